@@ -1,0 +1,301 @@
+"""ctypes front end of the fp64 MALA oracle (``mala_oracle.c``) -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module; the
+product path never does.  The C functions work on ONE query head and its key/value head, exactly
+as the paper's Methodology section writes the operator; this file adds nothing but the batch /
+head loops (contiguous GQA groups: ``h_kv = h_q // (Hq // Hkv)``), the summation of dK, dV over
+the query heads that share a KV head, and array marshalling.
+
+Tensors are ``[B, N, H, d]`` (torch tensors of any float dtype, or numpy arrays); every head slice
+is widened to float64 before it reaches C.  lse / D are ``[B, Hq, N]``.  Tile masks use the C
+encoding: 0 = not legal, 1 = skipped, 2 = retained; ``crit`` is the tile criterion C (skip iff
+C < 0), NaN where not legal.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mala_oracle.c")
+_LIB = os.path.join(_HERE, "libmala_oracle.so")
+_lib = None
+
+ILLEGAL, SKIPPED, RETAINED = 0, 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (strict IEEE, OpenMP)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fno-fast-math", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"]
+        subprocess.check_call(cmd)
+    return _LIB
+
+
+_D = ctypes.POINTER(ctypes.c_double)
+_I = ctypes.POINTER(ctypes.c_int)
+_U8 = ctypes.POINTER(ctypes.c_uint8)
+_ci, _cd = ctypes.c_int, ctypes.c_double
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(_LIB)
+        L.mala_oracle_threads.restype = _ci
+        L.mala_oracle_dense_fwd.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _ci, _ci, _ci, _D, _D]
+        L.mala_oracle_dense_bwd.argtypes = [_D, _D, _D, _D, _ci, _ci, _cd, _ci, _D, _D, _D]
+        L.mala_oracle_fwd.argtypes = [_D, _D, _D, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D, _D, _U8, _D]
+        L.mala_oracle_bwd_D.argtypes = [_D, _D, _ci, _ci, _D]
+        L.mala_oracle_bwd.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I,
+                                      _D, _D, _D, _U8, _D]
+        L.mala_oracle_bwd_dq.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D]
+        L.mala_oracle_decode_tiles_per_split.argtypes = [_ci, _ci, _ci]
+        L.mala_oracle_decode_splits.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _D, _D, _U8, _D]
+        L.mala_oracle_decode_merge.argtypes = [_D, _D, _ci, _ci, _ci, _D, _D]
+        for f in ("mala_oracle_dense_fwd", "mala_oracle_dense_bwd", "mala_oracle_fwd", "mala_oracle_bwd_D",
+                  "mala_oracle_bwd", "mala_oracle_bwd_dq", "mala_oracle_decode_tiles_per_split",
+                  "mala_oracle_decode_splits", "mala_oracle_decode_merge"):
+            getattr(L, f).restype = _ci
+        _lib = L
+    return _lib
+
+
+def threads() -> int:
+    return int(lib().mala_oracle_threads())
+
+
+def _np(x) -> np.ndarray:
+    """float64 contiguous numpy copy of a torch tensor / numpy array (exact for bf16, fp32)."""
+    if hasattr(x, "detach"):
+        import torch
+        x = x.detach().cpu().to(torch.float64).numpy()
+    return np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+
+
+def _head(x, b: int, h: int) -> np.ndarray:
+    return _np(x[b, :, h, :])
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(_D)
+
+
+def _ip(a):
+    return a.ctypes.data_as(_I) if a is not None else None
+
+
+def _u8(a: np.ndarray):
+    return a.ctypes.data_as(_U8)
+
+
+def _ck(rc: int, what: str):
+    if rc != 0:
+        raise ValueError(f"oracle {what} rejected its arguments (rc={rc})")
+
+
+def dense_fwd(q, k, v, scale: float, causal: bool = True):
+    """FullAttn by its definition.  Returns o [B,N,Hq,d], lse [B,Hq,N]."""
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    o = np.zeros((B, N, Hq, d))
+    lse = np.zeros((B, Hq, N))
+    for b in range(B):
+        for h in range(Hq):
+            Q, K, V = _head(q, b, h), _head(k, b, h // G), _head(v, b, h // G)
+            O = np.zeros((N, d))
+            _ck(lib().mala_oracle_dense_fwd(_p(Q), _p(K), _p(V), N, K.shape[0], d, scale, int(causal), 0, N,
+                                            _p(O), _p(lse[b, h])), "dense_fwd")
+            o[b, :, h, :] = O
+    return o, lse
+
+
+def dense_bwd(q, k, v, do, scale: float, causal: bool = True):
+    """FullAttn gradients by the closed forms.  Returns dq [B,N,Hq,d], dk, dv [B,N,Hkv,d]."""
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    dq = np.zeros((B, N, Hq, d))
+    dk = np.zeros((B, N, Hkv, d))
+    dv = np.zeros((B, N, Hkv, d))
+    for b in range(B):
+        for h in range(Hq):
+            Q, K, V, dO = _head(q, b, h), _head(k, b, h // G), _head(v, b, h // G), _head(do, b, h)
+            a, c, e = np.zeros((N, d)), np.zeros((N, d)), np.zeros((N, d))
+            _ck(lib().mala_oracle_dense_bwd(_p(Q), _p(K), _p(V), _p(dO), N, d, scale, int(causal), _p(a), _p(c),
+                                            _p(e)), "dense_bwd")
+            dq[b, :, h, :] = a
+            dk[b, :, h // G, :] += c
+            dv[b, :, h // G, :] += e
+    return dq, dk, dv
+
+
+def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True, units=None):
+    """Algorithm 1.  ``units``: optional list of (b, h_q, i) query blocks; rows of other blocks stay NaN.
+
+    Returns dict(o [B,N,Hq,d], lse [B,Hq,N], mask [B,Hq,Tr,Tc] uint8, crit [B,Hq,Tr,Tc]).
+    """
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    Tr, Tc = -(-N // Bq), -(-N // Bk)
+    o = np.full((B, N, Hq, d), np.nan)
+    lse = np.full((B, Hq, N), np.nan)
+    mask = np.zeros((B, Hq, Tr, Tc), dtype=np.uint8)
+    crit = np.full((B, Hq, Tr, Tc), np.nan)
+    heads = {}
+    if units is None:
+        for b in range(B):
+            for h in range(Hq):
+                heads[(b, h)] = None
+    else:
+        for (b, h, i) in units:
+            heads.setdefault((b, h), []).append(int(i))
+    for (b, h), blocks in heads.items():
+        Q, K, V = _head(q, b, h), _head(k, b, h // G), _head(v, b, h // G)
+        O = np.full((N, d), np.nan)
+        l = np.full((N,), np.nan)
+        m = np.zeros((Tr, Tc), dtype=np.uint8)
+        c = np.full((Tr, Tc), np.nan)
+        bl = np.asarray(blocks, dtype=np.int32) if blocks is not None else None
+        _ck(lib().mala_oracle_fwd(_p(Q), _p(K), _p(V), N, d, scale, tau, Bq, Bk, int(causal),
+                                  0 if bl is None else len(bl), _ip(bl), _p(O), _p(l), _u8(m), _p(c)), "fwd")
+        o[b, :, h, :] = O
+        lse[b, h] = l
+        mask[b, h] = m
+        crit[b, h] = c
+    return dict(o=o, lse=lse, mask=mask, crit=crit)
+
+
+def bwd(q, k, v, o, do, lse, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True,
+        key_units=None, dq_units=None):
+    """Algorithm 2 with the given forward output ``o`` and saved ``lse``.
+
+    Full run (both unit lists None): dq, dk, dv complete.  With ``key_units`` = [(b, h_kv, j)] only
+    those key blocks are run: their dK/dV rows (summed over the group's query heads) are exact and
+    everything else is NaN.  With ``dq_units`` = [(b, h_q, i)] the dQ rows of those query blocks are
+    computed from all their legal key blocks.
+    Returns dict(dq, dk, dv, mask [B,Hq,Tc,Tr], crit [B,Hq,Tc,Tr]).
+    """
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    Tr, Tc = -(-N // Bq), -(-N // Bk)
+    full = key_units is None and dq_units is None
+    dq = np.zeros((B, N, Hq, d)) if full else np.full((B, N, Hq, d), np.nan)
+    dk = np.zeros((B, N, Hkv, d)) if full else np.full((B, N, Hkv, d), np.nan)
+    dv = np.zeros((B, N, Hkv, d)) if full else np.full((B, N, Hkv, d), np.nan)
+    mask = np.zeros((B, Hq, Tc, Tr), dtype=np.uint8)
+    crit = np.full((B, Hq, Tc, Tr), np.nan)
+
+    def head_inputs(b, h):
+        Q, K, V, dO = _head(q, b, h), _head(k, b, h // G), _head(v, b, h // G), _head(do, b, h)
+        O = _head(o, b, h)
+        l = _np(lse[b, h])
+        D = np.zeros((N,))
+        lib().mala_oracle_bwd_D(_p(O), _p(dO), N, d, _p(D))
+        return Q, K, V, dO, l, D
+
+    groups = {}
+    if full:
+        for b in range(B):
+            for g in range(Hkv):
+                groups[(b, g)] = None
+    elif key_units is not None:
+        for (b, g, j) in key_units:
+            groups.setdefault((b, g), []).append(int(j))
+    for (b, g), blocks in groups.items():
+        bl = np.asarray(blocks, dtype=np.int32) if blocks is not None else None
+        rows = None
+        if bl is not None:
+            rows = np.concatenate([np.arange(j * Bk, min(N, (j + 1) * Bk)) for j in bl])
+            dk[b, rows, g, :] = 0.0
+            dv[b, rows, g, :] = 0.0
+        for h in range(g * G, (g + 1) * G):
+            Q, K, V, dO, l, D = head_inputs(b, h)
+            a = np.zeros((N, d))
+            c = np.zeros((N, d))
+            e = np.zeros((N, d))
+            m = np.zeros((Tc, Tr), dtype=np.uint8)
+            cr = np.full((Tc, Tr), np.nan)
+            _ck(lib().mala_oracle_bwd(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, d, scale, tau, Bq, Bk,
+                                      int(causal), 0 if bl is None else len(bl), _ip(bl),
+                                      _p(a) if full else None, _p(c), _p(e), _u8(m), _p(cr)), "bwd")
+            if full:
+                dq[b, :, h, :] = a
+                dk[b, :, g, :] += c
+                dv[b, :, g, :] += e
+                mask[b, h] = m
+                crit[b, h] = cr
+            else:
+                dk[b, rows, g, :] += c[rows]
+                dv[b, rows, g, :] += e[rows]
+                mask[b, h, bl] = m[bl]
+                crit[b, h, bl] = cr[bl]
+    if dq_units is not None:
+        heads = {}
+        for (b, h, i) in dq_units:
+            heads.setdefault((b, h), []).append(int(i))
+        for (b, h), blocks in heads.items():
+            bl = np.asarray(blocks, dtype=np.int32)
+            Q, K, V, dO, l, D = head_inputs(b, h)
+            a = np.full((N, d), np.nan)
+            _ck(lib().mala_oracle_bwd_dq(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, d, scale, tau, Bq, Bk,
+                                         int(causal), len(bl), _ip(bl), _p(a)), "bwd_dq")
+            rows = np.concatenate([np.arange(i * Bq, min(N, (i + 1) * Bq)) for i in bl])
+            dq[b, rows, h, :] = a[rows]
+    return dict(dq=dq, dk=dk, dv=dv, mask=mask, crit=crit)
+
+
+def decode(q, kcache, vcache, scale: float, tau: float, num_splits: int, Bk: int, units=None,
+           packed_rows: bool = True):
+    """Split-KV decode of one new token per sequence.
+
+    q [B,Hq,d] (or [B,1,Hq,d]); caches [B,Nk,Hkv,d].  ``units``: optional list of (b, h_kv); other
+    entries stay NaN.  ``packed_rows``: the Hq/Hkv query heads of one KV head form the rows of one
+    tile (one row that needs a tile retains it for all); False runs every query head alone.
+    Returns dict(o [B,Hq,d], lse [B,Hq], mask [B,Hkv,S,tps] (packed) or [B,Hq,S,tps], crit, o_part, lse_part).
+    """
+    if len(q.shape) == 4:
+        q = q[:, 0]
+    B, Hq, d = q.shape
+    Nk, Hkv = kcache.shape[1], kcache.shape[2]
+    G = Hq // Hkv
+    tps = int(lib().mala_oracle_decode_tiles_per_split(Nk, num_splits, Bk))
+    o = np.full((B, Hq, d), np.nan)
+    lse = np.full((B, Hq), np.nan)
+    nm = Hkv if packed_rows else Hq
+    mask = np.zeros((B, nm, num_splits, tps), dtype=np.uint8)
+    crit = np.full((B, nm, num_splits, tps), np.nan)
+    o_part = np.full((B, Hq, num_splits, d), np.nan)
+    lse_part = np.full((B, Hq, num_splits), np.nan)
+    if units is None:
+        units = [(b, g) for b in range(B) for g in range(Hkv)]
+    for (b, g) in units:
+        K, V = _head(kcache, b, g), _head(vcache, b, g)
+        row_sets = [list(range(g * G, (g + 1) * G))] if packed_rows else [[h] for h in range(g * G, (g + 1) * G)]
+        for hs in row_sets:
+            R = len(hs)
+            Q = _np(q[b, hs[0]:hs[-1] + 1, :])
+            op = np.zeros((num_splits, R, d))
+            lp = np.zeros((num_splits, R))
+            m = np.zeros((num_splits, tps), dtype=np.uint8)
+            c = np.full((num_splits, tps), np.nan)
+            _ck(lib().mala_oracle_decode_splits(_p(Q), _p(K), _p(V), R, Nk, d, scale, tau, num_splits, Bk, _p(op),
+                                                _p(lp), _u8(m), _p(c)), "decode_splits")
+            oo = np.zeros((R, d))
+            ll = np.zeros((R,))
+            _ck(lib().mala_oracle_decode_merge(_p(op), _p(lp), num_splits, R, d, _p(oo), _p(ll)), "decode_merge")
+            o[b, hs[0]:hs[-1] + 1] = oo
+            lse[b, hs[0]:hs[-1] + 1] = ll
+            o_part[b, hs[0]:hs[-1] + 1] = op.transpose(1, 0, 2)
+            lse_part[b, hs[0]:hs[-1] + 1] = lp.T
+            mi = g if packed_rows else hs[0]
+            mask[b, mi] = m
+            crit[b, mi] = c
+    return dict(o=o, lse=lse, mask=mask, crit=crit, o_part=o_part, lse_part=lse_part)

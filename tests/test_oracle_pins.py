@@ -1,0 +1,480 @@
+"""Pins of the fp64 oracle against things other than itself (CPU only).
+
+Each test states what fixes the expected value: the paper's equations re-stated independently
+(explicit key sets and direct sums, ratio form of Eq. 2), textbook softmax, finite differences,
+closed forms, Proposition 1, the nesting property, special cases that reduce to dense attention.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import mala_oracle as orc
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+def peaky_inputs(N, d, seed, Hq=1, Hkv=1, B=1, boost=4.0, retrieval=True):
+    """Random heads with a strong self key (and a few far retrieval keys) so that tiles do get skipped."""
+    r = _rng(seed)
+    q = r.standard_normal((B, N, Hq, d))
+    k = r.standard_normal((B, N, Hkv, d))
+    v = r.standard_normal((B, N, Hkv, d))
+    k *= math.sqrt(d) / np.linalg.norm(k, axis=-1, keepdims=True)
+    G = Hq // Hkv
+    for b in range(B):
+        for h in range(Hq):
+            q[b, :, h] += boost * k[b, :, h // G]
+            if retrieval:
+                for i in range(8, N, 23):
+                    j = int(r.integers(0, i))
+                    q[b, i, h] += boost * k[b, j, h // G]
+    return q, k, v
+
+
+# ------------------------------------------------------------------------------------------------
+# independent restatements used as pins
+# ------------------------------------------------------------------------------------------------
+def textbook_attention(Q, K, V, scale):
+    N = Q.shape[0]
+    O = np.zeros_like(V[:N])
+    lse = np.zeros(N)
+    for q in range(N):
+        e = np.array([math.exp(scale * float(Q[q] @ K[k])) for k in range(q + 1)])
+        p = e / e.sum()
+        O[q] = sum(p[k] * V[k] for k in range(q + 1))
+        lse[q] = math.log(e.sum())
+    return O, lse
+
+
+def brute_mala_fwd(Q, K, V, scale, tau, Bq, Bk):
+    """Eqs. 1-2 with explicit retained key sets and direct summation; ratio form of the test."""
+    N = Q.shape[0]
+    S = scale * (Q @ K.T)
+    Tr, Tc = -(-N // Bq), -(-N // Bk)
+    mask = np.zeros((Tr, Tc), dtype=np.uint8)
+    O = np.zeros((N, V.shape[1]))
+    lse = np.zeros(N)
+    for i in range(Tr):
+        rows = list(range(i * Bq, min(N, (i + 1) * Bq)))
+        R = {q: [] for q in rows}
+        for j in reversed(range(Tc)):
+            keys = list(range(j * Bk, min(N, (j + 1) * Bk)))
+            if keys[0] > rows[-1]:
+                continue
+            skip = True
+            for q in rows:
+                legal = [k for k in keys if k <= q]
+                if not legal:
+                    continue                      # row does not constrain the tile
+                Zt = sum(math.exp(S[q, k]) for k in R[q])
+                if Zt == 0.0:
+                    skip = False                  # first legal tile of a row is always kept
+                    continue
+                ratio = math.exp(max(S[q, k] for k in legal)) / Zt
+                if not (ratio < tau / (q + 1)):
+                    skip = False
+            mask[i, j] = 1 if skip else 2
+            if not skip:
+                for q in rows:
+                    R[q] += [k for k in keys if k <= q]
+        for q in rows:
+            Z = sum(math.exp(S[q, k]) for k in R[q])
+            O[q] = sum(math.exp(S[q, k]) / Z * V[k] for k in R[q])
+            lse[q] = math.log(Z)
+    return O, lse, mask
+
+
+def brute_mala_bwd(Q, K, V, dO, O, lse, scale, tau, Bq, Bk):
+    """Eq. 4 per tile with the saved lse, then the attention-backward equations restricted to the
+    retained tiles, written with whole-matrix products."""
+    N = Q.shape[0]
+    S = scale * (Q @ K.T)                                       # [q, k]
+    Tr, Tc = -(-N // Bq), -(-N // Bk)
+    mask = np.zeros((Tc, Tr), dtype=np.uint8)
+    keep = np.zeros((N, N), dtype=bool)
+    for j in range(Tc):
+        for i in range(Tr):
+            qs = range(i * Bq, min(N, (i + 1) * Bq))
+            ks = range(j * Bk, min(N, (j + 1) * Bk))
+            ent = [(q, k) for q in qs for k in ks if k <= q]
+            if not ent:
+                continue
+            skip = all(math.exp(S[q, k] - lse[q]) < tau / (q + 1) for (q, k) in ent)
+            mask[j, i] = 1 if skip else 2
+            if not skip:
+                for (q, k) in ent:
+                    keep[q, k] = True
+    P = np.where(keep, np.exp(S - lse[:, None]), 0.0)
+    D = (O * dO).sum(axis=1)
+    dP = dO @ V.T
+    dS = P * (dP - D[:, None])
+    return scale * dS @ K, scale * dS.T @ Q, P.T @ dO, mask
+
+
+# ------------------------------------------------------------------------------------------------
+# FullAttn (tau = 0)
+# ------------------------------------------------------------------------------------------------
+def test_dense_fwd_is_textbook_softmax():
+    q, k, v = peaky_inputs(37, 8, 1, boost=0.5)
+    o, lse = orc.dense_fwd(q, k, v, 0.3)
+    O, L = textbook_attention(q[0, :, 0], k[0, :, 0], v[0, :, 0], 0.3)
+    assert np.allclose(o[0, :, 0], O, rtol=0, atol=1e-12)
+    assert np.allclose(lse[0, 0], L, rtol=0, atol=1e-12)
+
+
+def test_dense_bwd_matches_finite_differences():
+    N, d, scale = 12, 4, 0.7
+    q, k, v = peaky_inputs(N, d, 2, boost=0.3)
+    do = _rng(3).standard_normal((1, N, 1, d))
+    dq, dk, dv = orc.dense_bwd(q, k, v, do, scale)
+
+    def loss(qq, kk, vv):
+        o, _ = orc.dense_fwd(qq, kk, vv, scale)
+        return float((o * do).sum())
+
+    eps = 1e-6
+    for (x, g, name) in ((q, dq, "dq"), (k, dk, "dk"), (v, dv, "dv")):
+        num = np.zeros_like(x)
+        for idx in np.ndindex(*x.shape):
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps
+            xm[idx] -= eps
+            args_p = [q, k, v]
+            args_m = [q, k, v]
+            pos = {"dq": 0, "dk": 1, "dv": 2}[name]
+            args_p[pos], args_m[pos] = xp, xm
+            num[idx] = (loss(*args_p) - loss(*args_m)) / (2 * eps)
+        assert np.linalg.norm(num - g) <= 1e-6 * max(1.0, np.linalg.norm(g)), name
+
+
+def test_dense_bwd_gqa_sums_group_heads():
+    q, k, v = peaky_inputs(16, 4, 4, Hq=4, Hkv=2, boost=0.3)
+    do = _rng(5).standard_normal(q.shape)
+    dq, dk, dv = orc.dense_bwd(q, k, v, do, 0.5)
+    for g in range(2):
+        acc_k = np.zeros((16, 4))
+        acc_v = np.zeros((16, 4))
+        for h in (2 * g, 2 * g + 1):
+            a, c, e = orc.dense_bwd(q[:, :, h:h + 1], k[:, :, g:g + 1], v[:, :, g:g + 1], do[:, :, h:h + 1], 0.5)
+            assert np.allclose(dq[0, :, h], a[0, :, 0], atol=1e-13)
+            acc_k += c[0, :, 0]
+            acc_v += e[0, :, 0]
+        assert np.allclose(dk[0, :, g], acc_k, atol=1e-12)
+        assert np.allclose(dv[0, :, g], acc_v, atol=1e-12)
+
+
+@pytest.mark.parametrize("N,Bq,Bk", [(64, 8, 8), (50, 8, 8), (50, 16, 4), (33, 4, 16), (20, 32, 32)])
+def test_tau_zero_recovers_fullattn(N, Bq, Bk):
+    d, scale = 8, 0.35
+    q, k, v = peaky_inputs(N, d, 6, Hq=2, Hkv=1)
+    do = _rng(7).standard_normal(q.shape)
+    o_d, lse_d = orc.dense_fwd(q, k, v, scale)
+    f = orc.fwd(q, k, v, scale, 0.0, Bq, Bk)
+    assert np.allclose(f["o"], o_d, atol=1e-12) and np.allclose(f["lse"], lse_d, atol=1e-12)
+    assert not (f["mask"] == orc.SKIPPED).any()
+    dq_d, dk_d, dv_d = orc.dense_bwd(q, k, v, do, scale)
+    g = orc.bwd(q, k, v, f["o"], do, f["lse"], scale, 0.0, Bq, Bk)
+    for a, b_ in ((g["dq"], dq_d), (g["dk"], dk_d), (g["dv"], dv_d)):
+        assert np.allclose(a, b_, atol=1e-10)
+    assert not (g["mask"] == orc.SKIPPED).any()
+
+
+# ------------------------------------------------------------------------------------------------
+# the online rule (Eqs. 1-3, Algorithm 1)
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N,Bq,Bk,tau", [(64, 8, 8, 1e-2), (61, 8, 8, 1e-1), (48, 16, 4, 1e-2), (40, 4, 8, 1.0),
+                                         (24, 1, 1, 1e-1)])
+def test_fwd_matches_bruteforce_key_sets(N, Bq, Bk, tau):
+    d, scale = 32, 1.0 / math.sqrt(32)
+    q, k, v = peaky_inputs(N, d, 11 + N, boost=5.0)
+    f = orc.fwd(q, k, v, scale, tau, Bq, Bk)
+    O, L, M = brute_mala_fwd(q[0, :, 0], k[0, :, 0], v[0, :, 0], scale, tau, Bq, Bk)
+    assert (np.abs(f["crit"][np.isfinite(f["crit"])]) > 1e-9).all()
+    assert (f["mask"][0, 0] == M).all()
+    assert (M == 1).sum() > 0, "workload must exercise skipping"
+    assert np.allclose(f["o"][0, :, 0], O, atol=1e-11) and np.allclose(f["lse"][0, 0], L, atol=1e-11)
+
+
+def test_fwd_bq_larger_than_bk_rows_without_legal_keys_do_not_constrain():
+    # with B_q = 16, B_k = 4 the first tiles visited have no legal key for the early rows of a block
+    N, d, scale, tau = 32, 4, 0.5, 1e-1
+    q, k, v = peaky_inputs(N, d, 21, boost=6.0)
+    f = orc.fwd(q, k, v, scale, tau, 16, 4)
+    O, L, M = brute_mala_fwd(q[0, :, 0], k[0, :, 0], v[0, :, 0], scale, tau, 16, 4)
+    assert (f["mask"][0, 0] == M).all() and np.isfinite(f["lse"]).all()
+    assert np.allclose(f["o"][0, :, 0], O, atol=1e-11)
+
+
+def test_fwd_first_tile_retained_rows_nonempty_and_illegal_tiles_uncounted():
+    q, k, v = peaky_inputs(96, 8, 31, Hq=2, Hkv=2, boost=6.0)
+    f = orc.fwd(q, k, v, 0.35, 1.0, 8, 8)
+    m = f["mask"]
+    for i in range(12):
+        assert (m[:, :, i, i] == orc.RETAINED).all()
+        assert (m[:, :, i, i + 1:] == orc.ILLEGAL).all()
+        assert (m[:, :, i, :i + 1] != orc.ILLEGAL).all()
+    assert np.isfinite(f["lse"]).all() and np.isfinite(f["o"]).all()
+    assert np.isnan(f["crit"][m == orc.ILLEGAL]).all()
+
+
+@pytest.mark.parametrize("tau", [1e-3, 1e-1, 1.0, 4.0])
+def test_proposition1_omitted_mass_and_output_bounds(tau):
+    N, d, scale = 128, 32, 1.0 / math.sqrt(32)
+    q, k, v = peaky_inputs(N, d, 41, Hq=2, Hkv=1, boost=4.0)
+    o_d, lse_d = orc.dense_fwd(q, k, v, scale)
+    f = orc.fwd(q, k, v, scale, tau, 8, 8)
+    eps = 1.0 - np.exp(f["lse"] - lse_d)                       # omitted mass from the two normalizers
+    assert (eps >= -1e-12).all() and (eps <= tau / (1 + tau) + 1e-12).all()
+    vmax = np.linalg.norm(v, axis=-1).max()
+    err = np.linalg.norm(f["o"] - o_d, axis=-1)
+    assert (err <= 2 * tau / (1 + tau) * vmax + 1e-12).all()
+    if tau >= 1e-1:
+        assert (f["mask"] == orc.SKIPPED).sum() > 0
+
+
+def test_closed_form_zero_queries_uniform_rows():
+    N, d = 40, 4
+    r = _rng(51)
+    q = np.zeros((1, N, 1, d))
+    k, v = r.standard_normal((1, N, 1, d)), r.standard_normal((1, N, 1, d))
+    for tau in (1e-3, 1.0):
+        f = orc.fwd(q, k, v, 0.5, tau, 8, 8)
+        assert not (f["mask"] == orc.SKIPPED).any()            # ratio 1/Z_t >= 1/L_q >= tau/L_q
+        mean = np.cumsum(v[0, :, 0], axis=0) / np.arange(1, N + 1)[:, None]
+        assert np.allclose(f["o"][0, :, 0], mean, atol=1e-13)
+        assert np.allclose(f["lse"][0, 0], np.log(np.arange(1, N + 1)), atol=1e-13)
+
+
+def _one_hot_case(N, C):
+    q = np.zeros((1, N, 1, N))
+    k = np.zeros((1, N, 1, N))
+    for t in range(N):
+        q[0, t, 0, t] = C
+        k[0, t, 0, t] = 1.0
+    v = _rng(61).standard_normal((1, N, 1, 3))
+    return q, k, np.concatenate([v, np.zeros((1, N, 1, N - 3))], axis=-1)
+
+
+def _one_hot_expected_mask(N, B, C, tau):
+    T = N // B
+    m = np.zeros((T, T), dtype=np.uint8)
+    for i in range(T):
+        Z = [math.exp(C) + r for r in range(B)]                # after the diagonal tile: self key + r zeros
+        m[i, i] = 2
+        for j in range(i - 1, -1, -1):
+            skip = all(1.0 / Z[r] < tau / (i * B + r + 1) for r in range(B))
+            m[i, j] = 1 if skip else 2
+            if not skip:
+                Z = [z + B for z in Z]
+    return m
+
+
+@pytest.mark.parametrize("C", [3.0, 7.0, 8.0, 10.0])
+def test_closed_form_one_boosted_key_per_row(C):
+    N, B, tau = 64, 8, 1e-2
+    q, k, v = _one_hot_case(N, C)
+    f = orc.fwd(q, k, v, 1.0, tau, B, B)
+    assert (f["mask"][0, 0] == _one_hot_expected_mask(N, B, C, tau)).all()
+
+
+def test_closed_form_threshold_crossing_at_predicted_boost():
+    # block 1 (rows 8..15), tile (1,0): the binding row is the last one, r = 7, L = 16:
+    # skipped iff 1/(e^C + 7) < tau/16  <=>  C > log(16/tau - 7)
+    N, B, tau = 64, 8, 1e-2
+    Cstar = math.log(16 / tau - 7)
+    for C, expect in ((Cstar - 1e-6, orc.RETAINED), (Cstar + 1e-6, orc.SKIPPED)):
+        q, k, v = _one_hot_case(N, C)
+        f = orc.fwd(q, k, v, 1.0, tau, B, B, units=[(0, 0, 1)])
+        assert f["mask"][0, 0, 1, 0] == expect
+        assert abs(f["crit"][0, 0, 1, 0]) < 1e-5
+
+
+def test_single_tile_is_dense_for_any_tau():
+    q, k, v = peaky_inputs(30, 8, 71, boost=6.0)
+    o_d, lse_d = orc.dense_fwd(q, k, v, 0.4)
+    f = orc.fwd(q, k, v, 0.4, 10.0, 32, 32)
+    assert np.allclose(f["o"], o_d, atol=1e-12) and np.allclose(f["lse"], lse_d, atol=1e-12)
+
+
+def test_per_element_rule_when_tiles_are_single_entries():
+    N, d, scale, tau = 20, 4, 0.5, 0.3
+    q, k, v = peaky_inputs(N, d, 81, boost=4.0)
+    f = orc.fwd(q, k, v, scale, tau, 1, 1)
+    S = scale * q[0, :, 0] @ k[0, :, 0].T
+    for i in range(N):
+        Z = 0.0
+        for j in range(i, -1, -1):
+            keep = (Z == 0.0) or not (math.exp(S[i, j]) / Z < tau / (i + 1))
+            assert f["mask"][0, 0, i, j] == (2 if keep else 1)
+            if keep:
+                Z += math.exp(S[i, j])
+        assert abs(f["lse"][0, 0, i] - math.log(Z)) < 1e-12
+
+
+def test_tau_monotonicity_of_forward_support():
+    # if tau1 (1 + tau2) <= tau2 the support under tau1 contains the support under tau2
+    q, k, v = peaky_inputs(128, 32, 91, boost=6.0)
+    taus = [0.0, 1e-5, 1e-4, 1e-3, 1e-1]
+    masks = [orc.fwd(q, k, v, 1.0 / math.sqrt(32), t, 8, 8)["mask"] for t in taus]
+    for a, b_ in zip(masks[:-1], masks[1:]):
+        assert ((b_ == orc.RETAINED) <= (a == orc.RETAINED)).all()
+    assert (masks[-1] == orc.SKIPPED).sum() > (masks[1] == orc.SKIPPED).sum()
+
+
+def test_fwd_units_select_blocks_and_match_full_run():
+    q, k, v = peaky_inputs(70, 8, 101, Hq=2, Hkv=1, boost=5.0)
+    full = orc.fwd(q, k, v, 0.35, 1e-1, 8, 8)
+    part = orc.fwd(q, k, v, 0.35, 1e-1, 8, 8, units=[(0, 1, 3), (0, 1, 8)])
+    for i in (3, 8):
+        rows = slice(i * 8, min(70, i * 8 + 8))
+        assert np.array_equal(part["o"][0, rows, 1], full["o"][0, rows, 1])
+        assert np.array_equal(part["mask"][0, 1, i], full["mask"][0, 1, i])
+    assert np.isnan(part["o"][0, :, 0]).all() and np.isnan(part["o"][0, 0:24, 1]).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# the offline rule (Eq. 4, Algorithm 2)
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N,Bq,Bk,tau", [(64, 8, 8, 1e-2), (61, 8, 8, 1e-1), (48, 4, 8, 1.0), (48, 16, 4, 1e-1)])
+def test_bwd_matches_bruteforce_and_is_nested(N, Bq, Bk, tau):
+    d, scale = 32, 1.0 / math.sqrt(32)
+    q, k, v = peaky_inputs(N, d, 111 + N, boost=5.0)
+    do = _rng(112).standard_normal(q.shape)
+    f = orc.fwd(q, k, v, scale, tau, Bq, Bk)
+    g = orc.bwd(q, k, v, f["o"], do, f["lse"], scale, tau, Bq, Bk)
+    dQ, dK, dV, M = brute_mala_bwd(q[0, :, 0], k[0, :, 0], v[0, :, 0], do[0, :, 0], f["o"][0, :, 0], f["lse"][0, 0],
+                                   scale, tau, Bq, Bk)
+    assert (g["mask"][0, 0] == M).all()
+    assert np.allclose(g["dq"][0, :, 0], dQ, atol=1e-11)
+    assert np.allclose(g["dk"][0, :, 0], dK, atol=1e-11)
+    assert np.allclose(g["dv"][0, :, 0], dV, atol=1e-11)
+    # nesting: every tile kept by backward was kept by forward (same partition), none stored
+    fm = f["mask"][0, 0]
+    bm = g["mask"][0, 0].T
+    assert ((bm == orc.RETAINED) <= (fm == orc.RETAINED)).all()
+    assert ((bm == orc.ILLEGAL) == (fm == orc.ILLEGAL)).all()
+    assert (bm == orc.SKIPPED).sum() >= (fm == orc.SKIPPED).sum() > 0
+
+
+def test_bwd_may_skip_the_diagonal_tile():
+    # rows whose mass sits on one far key: the diagonal tile falls below tau/L under the final normalizer
+    N, B, d = 32, 8, 32
+    r = _rng(121)
+    k = np.zeros((1, N, 1, d))
+    for t in range(N):
+        k[0, t, 0, t] = 1.0
+    q = np.zeros((1, N, 1, d))
+    q[0, :, 0, 0] = 30.0                                        # every query points at key 0
+    v = r.standard_normal((1, N, 1, d))
+    do = r.standard_normal((1, N, 1, d))
+    f = orc.fwd(q, k, v, 1.0, 1e-2, B, B)
+    g = orc.bwd(q, k, v, f["o"], do, f["lse"], 1.0, 1e-2, B, B)
+    assert (f["mask"][0, 0].diagonal() == orc.RETAINED).all()
+    assert (g["mask"][0, 0].diagonal()[1:] == orc.SKIPPED).all()
+    assert (g["mask"][0, 0, 0, :] == orc.RETAINED).all()
+
+
+def test_bwd_key_units_and_dq_units_match_full_run():
+    N, Bq, Bk, d, scale, tau = 72, 8, 8, 8, 0.35, 1e-1
+    q, k, v = peaky_inputs(N, d, 131, Hq=4, Hkv=2, boost=5.0)
+    do = _rng(132).standard_normal(q.shape)
+    f = orc.fwd(q, k, v, scale, tau, Bq, Bk)
+    full = orc.bwd(q, k, v, f["o"], do, f["lse"], scale, tau, Bq, Bk)
+    part = orc.bwd(q, k, v, f["o"], do, f["lse"], scale, tau, Bq, Bk, key_units=[(0, 1, 2), (0, 0, 8)],
+                   dq_units=[(0, 3, 5)])
+    assert np.allclose(part["dk"][0, 16:24, 1], full["dk"][0, 16:24, 1], atol=1e-12)
+    assert np.allclose(part["dv"][0, 64:72, 0], full["dv"][0, 64:72, 0], atol=1e-12)
+    assert np.allclose(part["dq"][0, 40:48, 3], full["dq"][0, 40:48, 3], atol=1e-12)
+    assert np.array_equal(part["mask"][0, 2:4, 2], full["mask"][0, 2:4, 2])
+    assert np.isnan(part["dk"][0, 0:8, 1]).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# split-KV decode
+# ------------------------------------------------------------------------------------------------
+def _decode_inputs(Nk, d, G, seed, gate=True):
+    r = _rng(seed)
+    q = r.standard_normal((1, G, d))
+    kc = r.standard_normal((1, Nk, 1, d))
+    vc = r.standard_normal((1, Nk, 1, d))
+    if gate:                                                    # most keys far below a few live ones
+        live = r.random(Nk) < 0.1
+        live[-4:] = True
+        kc[0, :, 0, d - 1] = np.where(live, 0.0, -6.0)
+        q[0, :, d - 1] = 6.0
+    return q, kc, vc
+
+
+@pytest.mark.parametrize("S", [1, 3, 8])
+def test_decode_tau_zero_any_split_count_is_dense(S):
+    q, kc, vc = _decode_inputs(100, 8, 4, 141)
+    dec = orc.decode(q, kc, vc, 0.4, 0.0, S, 8)
+    for h in range(4):
+        e = np.exp(0.4 * kc[0, :, 0] @ q[0, h])
+        assert np.allclose(dec["o"][0, h], (e / e.sum()) @ vc[0, :, 0], atol=1e-12)
+        assert abs(dec["lse"][0, h] - math.log(e.sum())) < 1e-12
+    assert not (dec["mask"] == orc.SKIPPED).any()
+
+
+@pytest.mark.parametrize("packed", [True, False])
+def test_decode_rule_bruteforce_per_split_and_mass_bound(packed):
+    Nk, d, G, S, Bk, scale, tau = 96, 8, 4, 3, 8, 0.5, 0.5
+    q, kc, vc = _decode_inputs(Nk, d, G, 151)
+    dec = orc.decode(q, kc, vc, scale, tau, S, Bk, packed_rows=packed)
+    sc = scale * kc[0, :, 0] @ q[0].T                            # [Nk, G]
+    chunk = 32
+    row_sets = [list(range(G))] if packed else [[h] for h in range(G)]
+    assert (dec["mask"] == orc.SKIPPED).sum() > 0
+    for ri, hs in enumerate(row_sets):
+        for s in range(S):
+            kept = []
+            for t in reversed(range(chunk // Bk)):
+                keys = list(range(s * chunk + t * Bk, s * chunk + (t + 1) * Bk))
+                skip = True
+                for h in hs:
+                    Z = sum(math.exp(sc[k_, h]) for k_ in kept)
+                    if Z == 0.0 or not (math.exp(max(sc[k_, h] for k_ in keys)) / Z < tau / Nk):
+                        skip = False
+                assert dec["mask"][0, ri, s, t] == (1 if skip else 2)
+                if not skip:
+                    kept += keys
+            for h in hs:
+                Z = sum(math.exp(sc[k_, h]) for k_ in kept)
+                assert abs(dec["lse_part"][0, h, s] - math.log(Z)) < 1e-12
+    # Proposition 1 carries over to the merged result (each omitted key is below tau/L of a partial Z)
+    for h in range(G):
+        lse_d = math.log(np.exp(sc[:, h]).sum())
+        eps = 1.0 - math.exp(dec["lse"][0, h] - lse_d)
+        assert -1e-12 <= eps <= tau / (1 + tau) + 1e-12
+
+
+def test_decode_merge_is_logsumexp_weighted_mean():
+    r = _rng(161)
+    op = r.standard_normal((1, 2, 5, 3))
+    lp = r.standard_normal((1, 2, 5))
+    L = orc.lib()
+    import ctypes
+    for h in range(2):
+        o = np.zeros((1, 3))
+        l = np.zeros((1,))
+        a = np.ascontiguousarray(op[0, h][:, None, :])
+        b_ = np.ascontiguousarray(lp[0, h][:, None])
+        L.mala_oracle_decode_merge(a.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+                                   b_.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), 5, 1, 3,
+                                   o.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+                                   l.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
+        w = np.exp(lp[0, h])
+        assert np.allclose(o[0], (w / w.sum()) @ op[0, h], atol=1e-13)
+        assert abs(l[0] - math.log(w.sum())) < 1e-13
+
+
+def test_decode_ragged_cache_and_empty_trailing_split():
+    q, kc, vc = _decode_inputs(70, 8, 2, 171, gate=False)
+    dec = orc.decode(q, kc, vc, 0.4, 0.0, 5, 16)                 # chunk = 16, 5 splits cover 80 > 70 keys
+    assert np.isneginf(dec["lse_part"]).sum() == 0                # 70 keys -> split 4 holds keys 64..69
+    dec2 = orc.decode(q, kc, vc, 0.4, 0.0, 8, 16)                # chunk = 16, splits 5..7 are empty
+    assert np.isneginf(dec2["lse_part"][0, :, 5:]).all()
+    assert np.allclose(dec["o"], dec2["o"], atol=1e-13)
