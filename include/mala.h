@@ -1,0 +1,111 @@
+/*
+ * libmala -- C ABI of the B200 (sm_100a) MassAlloc Attention (MALA) hot path.
+ *
+ * The operator is the one the paper's Methodology section states for a query head and its
+ * key/value head: QK^T scores are formed for every legal causal tile; a forward tile is skipped
+ * when, for every relevant row, rowmax(S) - m - log(l) < log(tau / L_q) (Eq. 3, Algorithm 1);
+ * a backward tile is skipped when S - lse < log(tau / L_q) on all its valid entries (Eq. 4,
+ * Algorithm 2); split-KV decode applies the forward rule per split against the split's partial
+ * normalizer with L = N_k and merges the partials ("Fused decoding execution").  tau = 0 selects
+ * the dense FullAttn kernels (Section 2.3: tau -> 0 recovers FullAttn).
+ *
+ * Conventions common to all calls
+ *   - Every pointer is a DEVICE pointer owned by the caller unless stated otherwise; the library
+ *     never frees or retains one.  Tensors are bf16 views [B, N, H, d] given as a base pointer and
+ *     element strides (sb, sn, sh); the last dimension is contiguous.  Base pointers must be
+ *     16-byte aligned and all strides multiples of 8 elements (16 bytes).
+ *   - d is 64 or 128.  Hq must be a multiple of Hkv; query head h uses key/value head
+ *     h / (Hq / Hkv).  N may be any positive length (the last tile may be ragged).
+ *   - scale (> 0, finite) multiplies the fp32 scores; lse is in nats, of the scaled scores, over
+ *     the retained set.  tau >= 0, finite.
+ *   - Tile partition: mala_tile_shape() reports it; forward and backward use the same partition.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t, may be NULL for the default
+ *     stream), allocate nothing and never synchronise.  `ws` is caller-provided scratch of at
+ *     least mala_workspace_bytes() bytes, 256-byte aligned; its contents are undefined afterwards.
+ *   - Return value: MALA_OK or a negative MALA_ERR_* code; nothing is launched on error.
+ *     A bounded device-side wait that expires does not hang: the kernels finish, later launches
+ *     become no-ops, and mala_device_status() reports MALA_ERR_DEVICE_TIMEOUT until cleared.
+ */
+#ifndef MALA_H_
+#define MALA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MALA_OK 0
+#define MALA_ERR_INVALID_ARG (-1)        /* NULL pointer, non-positive size, bad tau / scale */
+#define MALA_ERR_UNSUPPORTED (-2)        /* d not in {64,128}, Hq % Hkv != 0, too many splits ... */
+#define MALA_ERR_MISALIGNED (-3)         /* pointer / stride alignment rules above violated */
+#define MALA_ERR_WORKSPACE_TOO_SMALL (-4)
+#define MALA_ERR_WRONG_ARCH (-5)         /* current device is not compute capability 10.x */
+#define MALA_ERR_CUDA (-6)               /* a CUDA runtime call or launch failed */
+#define MALA_ERR_TENSOR_MAP (-7)         /* the driver rejected a TMA tensor map */
+#define MALA_ERR_DEVICE_TIMEOUT (-8)     /* a bounded device-side wait expired (status word) */
+
+#define MALA_OP_FWD 0
+#define MALA_OP_BWD 1
+#define MALA_OP_DECODE 2
+
+typedef struct { const void* p; int64_t sb, sn, sh; } mala_tin;   /* read-only bf16 [B,N,H,d] view */
+typedef struct { void* p; int64_t sb, sn, sh; } mala_tout;        /* written bf16 [B,N,H,d] view */
+
+/* Optional telemetry (any member may be NULL; the struct pointer itself may be NULL).
+ *   retained_per_block : u32, overwritten.  fwd [B,Hq,Tr] (per query block), bwd [B,Hq,Tc] (per key
+ *                        block and query head), decode [B,Hkv,num_splits].
+ *   tile_bitmask       : u32 words, overwritten.  fwd [B,Hq,Tr,ceil(Tc/32)], bit j of row i set iff
+ *                        tile (i,j) was retained; bwd [B,Hq,Tc,ceil(Tr/32)], bit i of row j;
+ *                        decode [B,Hkv,num_splits,ceil(tiles_per_split/32)].  Meant for parity checks.
+ *   totals             : u64[2], ACCUMULATED: += retained tiles, += legal (visited) tiles. */
+typedef struct {
+  uint32_t* retained_per_block;
+  uint32_t* tile_bitmask;
+  uint64_t* totals;
+} mala_stats;
+
+/* Algorithm 1 (forward / prefill).  q [B,N,Hq,d]; k, v [B,N,Hkv,d]; o [B,N,Hq,d]; lse fp32 [B,Hq,N].
+ * causal != 0: equal-length causal attention, L_q = q + 1, tiles visited from the diagonal toward
+ * earlier keys.  causal == 0: every key legal, L_q = N, tiles visited from the last to the first. */
+int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
+             int Hkv, int N, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
+             void* cuda_stream);
+
+/* Algorithm 2 (backward).  o, dout [B,N,Hq,d]; lse as written by mala_fwd; dq [B,N,Hq,d];
+ * dk, dv [B,N,Hkv,d] (summed over the query heads of the group).  D = rowsum(O o dO) is computed
+ * from the given o.  dQ is accumulated in fp32 in the workspace and converted at the end. */
+int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
+             mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d, int causal,
+             float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Split-KV decode of one new token per sequence ("Fused decoding execution").  q [B,1,Hq,d] (sn is
+ * ignored); kcache, vcache [B,Nk,Hkv,d], the newest token's key/value included; o [B,1,Hq,d];
+ * lse_opt fp32 [B,Hq] or NULL.  The Hq/Hkv query heads of one KV head are the rows of one tile; the
+ * key range is cut into num_splits contiguous chunks of ceil(ceil(Nk/num_splits)/128)*128 keys,
+ * each visited newest tile first with its own running state, L = Nk; partials are merged by the
+ * normalizer-aware reduction.  Requires Hq/Hkv <= 16. */
+int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
+                int B, int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws,
+                size_t ws_bytes, void* cuda_stream);
+
+/* Scratch bytes needed by one call of `op` (MALA_OP_*); N is Nk for decode; num_splits is ignored
+ * for fwd / bwd.  Returns 0 for unsupported arguments. */
+size_t mala_workspace_bytes(int op, int B, int Hq, int Hkv, int N, int d, int num_splits);
+
+/* Tile partition of `op` for head size d: Bq query rows x Bk keys.  For decode Bq is reported as 0
+ * (the rows are the Hq/Hkv packed query heads).  Returns MALA_OK or MALA_ERR_UNSUPPORTED. */
+int mala_tile_shape(int op, int d, int* Bq, int* Bk);
+
+/* Reads the current device's status word into *code_out (MALA_OK or MALA_ERR_DEVICE_TIMEOUT) and, if
+ * clear != 0, resets it.  Synchronises the device.  HOST pointer. */
+int mala_device_status(int* code_out, int clear);
+
+const char* mala_strerror(int code);
+int mala_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MALA_H_ */

@@ -1,0 +1,239 @@
+// Host side of libmala: argument validation, TMA tensor-map creation, workspace carving and kernel
+// launches behind the C ABI declared in include/mala.h.  No torch types, no allocation, no sync.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <mutex>
+
+#include "../../include/mala.h"
+#include "mala_bwd.cuh"
+#include "mala_decode.cuh"
+#include "mala_fwd.cuh"
+#include "tensor_map.h"
+
+namespace mala {
+
+// Sticky per-device status word written by kernels whose bounded waits expire.
+__device__ int g_mala_status;
+
+static std::mutex g_mu;
+static int* g_status_ptr[64];
+static bool g_attr_done[64];
+
+static int current_device_checked(int* dev_out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MALA_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return MALA_ERR_UNSUPPORTED;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MALA_ERR_CUDA;
+  if (major != 10) return MALA_ERR_WRONG_ARCH;
+  *dev_out = dev;
+  return MALA_OK;
+}
+
+template <typename K>
+static bool set_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+// One-time per-device set-up: status word address and dynamic shared memory limits.
+static int device_setup(int dev, int** status_out) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  if (!g_status_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_mala_status) != cudaSuccess) return MALA_ERR_CUDA;
+    g_status_ptr[dev] = (int*)ptr;
+  }
+  if (!g_attr_done[dev]) {
+    bool ok = true;
+    ok = ok && set_smem(mala_fwd_kernel<128, false>, FwdCfg<128, false>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<128, true>, FwdCfg<128, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<64, false>, FwdCfg<64, false>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<64, true>, FwdCfg<64, true>::kSmemBytes);
+    ok = ok && bwd_set_attributes();
+    ok = ok && decode_set_attributes();
+    if (!ok) return MALA_ERR_CUDA;
+    g_attr_done[dev] = true;
+  }
+  *status_out = g_status_ptr[dev];
+  return MALA_OK;
+}
+
+static bool aligned16(const void* p) { return (((uintptr_t)p) & 15) == 0; }
+static bool stride_ok(int64_t s) { return s >= 0 && (s % 8) == 0; }
+
+// bf16 [B,N,H,d] view: pointer and strides legal for TMA and 16-byte vector access
+static int check_view(const void* p, int64_t sb, int64_t sn, int64_t sh, int B, int N, int H) {
+  if (!p) return MALA_ERR_INVALID_ARG;
+  if (!aligned16(p)) return MALA_ERR_MISALIGNED;
+  if ((B > 1 && !stride_ok(sb)) || (N > 1 && !stride_ok(sn)) || (H > 1 && !stride_ok(sh))) return MALA_ERR_MISALIGNED;
+  if ((B > 1 && sb == 0) || (N > 1 && sn == 0) || (H > 1 && sh == 0)) return MALA_ERR_INVALID_ARG;
+  return MALA_OK;
+}
+
+static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float tau) {
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0) return MALA_ERR_INVALID_ARG;
+  if (!(tau >= 0.f) || !isfinite(tau)) return MALA_ERR_INVALID_ARG;
+  if (!(scale > 0.f) || !isfinite(scale)) return MALA_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return MALA_ERR_UNSUPPORTED;
+  if (Hq % Hkv != 0) return MALA_ERR_UNSUPPORTED;
+  if (B > 65535 || Hq > 65535) return MALA_ERR_UNSUPPORTED;
+  return MALA_OK;
+}
+
+#define MALA_TRY(expr)              \
+  do {                              \
+    const int rc_ = (expr);         \
+    if (rc_ != MALA_OK) return rc_; \
+  } while (0)
+
+static const float kLog2e = 1.4426950408889634f;
+
+template <int D, bool kDense>
+static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                      cudaStream_t stream) {
+  dim3 grid(p.Tr, p.Hq, p.B);
+  mala_fwd_kernel<D, kDense><<<grid, FwdCfg<D, kDense>::kThreads, FwdCfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
+  return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
+}
+
+}  // namespace mala
+
+using namespace mala;
+
+extern "C" {
+
+int mala_version(void) { return 100; }
+
+const char* mala_strerror(int code) {
+  switch (code) {
+    case MALA_OK: return "ok";
+    case MALA_ERR_INVALID_ARG: return "invalid argument";
+    case MALA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case MALA_ERR_MISALIGNED: return "pointer or stride not 16-byte aligned";
+    case MALA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case MALA_ERR_WRONG_ARCH: return "device is not sm_100";
+    case MALA_ERR_CUDA: return "CUDA runtime error";
+    case MALA_ERR_TENSOR_MAP: return "TMA tensor map rejected";
+    case MALA_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown error";
+  }
+}
+
+int mala_tile_shape(int op, int d, int* Bq, int* Bk) {
+  if (!Bq || !Bk) return MALA_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return MALA_ERR_UNSUPPORTED;
+  if (op == MALA_OP_FWD || op == MALA_OP_BWD) { *Bq = 128; *Bk = 128; return MALA_OK; }
+  if (op == MALA_OP_DECODE) { *Bq = 0; *Bk = 128; return MALA_OK; }
+  return MALA_ERR_UNSUPPORTED;
+}
+
+size_t mala_workspace_bytes(int op, int B, int Hq, int Hkv, int N, int d, int num_splits) {
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || (d != 64 && d != 128)) return 0;
+  if (op == MALA_OP_FWD) return 256;
+  if (op == MALA_OP_BWD) return bwd_workspace_bytes(B, Hq, N, d);
+  if (op == MALA_OP_DECODE) return num_splits > 0 ? decode_workspace_bytes(B, Hq, d, num_splits) : 0;
+  return 0;
+}
+
+int mala_device_status(int* code_out, int clear) {
+  if (!code_out) return MALA_ERR_INVALID_ARG;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  if (cudaDeviceSynchronize() != cudaSuccess) return MALA_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpy(&v, status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MALA_ERR_CUDA;
+  *code_out = v;
+  if (clear && v != 0) {
+    const int zero = 0;
+    if (cudaMemcpy(status, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return MALA_ERR_CUDA;
+  }
+  return MALA_OK;
+}
+
+int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
+             int Hkv, int N, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
+             void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
+  if (!lse) return MALA_ERR_INVALID_ARG;
+  MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, N, Hq));
+  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, N, Hkv));
+  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, N, Hkv));
+  MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, N, Hq));
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+  CUtensorMap tq, tk, tv;
+  if (!make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
+      !make_tensor_map_bnhd(&tk, k.p, B, N, Hkv, d, k.sb, k.sn, k.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, v.p, B, N, Hkv, d, v.sb, v.sn, v.sh, 128))
+    return MALA_ERR_TENSOR_MAP;
+
+  FwdParams p;
+  p.o = (__nv_bfloat16*)o.p; p.o_sb = o.sb; p.o_sn = o.sn; p.o_sh = o.sh;
+  p.lse = lse;
+  p.retained = st ? st->retained_per_block : nullptr;
+  p.bitmask = st ? st->tile_bitmask : nullptr;
+  p.totals = st ? (unsigned long long*)st->totals : nullptr;
+  p.status = status;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Tr = (N + 127) / 128; p.words = (p.Tr + 31) / 32; p.causal = causal ? 1 : 0;
+  p.scale_log2 = scale * kLog2e;
+  p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
+  if (p.bitmask) {
+    if (cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * p.Tr * p.words * sizeof(uint32_t), stream) != cudaSuccess)
+      return MALA_ERR_CUDA;
+  }
+  const bool dense = (tau == 0.f);
+  if (d == 128) return dense ? launch_fwd<128, true>(tq, tk, tv, p, stream) : launch_fwd<128, false>(tq, tk, tv, p, stream);
+  return dense ? launch_fwd<64, true>(tq, tk, tv, p, stream) : launch_fwd<64, false>(tq, tk, tv, p, stream);
+}
+
+int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
+             mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d, int causal,
+             float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+  MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
+  if (!lse || !ws) return MALA_ERR_INVALID_ARG;
+  MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, N, Hq));
+  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, N, Hkv));
+  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, N, Hkv));
+  MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, N, Hq));
+  MALA_TRY(check_view(dout.p, dout.sb, dout.sn, dout.sh, B, N, Hq));
+  MALA_TRY(check_view(dq.p, dq.sb, dq.sn, dq.sh, B, N, Hq));
+  MALA_TRY(check_view(dk.p, dk.sb, dk.sn, dk.sh, B, N, Hkv));
+  MALA_TRY(check_view(dv.p, dv.sb, dv.sn, dv.sh, B, N, Hkv));
+  if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
+  if (ws_bytes < bwd_workspace_bytes(B, Hq, N, d)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, N, d, causal ? 1 : 0, scale, tau, ws, status,
+                    (cudaStream_t)cuda_stream);
+}
+
+int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
+                int B, int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws,
+                size_t ws_bytes, void* cuda_stream) {
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  if (num_splits <= 0 || !ws) return MALA_ERR_INVALID_ARG;
+  if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
+  MALA_TRY(check_view(kcache.p, kcache.sb, kcache.sn, kcache.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(vcache.p, vcache.sb, vcache.sn, vcache.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
+  if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
+  if (ws_bytes < decode_workspace_bytes(B, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  return decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
+                       (cudaStream_t)cuda_stream);
+}
+
+}  // extern "C"

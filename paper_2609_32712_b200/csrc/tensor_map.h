@@ -1,0 +1,47 @@
+// Host-side creation of TMA tensor maps for bf16 tensors viewed as [B, N, H, d] with arbitrary
+// element strides (last dimension contiguous).  The driver entry point is looked up at run time so
+// the library has no link-time dependency on libcuda.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mala {
+
+typedef CUresult (*PFN_tensorMapEncodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                             CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                             CUtensorMapFloatOOBfill);
+
+inline PFN_tensorMapEncodeTiled tensor_map_encoder() {
+  static PFN_tensorMapEncodeTiled fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (PFN_tensorMapEncodeTiled)p;
+  }
+  return fn;
+}
+
+// Tensor map over a bf16 [B, N, H, d] view: coordinates (c, n, h, b), box = 64 columns x box_rows rows,
+// 128-byte swizzle, out-of-range rows read as zero.  Returns false if the driver rejects it
+// (base not 16-byte aligned, a stride not a multiple of 16 bytes, ...).
+inline bool make_tensor_map_bnhd(CUtensorMap* out, const void* base, int B, int N, int H, int d, int64_t sb,
+                                 int64_t sn, int64_t sh, int box_rows) {
+  PFN_tensorMapEncodeTiled enc = tensor_map_encoder();
+  if (!enc) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+  // strides of dimensions 1..3 in bytes; a stride of a size-1 dimension only needs to be legal
+  auto legal = [&](int64_t s, int n) -> cuuint64_t { return (n == 1 || s <= 0) ? (cuuint64_t)d * 2 : (cuuint64_t)s * 2; };
+  cuuint64_t strides[3] = {legal(sn, N), legal(sh, H), legal(sb, B)};
+  cuuint32_t box[4] = {64u, (cuuint32_t)box_rows, 1u, 1u};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace mala

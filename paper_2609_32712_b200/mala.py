@@ -1,0 +1,168 @@
+"""ctypes binding of ``libmala.so`` (C ABI in ``include/mala.h``): argument marshalling only.
+
+PyTorch is used for device memory and the current stream; every step of the attention path runs in
+the library's kernels.  There is no CPU or eager fallback: if the library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIBPATH = os.path.join(_HERE, "libmala.so")
+_lib = None
+
+OP_FWD, OP_BWD, OP_DECODE = 0, 1, 2
+
+
+class MalaError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {lib().mala_strerror(code).decode()} (code {code})")
+        self.code = code
+
+
+class _TIn(ctypes.Structure):
+    _fields_ = [("p", ctypes.c_void_p), ("sb", ctypes.c_int64), ("sn", ctypes.c_int64), ("sh", ctypes.c_int64)]
+
+
+class _TOut(ctypes.Structure):
+    _fields_ = [("p", ctypes.c_void_p), ("sb", ctypes.c_int64), ("sn", ctypes.c_int64), ("sh", ctypes.c_int64)]
+
+
+class _Stats(ctypes.Structure):
+    _fields_ = [("retained_per_block", ctypes.c_void_p), ("tile_bitmask", ctypes.c_void_p),
+                ("totals", ctypes.c_void_p)]
+
+
+def lib():
+    """Loads libmala.so (built in-tree by ``paper_2609_32712_b200.build``); fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIBPATH):
+            raise ImportError(f"{_LIBPATH} is missing: run `python -m paper_2609_32712_b200.build` (needs nvcc)")
+        L = ctypes.CDLL(_LIBPATH)
+        i, f, vp, sz = ctypes.c_int, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
+        L.mala_fwd.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, f, f, vp, sz, vp]
+        L.mala_bwd.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, _TOut, _TOut, _TOut, ctypes.POINTER(_Stats),
+                               i, i, i, i, i, i, f, f, vp, sz, vp]
+        L.mala_decode.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp, sz, vp]
+        L.mala_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
+        L.mala_workspace_bytes.restype = sz
+        L.mala_tile_shape.argtypes = [i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
+        L.mala_device_status.argtypes = [ctypes.POINTER(i), i]
+        L.mala_strerror.argtypes = [i]
+        L.mala_strerror.restype = ctypes.c_char_p
+        L.mala_version.restype = i
+        for n in ("mala_fwd", "mala_bwd", "mala_decode", "mala_tile_shape", "mala_device_status"):
+            getattr(L, n).restype = i
+        _lib = L
+    return _lib
+
+
+def _view(t: torch.Tensor, cls):
+    assert t.dtype == torch.bfloat16 and t.dim() == 4 and t.stride(3) == 1, "expects bf16 [B,N,H,d], last dim contiguous"
+    return cls(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def tile_shape(op: int, d: int):
+    bq, bk = ctypes.c_int(0), ctypes.c_int(0)
+    rc = lib().mala_tile_shape(op, d, ctypes.byref(bq), ctypes.byref(bk))
+    if rc != 0:
+        raise MalaError(rc, "mala_tile_shape")
+    return bq.value, bk.value
+
+
+def workspace_bytes(op: int, B: int, Hq: int, Hkv: int, N: int, d: int, num_splits: int = 0) -> int:
+    return int(lib().mala_workspace_bytes(op, B, Hq, Hkv, N, d, num_splits))
+
+
+def device_status(clear: bool = True) -> int:
+    code = ctypes.c_int(0)
+    rc = lib().mala_device_status(ctypes.byref(code), int(clear))
+    if rc != 0:
+        raise MalaError(rc, "mala_device_status")
+    return code.value
+
+
+class Stats:
+    """Device tensors for the optional telemetry of one call."""
+
+    def __init__(self, retained_shape, words: int, device):
+        self.retained = torch.zeros(retained_shape, dtype=torch.int32, device=device)
+        self.bitmask = torch.zeros(tuple(retained_shape) + (words,), dtype=torch.int32, device=device)
+        self.totals = torch.zeros(2, dtype=torch.int64, device=device)
+        self.c = _Stats(self.retained.data_ptr(), self.bitmask.data_ptr(), self.totals.data_ptr())
+
+    def mask(self, n_bits: int) -> torch.Tensor:
+        """Boolean [..., n_bits] expansion of the bitmask (bit x of a row = tile x retained)."""
+        w = self.bitmask.to(torch.int64) & 0xFFFFFFFF
+        bits = (w.unsqueeze(-1) >> torch.arange(32, device=w.device)) & 1
+        return bits.flatten(-2)[..., :n_bits].bool()
+
+
+def _ws(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+def fwd(q, k, v, scale: float, tau: float, causal: bool = True, stats: bool = False, out=None, lse=None, ws=None):
+    """mala_fwd: returns (o [B,N,Hq,d] bf16, lse [B,Hq,N] fp32, Stats or None)."""
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq, N), dtype=torch.float32, device=q.device) if lse is None else lse
+    T = -(-N // 128)
+    st = Stats((B, Hq, T), -(-T // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_FWD, B, Hq, Hkv, N, d), q.device) if ws is None else ws
+    rc = lib().mala_fwd(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TOut), lse.data_ptr(),
+                        ctypes.byref(st.c) if st else None, B, Hq, Hkv, N, d, int(causal), scale, tau,
+                        ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_fwd")
+    return o, lse, st
+
+
+def bwd(q, k, v, o, do, lse, scale: float, tau: float, causal: bool = True, stats: bool = False, ws=None,
+        dq=None, dk=None, dv=None):
+    """mala_bwd: returns (dq, dk, dv, Stats or None)."""
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    T = -(-N // 128)
+    st = Stats((B, Hq, T), -(-T // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_BWD, B, Hq, Hkv, N, d), q.device) if ws is None else ws
+    rc = lib().mala_bwd(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TIn), _view(do, _TIn),
+                        lse.data_ptr(), _view(dq, _TOut), _view(dk, _TOut), _view(dv, _TOut),
+                        ctypes.byref(st.c) if st else None, B, Hq, Hkv, N, d, int(causal), scale, tau,
+                        ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_bwd")
+    return dq, dk, dv, st
+
+
+def decode(q, kcache, vcache, scale: float, tau: float, num_splits: int, stats: bool = False, ws=None, out=None,
+           want_lse: bool = True):
+    """mala_decode: q [B,1,Hq,d]; returns (o [B,1,Hq,d] bf16, lse [B,Hq] fp32 or None, Stats or None)."""
+    B, one, Hq, d = q.shape
+    assert one == 1
+    Nk, Hkv = kcache.shape[1], kcache.shape[2]
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    tps = -(-(-(-Nk // num_splits)) // 128)
+    st = Stats((B, Hkv, num_splits), -(-tps // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_DECODE, B, Hq, Hkv, Nk, d, num_splits), q.device) if ws is None else ws
+    rc = lib().mala_decode(_view(q, _TIn), _view(kcache, _TIn), _view(vcache, _TIn), _view(o, _TOut),
+                           lse.data_ptr() if lse is not None else None, ctypes.byref(st.c) if st else None,
+                           B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_decode")
+    return o, lse, st
