@@ -1,11 +1,666 @@
+// MALA backward (Algorithm 2) for sm_100a.
+//
+//   bwd_preprocess_kernel : D = rowsum(O o dO), lse in the log2 domain and the per-query test offset
+//                           lse2 + log2(tau / L_q), all padded to whole tiles (HBM-bound).
+//   mala_bwd_kernel       : one CTA per (key block j, KV head, batch).  K_j, V_j stay in shared memory;
+//                           for every query head of the group and every query block i >= j (ascending)
+//                           S^T = K_j Q_i^T is recomputed on tensor cores and tested against the saved
+//                           lse (Eq. 4).  Only retained tiles load dO and run dP^T = V dO^T, P^T,
+//                           dS^T = P^T o (dP^T - D), dV += P^T dO, dK += dS^T Q, dQ_i += dS K_j.
+//                           dK, dV accumulate in TMEM; dQ tiles are added to an fp32 accumulator in
+//                           global memory with vector reductions.
+//   bwd_convert_dq_kernel : dq = bf16(scale * accumulator).
+//
+// Warp roles of the main kernel (320 threads):
+//   warp 0     TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
+//   warp 1     UMMA issuer (and, in the MALA kernel, the on-demand dO loads)
+//   warps 2-5  compute group, one thread per key row of the transposed tile
+//   warps 6-9  dQ group, one thread per query row of the dQ tile
 #pragma once
+#include <cuda_runtime.h>
+
 #include "../../include/mala.h"
 #include "sm100_ptx.cuh"
+#include "tensor_map.h"
+
 namespace mala {
-inline bool bwd_set_attributes() { return true; }
-inline size_t bwd_workspace_bytes(int B, int Hq, int N, int d) { return 256; }
-inline int bwd_launch(mala_tin, mala_tin, mala_tin, mala_tin, mala_tin, const float*, mala_tout, mala_tout, mala_tout,
-                      const mala_stats*, int, int, int, int, int, int, float, float, void*, int*, cudaStream_t) {
-  return MALA_ERR_UNSUPPORTED;
+
+struct BwdParams {
+  const float* lse2;    // [B,Hq,Np] lse * log2(e); +inf on padding rows
+  const float* bq;      // [B,Hq,Np] lse2 + log2(tau / L_q); +inf on padding rows
+  const float* Dq;      // [B,Hq,Np] rowsum(O o dO); 0 on padding rows
+  float* dq_acc;        // [B,Hq,Np,D] fp32
+  __nv_bfloat16* dk; int64_t dk_sb, dk_sn, dk_sh;
+  __nv_bfloat16* dv; int64_t dv_sb, dv_sn, dv_sh;
+  uint32_t* retained;   // [B,Hq,Tc] or null
+  uint32_t* bitmask;    // [B,Hq,Tc,words] or null (zero-filled by the host)
+  unsigned long long* totals;
+  int* status;
+  int B, Hq, Hkv, N, Np, T, words, causal;
+  float scale, scale_log2;
+};
+
+template <int D>
+struct BwdCfg {
+  static constexpr int kPanels = D / 64;
+  static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kDsBytes = 128 * 128 * 2;
+  // K, V, Q x2, dO x2.  dS^T (32 KB) of a retained tile overwrites that tile's dO stage once dP and dV
+  // have consumed it (D = 128); for D = 64 a dO stage is too small, so two separate dS stages follow.
+  static constexpr int kSmemBytes = 6 * kTileBytes + (D == 128 ? 0 : 2 * kDsBytes) + 1024;
+  static constexpr int kThreads = 320;
+  static constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
+};
+
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
+
+template <int D, bool kDense>
+__global__ void __launch_bounds__(320, 1)
+mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
+                const BwdParams p) {
+  using Cfg = BwdCfg<D>;
+  constexpr int PAN = Cfg::kPanels;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sK = smem;
+  uint8_t* sV = sK + Cfg::kTileBytes;
+  uint8_t* sQ = sV + Cfg::kTileBytes;          // 2 stages
+  uint8_t* sDO = sQ + 2 * Cfg::kTileBytes;     // 2 stages
+  // dS^T stages, [2 halves][128 key rows][64 q] bf16, 128B swizzle
+  uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
+
+  __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
+      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar;
+  __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int flag[3];
+  __shared__ int dq_info;
+  __shared__ int early_exit;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int j = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
+  const int G = p.Hq / p.Hkv;
+  const int i0 = p.causal ? j : 0;
+  const int ni = p.T - i0;
+  const int n_tot = G * ni;
+  int* status = p.status;
+
+  if (tid == 0) {
+    early_exit = (*(volatile int*)status != 0);
+    mbar_init(&kv_full, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1);
+      mbar_init(&do_full[s], 1); mbar_init(&do_empty[s], 1);
+      mbar_init(&vote_bar[s], 4);
+    }
+    mbar_init(&s_full, 1); mbar_init(&p_full, 4); mbar_init(&dp_full, 1); mbar_init(&ds_full, 4);
+    mbar_init(&dv_done, 1); mbar_init(&grp_bar, 4); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
+    mbar_init(&fin_bar, 1);
+    flag[0] = flag[1] = flag[2] = 0;
+    dq_info = -1;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (early_exit) return;
+  if (warp == 0) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tb = tmem_base_s;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmDO);
+      mbar_arrive_expect_tx(&kv_full, 2 * Cfg::kTileBytes);
+      for (int pn = 0; pn < PAN; ++pn) {
+        tma_load_4d(sK + pn * 16384, &tmK, &kv_full, pn * 64, j * 128, hkv, b);
+        tma_load_4d(sV + pn * 16384, &tmV, &kv_full, pn * 64, j * 128, hkv, b);
+      }
+      bool ok = true;
+      int issued = 0;
+      for (int n = 0; n < n_tot && ok; ++n) {
+        const int s = n & 1, hq = hkv * G + n / ni, i = i0 + n % ni;
+        ok = mbar_wait(&q_empty[s], ((n >> 1) & 1) ^ 1, status);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
+        for (int pn = 0; pn < PAN; ++pn)
+          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, i * 128, hq, b);
+        if (kDense) {
+          ok = mbar_wait(&do_empty[s], ((n >> 1) & 1) ^ 1, status);
+          if (!ok) { mbar_wait(&q_full[s], (n >> 1) & 1, status); break; }
+          mbar_arrive_expect_tx(&do_full[s], Cfg::kTileBytes);
+          for (int pn = 0; pn < PAN; ++pn)
+            tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, i * 128, hq, b);
+        }
+        issued = n + 1;
+      }
+      if (!ok) {
+        mbar_wait(&kv_full, 0, status);
+        for (int n = (issued > 2 ? issued - 2 : 0); n < issued; ++n) {
+          mbar_wait(&q_full[n & 1], (n >> 1) & 1, status);
+          if (kDense) mbar_wait(&do_full[n & 1], (n >> 1) & 1, status);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);    // S^T, dP^T
+      constexpr uint32_t idesc_dv = make_idesc_bf16(128, D, false, true);      // dV (A in TMEM), dK
+      constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);       // dQ
+      const uint32_t aK = smem_u32(sK), aV = smem_u32(sV), aQ = smem_u32(sQ), aDO = smem_u32(sDO), aDS = smem_u32(sDS);
+      bool ok = mbar_wait(&kv_full, 0, status);
+      int r = 0;   // retained tiles so far
+      auto issue_qk = [&](int n) -> bool {
+        const int s = n & 1;
+        if (!mbar_wait(&q_full[s], (n >> 1) & 1, status)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+          mma_ss(tmem_addr(tb, 0, Cfg::kColS), make_smem_desc(aK + off, 16, 1024),
+                 make_smem_desc(aQ + s * Cfg::kTileBytes + off, 16, 1024), idesc_s, k > 0);
+        }
+        tc_commit(&s_full);
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int n = 0; n < n_tot && ok; ++n) {
+        const int s = n & 1, hq = hkv * G + n / ni, i = i0 + n % ni;
+        bool retain = true;
+        if (!kDense) {
+          ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
+          if (!ok) break;
+          retain = (*(volatile int*)&flag[n % 3]) != 0;
+        }
+        const int ds = r & 1;   // dO stage
+        if (retain) {
+          if (!kDense) {
+            ok = mbar_wait(&do_empty[ds], ((r >> 1) & 1) ^ 1, status);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&do_full[ds], Cfg::kTileBytes);
+            for (int pn = 0; pn < PAN; ++pn)
+              tma_load_4d(sDO + ds * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[ds], pn * 64, i * 128, hq, b);
+          }
+          if (r > 0) {   // the dQ tile of the previous retained tile (aliased with dP) has been read out
+            ok = mbar_wait(&dq_empty, (r - 1) & 1, status);
+            if (!ok) break;
+          }
+          ok = mbar_wait(&do_full[ds], (r >> 1) & 1, status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {   // dP^T = V dO^T
+            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), make_smem_desc(aV + off, 16, 1024),
+                   make_smem_desc(aDO + ds * Cfg::kTileBytes + off, 16, 1024), idesc_s, k > 0);
+          }
+          tc_commit(&dp_full);
+          ok = mbar_wait(&p_full, r & 1, status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < 8; ++k)   // dV += P^T dO
+            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + k * 8),
+                   make_smem_desc(aDO + ds * Cfg::kTileBytes + k * 2048, 16384, 1024), idesc_dv,
+                   (r > 0 || k > 0) ? 1u : 0u);
+          tc_commit(&dv_done);
+        }
+        // the score buffer is free again: recompute the next tile's scores while dS is being formed
+        if (n + 1 < n_tot) { ok = issue_qk(n + 1); if (!ok) break; }
+        if (retain) {
+          ok = mbar_wait(&ds_full, r & 1, status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {   // dK += dS^T Q
+            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDK), make_smem_desc(aDS + ds * Cfg::kDsBytes + off, 16, 1024),
+                   make_smem_desc(aQ + s * Cfg::kTileBytes + k * 2048, 16384, 1024), idesc_dv,
+                   (r > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(&q_empty[s]);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j  (into the dP columns)
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), make_smem_desc(aDS + ds * Cfg::kDsBytes + k * 2048, 16384, 1024),
+                   make_smem_desc(aK + k * 2048, 16384, 1024), idesc_dq, k > 0);
+          tc_commit(&do_empty[ds]);   // dO stage (and the dS^T stored over it) is free once dK, dQ retire
+          *(volatile int*)&dq_info = n;
+          mbar_arrive(&dq_info_bar);
+          tc_commit(&dq_full);
+          ++r;
+        } else {
+          mbar_arrive(&q_empty[s]);
+        }
+      }
+      // tell the dQ group that nothing more will come, then wait for every MMA to retire
+      bool ok2 = true;
+      if (r > 0) ok2 = mbar_wait(&dq_empty, (r - 1) & 1, status);
+      if (ok2) { *(volatile int*)&dq_info = -1; mbar_arrive(&dq_info_bar); }
+      tc_commit(&fin_bar);
+      mbar_wait(&fin_bar, 0, status);
+      if (!ok && !kDense) {
+        for (int u = (r > 1 ? r - 1 : 0); u <= r; ++u) mbar_wait(&do_full[u & 1], (u >> 1) & 1, status);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ compute group: thread = key row
+    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
+    const int rl = (int)lane_base + lane;
+    const bool valid_key = (j * 128 + rl) < p.N;
+    const float c2 = p.scale_log2;
+    const bool stat_thread = (warp == 2 && lane == 0);
+    bool ok = true;
+    int r = 0;
+    int r_head = 0;
+    uint32_t bm_bits = 0;
+    int bm_word = -1;
+
+    auto vec_index = [&](int n) -> size_t {
+      const int hq = hkv * G + n / ni, i = i0 + n % ni;
+      return ((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128 + rl;
+    };
+    // per-query vectors of tile 0 into slot 0, made visible by a first pass through vote_bar[1]
+    {
+      const size_t x = vec_index(0);
+      vec[0][0][rl] = p.lse2[x];
+      vec[0][1][rl] = p.bq[x];
+      vec[0][2][rl] = p.Dq[x];
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&grp_bar);
+    ok = mbar_wait(&grp_bar, 0, status);
+    ok = __all_sync(0xffffffffu, ok);
+
+    for (int n = 0; n < n_tot && ok; ++n) {
+      const int hq_n = n / ni, i = i0 + n % ni;
+      const int slot = n % 3;
+      // prefetch the per-query vectors of the next tile
+      float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
+      if (n + 1 < n_tot) {
+        const size_t x = vec_index(n + 1);
+        nx0 = p.lse2[x]; nx1 = p.bq[x]; nx2 = p.Dq[x];
+      }
+      ok = mbar_wait(&s_full, n & 1, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t s0[32], s1[32], s2[32], s3[32];
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 0), s0);
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 32), s1);
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 64), s2);
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 96), s3);
+      tmem_wait_ld();
+      if (p.causal && i == j) {   // diagonal tile: entry (key rl, query e) is legal iff rl <= e
+        const uint32_t ninf = 0xff800000u;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          if (e < rl) s0[e] = ninf;
+          if (e + 32 < rl) s1[e] = ninf;
+          if (e + 64 < rl) s2[e] = ninf;
+          if (e + 96 < rl) s3[e] = ninf;
+        }
+      }
+      // publish the next tile's vectors (slot (n+1) % 3 was last read two tiles ago)
+      {
+        const int ns = (n + 1) % 3;
+        vec[ns][0][rl] = nx0; vec[ns][1][rl] = nx1; vec[ns][2][rl] = nx2;
+      }
+      bool retain = true;
+      {
+        // Eq. 4: skip iff s - lse_q < log(tau / L_q) on every valid entry
+        bool vote = false;
+        if (!kDense) {
+          float crit = -INFINITY;
+          const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float4 x0 = bb[e], x1 = bb[8 + e], x2 = bb[16 + e], x3 = bb[24 + e];
+            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s0[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(s0[4 * e + 1]), c2, -x0.y)),
+                                     fmaxf(fmaf(__uint_as_float(s0[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(s0[4 * e + 3]), c2, -x0.w))));
+            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s1[4 * e + 0]), c2, -x1.x), fmaf(__uint_as_float(s1[4 * e + 1]), c2, -x1.y)),
+                                     fmaxf(fmaf(__uint_as_float(s1[4 * e + 2]), c2, -x1.z), fmaf(__uint_as_float(s1[4 * e + 3]), c2, -x1.w))));
+            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s2[4 * e + 0]), c2, -x2.x), fmaf(__uint_as_float(s2[4 * e + 1]), c2, -x2.y)),
+                                     fmaxf(fmaf(__uint_as_float(s2[4 * e + 2]), c2, -x2.z), fmaf(__uint_as_float(s2[4 * e + 3]), c2, -x2.w))));
+            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s3[4 * e + 0]), c2, -x3.x), fmaf(__uint_as_float(s3[4 * e + 1]), c2, -x3.y)),
+                                     fmaxf(fmaf(__uint_as_float(s3[4 * e + 2]), c2, -x3.z), fmaf(__uint_as_float(s3[4 * e + 3]), c2, -x3.w))));
+          }
+          vote = valid_key && !(crit < 0.f);
+        }
+        const bool any = __any_sync(0xffffffffu, vote);
+        if (lane == 0) {
+          if (any) *(volatile int*)&flag[n % 3] = 1;
+          if (warp == 2) *(volatile int*)&flag[(n + 1) % 3] = 0;
+          tc_fence_before();
+          mbar_arrive(&vote_bar[n & 1]);
+        }
+        ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (!kDense) retain = (*(volatile int*)&flag[n % 3]) != 0;
+      }
+      if (stat_thread && n % ni == 0) { r_head = 0; bm_bits = 0; bm_word = -1; }
+      if (retain) {
+        if (stat_thread) {
+          ++r_head;
+          if (p.bitmask) {
+            uint32_t* bm_row = p.bitmask + ((size_t)(b * p.Hq + hkv * G + hq_n) * p.T + j) * p.words;
+            if ((i >> 5) != bm_word) {
+              if (bm_word >= 0) bm_row[bm_word] = bm_bits;
+              bm_word = i >> 5;
+              bm_bits = 0;
+            }
+            bm_bits |= 1u << (i & 31);
+          }
+        }
+        // P^T = exp2(s * c2 - lse2_q) (bf16): kept packed in registers and written over S^T in TMEM
+        uint32_t pk[64];
+        const float4* ll = reinterpret_cast<const float4*>(vec[slot][0]);
+#define MALA_BWD_P(SRC, CH)                                                                  \
+        {                                                                                    \
+          _Pragma("unroll") for (int e = 0; e < 8; ++e) {                                    \
+            const float4 x = ll[(CH) * 8 + e];                                               \
+            const float p0 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 0]), c2, -x.x));     \
+            const float p1 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 1]), c2, -x.y));     \
+            const float p2 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 2]), c2, -x.z));     \
+            const float p3 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 3]), c2, -x.w));     \
+            pk[(CH) * 16 + 2 * e] = pack_bf16x2(p0, p1);                                     \
+            pk[(CH) * 16 + 2 * e + 1] = pack_bf16x2(p2, p3);                                 \
+          }                                                                                  \
+          uint32_t tmp[16];                                                                  \
+          _Pragma("unroll") for (int e = 0; e < 16; ++e) tmp[e] = pk[(CH) * 16 + e];         \
+          tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + (CH) * 16), tmp);                \
+        }
+        MALA_BWD_P(s0, 0)
+        MALA_BWD_P(s1, 1)
+        MALA_BWD_P(s2, 2)
+        MALA_BWD_P(s3, 3)
+#undef MALA_BWD_P
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full);
+        // dS^T = P^T o (dP^T - D_q), bf16, into shared memory for the dK and dQ MMAs
+        // dS^T goes where this tile's dO lies (D = 128): wait until dP and dV have consumed it
+        ok = mbar_wait(&dp_full, r & 1, status);
+        if (ok) ok = mbar_wait(&dv_done, r & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const float4* dd = reinterpret_cast<const float4*>(vec[slot][2]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t dp[32];
+          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + c * 32), dp);
+          tmem_wait_ld();
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const float4 x = dd[c * 8 + v * 2 + u];
+              const uint32_t pa = pk[c * 16 + v * 4 + 2 * u], pb = pk[c * 16 + v * 4 + 2 * u + 1];
+              const float p0 = __uint_as_float(pa << 16), p1 = __uint_as_float(pa & 0xffff0000u);
+              const float p2 = __uint_as_float(pb << 16), p3 = __uint_as_float(pb & 0xffff0000u);
+              const float d0 = p0 * (__uint_as_float(dp[v * 8 + u * 4 + 0]) - x.x);
+              const float d1 = p1 * (__uint_as_float(dp[v * 8 + u * 4 + 1]) - x.y);
+              const float d2 = p2 * (__uint_as_float(dp[v * 8 + u * 4 + 2]) - x.z);
+              const float d3 = p3 * (__uint_as_float(dp[v * 8 + u * 4 + 3]) - x.w);
+              w[2 * u] = pack_bf16x2(d0, d1);
+              w[2 * u + 1] = pack_bf16x2(d2, d3);
+            }
+            const uint32_t col = (uint32_t)((c & 1) * 32 + v * 8);
+            *reinterpret_cast<uint4*>(sDS + (r & 1) * Cfg::kDsBytes + (c >> 1) * 16384 + sw128_offset((uint32_t)rl, col)) =
+                make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ds_full);
+        ++r;
+      }
+      if (stat_thread && (n % ni == ni - 1)) {   // last tile of this query head
+        const size_t row = (size_t)(b * p.Hq + hkv * G + hq_n) * p.T + j;
+        if (p.bitmask && bm_word >= 0) p.bitmask[row * p.words + bm_word] = bm_bits;
+        if (p.retained) p.retained[row] = (uint32_t)r_head;
+        if (p.totals) {
+          atomicAdd(&p.totals[0], (unsigned long long)r_head);
+          atomicAdd(&p.totals[1], (unsigned long long)ni);
+        }
+      }
+    }
+
+    // epilogue: dK_j (x scale), dV_j -> global
+    if (ok) {
+      ok = mbar_wait(&fin_bar, 0, status);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      const int key = j * 128 + rl;
+      __nv_bfloat16* dvrow = p.dv + (int64_t)b * p.dv_sb + (int64_t)key * p.dv_sn + (int64_t)hkv * p.dv_sh;
+      __nv_bfloat16* dkrow = p.dk + (int64_t)b * p.dk_sb + (int64_t)key * p.dk_sn + (int64_t)hkv * p.dk_sh;
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        __nv_bfloat16* out = which ? dkrow : dvrow;
+        const float f = which ? p.scale : 1.f;
+        const uint32_t col0 = which ? Cfg::kColDK : Cfg::kColDV;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          if (r > 0) {
+            tmem_ld_x32(tmem_addr(tb, lane_base, col0 + c * 32), o);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = 0u;
+          }
+          if (valid_key) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint4 w;
+              w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * f, __uint_as_float(o[8 * v + 1]) * f);
+              w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * f, __uint_as_float(o[8 * v + 3]) * f);
+              w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * f, __uint_as_float(o[8 * v + 5]) * f);
+              w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * f, __uint_as_float(o[8 * v + 7]) * f);
+              *reinterpret_cast<uint4*>(out + c * 32 + v * 8) = w;
+            }
+          }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ dQ group: thread = query row
+    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
+    const int rl = (int)lane_base + lane;
+    for (int k = 0;; ++k) {
+      bool ok = mbar_wait(&dq_info_bar, k & 1, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const int n = *(volatile int*)&dq_info;
+      if (n < 0) break;
+      ok = mbar_wait(&dq_full, k & 1, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int hq = hkv * G + n / ni, i = i0 + n % ni;
+      float* dst = p.dq_acc + (((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128 + rl) * D;
+      uint32_t a0[32], a1[32];
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 0), a0);
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 32), a1);
+      uint32_t a2[32], a3[32];
+      if (D == 128) {
+        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 64), a2);
+        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 96), a3);
+      }
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused; the adds continue from registers
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {
+        red_add_v4(dst + v * 4, __uint_as_float(a0[4 * v]), __uint_as_float(a0[4 * v + 1]), __uint_as_float(a0[4 * v + 2]), __uint_as_float(a0[4 * v + 3]));
+        red_add_v4(dst + 32 + v * 4, __uint_as_float(a1[4 * v]), __uint_as_float(a1[4 * v + 1]), __uint_as_float(a1[4 * v + 2]), __uint_as_float(a1[4 * v + 3]));
+      }
+      if (D == 128) {
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+          red_add_v4(dst + 64 + v * 4, __uint_as_float(a2[4 * v]), __uint_as_float(a2[4 * v + 1]), __uint_as_float(a2[4 * v + 2]), __uint_as_float(a2[4 * v + 3]));
+          red_add_v4(dst + 96 + v * 4, __uint_as_float(a3[4 * v]), __uint_as_float(a3[4 * v + 1]), __uint_as_float(a3[4 * v + 2]), __uint_as_float(a3[4 * v + 3]));
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+// D = rowsum(O o dO), lse2 = lse * log2(e), bq = lse2 + log2(tau / L_q); one warp per (b, h, row).
+__global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sn, int64_t o_sh,
+                                      const __nv_bfloat16* __restrict__ dout, int64_t d_sb, int64_t d_sn, int64_t d_sh,
+                                      const float* __restrict__ lse, float* __restrict__ lse2, float* __restrict__ bq,
+                                      float* __restrict__ Dq, int B, int Hq, int N, int Np, int d, int causal,
+                                      float log2_tau) {
+  const int warps_per_block = blockDim.x >> 5;
+  const long long w = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const long long total = (long long)B * Hq * Np;
+  if (w >= total) return;
+  const int row = (int)(w % Np);
+  const int h = (int)((w / Np) % Hq);
+  const int b = (int)(w / ((long long)Np * Hq));
+  if (row >= N) {
+    if (lane == 0) { lse2[w] = INFINITY; bq[w] = INFINITY; Dq[w] = 0.f; }
+    return;
+  }
+  const __nv_bfloat16* op = o + b * o_sb + row * o_sn + h * o_sh;
+  const __nv_bfloat16* dp = dout + b * d_sb + row * d_sn + h * d_sh;
+  float acc = 0.f;
+  for (int c = lane * 2; c < d; c += 64) {
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(op + c);
+    const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dp + c);
+    acc += __bfloat162float(a.x) * __bfloat162float(g.x) + __bfloat162float(a.y) * __bfloat162float(g.y);
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+  if (lane == 0) {
+    const float l2 = lse[((size_t)b * Hq + h) * N + row] * 1.4426950408889634f;
+    const float L = causal ? (float)(row + 1) : (float)N;
+    lse2[w] = l2;
+    bq[w] = l2 + (log2_tau - log2f(L));
+    Dq[w] = acc;
+  }
+}
+
+// dq = bf16(scale * acc); one thread per 8 output elements
+__global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int64_t sb,
+                                      int64_t sn, int64_t sh, int B, int Hq, int N, int Np, int d, float scale) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = d / 8;
+  const long long total = (long long)B * Hq * N * per_row;
+  if (idx >= total) return;
+  const int c = (int)(idx % per_row) * 8;
+  const int row = (int)((idx / per_row) % N);
+  const int h = (int)((idx / ((long long)per_row * N)) % Hq);
+  const int b = (int)(idx / ((long long)per_row * N * Hq));
+  const float4* src = reinterpret_cast<const float4*>(acc + (((size_t)b * Hq + h) * Np + row) * d + c);
+  const float4 x = src[0], y = src[1];
+  uint4 w;
+  w.x = pack_bf16x2(x.x * scale, x.y * scale);
+  w.y = pack_bf16x2(x.z * scale, x.w * scale);
+  w.z = pack_bf16x2(y.x * scale, y.y * scale);
+  w.w = pack_bf16x2(y.z * scale, y.w * scale);
+  *reinterpret_cast<uint4*>(dq + b * sb + row * sn + h * sh + c) = w;
+}
+
+inline size_t bwd_align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+inline size_t bwd_workspace_bytes(int B, int Hq, int N, int d) {
+  const size_t Np = (size_t)((N + 127) / 128) * 128;
+  return bwd_align256((size_t)B * Hq * Np * d * sizeof(float)) + 3 * bwd_align256((size_t)B * Hq * Np * sizeof(float));
+}
+
+inline bool bwd_set_attributes() {
+  bool ok = true;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes) == cudaSuccess;
+  return ok;
+}
+
+template <int D, bool kDense>
+inline int bwd_launch_main(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
+                           const BwdParams& p, cudaStream_t stream) {
+  dim3 grid(p.T, p.Hkv, p.B);
+  mala_bwd_kernel<D, kDense><<<grid, BwdCfg<D>::kThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, p);
+  return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
+}
+
+inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
+                      mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d,
+                      int causal, float scale, float tau, void* ws, int* status, cudaStream_t stream) {
+  const int T = (N + 127) / 128, Np = T * 128;
+  uint8_t* w = (uint8_t*)ws;
+  float* acc = (float*)w;
+  w += bwd_align256((size_t)B * Hq * Np * d * sizeof(float));
+  const size_t vbytes = bwd_align256((size_t)B * Hq * Np * sizeof(float));
+  float* lse2 = (float*)w;
+  float* bq = (float*)(w + vbytes);
+  float* Dq = (float*)(w + 2 * vbytes);
+
+  CUtensorMap tq, tk, tv, tdo;
+  if (!make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
+      !make_tensor_map_bnhd(&tk, k.p, B, N, Hkv, d, k.sb, k.sn, k.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, v.p, B, N, Hkv, d, v.sb, v.sn, v.sh, 128) ||
+      !make_tensor_map_bnhd(&tdo, dout.p, B, N, Hq, d, dout.sb, dout.sn, dout.sh, 128))
+    return MALA_ERR_TENSOR_MAP;
+
+  if (cudaMemsetAsync(acc, 0, (size_t)B * Hq * Np * d * sizeof(float), stream) != cudaSuccess) return MALA_ERR_CUDA;
+  BwdParams p;
+  p.lse2 = lse2; p.bq = bq; p.Dq = Dq; p.dq_acc = acc;
+  p.dk = (__nv_bfloat16*)dk.p; p.dk_sb = dk.sb; p.dk_sn = dk.sn; p.dk_sh = dk.sh;
+  p.dv = (__nv_bfloat16*)dv.p; p.dv_sb = dv.sb; p.dv_sn = dv.sn; p.dv_sh = dv.sh;
+  p.retained = st ? st->retained_per_block : nullptr;
+  p.bitmask = st ? st->tile_bitmask : nullptr;
+  p.totals = st ? (unsigned long long*)st->totals : nullptr;
+  p.status = status;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Np = Np; p.T = T; p.words = (T + 31) / 32; p.causal = causal;
+  p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
+  if (p.bitmask &&
+      cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * T * p.words * sizeof(uint32_t), stream) != cudaSuccess)
+    return MALA_ERR_CUDA;
+
+  {
+    const long long rows = (long long)B * Hq * Np;
+    const int wpb = 8;
+    const unsigned blocks = (unsigned)((rows + wpb - 1) / wpb);
+    bwd_preprocess_kernel<<<blocks, wpb * 32, 0, stream>>>((const __nv_bfloat16*)o.p, o.sb, o.sn, o.sh,
+                                                          (const __nv_bfloat16*)dout.p, dout.sb, dout.sn, dout.sh, lse,
+                                                          lse2, bq, Dq, B, Hq, N, Np, d, causal,
+                                                          tau > 0.f ? log2f(tau) : -INFINITY);
+    if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
+  }
+  const bool dense = (tau == 0.f);
+  int rc;
+  if (d == 128) rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, p, stream);
+  else rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, p, stream);
+  if (rc != MALA_OK) return rc;
+  {
+    const long long total = (long long)B * Hq * N * (d / 8);
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(acc, (__nv_bfloat16*)dq.p, dq.sb, dq.sn, dq.sh, B, Hq, N, Np, d,
+                                                      scale);
+    if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
+  }
+  return MALA_OK;
+}
+
 }  // namespace mala

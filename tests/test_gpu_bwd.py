@@ -1,0 +1,99 @@
+"""GPU parity of mala_bwd (through the C ABI) against the fp64 oracle.
+
+Isolated runs give the oracle the SAME forward output o (bf16) and saved lse (fp32) that the GPU backward
+receives (those written by mala_fwd), so that only the backward kernels are under test; end-to-end runs
+compare GPU fwd -> bwd with oracle fwd -> bwd in fp64."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_32712_b200 import workloads as W
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mala():
+    from paper_2609_32712_b200 import mala as m
+    m.lib()
+    return m
+
+
+def _check_bwd_masks(st, ref, B, Hq, T, causal, band_extra=0.0):
+    gm = st.mask(T).cpu().numpy()                       # [B,Hq,Tc,Tr]
+    flips = 0
+    for b in range(B):
+        for h in range(Hq):
+            for j in range(T):
+                om, oc = ref["mask"][b, h, j], ref["crit"][b, h, j]
+                for i in range(T):
+                    if om[i] == 0:
+                        assert not gm[b, h, j, i]
+                        continue
+                    if bool(gm[b, h, j, i]) != (om[i] == 2):
+                        assert abs(oc[i]) <= parity.MASK_BAND + band_extra, (b, h, j, i, oc[i])
+                        flips += 1
+                assert int(st.retained[b, h, j]) == int(gm[b, h, j].sum())
+    return flips
+
+
+def _run_isolated(mala, oracle, w, tau, causal=True):
+    q, k, v, do = (w[x].cuda() for x in ("q", "k", "v", "do"))
+    B, N, Hq, d = q.shape
+    o, lse, fst = mala.fwd(q, k, v, w["scale"], tau, causal=causal, stats=True)
+    dq, dk, dv, st = mala.bwd(q, k, v, o, do, lse, w["scale"], tau, causal=causal, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    Bq, Bk = mala.tile_shape(mala.OP_BWD, d)
+    ref = oracle.bwd(w["q"], w["k"], w["v"], o.float().cpu(), w["do"], lse.cpu().numpy(), w["scale"], tau, Bq, Bk,
+                     causal=causal)
+    T = -(-N // Bq)
+    flips = _check_bwd_masks(st, ref, B, Hq, T, causal)
+    e = [parity.check_grad(dq.float().cpu().numpy(), ref["dq"], "dq"),
+         parity.check_grad(dk.float().cpu().numpy(), ref["dk"], "dk"),
+         parity.check_grad(dv.float().cpu().numpy(), ref["dv"], "dv")]
+    # nesting: backward support inside forward support, same partition, nothing stored
+    fm = fst.mask(T).cpu().numpy()
+    bm = st.mask(T).cpu().numpy().transpose(0, 1, 3, 2)
+    assert (bm <= fm).all()
+    return dict(flips=flips, err=e, skipped=int((ref["mask"] == 1).sum()), retained=int((ref["mask"] == 2).sum()),
+                totals=st.totals.cpu().numpy())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("N,d,Hq,Hkv", [(128, 128, 1, 1), (384, 128, 2, 1), (333, 128, 4, 2), (512, 64, 2, 2),
+                                        (200, 64, 2, 1)])
+def test_bwd_small_shapes_literal(mala, oracle, N, d, Hq, Hkv, tau):
+    w = W.custom_prefill(2, Hq, Hkv, N, d, seed=N + d)
+    _run_isolated(mala, oracle, w, tau)
+
+
+@pytest.mark.parametrize("tau", [1e-5, 1e-4, 1e-3, 1.0])
+@pytest.mark.parametrize("N,d", [(1024, 128), (1000, 128), (1024, 64)])
+def test_bwd_skipping_regime(mala, oracle, N, d, tau):
+    w = W.custom_prefill(1, 4, 2, N, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=7, preset="R")
+    res = _run_isolated(mala, oracle, w, tau)
+    assert res["skipped"] > 0
+    assert res["totals"][1] == res["retained"] + res["skipped"]
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-3])
+def test_bwd_cfg1_end_to_end(mala, oracle, tau):
+    w = W.make_prefill(W.prefill_config("cfg1"))
+    q, k, v, do = (w[x].cuda() for x in ("q", "k", "v", "do"))
+    o, lse, _ = mala.fwd(q, k, v, w["scale"], tau)
+    dq, dk, dv, st = mala.bwd(q, k, v, o, do, lse, w["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    f = oracle.fwd(w["q"], w["k"], w["v"], w["scale"], tau, 128, 128)
+    g = oracle.bwd(w["q"], w["k"], w["v"], f["o"], w["do"], f["lse"], w["scale"], tau, 128, 128)
+    _check_bwd_masks(st, g, 1, 2, 8, True, band_extra=1e-3)
+    parity.check_grad(dq.float().cpu().numpy(), g["dq"], "dq")
+    parity.check_grad(dk.float().cpu().numpy(), g["dk"], "dk")
+    parity.check_grad(dv.float().cpu().numpy(), g["dv"], "dv")
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-2])
+def test_bwd_non_causal(mala, oracle, tau):
+    w = W.custom_prefill(1, 2, 1, 300, 128, head_types=["peaked", "diffuse"], seed=5, preset="R")
+    _run_isolated(mala, oracle, w, tau, causal=False)
