@@ -1,11 +1,99 @@
+// Split-KV decode ("Fused decoding execution"): the split kernel is the decode mode of the forward
+// kernel template (mala_fwd.cuh); this file holds the normalizer-aware merge of the split partials,
+// the workspace layout and the launch code.
 #pragma once
+#include <cuda_runtime.h>
+
 #include "../../include/mala.h"
-#include "sm100_ptx.cuh"
+#include "mala_fwd.cuh"
+#include "tensor_map.h"
+
 namespace mala {
-inline bool decode_set_attributes() { return true; }
-inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) { return 256; }
-inline int decode_launch(mala_tin, mala_tin, mala_tin, mala_tout, float*, const mala_stats*, int, int, int, int, int,
-                         float, float, int, void*, int*, cudaStream_t) {
-  return MALA_ERR_UNSUPPORTED;
+
+// lse = log sum_s exp(lse_s), o = sum_s exp(lse_s - lse) o_s; one block per (b, query head), one thread
+// per output column.
+template <int D>
+__global__ void __launch_bounds__(D)
+decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part, __nv_bfloat16* __restrict__ o,
+                    int64_t o_sb, int64_t o_sh, float* __restrict__ lse_out, int Hq, int num_splits) {
+  const int bh = blockIdx.x, b = bh / Hq, h = bh % Hq, c = threadIdx.x;
+  const float* lp = lse_part + (size_t)bh * num_splits;
+  float mx = -INFINITY;
+  for (int s = 0; s < num_splits; ++s) mx = fmaxf(mx, lp[s]);
+  float Z = 0.f, acc = 0.f;
+  for (int s = 0; s < num_splits; ++s) {
+    const float ls = lp[s];
+    if (ls == -INFINITY) continue;
+    const float w = exp2f((ls - mx) * 1.4426950408889634f);
+    Z += w;
+    acc += w * o_part[((size_t)bh * num_splits + s) * D + c];
+  }
+  o[b * o_sb + h * o_sh + c] = __float2bfloat16(acc / Z);
+  if (lse_out && c == 0) lse_out[bh] = mx + logf(Z);
 }
+
+inline size_t decode_align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) {
+  return decode_align256((size_t)B * Hq * S * d * sizeof(float)) + decode_align256((size_t)B * Hq * S * sizeof(float));
+}
+
+inline bool decode_set_attributes() {
+  bool ok = true;
+  ok = ok && cudaFuncSetAttribute(mala_fwd_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128, false>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_fwd_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128, true>::kSmemBytes) == cudaSuccess;
+  return ok;
+}
+
+// Launches the split kernel and the merge on `stream`.  o_part / lse_part: caller-provided scratch of
+// decode_workspace_bytes() bytes in total (o_part first).
+inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala_tout o, float* lse_opt,
+                                      const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
+                                      float tau, int num_splits, float* o_part, float* lse_part, int* status,
+                                      cudaStream_t stream) {
+  if (d != 128) return MALA_ERR_UNSUPPORTED;
+  const int per = (Nk + num_splits - 1) / num_splits;
+  const int tps = (per + 127) / 128;
+
+  CUtensorMap tq, tk, tv;
+  // q [B,1,Hq,d] viewed with the heads as rows: one 128-row box starting at the group's first head
+  if (!make_tensor_map_bnhd(&tq, q.p, B, Hq, 1, d, q.sb, q.sh, 0, 128) ||
+      !make_tensor_map_bnhd(&tk, kc.p, B, Nk, Hkv, d, kc.sb, kc.sn, kc.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, vc.p, B, Nk, Hkv, d, vc.sb, vc.sn, vc.sh, 128))
+    return MALA_ERR_TENSOR_MAP;
+
+  FwdParams p;
+  p.o = nullptr; p.o_sb = p.o_sn = p.o_sh = 0; p.lse = nullptr;
+  p.retained = st ? st->retained_per_block : nullptr;
+  p.bitmask = st ? st->tile_bitmask : nullptr;
+  p.totals = st ? (unsigned long long*)st->totals : nullptr;
+  p.status = status;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = Nk; p.Tr = 0; p.words = (tps + 31) / 32; p.causal = 0;
+  p.o_part = o_part; p.lse_part = lse_part; p.tps = tps; p.num_splits = num_splits;
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
+  if (p.bitmask &&
+      cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hkv * num_splits * p.words * sizeof(uint32_t), stream) != cudaSuccess)
+    return MALA_ERR_CUDA;
+
+  dim3 grid(num_splits, Hkv, B);
+  if (tau == 0.f)
+    mala_fwd_kernel<128, true, true><<<grid, 192, FwdCfg<128, true>::kSmemBytes, stream>>>(tq, tk, tv, p);
+  else
+    mala_fwd_kernel<128, false, true><<<grid, 192, FwdCfg<128, false>::kSmemBytes, stream>>>(tq, tk, tv, p);
+  if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
+  decode_merge_kernel<128><<<B * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb, o.sh, lse_opt, Hq,
+                                                       num_splits);
+  return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
+}
+
+inline int decode_launch(mala_tin q, mala_tin kc, mala_tin vc, mala_tout o, float* lse_opt, const mala_stats* st, int B,
+                         int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws, int* status,
+                         cudaStream_t stream) {
+  float* o_part = (float*)ws;
+  float* lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Hq * num_splits * d * sizeof(float)));
+  return decode_launch_with_scratch(q, kc, vc, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, o_part,
+                                    lse_part, status, stream);
+}
+
 }  // namespace mala

@@ -1,4 +1,4 @@
-// MALA forward (Algorithm 1) for sm_100a.
+// MALA forward (Algorithm 1) and split-KV decode ("Fused decoding execution") for sm_100a.
 //
 // One CTA owns one 128-row query block of one (batch, query head) and walks its legal key blocks
 // from the diagonal toward earlier keys.  Warp roles (192 threads):
@@ -10,6 +10,12 @@
 //                 votes on retention (Eq. 3), and for retained tiles writes P (bf16) over S in TMEM
 //                 and keeps the running (m, l); O is rescaled lazily in TMEM.
 // All synchronisation is by mbarriers with bounded waits.
+//
+// Decode mode (kDecode): one CTA owns one split of one (batch, KV head).  The rows of its "query
+// block" are the G = Hq/Hkv query heads that share the KV head (rows G..127 of the tile hold other
+// heads or zeros and are ignored), L = Nk for every row, tiles of the split are visited newest
+// first, and the CTA writes a normalised fp32 partial output and its log-normalizer per head.  Only
+// one softmax warp (TMEM lanes 0..31) is active.
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -24,6 +30,10 @@ struct FwdParams {
   unsigned long long* totals;    // [2] or null
   int* status;
   int B, Hq, Hkv, N, Tr, words, causal;
+  // decode only
+  float* o_part;                 // [B, Hq, num_splits, D] fp32, normalised per split
+  float* lse_part;               // [B, Hq, num_splits] natural log; -inf for an empty split
+  int tps, num_splits;           // tiles per split, number of splits (N is Nk)
   float scale_log2;              // scale * log2(e)
   float log2_tau;                // log2(tau); unused by the dense kernel
 };
@@ -40,7 +50,7 @@ struct FwdCfg {
   static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
 };
 
-template <int D, bool kDense>
+template <int D, bool kDense, bool kDecode>
 __global__ void __launch_bounds__(192, 1)
 mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const FwdParams p) {
@@ -59,12 +69,30 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __shared__ int early_exit;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int i = p.Tr - 1 - (int)blockIdx.x;   // longest blocks first
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int hkv = h / (p.Hq / p.Hkv);
-  const int Tc = p.Tr;
-  const int T = p.causal ? (i + 1) : Tc;      // tiles to visit
-  const int j0 = p.causal ? i : (Tc - 1);     // first visited key block
+  const int G = p.Hq / p.Hkv;
+  const int b = blockIdx.z;
+  int i, h, hkv, T, j0, q_row, q_head;
+  if (kDecode) {
+    const int split = blockIdx.x;
+    hkv = blockIdx.y;
+    h = hkv * G;
+    i = split;
+    const int lo = split * p.tps * 128;
+    const int hi = min(p.N, lo + p.tps * 128);
+    T = hi > lo ? (hi - lo + 127) / 128 : 0;   // legal tiles of this split
+    j0 = lo / 128 + T - 1;                     // newest tile first
+    q_row = hkv * G;                           // rows of the Q tile are query heads
+    q_head = 0;
+  } else {
+    i = p.Tr - 1 - (int)blockIdx.x;            // longest blocks first
+    h = blockIdx.y;
+    hkv = h / G;
+    T = p.causal ? (i + 1) : p.Tr;             // tiles to visit
+    j0 = p.causal ? i : (p.Tr - 1);            // first visited key block
+    q_row = i * 128;
+    q_head = h;
+  }
+  constexpr int kSoftmaxWarps = kDecode ? 1 : 4;
   int* status = p.status;
 
   if (tid == 0) {
@@ -72,7 +100,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init(&q_full, 1);
     for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); }
     for (int s = 0; s < VS; ++s) { mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&s_full[s], 1); mbar_init(&vote_bar[s], 4); mbar_init(&p_full[s], 4); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&s_full[s], 1); mbar_init(&vote_bar[s], kSoftmaxWarps); mbar_init(&p_full[s], kSoftmaxWarps);
+    }
     mbar_init(&o_done, 1);
     mbar_init(&fin_bar, 1);
     flag[0] = flag[1] = flag[2] = 0;
@@ -91,7 +121,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
       mbar_arrive_expect_tx(&q_full, Cfg::kTileBytes);
-      for (int pn = 0; pn < PAN; ++pn) tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, i * 128, h, b);
+      for (int pn = 0; pn < PAN; ++pn) tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, q_row, q_head, b);
       int issued = 0;
       bool ok = true;
       for (int t = 0; t < T && ok; ++t) {
@@ -142,7 +172,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ++v_issued;
         return true;
       };
-      if (ok) ok = issue_qk(0);
+      if (ok && T > 0) ok = issue_qk(0);
       if (kDense) {
         for (int t = 0; t < VS - 1 && t < T && ok; ++t) ok = issue_v(t);
       }
@@ -182,22 +212,24 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int u = (v_issued > VS ? v_issued - VS : 0); u < v_issued; ++u) mbar_wait(&v_full[u % VS], (u / VS) & 1, status);
       }
     }
-  } else {
+  } else if (!kDecode || warp == 4) {
     // ------------------------------------------------------------------ softmax group: one thread per row
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;            // row inside the block
-    const int row = i * 128 + rl;
-    const bool valid = row < p.N;
+    const int row = kDecode ? rl : i * 128 + rl;
+    const bool valid = kDecode ? (rl < G) : (row < p.N);
     const float c2 = p.scale_log2;
-    const float Lq = p.causal ? (float)(row + 1) : (float)p.N;
+    const float Lq = (p.causal && !kDecode) ? (float)(row + 1) : (float)p.N;
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f(Lq));
     float m_ref = -INFINITY, l = 0.f;
     int r = 0;                                       // retained tiles so far
     bool ok = true;
     uint32_t bm_bits = 0;
     int bm_word = -1;
-    const bool stat_thread = (warp == 2 && lane == 0);
-    uint32_t* bm_row = p.bitmask ? p.bitmask + ((size_t)(b * p.Hq + h) * p.Tr + i) * p.words : nullptr;
+    const bool stat_thread = (warp == (kDecode ? 4 : 2) && lane == 0);
+    // telemetry row: (b, h, query block) in prefill, (b, hkv, split) in decode
+    const size_t stat_row = kDecode ? ((size_t)(b * p.Hkv + hkv) * p.num_splits + i) : ((size_t)(b * p.Hq + h) * p.Tr + i);
+    uint32_t* bm_row = p.bitmask ? p.bitmask + stat_row * p.words : nullptr;
 
     for (int t = 0; t < T; ++t) {
       const int j = j0 - t;
@@ -214,7 +246,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tmem_wait_ld();
       if (t == 0) {
         // first visited tile: causal diagonal and / or the ragged end of the key range
-        const int lim = p.causal ? rl : (p.N - 1 - j * 128);
+        const int lim = (p.causal && !kDecode) ? rl : (p.N - 1 - j * 128);
         const uint32_t ninf = 0xff800000u;
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
@@ -240,7 +272,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
           if (any) *(volatile int*)&flag[t % 3] = 1;
-          if (warp == 2) *(volatile int*)&flag[(t + 1) % 3] = 0;
+          if (warp == (kDecode ? 4 : 2)) *(volatile int*)&flag[(t + 1) % 3] = 0;
           tc_fence_before();
           mbar_arrive(&vote_bar[t & 1]);
         }
@@ -251,12 +283,13 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       if (!retain) continue;   // m, l, O unchanged; no exp, no P, no V load, no PV
       if (stat_thread && bm_row) {
-        if ((j >> 5) != bm_word) {
+        const int bit = kDecode ? (T - 1 - t) : j;   // decode: tile index inside the split
+        if ((bit >> 5) != bm_word) {
           if (bm_word >= 0) bm_row[bm_word] = bm_bits;
-          bm_word = j >> 5;
+          bm_word = bit >> 5;
           bm_bits = 0;
         }
-        bm_bits |= 1u << (j & 31);
+        bm_bits |= 1u << (bit & 31);
       }
       // running maximum with lazy rescaling: the reference m_ref only moves when the row maximum
       // grew by more than 2^8, so P stays <= 256 and O is rarely touched
@@ -311,6 +344,45 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ++r;
     }
 
+    if (kDecode) {
+      if (ok && T > 0) {
+        ok = mbar_wait(&o_done, (r - 1) & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (ok) {
+        // partial output of this split: O / l in fp32 and its log-normalizer (empty split: 0, -inf)
+        tc_fence_after();
+        const float inv = T > 0 ? 1.f / l : 0.f;
+        const size_t prow = ((size_t)b * p.Hq + h + rl) * p.num_splits + i;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          if (T > 0) {
+            tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColO + c * 32), o);
+            tmem_wait_ld();
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = 0u;
+          }
+          if (valid) {
+            float4* dst = reinterpret_cast<float4*>(p.o_part + prow * D + c * 32);
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+              dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
+                                   __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
+          }
+        }
+        if (valid) p.lse_part[prow] = T > 0 ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        if (stat_thread) {
+          if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
+          if (p.retained) p.retained[stat_row] = (uint32_t)r;
+          if (p.totals) {
+            atomicAdd(&p.totals[0], (unsigned long long)r);
+            atomicAdd(&p.totals[1], (unsigned long long)T);
+          }
+        }
+      }
+    } else {
     if (ok) {
       // finalize: O <- O / l, lse <- m + log l
       ok = mbar_wait(&o_done, (r - 1) & 1, status);
@@ -340,12 +412,13 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (valid) p.lse[((size_t)b * p.Hq + h) * p.N + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
       if (stat_thread) {
         if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
-        if (p.retained) p.retained[(size_t)(b * p.Hq + h) * p.Tr + i] = (uint32_t)r;
+        if (p.retained) p.retained[stat_row] = (uint32_t)r;
         if (p.totals) {
           atomicAdd(&p.totals[0], (unsigned long long)r);
           atomicAdd(&p.totals[1], (unsigned long long)T);
         }
       }
+    }
     }
   }
 

@@ -1,0 +1,82 @@
+"""GPU parity of mala_decode (split-KV decode through the C ABI) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_32712_b200 import workloads as W
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mala():
+    from paper_2609_32712_b200 import mala as m
+    m.lib()
+    return m
+
+
+def _run_and_check(mala, oracle, w, tau, num_splits, units=None):
+    q, kc, vc = (w[x].cuda() for x in ("q", "kcache", "vcache"))
+    B, _, Hq, d = q.shape
+    Nk, Hkv = kc.shape[1], kc.shape[2]
+    G = Hq // Hkv
+    o, lse, st = mala.decode(q, kc, vc, w["scale"], tau, num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    _, Bk = mala.tile_shape(mala.OP_DECODE, d)
+    ref = oracle.decode(w["q"], w["kcache"], w["vcache"], w["scale"], tau, num_splits, Bk, units=units)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()                    # [B,Hkv,S,tps]
+    if units is None:
+        units = [(b, g) for b in range(B) for g in range(Hkv)]
+    o_c, lse_c = o.float().cpu().numpy()[:, 0], lse.cpu().numpy()
+    skipped = retained = flips = 0
+    for (b, g) in units:
+        for s in range(num_splits):
+            flips += parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s],
+                                       list(range(tps - 1, -1, -1)), tau, Nk, Bk)
+            assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
+        hs = slice(g * G, (g + 1) * G)
+        parity.check_output(o_c[b, hs], ref["o"][b, hs])
+        assert np.abs(lse_c[b, hs] - ref["lse"][b, hs]).max() <= parity.LSE_ABS
+        skipped += int((ref["mask"][b, g] == 1).sum())
+        retained += int((ref["mask"][b, g] == 2).sum())
+    return dict(skipped=skipped, retained=retained, flips=flips, totals=st.totals.cpu().numpy())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv", [(128, 1, 4, 1), (1024, 4, 8, 2), (1000, 3, 4, 4), (4096, 8, 16, 2),
+                                          (700, 8, 2, 1)])
+def test_decode_literal(mala, oracle, Nk, S, Hq, Hkv, tau):
+    w = W.custom_decode(2, Hq, Hkv, Nk, 128, S, seed=Nk + S)
+    _run_and_check(mala, oracle, w, tau, S)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("Nk,S", [(8192, 8), (8192, 2), (5000, 4)])
+def test_decode_gated_keys_skip_value_tiles(mala, oracle, Nk, S, tau):
+    w = W.custom_decode(2, 8, 2, Nk, 128, S, group_types=["diffuse", "peaked"], seed=3, preset="D")
+    res = _run_and_check(mala, oracle, w, tau, S)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+    assert res["totals"][1] == res["retained"] + res["skipped"]
+
+
+def test_decode_tau_zero_is_split_invariant(mala):
+    w = W.custom_decode(1, 8, 2, 4096, 128, 4, seed=11)
+    q, kc, vc = (w[x].cuda() for x in ("q", "kcache", "vcache"))
+    o1, l1, _ = mala.decode(q, kc, vc, w["scale"], 0.0, 1)
+    o2, l2, _ = mala.decode(q, kc, vc, w["scale"], 0.0, 16)
+    assert (o1.float() - o2.float()).abs().max() <= 1e-2
+    assert (l1 - l2).abs().max() <= 1e-4
+
+
+def test_decode_strided_cache_view(mala, oracle):
+    # caches stored [B, Hkv, Nk, d] and passed as a permuted view
+    w = W.custom_decode(1, 4, 2, 1024, 128, 4, seed=13)
+    q = w["q"].cuda()
+    kc = w["kcache"].cuda().permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    vc = w["vcache"].cuda().permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    o, lse, _ = mala.decode(q, kc, vc, w["scale"], 0.0, 4)
+    ref = oracle.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 0.0, 4, 128)
+    parity.check_output(o.float().cpu().numpy()[:, 0], ref["o"])
