@@ -1,0 +1,442 @@
+#!/usr/bin/env python
+"""Benchmark of the MALA attention hot path on B200 (one process per GPU).
+
+A step is one pass of the whole path -- mala_fwd then mala_bwd at tolerance tau -- over one batch of
+seeded synthetic input of the benchmark definition's 32K configuration (cfg3; --workload selects
+another).  `value` is dense-equivalent TFLOP/s of fwd+bwd (FullAttn FLOP model: 4*B*Hq*N^2*d/2 forward,
+2.5x that backward) with inputs resident in HBM; `e2e` is the same metric with pinned-host inputs copied
+in and results copied out every step.  The line also carries, under `detail`, fwd / bwd latency of the
+MALA and dense kernels on cfg3 / cfg4 (literal and paper-regime "R" inputs), decode latency on cfg5
+(literal and gated "D" inputs) and the skipped-tile fractions.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+TILE = 128
+
+
+def fwd_dense_equiv_flops(B, Hq, N, d):
+    return 4.0 * B * Hq * N * N * d / 2.0
+
+
+def bwd_dense_equiv_flops(B, Hq, N, d):
+    return 2.5 * fwd_dense_equiv_flops(B, Hq, N, d)
+
+
+def fwd_executed_flops(legal, retained, d):
+    return (legal + retained) * 2.0 * TILE * TILE * d
+
+
+def bwd_executed_flops(legal, retained, d):
+    return (legal + 4.0 * retained) * 2.0 * TILE * TILE * d
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while a region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        busy = [x for x in sm if x > 0.5 * max(sm)] if sm else []
+        return dict(sm_mhz=statistics.median(busy) if busy else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def max_over_ranks(value: float, device) -> float:
+    """Maximum of a per-rank scalar over all ranks of the default process group (identity if none)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_rank_step: float, world: int, ms_per_step: float) -> float:
+    """Aggregate TFLOP/s of `world` replicas that each process flops_per_rank_step in ms_per_step (max over ranks)."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
+def time_cuda(fn, warmup, iters):
+    """Average milliseconds per call of fn(), CUDA events on the current stream."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+class PrefillCase:
+    """Device-resident inputs, outputs and scratch of one prefill configuration."""
+
+    def __init__(self, name, preset, device, seed_offset=0):
+        import torch
+        from paper_2609_32712_b200 import mala, workloads as W
+        self.mala = mala
+        self.cfg = W.prefill_config(name)
+        self.preset = preset
+        w = W.make_prefill(self.cfg, preset=preset, device=device, seed=self.cfg.seed + seed_offset)
+        self.q, self.k, self.v, self.do = w["q"], w["k"], w["v"], w["do"]
+        self.scale = w["scale"]
+        c = self.cfg
+        self.o = torch.empty_like(self.q)
+        self.lse = torch.empty((c.B, c.Hq, c.N), dtype=torch.float32, device=device)
+        self.dq, self.dk, self.dv = torch.empty_like(self.q), torch.empty_like(self.k), torch.empty_like(self.v)
+        self.ws = torch.empty(mala.workspace_bytes(mala.OP_BWD, c.B, c.Hq, c.Hkv, c.N, c.d), dtype=torch.uint8,
+                              device=device)
+        self.fwd_de = fwd_dense_equiv_flops(c.B, c.Hq, c.N, c.d)
+        self.bwd_de = bwd_dense_equiv_flops(c.B, c.Hq, c.N, c.d)
+
+    def fwd(self, tau, stats=False):
+        return self.mala.fwd(self.q, self.k, self.v, self.scale, tau, out=self.o, lse=self.lse, stats=stats, ws=self.ws)
+
+    def bwd(self, tau, stats=False):
+        return self.mala.bwd(self.q, self.k, self.v, self.o, self.do, self.lse, self.scale, tau, ws=self.ws,
+                             dq=self.dq, dk=self.dk, dv=self.dv, stats=stats)
+
+    def step(self, tau):
+        self.fwd(tau)
+        self.bwd(tau)
+
+    def tile_stats(self, tau):
+        import torch
+        _, _, fs = self.fwd(tau, stats=True)
+        _, _, _, bs = self.bwd(tau, stats=True)
+        torch.cuda.synchronize()
+        f, b = fs.totals.cpu().tolist(), bs.totals.cpu().tolist()
+        return dict(fwd_retained=f[0], fwd_legal=f[1], bwd_retained=b[0], bwd_legal=b[1])
+
+    def input_bytes(self):
+        return sum(t.numel() * t.element_size() for t in (self.q, self.k, self.v, self.do))
+
+
+def oracle_sample(case, tau, o_gpu, lse_gpu):
+    """Times the fp64 oracle on a bounded sample of the case's tiles (forward: some query blocks,
+    backward: some key blocks).  Returns (dense-equivalent FLOPs of the sample, seconds, description)."""
+    from oracle import mala_oracle as orc
+    c = case.cfg
+    T = -(-c.N // TILE)
+    G = c.Hq // c.Hkv
+    nb = min(16, T)
+    fwd_blocks = sorted({max(0, T * (x + 1) // nb - 1) for x in range(nb)})
+    fwd_units = [(0, h, i) for h in sorted({0, c.Hq - 1}) for i in fwd_blocks]
+    bwd_blocks = sorted({min(T - 1, T // 2 + T * x // (2 * nb)) for x in range(nb)})
+    bwd_units = [(0, 0, j) for j in bwd_blocks]
+    tile_flops = 2.0 * TILE * TILE * c.d
+    flops = sum((i + 1) * 2 * tile_flops for (_, _, i) in fwd_units)
+    flops += sum(G * (T - j) * 5 * tile_flops for (_, _, j) in bwd_units)
+    t0 = time.perf_counter()
+    orc.fwd(case.q, case.k, case.v, case.scale, tau, TILE, TILE, units=fwd_units)
+    orc.bwd(case.q, case.k, case.v, o_gpu, case.do, lse_gpu.cpu().numpy(), case.scale, tau, TILE, TILE,
+            key_units=bwd_units)
+    dt = time.perf_counter() - t0
+    what = (f"{c.name} {case.preset}: oracle fwd on {len(fwd_blocks)} query blocks (every T/{nb}-th) of heads 0 and "
+            f"{c.Hq - 1} + oracle bwd on {len(bwd_blocks)} key blocks of the upper half of KV head 0 "
+            f"({flops / 1e9:.1f} dense-equivalent GFLOP of fp64 work)")
+    return flops, dt, what
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample of the same workload per step."""
+    if rank != 0:
+        return
+    import torch
+    from oracle import mala_oracle as orc
+    from paper_2609_32712_b200 import workloads as W
+
+    class Host:
+        pass
+    cfg = W.prefill_config(args.workload)
+    w = W.make_prefill(cfg, preset=args.preset, device="cpu")
+    case = Host()
+    case.cfg, case.preset, case.scale = cfg, args.preset, w["scale"]
+    case.q, case.k, case.v, case.do = w["q"], w["k"], w["v"], w["do"]
+    T = -(-cfg.N // TILE)
+    # the sampled backward needs o and lse of the sampled rows only through D and lse; use the oracle's own forward
+    # on the rows that the sampled key block touches (the last T//64 query blocks)
+    units = [(0, h, i) for h in range(cfg.Hq // cfg.Hkv) for i in range(T // 2, T)]
+    f = orc.fwd(case.q, case.k, case.v, case.scale, args.tau, TILE, TILE, units=units)
+    o = torch.from_numpy(f["o"]).nan_to_num(0.0)
+    lse = torch.from_numpy(f["lse"]).nan_to_num(0.0)
+    times, flops = [], 0.0
+    what = ""
+    for s in range(args.warmup + args.steps):
+        fl, dt, what = oracle_sample(case, args.tau, o, lse)
+        if s >= args.warmup:
+            times.append(dt)
+            flops = fl
+    sec = sum(times) / len(times)
+    val = flops / sec / 1e12
+    print(json.dumps({
+        "impl": "reference", "metric": "mala_fwd_bwd_dense_equiv_tflops", "value": val, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload} {args.preset} tau={args.tau}", "sample": what},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": what},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="mala", choices=["mala", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--preset", default="literal", choices=["literal", "R"])
+    ap.add_argument("--tau", type=float, default=1e-4)
+    ap.add_argument("--detail-iters", type=int, default=10, help="timed iterations of each detail measurement")
+    ap.add_argument("--no-detail", action="store_true", help="skip the per-config detail table")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_32712_b200 import mala, workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    mala.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    warmup = max(args.warmup, 3)
+    peaks = load_peaks()
+
+    # ---------------------------------------------------------------- main timed region (inputs in HBM)
+    case = PrefillCase(args.workload, args.preset, dev, seed_offset=rank)
+    c = case.cfg
+    tau = args.tau
+    for _ in range(warmup):
+        case.step(tau)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * args.steps + 1)]
+    ev[0].record()
+    for s in range(args.steps):
+        case.fwd(tau)
+        ev[3 * s + 1].record()
+        case.bwd(tau)
+        ev[3 * s + 2].record()
+        ev[3 * s + 3].record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = ev[0].elapsed_time(ev[3 * args.steps])
+    fwd_ms = sum((ev[3 * s].elapsed_time(ev[3 * s + 1]) for s in range(args.steps))) / args.steps
+    bwd_ms = sum((ev[3 * s + 1].elapsed_time(ev[3 * s + 2]) for s in range(args.steps))) / args.steps
+    total_ms = max_over_ranks(total_ms, dev)
+    assert mala.device_status() == 0, "a device-side wait expired"
+    ms_per_step = total_ms / args.steps
+    step_flops = case.fwd_de + case.bwd_de
+    value = whole_job_value(step_flops, world, ms_per_step)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    ts = case.tile_stats(tau)
+    # roofline of the dominant kernel (the backward main kernel): executed tile FLOPs / launch duration
+    bwd_exec = bwd_executed_flops(ts["bwd_legal"], ts["bwd_retained"], c.d)
+    fwd_exec = fwd_executed_flops(ts["fwd_legal"], ts["fwd_retained"], c.d)
+    ach = bwd_exec / (bwd_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "mala_bwd_kernel", "achieved": ach, "peak": peaks["tflops_sustained"],
+                "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": None,
+                "peak_source": f"{peaks['source']} (bf16 matmul, sustained)",
+                "note": "duration = whole mala_bwd call (preprocess + main + dQ convert), so frac is a lower bound",
+                "fwd": {"kernel": "mala_fwd_kernel", "achieved": fwd_exec / (fwd_ms * 1e-3) / 1e12,
+                        "frac": fwd_exec / (fwd_ms * 1e-3) / 1e12 / peaks["tflops_sustained"]}}
+
+    # ---------------------------------------------------------------- end to end: host buffers, copies timed
+    host_in = [t.cpu().pin_memory() for t in (case.q, case.k, case.v, case.do)]
+    host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in (case.o, case.dq, case.dk, case.dv)]
+    dev_in = (case.q, case.k, case.v, case.do)
+    dev_out = (case.o, case.dq, case.dk, case.dv)
+
+    def e2e_step():
+        for d_, h_ in zip(dev_in, host_in):
+            d_.copy_(h_, non_blocking=True)
+        case.step(tau)
+        for h_, d_ in zip(host_out, dev_out):
+            h_.copy_(d_, non_blocking=True)
+
+    e2e_iters = max(1, min(args.steps, 5))
+    e2e_ms = time_cuda(e2e_step, 1, e2e_iters)
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+    e2e = {"value": step_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    del host_in, host_out
+
+    # ---------------------------------------------------------------- CPU baseline: the oracle on a bounded sample
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import mala_oracle as orc
+        case.fwd(tau)
+        torch.cuda.synchronize()
+        fl, dt, what = oracle_sample(case, tau, case.o.float().cpu(), case.lse)
+        cpu_baseline = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle",
+                        "sample": what, "seconds": dt}
+
+    # ---------------------------------------------------------------- detail: MALA vs dense, per config
+    detail = {}
+    if world == 1 and not args.no_detail:
+        it = args.detail_iters
+        for name in ("cfg3", "cfg4"):
+            for preset in ("literal", "R"):
+                cs = case if (name == args.workload and preset == args.preset) else PrefillCase(name, preset, dev)
+                cc = cs.cfg
+                row = {}
+                for label, t_ in (("mala", tau), ("dense", 0.0)):
+                    f_ms = time_cuda(lambda: cs.fwd(t_), 3, it)
+                    b_ms = time_cuda(lambda: cs.bwd(t_), 3, it)
+                    row[label] = {"fwd_ms": f_ms, "bwd_ms": b_ms,
+                                  "fwd_dense_equiv_tflops": cs.fwd_de / f_ms / 1e9,
+                                  "bwd_dense_equiv_tflops": cs.bwd_de / b_ms / 1e9}
+                st = cs.tile_stats(tau)
+                row["fwd_retained_frac"] = st["fwd_retained"] / st["fwd_legal"]
+                row["bwd_retained_frac"] = st["bwd_retained"] / st["bwd_legal"]
+                row["fwd_slots_per_query"] = st["fwd_retained"] * TILE * TILE / (cc.B * cc.Hq * cc.N)
+                row["bwd_slots_per_query"] = st["bwd_retained"] * TILE * TILE / (cc.B * cc.Hq * cc.N)
+                row["fwd_tensor_frac_on_executed"] = (fwd_executed_flops(st["fwd_legal"], st["fwd_retained"], cc.d)
+                                                      / (row["mala"]["fwd_ms"] * 1e-3) / 1e12 / peaks["tflops_sustained"])
+                row["bwd_tensor_frac_on_executed"] = (bwd_executed_flops(st["bwd_legal"], st["bwd_retained"], cc.d)
+                                                      / (row["mala"]["bwd_ms"] * 1e-3) / 1e12 / peaks["tflops_sustained"])
+                row["speedup_fwd"] = row["dense"]["fwd_ms"] / row["mala"]["fwd_ms"]
+                row["speedup_bwd"] = row["dense"]["bwd_ms"] / row["mala"]["bwd_ms"]
+                detail[f"{name}_{preset}"] = row
+                if cs is not case:
+                    del cs
+                    torch.cuda.empty_cache()
+        # decode (cfg5): HBM roofline = bytes that must be read (K always, V of retained tiles) / time
+        dcfg = W.decode_config("cfg5")
+        for preset in ("literal", "D"):
+            wd = W.make_decode(dcfg, preset=preset, device=dev)
+            qd, kc, vc = wd["q"], wd["kcache"], wd["vcache"]
+            wsd = torch.empty(mala.workspace_bytes(mala.OP_DECODE, dcfg.B, dcfg.Hq, dcfg.Hkv, dcfg.Nk, dcfg.d,
+                                                   dcfg.num_splits), dtype=torch.uint8, device=dev)
+            od = torch.empty_like(qd)
+            row = {}
+            for label, t_ in (("mala", tau), ("dense", 0.0)):
+                us = 1e3 * time_cuda(lambda: mala.decode(qd, kc, vc, wd["scale"], t_, dcfg.num_splits, ws=wsd, out=od,
+                                                          want_lse=False), 25, 100)
+                _, _, st = mala.decode(qd, kc, vc, wd["scale"], t_, dcfg.num_splits, ws=wsd, out=od, stats=True)
+                torch.cuda.synchronize()
+                ret, leg = st.totals.cpu().tolist()
+                need = (leg + ret) * TILE * dcfg.d * 2          # K tiles always, V tiles if retained
+                row[label] = {"us": us, "retained_frac": ret / leg, "needed_gb": need / 1e9,
+                              "achieved_gbs": need / (us * 1e-6) / 1e9,
+                              "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+            row["speedup"] = row["dense"]["us"] / row["mala"]["us"]
+            detail[f"cfg5_{preset}"] = row
+            del wd, qd, kc, vc, wsd
+            torch.cuda.empty_cache()
+
+    out = {
+        "metric": "mala_fwd_bwd_dense_equiv_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{c.name} {args.preset}: causal GQA B={c.B} Hq={c.Hq} Hkv={c.Hkv} N={c.N} d={c.d}, "
+                               f"tau={tau}, fwd+bwd per step",
+                   "l2": f"inputs {case.input_bytes() / 1e6:.0f} MB per step exceed the 126 MB L2 (no flush needed)",
+                   "parallelism": "replicas (one head slice per GPU, no collective)" if world > 1 else "single GPU"},
+        "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
+        "fwd_retained_frac": ts["fwd_retained"] / ts["fwd_legal"], "bwd_retained_frac": ts["bwd_retained"] / ts["bwd_legal"],
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * args.steps,
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "detail": detail,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
