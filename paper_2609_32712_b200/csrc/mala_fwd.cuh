@@ -346,7 +346,8 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
     if (kDecode) {
       if (ok && T > 0) {
-        ok = mbar_wait(&o_done, (r - 1) & 1, status);
+        // every PV has retired (o_done's parity alone cannot tell one pending PV from two)
+        ok = mbar_wait(&fin_bar, 0, status);
         ok = __all_sync(0xffffffffu, ok);
       }
       if (ok) {
@@ -384,8 +385,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
     } else {
     if (ok) {
-      // finalize: O <- O / l, lse <- m + log l
-      ok = mbar_wait(&o_done, (r - 1) & 1, status);
+      // finalize: O <- O / l, lse <- m + log l, once every PV has retired (the issuer commits fin_bar
+      // after its last MMA; o_done's parity alone cannot tell one pending PV from two)
+      ok = mbar_wait(&fin_bar, 0, status);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {

@@ -1,0 +1,133 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot run 32K / 128K attention in full, so forward query blocks, backward key blocks / dQ
+query blocks and decode (batch, KV head) units are sampled and computed one by one; properties that hold
+at any size (nesting, tau = 0 retains everything, omitted-mass bound from the two normalizers) are checked
+over the whole output."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_32712_b200 import workloads as W
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mala():
+    from paper_2609_32712_b200 import mala as m
+    m.lib()
+    return m
+
+
+def _prefill_sampled(mala, oracle, name, preset, tau, fwd_units, key_units, dq_units):
+    cfg = W.prefill_config(name)
+    w = W.make_prefill(cfg, preset=preset, device="cuda")
+    q, k, v, do = w["q"], w["k"], w["v"], w["do"]
+    B, N, Hq, d = q.shape
+    T = -(-N // 128)
+    o, lse, fst = mala.fwd(q, k, v, w["scale"], tau, stats=True)
+    dq, dk, dv, bst = mala.bwd(q, k, v, o, do, lse, w["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    fm = fst.mask(T)
+    bm = bst.mask(T)
+    # properties over the whole problem
+    assert (bm.transpose(2, 3) <= fm).all(), "backward support must be nested in forward support"
+    tri = torch.tril(torch.ones(T, T, dtype=torch.bool, device=fm.device))
+    assert not (fm & ~tri).any() and fm.diagonal(dim1=2, dim2=3).all()
+    if tau == 0.0:
+        assert (fm == tri).all() and (bm.transpose(2, 3) == tri).all()
+    else:
+        o_d, lse_d, _ = mala.fwd(q, k, v, w["scale"], 0.0)
+        eps = 1.0 - torch.exp(lse - lse_d)
+        assert eps.max() <= tau / (1 + tau) + 1e-3 and eps.min() >= -1e-3      # Proposition 1 (fp32 normalizers)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(dq.float()).all()
+    assert torch.isfinite(dk.float()).all() and torch.isfinite(dv.float()).all()
+
+    # sampled forward blocks
+    ref = oracle.fwd(q, k, v, w["scale"], tau, 128, 128, units=fwd_units)
+    fmc = fm.cpu().numpy()
+    for (b, h, i) in fwd_units:
+        rows = slice(i * 128, min(N, (i + 1) * 128))
+        parity.check_mask(fmc[b, h, i], ref["mask"][b, h, i], ref["crit"][b, h, i], list(range(i, -1, -1)), tau,
+                          i * 128 + 1)
+        parity.check_output(o[b, rows, h].float().cpu().numpy(), ref["o"][b, rows, h])
+        assert np.abs(lse[b, h, rows].cpu().numpy() - ref["lse"][b, h, rows]).max() <= parity.LSE_ABS
+    # sampled backward blocks, fed with the same o / lse the GPU backward saw
+    g = oracle.bwd(q, k, v, o, do, lse.cpu().numpy(), w["scale"], tau, 128, 128, key_units=key_units,
+                   dq_units=dq_units)
+    bmc = bm.cpu().numpy()
+    G = Hq // k.shape[2]
+    for (b, hk, j) in key_units:
+        rows = slice(j * 128, min(N, (j + 1) * 128))
+        parity.check_grad(dk[b, rows, hk].float().cpu().numpy(), g["dk"][b, rows, hk], f"dk block {j}")
+        parity.check_grad(dv[b, rows, hk].float().cpu().numpy(), g["dv"][b, rows, hk], f"dv block {j}")
+        for h in range(hk * G, (hk + 1) * G):
+            om, oc = g["mask"][b, h, j], g["crit"][b, h, j]
+            for i in range(T):
+                if bool(bmc[b, h, j, i]) != (om[i] == 2):
+                    assert om[i] != 0 and abs(oc[i]) <= parity.MASK_BAND, (h, j, i, oc[i])
+    for (b, h, i) in dq_units:
+        rows = slice(i * 128, min(N, (i + 1) * 128))
+        parity.check_grad(dq[b, rows, h].float().cpu().numpy(), g["dq"][b, rows, h], f"dq block {i}")
+    return float(fm.sum()) / float(tri.sum() * B * Hq)
+
+
+@pytest.mark.parametrize("preset", ["literal", "R"])
+@pytest.mark.parametrize("tau", [0.0, 1e-5, 1e-4, 1e-3])
+def test_cfg2_8k(mala, oracle, preset, tau):
+    T = 64
+    fwd_units = [(0, 0, 0), (0, 3, 17), (0, 9, T - 1), (0, 15, 40)]
+    key_units = [(0, 0, T - 1), (0, 2, 50), (0, 3, 30)]
+    dq_units = [(0, 1, 5), (0, 12, T - 1)]
+    frac = _prefill_sampled(mala, oracle, "cfg2", preset, tau, fwd_units, key_units, dq_units)
+    if preset == "R" and tau > 0:
+        assert frac < 0.8
+
+
+@pytest.mark.parametrize("preset,tau", [("literal", 1e-4), ("R", 1e-4), ("literal", 0.0)])
+def test_cfg3_32k(mala, oracle, preset, tau):
+    T = 256
+    fwd_units = [(0, 0, T - 1), (0, 1, 100), (0, 2, 200), (0, 31, 7)]
+    key_units = [(0, 0, T - 2), (0, 5, 200)]
+    dq_units = [(0, 6, 130)]
+    _prefill_sampled(mala, oracle, "cfg3", preset, tau, fwd_units, key_units, dq_units)
+
+
+@pytest.mark.parametrize("preset,tau", [("R", 1e-4), ("literal", 0.0)])
+def test_cfg4_128k(mala, oracle, preset, tau):
+    T = 1024
+    fwd_units = [(0, 1, T - 1), (0, 2, 300), (0, 4, 3)]
+    key_units = [(0, 1, T - 3), (0, 0, 900)]
+    dq_units = [(0, 7, 257)]
+    _prefill_sampled(mala, oracle, "cfg4", preset, tau, fwd_units, key_units, dq_units)
+
+
+@pytest.mark.parametrize("preset,tau", [("literal", 0.0), ("literal", 1e-4), ("D", 1e-4)])
+def test_cfg5_decode_128k(mala, oracle, preset, tau):
+    cfg = W.decode_config("cfg5")
+    w = W.make_decode(cfg, preset=preset, device="cuda")
+    q, kc, vc = w["q"], w["kcache"], w["vcache"]
+    o, lse, st = mala.decode(q, kc, vc, w["scale"], tau, cfg.num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert torch.isfinite(o.float()).all()
+    units = [(0, 0), (3, 1), (5, 2), (7, 7)]
+    ref = oracle.decode(q, kc, vc, w["scale"], tau, cfg.num_splits, 128, units=units)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    G = cfg.Hq // cfg.Hkv
+    for (b, g) in units:
+        for s in range(cfg.num_splits):
+            parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                              tau, cfg.Nk)
+        hs = slice(g * G, (g + 1) * G)
+        parity.check_output(o[b, 0, hs].float().cpu().numpy(), ref["o"][b, hs])
+        assert np.abs(lse[b, hs].cpu().numpy() - ref["lse"][b, hs]).max() <= parity.LSE_ABS
+    if preset == "D":
+        tot = st.totals.cpu().numpy()
+        assert tot[0] < tot[1]
+    if tau == 0.0:
+        assert gm.all()
