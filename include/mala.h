@@ -45,6 +45,10 @@ extern "C" {
 #define MALA_ERR_CUDA (-6)               /* a CUDA runtime call or launch failed */
 #define MALA_ERR_TENSOR_MAP (-7)         /* the driver rejected a TMA tensor map */
 #define MALA_ERR_DEVICE_TIMEOUT (-8)     /* a bounded device-side wait expired (status word) */
+#define MALA_ERR_STATIC_SCRATCH_EXCEEDED (-9) /* mala_decode_static: problem exceeds the built-in scratch */
+
+/* Size of the scratch array compiled into the library for mala_decode_static (24 MiB per device). */
+#define MALA_STATIC_SCRATCH_BYTES (24u << 20)
 
 #define MALA_OP_FWD 0
 #define MALA_OP_BWD 1
@@ -89,6 +93,34 @@ int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, cons
 int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
                 int B, int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws,
                 size_t ws_bytes, void* cuda_stream);
+
+/* Decode for callers that cannot allocate device memory.  (The paper has no counterpart: this entry point
+ * exists for integration reasons only and computes exactly what mala_decode computes.)
+ *
+ * Some callers of this library have no way to obtain scratch memory at the point of the call: code
+ * that runs inside a serving engine's pre-sized memory plan where every byte of the device pool is
+ * already assigned, a plug-in that receives only its input and output buffers from the host framework,
+ * or a latency-critical path that must not touch an allocator (cudaMalloc synchronises the device and
+ * may fail under fragmentation).  For them this variant keeps the split partials -- the only scratch
+ * the decode path needs -- in an array that is part of the library image: MALA_STATIC_SCRATCH_BYTES of
+ * global memory on every GPU that loads the library, held until the process exits.  The caller still
+ * passes all inputs and outputs; the call itself allocates nothing and frees nothing.
+ *
+ * Limits and rules
+ *   - mala_workspace_bytes(MALA_OP_DECODE, ...) for the same arguments must not exceed
+ *     MALA_STATIC_SCRATCH_BYTES; otherwise nothing is launched and
+ *     MALA_ERR_STATIC_SCRATCH_EXCEEDED is returned (use fewer splits, or mala_decode with your own ws).
+ *   - All calls on one device share the one array.  Two calls whose kernels can overlap on the GPU
+ *     (different streams, or different host threads on different streams) race on it and give wrong
+ *     results: keep calls on a device in one stream, or order them with events.  The array keeps the
+ *     previous call's contents between calls; the kernels overwrite every entry they later read, so no
+ *     clearing is needed.
+ *   - The first call on each device looks up the array's device address (a one-time
+ *     cudaGetSymbolAddress with that device current).  Make that first call outside any stream capture.
+ *   - No telemetry (mala_stats) is available through this entry point.
+ * Arguments, layouts, result and error codes otherwise as mala_decode. */
+int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, int B, int Hq,
+                       int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* cuda_stream);
 
 /* Scratch bytes needed by one call of `op` (MALA_OP_*); N is Nk for decode; num_splits is ignored
  * for fwd / bwd.  Returns 0 for unsupported arguments. */

@@ -19,6 +19,24 @@ static std::mutex g_mu;
 static int* g_status_ptr[64];
 static bool g_attr_done[64];
 
+// Built-in scratch of mala_decode_static: the split partials of one decode call.  Every device that
+// loads the library holds these bytes until the process exits.  In host code the array's name is only
+// a stand-in for the symbol, not a device address, so its address is looked up per device below.
+static __device__ __align__(256) unsigned char g_decode_scratch[MALA_STATIC_SCRATCH_BYTES];
+static unsigned char* g_decode_scratch_ptr[64];
+
+// Device address of the built-in scratch on device `dev` (which must be current); looked up once.
+static int static_scratch_address(int dev, unsigned char** out) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  if (!g_decode_scratch_ptr[dev]) {
+    unsigned char* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_decode_scratch) != cudaSuccess || !ptr) return MALA_ERR_CUDA;
+    g_decode_scratch_ptr[dev] = ptr;
+  }
+  *out = g_decode_scratch_ptr[dev];
+  return MALA_OK;
+}
+
 static int current_device_checked(int* dev_out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return MALA_ERR_CUDA;
@@ -115,6 +133,7 @@ const char* mala_strerror(int code) {
     case MALA_ERR_CUDA: return "CUDA runtime error";
     case MALA_ERR_TENSOR_MAP: return "TMA tensor map rejected";
     case MALA_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+    case MALA_ERR_STATIC_SCRATCH_EXCEEDED: return "problem needs more than the library's built-in scratch";
     default: return "unknown error";
   }
 }
@@ -235,6 +254,31 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
   MALA_TRY(device_setup(dev, &status));
   return decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
                        (cudaStream_t)cuda_stream);
+}
+
+int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, int B, int Hq,
+                       int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* cuda_stream) {
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  if (num_splits <= 0) return MALA_ERR_INVALID_ARG;
+  if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
+  MALA_TRY(check_view(kcache.p, kcache.sb, kcache.sn, kcache.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(vcache.p, vcache.sb, vcache.sn, vcache.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
+  if (decode_workspace_bytes(B, Hq, d, num_splits) > (size_t)MALA_STATIC_SCRATCH_BYTES)
+    return MALA_ERR_STATIC_SCRATCH_EXCEEDED;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  unsigned char* scratch = nullptr;
+  MALA_TRY(static_scratch_address(dev, &scratch));
+  float* o_part = (float*)scratch;
+  float* lse_part = (float*)(scratch + decode_align256((size_t)B * Hq * num_splits * d * sizeof(float)));
+  // every (batch, head, split) entry of both arrays is written by the split kernel (empty splits
+  // included) before the merge reads it, so nothing left over from an earlier call is ever read
+  return decode_launch_with_scratch(q, kcache, vcache, o, lse_opt, nullptr, B, Hq, Hkv, Nk, d, scale, tau, num_splits,
+                                    o_part, lse_part, status, (cudaStream_t)cuda_stream);
 }
 
 }  // extern "C"

@@ -50,6 +50,8 @@ def lib():
         L.mala_bwd.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, _TOut, _TOut, _TOut, ctypes.POINTER(_Stats),
                                i, i, i, i, i, i, f, f, vp, sz, vp]
         L.mala_decode.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp, sz, vp]
+        L.mala_decode_static.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, i, i, i, i, i, f, f, i, vp]
+        L.mala_decode_static.restype = i
         L.mala_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
         L.mala_workspace_bytes.restype = sz
         L.mala_tile_shape.argtypes = [i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
@@ -166,3 +168,27 @@ def decode(q, kcache, vcache, scale: float, tau: float, num_splits: int, stats: 
     if rc != 0:
         raise MalaError(rc, "mala_decode")
     return o, lse, st
+
+
+STATIC_SCRATCH_BYTES = 24 << 20
+
+
+def decode_static(q, kcache, vcache, scale: float, tau: float, num_splits: int, out=None, want_lse: bool = True):
+    """mala_decode_static: decode without any caller-provided scratch.
+
+    For callers that cannot allocate device memory at the point of the call (a fixed memory plan, a plug-in
+    that only receives its inputs and outputs, a path that must not touch the allocator).  The split partials
+    live in a 24 MiB array inside the library image; calls on one device must not overlap on the GPU.  Only
+    the output tensors are created here when the caller does not pass them.
+    Returns (o [B,1,Hq,d] bf16, lse [B,Hq] fp32 or None)."""
+    B, one, Hq, d = q.shape
+    assert one == 1
+    Nk, Hkv = kcache.shape[1], kcache.shape[2]
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    rc = lib().mala_decode_static(_view(q, _TIn), _view(kcache, _TIn), _view(vcache, _TIn), _view(o, _TOut),
+                                  lse.data_ptr() if lse is not None else None, B, Hq, Hkv, Nk, d, scale, tau,
+                                  num_splits, _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_decode_static")
+    return o, lse
