@@ -8,14 +8,14 @@
 //                           lse (Eq. 4).  Only retained tiles load dO and run dP^T = V dO^T, P^T,
 //                           dS^T = P^T o (dP^T - D), dV += P^T dO, dK += dS^T Q, dQ_i += dS K_j.
 //                           dK, dV accumulate in TMEM; dQ tiles are added to an fp32 accumulator in
-//                           global memory with vector reductions.
+//                           global memory by TMA reduce-add from shared memory.
 //   bwd_convert_dq_kernel : dq = bf16(scale * accumulator).
 //
-// Warp roles of the main kernel (320 threads):
+// Warp roles of the main kernel (448 threads):
 //   warp 0     TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
 //   warp 1     UMMA issuer (and, in the MALA kernel, the on-demand dO loads)
-//   warps 2-5  compute group, one thread per key row of the transposed tile
-//   warps 6-9  dQ group, one thread per query row of the dQ tile
+//   warps 2-9  compute group, two threads per key row of the transposed tile (64 query columns each)
+//   warps 10-13 dQ group, one thread per query row of the dQ tile
 #pragma once
 #include <cuda_runtime.h>
 
@@ -48,7 +48,7 @@ struct BwdCfg {
   // K, V, Q x2, dO x2.  dS^T (32 KB) of a retained tile overwrites that tile's dO stage once dP and dV
   // have consumed it (D = 128); for D = 64 a dO stage is too small, so two separate dS stages follow.
   static constexpr int kSmemBytes = 6 * kTileBytes + (D == 128 ? 0 : 2 * kDsBytes) + 1024;
-  static constexpr int kThreads = 320;
+  static constexpr int kThreads = 448;
   static constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
 };
 
@@ -57,10 +57,10 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 }
 
 template <int D, bool kDense>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(448, 1)
 mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
-                const BwdParams p) {
+                const __grid_constant__ CUtensorMap tmAcc, const BwdParams p) {
   using Cfg = BwdCfg<D>;
   constexpr int PAN = Cfg::kPanels;
   extern __shared__ uint8_t smem_raw[];
@@ -73,7 +73,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
 
   __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
-      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar;
+      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free;
   __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[3];
@@ -94,11 +94,12 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int s = 0; s < 2; ++s) {
       mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1);
       mbar_init(&do_full[s], 1); mbar_init(&do_empty[s], 1);
-      mbar_init(&vote_bar[s], 4);
+      mbar_init(&vote_bar[s], 8);
     }
-    mbar_init(&s_full, 1); mbar_init(&p_full, 4); mbar_init(&dp_full, 1); mbar_init(&ds_full, 4);
-    mbar_init(&dv_done, 1); mbar_init(&grp_bar, 4); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
+    mbar_init(&s_full, 1); mbar_init(&p_full, 8); mbar_init(&dp_full, 1); mbar_init(&ds_full, 8);
+    mbar_init(&dv_done, 1); mbar_init(&grp_bar, 8); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
     mbar_init(&fin_bar, 1);
+    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1);
     flag[0] = flag[1] = flag[2] = 0;
     dq_info = -1;
     mbar_fence_init();
@@ -223,7 +224,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                    make_smem_desc(aQ + s * Cfg::kTileBytes + k * 2048, 16384, 1024), idesc_dv,
                    (r > 0 || k > 0) ? 1u : 0u);
           }
-          tc_commit(&q_empty[s]);
+          // (the Q stage is released by the dQ group, which stages the dQ tile in it after these MMAs)
 #pragma unroll
           for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j  (into the dP columns)
             mma_ss(tmem_addr(tb, 0, Cfg::kColDP), make_smem_desc(aDS + ds * Cfg::kDsBytes + k * 2048, 16384, 1024),
@@ -247,10 +248,13 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int u = (r > 1 ? r - 1 : 0); u <= r; ++u) mbar_wait(&do_full[u & 1], (u >> 1) & 1, status);
       }
     }
-  } else if (warp < 6) {
-    // ------------------------------------------------------------------ compute group: thread = key row
+  } else if (warp < 10) {
+    // ------------------------------------------------------------------ compute group
+    // Two threads per key row: warps 2-5 own query columns 0..63 of the transposed tile, warps 6-9
+    // columns 64..127 (both warps of a pair reach the same TMEM lane quadrant).
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
+    const int hf = (warp - 2) >> 2;                 // column half
     const bool valid_key = (j * 128 + rl) < p.N;
     const float c2 = p.scale_log2;
     const bool stat_thread = (warp == 2 && lane == 0);
@@ -264,8 +268,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
       return ((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128 + rl;
     };
-    // per-query vectors of tile 0 into slot 0, made visible by a first pass through vote_bar[1]
-    {
+    // per-query vectors of tile 0 into slot 0 (published by the first column half), then a group sync
+    if (hf == 0) {
       const size_t x = vec_index(0);
       vec[0][0][rl] = p.lse2[x];
       vec[0][1][rl] = p.bq[x];
@@ -281,7 +285,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int slot = n % 3;
       // prefetch the per-query vectors of the next tile
       float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
-      if (n + 1 < n_tot) {
+      if (hf == 0 && n + 1 < n_tot) {
         const size_t x = vec_index(n + 1);
         nx0 = p.lse2[x]; nx1 = p.bq[x]; nx2 = p.Dq[x];
       }
@@ -289,24 +293,21 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s0[32], s1[32], s2[32], s3[32];
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 0), s0);
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 32), s1);
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 64), s2);
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + 96), s3);
+      uint32_t s0[32], s1[32];
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 0), s0);
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 32), s1);
       tmem_wait_ld();
-      if (p.causal && i == j) {   // diagonal tile: entry (key rl, query e) is legal iff rl <= e
+      if (p.causal && i == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
         const uint32_t ninf = 0xff800000u;
+        const int c0 = hf * 64;
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-          if (e < rl) s0[e] = ninf;
-          if (e + 32 < rl) s1[e] = ninf;
-          if (e + 64 < rl) s2[e] = ninf;
-          if (e + 96 < rl) s3[e] = ninf;
+          if (c0 + e < rl) s0[e] = ninf;
+          if (c0 + e + 32 < rl) s1[e] = ninf;
         }
       }
       // publish the next tile's vectors (slot (n+1) % 3 was last read two tiles ago)
-      {
+      if (hf == 0) {
         const int ns = (n + 1) % 3;
         vec[ns][0][rl] = nx0; vec[ns][1][rl] = nx1; vec[ns][2][rl] = nx2;
       }
@@ -316,18 +317,14 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         bool vote = false;
         if (!kDense) {
           float crit = -INFINITY;
-          const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]);
+          const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]) + hf * 16;
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            const float4 x0 = bb[e], x1 = bb[8 + e], x2 = bb[16 + e], x3 = bb[24 + e];
+            const float4 x0 = bb[e], x1 = bb[8 + e];
             crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s0[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(s0[4 * e + 1]), c2, -x0.y)),
                                      fmaxf(fmaf(__uint_as_float(s0[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(s0[4 * e + 3]), c2, -x0.w))));
             crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s1[4 * e + 0]), c2, -x1.x), fmaf(__uint_as_float(s1[4 * e + 1]), c2, -x1.y)),
                                      fmaxf(fmaf(__uint_as_float(s1[4 * e + 2]), c2, -x1.z), fmaf(__uint_as_float(s1[4 * e + 3]), c2, -x1.w))));
-            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s2[4 * e + 0]), c2, -x2.x), fmaf(__uint_as_float(s2[4 * e + 1]), c2, -x2.y)),
-                                     fmaxf(fmaf(__uint_as_float(s2[4 * e + 2]), c2, -x2.z), fmaf(__uint_as_float(s2[4 * e + 3]), c2, -x2.w))));
-            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s3[4 * e + 0]), c2, -x3.x), fmaf(__uint_as_float(s3[4 * e + 1]), c2, -x3.y)),
-                                     fmaxf(fmaf(__uint_as_float(s3[4 * e + 2]), c2, -x3.z), fmaf(__uint_as_float(s3[4 * e + 3]), c2, -x3.w))));
           }
           vote = valid_key && !(crit < 0.f);
         }
@@ -338,6 +335,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_before();
           mbar_arrive(&vote_bar[n & 1]);
         }
+        // this barrier also orders every thread's S^T loads before any thread's P^T stores below
         ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -358,8 +356,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
         // P^T = exp2(s * c2 - lse2_q) (bf16): kept packed in registers and written over S^T in TMEM
-        uint32_t pk[64];
-        const float4* ll = reinterpret_cast<const float4*>(vec[slot][0]);
+        uint32_t pk[32];
+        const float4* ll = reinterpret_cast<const float4*>(vec[slot][0]) + hf * 16;
 #define MALA_BWD_P(SRC, CH)                                                                  \
         {                                                                                    \
           _Pragma("unroll") for (int e = 0; e < 8; ++e) {                                    \
@@ -373,12 +371,10 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }                                                                                  \
           uint32_t tmp[16];                                                                  \
           _Pragma("unroll") for (int e = 0; e < 16; ++e) tmp[e] = pk[(CH) * 16 + e];         \
-          tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + (CH) * 16), tmp);                \
+          tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 32 + (CH) * 16), tmp);      \
         }
         MALA_BWD_P(s0, 0)
         MALA_BWD_P(s1, 1)
-        MALA_BWD_P(s2, 2)
-        MALA_BWD_P(s3, 3)
 #undef MALA_BWD_P
         tmem_wait_st();
         tc_fence_before();
@@ -391,11 +387,11 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const float4* dd = reinterpret_cast<const float4*>(vec[slot][2]);
+        const float4* dd = reinterpret_cast<const float4*>(vec[slot][2]) + hf * 16;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
           uint32_t dp[32];
-          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + c * 32), dp);
+          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + hf * 64 + c * 32), dp);
           tmem_wait_ld();
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
@@ -413,8 +409,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
               w[2 * u] = pack_bf16x2(d0, d1);
               w[2 * u + 1] = pack_bf16x2(d2, d3);
             }
-            const uint32_t col = (uint32_t)((c & 1) * 32 + v * 8);
-            *reinterpret_cast<uint4*>(sDS + (r & 1) * Cfg::kDsBytes + (c >> 1) * 16384 + sw128_offset((uint32_t)rl, col)) =
+            const uint32_t col = (uint32_t)(c * 32 + v * 8);
+            *reinterpret_cast<uint4*>(sDS + (r & 1) * Cfg::kDsBytes + hf * 16384 + sw128_offset((uint32_t)rl, col)) =
                 make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
@@ -435,7 +431,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
     }
 
-    // epilogue: dK_j (x scale), dV_j -> global
+    // epilogue: dK_j (x scale), dV_j -> global; each thread of a pair stores half of the columns of its row
     if (ok) {
       ok = mbar_wait(&fin_bar, 0, status);
       ok = __all_sync(0xffffffffu, ok);
@@ -451,7 +447,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const float f = which ? p.scale : 1.f;
         const uint32_t col0 = which ? Cfg::kColDK : Cfg::kColDV;
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int cc = 0; cc < D / 64; ++cc) {
+          const int c = hf * (D / 64) + cc;
           uint32_t o[32];
           if (r > 0) {
             tmem_ld_x32(tmem_addr(tb, lane_base, col0 + c * 32), o);
@@ -476,8 +473,15 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------------ dQ group: thread = query row
+    // Each retained tile's dQ (fp32, 128 x D) is staged in the tile's own Q stage -- free once dK and dQ
+    // have retired -- in 32-column swizzled panels and added to the global accumulator by TMA
+    // reduce-add; the Q stage is handed back to the producer when the TMA has read it.
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
+    const bool elected = (warp == 10 && lane == 0);
+    constexpr int kPanelsPerRound = (D == 128) ? 2 : 1;   // 16 KB panels that fit in one Q stage
+    uint32_t full_phase = 0, free_phase = 0;
+    if (elected) tma_prefetch_desc(&tmAcc);
     for (int k = 0;; ++k) {
       bool ok = mbar_wait(&dq_info_bar, k & 1, status);
       ok = __all_sync(0xffffffffu, ok);
@@ -489,32 +493,53 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
-      float* dst = p.dq_acc + (((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128 + rl) * D;
-      uint32_t a0[32], a1[32];
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 0), a0);
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 32), a1);
-      uint32_t a2[32], a3[32];
-      if (D == 128) {
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 64), a2);
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 96), a3);
-      }
-      tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused; the adds continue from registers
+      const int row0 = (int)(((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128);
+      uint8_t* stg = sQ + (n & 1) * Cfg::kTileBytes;
 #pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        red_add_v4(dst + v * 4, __uint_as_float(a0[4 * v]), __uint_as_float(a0[4 * v + 1]), __uint_as_float(a0[4 * v + 2]), __uint_as_float(a0[4 * v + 3]));
-        red_add_v4(dst + 32 + v * 4, __uint_as_float(a1[4 * v]), __uint_as_float(a1[4 * v + 1]), __uint_as_float(a1[4 * v + 2]), __uint_as_float(a1[4 * v + 3]));
-      }
-      if (D == 128) {
-#pragma unroll
-        for (int v = 0; v < 8; ++v) {
-          red_add_v4(dst + 64 + v * 4, __uint_as_float(a2[4 * v]), __uint_as_float(a2[4 * v + 1]), __uint_as_float(a2[4 * v + 2]), __uint_as_float(a2[4 * v + 3]));
-          red_add_v4(dst + 96 + v * 4, __uint_as_float(a3[4 * v]), __uint_as_float(a3[4 * v + 1]), __uint_as_float(a3[4 * v + 2]), __uint_as_float(a3[4 * v + 3]));
+      for (int round = 0; round < 2; ++round) {
+        if (round > 0) {   // the panels are still being read by the previous round's reduce
+          if (elected) { bulk_wait_read_all(); mbar_arrive(&stg_free); }
+          ok = mbar_wait(&stg_free, free_phase & 1, status);
+          ok = __all_sync(0xffffffffu, ok);
+          ++free_phase;
+          if (!ok) break;
         }
+#pragma unroll
+        for (int cc = 0; cc < kPanelsPerRound; ++cc) {
+          const int chunk = round * kPanelsPerRound + cc;
+          uint32_t a[32];
+          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + chunk * 32), a);
+          tmem_wait_ld();
+          if (round == 1 && cc == kPanelsPerRound - 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused by the next dP
+          }
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            *reinterpret_cast<uint4*>(stg + cc * 16384 + rl * 128 + ((v ^ (rl & 7)) << 4)) =
+                make_uint4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&stg_full);
+        if (elected) {
+          ok = mbar_wait(&stg_full, full_phase & 1, status);
+          if (ok) {
+#pragma unroll
+            for (int cc = 0; cc < kPanelsPerRound; ++cc)
+              tma_reduce_add_2d(&tmAcc, stg + cc * 16384, (round * kPanelsPerRound + cc) * 32, row0);
+            bulk_commit_group();
+          }
+        }
+        ++full_phase;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
       }
+      if (!ok) break;
+      if (elected) { bulk_wait_read_all(); mbar_arrive(&q_empty[n & 1]); }
     }
+    if (elected) bulk_wait_all();
   }
 
   tc_fence_before();
@@ -598,9 +623,9 @@ inline bool bwd_set_attributes() {
 
 template <int D, bool kDense>
 inline int bwd_launch_main(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
-                           const BwdParams& p, cudaStream_t stream) {
+                           const CUtensorMap& tacc, const BwdParams& p, cudaStream_t stream) {
   dim3 grid(p.T, p.Hkv, p.B);
-  mala_bwd_kernel<D, kDense><<<grid, BwdCfg<D>::kThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, p);
+  mala_bwd_kernel<D, kDense><<<grid, BwdCfg<D>::kThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, tacc, p);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
@@ -616,8 +641,9 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   float* bq = (float*)(w + vbytes);
   float* Dq = (float*)(w + 2 * vbytes);
 
-  CUtensorMap tq, tk, tv, tdo;
-  if (!make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
+  CUtensorMap tq, tk, tv, tdo, tacc;
+  if (!make_tensor_map_f32_rows(&tacc, acc, (uint64_t)B * Hq * Np, d, 128) ||
+      !make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
       !make_tensor_map_bnhd(&tk, k.p, B, N, Hkv, d, k.sb, k.sn, k.sh, 128) ||
       !make_tensor_map_bnhd(&tv, v.p, B, N, Hkv, d, v.sb, v.sn, v.sh, 128) ||
       !make_tensor_map_bnhd(&tdo, dout.p, B, N, Hq, d, dout.sb, dout.sn, dout.sh, 128))
@@ -650,8 +676,8 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   }
   const bool dense = (tau == 0.f);
   int rc;
-  if (d == 128) rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, p, stream);
-  else rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, p, stream);
+  if (d == 128) rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, tacc, p, stream);
+  else rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, tacc, p, stream);
   if (rc != MALA_OK) return rc;
   {
     const long long total = (long long)B * Hq * N * (d / 8);
