@@ -153,18 +153,27 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);    // S^T, dP^T
       constexpr uint32_t idesc_dv = make_idesc_bf16(128, D, false, true);      // dV (A in TMEM), dK
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);       // dQ
-      const uint32_t aK = smem_u32(sK), aV = smem_u32(sV), aQ = smem_u32(sQ), aDO = smem_u32(sDO), aDS = smem_u32(sDS);
+      // descriptors are built once; per MMA only the start-address field is advanced
+      const uint64_t dKk = make_smem_desc(smem_u32(sK), 16, 1024);        // K_j as K-major A (S^T)
+      const uint64_t dKm = make_smem_desc(smem_u32(sK), 16384, 1024);     // K_j as MN-major B (dQ)
+      const uint64_t dVk = make_smem_desc(smem_u32(sV), 16, 1024);        // V_j as K-major A (dP^T)
+      const uint64_t dQk0 = make_smem_desc(smem_u32(sQ), 16, 1024);       // Q stage 0 as K-major B (S^T)
+      const uint64_t dQm0 = make_smem_desc(smem_u32(sQ), 16384, 1024);    // Q stage 0 as MN-major B (dK)
+      const uint64_t dDOk0 = make_smem_desc(smem_u32(sDO), 16, 1024);     // dO stage 0 as K-major B (dP^T)
+      const uint64_t dDOm0 = make_smem_desc(smem_u32(sDO), 16384, 1024);  // dO stage 0 as MN-major B (dV)
+      const uint64_t dDSk0 = make_smem_desc(smem_u32(sDS), 16, 1024);     // dS^T stage 0 as K-major A (dK)
+      const uint64_t dDSm0 = make_smem_desc(smem_u32(sDS), 16384, 1024);  // dS^T stage 0 as MN-major A (dQ)
       bool ok = mbar_wait(&kv_full, 0, status);
       int r = 0;   // retained tiles so far
       auto issue_qk = [&](int n) -> bool {
         const int s = n & 1;
         if (!mbar_wait(&q_full[s], (n >> 1) & 1, status)) return false;
         tc_fence_after();
+        const uint64_t dQk = desc_advance(dQk0, s * Cfg::kTileBytes);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-          mma_ss(tmem_addr(tb, 0, Cfg::kColS), make_smem_desc(aK + off, 16, 1024),
-                 make_smem_desc(aQ + s * Cfg::kTileBytes + off, 16, 1024), idesc_s, k > 0);
+          mma_ss(tmem_addr(tb, 0, Cfg::kColS), desc_advance(dKk, off), desc_advance(dQk, off), idesc_s, k > 0);
         }
         tc_commit(&s_full);
         return true;
@@ -194,11 +203,13 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           ok = mbar_wait(&do_full[ds], (r >> 1) & 1, status);
           if (!ok) break;
           tc_fence_after();
+          const uint64_t dDOk = desc_advance(dDOk0, ds * Cfg::kTileBytes);
+          const uint64_t dDOm = desc_advance(dDOm0, ds * Cfg::kTileBytes);
+          const uint32_t acc0 = r > 0 ? 1u : 0u;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {   // dP^T = V dO^T
             const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), make_smem_desc(aV + off, 16, 1024),
-                   make_smem_desc(aDO + ds * Cfg::kTileBytes + off, 16, 1024), idesc_s, k > 0);
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dVk, off), desc_advance(dDOk, off), idesc_s, k > 0);
           }
           tc_commit(&dp_full);
           ok = mbar_wait(&p_full, r & 1, status);
@@ -206,9 +217,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < 8; ++k)   // dV += P^T dO
-            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + k * 8),
-                   make_smem_desc(aDO + ds * Cfg::kTileBytes + k * 2048, 16384, 1024), idesc_dv,
-                   (r > 0 || k > 0) ? 1u : 0u);
+            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + k * 8), desc_advance(dDOm, k * 2048),
+                   idesc_dv, k > 0 ? 1u : acc0);
           tc_commit(&dv_done);
         }
         // the score buffer is free again: recompute the next tile's scores while dS is being formed
@@ -217,18 +227,20 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           ok = mbar_wait(&ds_full, r & 1, status);
           if (!ok) break;
           tc_fence_after();
+          const uint64_t dDSk = desc_advance(dDSk0, ds * Cfg::kDsBytes), dDSm = desc_advance(dDSm0, ds * Cfg::kDsBytes);
+          const uint64_t dQm = desc_advance(dQm0, s * Cfg::kTileBytes);
+          const uint32_t acc1 = r > 0 ? 1u : 0u;
 #pragma unroll
           for (int k = 0; k < 8; ++k) {   // dK += dS^T Q
             const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tmem_addr(tb, 0, Cfg::kColDK), make_smem_desc(aDS + ds * Cfg::kDsBytes + off, 16, 1024),
-                   make_smem_desc(aQ + s * Cfg::kTileBytes + k * 2048, 16384, 1024), idesc_dv,
-                   (r > 0 || k > 0) ? 1u : 0u);
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDK), desc_advance(dDSk, off), desc_advance(dQm, k * 2048), idesc_dv,
+                   k > 0 ? 1u : acc1);
           }
           // (the Q stage is released by the dQ group, which stages the dQ tile in it after these MMAs)
 #pragma unroll
           for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j  (into the dP columns)
-            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), make_smem_desc(aDS + ds * Cfg::kDsBytes + k * 2048, 16384, 1024),
-                   make_smem_desc(aK + k * 2048, 16384, 1024), idesc_dq, k > 0);
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
+                   k > 0);
           tc_commit(&do_empty[ds]);   // dO stage (and the dS^T stored over it) is free once dK, dQ retire
           *(volatile int*)&dq_info = n;
           mbar_arrive(&dq_info_bar);

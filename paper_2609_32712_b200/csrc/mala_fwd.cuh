@@ -143,7 +143,10 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (lane == 0) {
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, false, true);
-      const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
+      // descriptors are built once; per MMA only the start-address field is advanced
+      const uint64_t dQ = make_smem_desc(smem_u32(sQ), 16, 1024);
+      const uint64_t dK0 = make_smem_desc(smem_u32(sK), 16, 1024);
+      const uint64_t dV0 = make_smem_desc(smem_u32(sV), 16384, 1024);
       bool ok = mbar_wait(&q_full, 0, status);
       int v_issued = 0;   // V tiles requested so far
       int r = 0;          // PV MMAs issued so far (retained tiles)
@@ -153,11 +156,11 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!mbar_wait(&k_full[s], (t / KS) & 1, status)) return false;
         tc_fence_after();
         const uint32_t dS = tmem_addr(tb, 0, (t & 1) ? Cfg::kColS1 : Cfg::kColS0);
+        const uint64_t dK = desc_advance(dK0, s * Cfg::kTileBytes);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-          mma_ss(dS, make_smem_desc(aQ + off, 16, 1024), make_smem_desc(aK + s * Cfg::kTileBytes + off, 16, 1024),
-                 idesc_qk, k > 0);
+          mma_ss(dS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0);
         }
         tc_commit(&k_empty[s]);
         tc_commit(&s_full[t & 1]);
@@ -195,10 +198,11 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_after();
           const uint32_t aP = tmem_addr(tb, 0, (t & 1) ? Cfg::kColS1 : Cfg::kColS0);
           const uint32_t dO = tmem_addr(tb, 0, Cfg::kColO);
+          const uint64_t dV = desc_advance(dV0, s * Cfg::kTileBytes);
+          const uint32_t acc0 = r > 0 ? 1u : 0u;
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            mma_ts(dO, aP + k * 8, make_smem_desc(aV + s * Cfg::kTileBytes + k * 2048, 16384, 1024), idesc_pv,
-                   (r > 0 || k > 0) ? 1u : 0u);
+            mma_ts(dO, aP + k * 8, desc_advance(dV, k * 2048), idesc_pv, k > 0 ? 1u : acc0);
           tc_commit(&v_empty[s]);
           tc_commit(&o_done);
           ++r;

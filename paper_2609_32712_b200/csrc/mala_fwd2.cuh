@@ -1,0 +1,397 @@
+// MALA forward (Algorithm 1) for sm_100a, prefill version: two query blocks per CTA.
+//
+// One CTA owns the two consecutive 128-row query blocks A = 2c and B = 2c+1 of one (batch, query
+// head).  They share the K tiles; each block has its own UMMA-issuing thread, softmax warpgroup,
+// score buffer, V stage and output accumulator (TMEM: S_A, S_B, O_A, O_B = 512 columns).  A thread
+// that issues tcgen05.mma stalls until the tensor pipe accepts the instruction, so the waits and
+// commits of one block's issuer run while the other block's MMAs execute, and one block's rows are in
+// the softmax path while the pipe works for the other block.
+// Each block keeps the semantics of Algorithm 1 on its own: its tiles are visited from ITS diagonal
+// toward earlier keys, the test for a tile uses the state left by that block's previous retained tile,
+// and a skipped tile issues no exp, no P, no V load and no PV.
+//
+// Warp roles (384 threads):
+//   warp 0       TMA producer: Q_A, Q_B once, K ring (a K stage is released when both issuers are done)
+//   warp 1, 2    UMMA issuers of block A and B: S_X = Q_X K^T for every tile, then (after the vote) the V
+//                load of that block and O_X += P_X V; the next QK of X follows its PV in program order, so
+//                the single score buffer of X is reused in tensor-pipe order without a barrier
+//   warps 4-7    softmax group of block A, warps 8-11 of block B (one thread per query row)
+// All synchronisation is by mbarriers with bounded waits.
+#pragma once
+#include "mala_fwd.cuh"
+
+namespace mala {
+
+template <int D, bool kDense>
+struct Fwd2Cfg {
+  static constexpr int kPanels = D / 64;
+  static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kKStages = 3;
+  // Q_A, Q_B, K ring, V_A, V_B
+  static constexpr int kSmemBytes = (2 + kKStages + 2) * kTileBytes + 1024;
+  static constexpr int kThreads = 384;
+  static constexpr uint32_t kTmemCols = 512;
+};
+
+template <int D, bool kDense>
+__global__ void __launch_bounds__(384, 1)
+mala_fwd2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const FwdParams p) {
+  using Cfg = Fwd2Cfg<D, kDense>;
+  constexpr int KS = Cfg::kKStages, PAN = Cfg::kPanels;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;                               // [2] blocks A, B
+  uint8_t* sK = sQ + 2 * Cfg::kTileBytes;
+  uint8_t* sV = sK + KS * Cfg::kTileBytes;          // [2] blocks A, B
+
+  __shared__ uint64_t q_full, k_full[KS], k_empty[KS], v_full[2], v_empty[2], s_full[2], vote_bar[2], p_full[2],
+      fin_bar, turn_bar[2];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int flag[2][3];
+  __shared__ int early_exit;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = p.Hq / p.Hkv;
+  const int b = blockIdx.z, h = blockIdx.y, hkv = h / G;
+  const int npairs = (p.Tr + 1) / 2;
+  const int c = npairs - 1 - (int)blockIdx.x;        // longest pairs first
+  const int iA = 2 * c, iB = 2 * c + 1;
+  const bool hasB = iB < p.Tr;
+  // key steps u = 0 .. U-1 visit key block j0 - u; block X takes part from step first[X] on
+  const int j0 = p.causal ? (hasB ? iB : iA) : (p.Tr - 1);
+  const int U = j0 + 1;
+  const int firstA = p.causal ? (j0 - iA) : 0;       // 1 when B exists (B's diagonal is not legal for A)
+  int* status = p.status;
+
+  if (tid == 0) {
+    early_exit = (*(volatile int*)status != 0);
+    mbar_init(&q_full, 1);
+    for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 2); }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&v_full[x], 1); mbar_init(&v_empty[x], kDense ? 2 : 1);
+      mbar_init(&s_full[x], 1); mbar_init(&vote_bar[x], 4); mbar_init(&p_full[x], 4);
+      flag[x][0] = flag[x][1] = flag[x][2] = 0;
+    }
+    mbar_init(&fin_bar, 2);
+    mbar_init(&turn_bar[0], 4); mbar_init(&turn_bar[1], 4);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (early_exit) return;
+  if (warp == 0) { tmem_alloc(&tmem_base_s, Cfg::kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tb = tmem_base_s;
+  if (warp < 4) {
+  // warps 0-3 (producer, issuers) need few registers; the two softmax warpgroups take the rest
+  reg_dealloc<72>();
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer: Q_A, Q_B, K ring
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+      mbar_arrive_expect_tx(&q_full, (hasB ? 2 : 1) * Cfg::kTileBytes);
+      for (int pn = 0; pn < PAN; ++pn) {
+        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, iA * 128, h, b);
+        if (hasB) tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, iB * 128, h, b);
+      }
+      int issued = 0, v_issued = 0, s = 0;
+      uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
+      bool ok = true;
+      for (int u = 0; u < U && ok; ++u) {
+        ok = mbar_wait(&k_empty[s], par, status);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
+        for (int pn = 0; pn < PAN; ++pn)
+          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, (j0 - u) * 128, hkv, b);
+        issued = u + 1;
+        if (++s == KS) { s = 0; par ^= 1; }
+        if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
+          ok = mbar_wait(&v_empty[u & 1], ((u >> 1) & 1) ^ 1, status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
+          for (int pn = 0; pn < PAN; ++pn)
+            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, (j0 - u) * 128, hkv, b);
+          v_issued = u + 1;
+        }
+      }
+      if (!ok) {
+        mbar_wait(&q_full, 0, status);
+        for (int u = (issued > KS ? issued - KS : 0); u < issued; ++u) mbar_wait(&k_full[u % KS], (u / KS) & 1, status);
+        for (int u = (v_issued > 2 ? v_issued - 2 : 0); u < v_issued; ++u) mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
+      }
+    }
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------------------------------------------ UMMA issuer of block x (+ its V loads)
+    const int x = warp - 1;
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, false, true);
+      const bool present_x = (x == 0) || hasB;
+      const int first = (x == 0) ? firstA : 0;
+      const uint64_t dQ = make_smem_desc(smem_u32(sQ + x * Cfg::kTileBytes), 16, 1024);
+      const uint64_t dK0 = make_smem_desc(smem_u32(sK), 16, 1024);
+      const uint64_t dV0 = make_smem_desc(smem_u32(sV), 16384, 1024);
+      const uint32_t tS = tmem_addr(tb, 0, x * 128), tO = tmem_addr(tb, 0, 256 + x * 128);
+      bool ok = mbar_wait(&q_full, 0, status);
+      int r = 0;                       // PVs issued (retained tiles); also counts this block's V loads
+      int s = 0;                       // K stage of step u
+      uint32_t kpar = 0;               // parity of k_full[s] for step u
+      for (int u = 0; u < U && ok; ++u) {
+        ok = mbar_wait(&k_full[s], kpar, status);
+        if (!ok) break;
+        if (!present_x || u < first) {
+          mbar_arrive(&k_empty[s]);    // this block has no tile at this step
+          if (kDense) {                // release the shared V stage too, paced by its arrival
+            ok = mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
+            if (!ok) break;
+            mbar_arrive(&v_empty[u & 1]);
+          }
+        } else {
+          const int t = u - first;     // tile index of this block
+          tc_fence_after();
+          const uint64_t dK = desc_advance(dK0, s * Cfg::kTileBytes);
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+            mma_ss(tS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0);
+          }
+          tc_commit(&k_empty[s]);
+          tc_commit(&s_full[x]);
+          bool retain = true;
+          if (!kDense) {
+            ok = mbar_wait(&vote_bar[x], t & 1, status);
+            if (!ok) break;
+            retain = (*(volatile int*)&flag[x][t % 3]) != 0;
+          }
+          if (retain) {
+            // MALA: V is loaded on demand into this block's own stage (free once its previous PV retired);
+            // dense: V(u) sits in the shared ring stage u & 1
+            const int vs = kDense ? (u & 1) : x;
+            const uint32_t vpar = kDense ? ((u >> 1) & 1) : (r & 1);
+            if (!kDense) {
+              ok = mbar_wait(&v_empty[x], (r & 1) ^ 1, status);
+              if (!ok) break;
+              mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
+              for (int pn = 0; pn < PAN; ++pn)
+                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, (j0 - u) * 128, hkv, b);
+            }
+            ok = mbar_wait(&p_full[x], r & 1, status);
+            if (ok) ok = mbar_wait(&v_full[vs], vpar, status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t acc0 = r > 0 ? 1u : 0u;
+            const uint64_t dVs = desc_advance(dV0, vs * Cfg::kTileBytes);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, k > 0 ? 1u : acc0);
+            tc_commit(&v_empty[vs]);
+            ++r;
+          }
+        }
+        if (++s == KS) { s = 0; kpar ^= 1; }
+      }
+      // every MMA of this block has retired (and every V copy landed) before the CTA may exit
+      tc_commit(&fin_bar);
+      mbar_wait(&fin_bar, 0, status);
+      if (!kDense && !ok && r > 0) mbar_wait(&v_full[x], (r - 1) & 1, status);
+    }
+  }
+  } else {
+    reg_alloc<208>();
+    // ------------------------------------------------------------------ softmax groups: one thread per row
+    const int x = (warp - 4) >> 2;                   // 0 = block A, 1 = block B
+    const int i = x ? iB : iA;
+    const bool present_x = (x == 0) || hasB;
+    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
+    const int rl = (int)lane_base + lane;
+    const int row = i * 128 + rl;
+    const bool valid = row < p.N;
+    const float c2 = p.scale_log2;
+    const float Lq = p.causal ? (float)(row + 1) : (float)p.N;
+    const float theta = kDense ? -INFINITY : (p.log2_tau - log2f(Lq));
+    const uint32_t colS = (uint32_t)x * 128u, colO = 256u + (uint32_t)x * 128u;
+    const int first = (x == 0) ? firstA : 0;
+    const int T = present_x ? (U - first) : 0;       // tiles of this block
+    float m_ref = -INFINITY, l = 0.f;
+    int r = 0;
+    bool ok = true;
+    uint32_t bm_bits = 0;
+    int bm_word = -1;
+    const bool stat_thread = ((warp & 3) == 0 && lane == 0);
+    const size_t stat_row = (size_t)(b * p.Hq + h) * p.Tr + i;
+    uint32_t* bm_row = (p.bitmask && present_x) ? p.bitmask + stat_row * p.words : nullptr;
+
+    for (int t = 0; t < T; ++t) {
+      const int j = j0 - first - t;
+      ok = mbar_wait(&s_full[x], t & 1, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t s0[32], s1[32], s2[32], s3[32];
+      tmem_ld_x32(tmem_addr(tb, lane_base, colS + 0), s0);
+      tmem_ld_x32(tmem_addr(tb, lane_base, colS + 32), s1);
+      tmem_ld_x32(tmem_addr(tb, lane_base, colS + 64), s2);
+      tmem_ld_x32(tmem_addr(tb, lane_base, colS + 96), s3);
+      tmem_wait_ld();
+      if (t == 0) {
+        // first visited tile: causal diagonal and / or the ragged end of the key range
+        const int lim = p.causal ? rl : (p.N - 1 - j * 128);
+        const uint32_t ninf = 0xff800000u;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          if (e > lim) s0[e] = ninf;
+          if (e + 32 > lim) s1[e] = ninf;
+          if (e + 64 > lim) s2[e] = ninf;
+          if (e + 96 > lim) s3[e] = ninf;
+        }
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        mx0 = fmaxf(mx0, fmaxf(__uint_as_float(s0[e]), __uint_as_float(s1[e])));
+        mx1 = fmaxf(mx1, fmaxf(__uint_as_float(s2[e]), __uint_as_float(s3[e])));
+      }
+      const float mt = fmaxf(mx0, mx1) * c2;   // row maximum of the scaled scores, log2 domain
+      bool retain = true;
+      if (!kDense) {
+        // Eq. 3: skip iff rowmax - (m + log l) < log(tau / L) for every valid row
+        bool vote;
+        if (l == 0.f) vote = valid;   // nothing retained yet: the log-ratio is +inf
+        else vote = valid && !(((mt - (m_ref + log2f(l))) - theta) < 0.f);
+        const bool any = __any_sync(0xffffffffu, vote);
+        if (lane == 0) {
+          if (any) *(volatile int*)&flag[x][t % 3] = 1;
+          if ((warp & 3) == 0) *(volatile int*)&flag[x][(t + 1) % 3] = 0;
+          tc_fence_before();
+          mbar_arrive(&vote_bar[x]);
+        }
+        ok = mbar_wait(&vote_bar[x], t & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        retain = (*(volatile int*)&flag[x][t % 3]) != 0;
+      }
+      if (!retain) continue;   // m, l, O unchanged; no exp, no P, no PV
+      if (stat_thread && bm_row) {
+        if ((j >> 5) != bm_word) {
+          if (bm_word >= 0) bm_row[bm_word] = bm_bits;
+          bm_word = j >> 5;
+          bm_bits = 0;
+        }
+        bm_bits |= 1u << (j & 31);
+      }
+      // Lazy rescaling: the reference maximum only moves when the row maximum grew by more than 2^8.
+      // The scores of this tile were produced after every earlier PV of this block (same tensor pipe,
+      // program order), so O may be touched here without a further wait.
+      if (r == 0) {
+        m_ref = mt;
+      } else {
+        const bool need = mt > m_ref + 8.f;
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = fmaxf(m_ref, mt);
+          const float alpha = fast_exp2(m_ref - m_new);
+          l *= alpha;
+          m_ref = m_new;
+#pragma unroll
+          for (int cc = 0; cc < D / 32; ++cc) {
+            uint32_t o[32];
+            tmem_ld_x32(tmem_addr(tb, lane_base, colO + cc * 32), o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st_x32(tmem_addr(tb, lane_base, colO + cc * 32), o);
+          }
+        }
+      }
+      // Dense kernel: the two softmax groups take turns in the exponential phase (B(0), A(0), B(1), A(1), ...)
+      // so that one block's exponentials run while the tensor pipe works for the other block, instead of
+      // both groups contending for the MUFU at the same time and then for the tensor pipe at the same time.
+      // A's tile t follows B's tile of the same key step (t + firstA); B's tile t follows A's tile of the previous
+      // step (t - 1 - firstA).  turn_bar[0] counts B's finished exp phases from tile firstA on, turn_bar[1] A's, so
+      // every waiter sees the phases in sequence.
+      if (kDense && hasB) {
+        const int idx = (x == 0) ? t : (t - 1 - firstA);
+        if (idx >= 0) {
+          ok = mbar_wait(&turn_bar[x], idx & 1, status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
+      }
+      // P = exp2(s * c2 - m_ref), row sum in fp32 before the bf16 cast, P written over S
+      const float nm = -m_ref;
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+      uint32_t pk[16];
+#define MALA_P_CHUNK(SRC, COL)                                                         \
+      {                                                                                \
+        _Pragma("unroll") for (int e = 0; e < 8; ++e) {                                \
+          const float p0 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e]), c2, nm));        \
+          const float p1 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 1]), c2, nm));    \
+          const float p2 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 2]), c2, nm));    \
+          const float p3 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 3]), c2, nm));    \
+          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;                              \
+          pk[2 * e] = pack_bf16x2(p0, p1);                                             \
+          pk[2 * e + 1] = pack_bf16x2(p2, p3);                                         \
+        }                                                                              \
+        tmem_st_x16(tmem_addr(tb, lane_base, colS + (COL)), pk);                       \
+      }
+      MALA_P_CHUNK(s0, 0)
+      MALA_P_CHUNK(s1, 16)
+      MALA_P_CHUNK(s2, 32)
+      MALA_P_CHUNK(s3, 48)
+#undef MALA_P_CHUNK
+      l += (sum0 + sum1) + (sum2 + sum3);
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&p_full[x]);
+        if (kDense && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);   // the other group's turn
+      }
+      ++r;
+    }
+
+    if (ok && present_x) {
+      // finalize once every PV has retired: O <- O / l, lse <- m + log l
+      ok = mbar_wait(&fin_bar, 0, status);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok && present_x) {
+      tc_fence_after();
+      const float inv = 1.f / l;
+      __nv_bfloat16* orow = p.o + (int64_t)b * p.o_sb + (int64_t)row * p.o_sn + (int64_t)h * p.o_sh;
+#pragma unroll
+      for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t o[32];
+        tmem_ld_x32(tmem_addr(tb, lane_base, colO + cc * 32), o);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + cc * 32 + v * 8) = w;
+          }
+        }
+      }
+      if (valid) p.lse[((size_t)b * p.Hq + h) * p.N + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      if (stat_thread) {
+        if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
+        if (p.retained) p.retained[stat_row] = (uint32_t)r;
+        if (p.totals) {
+          atomicAdd(&p.totals[0], (unsigned long long)r);
+          atomicAdd(&p.totals[1], (unsigned long long)T);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tb, Cfg::kTmemCols);
+}
+
+}  // namespace mala

@@ -58,6 +58,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
   return true;
 }
 
+// Register re-allocation between the warpgroups of a CTA (executed by all four warps of a warpgroup)
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
 // generic-proxy writes to shared memory made visible to the async proxy (TMA, tcgen05.mma)
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -142,6 +146,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
   d |= (uint64_t)2 << 61;  // SWIZZLE_128B
   return d;
 }
+
+// Descriptor of the same tile `bytes` further on in shared memory (bytes a multiple of 16; the
+// 14-bit start-address field counts 16-byte units and never carries within the 256 KB window).
+// Building descriptors once and advancing them keeps the single issuing thread ahead of the tensor pipe.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
 
 // Instruction descriptor of tcgen05.mma kind::f16: bf16 A and B, fp32 accumulate, M x N tile.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
