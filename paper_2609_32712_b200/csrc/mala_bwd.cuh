@@ -11,11 +11,11 @@
 //                           global memory by TMA reduce-add from shared memory.
 //   bwd_convert_dq_kernel : dq = bf16(scale * accumulator).
 //
-// Warp roles of the main kernel (448 threads):
-//   warp 0     TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
-//   warp 1     UMMA issuer (and, in the MALA kernel, the on-demand dO loads)
-//   warps 2-9  compute group, two threads per key row of the transposed tile (64 query columns each)
-//   warps 10-13 dQ group, one thread per query row of the dQ tile
+// Warp roles of the main kernel (512 threads; registers are re-split between the warpgroups):
+//   warp 0      TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
+//   warp 1      UMMA issuer (and, in the MALA kernel, the on-demand dO loads); warps 2-3 idle
+//   warps 4-11  compute group, two threads per key row of the transposed tile (64 query columns each)
+//   warps 12-15 dQ group, one thread per query row of the dQ tile
 #pragma once
 #include <cuda_runtime.h>
 
@@ -48,7 +48,7 @@ struct BwdCfg {
   // K, V, Q x2, dO x2.  dS^T (32 KB) of a retained tile overwrites that tile's dO stage once dP and dV
   // have consumed it (D = 128); for D = 64 a dO stage is too small, so two separate dS stages follow.
   static constexpr int kSmemBytes = 6 * kTileBytes + (D == 128 ? 0 : 2 * kDsBytes) + 1024;
-  static constexpr int kThreads = 448;
+  static constexpr int kThreads = 512;
   static constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
 };
 
@@ -57,7 +57,7 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 }
 
 template <int D, bool kDense>
-__global__ void __launch_bounds__(448, 1)
+__global__ void __launch_bounds__(512, 1)
 mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
                 const __grid_constant__ CUtensorMap tmAcc, const BwdParams p) {
@@ -73,7 +73,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
 
   __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
-      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free;
+      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free, ds_free;
   __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[3];
@@ -99,7 +99,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init(&s_full, 1); mbar_init(&p_full, 8); mbar_init(&dp_full, 1); mbar_init(&ds_full, 8);
     mbar_init(&dv_done, 1); mbar_init(&grp_bar, 8); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
     mbar_init(&fin_bar, 1);
-    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1);
+    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1); mbar_init(&ds_free, 1);
     flag[0] = flag[1] = flag[2] = 0;
     dq_info = -1;
     mbar_fence_init();
@@ -112,6 +112,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
 
+  if (warp < 4) {
+  reg_dealloc<56>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -231,20 +233,20 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const uint64_t dQm = desc_advance(dQm0, s * Cfg::kTileBytes);
           const uint32_t acc1 = r > 0 ? 1u : 0u;
 #pragma unroll
+          for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j  (into the dP columns), first: its read-out takes longest
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
+                   k > 0);
+          *(volatile int*)&dq_info = n * 2 + ds;
+          mbar_arrive(&dq_info_bar);
+          tc_commit(&dq_full);
+#pragma unroll
           for (int k = 0; k < 8; ++k) {   // dK += dS^T Q
             const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
             mma_ss(tmem_addr(tb, 0, Cfg::kColDK), desc_advance(dDSk, off), desc_advance(dQm, k * 2048), idesc_dv,
                    k > 0 ? 1u : acc1);
           }
-          // (the Q stage is released by the dQ group, which stages the dQ tile in it after these MMAs)
-#pragma unroll
-          for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j  (into the dP columns)
-            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
-                   k > 0);
-          tc_commit(&do_empty[ds]);   // dO stage (and the dS^T stored over it) is free once dK, dQ retire
-          *(volatile int*)&dq_info = n;
-          mbar_arrive(&dq_info_bar);
-          tc_commit(&dq_full);
+          tc_commit(&q_empty[s]);
+          tc_commit(&ds_free);   // dS^T has been consumed: the dQ group may stage the dQ tile in that stage
           ++r;
         } else {
           mbar_arrive(&q_empty[s]);
@@ -260,16 +262,17 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int u = (r > 1 ? r - 1 : 0); u <= r; ++u) mbar_wait(&do_full[u & 1], (u >> 1) & 1, status);
       }
     }
-  } else if (warp < 10) {
+  }
+  } else if (warp < 12) {
     // ------------------------------------------------------------------ compute group
     // Two threads per key row: warps 2-5 own query columns 0..63 of the transposed tile, warps 6-9
     // columns 64..127 (both warps of a pair reach the same TMEM lane quadrant).
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
-    const int hf = (warp - 2) >> 2;                 // column half
+    const int hf = (warp - 4) >> 2;                 // column half
     const bool valid_key = (j * 128 + rl) < p.N;
     const float c2 = p.scale_log2;
-    const bool stat_thread = (warp == 2 && lane == 0);
+    const bool stat_thread = (warp == 4 && lane == 0);
     bool ok = true;
     int r = 0;
     int r_head = 0;
@@ -343,7 +346,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
           if (any) *(volatile int*)&flag[n % 3] = 1;
-          if (warp == 2) *(volatile int*)&flag[(n + 1) % 3] = 0;
+          if (warp == 4) *(volatile int*)&flag[(n + 1) % 3] = 0;
           tc_fence_before();
           mbar_arrive(&vote_bar[n & 1]);
         }
@@ -485,30 +488,46 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------------ dQ group: thread = query row
-    // Each retained tile's dQ (fp32, 128 x D) is staged in the tile's own Q stage -- free once dK and dQ
-    // have retired -- in 32-column swizzled panels and added to the global accumulator by TMA
-    // reduce-add; the Q stage is handed back to the producer when the TMA has read it.
+    // Each retained tile's dQ (fp32, 128 x D) is read out of TMEM into registers at once (so the dP / dQ
+    // columns are free for the next tile right away), then staged in 32-column swizzled panels in the
+    // tile's dS^T stage -- free once dK has retired -- and added to the global accumulator by TMA
+    // reduce-add.  The stage goes back to the dO ring when the TMA has read it.
+    reg_alloc<200>();
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
-    const bool elected = (warp == 10 && lane == 0);
-    constexpr int kPanelsPerRound = (D == 128) ? 2 : 1;   // 16 KB panels that fit in one Q stage
+    const bool elected = (warp == 12 && lane == 0);
     uint32_t full_phase = 0, free_phase = 0;
     if (elected) tma_prefetch_desc(&tmAcc);
     for (int k = 0;; ++k) {
       bool ok = mbar_wait(&dq_info_bar, k & 1, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      const int n = *(volatile int*)&dq_info;
-      if (n < 0) break;
+      const int info = *(volatile int*)&dq_info;
+      if (info < 0) break;
+      const int n = info >> 1, ds = info & 1;
       ok = mbar_wait(&dq_full, k & 1, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      uint32_t a0[32], a1[32], a2[32], a3[32];
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 0), a0);
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 32), a1);
+      if (D == 128) {
+        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 64), a2);
+        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 96), a3);
+      }
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused by the next dP
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
       const int row0 = (int)(((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128);
-      uint8_t* stg = sQ + (n & 1) * Cfg::kTileBytes;
+      uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // two 16 KB panels
+      ok = mbar_wait(&ds_free, k & 1, status);     // dK has consumed dS^T
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
 #pragma unroll
-      for (int round = 0; round < 2; ++round) {
+      for (int round = 0; round < D / 64; ++round) {
         if (round > 0) {   // the panels are still being read by the previous round's reduce
           if (elected) { bulk_wait_read_all(); mbar_arrive(&stg_free); }
           ok = mbar_wait(&stg_free, free_phase & 1, status);
@@ -517,20 +536,15 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (!ok) break;
         }
 #pragma unroll
-        for (int cc = 0; cc < kPanelsPerRound; ++cc) {
-          const int chunk = round * kPanelsPerRound + cc;
-          uint32_t a[32];
-          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + chunk * 32), a);
-          tmem_wait_ld();
-          if (round == 1 && cc == kPanelsPerRound - 1) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused by the next dP
+        for (int v = 0; v < 8; ++v) {
+          const uint32_t off = rl * 128 + ((v ^ (rl & 7)) << 4);
+          if (round == 0) {
+            *reinterpret_cast<uint4*>(stg + off) = make_uint4(a0[4 * v], a0[4 * v + 1], a0[4 * v + 2], a0[4 * v + 3]);
+            *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a1[4 * v], a1[4 * v + 1], a1[4 * v + 2], a1[4 * v + 3]);
+          } else {
+            *reinterpret_cast<uint4*>(stg + off) = make_uint4(a2[4 * v], a2[4 * v + 1], a2[4 * v + 2], a2[4 * v + 3]);
+            *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a3[4 * v], a3[4 * v + 1], a3[4 * v + 2], a3[4 * v + 3]);
           }
-#pragma unroll
-          for (int v = 0; v < 8; ++v)
-            *reinterpret_cast<uint4*>(stg + cc * 16384 + rl * 128 + ((v ^ (rl & 7)) << 4)) =
-                make_uint4(a[4 * v], a[4 * v + 1], a[4 * v + 2], a[4 * v + 3]);
         }
         fence_proxy_async_smem();
         __syncwarp();
@@ -538,9 +552,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (elected) {
           ok = mbar_wait(&stg_full, full_phase & 1, status);
           if (ok) {
-#pragma unroll
-            for (int cc = 0; cc < kPanelsPerRound; ++cc)
-              tma_reduce_add_2d(&tmAcc, stg + cc * 16384, (round * kPanelsPerRound + cc) * 32, row0);
+            tma_reduce_add_2d(&tmAcc, stg, round * 64, row0);
+            tma_reduce_add_2d(&tmAcc, stg + 16384, round * 64 + 32, row0);
             bulk_commit_group();
           }
         }
@@ -549,7 +562,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
       }
       if (!ok) break;
-      if (elected) { bulk_wait_read_all(); mbar_arrive(&q_empty[n & 1]); }
+      if (elected) { bulk_wait_read_all(); mbar_arrive(&do_empty[ds]); }   // stage back to the dO ring
     }
     if (elected) bulk_wait_all();
   }
