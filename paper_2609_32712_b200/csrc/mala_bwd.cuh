@@ -11,11 +11,16 @@
 //                           global memory by TMA reduce-add from shared memory.
 //   bwd_convert_dq_kernel : dq = bf16(scale * accumulator).
 //
-// Warp roles of the main kernel (512 threads; registers are re-split between the warpgroups):
-//   warp 0      TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
-//   warp 1      UMMA issuer (and, in the MALA kernel, the on-demand dO loads); warps 2-3 idle
-//   warps 4-11  compute group, two threads per key row of the transposed tile (64 query columns each)
-//   warps 12-15 dQ group, one thread per query row of the dQ tile
+// Warp roles of the main kernel (768 threads; registers are re-split between the warpgroups):
+//   warp 0       TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
+//   warp 1       UMMA issuer (and, in the MALA kernel, the on-demand dO loads); warps 2-3 idle
+//   warps 4-11   score group: reads S^T, applies Eq. 4 and votes; retained tiles: P^T -> TMEM
+//   warps 12-19  dS group: takes P^T back out of TMEM (so the score buffer can be reused for the next
+//                tile at once), waits for dP^T and forms dS^T in shared memory
+//   warps 20-23  dQ group, one thread per query row of the dQ tile
+// Registers released by warps 0-3 (setmaxnreg) go to the dS and dQ groups.
+// Score and dS groups use two threads per key row (64 query columns each); while the dS group and the
+// tensor pipe finish tile n, the score group already works on tile n+1.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -48,7 +53,7 @@ struct BwdCfg {
   // K, V, Q x2, dO x2.  dS^T (32 KB) of a retained tile overwrites that tile's dO stage once dP and dV
   // have consumed it (D = 128); for D = 64 a dO stage is too small, so two separate dS stages follow.
   static constexpr int kSmemBytes = 6 * kTileBytes + (D == 128 ? 0 : 2 * kDsBytes) + 1024;
-  static constexpr int kThreads = 512;
+  static constexpr int kThreads = 768;
   static constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
 };
 
@@ -57,7 +62,7 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 }
 
 template <int D, bool kDense>
-__global__ void __launch_bounds__(512, 1)
+__global__ void __launch_bounds__(768, 1)
 mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
                 const __grid_constant__ CUtensorMap tmAcc, const BwdParams p) {
@@ -73,8 +78,9 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
 
   __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
-      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free, ds_free;
+      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free, ds_free, pt_read;
   __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
+  __shared__ __align__(16) float dq_ring[2][128];  // D of the retained tiles, for the dS group
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[3];
   __shared__ int dq_info;
@@ -99,7 +105,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init(&s_full, 1); mbar_init(&p_full, 8); mbar_init(&dp_full, 1); mbar_init(&ds_full, 8);
     mbar_init(&dv_done, 1); mbar_init(&grp_bar, 8); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
     mbar_init(&fin_bar, 1);
-    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1); mbar_init(&ds_free, 1);
+    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1); mbar_init(&ds_free, 1); mbar_init(&pt_read, 8);
     flag[0] = flag[1] = flag[2] = 0;
     dq_info = -1;
     mbar_fence_init();
@@ -113,7 +119,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tb = tmem_base_s;
 
   if (warp < 4) {
-  reg_dealloc<56>();
+  reg_dealloc<48>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -219,11 +225,13 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < 8; ++k)   // dV += P^T dO
-            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + k * 8), desc_advance(dDOm, k * 2048),
-                   idesc_dv, k > 0 ? 1u : acc0);
+            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + (k >> 2) * 64 + (k & 3) * 8),
+                   desc_advance(dDOm, k * 2048), idesc_dv, k > 0 ? 1u : acc0);
           tc_commit(&dv_done);
         }
-        // the score buffer is free again: recompute the next tile's scores while dS is being formed
+        // the score buffer is free once dV has been issued and the dS group holds P^T in registers:
+        // recompute the next tile's scores while dS is being formed
+        if (retain) { ok = mbar_wait(&pt_read, r & 1, status); if (!ok) break; }
         if (n + 1 < n_tot) { ok = issue_qk(n + 1); if (!ok) break; }
         if (retain) {
           ok = mbar_wait(&ds_full, r & 1, status);
@@ -264,9 +272,11 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   }
   } else if (warp < 12) {
-    // ------------------------------------------------------------------ compute group
-    // Two threads per key row: warps 2-5 own query columns 0..63 of the transposed tile, warps 6-9
+    // ------------------------------------------------------------------ score group
+    // Two threads per key row: warps 4-7 own query columns 0..63 of the transposed tile, warps 8-11
     // columns 64..127 (both warps of a pair reach the same TMEM lane quadrant).
+    // Each thread stays inside its own 64 TMEM columns: S^T is read once for the test and once more for
+    // P^T, whose packed columns (hf * 64 + 0..31) overwrite only score columns this thread has consumed.
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const int hf = (warp - 4) >> 2;                 // column half
@@ -308,17 +318,29 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s0[32], s1[32];
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 0), s0);
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 32), s1);
-      tmem_wait_ld();
-      if (p.causal && i == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
-        const uint32_t ninf = 0xff800000u;
-        const int c0 = hf * 64;
+      const bool diag = p.causal && i == j;   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
+      const uint32_t ninf = 0xff800000u;
+      // pass 1 (MALA only), Eq. 4: skip iff s - lse_q < log(tau / L_q) on every valid entry
+      float crit = -INFINITY;
+      if (!kDense) {
+        const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]) + hf * 16;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          if (c0 + e < rl) s0[e] = ninf;
-          if (c0 + e + 32 < rl) s1[e] = ninf;
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sc[32];
+          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + c * 32), sc);
+          tmem_wait_ld();
+          if (diag) {
+            const int c0 = hf * 64 + c * 32;
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (c0 + e < rl) sc[e] = ninf;
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float4 x0 = bb[c * 8 + e];
+            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y)),
+                                     fmaxf(fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w))));
+          }
         }
       }
       // publish the next tile's vectors (slot (n+1) % 3 was last read two tiles ago)
@@ -328,21 +350,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       bool retain = true;
       {
-        // Eq. 4: skip iff s - lse_q < log(tau / L_q) on every valid entry
-        bool vote = false;
-        if (!kDense) {
-          float crit = -INFINITY;
-          const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]) + hf * 16;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const float4 x0 = bb[e], x1 = bb[8 + e];
-            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s0[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(s0[4 * e + 1]), c2, -x0.y)),
-                                     fmaxf(fmaf(__uint_as_float(s0[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(s0[4 * e + 3]), c2, -x0.w))));
-            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(s1[4 * e + 0]), c2, -x1.x), fmaf(__uint_as_float(s1[4 * e + 1]), c2, -x1.y)),
-                                     fmaxf(fmaf(__uint_as_float(s1[4 * e + 2]), c2, -x1.z), fmaf(__uint_as_float(s1[4 * e + 3]), c2, -x1.w))));
-          }
-          vote = valid_key && !(crit < 0.f);
-        }
+        const bool vote = !kDense && valid_key && !(crit < 0.f);
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
           if (any) *(volatile int*)&flag[n % 3] = 1;
@@ -350,7 +358,6 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_before();
           mbar_arrive(&vote_bar[n & 1]);
         }
-        // this barrier also orders every thread's S^T loads before any thread's P^T stores below
         ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -370,69 +377,37 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             bm_bits |= 1u << (i & 31);
           }
         }
-        // P^T = exp2(s * c2 - lse2_q) (bf16): kept packed in registers and written over S^T in TMEM
-        uint32_t pk[32];
+        // D of this tile's queries for the dS group (which may lag behind by more than the vector slots)
+        if (hf == 0) dq_ring[r & 1][rl] = vec[slot][2][rl];
+        // pass 2: P^T = exp2(s * c2 - lse2_q) (bf16), written over S^T in TMEM as the A operand of dV
         const float4* ll = reinterpret_cast<const float4*>(vec[slot][0]) + hf * 16;
-#define MALA_BWD_P(SRC, CH)                                                                  \
-        {                                                                                    \
-          _Pragma("unroll") for (int e = 0; e < 8; ++e) {                                    \
-            const float4 x = ll[(CH) * 8 + e];                                               \
-            const float p0 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 0]), c2, -x.x));     \
-            const float p1 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 1]), c2, -x.y));     \
-            const float p2 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 2]), c2, -x.z));     \
-            const float p3 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 3]), c2, -x.w));     \
-            pk[(CH) * 16 + 2 * e] = pack_bf16x2(p0, p1);                                     \
-            pk[(CH) * 16 + 2 * e + 1] = pack_bf16x2(p2, p3);                                 \
-          }                                                                                  \
-          uint32_t tmp[16];                                                                  \
-          _Pragma("unroll") for (int e = 0; e < 16; ++e) tmp[e] = pk[(CH) * 16 + e];         \
-          tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 32 + (CH) * 16), tmp);      \
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sc[32], pk[16];
+          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + c * 32), sc);
+          tmem_wait_ld();
+          if (diag) {
+            const int c0 = hf * 64 + c * 32;
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (c0 + e < rl) sc[e] = ninf;
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float4 x = ll[c * 8 + e];
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x.x));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x.y));
+            const float p2 = fast_exp2(fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x.z));
+            const float p3 = fast_exp2(fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x.w));
+            pk[2 * e] = pack_bf16x2(p0, p1);
+            pk[2 * e + 1] = pack_bf16x2(p2, p3);
+          }
+          tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + c * 16), pk);
         }
-        MALA_BWD_P(s0, 0)
-        MALA_BWD_P(s1, 1)
-#undef MALA_BWD_P
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full);
-        // dS^T = P^T o (dP^T - D_q), bf16, into shared memory for the dK and dQ MMAs
-        // dS^T goes where this tile's dO lies (D = 128): wait until dP and dV have consumed it
-        ok = mbar_wait(&dp_full, r & 1, status);
-        if (ok) ok = mbar_wait(&dv_done, r & 1, status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after();
-        const float4* dd = reinterpret_cast<const float4*>(vec[slot][2]) + hf * 16;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t dp[32];
-          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + hf * 64 + c * 32), dp);
-          tmem_wait_ld();
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint32_t w[4];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const float4 x = dd[c * 8 + v * 2 + u];
-              const uint32_t pa = pk[c * 16 + v * 4 + 2 * u], pb = pk[c * 16 + v * 4 + 2 * u + 1];
-              const float p0 = __uint_as_float(pa << 16), p1 = __uint_as_float(pa & 0xffff0000u);
-              const float p2 = __uint_as_float(pb << 16), p3 = __uint_as_float(pb & 0xffff0000u);
-              const float d0 = p0 * (__uint_as_float(dp[v * 8 + u * 4 + 0]) - x.x);
-              const float d1 = p1 * (__uint_as_float(dp[v * 8 + u * 4 + 1]) - x.y);
-              const float d2 = p2 * (__uint_as_float(dp[v * 8 + u * 4 + 2]) - x.z);
-              const float d3 = p3 * (__uint_as_float(dp[v * 8 + u * 4 + 3]) - x.w);
-              w[2 * u] = pack_bf16x2(d0, d1);
-              w[2 * u + 1] = pack_bf16x2(d2, d3);
-            }
-            const uint32_t col = (uint32_t)(c * 32 + v * 8);
-            *reinterpret_cast<uint4*>(sDS + (r & 1) * Cfg::kDsBytes + hf * 16384 + sw128_offset((uint32_t)rl, col)) =
-                make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ds_full);
         ++r;
       }
       if (stat_thread && (n % ni == ni - 1)) {   // last tile of this query head
@@ -486,16 +461,81 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
       }
     }
-  } else {
-    // ------------------------------------------------------------------ dQ group: thread = query row
-    // Each retained tile's dQ (fp32, 128 x D) is read out of TMEM into registers at once (so the dP / dQ
-    // columns are free for the next tile right away), then staged in 32-column swizzled panels in the
-    // tile's dS^T stage -- free once dK has retired -- and added to the global accumulator by TMA
-    // reduce-add.  The stage goes back to the dO ring when the TMA has read it.
-    reg_alloc<200>();
+  } else if (warp < 20) {
+    // ------------------------------------------------------------------ dS group
+    // Per retained tile: P^T (bf16, this thread's 64 query columns) back out of TMEM, then
+    // dS^T = P^T o (dP^T - D_q) as bf16 into the tile's dS^T stage for the dK and dQ MMAs.
+    reg_alloc<88>();
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
-    const bool elected = (warp == 12 && lane == 0);
+    const int hf = (warp - 12) >> 2;
+    for (int r = 0;; ++r) {
+      // the issuer's final commit ends the loop: no retained tile follows
+      bool ok = mbar_wait_either(&p_full, r & 1, &fin_bar, 0, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      if (!mbar_try_wait(&p_full, r & 1)) break;   // woken by fin_bar
+      tc_fence_after();
+      uint32_t pk[32];
+      {
+        uint32_t t0[16], t1[16];
+        tmem_ld_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 0), t0);
+        tmem_ld_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 16), t1);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) { pk[e] = t0[e]; pk[16 + e] = t1[e]; }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&pt_read);        // the score buffer may be overwritten
+      // dS^T goes where this tile's dO lies (D = 128): wait until dP and dV have consumed it
+      ok = mbar_wait(&dp_full, r & 1, status);
+      if (ok) ok = mbar_wait(&dv_done, r & 1, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const float4* dd = reinterpret_cast<const float4*>(dq_ring[r & 1]) + hf * 16;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t dp[32];
+        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + hf * 64 + c * 32), dp);
+        tmem_wait_ld();
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          uint32_t w[4];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const float4 x = dd[c * 8 + v * 2 + u];
+            const uint32_t pa = pk[c * 16 + v * 4 + 2 * u], pb = pk[c * 16 + v * 4 + 2 * u + 1];
+            const float p0 = __uint_as_float(pa << 16), p1 = __uint_as_float(pa & 0xffff0000u);
+            const float p2 = __uint_as_float(pb << 16), p3 = __uint_as_float(pb & 0xffff0000u);
+            const float d0 = p0 * (__uint_as_float(dp[v * 8 + u * 4 + 0]) - x.x);
+            const float d1 = p1 * (__uint_as_float(dp[v * 8 + u * 4 + 1]) - x.y);
+            const float d2 = p2 * (__uint_as_float(dp[v * 8 + u * 4 + 2]) - x.z);
+            const float d3 = p3 * (__uint_as_float(dp[v * 8 + u * 4 + 3]) - x.w);
+            w[2 * u] = pack_bf16x2(d0, d1);
+            w[2 * u + 1] = pack_bf16x2(d2, d3);
+          }
+          const uint32_t col = (uint32_t)(c * 32 + v * 8);
+          *reinterpret_cast<uint4*>(sDS + (r & 1) * Cfg::kDsBytes + hf * 16384 + sw128_offset((uint32_t)rl, col)) =
+              make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ds_full);
+    }
+  } else {
+    // ------------------------------------------------------------------ dQ group: thread = query row
+    // Each retained tile's dQ (fp32, 128 x D) is read out of TMEM 64 columns at a time, staged as two
+    // 32-column swizzled panels in the tile's dS^T stage -- free once dK has retired -- and added to the
+    // global accumulator by TMA reduce-add.  The dP / dQ columns are released as soon as the last
+    // columns are in registers; the stage goes back to the dO ring when the TMA has read it.
+    reg_alloc<88>();
+    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
+    const int rl = (int)lane_base + lane;
+    const bool elected = (warp == 20 && lane == 0);
     uint32_t full_phase = 0, free_phase = 0;
     if (elected) tma_prefetch_desc(&tmAcc);
     for (int k = 0;; ++k) {
@@ -509,25 +549,25 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t a0[32], a1[32], a2[32], a3[32];
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 0), a0);
-      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 32), a1);
-      if (D == 128) {
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 64), a2);
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + 96), a3);
-      }
-      tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused by the next dP
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
       const int row0 = (int)(((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128);
       uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // two 16 KB panels
-      ok = mbar_wait(&ds_free, k & 1, status);     // dK has consumed dS^T
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
 #pragma unroll
       for (int round = 0; round < D / 64; ++round) {
+        uint32_t a0[32], a1[32];
+        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + round * 64 + 0), a0);
+        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + round * 64 + 32), a1);
+        tmem_wait_ld();
+        if (round == D / 64 - 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused by the next dP
+        }
+        if (round == 0) {  // dK has consumed dS^T: its stage may be overwritten
+          ok = mbar_wait(&ds_free, k & 1, status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
         if (round > 0) {   // the panels are still being read by the previous round's reduce
           if (elected) { bulk_wait_read_all(); mbar_arrive(&stg_free); }
           ok = mbar_wait(&stg_free, free_phase & 1, status);
@@ -538,13 +578,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
         for (int v = 0; v < 8; ++v) {
           const uint32_t off = rl * 128 + ((v ^ (rl & 7)) << 4);
-          if (round == 0) {
-            *reinterpret_cast<uint4*>(stg + off) = make_uint4(a0[4 * v], a0[4 * v + 1], a0[4 * v + 2], a0[4 * v + 3]);
-            *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a1[4 * v], a1[4 * v + 1], a1[4 * v + 2], a1[4 * v + 3]);
-          } else {
-            *reinterpret_cast<uint4*>(stg + off) = make_uint4(a2[4 * v], a2[4 * v + 1], a2[4 * v + 2], a2[4 * v + 3]);
-            *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a3[4 * v], a3[4 * v + 1], a3[4 * v + 2], a3[4 * v + 3]);
-          }
+          *reinterpret_cast<uint4*>(stg + off) = make_uint4(a0[4 * v], a0[4 * v + 1], a0[4 * v + 2], a0[4 * v + 3]);
+          *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a1[4 * v], a1[4 * v + 1], a1[4 * v + 2], a1[4 * v + 3]);
         }
         fence_proxy_async_smem();
         __syncwarp();

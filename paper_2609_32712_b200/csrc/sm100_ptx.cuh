@@ -62,6 +62,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* s
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
+// Bounded wait until either of two phases has completed (used where a consumer must also notice
+// that its producer has finished for good).
+__device__ __forceinline__ bool mbar_wait_either(uint64_t* bar_a, uint32_t parity_a, uint64_t* bar_b, uint32_t parity_b,
+                                                 int* status) {
+  const long long t0 = clock64();
+  uint32_t it = 0;
+  while (!mbar_try_wait(bar_a, parity_a) && !mbar_try_wait(bar_b, parity_b)) {
+    if (((++it) & 0xff) == 0) {
+      if (*(volatile int*)status != 0) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        atomicCAS(status, 0, kDevTimeout);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
 // generic-proxy writes to shared memory made visible to the async proxy (TMA, tcgen05.mma)
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
