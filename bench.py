@@ -327,11 +327,14 @@ def main():
     bwd_exec = bwd_executed_flops(ts["bwd_legal"], ts["bwd_retained"], c.d)
     fwd_exec = fwd_executed_flops(ts["fwd_legal"], ts["fwd_retained"], c.d)
     ach = bwd_exec / (bwd_ms * 1e-3) / 1e12
+    # DRAM bytes of one mala_bwd_kernel launch from the committed ncu capture of the same workload
+    # (profiles/mala_bwd_kernel_cfg3_literal_tau1e-4.txt: dram__bytes.sum.per_second x gpu__time_duration.sum)
+    traffic = {("cfg3", "literal", 1e-4): 68.939162e9 * 31.962048e-3}.get((args.workload, args.preset, tau))
     roofline = {"bound": "tensor", "kernel": "mala_bwd_kernel", "achieved": ach, "peak": peaks["tflops_sustained"],
-                "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": None,
+                "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": traffic,
                 "peak_source": f"{peaks['source']} (bf16 matmul, sustained)",
                 "note": "duration = whole mala_bwd call (preprocess + main + dQ convert), so frac is a lower bound",
-                "fwd": {"kernel": "mala_fwd_kernel", "achieved": fwd_exec / (fwd_ms * 1e-3) / 1e12,
+                "fwd": {"kernel": "mala_fwd2_kernel", "achieved": fwd_exec / (fwd_ms * 1e-3) / 1e12,
                         "frac": fwd_exec / (fwd_ms * 1e-3) / 1e12 / peaks["tflops_sustained"]}}
 
     # ---------------------------------------------------------------- end to end: host buffers, copies timed

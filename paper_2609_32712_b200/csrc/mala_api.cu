@@ -64,8 +64,6 @@ static int device_setup(int dev, int** status_out) {
   }
   if (!g_attr_done[dev]) {
     bool ok = true;
-    ok = ok && set_smem(mala_fwd_kernel<128, false, false>, FwdCfg<128, false>::kSmemBytes);
-    ok = ok && set_smem(mala_fwd_kernel<64, false, false>, FwdCfg<64, false>::kSmemBytes);
     ok = ok && set_smem(mala_fwd2_kernel<128, true>, Fwd2Cfg<128, true>::kSmemBytes);
     ok = ok && set_smem(mala_fwd2_kernel<128, false>, Fwd2Cfg<128, false>::kSmemBytes);
     ok = ok && set_smem(mala_fwd2_kernel<64, false>, Fwd2Cfg<64, false>::kSmemBytes);
@@ -109,20 +107,12 @@ static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float
 
 static const float kLog2e = 1.4426950408889634f;
 
-// Forward launch.  The dense path (tau = 0) runs two query blocks per CTA (mala_fwd2_kernel): its time
-// goes into the softmax path of every tile, which two warpgroups share better.  The MALA path runs one
-// query block per CTA with two score buffers (mala_fwd_kernel), so that QK^T of the next tile overlaps
-// the retention decision of the current one -- the faster arrangement when most tiles are skipped.
+// Forward (prefill) launch: two query blocks per CTA.  (The one-block kernel of mala_fwd.cuh serves decode.)
 template <int D, bool kDense>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                       cudaStream_t stream) {
-  if (true) {
-    dim3 grid((p.Tr + 1) / 2, p.Hq, p.B);
-    mala_fwd2_kernel<D, kDense><<<grid, Fwd2Cfg<D, kDense>::kThreads, Fwd2Cfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
-  } else {
-    dim3 grid(p.Tr, p.Hq, p.B);
-    mala_fwd_kernel<D, false, false><<<grid, FwdCfg<D, false>::kThreads, FwdCfg<D, false>::kSmemBytes, stream>>>(tq, tk, tv, p);
-  }
+  dim3 grid((p.Tr + 1) / 2, p.Hq, p.B);
+  mala_fwd2_kernel<D, kDense><<<grid, Fwd2Cfg<D, kDense>::kThreads, Fwd2Cfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
