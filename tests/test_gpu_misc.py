@@ -1,0 +1,117 @@
+"""GPU checks beyond plain parity: strided tensor views, run-to-run determinism, tau-monotonic support,
+ragged mid-size shapes in the skipping regime, and error reporting through the binding."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_32712_b200 import workloads as W
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mala():
+    from paper_2609_32712_b200 import mala as m
+    m.lib()
+    return m
+
+
+def _bhnd_view(t):
+    """Same values, stored [B,H,N,d] and viewed as [B,N,H,d] (strides sn = d, sh = N*d)."""
+    return t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+
+
+def test_strided_views_give_identical_results(mala):
+    w = W.custom_prefill(2, 4, 2, 640, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=31, preset="R")
+    q, k, v, do = (w[x].cuda() for x in ("q", "k", "v", "do"))
+    tau = 1e-4
+    o, lse, st = mala.fwd(q, k, v, w["scale"], tau, stats=True)
+    dq, dk, dv, _ = mala.bwd(q, k, v, o, do, lse, w["scale"], tau)
+    qs, ks, vs, dos = (_bhnd_view(t) for t in (q, k, v, do))
+    assert qs.stride() != q.stride()
+    o2 = _bhnd_view(torch.empty_like(q))
+    o2, lse2, st2 = mala.fwd(qs, ks, vs, w["scale"], tau, stats=True, out=o2)
+    dq2, dk2, dv2 = (_bhnd_view(torch.empty_like(t)) for t in (q, k, v))
+    mala.bwd(qs, ks, vs, o2, dos, lse2, w["scale"], tau, dq=dq2, dk=dk2, dv=dv2)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2) and torch.equal(lse, lse2) and torch.equal(st.bitmask, st2.bitmask)
+    assert torch.equal(dk, dk2) and torch.equal(dv, dv2)
+    assert (dq.float() - dq2.float()).abs().max() <= 1e-2 * dq.float().abs().max()   # fp32 adds in another order
+
+
+def test_forward_and_mask_are_deterministic(mala):
+    w = W.custom_prefill(1, 4, 2, 2048, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=33, preset="R")
+    q, k, v, do = (w[x].cuda() for x in ("q", "k", "v", "do"))
+    runs = []
+    for _ in range(3):
+        o, lse, st = mala.fwd(q, k, v, w["scale"], 1e-4, stats=True)
+        dq, dk, dv, bst = mala.bwd(q, k, v, o, do, lse, w["scale"], 1e-4, stats=True)
+        torch.cuda.synchronize()
+        runs.append((o.clone(), lse.clone(), st.bitmask.clone(), dk.clone(), dv.clone(), bst.bitmask.clone(), dq.clone()))
+    for r in runs[1:]:
+        for a, b in zip(runs[0][:6], r[:6]):
+            assert torch.equal(a, b)
+        assert (runs[0][6].float() - r[6].float()).abs().max() <= 1e-2 * runs[0][6].float().abs().max()
+
+
+def test_support_shrinks_as_tau_grows(mala):
+    # tau1 (1 + tau2) <= tau2 for consecutive values: the support under tau1 contains the support under tau2
+    w = W.custom_prefill(1, 4, 2, 4096, 128, head_types=["peaked", "peaked", "sink", "diffuse"], seed=35, preset="R")
+    q, k, v = (w[x].cuda() for x in ("q", "k", "v"))
+    masks = []
+    for tau in (0.0, 1e-5, 1e-4, 1e-3, 1e-1, 1.0):
+        _, _, st = mala.fwd(q, k, v, w["scale"], tau, stats=True)
+        masks.append(st.mask(32))
+    for a, b in zip(masks[:-1], masks[1:]):
+        assert (b <= a).all()
+    assert masks[-1].sum() < masks[1].sum()
+
+
+@pytest.mark.parametrize("N,d,tau", [(3000, 128, 1e-4), (2900, 64, 1e-3), (5000, 128, 1.0)])
+def test_ragged_mid_size_sampled(mala, oracle, N, d, tau):
+    w = W.custom_prefill(1, 4, 2, N, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=N, preset="R")
+    q, k, v, do = (w[x].cuda() for x in ("q", "k", "v", "do"))
+    T = -(-N // 128)
+    o, lse, fst = mala.fwd(q, k, v, w["scale"], tau, stats=True)
+    dq, dk, dv, bst = mala.bwd(q, k, v, o, do, lse, w["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    fwd_units = [(0, 1, T - 1), (0, 2, T // 2), (0, 3, 1)]
+    ref = oracle.fwd(w["q"], w["k"], w["v"], w["scale"], tau, 128, 128, units=fwd_units)
+    fm = fst.mask(T).cpu().numpy()
+    for (b, h, i) in fwd_units:
+        rows = slice(i * 128, min(N, (i + 1) * 128))
+        parity.check_mask(fm[b, h, i], ref["mask"][b, h, i], ref["crit"][b, h, i], list(range(i, -1, -1)), tau, i * 128 + 1)
+        parity.check_output(o[b, rows, h].float().cpu().numpy(), ref["o"][b, rows, h])
+    g = oracle.bwd(w["q"], w["k"], w["v"], o.float().cpu(), w["do"], lse.cpu().numpy(), w["scale"], tau, 128, 128,
+                   key_units=[(0, 0, T - 1), (0, 1, T // 3)], dq_units=[(0, 2, T - 1)])
+    for (b, hk, j) in [(0, 0, T - 1), (0, 1, T // 3)]:
+        rows = slice(j * 128, min(N, (j + 1) * 128))
+        parity.check_grad(dk[b, rows, hk].float().cpu().numpy(), g["dk"][b, rows, hk], "dk")
+        parity.check_grad(dv[b, rows, hk].float().cpu().numpy(), g["dv"][b, rows, hk], "dv")
+    rows = slice((T - 1) * 128, N)
+    parity.check_grad(dq[0, rows, 2].float().cpu().numpy(), g["dq"][0, rows, 2], "dq")
+    assert (bst.mask(T).transpose(2, 3) <= fst.mask(T)).all()
+
+
+def test_binding_reports_errors(mala):
+    q = torch.zeros(1, 256, 2, 128, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(1, 2, 256, device="cuda")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(mala.MalaError) as e:
+        mala.bwd(q, q, q, q, q, lse, 0.1, 1e-4, ws=small)
+    assert e.value.code == -4
+    with pytest.raises(mala.MalaError) as e:
+        mala.fwd(q, q, q, 0.1, -1.0)
+    assert e.value.code == -1
+    q96 = torch.zeros(1, 256, 2, 96, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(mala.MalaError) as e:
+        mala.fwd(q96, q96, q96, 0.1, 0.0)
+    assert e.value.code == -2
+    q64 = torch.zeros(1, 1, 2, 64, dtype=torch.bfloat16, device="cuda")
+    kv64 = torch.zeros(1, 256, 2, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(mala.MalaError) as e:        # decode supports d = 128 only
+        mala.decode(q64, kv64, kv64, 0.1, 0.0, 2)
+    assert e.value.code == -2
+    assert mala.device_status() == 0
