@@ -1,11 +1,11 @@
-// Split-KV decode ("Fused decoding execution"): the split kernel is the decode mode of the forward
-// kernel template (mala_fwd.cuh); this file holds the normalizer-aware merge of the split partials,
-// the workspace layout and the launch code.
+// Split-KV decode ("Fused decoding execution"): the persistent split kernel lives in
+// mala_decode_split.cuh; this file holds the normalizer-aware merge of the split partials, the
+// workspace layout and the launch code.
 #pragma once
 #include <cuda_runtime.h>
 
 #include "../../include/mala.h"
-#include "mala_fwd.cuh"
+#include "mala_decode_split.cuh"
 #include "tensor_map.h"
 
 namespace mala {
@@ -40,8 +40,8 @@ inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) {
 
 inline bool decode_set_attributes() {
   bool ok = true;
-  ok = ok && cudaFuncSetAttribute(mala_fwd_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128, false>::kSmemBytes) == cudaSuccess;
-  ok = ok && cudaFuncSetAttribute(mala_fwd_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<128, true>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
   return ok;
 }
 
@@ -54,33 +54,38 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   if (d != 128) return MALA_ERR_UNSUPPORTED;
   const int per = (Nk + num_splits - 1) / num_splits;
   const int tps = (per + 127) / 128;
+  if ((long long)B * Hkv * num_splits > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
 
   CUtensorMap tq, tk, tv;
-  // q [B,1,Hq,d] viewed with the heads as rows: one 128-row box starting at the group's first head
-  if (!make_tensor_map_bnhd(&tq, q.p, B, Hq, 1, d, q.sb, q.sh, 0, 128) ||
+  // q [B,1,Hq,d] viewed with the heads as rows: one 16-row box starting at the group's first head
+  if (!make_tensor_map_bnhd(&tq, q.p, B, Hq, 1, d, q.sb, q.sh, 0, 16) ||
       !make_tensor_map_bnhd(&tk, kc.p, B, Nk, Hkv, d, kc.sb, kc.sn, kc.sh, 128) ||
       !make_tensor_map_bnhd(&tv, vc.p, B, Nk, Hkv, d, vc.sb, vc.sn, vc.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
-  FwdParams p;
-  p.o = nullptr; p.o_sb = p.o_sn = p.o_sh = 0; p.lse = nullptr;
+  DecParams p;
+  p.o_part = o_part; p.lse_part = lse_part;
   p.retained = st ? st->retained_per_block : nullptr;
   p.bitmask = st ? st->tile_bitmask : nullptr;
   p.totals = st ? (unsigned long long*)st->totals : nullptr;
   p.status = status;
-  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = Nk; p.Tr = 0; p.words = (tps + 31) / 32; p.causal = 0;
-  p.o_part = o_part; p.lse_part = lse_part; p.tps = tps; p.num_splits = num_splits;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Nk = Nk; p.tps = tps; p.num_splits = num_splits; p.words = (tps + 31) / 32;
+  p.n_items = B * Hkv * num_splits;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
   if (p.bitmask &&
       cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hkv * num_splits * p.words * sizeof(uint32_t), stream) != cudaSuccess)
     return MALA_ERR_CUDA;
 
-  dim3 grid(num_splits, Hkv, B);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return MALA_ERR_CUDA;
+  const int grid = p.n_items < sms ? p.n_items : sms;   // persistent: one CTA per SM
   if (tau == 0.f)
-    mala_fwd_kernel<128, true, true><<<grid, 192, FwdCfg<128, true>::kSmemBytes, stream>>>(tq, tk, tv, p);
+    mala_decode_split_kernel<true><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);
   else
-    mala_fwd_kernel<128, false, true><<<grid, 192, FwdCfg<128, false>::kSmemBytes, stream>>>(tq, tk, tv, p);
+    mala_decode_split_kernel<false><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   decode_merge_kernel<128><<<B * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb, o.sh, lse_opt, Hq,
                                                        num_splits);
