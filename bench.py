@@ -334,7 +334,7 @@ def main():
                 "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": traffic,
                 "peak_source": f"{peaks['source']} (bf16 matmul, sustained)",
                 "note": "duration = whole mala_bwd call (preprocess + main + dQ convert), so frac is a lower bound",
-                "fwd": {"kernel": "mala_fwd2_kernel", "achieved": fwd_exec / (fwd_ms * 1e-3) / 1e12,
+                "fwd": {"kernel": "mala_fwd_kernel", "achieved": fwd_exec / (fwd_ms * 1e-3) / 1e12,
                         "frac": fwd_exec / (fwd_ms * 1e-3) / 1e12 / peaks["tflops_sustained"]}}
 
     # ---------------------------------------------------------------- end to end: host buffers, copies timed

@@ -8,7 +8,6 @@
 #include "mala_bwd.cuh"
 #include "mala_decode.cuh"
 #include "mala_fwd.cuh"
-#include "mala_fwd2.cuh"
 #include "tensor_map.h"
 
 namespace mala {
@@ -64,10 +63,10 @@ static int device_setup(int dev, int** status_out) {
   }
   if (!g_attr_done[dev]) {
     bool ok = true;
-    ok = ok && set_smem(mala_fwd2_kernel<128, true>, Fwd2Cfg<128, true>::kSmemBytes);
-    ok = ok && set_smem(mala_fwd2_kernel<128, false>, Fwd2Cfg<128, false>::kSmemBytes);
-    ok = ok && set_smem(mala_fwd2_kernel<64, false>, Fwd2Cfg<64, false>::kSmemBytes);
-    ok = ok && set_smem(mala_fwd2_kernel<64, true>, Fwd2Cfg<64, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<128, true>, FwdCfg<128, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<128, false>, FwdCfg<128, false>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<64, false>, FwdCfg<64, false>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<64, true>, FwdCfg<64, true>::kSmemBytes);
     ok = ok && bwd_set_attributes();
     ok = ok && decode_set_attributes();
     if (!ok) return MALA_ERR_CUDA;
@@ -107,12 +106,12 @@ static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float
 
 static const float kLog2e = 1.4426950408889634f;
 
-// Forward (prefill) launch: two query blocks per CTA.  (The one-block kernel of mala_fwd.cuh serves decode.)
+// Forward (prefill) launch: two query blocks per CTA.
 template <int D, bool kDense>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                       cudaStream_t stream) {
   dim3 grid((p.Tr + 1) / 2, p.Hq, p.B);
-  mala_fwd2_kernel<D, kDense><<<grid, Fwd2Cfg<D, kDense>::kThreads, Fwd2Cfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
+  mala_fwd_kernel<D, kDense><<<grid, FwdCfg<D, kDense>::kThreads, FwdCfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
@@ -205,7 +204,6 @@ int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const 
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Tr = (N + 127) / 128; p.words = (p.Tr + 31) / 32; p.causal = causal ? 1 : 0;
   p.scale_log2 = scale * kLog2e;
   p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
-  p.o_part = nullptr; p.lse_part = nullptr; p.tps = 0; p.num_splits = 0;
   if (p.bitmask) {
     if (cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * p.Tr * p.words * sizeof(uint32_t), stream) != cudaSuccess)
       return MALA_ERR_CUDA;

@@ -1,21 +1,22 @@
-// MALA forward (Algorithm 1) and split-KV decode ("Fused decoding execution") for sm_100a.
+// MALA forward (Algorithm 1) for sm_100a, prefill version: two query blocks per CTA.
 //
-// One CTA owns one 128-row query block of one (batch, query head) and walks its legal key blocks
-// from the diagonal toward earlier keys.  Warp roles (192 threads):
-//   warp 0      : TMA producer for Q (once) and the K ring
-//   warp 1      : UMMA issuer.  S = Q K^T for EVERY tile into one of two TMEM score buffers; after the
-//                 retention decision of a tile it issues the V load and, once P is ready, O += P V.
-//                 A skipped tile issues no V load and no PV MMA.
-//   warps 2..5  : softmax group, one thread per query row.  Reads S from TMEM, forms the row maximum,
-//                 votes on retention (Eq. 3), and for retained tiles writes P (bf16) over S in TMEM
-//                 and keeps the running (m, l); O is rescaled lazily in TMEM.
+// One CTA owns the two consecutive 128-row query blocks A = 2c and B = 2c+1 of one (batch, query
+// head).  They share the K tiles; each block has its own UMMA-issuing thread, softmax warpgroup,
+// score buffer, V stage and output accumulator (TMEM: S_A, S_B, O_A, O_B = 512 columns).  A thread
+// that issues tcgen05.mma stalls until the tensor pipe accepts the instruction, so the waits and
+// commits of one block's issuer run while the other block's MMAs execute, and one block's rows are in
+// the softmax path while the pipe works for the other block.
+// Each block keeps the semantics of Algorithm 1 on its own: its tiles are visited from ITS diagonal
+// toward earlier keys, the test for a tile uses the state left by that block's previous retained tile,
+// and a skipped tile issues no exp, no P, no V load and no PV.
+//
+// Warp roles (384 threads):
+//   warp 0       TMA producer: Q_A, Q_B once, K ring (a K stage is released when both issuers are done)
+//   warp 1, 2    UMMA issuers of block A and B: S_X = Q_X K^T for every tile, then (after the vote) the V
+//                load of that block and O_X += P_X V; the next QK of X follows its PV in program order, so
+//                the single score buffer of X is reused in tensor-pipe order without a barrier
+//   warps 4-7    softmax group of block A, warps 8-11 of block B (one thread per query row)
 // All synchronisation is by mbarriers with bounded waits.
-//
-// Decode mode (kDecode): one CTA owns one split of one (batch, KV head).  The rows of its "query
-// block" are the G = Hq/Hkv query heads that share the KV head (rows G..127 of the tile hold other
-// heads or zeros and are ignored), L = Nk for every row, tiles of the split are visited newest
-// first, and the CTA writes a normalised fp32 partial output and its log-normalizer per head.  Only
-// one softmax warp (TMEM lanes 0..31) is active.
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -30,82 +31,63 @@ struct FwdParams {
   unsigned long long* totals;    // [2] or null
   int* status;
   int B, Hq, Hkv, N, Tr, words, causal;
-  // decode only
-  float* o_part;                 // [B, Hq, num_splits, D] fp32, normalised per split
-  float* lse_part;               // [B, Hq, num_splits] natural log; -inf for an empty split
-  int tps, num_splits;           // tiles per split, number of splits (N is Nk)
   float scale_log2;              // scale * log2(e)
   float log2_tau;                // log2(tau); unused by the dense kernel
 };
 
 template <int D, bool kDense>
 struct FwdCfg {
-  static constexpr int kPanels = D / 64;                 // 64-column swizzle panels per tile
+  static constexpr int kPanels = D / 64;
   static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kKStages = (D == 128) ? (kDense ? 3 : 4) : 4;
-  static constexpr int kVStages = (D == 128) ? (kDense ? 3 : 2) : 3;
-  static constexpr int kSmemBytes = (1 + kKStages + kVStages) * kTileBytes + 1024;
-  static constexpr int kThreads = 192;
+  static constexpr int kKStages = 3;
+  // Q_A, Q_B, K ring, V_A, V_B
+  static constexpr int kSmemBytes = (2 + kKStages + 2) * kTileBytes + 1024;
+  static constexpr int kThreads = 384;
   static constexpr uint32_t kTmemCols = 512;
-  static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
 };
 
-template <int D, bool kDense, bool kDecode>
-__global__ void __launch_bounds__(192, 1)
+template <int D, bool kDense>
+__global__ void __launch_bounds__(384, 1)
 mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                const __grid_constant__ CUtensorMap tmV, const FwdParams p) {
+                 const __grid_constant__ CUtensorMap tmV, const FwdParams p) {
   using Cfg = FwdCfg<D, kDense>;
-  constexpr int KS = Cfg::kKStages, VS = Cfg::kVStages, PAN = Cfg::kPanels;
+  constexpr int KS = Cfg::kKStages, PAN = Cfg::kPanels;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;
-  uint8_t* sK = sQ + Cfg::kTileBytes;
-  uint8_t* sV = sK + KS * Cfg::kTileBytes;
+  uint8_t* sQ = smem;                               // [2] blocks A, B
+  uint8_t* sK = sQ + 2 * Cfg::kTileBytes;
+  uint8_t* sV = sK + KS * Cfg::kTileBytes;          // [2] blocks A, B
 
-  __shared__ uint64_t q_full, k_full[KS], k_empty[KS], s_full[2], vote_bar[2], p_full[2], v_full[VS], v_empty[VS],
-      o_done, fin_bar;
+  __shared__ uint64_t q_full, k_full[KS], k_empty[KS], v_full[2], v_empty[2], s_full[2], vote_bar[2], p_full[2],
+      fin_bar, turn_bar[2];
   __shared__ uint32_t tmem_base_s;
-  __shared__ int flag[3];
+  __shared__ int flag[2][3];
   __shared__ int early_exit;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.Hq / p.Hkv;
-  const int b = blockIdx.z;
-  int i, h, hkv, T, j0, q_row, q_head;
-  if (kDecode) {
-    const int split = blockIdx.x;
-    hkv = blockIdx.y;
-    h = hkv * G;
-    i = split;
-    const int lo = split * p.tps * 128;
-    const int hi = min(p.N, lo + p.tps * 128);
-    T = hi > lo ? (hi - lo + 127) / 128 : 0;   // legal tiles of this split
-    j0 = lo / 128 + T - 1;                     // newest tile first
-    q_row = hkv * G;                           // rows of the Q tile are query heads
-    q_head = 0;
-  } else {
-    i = p.Tr - 1 - (int)blockIdx.x;            // longest blocks first
-    h = blockIdx.y;
-    hkv = h / G;
-    T = p.causal ? (i + 1) : p.Tr;             // tiles to visit
-    j0 = p.causal ? i : (p.Tr - 1);            // first visited key block
-    q_row = i * 128;
-    q_head = h;
-  }
-  constexpr int kSoftmaxWarps = kDecode ? 1 : 4;
+  const int b = blockIdx.z, h = blockIdx.y, hkv = h / G;
+  const int npairs = (p.Tr + 1) / 2;
+  const int c = npairs - 1 - (int)blockIdx.x;        // longest pairs first
+  const int iA = 2 * c, iB = 2 * c + 1;
+  const bool hasB = iB < p.Tr;
+  // key steps u = 0 .. U-1 visit key block j0 - u; block X takes part from step first[X] on
+  const int j0 = p.causal ? (hasB ? iB : iA) : (p.Tr - 1);
+  const int U = j0 + 1;
+  const int firstA = p.causal ? (j0 - iA) : 0;       // 1 when B exists (B's diagonal is not legal for A)
   int* status = p.status;
 
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
     mbar_init(&q_full, 1);
-    for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); }
-    for (int s = 0; s < VS; ++s) { mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&s_full[s], 1); mbar_init(&vote_bar[s], kSoftmaxWarps); mbar_init(&p_full[s], kSoftmaxWarps);
+    for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 2); }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&v_full[x], 1); mbar_init(&v_empty[x], kDense ? 2 : 1);
+      mbar_init(&s_full[x], 1); mbar_init(&vote_bar[x], 4); mbar_init(&p_full[x], 4);
+      flag[x][0] = flag[x][1] = flag[x][2] = 0;
     }
-    mbar_init(&o_done, 1);
-    mbar_init(&fin_bar, 1);
-    flag[0] = flag[1] = flag[2] = 0;
+    mbar_init(&fin_bar, 2);
+    mbar_init(&turn_bar[0], 4); mbar_init(&turn_bar[1], 4);
     mbar_fence_init();
   }
   __syncthreads();
@@ -115,133 +97,151 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
-
+  if (warp < 4) {
+  // warps 0-3 (producer, issuers) need few registers; the two softmax warpgroups take the rest
+  reg_dealloc<72>();
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer: Q, K ring
+    // ------------------------------------------------------------------ TMA producer: Q_A, Q_B, K ring
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-      mbar_arrive_expect_tx(&q_full, Cfg::kTileBytes);
-      for (int pn = 0; pn < PAN; ++pn) tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, q_row, q_head, b);
-      int issued = 0;
+      mbar_arrive_expect_tx(&q_full, (hasB ? 2 : 1) * Cfg::kTileBytes);
+      for (int pn = 0; pn < PAN; ++pn) {
+        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, iA * 128, h, b);
+        if (hasB) tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, iB * 128, h, b);
+      }
+      int issued = 0, v_issued = 0, s = 0;
+      uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
       bool ok = true;
-      for (int t = 0; t < T && ok; ++t) {
-        const int s = t % KS;
-        ok = mbar_wait(&k_empty[s], ((t / KS) & 1) ^ 1, status);
+      for (int u = 0; u < U && ok; ++u) {
+        ok = mbar_wait(&k_empty[s], par, status);
         if (!ok) break;
         mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, (j0 - t) * 128, hkv, b);
-        issued = t + 1;
+          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, (j0 - u) * 128, hkv, b);
+        issued = u + 1;
+        if (++s == KS) { s = 0; par ^= 1; }
+        if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
+          ok = mbar_wait(&v_empty[u & 1], ((u >> 1) & 1) ^ 1, status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
+          for (int pn = 0; pn < PAN; ++pn)
+            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, (j0 - u) * 128, hkv, b);
+          v_issued = u + 1;
+        }
       }
-      if (!ok) {  // drain our own copies before leaving
+      if (!ok) {
         mbar_wait(&q_full, 0, status);
-        for (int t = (issued > KS ? issued - KS : 0); t < issued; ++t) mbar_wait(&k_full[t % KS], (t / KS) & 1, status);
+        for (int u = (issued > KS ? issued - KS : 0); u < issued; ++u) mbar_wait(&k_full[u % KS], (u / KS) & 1, status);
+        for (int u = (v_issued > 2 ? v_issued - 2 : 0); u < v_issued; ++u) mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ UMMA issuer (+ V loads)
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------------------------------------------ UMMA issuer of block x (+ its V loads)
+    const int x = warp - 1;
     if (lane == 0) {
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, false, true);
-      // descriptors are built once; per MMA only the start-address field is advanced
-      const uint64_t dQ = make_smem_desc(smem_u32(sQ), 16, 1024);
+      const bool present_x = (x == 0) || hasB;
+      const int first = (x == 0) ? firstA : 0;
+      const uint64_t dQ = make_smem_desc(smem_u32(sQ + x * Cfg::kTileBytes), 16, 1024);
       const uint64_t dK0 = make_smem_desc(smem_u32(sK), 16, 1024);
       const uint64_t dV0 = make_smem_desc(smem_u32(sV), 16384, 1024);
+      const uint32_t tS = tmem_addr(tb, 0, x * 128), tO = tmem_addr(tb, 0, 256 + x * 128);
       bool ok = mbar_wait(&q_full, 0, status);
-      int v_issued = 0;   // V tiles requested so far
-      int r = 0;          // PV MMAs issued so far (retained tiles)
-      uint32_t pcount[2] = {0, 0};
-      auto issue_qk = [&](int t) -> bool {
-        const int s = t % KS;
-        if (!mbar_wait(&k_full[s], (t / KS) & 1, status)) return false;
-        tc_fence_after();
-        const uint32_t dS = tmem_addr(tb, 0, (t & 1) ? Cfg::kColS1 : Cfg::kColS0);
-        const uint64_t dK = desc_advance(dK0, s * Cfg::kTileBytes);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-          mma_ss(dS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0);
-        }
-        tc_commit(&k_empty[s]);
-        tc_commit(&s_full[t & 1]);
-        return true;
-      };
-      auto issue_v = [&](int t) -> bool {   // V of visited tile t into stage v_issued % VS
-        const int s = v_issued % VS;
-        if (!mbar_wait(&v_empty[s], ((v_issued / VS) & 1) ^ 1, status)) return false;
-        mbar_arrive_expect_tx(&v_full[s], Cfg::kTileBytes);
-        for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sV + s * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[s], pn * 64, (j0 - t) * 128, hkv, b);
-        ++v_issued;
-        return true;
-      };
-      if (ok && T > 0) ok = issue_qk(0);
-      if (kDense) {
-        for (int t = 0; t < VS - 1 && t < T && ok; ++t) ok = issue_v(t);
-      }
-      for (int t = 0; t < T && ok; ++t) {
-        if (t + 1 < T) { ok = issue_qk(t + 1); if (!ok) break; }
-        bool retain = true;
-        if (!kDense) {
-          ok = mbar_wait(&vote_bar[t & 1], (t >> 1) & 1, status);
-          if (!ok) break;
-          retain = (*(volatile int*)&flag[t % 3]) != 0;
-          if (retain) { ok = issue_v(t); if (!ok) break; }
-        }
-        if (retain) {
-          const int s = r % VS;
-          ok = mbar_wait(&p_full[t & 1], pcount[t & 1] & 1, status);
-          if (!ok) break;
-          ++pcount[t & 1];
-          ok = mbar_wait(&v_full[s], (r / VS) & 1, status);
-          if (!ok) break;
+      int r = 0;                       // PVs issued (retained tiles); also counts this block's V loads
+      int s = 0;                       // K stage of step u
+      uint32_t kpar = 0;               // parity of k_full[s] for step u
+      for (int u = 0; u < U && ok; ++u) {
+        ok = mbar_wait(&k_full[s], kpar, status);
+        if (!ok) break;
+        if (!present_x || u < first) {
+          mbar_arrive(&k_empty[s]);    // this block has no tile at this step
+          if (kDense) {                // release the shared V stage too, paced by its arrival
+            ok = mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
+            if (!ok) break;
+            mbar_arrive(&v_empty[u & 1]);
+          }
+        } else {
+          const int t = u - first;     // tile index of this block
           tc_fence_after();
-          const uint32_t aP = tmem_addr(tb, 0, (t & 1) ? Cfg::kColS1 : Cfg::kColS0);
-          const uint32_t dO = tmem_addr(tb, 0, Cfg::kColO);
-          const uint64_t dV = desc_advance(dV0, s * Cfg::kTileBytes);
-          const uint32_t acc0 = r > 0 ? 1u : 0u;
+          const uint64_t dK = desc_advance(dK0, s * Cfg::kTileBytes);
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            mma_ts(dO, aP + k * 8, desc_advance(dV, k * 2048), idesc_pv, k > 0 ? 1u : acc0);
-          tc_commit(&v_empty[s]);
-          tc_commit(&o_done);
-          ++r;
-          if (kDense && t + VS - 1 < T) { ok = issue_v(t + VS - 1); if (!ok) break; }
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+            mma_ss(tS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0);
+          }
+          tc_commit(&k_empty[s]);
+          tc_commit(&s_full[x]);
+          bool retain = true;
+          if (!kDense) {
+            ok = mbar_wait(&vote_bar[x], t & 1, status);
+            if (!ok) break;
+            retain = (*(volatile int*)&flag[x][t % 3]) != 0;
+          }
+          if (retain) {
+            // MALA: V is loaded on demand into this block's own stage (free once its previous PV retired);
+            // dense: V(u) sits in the shared ring stage u & 1
+            const int vs = kDense ? (u & 1) : x;
+            const uint32_t vpar = kDense ? ((u >> 1) & 1) : (r & 1);
+            if (!kDense) {
+              ok = mbar_wait(&v_empty[x], (r & 1) ^ 1, status);
+              if (!ok) break;
+              mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
+              for (int pn = 0; pn < PAN; ++pn)
+                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, (j0 - u) * 128, hkv, b);
+            }
+            ok = mbar_wait(&p_full[x], r & 1, status);
+            if (ok) ok = mbar_wait(&v_full[vs], vpar, status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t acc0 = r > 0 ? 1u : 0u;
+            const uint64_t dVs = desc_advance(dV0, vs * Cfg::kTileBytes);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, k > 0 ? 1u : acc0);
+            tc_commit(&v_empty[vs]);
+            ++r;
+          }
         }
+        if (++s == KS) { s = 0; kpar ^= 1; }
       }
-      // all MMAs retired and all requested V copies landed before the CTA may exit
+      // every MMA of this block has retired (and every V copy landed) before the CTA may exit
       tc_commit(&fin_bar);
       mbar_wait(&fin_bar, 0, status);
-      if (!ok) {
-        for (int u = (v_issued > VS ? v_issued - VS : 0); u < v_issued; ++u) mbar_wait(&v_full[u % VS], (u / VS) & 1, status);
-      }
+      if (!kDense && !ok && r > 0) mbar_wait(&v_full[x], (r - 1) & 1, status);
     }
-  } else if (!kDecode || warp == 4) {
-    // ------------------------------------------------------------------ softmax group: one thread per row
+  }
+  } else {
+    reg_alloc<208>();
+    // ------------------------------------------------------------------ softmax groups: one thread per row
+    const int x = (warp - 4) >> 2;                   // 0 = block A, 1 = block B
+    const int i = x ? iB : iA;
+    const bool present_x = (x == 0) || hasB;
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
-    const int rl = (int)lane_base + lane;            // row inside the block
-    const int row = kDecode ? rl : i * 128 + rl;
-    const bool valid = kDecode ? (rl < G) : (row < p.N);
+    const int rl = (int)lane_base + lane;
+    const int row = i * 128 + rl;
+    const bool valid = row < p.N;
     const float c2 = p.scale_log2;
-    const float Lq = (p.causal && !kDecode) ? (float)(row + 1) : (float)p.N;
+    const float Lq = p.causal ? (float)(row + 1) : (float)p.N;
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f(Lq));
+    const uint32_t colS = (uint32_t)x * 128u, colO = 256u + (uint32_t)x * 128u;
+    const int first = (x == 0) ? firstA : 0;
+    const int T = present_x ? (U - first) : 0;       // tiles of this block
     float m_ref = -INFINITY, l = 0.f;
-    int r = 0;                                       // retained tiles so far
+    int r = 0;
     bool ok = true;
     uint32_t bm_bits = 0;
     int bm_word = -1;
-    const bool stat_thread = (warp == (kDecode ? 4 : 2) && lane == 0);
-    // telemetry row: (b, h, query block) in prefill, (b, hkv, split) in decode
-    const size_t stat_row = kDecode ? ((size_t)(b * p.Hkv + hkv) * p.num_splits + i) : ((size_t)(b * p.Hq + h) * p.Tr + i);
-    uint32_t* bm_row = p.bitmask ? p.bitmask + stat_row * p.words : nullptr;
+    const bool stat_thread = ((warp & 3) == 0 && lane == 0);
+    const size_t stat_row = (size_t)(b * p.Hq + h) * p.Tr + i;
+    uint32_t* bm_row = (p.bitmask && present_x) ? p.bitmask + stat_row * p.words : nullptr;
 
     for (int t = 0; t < T; ++t) {
-      const int j = j0 - t;
-      ok = mbar_wait(&s_full[t & 1], (t >> 1) & 1, status);
+      const int j = j0 - first - t;
+      ok = mbar_wait(&s_full[x], t & 1, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t colS = (t & 1) ? Cfg::kColS1 : Cfg::kColS0;
       uint32_t s0[32], s1[32], s2[32], s3[32];
       tmem_ld_x32(tmem_addr(tb, lane_base, colS + 0), s0);
       tmem_ld_x32(tmem_addr(tb, lane_base, colS + 32), s1);
@@ -250,7 +250,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tmem_wait_ld();
       if (t == 0) {
         // first visited tile: causal diagonal and / or the ragged end of the key range
-        const int lim = (p.causal && !kDecode) ? rl : (p.N - 1 - j * 128);
+        const int lim = p.causal ? rl : (p.N - 1 - j * 128);
         const uint32_t ninf = 0xff800000u;
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
@@ -260,13 +260,13 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (e + 96 > lim) s3[e] = ninf;
         }
       }
-      float mx = -INFINITY;
+      float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
       for (int e = 0; e < 32; ++e) {
-        mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(s0[e]), __uint_as_float(s1[e])),
-                             fmaxf(__uint_as_float(s2[e]), __uint_as_float(s3[e]))));
+        mx0 = fmaxf(mx0, fmaxf(__uint_as_float(s0[e]), __uint_as_float(s1[e])));
+        mx1 = fmaxf(mx1, fmaxf(__uint_as_float(s2[e]), __uint_as_float(s3[e])));
       }
-      const float mt = mx * c2;   // row maximum of the scaled scores, log2 domain
+      const float mt = fmaxf(mx0, mx1) * c2;   // row maximum of the scaled scores, log2 domain
       bool retain = true;
       if (!kDense) {
         // Eq. 3: skip iff rowmax - (m + log l) < log(tau / L) for every valid row
@@ -275,133 +275,108 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         else vote = valid && !(((mt - (m_ref + log2f(l))) - theta) < 0.f);
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
-          if (any) *(volatile int*)&flag[t % 3] = 1;
-          if (warp == (kDecode ? 4 : 2)) *(volatile int*)&flag[(t + 1) % 3] = 0;
+          if (any) *(volatile int*)&flag[x][t % 3] = 1;
+          if ((warp & 3) == 0) *(volatile int*)&flag[x][(t + 1) % 3] = 0;
           tc_fence_before();
-          mbar_arrive(&vote_bar[t & 1]);
+          mbar_arrive(&vote_bar[x]);
         }
-        ok = mbar_wait(&vote_bar[t & 1], (t >> 1) & 1, status);
+        ok = mbar_wait(&vote_bar[x], t & 1, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        retain = (*(volatile int*)&flag[t % 3]) != 0;
+        retain = (*(volatile int*)&flag[x][t % 3]) != 0;
       }
-      if (!retain) continue;   // m, l, O unchanged; no exp, no P, no V load, no PV
+      if (!retain) continue;   // m, l, O unchanged; no exp, no P, no PV
       if (stat_thread && bm_row) {
-        const int bit = kDecode ? (T - 1 - t) : j;   // decode: tile index inside the split
-        if ((bit >> 5) != bm_word) {
+        if ((j >> 5) != bm_word) {
           if (bm_word >= 0) bm_row[bm_word] = bm_bits;
-          bm_word = bit >> 5;
+          bm_word = j >> 5;
           bm_bits = 0;
         }
-        bm_bits |= 1u << (bit & 31);
+        bm_bits |= 1u << (j & 31);
       }
-      // running maximum with lazy rescaling: the reference m_ref only moves when the row maximum
-      // grew by more than 2^8, so P stays <= 256 and O is rarely touched
+      // Lazy rescaling: the reference maximum only moves when the row maximum grew by more than 2^8.
+      // The scores of this tile were produced after every earlier PV of this block (same tensor pipe,
+      // program order), so O may be touched here without a further wait.
       if (r == 0) {
         m_ref = mt;
       } else {
         const bool need = mt > m_ref + 8.f;
         if (__any_sync(0xffffffffu, need)) {
-          ok = mbar_wait(&o_done, (r - 1) & 1, status);   // PV of the previous retained tile has landed
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
           const float m_new = fmaxf(m_ref, mt);
           const float alpha = fast_exp2(m_ref - m_new);
           l *= alpha;
           m_ref = m_new;
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
+          for (int cc = 0; cc < D / 32; ++cc) {
             uint32_t o[32];
-            tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColO + c * 32), o);
+            tmem_ld_x32(tmem_addr(tb, lane_base, colO + cc * 32), o);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st_x32(tmem_addr(tb, lane_base, Cfg::kColO + c * 32), o);
+            tmem_st_x32(tmem_addr(tb, lane_base, colO + cc * 32), o);
           }
+        }
+      }
+      // Dense kernel: the two softmax groups take turns in the exponential phase (B(0), A(0), B(1), A(1), ...)
+      // so that one block's exponentials run while the tensor pipe works for the other block, instead of
+      // both groups contending for the MUFU at the same time and then for the tensor pipe at the same time.
+      // A's tile t follows B's tile of the same key step (t + firstA); B's tile t follows A's tile of the previous
+      // step (t - 1 - firstA).  turn_bar[0] counts B's finished exp phases from tile firstA on, turn_bar[1] A's, so
+      // every waiter sees the phases in sequence.
+      if (kDense && hasB) {
+        const int idx = (x == 0) ? t : (t - 1 - firstA);
+        if (idx >= 0) {
+          ok = mbar_wait(&turn_bar[x], idx & 1, status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
         }
       }
       // P = exp2(s * c2 - m_ref), row sum in fp32 before the bf16 cast, P written over S
       const float nm = -m_ref;
-      float sum = 0.f;
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
       uint32_t pk[16];
-#define MALA_P_CHUNK(SRC, COL)                                                     \
-      {                                                                            \
-        _Pragma("unroll") for (int e = 0; e < 16; ++e) {                           \
-          const float p0 = fast_exp2(fmaf(__uint_as_float(SRC[2 * e]), c2, nm));    \
-          const float p1 = fast_exp2(fmaf(__uint_as_float(SRC[2 * e + 1]), c2, nm));\
-          sum += p0 + p1;                                                          \
-          pk[e] = pack_bf16x2(p0, p1);                                             \
-        }                                                                          \
-        tmem_st_x16(tmem_addr(tb, lane_base, colS + (COL)), pk);                   \
+#define MALA_P_CHUNK(SRC, COL)                                                         \
+      {                                                                                \
+        _Pragma("unroll") for (int e = 0; e < 8; ++e) {                                \
+          const float p0 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e]), c2, nm));        \
+          const float p1 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 1]), c2, nm));    \
+          const float p2 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 2]), c2, nm));    \
+          const float p3 = fast_exp2(fmaf(__uint_as_float(SRC[4 * e + 3]), c2, nm));    \
+          sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;                              \
+          pk[2 * e] = pack_bf16x2(p0, p1);                                             \
+          pk[2 * e + 1] = pack_bf16x2(p2, p3);                                         \
+        }                                                                              \
+        tmem_st_x16(tmem_addr(tb, lane_base, colS + (COL)), pk);                       \
       }
       MALA_P_CHUNK(s0, 0)
       MALA_P_CHUNK(s1, 16)
       MALA_P_CHUNK(s2, 32)
       MALA_P_CHUNK(s3, 48)
 #undef MALA_P_CHUNK
-      l += sum;
+      l += (sum0 + sum1) + (sum2 + sum3);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[t & 1]);
+      if (lane == 0) {
+        mbar_arrive(&p_full[x]);
+        if (kDense && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);   // the other group's turn
+      }
       ++r;
     }
 
-    if (kDecode) {
-      if (ok && T > 0) {
-        // every PV has retired (o_done's parity alone cannot tell one pending PV from two)
-        ok = mbar_wait(&fin_bar, 0, status);
-        ok = __all_sync(0xffffffffu, ok);
-      }
-      if (ok) {
-        // partial output of this split: O / l in fp32 and its log-normalizer (empty split: 0, -inf)
-        tc_fence_after();
-        const float inv = T > 0 ? 1.f / l : 0.f;
-        const size_t prow = ((size_t)b * p.Hq + h + rl) * p.num_splits + i;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          if (T > 0) {
-            tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColO + c * 32), o);
-            tmem_wait_ld();
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = 0u;
-          }
-          if (valid) {
-            float4* dst = reinterpret_cast<float4*>(p.o_part + prow * D + c * 32);
-#pragma unroll
-            for (int v = 0; v < 8; ++v)
-              dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
-                                   __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
-          }
-        }
-        if (valid) p.lse_part[prow] = T > 0 ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
-        if (stat_thread) {
-          if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
-          if (p.retained) p.retained[stat_row] = (uint32_t)r;
-          if (p.totals) {
-            atomicAdd(&p.totals[0], (unsigned long long)r);
-            atomicAdd(&p.totals[1], (unsigned long long)T);
-          }
-        }
-      }
-    } else {
-    if (ok) {
-      // finalize: O <- O / l, lse <- m + log l, once every PV has retired (the issuer commits fin_bar
-      // after its last MMA; o_done's parity alone cannot tell one pending PV from two)
+    if (ok && present_x) {
+      // finalize once every PV has retired: O <- O / l, lse <- m + log l
       ok = mbar_wait(&fin_bar, 0, status);
       ok = __all_sync(0xffffffffu, ok);
     }
-    if (ok) {
+    if (ok && present_x) {
       tc_fence_after();
       const float inv = 1.f / l;
       __nv_bfloat16* orow = p.o + (int64_t)b * p.o_sb + (int64_t)row * p.o_sn + (int64_t)h * p.o_sh;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int cc = 0; cc < D / 32; ++cc) {
         uint32_t o[32];
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColO + c * 32), o);
+        tmem_ld_x32(tmem_addr(tb, lane_base, colO + cc * 32), o);
         tmem_wait_ld();
         if (valid) {
 #pragma unroll
@@ -411,7 +386,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
             w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
             w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+            *reinterpret_cast<uint4*>(orow + cc * 32 + v * 8) = w;
           }
         }
       }
@@ -424,7 +399,6 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           atomicAdd(&p.totals[1], (unsigned long long)T);
         }
       }
-    }
     }
   }
 
