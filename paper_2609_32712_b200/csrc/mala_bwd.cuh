@@ -14,13 +14,12 @@
 // Warp roles of the main kernel (768 threads; registers are re-split between the warpgroups):
 //   warp 0       TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
 //   warp 1       UMMA issuer (and, in the MALA kernel, the on-demand dO loads); warps 2-3 idle
-//   warps 4-11   score group: reads S^T, applies Eq. 4 and votes; retained tiles: P^T -> TMEM
-//   warps 12-19  dS group: takes P^T back out of TMEM (so the score buffer can be reused for the next
-//                tile at once), waits for dP^T and forms dS^T in shared memory
-//   warps 20-23  dQ group, one thread per query row of the dQ tile
-// Registers released by warps 0-3 (setmaxnreg) go to the dS and dQ groups.
-// Score and dS groups use two threads per key row (64 query columns each); while the dS group and the
-// tensor pipe finish tile n, the score group already works on tile n+1.
+//   warps 4-19   score group, four threads per key row (32 query columns each): reads S^T once, applies
+//                Eq. 4 and votes; retained tiles: P^T -> TMEM (A operand of dV), then, with P^T still in
+//                registers, dS^T = P^T o (dP^T - D) -> shared memory (operand of dQ and dK)
+//   warps 20-23  dQ group, one thread per query row: takes the whole dQ tile out of TMEM at once (so that
+//                the next dP^T can be issued) and adds it to the global accumulator from shared memory
+// Registers released by warps 0-19 (setmaxnreg) go to the dQ group, which holds a 128-column row.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -74,9 +73,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
 
   __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
-      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free, ds_free, pt_read;
+      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free, ds_free;
   __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
-  __shared__ __align__(16) float dq_ring[2][128];  // D of the retained tiles, for the dS group
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[3];
   __shared__ int dq_info;
@@ -96,12 +94,12 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int s = 0; s < 2; ++s) {
       mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1);
       mbar_init(&do_full[s], 1); mbar_init(&do_empty[s], 1);
-      mbar_init(&vote_bar[s], 8);
+      mbar_init(&vote_bar[s], 16);
     }
-    mbar_init(&s_full, 1); mbar_init(&p_full, 8); mbar_init(&dp_full, 1); mbar_init(&ds_full, 8);
-    mbar_init(&dv_done, 1); mbar_init(&grp_bar, 8); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
+    mbar_init(&s_full, 1); mbar_init(&p_full, 16); mbar_init(&dp_full, 1); mbar_init(&ds_full, 16);
+    mbar_init(&dv_done, 1); mbar_init(&grp_bar, 16); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
     mbar_init(&fin_bar, 1);
-    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1); mbar_init(&ds_free, 1); mbar_init(&pt_read, 8);
+    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1); mbar_init(&ds_free, 1);
     flag[0] = flag[1] = flag[2] = 0;
     dq_info = -1;
     mbar_fence_init();
@@ -115,7 +113,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tb = tmem_base_s;
 
   if (warp < 4) {
-  reg_dealloc<48>();
+  reg_dealloc<40>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -153,7 +151,10 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    // All 32 lanes run this loop with identical values; MMAs, commits, arrivals and TMA loads are issued by
+    // one elected lane.
+    {
+      const uint32_t leader = elect_one();
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);    // S^T, dP^T
       constexpr uint32_t idesc_dv = make_idesc_bf16(128, D, false, true);      // dV (A in TMEM), dK
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);       // dQ
@@ -167,19 +168,19 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint64_t dDOm0 = make_smem_desc(smem_u32(sDO), 16384, 1024);  // dO stage 0 as MN-major B (dV)
       const uint64_t dDSk0 = make_smem_desc(smem_u32(sDS), 16, 1024);     // dS^T stage 0 as K-major A (dK)
       const uint64_t dDSm0 = make_smem_desc(smem_u32(sDS), 16384, 1024);  // dS^T stage 0 as MN-major A (dQ)
-      bool ok = mbar_wait(&kv_full, 0, status);
+      bool ok = mbar_wait_warp(&kv_full, 0, status);
       int r = 0;   // retained tiles so far
       auto issue_qk = [&](int n) -> bool {
         const int s = n & 1;
-        if (!mbar_wait(&q_full[s], (n >> 1) & 1, status)) return false;
+        if (!mbar_wait_warp(&q_full[s], (n >> 1) & 1, status)) return false;
         tc_fence_after();
         const uint64_t dQk = desc_advance(dQk0, s * Cfg::kTileBytes);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-          mma_ss(tmem_addr(tb, 0, Cfg::kColS), desc_advance(dKk, off), desc_advance(dQk, off), idesc_s, k > 0);
+          mma_ss(tmem_addr(tb, 0, Cfg::kColS), desc_advance(dKk, off), desc_advance(dQk, off), idesc_s, k > 0, leader);
         }
-        tc_commit(&s_full);
+        if (leader) tc_commit(&s_full);
         return true;
       };
       if (ok) ok = issue_qk(0);
@@ -187,24 +188,27 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int s = n & 1, hq = hkv * G + n / ni, i = i0 + n % ni;
         bool retain = true;
         if (!kDense) {
-          ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
+          ok = mbar_wait_warp(&vote_bar[n & 1], (n >> 1) & 1, status);
           if (!ok) break;
-          retain = (*(volatile int*)&flag[n % 3]) != 0;
+          retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[n % 3], 0) != 0;
         }
         const int ds = r & 1;   // dO stage
         if (retain) {
           if (!kDense) {
-            ok = mbar_wait(&do_empty[ds], ((r >> 1) & 1) ^ 1, status);
+            ok = mbar_wait_warp(&do_empty[ds], ((r >> 1) & 1) ^ 1, status);
             if (!ok) break;
-            mbar_arrive_expect_tx(&do_full[ds], Cfg::kTileBytes);
-            for (int pn = 0; pn < PAN; ++pn)
-              tma_load_4d(sDO + ds * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[ds], pn * 64, i * 128, hq, b);
+            if (leader) {
+              mbar_arrive_expect_tx(&do_full[ds], Cfg::kTileBytes);
+              for (int pn = 0; pn < PAN; ++pn)
+                tma_load_4d(sDO + ds * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[ds], pn * 64, i * 128, hq, b);
+            }
+            __syncwarp();
           }
           if (r > 0) {   // the dQ tile of the previous retained tile (aliased with dP) has been read out
-            ok = mbar_wait(&dq_empty, (r - 1) & 1, status);
+            ok = mbar_wait_warp(&dq_empty, (r - 1) & 1, status);
             if (!ok) break;
           }
-          ok = mbar_wait(&do_full[ds], (r >> 1) & 1, status);
+          ok = mbar_wait_warp(&do_full[ds], (r >> 1) & 1, status);
           if (!ok) break;
           tc_fence_after();
           const uint64_t dDOk = desc_advance(dDOk0, ds * Cfg::kTileBytes);
@@ -213,24 +217,23 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {   // dP^T = V dO^T
             const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dVk, off), desc_advance(dDOk, off), idesc_s, k > 0);
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dVk, off), desc_advance(dDOk, off), idesc_s, k > 0, leader);
           }
-          tc_commit(&dp_full);
-          ok = mbar_wait(&p_full, r & 1, status);
+          if (leader) tc_commit(&dp_full);
+          ok = mbar_wait_warp(&p_full, r & 1, status);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < 8; ++k)   // dV += P^T dO
-            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + (k >> 2) * 64 + (k & 3) * 8),
-                   desc_advance(dDOm, k * 2048), idesc_dv, k > 0 ? 1u : acc0);
-          tc_commit(&dv_done);
+            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + (k >> 1) * 32 + (k & 1) * 8),
+                   desc_advance(dDOm, k * 2048), idesc_dv, k > 0 ? 1u : acc0, leader);
+          if (leader) tc_commit(&dv_done);
         }
-        // the score buffer is free once dV has been issued and the dS group holds P^T in registers:
+        // the score buffer is free once dV has been issued (the score group keeps P^T in registers):
         // recompute the next tile's scores while dS is being formed
-        if (retain) { ok = mbar_wait(&pt_read, r & 1, status); if (!ok) break; }
         if (n + 1 < n_tot) { ok = issue_qk(n + 1); if (!ok) break; }
         if (retain) {
-          ok = mbar_wait(&ds_full, r & 1, status);
+          ok = mbar_wait_warp(&ds_full, r & 1, status);
           if (!ok) break;
           tc_fence_after();
           const uint64_t dDSk = desc_advance(dDSk0, ds * Cfg::kDsBytes), dDSm = desc_advance(dDSm0, ds * Cfg::kDsBytes);
@@ -239,43 +242,51 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j  (into the dP columns), first: its read-out takes longest
             mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
-                   k > 0);
-          *(volatile int*)&dq_info = n * 2 + ds;
-          mbar_arrive(&dq_info_bar);
-          tc_commit(&dq_full);
+                   k > 0, leader);
+          if (leader) {
+            *(volatile int*)&dq_info = n * 2 + ds;
+            mbar_arrive(&dq_info_bar);
+            tc_commit(&dq_full);
+          }
 #pragma unroll
           for (int k = 0; k < 8; ++k) {   // dK += dS^T Q
             const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
             mma_ss(tmem_addr(tb, 0, Cfg::kColDK), desc_advance(dDSk, off), desc_advance(dQm, k * 2048), idesc_dv,
-                   k > 0 ? 1u : acc1);
+                   k > 0 ? 1u : acc1, leader);
           }
-          tc_commit(&q_empty[s]);
-          tc_commit(&ds_free);   // dS^T has been consumed: the dQ group may stage the dQ tile in that stage
+          if (leader) {
+            tc_commit(&q_empty[s]);
+            tc_commit(&ds_free);   // dS^T has been consumed: the dQ group may stage the dQ tile in that stage
+          }
           ++r;
         } else {
-          mbar_arrive(&q_empty[s]);
+          if (leader) mbar_arrive(&q_empty[s]);
         }
       }
       // tell the dQ group that nothing more will come, then wait for every MMA to retire
+      __syncwarp();
       bool ok2 = true;
-      if (r > 0) ok2 = mbar_wait(&dq_empty, (r - 1) & 1, status);
-      if (ok2) { *(volatile int*)&dq_info = -1; mbar_arrive(&dq_info_bar); }
-      tc_commit(&fin_bar);
-      mbar_wait(&fin_bar, 0, status);
+      if (r > 0) ok2 = mbar_wait_warp(&dq_empty, (r - 1) & 1, status);
+      if (leader) {
+        if (ok2) { *(volatile int*)&dq_info = -1; mbar_arrive(&dq_info_bar); }
+        tc_commit(&fin_bar);
+      }
+      mbar_wait_warp(&fin_bar, 0, status);
       if (!ok && !kDense) {
-        for (int u = (r > 1 ? r - 1 : 0); u <= r; ++u) mbar_wait(&do_full[u & 1], (u >> 1) & 1, status);
+        for (int u = (r > 1 ? r - 1 : 0); u <= r; ++u) mbar_wait_warp(&do_full[u & 1], (u >> 1) & 1, status);
       }
     }
   }
-  } else if (warp < 12) {
+  } else if (warp < 20) {
     // ------------------------------------------------------------------ score group
-    // Two threads per key row: warps 4-7 own query columns 0..63 of the transposed tile, warps 8-11
-    // columns 64..127 (both warps of a pair reach the same TMEM lane quadrant).
-    // Each thread stays inside its own 64 TMEM columns: S^T is read once for the test and once more for
-    // P^T, whose packed columns (hf * 64 + 0..31) overwrite only score columns this thread has consumed.
+    // Four threads per key row: warps 4-7 own query columns 0..31 of the transposed tile, warps 8-11
+    // columns 32..63, and so on (the four warps of a row reach the same TMEM lane quadrant).  A thread
+    // reads its 32 score columns once; P^T (bf16, 16 packed columns) overwrites the first half of the
+    // thread's own score columns, so no thread ever touches a column another thread still has to read.
+    reg_dealloc<72>();
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
-    const int hf = (warp - 4) >> 2;                 // column half
+    const int qt = (warp - 4) >> 2;                 // column quarter
     const bool valid_key = (j * 128 + rl) < p.N;
     const float c2 = p.scale_log2;
     const bool stat_thread = (warp == 4 && lane == 0);
@@ -289,8 +300,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
       return ((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128 + rl;
     };
-    // per-query vectors of tile 0 into slot 0 (published by the first column half), then a group sync
-    if (hf == 0) {
+    // per-query vectors of tile 0 into slot 0 (published by the first column quarter), then a group sync
+    if (qt == 0) {
       const size_t x = vec_index(0);
       vec[0][0][rl] = p.lse2[x];
       vec[0][1][rl] = p.bq[x];
@@ -306,7 +317,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int slot = n % 3;
       // prefetch the per-query vectors of the next tile
       float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
-      if (hf == 0 && n + 1 < n_tot) {
+      if (qt == 0 && n + 1 < n_tot) {
         const size_t x = vec_index(n + 1);
         nx0 = p.lse2[x]; nx1 = p.bq[x]; nx2 = p.Dq[x];
       }
@@ -314,33 +325,29 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const bool diag = p.causal && i == j;   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
-      const uint32_t ninf = 0xff800000u;
-      // pass 1 (MALA only), Eq. 4: skip iff s - lse_q < log(tau / L_q) on every valid entry
+      uint32_t sc[32];
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + qt * 32), sc);
+      tmem_wait_ld();
+      if (p.causal && i == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
+        const uint32_t ninf = 0xff800000u;
+        const int c0 = qt * 32;
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (c0 + e < rl) sc[e] = ninf;
+      }
+      // Eq. 4 (MALA only): skip iff s - lse_q < log(tau / L_q) on every valid entry
       float crit = -INFINITY;
       if (!kDense) {
-        const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]) + hf * 16;
+        const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]) + qt * 8;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t sc[32];
-          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + c * 32), sc);
-          tmem_wait_ld();
-          if (diag) {
-            const int c0 = hf * 64 + c * 32;
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (c0 + e < rl) sc[e] = ninf;
-          }
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const float4 x0 = bb[c * 8 + e];
-            crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y)),
-                                     fmaxf(fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w))));
-          }
+        for (int e = 0; e < 8; ++e) {
+          const float4 x0 = bb[e];
+          crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y)),
+                                   fmaxf(fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w))));
         }
       }
       // publish the next tile's vectors (slot (n+1) % 3 was last read two tiles ago)
-      if (hf == 0) {
+      if (qt == 0) {
         const int ns = (n + 1) % 3;
         vec[ns][0][rl] = nx0; vec[ns][1][rl] = nx1; vec[ns][2][rl] = nx2;
       }
@@ -373,24 +380,13 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             bm_bits |= 1u << (i & 31);
           }
         }
-        // D of this tile's queries for the dS group (which may lag behind by more than the vector slots)
-        if (hf == 0) dq_ring[r & 1][rl] = vec[slot][2][rl];
-        // pass 2: P^T = exp2(s * c2 - lse2_q) (bf16), written over S^T in TMEM as the A operand of dV
-        const float4* ll = reinterpret_cast<const float4*>(vec[slot][0]) + hf * 16;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t sc[32], pk[16];
-          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + c * 32), sc);
-          tmem_wait_ld();
-          if (diag) {
-            const int c0 = hf * 64 + c * 32;
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (c0 + e < rl) sc[e] = ninf;
-          }
+        // P^T = exp2(s * c2 - lse2_q) (bf16), written over S^T in TMEM as the A operand of dV
+        uint32_t pk[16];
+        {
+          const float4* ll = reinterpret_cast<const float4*>(vec[slot][0]) + qt * 8;
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            const float4 x = ll[c * 8 + e];
+            const float4 x = ll[e];
             const float p0 = fast_exp2(fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x.x));
             const float p1 = fast_exp2(fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x.y));
             const float p2 = fast_exp2(fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x.z));
@@ -398,12 +394,48 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             pk[2 * e] = pack_bf16x2(p0, p1);
             pk[2 * e + 1] = pack_bf16x2(p2, p3);
           }
-          tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + c * 16), pk);
         }
+        tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + qt * 32), pk);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full);
+        // dS^T = P^T o (dP^T - D_q): values first, then, once dV has also finished reading the dO stage that
+        // dS^T overwrites (D = 128), into shared memory for the dQ and dK MMAs
+        ok = mbar_wait(&dp_full, r & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t w[16];
+        {
+          uint32_t dp[32];
+          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + qt * 32), dp);
+          tmem_wait_ld();
+          const float4* dd = reinterpret_cast<const float4*>(vec[slot][2]) + qt * 8;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float4 x = dd[e];
+            const uint32_t pa = pk[2 * e], pb = pk[2 * e + 1];
+            const float p0 = __uint_as_float(pa << 16), p1 = __uint_as_float(pa & 0xffff0000u);
+            const float p2 = __uint_as_float(pb << 16), p3 = __uint_as_float(pb & 0xffff0000u);
+            w[2 * e] = pack_bf16x2(p0 * (__uint_as_float(dp[4 * e + 0]) - x.x), p1 * (__uint_as_float(dp[4 * e + 1]) - x.y));
+            w[2 * e + 1] = pack_bf16x2(p2 * (__uint_as_float(dp[4 * e + 2]) - x.z), p3 * (__uint_as_float(dp[4 * e + 3]) - x.w));
+          }
+        }
+        ok = mbar_wait(&dv_done, r & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        {
+          uint8_t* dst = sDS + (r & 1) * Cfg::kDsBytes + (qt >> 1) * 16384;
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            *reinterpret_cast<uint4*>(dst + sw128_offset((uint32_t)rl, (uint32_t)((qt & 1) * 32 + v * 8))) =
+                make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ds_full);
         ++r;
       }
       if (stat_thread && (n % ni == ni - 1)) {   // last tile of this query head
@@ -417,7 +449,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
     }
 
-    // epilogue: dK_j (x scale), dV_j -> global; each thread of a pair stores half of the columns of its row
+    // epilogue: dK_j (x scale), dV_j -> global; the four threads of a row store a quarter of its columns each
     if (ok) {
       ok = mbar_wait(&fin_bar, 0, status);
       ok = __all_sync(0xffffffffu, ok);
@@ -432,9 +464,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         __nv_bfloat16* out = which ? dkrow : dvrow;
         const float f = which ? p.scale : 1.f;
         const uint32_t col0 = which ? Cfg::kColDK : Cfg::kColDV;
-#pragma unroll
-        for (int cc = 0; cc < D / 64; ++cc) {
-          const int c = hf * (D / 64) + cc;
+        if (qt < D / 32) {   // warp-uniform: D = 64 has two 32-column chunks, taken by the first two quarters
+          const int c = qt;
           uint32_t o[32];
           if (r > 0) {
             tmem_ld_x32(tmem_addr(tb, lane_base, col0 + c * 32), o);
@@ -457,78 +488,13 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
       }
     }
-  } else if (warp < 20) {
-    // ------------------------------------------------------------------ dS group
-    // Per retained tile: P^T (bf16, this thread's 64 query columns) back out of TMEM, then
-    // dS^T = P^T o (dP^T - D_q) as bf16 into the tile's dS^T stage for the dK and dQ MMAs.
-    reg_alloc<88>();
-    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
-    const int rl = (int)lane_base + lane;
-    const int hf = (warp - 12) >> 2;
-    for (int r = 0;; ++r) {
-      // the issuer's final commit ends the loop: no retained tile follows
-      bool ok = mbar_wait_either(&p_full, r & 1, &fin_bar, 0, status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      if (!mbar_try_wait(&p_full, r & 1)) break;   // woken by fin_bar
-      tc_fence_after();
-      uint32_t pk[32];
-      {
-        uint32_t t0[16], t1[16];
-        tmem_ld_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 0), t0);
-        tmem_ld_x16(tmem_addr(tb, lane_base, Cfg::kColS + hf * 64 + 16), t1);
-        tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 16; ++e) { pk[e] = t0[e]; pk[16 + e] = t1[e]; }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&pt_read);        // the score buffer may be overwritten
-      // dS^T goes where this tile's dO lies (D = 128): wait until dP and dV have consumed it
-      ok = mbar_wait(&dp_full, r & 1, status);
-      if (ok) ok = mbar_wait(&dv_done, r & 1, status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      const float4* dd = reinterpret_cast<const float4*>(dq_ring[r & 1]) + hf * 16;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t dp[32];
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + hf * 64 + c * 32), dp);
-        tmem_wait_ld();
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          uint32_t w[4];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const float4 x = dd[c * 8 + v * 2 + u];
-            const uint32_t pa = pk[c * 16 + v * 4 + 2 * u], pb = pk[c * 16 + v * 4 + 2 * u + 1];
-            const float p0 = __uint_as_float(pa << 16), p1 = __uint_as_float(pa & 0xffff0000u);
-            const float p2 = __uint_as_float(pb << 16), p3 = __uint_as_float(pb & 0xffff0000u);
-            const float d0 = p0 * (__uint_as_float(dp[v * 8 + u * 4 + 0]) - x.x);
-            const float d1 = p1 * (__uint_as_float(dp[v * 8 + u * 4 + 1]) - x.y);
-            const float d2 = p2 * (__uint_as_float(dp[v * 8 + u * 4 + 2]) - x.z);
-            const float d3 = p3 * (__uint_as_float(dp[v * 8 + u * 4 + 3]) - x.w);
-            w[2 * u] = pack_bf16x2(d0, d1);
-            w[2 * u + 1] = pack_bf16x2(d2, d3);
-          }
-          const uint32_t col = (uint32_t)(c * 32 + v * 8);
-          *reinterpret_cast<uint4*>(sDS + (r & 1) * Cfg::kDsBytes + hf * 16384 + sw128_offset((uint32_t)rl, col)) =
-              make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-      fence_proxy_async_smem();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ds_full);
-    }
   } else {
     // ------------------------------------------------------------------ dQ group: thread = query row
-    // Each retained tile's dQ (fp32, 128 x D) is read out of TMEM 64 columns at a time, staged as two
-    // 32-column swizzled panels in the tile's dS^T stage -- free once dK has retired -- and added to the
-    // global accumulator by TMA reduce-add.  The dP / dQ columns are released as soon as the last
-    // columns are in registers; the stage goes back to the dO ring when the TMA has read it.
-    reg_alloc<88>();
+    // Each retained tile's dQ (fp32, 128 x D) is taken out of TMEM in one go and the dP / dQ columns are
+    // released at once.  The row is then staged, 64 columns at a time, as two 32-column swizzled panels in
+    // the tile's dS^T stage -- free once dK has retired -- and added to the global accumulator by TMA
+    // reduce-add; the stage goes back to the dO ring when the TMA has read it.
+    reg_alloc<152>();
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const bool elected = (warp == 20 && lane == 0);
@@ -548,22 +514,18 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
       const int row0 = (int)(((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128);
       uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // two 16 KB panels
+      uint32_t a[D / 32][32];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + c * 32), a[c]);
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&dq_empty);       // TMEM columns may be reused by the next dP
+      ok = mbar_wait(&ds_free, k & 1, status);     // dK has consumed dS^T: its stage may be overwritten
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
 #pragma unroll
       for (int round = 0; round < D / 64; ++round) {
-        uint32_t a0[32], a1[32];
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + round * 64 + 0), a0);
-        tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + round * 64 + 32), a1);
-        tmem_wait_ld();
-        if (round == D / 64 - 1) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&dq_empty);   // TMEM columns may be reused by the next dP
-        }
-        if (round == 0) {  // dK has consumed dS^T: its stage may be overwritten
-          ok = mbar_wait(&ds_free, k & 1, status);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
         if (round > 0) {   // the panels are still being read by the previous round's reduce
           if (elected) { bulk_wait_read_all(); mbar_arrive(&stg_free); }
           ok = mbar_wait(&stg_free, free_phase & 1, status);
@@ -574,8 +536,10 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
         for (int v = 0; v < 8; ++v) {
           const uint32_t off = rl * 128 + ((v ^ (rl & 7)) << 4);
-          *reinterpret_cast<uint4*>(stg + off) = make_uint4(a0[4 * v], a0[4 * v + 1], a0[4 * v + 2], a0[4 * v + 3]);
-          *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a1[4 * v], a1[4 * v + 1], a1[4 * v + 2], a1[4 * v + 3]);
+          *reinterpret_cast<uint4*>(stg + off) =
+              make_uint4(a[2 * round][4 * v], a[2 * round][4 * v + 1], a[2 * round][4 * v + 2], a[2 * round][4 * v + 3]);
+          *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a[2 * round + 1][4 * v], a[2 * round + 1][4 * v + 1],
+                                                                    a[2 * round + 1][4 * v + 2], a[2 * round + 1][4 * v + 3]);
         }
         fence_proxy_async_smem();
         __syncwarp();

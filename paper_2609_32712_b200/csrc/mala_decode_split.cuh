@@ -131,7 +131,9 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer (+ on-demand V loads)
-    if (lane == 0) {
+    // All 32 lanes run this loop with identical values; MMAs, commits and TMA loads are issued by one elected lane.
+    {
+      const uint32_t leader = elect_one();
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, false, true);
       const uint64_t dQ0 = make_smem_desc(smem_u32(sQ), 16, 1024);
@@ -161,20 +163,22 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       auto issue_qk = [&](const Cur& c, int gq) -> bool {
         const int ip = c.ne & 1;
         if (q_seen < c.ne) {
-          if (!mbar_wait(&q_full[ip], (c.ne >> 1) & 1, status)) return false;
+          if (!mbar_wait_warp(&q_full[ip], (c.ne >> 1) & 1, status)) return false;
           q_seen = c.ne;
         }
-        if (!mbar_wait(&k_full[kc], kpar, status)) return false;
+        if (!mbar_wait_warp(&k_full[kc], kpar, status)) return false;
         tc_fence_after();
         const uint32_t dS = tmem_addr(tb, 0, (gq & 1) * 128);
         const uint64_t dQ = desc_advance(dQ0, ip * DecCfg::kQBytes), dK = desc_advance(dK0, kc * TB);
 #pragma unroll
         for (int k = 0; k < 8; ++k)   // Q panels lie 2 KB apart, K panels 16 KB
           mma_ss(dS, desc_advance(dQ, (k >> 2) * 2048 + (k & 3) * 32), desc_advance(dK, (k >> 2) * 16384 + (k & 3) * 32),
-                 idesc_qk, k > 0);
-        tc_commit(&k_empty[kc]);
-        tc_commit(&s_full[gq & 1]);
-        if (c.t == c.T - 1) tc_commit(&q_empty[ip]);   // last QK of the item: its Q stage may be refilled
+                 idesc_qk, k > 0, leader);
+        if (leader) {
+          tc_commit(&k_empty[kc]);
+          tc_commit(&s_full[gq & 1]);
+          if (c.t == c.T - 1) tc_commit(&q_empty[ip]);   // last QK of the item: its Q stage may be refilled
+        }
         if (++kc == KS) { kc = 0; kpar ^= 1; }
         return true;
       };
@@ -188,27 +192,30 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         if (nxt.valid) { ok = issue_qk(nxt, g + 1); if (!ok) break; }
         bool retain = true;
         if (!kDense) {
-          ok = mbar_wait(&vote_bar[g & 1], (g >> 1) & 1, status);
+          ok = mbar_wait_warp(&vote_bar[g & 1], (g >> 1) & 1, status);
           if (!ok) break;
-          retain = (*(volatile int*)&flag[g % 3]) != 0;
+          retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[g % 3], 0) != 0;
           if (retain) {   // V of this tile, on demand
-            ok = mbar_wait(&v_empty[vi], vipar, status);
+            ok = mbar_wait_warp(&v_empty[vi], vipar, status);
             if (!ok) break;
-            mbar_arrive_expect_tx(&v_full[vi], TB);
-            tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, (cur.j0 - cur.t) * 128, cur.hkv, cur.b);
-            tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, (cur.j0 - cur.t) * 128, cur.hkv, cur.b);
+            if (leader) {
+              mbar_arrive_expect_tx(&v_full[vi], TB);
+              tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, (cur.j0 - cur.t) * 128, cur.hkv, cur.b);
+              tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, (cur.j0 - cur.t) * 128, cur.hkv, cur.b);
+            }
+            __syncwarp();
             if (++vi == VS) { vi = 0; vipar ^= 1; }
           }
         }
         const int ip = cur.ne & 1;
         if (retain) {
-          ok = mbar_wait(&p_full[g & 1], ppar[g & 1], status);
+          ok = mbar_wait_warp(&p_full[g & 1], ppar[g & 1], status);
           if (!ok) break;
           ppar[g & 1] ^= 1;
-          ok = mbar_wait(&v_full[vc], vcpar, status);
+          ok = mbar_wait_warp(&v_full[vc], vcpar, status);
           if (!ok) break;
           if (r_item == 0 && cur.ne >= 2) {   // the softmax warp has read this accumulator's previous item
-            ok = mbar_wait(&o_free[ip], ((cur.ne >> 1) - 1) & 1, status);
+            ok = mbar_wait_warp(&o_free[ip], ((cur.ne >> 1) - 1) & 1, status);
             if (!ok) break;
           }
           tc_fence_after();
@@ -216,18 +223,18 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           const uint64_t dV = desc_advance(dV0, vc * TB);
           const uint32_t acc0 = r_item > 0 ? 1u : 0u;
 #pragma unroll
-          for (int k = 0; k < 8; ++k) mma_ts(dO, aP + k * 8, desc_advance(dV, k * 2048), idesc_pv, k > 0 ? 1u : acc0);
-          tc_commit(&v_empty[vc]);
-          tc_commit(&o_done);
+          for (int k = 0; k < 8; ++k) mma_ts(dO, aP + k * 8, desc_advance(dV, k * 2048), idesc_pv, k > 0 ? 1u : acc0, leader);
+          if (leader) { tc_commit(&v_empty[vc]); tc_commit(&o_done); }
           if (++vc == VS) { vc = 0; vcpar ^= 1; }
           ++r_item;
         }
-        if (cur.t == cur.T - 1) { tc_commit(&item_done[ip]); r_item = 0; }
+        if (cur.t == cur.T - 1) { if (leader) tc_commit(&item_done[ip]); r_item = 0; }
         cur = nxt;
         ++g;
       }
-      tc_commit(&fin_bar);
-      mbar_wait(&fin_bar, 0, status);
+      __syncwarp();
+      if (leader) tc_commit(&fin_bar);
+      mbar_wait_warp(&fin_bar, 0, status);
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
     }
   } else if (warp == 4) {

@@ -137,8 +137,11 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   } else if (warp == 1 || warp == 2) {
     // ------------------------------------------------------------------ UMMA issuer of block x (+ its V loads)
+    // All 32 lanes run this loop with identical values; MMAs, commits, arrivals and TMA loads are issued by
+    // one elected lane.
     const int x = warp - 1;
-    if (lane == 0) {
+    {
+      const uint32_t leader = elect_one();
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
       constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, false, true);
       const bool present_x = (x == 0) || hasB;
@@ -147,19 +150,19 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint64_t dK0 = make_smem_desc(smem_u32(sK), 16, 1024);
       const uint64_t dV0 = make_smem_desc(smem_u32(sV), 16384, 1024);
       const uint32_t tS = tmem_addr(tb, 0, x * 128), tO = tmem_addr(tb, 0, 256 + x * 128);
-      bool ok = mbar_wait(&q_full, 0, status);
+      bool ok = mbar_wait_warp(&q_full, 0, status);
       int r = 0;                       // PVs issued (retained tiles); also counts this block's V loads
       int s = 0;                       // K stage of step u
       uint32_t kpar = 0;               // parity of k_full[s] for step u
       for (int u = 0; u < U && ok; ++u) {
-        ok = mbar_wait(&k_full[s], kpar, status);
+        ok = mbar_wait_warp(&k_full[s], kpar, status);
         if (!ok) break;
         if (!present_x || u < first) {
-          mbar_arrive(&k_empty[s]);    // this block has no tile at this step
+          if (leader) mbar_arrive(&k_empty[s]);    // this block has no tile at this step
           if (kDense) {                // release the shared V stage too, paced by its arrival
-            ok = mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
+            ok = mbar_wait_warp(&v_full[u & 1], (u >> 1) & 1, status);
             if (!ok) break;
-            mbar_arrive(&v_empty[u & 1]);
+            if (leader) mbar_arrive(&v_empty[u & 1]);
           }
         } else {
           const int t = u - first;     // tile index of this block
@@ -168,15 +171,14 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
             const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0);
+            mma_ss(tS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0, leader);
           }
-          tc_commit(&k_empty[s]);
-          tc_commit(&s_full[x]);
+          if (leader) { tc_commit(&k_empty[s]); tc_commit(&s_full[x]); }
           bool retain = true;
           if (!kDense) {
-            ok = mbar_wait(&vote_bar[x], t & 1, status);
+            ok = mbar_wait_warp(&vote_bar[x], t & 1, status);
             if (!ok) break;
-            retain = (*(volatile int*)&flag[x][t % 3]) != 0;
+            retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[x][t % 3], 0) != 0;
           }
           if (retain) {
             // MALA: V is loaded on demand into this block's own stage (free once its previous PV retired);
@@ -184,31 +186,35 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const int vs = kDense ? (u & 1) : x;
             const uint32_t vpar = kDense ? ((u >> 1) & 1) : (r & 1);
             if (!kDense) {
-              ok = mbar_wait(&v_empty[x], (r & 1) ^ 1, status);
+              ok = mbar_wait_warp(&v_empty[x], (r & 1) ^ 1, status);
               if (!ok) break;
-              mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
-              for (int pn = 0; pn < PAN; ++pn)
-                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, (j0 - u) * 128, hkv, b);
+              if (leader) {
+                mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
+                for (int pn = 0; pn < PAN; ++pn)
+                  tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, (j0 - u) * 128, hkv, b);
+              }
+              __syncwarp();
             }
-            ok = mbar_wait(&p_full[x], r & 1, status);
-            if (ok) ok = mbar_wait(&v_full[vs], vpar, status);
+            ok = mbar_wait_warp(&p_full[x], r & 1, status);
+            if (ok) ok = mbar_wait_warp(&v_full[vs], vpar, status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t acc0 = r > 0 ? 1u : 0u;
             const uint64_t dVs = desc_advance(dV0, vs * Cfg::kTileBytes);
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-              mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, k > 0 ? 1u : acc0);
-            tc_commit(&v_empty[vs]);
+              mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, k > 0 ? 1u : acc0, leader);
+            if (leader) tc_commit(&v_empty[vs]);
             ++r;
           }
         }
         if (++s == KS) { s = 0; kpar ^= 1; }
       }
       // every MMA of this block has retired (and every V copy landed) before the CTA may exit
-      tc_commit(&fin_bar);
-      mbar_wait(&fin_bar, 0, status);
-      if (!kDense && !ok && r > 0) mbar_wait(&v_full[x], (r - 1) & 1, status);
+      __syncwarp();
+      if (leader) tc_commit(&fin_bar);
+      mbar_wait_warp(&fin_bar, 0, status);
+      if (!kDense && !ok && r > 0) mbar_wait_warp(&v_full[x], (r - 1) & 1, status);
     }
   }
   } else {
