@@ -8,8 +8,16 @@
 //                           lse (Eq. 4).  Only retained tiles load dO and run dP^T = V dO^T, P^T,
 //                           dS^T = P^T o (dP^T - D), dV += P^T dO, dK += dS^T Q, dQ_i += dS K_j.
 //                           dK, dV accumulate in TMEM; dQ tiles are added to an fp32 accumulator in
-//                           global memory by TMA reduce-add from shared memory.
-//   bwd_convert_dq_kernel : dq = bf16(scale * accumulator).
+//                           global memory, one half of the columns by vector reductions from registers
+//                           (red.global.add.v4.f32), the other half by TMA reduce-add from shared memory.
+//                           Either path alone is slower: an SM sustains about 25 B/clk of reductions, the
+//                           TMA path is starved of shared-memory bandwidth while SS MMAs run, and its source
+//                           buffer (32 KB, the tile's dS^T stage) is held until the reduction has read it.
+//                           Accumulator layout, per 128 x D tile (b, head, query block), D / 2 = h:
+//                             columns 0..h-1  : float (c / 4) * 512 + r * 4 + c % 4  (the 32 rows of a warp
+//                                               are 512 contiguous bytes of one column group)
+//                             columns h..D-1  : row-major [128][h] after those 128 * h floats
+//   bwd_convert_dq_kernel : dq = bf16(scale * accumulator), back in row-major order.
 //
 // Warp roles of the main kernel (768 threads; registers are re-split between the warpgroups):
 //   warp 0       TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
@@ -73,7 +81,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
 
   __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
-      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, stg_free, ds_free;
+      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, ds_free;
   __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[3];
@@ -99,7 +107,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_init(&s_full, 1); mbar_init(&p_full, 16); mbar_init(&dp_full, 1); mbar_init(&ds_full, 16);
     mbar_init(&dv_done, 1); mbar_init(&grp_bar, 16); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
     mbar_init(&fin_bar, 1);
-    mbar_init(&stg_full, 4); mbar_init(&stg_free, 1); mbar_init(&ds_free, 1);
+    mbar_init(&stg_full, 4); mbar_init(&ds_free, 1);
     flag[0] = flag[1] = flag[2] = 0;
     dq_info = -1;
     mbar_fence_init();
@@ -166,7 +174,6 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint64_t dQm0 = make_smem_desc(smem_u32(sQ), 16384, 1024);    // Q stage 0 as MN-major B (dK)
       const uint64_t dDOk0 = make_smem_desc(smem_u32(sDO), 16, 1024);     // dO stage 0 as K-major B (dP^T)
       const uint64_t dDOm0 = make_smem_desc(smem_u32(sDO), 16384, 1024);  // dO stage 0 as MN-major B (dV)
-      const uint64_t dDSk0 = make_smem_desc(smem_u32(sDS), 16, 1024);     // dS^T stage 0 as K-major A (dK)
       const uint64_t dDSm0 = make_smem_desc(smem_u32(sDS), 16384, 1024);  // dS^T stage 0 as MN-major A (dQ)
       bool ok = mbar_wait_warp(&kv_full, 0, status);
       int r = 0;   // retained tiles so far
@@ -236,26 +243,22 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           ok = mbar_wait_warp(&ds_full, r & 1, status);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t dDSk = desc_advance(dDSk0, ds * Cfg::kDsBytes), dDSm = desc_advance(dDSm0, ds * Cfg::kDsBytes);
+          const uint64_t dDSm = desc_advance(dDSm0, ds * Cfg::kDsBytes);
           const uint64_t dQm = desc_advance(dQm0, s * Cfg::kTileBytes);
           const uint32_t acc1 = r > 0 ? 1u : 0u;
 #pragma unroll
-          for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j  (into the dP columns), first: its read-out takes longest
+          for (int k = 0; k < 8; ++k)     // dK += dS^T Q, dS^T read from TMEM (the dP columns)
+            mma_ts(tmem_addr(tb, 0, Cfg::kColDK), tmem_addr(tb, 0, Cfg::kColDP + (k >> 1) * 32 + (k & 1) * 8),
+                   desc_advance(dQm, k * 2048), idesc_dv, k > 0 ? 1u : acc1, leader);
+          if (leader) tc_commit(&q_empty[s]);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j, into the dP columns (after dK has read dS^T from them)
             mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
                    k > 0, leader);
           if (leader) {
             *(volatile int*)&dq_info = n * 2 + ds;
             mbar_arrive(&dq_info_bar);
             tc_commit(&dq_full);
-          }
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {   // dK += dS^T Q
-            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tmem_addr(tb, 0, Cfg::kColDK), desc_advance(dDSk, off), desc_advance(dQm, k * 2048), idesc_dv,
-                   k > 0 ? 1u : acc1, leader);
-          }
-          if (leader) {
-            tc_commit(&q_empty[s]);
             tc_commit(&ds_free);   // dS^T has been consumed: the dQ group may stage the dQ tile in that stage
           }
           ++r;
@@ -422,6 +425,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             w[2 * e + 1] = pack_bf16x2(p2 * (__uint_as_float(dp[4 * e + 2]) - x.z), p3 * (__uint_as_float(dp[4 * e + 3]) - x.w));
           }
         }
+        // dS^T also goes to TMEM, over this thread's own (already consumed) dP^T columns: A operand of dK
+        tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColDP + qt * 32), w);
         ok = mbar_wait(&dv_done, r & 1, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -433,6 +438,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
         }
         fence_proxy_async_smem();
+        tmem_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&ds_full);
@@ -491,14 +497,14 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   } else {
     // ------------------------------------------------------------------ dQ group: thread = query row
     // Each retained tile's dQ (fp32, 128 x D) is taken out of TMEM in one go and the dP / dQ columns are
-    // released at once.  The row is then staged, 64 columns at a time, as two 32-column swizzled panels in
-    // the tile's dS^T stage -- free once dK has retired -- and added to the global accumulator by TMA
-    // reduce-add; the stage goes back to the dO ring when the TMA has read it.
+    // released at once.  The first D / 2 columns go to the global accumulator by vector reductions from
+    // registers; the others are staged as 32-column swizzled panels in the tile's dS^T stage -- free once
+    // dQ has retired -- and added by TMA reduce-add; the stage goes back to the dO ring when the TMA has
+    // read it.
     reg_alloc<152>();
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const bool elected = (warp == 20 && lane == 0);
-    uint32_t full_phase = 0, free_phase = 0;
     if (elected) tma_prefetch_desc(&tmAcc);
     for (int k = 0;; ++k) {
       bool ok = mbar_wait(&dq_info_bar, k & 1, status);
@@ -512,8 +518,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
-      const int row0 = (int)(((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128);
-      uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // two 16 KB panels
+      const int tile = (int)(((size_t)b * p.Hq + hq) * p.T + (size_t)i);
+      uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // D / 64 panels of 16 KB
       uint32_t a[D / 32][32];
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + c * 32), a[c]);
@@ -521,43 +527,40 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&dq_empty);       // TMEM columns may be reused by the next dP
-      ok = mbar_wait(&ds_free, k & 1, status);     // dK has consumed dS^T: its stage may be overwritten
+      {
+        float* acc = p.dq_acc + (size_t)tile * (128 * D) + rl * 4;
+#pragma unroll
+        for (int c = 0; c < D / 64; ++c)
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            red_add_v4(acc + (c * 8 + v) * 512, a[c][4 * v], a[c][4 * v + 1], a[c][4 * v + 2], a[c][4 * v + 3]);
+      }
+      ok = mbar_wait(&ds_free, k & 1, status);     // dQ and dK have consumed dS^T: its stage may be overwritten
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
 #pragma unroll
-      for (int round = 0; round < D / 64; ++round) {
-        if (round > 0) {   // the panels are still being read by the previous round's reduce
-          if (elected) { bulk_wait_read_all(); mbar_arrive(&stg_free); }
-          ok = mbar_wait(&stg_free, free_phase & 1, status);
-          ok = __all_sync(0xffffffffu, ok);
-          ++free_phase;
-          if (!ok) break;
-        }
+      for (int c = D / 64; c < D / 32; ++c) {
+        uint8_t* pan = stg + (c - D / 64) * 16384;
 #pragma unroll
-        for (int v = 0; v < 8; ++v) {
-          const uint32_t off = rl * 128 + ((v ^ (rl & 7)) << 4);
-          *reinterpret_cast<uint4*>(stg + off) =
-              make_uint4(a[2 * round][4 * v], a[2 * round][4 * v + 1], a[2 * round][4 * v + 2], a[2 * round][4 * v + 3]);
-          *reinterpret_cast<uint4*>(stg + 16384 + off) = make_uint4(a[2 * round + 1][4 * v], a[2 * round + 1][4 * v + 1],
-                                                                    a[2 * round + 1][4 * v + 2], a[2 * round + 1][4 * v + 3]);
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&stg_full);
-        if (elected) {
-          ok = mbar_wait(&stg_full, full_phase & 1, status);
-          if (ok) {
-            tma_reduce_add_2d(&tmAcc, stg, round * 64, row0);
-            tma_reduce_add_2d(&tmAcc, stg + 16384, round * 64 + 32, row0);
-            bulk_commit_group();
-          }
-        }
-        ++full_phase;
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        for (int v = 0; v < 8; ++v)
+          *reinterpret_cast<uint4*>(pan + rl * 128 + ((v ^ (rl & 7)) << 4)) =
+              make_uint4(a[c][4 * v], a[c][4 * v + 1], a[c][4 * v + 2], a[c][4 * v + 3]);
       }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&stg_full);
+      if (elected) {
+        ok = mbar_wait(&stg_full, k & 1, status);
+        if (ok) {
+#pragma unroll
+          for (int c = 0; c < D / 64; ++c) tma_reduce_add_3d(&tmAcc, stg + c * 16384, c * 32, 0, tile);
+          bulk_commit_group();
+          bulk_wait_read_all();
+        }
+        mbar_arrive(&do_empty[ds]);                // stage back to the dO ring
+      }
+      ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      if (elected) { bulk_wait_read_all(); mbar_arrive(&do_empty[ds]); }   // stage back to the dO ring
     }
     if (elected) bulk_wait_all();
   }
@@ -604,25 +607,41 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
   }
 }
 
-// dq = bf16(scale * acc); one thread per 8 output elements
+// dq = bf16(scale * acc); one thread per 8 output elements.  The accumulator is tiled (see the file header):
+// consecutive threads take consecutive rows of a tile.
 __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int64_t sb,
                                       int64_t sn, int64_t sh, int B, int Hq, int N, int Np, int d, float scale) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = d / 8;
-  const long long total = (long long)B * Hq * N * per_row;
+  const long long total = (long long)B * Hq * Np * per_row;
   if (idx >= total) return;
-  const int c = (int)(idx % per_row) * 8;
-  const int row = (int)((idx / per_row) % N);
-  const int h = (int)((idx / ((long long)per_row * N)) % Hq);
-  const int b = (int)(idx / ((long long)per_row * N * Hq));
-  const float4* src = reinterpret_cast<const float4*>(acc + (((size_t)b * Hq + h) * Np + row) * d + c);
-  const float4 x = src[0], y = src[1];
+  const int r = (int)(idx % 128);
+  const int cg = (int)((idx / 128) % per_row);             // columns 8 cg .. 8 cg + 7
+  const long long tile = idx / (128LL * per_row);          // (b * Hq + h) * (Np / 128) + i
+  const int T = Np / 128;
+  const int i = (int)(tile % T);
+  const int h = (int)((tile / T) % Hq);
+  const int b = (int)(tile / ((long long)T * Hq));
+  const int row = i * 128 + r;
+  if (row >= N) return;
+  const int half = d / 2;
+  const float* base = acc + (size_t)tile * 128 * d;
+  float4 x, y;
+  if (cg * 8 < half) {
+    const float* src = base + (size_t)(2 * cg) * 512 + r * 4;
+    x = *reinterpret_cast<const float4*>(src);
+    y = *reinterpret_cast<const float4*>(src + 512);
+  } else {
+    const float* src = base + (size_t)128 * half + (size_t)r * half + (cg * 8 - half);
+    x = *reinterpret_cast<const float4*>(src);
+    y = *reinterpret_cast<const float4*>(src + 4);
+  }
   uint4 w;
   w.x = pack_bf16x2(x.x * scale, x.y * scale);
   w.y = pack_bf16x2(x.z * scale, x.w * scale);
   w.z = pack_bf16x2(y.x * scale, y.y * scale);
   w.w = pack_bf16x2(y.z * scale, y.w * scale);
-  *reinterpret_cast<uint4*>(dq + b * sb + row * sn + h * sh + c) = w;
+  *reinterpret_cast<uint4*>(dq + b * sb + row * sn + h * sh + cg * 8) = w;
 }
 
 inline size_t bwd_align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -662,7 +681,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   float* Dq = (float*)(w + 2 * vbytes);
 
   CUtensorMap tq, tk, tv, tdo, tacc;
-  if (!make_tensor_map_f32_rows(&tacc, acc, (uint64_t)B * Hq * Np, d, 128) ||
+  if (!make_tensor_map_f32_tiles(&tacc, acc + 64 * d, (uint64_t)B * Hq * T, d / 2, (uint64_t)128 * d * sizeof(float)) ||
       !make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
       !make_tensor_map_bnhd(&tk, k.p, B, N, Hkv, d, k.sb, k.sn, k.sh, 128) ||
       !make_tensor_map_bnhd(&tv, v.p, B, N, Hkv, d, v.sb, v.sn, v.sh, 128) ||
@@ -700,7 +719,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   else rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, tacc, p, stream);
   if (rc != MALA_OK) return rc;
   {
-    const long long total = (long long)B * Hq * N * (d / 8);
+    const long long total = (long long)B * Hq * Np * (d / 8);
     const unsigned blocks = (unsigned)((total + 255) / 256);
     bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(acc, (__nv_bfloat16*)dq.p, dq.sb, dq.sn, dq.sh, B, Hq, N, Np, d,
                                                       scale);

@@ -44,16 +44,18 @@ inline bool make_tensor_map_bnhd(CUtensorMap* out, const void* base, int B, int 
   return r == CUDA_SUCCESS;
 }
 
-// Tensor map over a row-major fp32 matrix [rows, cols]: coordinates (col, row), box = 32 columns x
-// box_rows rows (128 bytes wide), 128-byte swizzle.  Used for TMA reduce-add of fp32 tiles.
-inline bool make_tensor_map_f32_rows(CUtensorMap* out, const void* base, uint64_t rows, int cols, int box_rows) {
+// Tensor map over fp32 tiles: `ntiles` row-major [128 rows x cols] blocks, `tile_stride_bytes` apart, first one at
+// `base`.  Coordinates (col, row, tile), box = 32 columns x 128 rows x 1 tile (128 bytes wide), 128-byte swizzle.
+// Used for TMA reduce-add of fp32 panels.
+inline bool make_tensor_map_f32_tiles(CUtensorMap* out, const void* base, uint64_t ntiles, int cols,
+                                      uint64_t tile_stride_bytes) {
   PFN_tensorMapEncodeTiled enc = tensor_map_encoder();
   if (!enc) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
-  cuuint32_t box[2] = {32u, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1u, 1u};
-  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+  cuuint64_t dims[3] = {(cuuint64_t)cols, 128u, (cuuint64_t)ntiles};
+  cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)tile_stride_bytes};
+  cuuint32_t box[3] = {32u, 128u, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
