@@ -140,20 +140,20 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
           tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, i * 128, hq, b);
-        if (kDense) {
-          ok = mbar_wait(&do_empty[s], ((n >> 1) & 1) ^ 1, status);
-          if (!ok) { mbar_wait(&q_full[s], (n >> 1) & 1, status); break; }
-          mbar_arrive_expect_tx(&do_full[s], Cfg::kTileBytes);
-          for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, i * 128, hq, b);
-        }
+        // dO of every tile is fetched ahead, retained or not (the vote comes too late to hide the copy behind it);
+        // a skipped tile's stage is handed straight back by the issuer
+        ok = mbar_wait(&do_empty[s], ((n >> 1) & 1) ^ 1, status);
+        if (!ok) { mbar_wait(&q_full[s], (n >> 1) & 1, status); break; }
+        mbar_arrive_expect_tx(&do_full[s], Cfg::kTileBytes);
+        for (int pn = 0; pn < PAN; ++pn)
+          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, i * 128, hq, b);
         issued = n + 1;
       }
       if (!ok) {
         mbar_wait(&kv_full, 0, status);
         for (int n = (issued > 2 ? issued - 2 : 0); n < issued; ++n) {
           mbar_wait(&q_full[n & 1], (n >> 1) & 1, status);
-          if (kDense) mbar_wait(&do_full[n & 1], (n >> 1) & 1, status);
+          mbar_wait(&do_full[n & 1], (n >> 1) & 1, status);
         }
       }
     }
@@ -192,30 +192,20 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       };
       if (ok) ok = issue_qk(0);
       for (int n = 0; n < n_tot && ok; ++n) {
-        const int s = n & 1, hq = hkv * G + n / ni, i = i0 + n % ni;
+        const int s = n & 1;
         bool retain = true;
         if (!kDense) {
           ok = mbar_wait_warp(&vote_bar[n & 1], (n >> 1) & 1, status);
           if (!ok) break;
           retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[n % 3], 0) != 0;
         }
-        const int ds = r & 1;   // dO stage
+        const int ds = s;       // dO stage (the dS^T / dQ staging of the tile reuses it)
         if (retain) {
-          if (!kDense) {
-            ok = mbar_wait_warp(&do_empty[ds], ((r >> 1) & 1) ^ 1, status);
-            if (!ok) break;
-            if (leader) {
-              mbar_arrive_expect_tx(&do_full[ds], Cfg::kTileBytes);
-              for (int pn = 0; pn < PAN; ++pn)
-                tma_load_4d(sDO + ds * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[ds], pn * 64, i * 128, hq, b);
-            }
-            __syncwarp();
-          }
           if (r > 0) {   // the dQ tile of the previous retained tile (aliased with dP) has been read out
             ok = mbar_wait_warp(&dq_empty, (r - 1) & 1, status);
             if (!ok) break;
           }
-          ok = mbar_wait_warp(&do_full[ds], (r >> 1) & 1, status);
+          ok = mbar_wait_warp(&do_full[ds], (n >> 1) & 1, status);
           if (!ok) break;
           tc_fence_after();
           const uint64_t dDOk = desc_advance(dDOk0, ds * Cfg::kTileBytes);
@@ -263,7 +253,10 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
           ++r;
         } else {
-          if (leader) mbar_arrive(&q_empty[s]);
+          // skipped tile: Q and the dO fetched ahead (once it has landed) go back to their rings
+          ok = mbar_wait_warp(&do_full[ds], (n >> 1) & 1, status);
+          if (!ok) break;
+          if (leader) { mbar_arrive(&q_empty[s]); mbar_arrive(&do_empty[ds]); }
         }
       }
       // tell the dQ group that nothing more will come, then wait for every MMA to retire
@@ -275,9 +268,6 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_commit(&fin_bar);
       }
       mbar_wait_warp(&fin_bar, 0, status);
-      if (!ok && !kDense) {
-        for (int u = (r > 1 ? r - 1 : 0); u <= r; ++u) mbar_wait_warp(&do_full[u & 1], (u >> 1) & 1, status);
-      }
     }
   }
   } else if (warp < 20) {
@@ -431,7 +421,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         {
-          uint8_t* dst = sDS + (r & 1) * Cfg::kDsBytes + (qt >> 1) * 16384;
+          uint8_t* dst = sDS + (n & 1) * Cfg::kDsBytes + (qt >> 1) * 16384;
 #pragma unroll
           for (int v = 0; v < 4; ++v)
             *reinterpret_cast<uint4*>(dst + sw128_offset((uint32_t)rl, (uint32_t)((qt & 1) * 32 + v * 8))) =

@@ -22,6 +22,10 @@
 
 namespace mala {
 
+#ifndef MALA_TURN_EARLY
+#define MALA_TURN_EARLY 1
+#endif
+
 struct FwdParams {
   __nv_bfloat16* o;
   int64_t o_sb, o_sn, o_sh;
@@ -58,7 +62,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sK = sQ + 2 * Cfg::kTileBytes;
   uint8_t* sV = sK + KS * Cfg::kTileBytes;          // [2] blocks A, B
 
-  __shared__ uint64_t q_full, k_full[KS], k_empty[KS], v_full[2], v_empty[2], s_full[2], vote_bar[2], p_full[2],
+  __shared__ uint64_t q_full, k_full[KS], k_empty[KS], v_full[2], v_empty[2], s_full[2], vote_bar[2], p_full[2][2],
       fin_bar, turn_bar[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[2][3];
@@ -83,7 +87,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 2); }
     for (int x = 0; x < 2; ++x) {
       mbar_init(&v_full[x], 1); mbar_init(&v_empty[x], kDense ? 2 : 1);
-      mbar_init(&s_full[x], 1); mbar_init(&vote_bar[x], 4); mbar_init(&p_full[x], 4);
+      mbar_init(&s_full[x], 1); mbar_init(&vote_bar[x], 4); mbar_init(&p_full[x][0], 4); mbar_init(&p_full[x][1], 4);
       flag[x][0] = flag[x][1] = flag[x][2] = 0;
     }
     mbar_init(&fin_bar, 2);
@@ -195,15 +199,23 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
               }
               __syncwarp();
             }
-            ok = mbar_wait_warp(&p_full[x], r & 1, status);
+            // P arrives in two halves of 64 keys: the first four k-steps of O += P V run while the second half
+            // of the exponentials is still being computed
+            ok = mbar_wait_warp(&p_full[x][0], r & 1, status);
             if (ok) ok = mbar_wait_warp(&v_full[vs], vpar, status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t acc0 = r > 0 ? 1u : 0u;
             const uint64_t dVs = desc_advance(dV0, vs * Cfg::kTileBytes);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
+            for (int k = 0; k < 4; ++k)
               mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, k > 0 ? 1u : acc0, leader);
+            ok = mbar_wait_warp(&p_full[x][1], r & 1, status);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int k = 4; k < 8; ++k)
+              mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, 1u, leader);
             if (leader) tc_commit(&v_empty[vs]);
             ++r;
           }
@@ -266,13 +278,22 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (e + 96 > lim) s3[e] = ninf;
         }
       }
-      float mx0 = -INFINITY, mx1 = -INFINITY;
+      float mx[8];
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        mx0 = fmaxf(mx0, fmaxf(__uint_as_float(s0[e]), __uint_as_float(s1[e])));
-        mx1 = fmaxf(mx1, fmaxf(__uint_as_float(s2[e]), __uint_as_float(s3[e])));
+      for (int q = 0; q < 8; ++q) mx[q] = -INFINITY;
+#pragma unroll
+      for (int e = 0; e < 32; e += 4) {   // eight independent chains
+        mx[0] = fmaxf(mx[0], fmaxf(__uint_as_float(s0[e]), __uint_as_float(s0[e + 1])));
+        mx[1] = fmaxf(mx[1], fmaxf(__uint_as_float(s0[e + 2]), __uint_as_float(s0[e + 3])));
+        mx[2] = fmaxf(mx[2], fmaxf(__uint_as_float(s1[e]), __uint_as_float(s1[e + 1])));
+        mx[3] = fmaxf(mx[3], fmaxf(__uint_as_float(s1[e + 2]), __uint_as_float(s1[e + 3])));
+        mx[4] = fmaxf(mx[4], fmaxf(__uint_as_float(s2[e]), __uint_as_float(s2[e + 1])));
+        mx[5] = fmaxf(mx[5], fmaxf(__uint_as_float(s2[e + 2]), __uint_as_float(s2[e + 3])));
+        mx[6] = fmaxf(mx[6], fmaxf(__uint_as_float(s3[e]), __uint_as_float(s3[e + 1])));
+        mx[7] = fmaxf(mx[7], fmaxf(__uint_as_float(s3[e + 2]), __uint_as_float(s3[e + 3])));
       }
-      const float mt = fmaxf(mx0, mx1) * c2;   // row maximum of the scaled scores, log2 domain
+      // row maximum of the scaled scores, log2 domain
+      const float mt = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * c2;
       bool retain = true;
       if (!kDense) {
         // Eq. 3: skip iff rowmax - (m + log l) < log(tau / L) for every valid row
@@ -356,7 +377,17 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       MALA_P_CHUNK(s0, 0)
       MALA_P_CHUNK(s1, 16)
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[x][0]);   // keys 0..63 of P are in place
       MALA_P_CHUNK(s2, 32)
+#if MALA_TURN_EARLY
+      // hand the exponential phase over a little before it ends: the other group needs a few hundred cycles
+      // to notice, and the MUFU would idle meanwhile
+      __syncwarp();
+      if (lane == 0 && kDense && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);
+#endif
       MALA_P_CHUNK(s3, 48)
 #undef MALA_P_CHUNK
       l += (sum0 + sum1) + (sum2 + sum3);
@@ -364,8 +395,10 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(&p_full[x]);
+        mbar_arrive(&p_full[x][1]);
+#if !MALA_TURN_EARLY
         if (kDense && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);   // the other group's turn
+#endif
       }
       ++r;
     }
