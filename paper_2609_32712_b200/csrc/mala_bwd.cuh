@@ -81,7 +81,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
 
   __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
-      ds_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, ds_free;
+      ds_full, dst_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, ds_free;
   __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[3];
@@ -104,7 +104,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_init(&do_full[s], 1); mbar_init(&do_empty[s], 1);
       mbar_init(&vote_bar[s], 16);
     }
-    mbar_init(&s_full, 1); mbar_init(&p_full, 16); mbar_init(&dp_full, 1); mbar_init(&ds_full, 16);
+    mbar_init(&s_full, 1); mbar_init(&p_full, 16); mbar_init(&dp_full, 1); mbar_init(&ds_full, 16); mbar_init(&dst_full, 16);
     mbar_init(&dv_done, 1); mbar_init(&grp_bar, 16); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
     mbar_init(&fin_bar, 1);
     mbar_init(&stg_full, 4); mbar_init(&ds_free, 1);
@@ -230,7 +230,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // recompute the next tile's scores while dS is being formed
         if (n + 1 < n_tot) { ok = issue_qk(n + 1); if (!ok) break; }
         if (retain) {
-          ok = mbar_wait_warp(&ds_full, r & 1, status);
+          ok = mbar_wait_warp(&dst_full, r & 1, status);
           if (!ok) break;
           tc_fence_after();
           const uint64_t dDSm = desc_advance(dDSm0, ds * Cfg::kDsBytes);
@@ -241,6 +241,9 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             mma_ts(tmem_addr(tb, 0, Cfg::kColDK), tmem_addr(tb, 0, Cfg::kColDP + (k >> 1) * 32 + (k & 1) * 8),
                    desc_advance(dQm, k * 2048), idesc_dv, k > 0 ? 1u : acc1, leader);
           if (leader) tc_commit(&q_empty[s]);
+          ok = mbar_wait_warp(&ds_full, r & 1, status);   // the shared-memory copy of dS^T
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
           for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j, into the dP columns (after dK has read dS^T from them)
             mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
@@ -354,10 +357,14 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_before();
           mbar_arrive(&vote_bar[n & 1]);
         }
-        ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (!kDense) retain = (*(volatile int*)&flag[n % 3]) != 0;
+        // A warp that found a retained entry knows the outcome (the vote is an OR) and goes straight on; a warp
+        // without one waits for the others (in the dense kernel this wait is the group's per-tile rendezvous).
+        if (kDense || !any) {
+          ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (!kDense) retain = (*(volatile int*)&flag[n % 3]) != 0;
+        }
       }
       if (stat_thread && n % ni == 0) { r_head = 0; bm_bits = 0; bm_word = -1; }
       if (retain) {
@@ -417,6 +424,10 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         // dS^T also goes to TMEM, over this thread's own (already consumed) dP^T columns: A operand of dK
         tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColDP + qt * 32), w);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&dst_full);       // dK may start while the shared-memory copy is written
         ok = mbar_wait(&dv_done, r & 1, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -428,8 +439,6 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
         }
         fence_proxy_async_smem();
-        tmem_wait_st();
-        tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&ds_full);
         ++r;

@@ -1,11 +1,11 @@
 // MALA forward (Algorithm 1) for sm_100a, prefill version: two query blocks per CTA.
 //
 // One CTA owns the two consecutive 128-row query blocks A = 2c and B = 2c+1 of one (batch, query
-// head).  They share the K tiles; each block has its own UMMA-issuing thread, softmax warpgroup,
-// score buffer, V stage and output accumulator (TMEM: S_A, S_B, O_A, O_B = 512 columns).  A thread
-// that issues tcgen05.mma stalls until the tensor pipe accepts the instruction, so the waits and
-// commits of one block's issuer run while the other block's MMAs execute, and one block's rows are in
-// the softmax path while the pipe works for the other block.
+// head).  They share the K tiles; each block has its own UMMA-issuing warp, softmax warpgroup,
+// score buffer, V stage and output accumulator (TMEM: S_A, S_B, O_A, O_B = 512 columns).  Per block the
+// chain S = QK^T -> row max -> exp -> O += PV -> next QK is strictly serial (P overwrites S: there is no
+// TMEM left for a second score buffer), so one block's rows are in the softmax path while the tensor
+// pipe works for the other block, and the two softmax groups take turns in the exponential phase.
 // Each block keeps the semantics of Algorithm 1 on its own: its tiles are visited from ITS diagonal
 // toward earlier keys, the test for a tile uses the state left by that block's previous retained tile,
 // and a skipped tile issues no exp, no P, no V load and no PV.
@@ -299,7 +299,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // Eq. 3: skip iff rowmax - (m + log l) < log(tau / L) for every valid row
         bool vote;
         if (l == 0.f) vote = valid;   // nothing retained yet: the log-ratio is +inf
-        else vote = valid && !(((mt - (m_ref + log2f(l))) - theta) < 0.f);
+        else vote = valid && !(((mt - (m_ref + __log2f(l))) - theta) < 0.f);
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
           if (any) *(volatile int*)&flag[x][t % 3] = 1;
@@ -307,12 +307,28 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_before();
           mbar_arrive(&vote_bar[x]);
         }
-        ok = mbar_wait(&vote_bar[x], t & 1, status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        retain = (*(volatile int*)&flag[x][t % 3]) != 0;
+        // A warp that found a retaining row knows the outcome (the vote is an OR) and goes straight on; only a warp
+        // without one has to wait for the other three.
+        if (!any) {
+          ok = mbar_wait(&vote_bar[x], t & 1, status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          retain = (*(volatile int*)&flag[x][t % 3]) != 0;
+        }
       }
-      if (!retain) continue;   // m, l, O unchanged; no exp, no P, no PV
+      if (!retain) {   // m, l, O unchanged; no exp, no P, no PV: take the turn (see below) and pass it on at once
+        if (!kDense && hasB) {
+          const int idx = (x == 0) ? t : (t - 1 - firstA);
+          if (idx >= 0) {
+            ok = mbar_wait(&turn_bar[x], idx & 1, status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          __syncwarp();
+          if (lane == 0 && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);
+        }
+        continue;
+      }
       if (stat_thread && bm_row) {
         if ((j >> 5) != bm_word) {
           if (bm_word >= 0) bm_row[bm_word] = bm_bits;
@@ -344,13 +360,14 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
       }
-      // Dense kernel: the two softmax groups take turns in the exponential phase (B(0), A(0), B(1), A(1), ...)
+      // The two softmax groups take turns in the exponential phase (B(0), A(0), B(1), A(1), ...; a skipped tile
+      // takes its turn and passes it on at once)
       // so that one block's exponentials run while the tensor pipe works for the other block, instead of
       // both groups contending for the MUFU at the same time and then for the tensor pipe at the same time.
       // A's tile t follows B's tile of the same key step (t + firstA); B's tile t follows A's tile of the previous
       // step (t - 1 - firstA).  turn_bar[0] counts B's finished exp phases from tile firstA on, turn_bar[1] A's, so
       // every waiter sees the phases in sequence.
-      if (kDense && hasB) {
+      if (hasB) {
         const int idx = (x == 0) ? t : (t - 1 - firstA);
         if (idx >= 0) {
           ok = mbar_wait(&turn_bar[x], idx & 1, status);
@@ -386,7 +403,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // hand the exponential phase over a little before it ends: the other group needs a few hundred cycles
       // to notice, and the MUFU would idle meanwhile
       __syncwarp();
-      if (lane == 0 && kDense && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);
+      if (lane == 0 && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);
 #endif
       MALA_P_CHUNK(s3, 48)
 #undef MALA_P_CHUNK
@@ -397,7 +414,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (lane == 0) {
         mbar_arrive(&p_full[x][1]);
 #if !MALA_TURN_EARLY
-        if (kDense && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);   // the other group's turn
+        if (hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);   // the other group's turn
 #endif
       }
       ++r;
