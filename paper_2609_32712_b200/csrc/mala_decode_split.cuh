@@ -8,10 +8,11 @@
 // over its items with the K (and, dense, V) rings, the score buffers and the two output accumulators
 // running on across item boundaries; there is no per-item launch, TMEM allocation or pipeline drain.
 //   warp 0  TMA producer: Q of the next item (16 rows), K ring; dense kernel: V ring one tile behind K
-//   warp 1  UMMA issuer: S = Q K^T one tile ahead of the decision; MALA kernel: V loaded only for retained
-//           tiles; O[item parity] += P V
+//   warp 1  UMMA issuer: S = Q K^T one tile ahead of the decision; MALA kernel: V loaded for retained tiles (and,
+//           ahead of its vote, for the tile after a retained one); O[item parity] += P V
 //   warp 4  softmax warp (TMEM lanes 0..31): row max, Eq. 3 vote, P, lazy rescale, partial output
-// K is always streamed; a skipped tile issues no exp, no P, no V load and no PV.
+// K is always streamed; a skipped tile issues no exp, no P and no PV, and reads no V unless its V copy had been
+// issued ahead of the vote (only the tile right after a retained one can be in that case).
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -182,6 +183,24 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         if (++kc == KS) { kc = 0; kpar ^= 1; }
         return true;
       };
+      // MALA kernel: a V tile is needed only if its tile is retained, which is known after the vote -- too late to hide
+      // an HBM round trip with one tile of look-ahead.  So the V copy of the next tile is issued ahead of its
+      // votes while tiles are being retained (one tile ahead after a retained tile, and always for the first tile
+      // of an item, which is retained by construction), as far as V stages are free.  A copy fetched for a tile
+      // that is then skipped is handed back to the ring unused once it has landed: only then is a V tile read that
+      // the method itself would not have read.
+      auto load_v = [&](const Cur& c) {
+        if (leader) {
+          mbar_arrive_expect_tx(&v_full[vi], TB);
+          tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, (c.j0 - c.t) * 128, c.hkv, c.b);
+          tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, (c.j0 - c.t) * 128, c.hkv, c.b);
+        }
+        __syncwarp();
+        if (++vi == VS) { vi = 0; vipar ^= 1; }
+      };
+      int v_upto = -1;                           // V copies have been issued for every retained tile <= v_upto and,
+      Cur sp;                                    // ahead of their votes, for the tiles in (g, v_upto]; sp = tile v_upto + 1
+      sp.valid = false;
       Cur cur, nxt;
       first_item(cur, blockIdx.x, 0);
       if (cur.valid) ok = issue_qk(cur, 0);
@@ -195,17 +214,19 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           ok = mbar_wait_warp(&vote_bar[g & 1], (g >> 1) & 1, status);
           if (!ok) break;
           retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[g % 3], 0) != 0;
-          if (retain) {   // V of this tile, on demand
-            ok = mbar_wait_warp(&v_empty[vi], vipar, status);
-            if (!ok) break;
-            if (leader) {
-              mbar_arrive_expect_tx(&v_full[vi], TB);
-              tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, (cur.j0 - cur.t) * 128, cur.hkv, cur.b);
-              tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, (cur.j0 - cur.t) * 128, cur.hkv, cur.b);
+          if (retain) {
+            if (v_upto < g) {   // V of this tile, on demand
+              ok = mbar_wait_warp(&v_empty[vi], vipar, status);
+              if (!ok) break;
+              load_v(cur);
             }
-            __syncwarp();
-            if (++vi == VS) { vi = 0; vipar ^= 1; }
+          } else if (v_upto >= g) {   // fetched ahead but not needed: back to the ring once it has landed
+            ok = mbar_wait_warp(&v_full[vc], vcpar, status);
+            if (!ok) break;
+            if (leader) mbar_arrive(&v_empty[vc]);
+            if (++vc == VS) { vc = 0; vcpar ^= 1; }
           }
+          if (v_upto < g) { v_upto = g; sp = nxt; }
         }
         const int ip = cur.ne & 1;
         if (retain) {
@@ -229,6 +250,14 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           ++r_item;
         }
         if (cur.t == cur.T - 1) { if (leader) tc_commit(&item_done[ip]); r_item = 0; }
+        if (!kDense) {
+          const int depth = (retain || (nxt.valid && nxt.t == 0)) ? 1 : 0;   // (two tiles ahead measured slower)
+          while (v_upto < g + depth && sp.valid && __all_sync(0xffffffffu, mbar_try_wait(&v_empty[vi], vipar))) {
+            load_v(sp);
+            ++v_upto;
+            advance(sp);
+          }
+        }
         cur = nxt;
         ++g;
       }
