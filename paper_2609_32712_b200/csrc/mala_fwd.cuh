@@ -156,71 +156,90 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint32_t tS = tmem_addr(tb, 0, x * 128), tO = tmem_addr(tb, 0, 256 + x * 128);
       bool ok = mbar_wait_warp(&q_full, 0, status);
       int r = 0;                       // PVs issued (retained tiles); also counts this block's V loads
-      int s = 0;                       // K stage of step u
-      uint32_t kpar = 0;               // parity of k_full[s] for step u
-      for (int u = 0; u < U && ok; ++u) {
+      int s = 0;                       // K stage of the next step to be scored
+      uint32_t kpar = 0;               // parity of k_full[s] for that step
+      // S = Q K^T of the step whose K sits in stage s (k_full already observed)
+      auto issue_qk = [&]() {
+        tc_fence_after();
+        const uint64_t dK = desc_advance(dK0, s * Cfg::kTileBytes);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+          mma_ss(tS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0, leader);
+        }
+        if (leader) { tc_commit(&k_empty[s]); tc_commit(&s_full[x]); }
+        if (++s == KS) { s = 0; kpar ^= 1; }
+      };
+      // steps at which this block has no tile (all of them for an absent block): only release the stages
+      int u = 0;
+      for (; u < U && ok && (!present_x || u < first); ++u) {
         ok = mbar_wait_warp(&k_full[s], kpar, status);
         if (!ok) break;
-        if (!present_x || u < first) {
-          if (leader) mbar_arrive(&k_empty[s]);    // this block has no tile at this step
-          if (kDense) {                // release the shared V stage too, paced by its arrival
-            ok = mbar_wait_warp(&v_full[u & 1], (u >> 1) & 1, status);
-            if (!ok) break;
-            if (leader) mbar_arrive(&v_empty[u & 1]);
-          }
-        } else {
-          const int t = u - first;     // tile index of this block
-          tc_fence_after();
-          const uint64_t dK = desc_advance(dK0, s * Cfg::kTileBytes);
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tS, desc_advance(dQ, off), desc_advance(dK, off), idesc_qk, k > 0, leader);
-          }
-          if (leader) { tc_commit(&k_empty[s]); tc_commit(&s_full[x]); }
-          bool retain = true;
-          if (!kDense) {
-            ok = mbar_wait_warp(&vote_bar[x], t & 1, status);
-            if (!ok) break;
-            retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[x][t % 3], 0) != 0;
-          }
-          if (retain) {
-            // MALA: V is loaded on demand into this block's own stage (free once its previous PV retired);
-            // dense: V(u) sits in the shared ring stage u & 1
-            const int vs = kDense ? (u & 1) : x;
-            const uint32_t vpar = kDense ? ((u >> 1) & 1) : (r & 1);
-            if (!kDense) {
-              ok = mbar_wait_warp(&v_empty[x], (r & 1) ^ 1, status);
-              if (!ok) break;
-              if (leader) {
-                mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
-                for (int pn = 0; pn < PAN; ++pn)
-                  tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, (j0 - u) * 128, hkv, b);
-              }
-              __syncwarp();
-            }
-            // P arrives in two halves of 64 keys: the first four k-steps of O += P V run while the second half
-            // of the exponentials is still being computed
-            ok = mbar_wait_warp(&p_full[x][0], r & 1, status);
-            if (ok) ok = mbar_wait_warp(&v_full[vs], vpar, status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t acc0 = r > 0 ? 1u : 0u;
-            const uint64_t dVs = desc_advance(dV0, vs * Cfg::kTileBytes);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, k > 0 ? 1u : acc0, leader);
-            ok = mbar_wait_warp(&p_full[x][1], r & 1, status);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int k = 4; k < 8; ++k)
-              mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, 1u, leader);
-            if (leader) tc_commit(&v_empty[vs]);
-            ++r;
-          }
+        if (leader) mbar_arrive(&k_empty[s]);
+        if (kDense) {                  // release the shared V stage too, paced by its arrival
+          ok = mbar_wait_warp(&v_full[u & 1], (u >> 1) & 1, status);
+          if (!ok) break;
+          if (leader) mbar_arrive(&v_empty[u & 1]);
         }
         if (++s == KS) { s = 0; kpar ^= 1; }
+      }
+      if (ok && u < U) {
+        ok = mbar_wait_warp(&k_full[s], kpar, status);
+        if (ok) issue_qk();
+      }
+      // Per tile: everything that does not depend on P (the next step's K, whose copy landed long ago) is observed
+      // before the wait for P, so that between the second half of P and the next S = Q K^T only the PV and QK
+      // issue themselves remain -- this warp runs a serial instruction stream, and every instruction on the path from
+      // "P is there" to "the next scores are there" lengthens the block's per-tile chain.
+      for (; u < U && ok; ++u) {
+        const int t = u - first;       // tile index of this block
+        const bool has_next = (u + 1 < U);
+        if (has_next) {
+          ok = mbar_wait_warp(&k_full[s], kpar, status);
+          if (!ok) break;
+        }
+        bool retain = true;
+        if (!kDense) {
+          ok = mbar_wait_warp(&vote_bar[x], t & 1, status);
+          if (!ok) break;
+          retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[x][t % 3], 0) != 0;
+        }
+        if (retain) {
+          // MALA: V is loaded on demand into this block's own stage (free once its previous PV retired);
+          // dense: V(u) sits in the shared ring stage u & 1
+          const int vs = kDense ? (u & 1) : x;
+          const uint32_t vpar = kDense ? ((u >> 1) & 1) : (r & 1);
+          if (!kDense) {
+            ok = mbar_wait_warp(&v_empty[x], (r & 1) ^ 1, status);
+            if (!ok) break;
+            if (leader) {
+              mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
+              for (int pn = 0; pn < PAN; ++pn)
+                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, (j0 - u) * 128, hkv, b);
+            }
+            __syncwarp();
+          }
+          const uint32_t acc0 = r > 0 ? 1u : 0u;
+          const uint64_t dVs = desc_advance(dV0, vs * Cfg::kTileBytes);
+          // P arrives in two halves of 64 keys: the first four k-steps of O += P V run while the second half
+          // of the exponentials is still being computed
+          ok = mbar_wait_warp(&v_full[vs], vpar, status);
+          if (ok) ok = mbar_wait_warp(&p_full[x][0], r & 1, status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, k > 0 ? 1u : acc0, leader);
+          ok = mbar_wait_warp(&p_full[x][1], r & 1, status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k = 4; k < 8; ++k)
+            mma_ts(tO, tS + k * 8, desc_advance(dVs, k * 2048), idesc_pv, 1u, leader);
+          if (leader) tc_commit(&v_empty[vs]);
+          ++r;
+        }
+        if (has_next) issue_qk();      // in tensor-pipe order after this tile's PV: the score buffer is reused
       }
       // every MMA of this block has retired (and every V copy landed) before the CTA may exit
       __syncwarp();
