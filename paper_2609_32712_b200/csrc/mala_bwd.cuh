@@ -133,8 +133,10 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       bool ok = true;
       int issued = 0;
-      for (int n = 0; n < n_tot && ok; ++n) {
-        const int s = n & 1, hq = hkv * G + n / ni, i = i0 + n % ni;
+      int hq = hkv * G, i = i0;   // tile n = (query head, query block), kept by increments: no division per tile
+      for (int n = 0; n < n_tot && ok; ++n, ++i) {
+        if (i == p.T) { i = i0; ++hq; }
+        const int s = n & 1;
         ok = mbar_wait(&q_empty[s], ((n >> 1) & 1) ^ 1, status);
         if (!ok) break;
         mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
@@ -292,13 +294,12 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     uint32_t bm_bits = 0;
     int bm_word = -1;
 
-    auto vec_index = [&](int n) -> size_t {
-      const int hq = hkv * G + n / ni, i = i0 + n % ni;
-      return ((size_t)b * p.Hq + hq) * p.Np + (size_t)i * 128 + rl;
+    auto vec_index = [&](int hq_local, int i) -> size_t {
+      return ((size_t)b * p.Hq + hkv * G + hq_local) * p.Np + (size_t)i * 128 + rl;
     };
     // per-query vectors of tile 0 into slot 0 (published by the first column quarter), then a group sync
     if (qt == 0) {
-      const size_t x = vec_index(0);
+      const size_t x = vec_index(0, i0);
       vec[0][0][rl] = p.lse2[x];
       vec[0][1][rl] = p.bq[x];
       vec[0][2][rl] = p.Dq[x];
@@ -308,13 +309,15 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     ok = mbar_wait(&grp_bar, 0, status);
     ok = __all_sync(0xffffffffu, ok);
 
-    for (int n = 0; n < n_tot && ok; ++n) {
-      const int hq_n = n / ni, i = i0 + n % ni;
-      const int slot = n % 3;
+    // tile n = (query head hq_n of the group, query block i): kept by increments, no division per tile
+    int hq_n = 0, i = i0, slot = 0;
+    for (int n = 0; n < n_tot && ok; ++n, ++i, slot = (slot == 2 ? 0 : slot + 1)) {
+      if (i == p.T) { i = i0; ++hq_n; }
+      const bool first_of_head = (i == i0), last_of_head = (i == p.T - 1);
       // prefetch the per-query vectors of the next tile
       float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
       if (qt == 0 && n + 1 < n_tot) {
-        const size_t x = vec_index(n + 1);
+        const size_t x = last_of_head ? vec_index(hq_n + 1, i0) : vec_index(hq_n, i + 1);
         nx0 = p.lse2[x]; nx1 = p.bq[x]; nx2 = p.Dq[x];
       }
       ok = mbar_wait(&s_full, n & 1, status);
@@ -344,7 +347,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       // publish the next tile's vectors (slot (n+1) % 3 was last read two tiles ago)
       if (qt == 0) {
-        const int ns = (n + 1) % 3;
+        const int ns = (slot == 2 ? 0 : slot + 1);
         vec[ns][0][rl] = nx0; vec[ns][1][rl] = nx1; vec[ns][2][rl] = nx2;
       }
       bool retain = true;
@@ -352,8 +355,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const bool vote = !kDense && valid_key && !(crit < 0.f);
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
-          if (any) *(volatile int*)&flag[n % 3] = 1;
-          if (warp == 4) *(volatile int*)&flag[(n + 1) % 3] = 0;
+          if (any) *(volatile int*)&flag[slot] = 1;
+          if (warp == 4) *(volatile int*)&flag[slot == 2 ? 0 : slot + 1] = 0;
           tc_fence_before();
           mbar_arrive(&vote_bar[n & 1]);
         }
@@ -363,10 +366,10 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          if (!kDense) retain = (*(volatile int*)&flag[n % 3]) != 0;
+          if (!kDense) retain = (*(volatile int*)&flag[slot]) != 0;
         }
       }
-      if (stat_thread && n % ni == 0) { r_head = 0; bm_bits = 0; bm_word = -1; }
+      if (stat_thread && first_of_head) { r_head = 0; bm_bits = 0; bm_word = -1; }
       if (retain) {
         if (stat_thread) {
           ++r_head;
@@ -443,7 +446,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (lane == 0) mbar_arrive(&ds_full);
         ++r;
       }
-      if (stat_thread && (n % ni == ni - 1)) {   // last tile of this query head
+      if (stat_thread && last_of_head) {   // last tile of this query head
         const size_t row = (size_t)(b * p.Hq + hkv * G + hq_n) * p.T + j;
         if (p.bitmask && bm_word >= 0) p.bitmask[row * p.words + bm_word] = bm_bits;
         if (p.retained) p.retained[row] = (uint32_t)r_head;
