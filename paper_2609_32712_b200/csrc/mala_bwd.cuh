@@ -345,14 +345,16 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                                    fmaxf(fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w))));
         }
       }
-      // publish the next tile's vectors (slot (n+1) % 3 was last read two tiles ago)
+      // publish the next tile's vectors.  Slot (n+1) % 3 was last read in tile n-2, which every warp has left:
+      // the scores of tile n only exist because all 16 warps delivered P^T of tile n-1, after their tile n-2.
+      // The readers in tile n+1 see the values through the chain arrive (P^T / vote) -> UMMA warp -> scores.
       if (qt == 0) {
         const int ns = (slot == 2 ? 0 : slot + 1);
         vec[ns][0][rl] = nx0; vec[ns][1][rl] = nx1; vec[ns][2][rl] = nx2;
       }
       bool retain = true;
-      {
-        const bool vote = !kDense && valid_key && !(crit < 0.f);
+      if (!kDense) {
+        const bool vote = valid_key && !(crit < 0.f);
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
           if (any) *(volatile int*)&flag[slot] = 1;
@@ -361,12 +363,12 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           mbar_arrive(&vote_bar[n & 1]);
         }
         // A warp that found a retained entry knows the outcome (the vote is an OR) and goes straight on; a warp
-        // without one waits for the others (in the dense kernel this wait is the group's per-tile rendezvous).
-        if (kDense || !any) {
+        // without one waits for the others.
+        if (!any) {
           ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          if (!kDense) retain = (*(volatile int*)&flag[slot]) != 0;
+          retain = (*(volatile int*)&flag[slot]) != 0;
         }
       }
       if (stat_thread && first_of_head) { r_head = 0; bm_bits = 0; bm_word = -1; }
