@@ -5,8 +5,9 @@
 //   mala_bwd_kernel       : one CTA per (key block j, KV head, batch).  K_j, V_j stay in shared memory;
 //                           for every query head of the group and every query block i >= j (ascending)
 //                           S^T = K_j Q_i^T is recomputed on tensor cores and tested against the saved
-//                           lse (Eq. 4).  Only retained tiles load dO and run dP^T = V dO^T, P^T,
-//                           dS^T = P^T o (dP^T - D), dV += P^T dO, dK += dS^T Q, dQ_i += dS K_j.
+//                           lse (Eq. 4).  Only retained tiles run dP^T = V dO^T, P^T,
+//                           dS^T = P^T o (dP^T - D), dV += P^T dO, dK += dS^T Q, dQ_i += dS K_j
+//                           (dO is fetched ahead for every tile: the vote comes too late to hide the copy).
 //                           dK, dV accumulate in TMEM; dQ tiles are added to an fp32 accumulator in
 //                           global memory, one half of the columns by vector reductions from registers
 //                           (red.global.add.v4.f32), the other half by TMA reduce-add from shared memory.
@@ -20,14 +21,19 @@
 //   bwd_convert_dq_kernel : dq = bf16(scale * accumulator), back in row-major order.
 //
 // Warp roles of the main kernel (768 threads; registers are re-split between the warpgroups):
-//   warp 0       TMA producer (K_j, V_j once; Q ring; in the dense kernel also the dO ring)
-//   warp 1       UMMA issuer (and, in the MALA kernel, the on-demand dO loads); warps 2-3 idle
+//   warp 0       TMA producer (K_j, V_j once; Q ring; dO ring)
+//   warp 1       UMMA warp (all 32 lanes run the issue loop, one elected lane issues); warps 2-3 idle
 //   warps 4-19   score group, four threads per key row (32 query columns each): reads S^T once, applies
 //                Eq. 4 and votes; retained tiles: P^T -> TMEM (A operand of dV), then, with P^T still in
-//                registers, dS^T = P^T o (dP^T - D) -> shared memory (operand of dQ and dK)
+//                registers, dS^T = P^T o (dP^T - D) -> TMEM (A operand of dK) and shared memory (operand of dQ)
 //   warps 20-23  dQ group, one thread per query row: takes the whole dQ tile out of TMEM at once (so that
-//                the next dP^T can be issued) and adds it to the global accumulator from shared memory
+//                the next dP^T can be issued) and adds it to the global accumulator
 // Registers released by warps 0-19 (setmaxnreg) go to the dQ group, which holds a 128-column row.
+// The warps run serial instruction streams at one dependent instruction per few cycles, so whatever a warp
+// executes between the barrier it waited on and the barrier it arrives on (or the MMA it issues) is on the
+// per-tile critical path: tile coordinates are kept by increments (no integer division per tile), waits whose
+// data arrived long ago come before the wait for fresh data, and a warp with a positive vote does not wait
+// for the group's vote.
 #pragma once
 #include <cuda_runtime.h>
 
