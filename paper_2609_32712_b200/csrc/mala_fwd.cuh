@@ -22,10 +22,6 @@
 
 namespace mala {
 
-#ifndef MALA_TURN_EARLY
-#define MALA_TURN_EARLY 1
-#endif
-
 struct FwdParams {
   __nv_bfloat16* o;
   int64_t o_sb, o_sn, o_sh;
@@ -418,24 +414,17 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(&p_full[x][0]);   // keys 0..63 of P are in place
       MALA_P_CHUNK(s2, 32)
-#if MALA_TURN_EARLY
       // hand the exponential phase over a little before it ends: the other group needs a few hundred cycles
       // to notice, and the MUFU would idle meanwhile
       __syncwarp();
       if (lane == 0 && hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);
-#endif
       MALA_P_CHUNK(s3, 48)
 #undef MALA_P_CHUNK
       l += (sum0 + sum1) + (sum2 + sum3);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&p_full[x][1]);
-#if !MALA_TURN_EARLY
-        if (hasB && (x == 0 || t >= firstA)) mbar_arrive(&turn_bar[1 - x]);   // the other group's turn
-#endif
-      }
+      if (lane == 0) mbar_arrive(&p_full[x][1]);
       ++r;
     }
 
