@@ -40,8 +40,11 @@ inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) {
 
 inline bool decode_set_attributes() {
   bool ok = true;
-  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
-  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
+#define MALA_DEC_ATTR(DENSE, GP) \
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
+  MALA_DEC_ATTR(false, 1) MALA_DEC_ATTR(false, 2) MALA_DEC_ATTR(false, 4) MALA_DEC_ATTR(false, 8) MALA_DEC_ATTR(false, 16)
+  MALA_DEC_ATTR(true, 1) MALA_DEC_ATTR(true, 2) MALA_DEC_ATTR(true, 4) MALA_DEC_ATTR(true, 8) MALA_DEC_ATTR(true, 16)
+#undef MALA_DEC_ATTR
   return ok;
 }
 
@@ -82,10 +85,18 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return MALA_ERR_CUDA;
   const int grid = p.n_items < sms ? p.n_items : sms;   // persistent: one CTA per SM
-  if (tau == 0.f)
-    mala_decode_split_kernel<true><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);
-  else
-    mala_decode_split_kernel<false><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);
+  const int G = Hq / Hkv;
+#define MALA_DEC_LAUNCH(GP)                                                                                          \
+  {                                                                                                                  \
+    if (tau == 0.f) mala_decode_split_kernel<true, GP><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    else mala_decode_split_kernel<false, GP><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);           \
+  }
+  if (G <= 1) MALA_DEC_LAUNCH(1)
+  else if (G <= 2) MALA_DEC_LAUNCH(2)
+  else if (G <= 4) MALA_DEC_LAUNCH(4)
+  else if (G <= 8) MALA_DEC_LAUNCH(8)
+  else MALA_DEC_LAUNCH(16)
+#undef MALA_DEC_LAUNCH
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   decode_merge_kernel<128><<<B * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb, o.sh, lse_opt, Hq,
                                                        num_splits);

@@ -1,18 +1,26 @@
 // Split-KV decode, split kernel ("Fused decoding execution") for sm_100a, head size 128.
 //
-// A work item is one split of one (batch, KV head): the G = Hq/Hkv query heads that share the KV head
-// are the rows of its tile (rows G..127 of the MMA tile read whatever follows the 16 loaded rows in
-// shared memory and are ignored), L = Nk for every row, the tiles of the split are visited newest
-// first with the item's own running (m, l), and the item ends with a normalised fp32 partial output
-// and its log-normalizer per head.  The kernel is HBM-bound, so it is persistent: one CTA per SM walks
-// over its items with the K (and, dense, V) rings, the score buffers and the two output accumulators
-// running on across item boundaries; there is no per-item launch, TMEM allocation or pipeline drain.
-//   warp 0  TMA producer: Q of the next item (16 rows), K ring; dense kernel: V ring one tile behind K
-//   warp 1  UMMA issuer: S = Q K^T one tile ahead of the decision; MALA kernel: V loaded for retained tiles (and,
-//           ahead of its vote, for the tile after a retained one); O[item parity] += P V
-//   warp 4  softmax warp (TMEM lanes 0..31): row max, Eq. 3 vote, P, lazy rescale, partial output
-// K is always streamed; a skipped tile issues no exp, no P and no PV, and reads no V unless its V copy had been
-// issued ahead of the vote (only the tile right after a retained one can be in that case).
+// A work item is one split of one (batch, KV head): the G = Hq/Hkv <= 16 query heads that share the KV head
+// are processed together, L = Nk for every head, the tiles of the split are visited newest first with the
+// item's own running (m, l), and the item ends with a normalised fp32 partial output and its log-normalizer
+// per head.  The kernel is HBM-bound, so it is persistent: one CTA per SM walks over its items with the K / V
+// rings and the score buffers running on across item boundaries.
+//
+// The problem is held transposed, keys (and output channels) in the TMEM lanes and the packed query heads as the
+// N = 16 columns of the MMAs:
+//     S^T [128 keys x 16]  = K_tile [128 x d] . Q^T [d x 16]        (A = K tile, B = Q tile, both K-major)
+//     O^T [d x 16]        += V_tile^T [d x 128 keys] . P^T [128 x 16]  (A = V tile read MN-major, B = P^T from smem)
+// so that all 128 softmax threads share a tile's work (16 scores each instead of one lane per head with 128), a
+// score buffer takes 16 TMEM columns (ring of four) and P^T is a 4 KB shared-memory tile (ring of four).
+//   warp 0     TMA producer: Q of the next item (16 rows), K ring; dense kernel: V ring one tile behind K
+//   warp 1     UMMA warp, event driven.  Three cursors walk over the tiles in order: S^T (as soon as a score
+//              buffer and the K tile are there), the vote (MALA kernel: the V copy of a retained tile is issued
+//              the moment its vote is known) and O^T += V^T P^T (as soon as P^T and V are there).  No step waits
+//              for another one's data, so the HBM latency of a V copy that can only be requested after the vote
+//              is hidden behind the tiles that follow.
+//   warps 4-7  softmax group, thread = key of the tile: per-head maxima and sums by warp shuffles and one small
+//              exchange per tile between the four warps, Eq. 3, P^T -> smem; lazy rescale of O^T
+// K is always streamed; a skipped tile issues no exp, no P, no V load and no PV.
 #pragma once
 #include "sm100_ptx.cuh"
 
@@ -32,13 +40,18 @@ struct DecParams {
 struct DecCfg {
   static constexpr int kTileBytes = 128 * 128 * 2;
   static constexpr int kQBytes = 4096;                   // 16 rows x 128 columns, two 2 KB panels
-  static constexpr int kKStages = 3, kVStages = 3;
-  static constexpr int kSmemBytes = 2 * kQBytes + (kKStages + kVStages) * kTileBytes + 1024;
-  static constexpr int kThreads = 160;
+  static constexpr int kPBytes = 4096;                   // P^T: 16 rows (heads) x 128 keys, two 2 KB panels
+  static constexpr int kKStages = 3, kVStages = 3, kPStages = 4, kSStages = 4;
+  static constexpr int kSmemBytes = 2 * kQBytes + (kKStages + kVStages) * kTileBytes + kPStages * kPBytes + 1024;
+  static constexpr int kThreads = 256;
+  static constexpr uint32_t kTmemCols = 128;             // S^T ring 4 x 16, O^T 2 x 16 (item parity)
+  static constexpr uint32_t kColO = 64;
 };
 
-template <bool kDense>
-__global__ void __launch_bounds__(160, 1)
+// GP: the number of packed heads rounded up to a power of two (compile-time, so that the per-head loops of the
+// softmax group unroll without branches)
+template <bool kDense, int GP>
+__global__ void __launch_bounds__(256, 1)
 mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                          const __grid_constant__ CUtensorMap tmV, const DecParams p) {
   constexpr int KS = DecCfg::kKStages, VS = DecCfg::kVStages, TB = DecCfg::kTileBytes;
@@ -47,11 +60,13 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   uint8_t* sQ = smem;                      // [2] item parity
   uint8_t* sK = sQ + 2 * DecCfg::kQBytes;
   uint8_t* sV = sK + KS * TB;
+  uint8_t* sP = sV + VS * TB;              // [4] P^T ring
 
-  __shared__ uint64_t q_full[2], q_empty[2], k_full[KS], k_empty[KS], v_full[VS], v_empty[VS], s_full[2],
-      vote_bar[2], p_full[2], o_done, item_done[2], o_free[2], fin_bar;
+  __shared__ uint64_t q_full[2], q_empty[2], k_full[KS], k_empty[KS], v_full[VS], v_empty[VS], s_full[4], s_free[4],
+      vote_bar[4], p_full[4], p_free[4], item_done[2], o_free[2], fin_bar, grp_a;
   __shared__ uint32_t tmem_base_s;
-  __shared__ int flag[3];
+  __shared__ int flag[4];
+  __shared__ float xch_max[2][4][16], xch_sum[2][4][16];   // the softmax group's per-tile exchange
   __shared__ int early_exit;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -61,19 +76,22 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&s_full[s], 1); mbar_init(&vote_bar[s], 1);
-      mbar_init(&p_full[s], 1); mbar_init(&item_done[s], 1); mbar_init(&o_free[s], 1);
+      mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&item_done[s], 1); mbar_init(&o_free[s], 4);
     }
     for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); }
     for (int s = 0; s < VS; ++s) { mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
-    mbar_init(&o_done, 1);
+    for (int s = 0; s < 4; ++s) {
+      mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4); mbar_init(&vote_bar[s], 1);
+      mbar_init(&p_full[s], 4); mbar_init(&p_free[s], 1);
+      flag[s] = 0;
+    }
     mbar_init(&fin_bar, 1);
-    flag[0] = flag[1] = flag[2] = 0;
+    mbar_init(&grp_a, 4);
     mbar_fence_init();
   }
   __syncthreads();
   if (early_exit) return;
-  if (warp == 0) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
+  if (warp == 0) { tmem_alloc(&tmem_base_s, DecCfg::kTmemCols); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -131,215 +149,243 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ UMMA issuer (+ on-demand V loads)
+    // ------------------------------------------------------------------ UMMA warp (+ on-demand V loads)
     // All 32 lanes run this loop with identical values; MMAs, commits and TMA loads are issued by one elected lane.
     {
       const uint32_t leader = elect_one();
-      constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false, false);
-      constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, false, true);
+      constexpr uint32_t idesc_qk = make_idesc_bf16(128, 16, false, false);
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, 16, true, false);
       const uint64_t dQ0 = make_smem_desc(smem_u32(sQ), 16, 1024);
       const uint64_t dK0 = make_smem_desc(smem_u32(sK), 16, 1024);
-      const uint64_t dV0 = make_smem_desc(smem_u32(sV), 16384, 1024);
-      bool ok = true;
-      // cursor over (non-empty item, tile) in processing order, and a second one running one tile ahead
-      struct Cur { int item, ne, t, T, b, hkv, split, j0; bool valid; };
-      auto first_item = [&](Cur& c, int from, int ne) {
+      const uint64_t dV0 = make_smem_desc(smem_u32(sV), 16384, 1024);   // V tile read MN-major (M = channel)
+      const uint64_t dP0 = make_smem_desc(smem_u32(sP), 16, 1024);
+      // cursor over (non-empty item, tile) in processing order; g = global tile number
+      struct Cur { int item, ne, t, T, b, hkv, j0, g; bool valid; };
+      auto first_item = [&](Cur& c, int from, int ne, int g) {
         c.valid = false;
+        c.g = g;
         for (int item = from; item < p.n_items; item += gridDim.x) {
           int b, hkv, split, T, j0;
           geometry(item, b, hkv, split, T, j0);
-          if (T > 0) { c = Cur{item, ne, 0, T, b, hkv, split, j0, true}; return; }
+          if (T > 0) { c.item = item; c.ne = ne; c.t = 0; c.T = T; c.b = b; c.hkv = hkv; c.j0 = j0; c.valid = true; return; }
         }
       };
       auto advance = [&](Cur& c) {
-        if (c.t + 1 < c.T) { ++c.t; return; }
-        first_item(c, c.item + gridDim.x, c.ne + 1);
+        if (c.t + 1 < c.T) { ++c.t; ++c.g; return; }
+        first_item(c, c.item + gridDim.x, c.ne + 1, c.g + 1);
       };
-      int g = 0;                                 // global tile counter (score buffer g & 1)
+      auto ready = [&](uint64_t* bar, uint32_t parity) -> bool { return __all_sync(0xffffffffu, mbar_test_wait(bar, parity)); };
+      Cur cq, cv, cp;                            // next tile to score, to take the vote of, to accumulate
+      first_item(cq, blockIdx.x, 0, 0);
+      cv = cq; cp = cq;
       int kc = 0; uint32_t kpar = 0;             // K ring consumer
-      int vi = 0; uint32_t vipar = 1;            // V ring producer side (MALA: loads issued here)
+      int vi = 0; uint32_t vipar = 1;            // V ring producer side (MALA: copies issued here)
       int vc = 0; uint32_t vcpar = 0;            // V ring consumer
-      uint32_t ppar[2] = {0, 0};
-      int q_seen = -1;                           // last non-empty item whose Q has been observed
-      auto issue_qk = [&](const Cur& c, int gq) -> bool {
-        const int ip = c.ne & 1;
-        if (q_seen < c.ne) {
-          if (!mbar_wait_warp(&q_full[ip], (c.ne >> 1) & 1, status)) return false;
-          q_seen = c.ne;
-        }
-        if (!mbar_wait_warp(&k_full[kc], kpar, status)) return false;
-        tc_fence_after();
-        const uint32_t dS = tmem_addr(tb, 0, (gq & 1) * 128);
-        const uint64_t dQ = desc_advance(dQ0, ip * DecCfg::kQBytes), dK = desc_advance(dK0, kc * TB);
+      uint32_t ret_bits = 0;                     // bit (g & 3): tile g was retained
+      int npv = 0;                               // PVs issued so far (P^T ring slot npv & 3)
+      int r_item = 0;                            // PVs of the accumulating cursor's item so far
+      bool ok = true;
+      long long t_progress = clock64();
+      uint32_t idle = 0;
+      while (cp.valid && ok) {
+        bool progress = false;
+        // ---- S^T of tile cq.g: its score buffer (g & 3) is free once the softmax group has read tile g - 4, and
+        //      at most four votes are outstanding (the size of their ring)
+        if (cq.valid && cq.g - cv.g < 4) {
+          const int ip = cq.ne & 1, sb = cq.g & 3;
+          if ((cq.g < 4 || ready(&s_free[sb], (uint32_t)(((cq.g >> 2) - 1) & 1))) &&
+              (cq.t > 0 || ready(&q_full[ip], (cq.ne >> 1) & 1)) && ready(&k_full[kc], kpar)) {
+            tc_fence_after();
+            const uint32_t dS = tmem_addr(tb, 0, (uint32_t)sb * 16u);
+            const uint64_t dQ = desc_advance(dQ0, ip * DecCfg::kQBytes), dK = desc_advance(dK0, kc * TB);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)   // Q panels lie 2 KB apart, K panels 16 KB
-          mma_ss(dS, desc_advance(dQ, (k >> 2) * 2048 + (k & 3) * 32), desc_advance(dK, (k >> 2) * 16384 + (k & 3) * 32),
-                 idesc_qk, k > 0, leader);
-        if (leader) {
-          tc_commit(&k_empty[kc]);
-          tc_commit(&s_full[gq & 1]);
-          if (c.t == c.T - 1) tc_commit(&q_empty[ip]);   // last QK of the item: its Q stage may be refilled
-        }
-        if (++kc == KS) { kc = 0; kpar ^= 1; }
-        return true;
-      };
-      // MALA kernel: a V tile is needed only if its tile is retained, which is known after the vote -- too late to hide
-      // an HBM round trip with one tile of look-ahead.  So the V copy of the next tile is issued ahead of its
-      // votes while tiles are being retained (one tile ahead after a retained tile, and always for the first tile
-      // of an item, which is retained by construction), as far as V stages are free.  A copy fetched for a tile
-      // that is then skipped is handed back to the ring unused once it has landed: only then is a V tile read that
-      // the method itself would not have read.
-      auto load_v = [&](const Cur& c) {
-        if (leader) {
-          mbar_arrive_expect_tx(&v_full[vi], TB);
-          tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, (c.j0 - c.t) * 128, c.hkv, c.b);
-          tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, (c.j0 - c.t) * 128, c.hkv, c.b);
-        }
-        __syncwarp();
-        if (++vi == VS) { vi = 0; vipar ^= 1; }
-      };
-      int v_upto = -1;                           // V copies have been issued for every retained tile <= v_upto and,
-      Cur sp;                                    // ahead of their votes, for the tiles in (g, v_upto]; sp = tile v_upto + 1
-      sp.valid = false;
-      Cur cur, nxt;
-      first_item(cur, blockIdx.x, 0);
-      if (cur.valid) ok = issue_qk(cur, 0);
-      int r_item = 0;
-      while (cur.valid && ok) {
-        nxt = cur;
-        advance(nxt);
-        if (nxt.valid) { ok = issue_qk(nxt, g + 1); if (!ok) break; }
-        bool retain = true;
-        if (!kDense) {
-          ok = mbar_wait_warp(&vote_bar[g & 1], (g >> 1) & 1, status);
-          if (!ok) break;
-          retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[g % 3], 0) != 0;
-          if (retain) {
-            if (v_upto < g) {   // V of this tile, on demand
-              ok = mbar_wait_warp(&v_empty[vi], vipar, status);
-              if (!ok) break;
-              load_v(cur);
+            for (int k = 0; k < 8; ++k)   // K panels lie 16 KB apart, Q panels 2 KB
+              mma_ss(dS, desc_advance(dK, (k >> 2) * 16384 + (k & 3) * 32), desc_advance(dQ, (k >> 2) * 2048 + (k & 3) * 32),
+                     idesc_qk, k > 0, leader);
+            if (leader) {
+              tc_commit(&k_empty[kc]);
+              tc_commit(&s_full[sb]);
+              if (cq.t == cq.T - 1) tc_commit(&q_empty[ip]);   // last S^T of the item: its Q stage may be refilled
             }
-          } else if (v_upto >= g) {   // fetched ahead but not needed: back to the ring once it has landed
-            ok = mbar_wait_warp(&v_full[vc], vcpar, status);
-            if (!ok) break;
-            if (leader) mbar_arrive(&v_empty[vc]);
-            if (++vc == VS) { vc = 0; vcpar ^= 1; }
+            if (++kc == KS) { kc = 0; kpar ^= 1; }
+            advance(cq);
+            progress = true;
           }
-          if (v_upto < g) { v_upto = g; sp = nxt; }
         }
-        const int ip = cur.ne & 1;
-        if (retain) {
-          ok = mbar_wait_warp(&p_full[g & 1], ppar[g & 1], status);
-          if (!ok) break;
-          ppar[g & 1] ^= 1;
-          ok = mbar_wait_warp(&v_full[vc], vcpar, status);
-          if (!ok) break;
-          if (r_item == 0 && cur.ne >= 2) {   // the softmax warp has read this accumulator's previous item
-            ok = mbar_wait_warp(&o_free[ip], ((cur.ne >> 1) - 1) & 1, status);
-            if (!ok) break;
+        // ---- vote of tile cv.g (dense: every tile is retained and V comes from the producer)
+        if (cv.valid && (!cq.valid || cv.g < cq.g) && cv.g - cp.g < 4) {   // (four tiles: the size of ret_bits)
+          if (kDense) {
+            ret_bits |= 1u << (cv.g & 3);
+            advance(cv);
+            progress = true;
+          } else if (ready(&vote_bar[cv.g & 3], (cv.g >> 2) & 1)) {
+            const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[cv.g & 3], 0) != 0;
+            if (!retain) {
+              ret_bits &= ~(1u << (cv.g & 3));
+              advance(cv);
+              progress = true;
+            } else if (ready(&v_empty[vi], vipar)) {   // V of this tile, on demand
+              if (leader) {
+                mbar_arrive_expect_tx(&v_full[vi], TB);
+                tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, (cv.j0 - cv.t) * 128, cv.hkv, cv.b);
+                tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, (cv.j0 - cv.t) * 128, cv.hkv, cv.b);
+              }
+              __syncwarp();
+              if (++vi == VS) { vi = 0; vipar ^= 1; }
+              ret_bits |= 1u << (cv.g & 3);
+              advance(cv);
+              progress = true;
+            }
           }
-          tc_fence_after();
-          const uint32_t aP = tmem_addr(tb, 0, (g & 1) * 128), dO = tmem_addr(tb, 0, 256 + ip * 128);
-          const uint64_t dV = desc_advance(dV0, vc * TB);
-          const uint32_t acc0 = r_item > 0 ? 1u : 0u;
+        }
+        // ---- O^T += V^T P^T of tile cp.g (or nothing, if it was skipped)
+        if (!cv.valid || cp.g < cv.g) {
+          const bool retain = (ret_bits >> (cp.g & 3)) & 1u;
+          bool done = !retain;
+          const int ip = cp.ne & 1, ps = npv & 3;
+          if (retain && ready(&p_full[ps], (uint32_t)((npv >> 2) & 1)) && ready(&v_full[vc], vcpar) &&
+              (r_item > 0 || cp.ne < 2 || ready(&o_free[ip], (uint32_t)(((cp.ne >> 1) - 1) & 1)))) {
+            // (first PV of an item: the softmax group has read this accumulator's previous item)
+            tc_fence_after();
+            const uint32_t dO = tmem_addr(tb, 0, DecCfg::kColO + (uint32_t)ip * 16u);
+            const uint64_t dV = desc_advance(dV0, vc * TB), dP = desc_advance(dP0, ps * DecCfg::kPBytes);
+            const uint32_t acc0 = r_item > 0 ? 1u : 0u;
 #pragma unroll
-          for (int k = 0; k < 8; ++k) mma_ts(dO, aP + k * 8, desc_advance(dV, k * 2048), idesc_pv, k > 0 ? 1u : acc0, leader);
-          if (leader) { tc_commit(&v_empty[vc]); tc_commit(&o_done); }
-          if (++vc == VS) { vc = 0; vcpar ^= 1; }
-          ++r_item;
-        }
-        if (cur.t == cur.T - 1) { if (leader) tc_commit(&item_done[ip]); r_item = 0; }
-        if (!kDense) {
-          const int depth = (retain || (nxt.valid && nxt.t == 0)) ? 1 : 0;   // (two tiles ahead measured slower)
-          while (v_upto < g + depth && sp.valid && __all_sync(0xffffffffu, mbar_try_wait(&v_empty[vi], vipar))) {
-            load_v(sp);
-            ++v_upto;
-            advance(sp);
+            for (int k = 0; k < 8; ++k)   // k-step = 16 keys: 2 KB further on in the V tile, 32 B in a P^T panel
+              mma_ss(dO, desc_advance(dV, k * 2048), desc_advance(dP, (k >> 2) * 2048 + (k & 3) * 32), idesc_pv,
+                     k > 0 ? 1u : acc0, leader);
+            if (leader) { tc_commit(&v_empty[vc]); tc_commit(&p_free[ps]); }
+            if (++vc == VS) { vc = 0; vcpar ^= 1; }
+            ++npv;
+            ++r_item;
+            done = true;
+          }
+          if (done) {
+            if (cp.t == cp.T - 1) { if (leader) tc_commit(&item_done[ip]); r_item = 0; }
+            advance(cp);
+            progress = true;
           }
         }
-        cur = nxt;
-        ++g;
+        if (progress) {
+          t_progress = clock64();
+          idle = 0;
+        } else {
+          // nothing could be done: back off (a warp that spins here takes issue slots from the softmax warp on
+          // its scheduler, and the whole group waits for that one at its barriers); bounded like every other wait
+          __nanosleep(100);
+          if (((++idle) & 0x3f) == 0) {
+            if (*(volatile int*)status != 0) ok = false;
+            else if (clock64() - t_progress > kWaitLimitCycles) { atomicCAS(status, 0, kDevTimeout); ok = false; }
+            ok = __all_sync(0xffffffffu, ok);
+          }
+        }
       }
       __syncwarp();
       if (leader) tc_commit(&fin_bar);
       mbar_wait_warp(&fin_bar, 0, status);
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
     }
-  } else if (warp == 4) {
-    // ------------------------------------------------------------------ softmax warp: lane = packed query head
-    const int rl = lane;
-    const bool valid = rl < G;
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax group: thread = key of the tile
+    // One exchange per tile between the four warps: every warp publishes the per-head maxima of its 32 keys of
+    // this tile together with its per-head sums of P of the previous retained tile; after one group barrier every
+    // thread holds the tile's row maxima and the up-to-date normalizers, evaluates Eq. 3 itself, and goes on.
+    const int w = warp & 3;
+    const uint32_t lane_base = (uint32_t)w * 32u;
+    const int kt = (int)lane_base + lane;          // key inside the tile; output channel in the epilogue
+    // rows G..15 of the P^T tiles are never written: clear the ring once so that those columns of O^T stay finite
+    for (int i = kt; i < DecCfg::kPStages * DecCfg::kPBytes / 16; i += 128) reinterpret_cast<uint4*>(sP)[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_proxy_async_smem();
     const float c2 = p.scale_log2;
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)p.Nk));
-    int g = 0, ne = 0, rg = 0;      // global tile counter, non-empty item ordinal, PVs requested so far
+    const bool head = (kt == 0);                   // the thread that keeps the telemetry
+    // The reference of the exponentials follows the scores only when they exceed it by 2^60: fp32 sums and bf16 P
+    // have the exponent range for it, and moving the reference means waiting until every PV issued so far has
+    // retired (their V copies included), which would stall this group for a whole HBM round trip.
+    constexpr float kRescaleGap = 60.f;
+    int g = 0, ne = 0, rg = 0;                     // global tile counter, non-empty item ordinal, retained tiles so far
+    uint32_t xc = 0;                               // exchanges so far (buffer xc & 1, barrier phase xc & 1)
     bool ok = true;
     for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
       int b, hkv, split, T, j0;
       geometry(item, b, hkv, split, T, j0);
-      const size_t prow = ((size_t)b * p.Hq + hkv * G + rl) * p.num_splits + split;
+      const size_t prow0 = ((size_t)b * p.Hq + hkv * G) * p.num_splits + split;   // head q: + q * num_splits
       const size_t stat_row = (size_t)(b * p.Hkv + hkv) * p.num_splits + split;
       if (T == 0) {   // empty split: (0, -inf)
-        if (valid) {
-          float4* dst = reinterpret_cast<float4*>(p.o_part + prow * 128);
-          for (int v = 0; v < 32; ++v) dst[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-          p.lse_part[prow] = -INFINITY;
-        }
-        if (lane == 0 && p.retained) p.retained[stat_row] = 0u;
+        for (int q = 0; q < G; ++q) p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = 0.f;
+        if (kt < G) p.lse_part[prow0 + (size_t)kt * p.num_splits] = -INFINITY;
+        if (head && p.retained) p.retained[stat_row] = 0u;
         continue;
       }
       const int ip = ne & 1;
-      const uint32_t colO = 256u + (uint32_t)ip * 128u;
-      float m_ref = -INFINITY, l = 0.f;
+      const uint32_t colO = DecCfg::kColO + (uint32_t)ip * 16u;
+      float m_ref[GP], l[GP], lgl[GP], ps_w[GP];   // ps_w: this warp's sums of P of the last retained tile
+#pragma unroll
+      for (int q = 0; q < GP; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; lgl[q] = -INFINITY; ps_w[q] = 0.f; }
       int r = 0;
+      bool pending_sum = false;
       uint32_t bm_bits = 0;
       int bm_word = -1;
       uint32_t* bm_row = p.bitmask ? p.bitmask + stat_row * p.words : nullptr;
+      // publishes this warp's (maxima, sums), waits for the group, returns the combined maxima in tmax and adds
+      // the combined sums to l
+      auto exchange = [&](const float (&mx_w)[GP], float (&tmax)[GP]) -> bool {
+        const int xb = xc & 1;
+        if (lane == 0) {
+#pragma unroll
+          for (int q = 0; q < GP; ++q) { xch_max[xb][w][q] = mx_w[q]; xch_sum[xb][w][q] = ps_w[q]; }
+          mbar_arrive(&grp_a);
+        }
+        bool k = mbar_wait(&grp_a, xc & 1, status);
+        k = __all_sync(0xffffffffu, k);
+        ++xc;
+        if (!k) return false;
+#pragma unroll
+        for (int q = 0; q < GP; ++q) {
+          tmax[q] = fmaxf(fmaxf(xch_max[xb][0][q], xch_max[xb][1][q]), fmaxf(xch_max[xb][2][q], xch_max[xb][3][q]));
+          if (pending_sum) {
+            l[q] += (xch_sum[xb][0][q] + xch_sum[xb][1][q]) + (xch_sum[xb][2][q] + xch_sum[xb][3][q]);
+            lgl[q] = __log2f(l[q]);
+          }
+        }
+        pending_sum = false;
+        return true;
+      };
       for (int t = 0; t < T; ++t, ++g) {
-        ok = mbar_wait(&s_full[g & 1], (g >> 1) & 1, status);
+        const int sb = g & 3;
+        ok = mbar_wait(&s_full[sb], (uint32_t)((g >> 2) & 1), status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t colS = (uint32_t)(g & 1) * 128u;
-        uint32_t s0[32], s1[32], s2[32], s3[32];
-        tmem_ld_x32(tmem_addr(tb, 0, colS + 0), s0);
-        tmem_ld_x32(tmem_addr(tb, 0, colS + 32), s1);
-        tmem_ld_x32(tmem_addr(tb, 0, colS + 64), s2);
-        tmem_ld_x32(tmem_addr(tb, 0, colS + 96), s3);
+        uint32_t sr[16];
+        tmem_ld_x16(tmem_addr(tb, lane_base, (uint32_t)sb * 16u), sr);
         tmem_wait_ld();
-        if (t == 0) {   // newest tile of the split: keys beyond the end of the cache
-          const int lim = p.Nk - 1 - j0 * 128;
-          const uint32_t ninf = 0xff800000u;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_free[sb]);     // the scores are in registers
+        const bool key_ok = ((j0 - t) * 128 + kt) < p.Nk;   // only the newest tile of the split can be ragged
+        float x[GP], mx[GP], tmax[GP];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            if (e > lim) s0[e] = ninf;
-            if (e + 32 > lim) s1[e] = ninf;
-            if (e + 64 > lim) s2[e] = ninf;
-            if (e + 96 > lim) s3[e] = ninf;
-          }
-        }
-        float mx0 = -INFINITY, mx1 = -INFINITY;
+        for (int q = 0; q < GP; ++q) { x[q] = (key_ok && q < G) ? __uint_as_float(sr[q]) * c2 : -INFINITY; mx[q] = x[q]; }
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          mx0 = fmaxf(mx0, fmaxf(__uint_as_float(s0[e]), __uint_as_float(s1[e])));
-          mx1 = fmaxf(mx1, fmaxf(__uint_as_float(s2[e]), __uint_as_float(s3[e])));
-        }
-        const float mt = fmaxf(mx0, mx1) * c2;
+        for (int s = 16; s > 0; s >>= 1)   // the reductions of the G heads run interleaved
+#pragma unroll
+          for (int q = 0; q < GP; ++q) mx[q] = fmaxf(mx[q], __shfl_xor_sync(0xffffffffu, mx[q], s));
+        ok = exchange(mx, tmax);
+        if (!ok) break;
+        // Eq. 3 against the split's partial normalizer: skip iff rowmax - (m + log l) < log(tau / Nk) for every head
         bool retain = true;
-        if (!kDense) {
-          // Eq. 3 against the split's partial normalizer: skip iff rowmax - (m + log l) < log(tau / Nk) for all rows
-          bool vote;
-          if (l == 0.f) vote = valid;
-          else vote = valid && !(((mt - (m_ref + log2f(l))) - theta) < 0.f);
-          retain = __any_sync(0xffffffffu, vote);
-          if (lane == 0) {
-            *(volatile int*)&flag[g % 3] = retain ? 1 : 0;
-            tc_fence_before();
-            mbar_arrive(&vote_bar[g & 1]);
-          }
+        if (!kDense && r > 0) {
+          retain = false;
+#pragma unroll
+          for (int q = 0; q < GP; ++q) retain = retain || (q < G && !(((tmax[q] - (m_ref[q] + lgl[q])) - theta) < 0.f));
+        }
+        if (!kDense && head) {
+          *(volatile int*)&flag[g & 3] = retain ? 1 : 0;
+          mbar_arrive(&vote_bar[g & 3]);
         }
         if (!retain) continue;
-        if (lane == 0 && bm_row) {
+        if (head && bm_row) {
           const int bit = T - 1 - t;   // tile index inside the split
           if ((bit >> 5) != bm_word) {
             if (bm_word >= 0) bm_row[bm_word] = bm_bits;
@@ -349,82 +395,95 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           bm_bits |= 1u << (bit & 31);
         }
         if (r == 0) {
-          m_ref = mt;
+#pragma unroll
+          for (int q = 0; q < GP; ++q) m_ref[q] = tmax[q];
         } else {
-          const bool need = mt > m_ref + 8.f;
-          if (__any_sync(0xffffffffu, need)) {
-            ok = mbar_wait(&o_done, (rg - 1) & 1, status);   // the previous PV has landed
+          float alpha[GP];
+          bool resc = false;
+#pragma unroll
+          for (int q = 0; q < GP; ++q) {
+            alpha[q] = 1.f;
+            if (q < G && tmax[q] > m_ref[q] + kRescaleGap) {   // lazy rescaling: the reference only moves when it has to
+              alpha[q] = fast_exp2(m_ref[q] - tmax[q]);
+              l[q] *= alpha[q];
+              lgl[q] = __log2f(l[q]);
+              m_ref[q] = tmax[q];
+              resc = true;
+            }
+          }
+          if (resc) {   // (the same decision in every thread: it only depends on exchanged values)
+            // every PV so far has landed: the latest one (number rg - 1) releases its P^T slot last.  (A parity wait
+            // must be neither ahead of nor two phases behind its barrier; per slot this one is exactly in step.)
+            ok = mbar_wait(&p_free[(rg - 1) & 3], (uint32_t)(((rg - 1) >> 2) & 1), status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const float m_new = fmaxf(m_ref, mt);
-            const float alpha = fast_exp2(m_ref - m_new);
-            l *= alpha;
-            m_ref = m_new;
+            uint32_t o[16];
+            tmem_ld_x16(tmem_addr(tb, lane_base, colO), o);
+            tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              uint32_t o[32];
-              tmem_ld_x32(tmem_addr(tb, 0, colO + c * 32), o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-              tmem_st_x32(tmem_addr(tb, 0, colO + c * 32), o);
-            }
+            for (int q = 0; q < GP; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
+            tmem_st_x16(tmem_addr(tb, lane_base, colO), o);
+            tmem_wait_st();
+            tc_fence_before();
           }
         }
-        const float nm = -m_ref;
-        float sum0 = 0.f, sum1 = 0.f;
-        uint32_t pk[16];
-#define MALA_DEC_P(SRC, COL)                                                           \
-        {                                                                              \
-          _Pragma("unroll") for (int e = 0; e < 16; ++e) {                             \
-            const float p0 = fast_exp2(fmaf(__uint_as_float(SRC[2 * e]), c2, nm));      \
-            const float p1 = fast_exp2(fmaf(__uint_as_float(SRC[2 * e + 1]), c2, nm));  \
-            sum0 += p0; sum1 += p1;                                                    \
-            pk[e] = pack_bf16x2(p0, p1);                                               \
-          }                                                                            \
-          tmem_st_x16(tmem_addr(tb, 0, colS + (COL)), pk);                             \
+        // P^T into slot rg & 3 of its ring, free once the PV that last read it has retired
+        const int ps = rg & 3;
+        if (rg >= 4) {
+          ok = mbar_wait(&p_free[ps], (uint32_t)(((rg >> 2) - 1) & 1), status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
         }
-        MALA_DEC_P(s0, 0)
-        MALA_DEC_P(s1, 16)
-        MALA_DEC_P(s2, 32)
-        MALA_DEC_P(s3, 48)
-#undef MALA_DEC_P
-        l += sum0 + sum1;
-        tmem_wait_st();
-        tc_fence_before();
+        {
+          uint8_t* dst = sP + ps * DecCfg::kPBytes + (kt >> 6) * 2048;
+          const uint32_t col = (uint32_t)(kt & 63);
+#pragma unroll
+          for (int q = 0; q < GP; ++q) {
+            ps_w[q] = (q < G) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
+            *reinterpret_cast<__nv_bfloat16*>(dst + sw128_offset((uint32_t)q, col)) = __float2bfloat16_rn(ps_w[q]);
+          }
+        }
+        fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_full[g & 1]);
+        if (lane == 0) mbar_arrive(&p_full[ps]);
+        // this warp's per-head sums of the tile (fp32, before the bf16 cast); they travel with the next exchange
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1)
+#pragma unroll
+          for (int q = 0; q < GP; ++q) ps_w[q] += __shfl_xor_sync(0xffffffffu, ps_w[q], s);
+        pending_sum = true;
         ++r;
         ++rg;
       }
       if (!ok) break;
+      if (pending_sum) {   // the sums of the last retained tile
+        float none[GP], dummy[GP];
+#pragma unroll
+        for (int q = 0; q < GP; ++q) none[q] = -INFINITY;
+        ok = exchange(none, dummy);
+        if (!ok) break;
+      }
       // partial output of this item once its last PV has retired: O / l in fp32 and the log-normalizer
       ok = mbar_wait(&item_done[ip], (ne >> 1) & 1, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const float inv = 1.f / l;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t o[32];
-        tmem_ld_x32(tmem_addr(tb, 0, colO + c * 32), o);
+      {
+        uint32_t o[16];
+        tmem_ld_x16(tmem_addr(tb, lane_base, colO), o);
         tmem_wait_ld();
-        if (c == 3) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&o_free[ip]);   // the accumulator may take the item after next
-        }
-        if (valid) {
-          float4* dst = reinterpret_cast<float4*>(p.o_part + prow * 128 + c * 32);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&o_free[ip]);   // the accumulator may take the item after next
 #pragma unroll
-          for (int v = 0; v < 8; ++v)
-            dst[v] = make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
-                                 __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
-        }
+        for (int q = 0; q < GP; ++q)
+          if (q < G) p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = __uint_as_float(o[q]) / l[q];
       }
-      if (valid) p.lse_part[prow] = (m_ref + log2f(l)) * 0.6931471805599453f;
-      if (lane == 0) {
+#pragma unroll
+      for (int q = 0; q < GP; ++q)
+        if (q < G && kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = (m_ref[q] + lgl[q]) * 0.6931471805599453f;
+      if (head) {
         if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
         if (p.retained) p.retained[stat_row] = (uint32_t)r;
         if (p.totals) {
@@ -438,7 +497,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tb, 512);
+  if (warp == 0) tmem_dealloc(tb, DecCfg::kTmemCols);
 }
 
 }  // namespace mala
