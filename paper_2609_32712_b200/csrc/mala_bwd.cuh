@@ -377,6 +377,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           retain = (*(volatile int*)&flag[slot]) != 0;
         }
       }
+      if (!kDense) retain = __all_sync(0xffffffffu, retain);   // same value in every lane: the branch below is uniform
       if (stat_thread && first_of_head) { r_head = 0; bm_bits = 0; bm_word = -1; }
       if (retain) {
         if (stat_thread) {

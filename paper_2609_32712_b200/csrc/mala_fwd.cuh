@@ -331,6 +331,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           retain = (*(volatile int*)&flag[x][t % 3]) != 0;
         }
       }
+      if (!kDense) retain = __all_sync(0xffffffffu, retain);   // same value in every lane: the branch below is uniform
       if (!retain) {   // m, l, O unchanged; no exp, no P, no PV: take the turn (see below) and pass it on at once
         if (!kDense && hasB) {
           const int idx = (x == 0) ? t : (t - 1 - firstA);
@@ -355,11 +356,12 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // Lazy rescaling: the reference maximum only moves when the row maximum grew by more than 2^8.
       // The scores of this tile were produced after every earlier PV of this block (same tensor pipe,
       // program order), so O may be touched here without a further wait.
+      // (warp votes stay out of conditional code: there the compiler has to re-converge the warp around each of them)
+      const bool need_any = __any_sync(0xffffffffu, r > 0 && mt > m_ref + 8.f);
       if (r == 0) {
         m_ref = mt;
       } else {
-        const bool need = mt > m_ref + 8.f;
-        if (__any_sync(0xffffffffu, need)) {
+        if (need_any) {
           const float m_new = fmaxf(m_ref, mt);
           const float alpha = fast_exp2(m_ref - m_new);
           l *= alpha;
@@ -382,13 +384,12 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // A's tile t follows B's tile of the same key step (t + firstA); B's tile t follows A's tile of the previous
       // step (t - 1 - firstA).  turn_bar[0] counts B's finished exp phases from tile firstA on, turn_bar[1] A's, so
       // every waiter sees the phases in sequence.
-      if (hasB) {
+      {
         const int idx = (x == 0) ? t : (t - 1 - firstA);
-        if (idx >= 0) {
-          ok = mbar_wait(&turn_bar[x], idx & 1, status);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
+        bool okw = true;
+        if (hasB && idx >= 0) okw = mbar_wait(&turn_bar[x], idx & 1, status);
+        ok = __all_sync(0xffffffffu, okw);
+        if (!ok) break;
       }
       // P = exp2(s * c2 - m_ref), row sum in fp32 before the bf16 cast, P written over S
       const float nm = -m_ref;
