@@ -306,6 +306,32 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     int g = 0, ne = 0, rg = 0;                     // global tile counter, non-empty item ordinal, retained tiles so far
     uint32_t xc = 0;                               // exchanges so far (buffer xc & 1, barrier phase xc & 1)
     bool ok = true;
+    // The partial output of an item needs its last PV, which trails this group by the V copies still in flight; it
+    // is therefore written two tiles into the NEXT item (or at that item's end), not where the item ends: the
+    // group never drains the pipeline at an item boundary.  Only O / l is deferred; everything else is known.
+    bool pend = false;
+    int pend_ip = 0, pend_ne = 0;
+    size_t pend_prow0 = 0;
+    float pend_l[GP];
+#pragma unroll
+    for (int q = 0; q < GP; ++q) pend_l[q] = 1.f;
+    auto flush = [&]() -> bool {
+      bool k = mbar_wait(&item_done[pend_ip], (uint32_t)((pend_ne >> 1) & 1), status);
+      k = __all_sync(0xffffffffu, k);
+      if (!k) return false;
+      tc_fence_after();
+      uint32_t o[16];
+      tmem_ld_x16(tmem_addr(tb, lane_base, DecCfg::kColO + (uint32_t)pend_ip * 16u), o);
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&o_free[pend_ip]);   // the accumulator may take the item after next
+#pragma unroll
+      for (int q = 0; q < GP; ++q)
+        if (q < G) p.o_part[(pend_prow0 + (size_t)q * p.num_splits) * 128 + kt] = __uint_as_float(o[q]) / pend_l[q];
+      pend = false;
+      return true;
+    };
     for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
       int b, hkv, split, T, j0;
       geometry(item, b, hkv, split, T, j0);
@@ -352,6 +378,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         return true;
       };
       for (int t = 0; t < T; ++t, ++g) {
+        if (pend && t == 2) { ok = flush(); if (!ok) break; }
         const int sb = g & 3;
         ok = mbar_wait(&s_full[sb], (uint32_t)((g >> 2) & 1), status);
         ok = __all_sync(0xffffffffu, ok);
@@ -464,22 +491,14 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         ok = exchange(none, dummy);
         if (!ok) break;
       }
-      // partial output of this item once its last PV has retired: O / l in fp32 and the log-normalizer
-      ok = mbar_wait(&item_done[ip], (ne >> 1) & 1, status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      {
-        uint32_t o[16];
-        tmem_ld_x16(tmem_addr(tb, lane_base, colO), o);
-        tmem_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&o_free[ip]);   // the accumulator may take the item after next
+      // the log-normalizer and the telemetry now; O / l (see above) once the item's last PV has retired
+      if (pend) { ok = flush(); if (!ok) break; }   // (a short item: the previous one is still pending)
+      pend = true;
+      pend_ip = ip;
+      pend_ne = ne;
+      pend_prow0 = prow0;
 #pragma unroll
-        for (int q = 0; q < GP; ++q)
-          if (q < G) p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = __uint_as_float(o[q]) / l[q];
-      }
+      for (int q = 0; q < GP; ++q) pend_l[q] = l[q];
 #pragma unroll
       for (int q = 0; q < GP; ++q)
         if (q < G && kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = (m_ref[q] + lgl[q]) * 0.6931471805599453f;
@@ -493,6 +512,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       }
       ++ne;
     }
+    if (ok && pend) flush();
   }
 
   tc_fence_before();
