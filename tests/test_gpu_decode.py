@@ -53,6 +53,15 @@ def test_decode_literal(mala, oracle, Nk, S, Hq, Hkv, tau):
     _run_and_check(mala, oracle, w, tau, S)
 
 
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv", [(300, 2, 6, 2), (2048, 16, 16, 1), (8192, 64, 10, 2), (1536, 4, 3, 1)])
+def test_decode_group_sizes_and_short_items(mala, oracle, Nk, S, Hq, Hkv, tau):
+    """Group sizes that are not powers of two (3, 5), the largest one (16), and more work items than SMs with one or
+    two tiles each (the partial output of an item is then written at the end of the next item)."""
+    w = W.custom_decode(2, Hq, Hkv, Nk, 128, S, seed=Nk + S + Hq)
+    _run_and_check(mala, oracle, w, tau, S)
+
+
 @pytest.mark.parametrize("tau", [1e-4, 1.0])
 @pytest.mark.parametrize("Nk,S", [(8192, 8), (8192, 2), (5000, 4)])
 def test_decode_gated_keys_skip_value_tiles(mala, oracle, Nk, S, tau):
