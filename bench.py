@@ -7,7 +7,8 @@ another).  `value` is dense-equivalent TFLOP/s of fwd+bwd (FullAttn FLOP model: 
 2.5x that backward) with inputs resident in HBM; `e2e` is the same metric with pinned-host inputs copied
 in and results copied out every step.  The line also carries, under `detail`, fwd / bwd latency of the
 MALA and dense kernels on cfg3 / cfg4 (literal and paper-regime "R" inputs), decode latency on cfg5
-(literal and gated "D" inputs) and the skipped-tile fractions.
+(literal and gated "D" inputs), the skipped-tile fractions, and for cfg3 R and cfg5 D the work / fidelity
+figures (retained slots, omitted mass, relative L2 against the dense path) at tau = 1e-4, 1e-2 and 1.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 """
@@ -175,6 +176,41 @@ class PrefillCase:
 
     def input_bytes(self):
         return sum(t.numel() * t.element_size() for t in (self.q, self.k, self.v, self.do))
+
+
+def fidelity(cs, taus, it):
+    """Work and operator fidelity of MALA against the in-library dense path on one configuration (the protocol
+    of Section 5.1 on synthetic states): retained slots per query in forward and backward, omitted softmax mass
+    eps = 1 - exp(lse_tau - lse_0) (bounded by tau / (1 + tau), Proposition 1), and relative L2 distance of O
+    and of dQ, dK, dV under a Rademacher upstream gradient."""
+    import torch
+    from paper_2609_32712_b200 import workloads as W
+    cc = cs.cfg
+    do_saved = cs.do
+    cs.do = W.rademacher_like(cs.q, seed=1000 + cc.seed)
+    cs.fwd(0.0)
+    cs.bwd(0.0)
+    ref = {n: getattr(cs, n).float() for n in ("o", "dq", "dk", "dv")}
+    nrm = {n: float(t.norm()) for n, t in ref.items()}
+    lse0 = cs.lse.clone()
+    dense_ms = (time_cuda(lambda: cs.fwd(0.0), 3, it), time_cuda(lambda: cs.bwd(0.0), 3, it))
+    rows = {}
+    for t_ in taus:
+        st = cs.tile_stats(t_)                      # leaves the MALA o, lse and gradients in the case's buffers
+        eps = 1.0 - torch.exp(cs.lse - lse0)
+        row = {"fwd_slots_per_query": st["fwd_retained"] * TILE * TILE / (cc.B * cc.Hq * cc.N),
+               "bwd_slots_per_query": st["bwd_retained"] * TILE * TILE / (cc.B * cc.Hq * cc.N),
+               "fwd_retained_frac": st["fwd_retained"] / st["fwd_legal"],
+               "bwd_retained_frac": st["bwd_retained"] / st["bwd_legal"],
+               "omitted_mass_max": float(eps.max()), "omitted_mass_mean": float(eps.mean()),
+               "omitted_mass_bound": t_ / (1.0 + t_)}
+        for n in ("o", "dq", "dk", "dv"):
+            row[f"rel_l2_{n}"] = float((getattr(cs, n).float() - ref[n]).norm()) / nrm[n]
+        f_ms, b_ms = time_cuda(lambda: cs.fwd(t_), 3, it), time_cuda(lambda: cs.bwd(t_), 3, it)
+        row.update(fwd_ms=f_ms, bwd_ms=b_ms, speedup_fwd=dense_ms[0] / f_ms, speedup_bwd=dense_ms[1] / b_ms)
+        rows[f"tau={t_:g}"] = row
+    cs.do = do_saved
+    return rows
 
 
 def oracle_sample(case, tau, o_gpu, lse_gpu):
@@ -394,6 +430,8 @@ def main():
                                                       / (row["mala"]["bwd_ms"] * 1e-3) / 1e12 / peaks["tflops_sustained"])
                 row["speedup_fwd"] = row["dense"]["fwd_ms"] / row["mala"]["fwd_ms"]
                 row["speedup_bwd"] = row["dense"]["bwd_ms"] / row["mala"]["bwd_ms"]
+                if name == "cfg3" and preset == "R":
+                    row["fidelity_vs_dense"] = fidelity(cs, (1e-4, 1e-2, 1.0), it)
                 detail[f"{name}_{preset}"] = row
                 if cs is not case:
                     del cs
@@ -418,6 +456,19 @@ def main():
                               "achieved_gbs": need / (us * 1e-6) / 1e9,
                               "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
             row["speedup"] = row["dense"]["us"] / row["mala"]["us"]
+            if preset == "D":                       # work and fidelity against the dense decode, tau up to 1
+                o0, lse0, _ = mala.decode(qd, kc, vc, wd["scale"], 0.0, dcfg.num_splits, ws=wsd)
+                o0, fid = o0.float(), {}
+                for t_ in (1e-4, 1e-2, 1.0):
+                    ot, lset, st = mala.decode(qd, kc, vc, wd["scale"], t_, dcfg.num_splits, ws=wsd, stats=True)
+                    ret, leg = st.totals.cpu().tolist()
+                    us = 1e3 * time_cuda(lambda: mala.decode(qd, kc, vc, wd["scale"], t_, dcfg.num_splits, ws=wsd,
+                                                              out=od, want_lse=False), 25, 100)
+                    fid[f"tau={t_:g}"] = {"us": us, "retained_frac": ret / leg,
+                                          "rel_l2_o": float((ot.float() - o0).norm() / o0.norm()),
+                                          "omitted_mass_max": float((1.0 - torch.exp(lset - lse0)).max()),
+                                          "speedup": row["dense"]["us"] / us}
+                row["fidelity_vs_dense"] = fid
             detail[f"cfg5_{preset}"] = row
             del wd, qd, kc, vc, wsd
             torch.cuda.empty_cache()

@@ -214,6 +214,14 @@ def make_decode(cfg: DecodeConfig, preset: str = "literal", device="cpu", seed: 
     return dict(q=q.to(bf), kcache=kc, vcache=vc, scale=cfg.scale, cfg=cfg, preset=preset)
 
 
+def rademacher_like(t: torch.Tensor, seed: int) -> torch.Tensor:
+    """Upstream gradient of +-1 entries (the Rademacher probe of the operator-fidelity protocol, Section 5.1)."""
+    gen = torch.Generator(device=t.device)
+    gen.manual_seed(seed)
+    bits = torch.randint(0, 2, t.shape, generator=gen, device=t.device, dtype=torch.int8)
+    return (bits * 2 - 1).to(t.dtype)
+
+
 def custom_prefill(B, Hq, Hkv, N, d, head_types=None, planted=4, seed=0, preset="literal", device="cpu"):
     """Small / odd-shaped cases for tests (any N, including ragged tails)."""
     if head_types is None:
