@@ -365,11 +365,13 @@ int mala_oracle_decode_tiles_per_split(int Nk, int num_splits, int Bk) {
   return (per + Bk - 1) / Bk;
 }
 
-int mala_oracle_decode_splits(const double* Q, const double* K, const double* V, int R, int Nk, int d,
-                              double scale, double tau, int num_splits, int Bk, double* o_part,
-                              double* lse_part, uint8_t* mask, double* crit) {
-  if (R <= 0 || Nk <= 0 || d <= 0 || num_splits <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
-  const int tps = mala_oracle_decode_tiles_per_split(Nk, num_splits, Bk);
+/* The same with the chunk length given (tps tiles of B_k keys per split) instead of derived from N_k: a batch
+ * of sequences of different lengths shares one layout of splits over the key positions, and a sequence shorter
+ * than a split's first position leaves that split empty.  N_k = 0 is allowed (every split empty). */
+int mala_oracle_decode_splits_tps(const double* Q, const double* K, const double* V, int R, int Nk, int d,
+                                  double scale, double tau, int num_splits, int tps, int Bk, double* o_part,
+                                  double* lse_part, uint8_t* mask, double* crit) {
+  if (R <= 0 || Nk < 0 || d <= 0 || num_splits <= 0 || tps <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
   const int chunk = tps * Bk;
   const double theta = log_threshold(tau, (double)Nk); /* L_0 = N_k, current token included */
 #pragma omp parallel for schedule(dynamic, 1)
@@ -432,6 +434,15 @@ int mala_oracle_decode_splits(const double* Q, const double* K, const double* V,
     free(m); free(l); free(acc); free(S); free(mt);
   }
   return 0;
+}
+
+int mala_oracle_decode_splits(const double* Q, const double* K, const double* V, int R, int Nk, int d,
+                              double scale, double tau, int num_splits, int Bk, double* o_part,
+                              double* lse_part, uint8_t* mask, double* crit) {
+  if (Nk <= 0 || num_splits <= 0 || Bk <= 0) return -1;
+  return mala_oracle_decode_splits_tps(Q, K, V, R, Nk, d, scale, tau, num_splits,
+                                       mala_oracle_decode_tiles_per_split(Nk, num_splits, Bk), Bk, o_part, lse_part,
+                                       mask, crit);
 }
 
 /* Normalizer-aware reduction of the split partials:

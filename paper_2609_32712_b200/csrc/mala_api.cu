@@ -256,6 +256,34 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
                        (cudaStream_t)cuda_stream);
 }
 
+int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* block_table,
+                      const int32_t* seqlens, mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq,
+                      int Hkv, int num_pages, int page_size, int max_pages_per_seq, int d, float scale, float tau,
+                      int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
+  if (page_size % 128 != 0 || (long long)max_pages_per_seq * page_size > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
+  const int Nk = max_pages_per_seq * page_size;   // the longest cache a sequence can hold
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  if (num_splits <= 0 || !ws) return MALA_ERR_INVALID_ARG;
+  if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  if ((((uintptr_t)block_table) & 3) != 0 || (((uintptr_t)seqlens) & 3) != 0) return MALA_ERR_MISALIGNED;
+  MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
+  MALA_TRY(check_view(kpages.p, kpages.sb, kpages.sn, kpages.sh, num_pages, page_size, Hkv));
+  MALA_TRY(check_view(vpages.p, vpages.sb, vpages.sn, vpages.sh, num_pages, page_size, Hkv));
+  MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
+  if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
+  if (ws_bytes < decode_workspace_bytes(B, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  DecPaging pg;
+  pg.block_table = block_table; pg.seqlens = seqlens; pg.bt_stride = max_pages_per_seq; pg.page_size = page_size;
+  pg.num_pages = num_pages;
+  return decode_launch(q, kpages, vpages, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
+                       (cudaStream_t)cuda_stream, &pg);
+}
+
 int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, int B, int Hq,
                        int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* cuda_stream) {
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));

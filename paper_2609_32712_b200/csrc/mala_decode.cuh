@@ -28,8 +28,9 @@ decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ 
     Z += w;
     acc += w * o_part[((size_t)bh * num_splits + s) * D + c];
   }
-  o[b * o_sb + h * o_sh + c] = __float2bfloat16(acc / Z);
-  if (lse_out && c == 0) lse_out[bh] = mx + logf(Z);
+  // (a sequence without keys has no split with mass: its output is 0 and its log-normalizer -inf)
+  o[b * o_sb + h * o_sh + c] = __float2bfloat16(Z > 0.f ? acc / Z : 0.f);
+  if (lse_out && c == 0) lse_out[bh] = Z > 0.f ? mx + logf(Z) : -INFINITY;
 }
 
 inline size_t decode_align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -48,13 +49,24 @@ inline bool decode_set_attributes() {
   return ok;
 }
 
+// A cache held in pages: kc / vc are [num_pages, page_size, Hkv, d] (sb = page stride), sequence b keeps its keys
+// 128*x .. in page block_table[b * bt_stride + x / (page_size / 128)], and holds seqlens[b] <= Nk keys.
+struct DecPaging {
+  const int* block_table;   // null: one contiguous cache per sequence
+  const int* seqlens;       // null: every sequence holds Nk keys
+  int bt_stride, page_size, num_pages;
+};
+
 // Launches the split kernel and the merge on `stream`.  o_part / lse_part: caller-provided scratch of
-// decode_workspace_bytes() bytes in total (o_part first).
+// decode_workspace_bytes() bytes in total (o_part first).  Nk: the longest cache (the splits are laid out for it).
 inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala_tout o, float* lse_opt,
                                       const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                                       float tau, int num_splits, float* o_part, float* lse_part, int* status,
-                                      cudaStream_t stream) {
+                                      cudaStream_t stream, const DecPaging* pg = nullptr) {
   if (d != 128) return MALA_ERR_UNSUPPORTED;
+  const bool paged = pg && pg->block_table;
+  if (paged && (pg->page_size <= 0 || pg->page_size % 128 != 0 || pg->num_pages <= 0 || pg->bt_stride <= 0))
+    return MALA_ERR_UNSUPPORTED;
   const int per = (Nk + num_splits - 1) / num_splits;
   const int tps = (per + 127) / 128;
   if ((long long)B * Hkv * num_splits > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
@@ -62,8 +74,10 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   CUtensorMap tq, tk, tv;
   // q [B,1,Hq,d] viewed with the heads as rows: one 16-row box starting at the group's first head
   if (!make_tensor_map_bnhd(&tq, q.p, B, Hq, 1, d, q.sb, q.sh, 0, 16) ||
-      !make_tensor_map_bnhd(&tk, kc.p, B, Nk, Hkv, d, kc.sb, kc.sn, kc.sh, 128) ||
-      !make_tensor_map_bnhd(&tv, vc.p, B, Nk, Hkv, d, vc.sb, vc.sn, vc.sh, 128))
+      !make_tensor_map_bnhd(&tk, kc.p, paged ? pg->num_pages : B, paged ? pg->page_size : Nk, Hkv, d, kc.sb, kc.sn,
+                            kc.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, vc.p, paged ? pg->num_pages : B, paged ? pg->page_size : Nk, Hkv, d, vc.sb, vc.sn,
+                            vc.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
   DecParams p;
@@ -72,6 +86,10 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   p.bitmask = st ? st->tile_bitmask : nullptr;
   p.totals = st ? (unsigned long long*)st->totals : nullptr;
   p.status = status;
+  p.seqlens = pg ? pg->seqlens : nullptr;
+  p.block_table = paged ? pg->block_table : nullptr;
+  p.bt_stride = paged ? pg->bt_stride : 0;
+  p.tpp = paged ? pg->page_size / 128 : 1;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Nk = Nk; p.tps = tps; p.num_splits = num_splits; p.words = (tps + 31) / 32;
   p.n_items = B * Hkv * num_splits;
   p.scale_log2 = scale * 1.4426950408889634f;
@@ -105,11 +123,11 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
 
 inline int decode_launch(mala_tin q, mala_tin kc, mala_tin vc, mala_tout o, float* lse_opt, const mala_stats* st, int B,
                          int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws, int* status,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, const DecPaging* pg = nullptr) {
   float* o_part = (float*)ws;
   float* lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Hq * num_splits * d * sizeof(float)));
   return decode_launch_with_scratch(q, kc, vc, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, o_part,
-                                    lse_part, status, stream);
+                                    lse_part, status, stream, pg);
 }
 
 }  // namespace mala

@@ -33,7 +33,11 @@ struct DecParams {
   uint32_t* bitmask;             // [B, Hkv, num_splits, words] or null (zero-filled by the host)
   unsigned long long* totals;    // [2] or null
   int* status;
-  int B, Hq, Hkv, Nk, tps, num_splits, words, n_items;
+  // Paged / variable-length caches (both null for one contiguous cache of Nk keys per sequence):
+  const int* seqlens;            // [B] keys held by sequence b (<= Nk); L = seqlens[b] for its rows
+  const int* block_table;        // [B, bt_stride] page of the tpp consecutive tiles number x*tpp .. x*tpp + tpp - 1
+  int bt_stride, tpp;            // tpp: tiles per page (page size / 128)
+  int B, Hq, Hkv, Nk, tps, num_splits, words, n_items;   // Nk: longest cache the splits are laid out for
   float scale_log2, log2_tau;
 };
 
@@ -66,6 +70,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       vote_bar[4], p_full[4], p_free[4], item_done[2], o_free[2], fin_bar, grp_a;
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[4];
+  __shared__ int v_row[8], v_outer[8];     // TMA coordinates of the V tile of tile g (ring; written by the producer)
   __shared__ float xch_max[2][4][16], xch_sum[2][4][16];   // the softmax group's per-tile exchange
   __shared__ int early_exit;
 
@@ -97,16 +102,29 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
 
-  // geometry of work item `item`: batch, KV head, split, number of legal tiles, newest key block
-  auto geometry = [&](int item, int& b, int& hkv, int& split, int& T, int& j0) {
+  // geometry of work item `item`: batch, KV head, split, number of legal tiles, newest key block, keys of the
+  // sequence
+  auto geometry = [&](int item, int& b, int& hkv, int& split, int& T, int& j0, int& nk) {
     split = item % p.num_splits;
     const int bh = item / p.num_splits;
     hkv = bh % p.Hkv;
     b = bh / p.Hkv;
+    nk = p.seqlens ? min(p.Nk, max(0, __ldg(p.seqlens + b))) : p.Nk;
     const int lo = split * p.tps * 128;
-    const int hi = min(p.Nk, lo + p.tps * 128);
+    const int hi = min(nk, lo + p.tps * 128);
     T = hi > lo ? (hi - lo + 127) / 128 : 0;
     j0 = lo / 128 + T - 1;
+  };
+  // TMA coordinates (key row, outermost index) of key block jt of sequence b
+  auto tile_coord = [&](int b, int jt, int& row, int& outer) {
+    if (p.block_table) {
+      const int pg = jt / p.tpp;
+      outer = __ldg(p.block_table + (size_t)b * p.bt_stride + pg);
+      row = (jt - pg * p.tpp) * 128;
+    } else {
+      outer = b;
+      row = jt * 128;
+    }
   };
 
   if (warp == 0) {
@@ -114,12 +132,13 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
       int ne = 0;                               // ordinal of the non-empty item
+      int g = 0;                                // global tile counter
       int ks = 0, vs = 0;
       uint32_t kpar = 1, vpar = 1;              // "empty" parities (first pass: free)
       bool ok = true;
       for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-        int b, hkv, split, T, j0;
-        geometry(item, b, hkv, split, T, j0);
+        int b, hkv, split, T, j0, nk;
+        geometry(item, b, hkv, split, T, j0, nk);
         if (T == 0) continue;
         const int ip = ne & 1;
         ok = mbar_wait(&q_empty[ip], ((ne >> 1) & 1) ^ 1, status);
@@ -127,19 +146,25 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         mbar_arrive_expect_tx(&q_full[ip], DecCfg::kQBytes);
         tma_load_4d(sQ + ip * DecCfg::kQBytes, &tmQ, &q_full[ip], 0, hkv * G, 0, b);
         tma_load_4d(sQ + ip * DecCfg::kQBytes + 2048, &tmQ, &q_full[ip], 64, hkv * G, 0, b);
-        for (int t = 0; t < T && ok; ++t) {
+        for (int t = 0; t < T && ok; ++t, ++g) {
+          int row, outer;
+          tile_coord(b, j0 - t, row, outer);     // (a page lookup is in flight while the slot is waited for)
           ok = mbar_wait(&k_empty[ks], kpar, status);
           if (!ok) break;
+          // The UMMA warp requests V of tile g from these coordinates after the vote.  It cannot be more than six
+          // tiles behind this one (K ring of three behind the S^T cursor, vote cursor at most four behind that),
+          // and it sees the two stores through the K tile's barrier.
+          if (!kDense) { v_row[g & 7] = row; v_outer[g & 7] = outer; }
           mbar_arrive_expect_tx(&k_full[ks], TB);
-          tma_load_4d(sK + ks * TB, &tmK, &k_full[ks], 0, (j0 - t) * 128, hkv, b);
-          tma_load_4d(sK + ks * TB + 16384, &tmK, &k_full[ks], 64, (j0 - t) * 128, hkv, b);
+          tma_load_4d(sK + ks * TB, &tmK, &k_full[ks], 0, row, hkv, outer);
+          tma_load_4d(sK + ks * TB + 16384, &tmK, &k_full[ks], 64, row, hkv, outer);
           if (++ks == KS) { ks = 0; kpar ^= 1; }
           if (kDense) {   // every tile is retained: V follows K
             ok = mbar_wait(&v_empty[vs], vpar, status);
             if (!ok) break;
             mbar_arrive_expect_tx(&v_full[vs], TB);
-            tma_load_4d(sV + vs * TB, &tmV, &v_full[vs], 0, (j0 - t) * 128, hkv, b);
-            tma_load_4d(sV + vs * TB + 16384, &tmV, &v_full[vs], 64, (j0 - t) * 128, hkv, b);
+            tma_load_4d(sV + vs * TB, &tmV, &v_full[vs], 0, row, hkv, outer);
+            tma_load_4d(sV + vs * TB + 16384, &tmV, &v_full[vs], 64, row, hkv, outer);
             if (++vs == VS) { vs = 0; vpar ^= 1; }
           }
         }
@@ -165,8 +190,8 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         c.valid = false;
         c.g = g;
         for (int item = from; item < p.n_items; item += gridDim.x) {
-          int b, hkv, split, T, j0;
-          geometry(item, b, hkv, split, T, j0);
+          int b, hkv, split, T, j0, nk;
+          geometry(item, b, hkv, split, T, j0, nk);
           if (T > 0) { c.item = item; c.ne = ne; c.t = 0; c.T = T; c.b = b; c.hkv = hkv; c.j0 = j0; c.valid = true; return; }
         }
       };
@@ -226,9 +251,10 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
               progress = true;
             } else if (ready(&v_empty[vi], vipar)) {   // V of this tile, on demand
               if (leader) {
+                const int row = *(volatile int*)&v_row[cv.g & 7], outer = *(volatile int*)&v_outer[cv.g & 7];
                 mbar_arrive_expect_tx(&v_full[vi], TB);
-                tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, (cv.j0 - cv.t) * 128, cv.hkv, cv.b);
-                tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, (cv.j0 - cv.t) * 128, cv.hkv, cv.b);
+                tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, row, cv.hkv, outer);
+                tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, row, cv.hkv, outer);
               }
               __syncwarp();
               if (++vi == VS) { vi = 0; vipar ^= 1; }
@@ -297,7 +323,6 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     for (int i = kt; i < DecCfg::kPStages * DecCfg::kPBytes / 16; i += 128) reinterpret_cast<uint4*>(sP)[i] = make_uint4(0u, 0u, 0u, 0u);
     fence_proxy_async_smem();
     const float c2 = p.scale_log2;
-    const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)p.Nk));
     const bool head = (kt == 0);                   // the thread that keeps the telemetry
     // The reference of the exponentials follows the scores only when they exceed it by 2^60: fp32 sums and bf16 P
     // have the exponent range for it, and moving the reference means waiting until every PV issued so far has
@@ -333,8 +358,9 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       return true;
     };
     for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-      int b, hkv, split, T, j0;
-      geometry(item, b, hkv, split, T, j0);
+      int b, hkv, split, T, j0, nk;
+      geometry(item, b, hkv, split, T, j0, nk);
+      const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)nk));   // L = keys of the sequence
       const size_t prow0 = ((size_t)b * p.Hq + hkv * G) * p.num_splits + split;   // head q: + q * num_splits
       const size_t stat_row = (size_t)(b * p.Hkv + hkv) * p.num_splits + split;
       if (T == 0) {   // empty split: (0, -inf)
@@ -390,7 +416,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_free[sb]);     // the scores are in registers
-        const bool key_ok = ((j0 - t) * 128 + kt) < p.Nk;   // only the newest tile of the split can be ragged
+        const bool key_ok = ((j0 - t) * 128 + kt) < nk;   // only the newest tile of the split can be ragged
         float x[GP], mx[GP], tmax[GP];
 #pragma unroll
         for (int q = 0; q < GP; ++q) { x[q] = (key_ok && q < G) ? __uint_as_float(sr[q]) * c2 : -INFINITY; mx[q] = x[q]; }

@@ -214,6 +214,34 @@ def make_decode(cfg: DecodeConfig, preset: str = "literal", device="cpu", seed: 
     return dict(q=q.to(bf), kcache=kc, vcache=vc, scale=cfg.scale, cfg=cfg, preset=preset)
 
 
+def paginate(kcache: torch.Tensor, vcache: torch.Tensor, page_size: int, seqlens=None, seed: int = 0,
+             spare_pages: int = 3):
+    """Serving-side layout of a decode workload: the contiguous caches [B,Nk,Hkv,d] are cut into pages of
+    ``page_size`` keys that are scattered over a shuffled pool of B*ceil(Nk/page_size) + spare_pages pages.
+    Slots that no sequence uses (beyond ``seqlens[b]``, spare pages) hold finite junk, and block-table entries of
+    pages a sequence does not reach point outside the pool.  Returns (kpages, vpages, block_table int32
+    [B, max_pages], seqlens int32 [B])."""
+    B, Nk, Hkv, d = kcache.shape
+    dev = kcache.device
+    mp = -(-Nk // page_size)
+    pool = B * mp + spare_pages
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    perm = torch.randperm(pool, generator=gen)
+    lens = [Nk] * B if seqlens is None else [int(x) for x in seqlens]
+    kp = (8.0 * torch.randn((pool, page_size, Hkv, d), generator=gen)).to(kcache.dtype).to(dev)
+    vp = (8.0 * torch.randn((pool, page_size, Hkv, d), generator=gen)).to(vcache.dtype).to(dev)
+    bt = torch.full((B, mp), pool + 5, dtype=torch.int32)
+    for b in range(B):
+        for x in range(-(-lens[b] // page_size)):
+            n = min(page_size, lens[b] - x * page_size)
+            pg = int(perm[b * mp + x])
+            bt[b, x] = pg
+            kp[pg, :n] = kcache[b, x * page_size:x * page_size + n]
+            vp[pg, :n] = vcache[b, x * page_size:x * page_size + n]
+    return kp, vp, bt.to(dev), torch.tensor(lens, dtype=torch.int32, device=dev)
+
+
 def rademacher_like(t: torch.Tensor, seed: int) -> torch.Tensor:
     """Upstream gradient of +-1 entries (the Rademacher probe of the operator-fidelity protocol, Section 5.1)."""
     gen = torch.Generator(device=t.device)

@@ -89,3 +89,82 @@ def test_decode_strided_cache_view(mala, oracle):
     o, lse, _ = mala.decode(q, kc, vc, w["scale"], 0.0, 4)
     ref = oracle.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 0.0, 4, 128)
     parity.check_output(o.float().cpu().numpy()[:, 0], ref["o"])
+
+
+def _run_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0):
+    kp, vp, bt, lens = W.paginate(w["kcache"], w["vcache"], page_size, seqlens=seqlens, seed=seed)
+    q = w["q"].cuda()
+    B, _, Hq, d = q.shape
+    Hkv = kp.shape[2]
+    G = Hq // Hkv
+    o, lse, st = mala.decode_paged(q, kp.cuda(), vp.cuda(), bt.cuda(), lens.cuda() if seqlens is not None else None,
+                                   w["scale"], tau, num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    _, Bk = mala.tile_shape(mala.OP_DECODE, d)
+    ref = oracle.decode_paged(w["q"], kp, vp, bt.numpy(), lens.numpy() if seqlens is not None else None, w["scale"],
+                              tau, num_splits, Bk)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy()[:, 0], lse.cpu().numpy()
+    skipped = retained = 0
+    for b in range(B):
+        n = int(lens[b])
+        for g in range(Hkv):
+            for s in range(num_splits):
+                parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                                  tau, max(n, 1), Bk)
+                assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
+            hs = slice(g * G, (g + 1) * G)
+            parity.check_output(o_c[b, hs], ref["o"][b, hs])
+            if n > 0:
+                assert np.abs(lse_c[b, hs] - ref["lse"][b, hs]).max() <= parity.LSE_ABS
+            else:
+                assert np.isneginf(lse_c[b, hs]).all() and (o_c[b, hs] == 0).all()
+            skipped += int((ref["mask"][b, g] == 1).sum())
+            retained += int((ref["mask"][b, g] == 2).sum())
+    tot = st.totals.cpu().numpy()
+    assert tot[1] == retained + skipped
+    return dict(skipped=skipped, retained=retained)
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv,page,lens", [
+    (1024, 4, 8, 2, 128, None),                        # one tile per page, every sequence full
+    (2048, 4, 4, 1, 256, [2048, 1000, 129]),           # two tiles per page, ragged lengths, empty trailing splits
+    (1536, 3, 6, 2, 512, [1, 1536, 0, 700]),           # a split per page; one key; no key at all
+    (8192, 64, 8, 2, 128, [8192, 5000, 128, 3333]),    # more work items than SMs, one tile each
+])
+def test_decode_paged_literal(mala, oracle, Nk, S, Hq, Hkv, page, lens, tau):
+    B = 2 if lens is None else len(lens)
+    w = W.custom_decode(B, Hq, Hkv, Nk, 128, S, seed=Nk + S + page)
+    _run_paged(mala, oracle, w, tau, S, page, lens, seed=page)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+def test_decode_paged_gated_keys_skip_value_tiles(mala, oracle, tau):
+    w = W.custom_decode(3, 8, 2, 8192, 128, 8, group_types=["diffuse", "peaked"], seed=5, preset="D")
+    res = _run_paged(mala, oracle, w, tau, 8, 256, [8192, 4096 + 77, 2500], seed=9)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+
+
+def test_decode_paged_identity_table_equals_contiguous_call(mala):
+    # pages laid out in order are the contiguous cache: both entry points must give the same bits
+    w = W.custom_decode(2, 8, 2, 4096, 128, 8, group_types=["diffuse", "peaked"], seed=21, preset="D")
+    q, kc, vc = (w[x].cuda() for x in ("q", "kcache", "vcache"))
+    bt = torch.arange(2 * 16, dtype=torch.int32, device="cuda").reshape(2, 16)
+    for tau in (0.0, 1e-4):
+        o1, l1, s1 = mala.decode(q, kc, vc, w["scale"], tau, 8, stats=True)
+        o2, l2, s2 = mala.decode_paged(q, kc.reshape(32, 256, 2, 128), vc.reshape(32, 256, 2, 128), bt, None,
+                                       w["scale"], tau, 8, stats=True)
+        assert torch.equal(o1, o2) and torch.equal(l1, l2)
+        assert torch.equal(s1.retained, s2.retained)
+
+
+def test_decode_paged_rejects_pages_that_are_not_whole_tiles(mala):
+    q = torch.zeros((1, 1, 4, 128), dtype=torch.bfloat16, device="cuda")
+    pages = torch.zeros((4, 64, 1, 128), dtype=torch.bfloat16, device="cuda")
+    bt = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
+    with pytest.raises(mala.MalaError) as e:
+        mala.decode_paged(q, pages, pages, bt, None, 0.1, 0.0, 1)
+    assert e.value.code < 0

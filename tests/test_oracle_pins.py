@@ -478,3 +478,79 @@ def test_decode_ragged_cache_and_empty_trailing_split():
     dec2 = orc.decode(q, kc, vc, 0.4, 0.0, 8, 16)                # chunk = 16, splits 5..7 are empty
     assert np.isneginf(dec2["lse_part"][0, :, 5:]).all()
     assert np.allclose(dec["o"], dec2["o"], atol=1e-13)
+
+
+# ------------------------------------------------------------------ paged cache, one length per sequence
+def _paged_inputs(B, Nmax, d, G, page, lens, seed):
+    """Contiguous caches of B sequences cut into pages that are scattered over a shuffled pool; slots that no
+    sequence uses hold large finite junk."""
+    r = _rng(seed)
+    q = r.standard_normal((B, G, d))
+    kc = r.standard_normal((B, Nmax, 1, d))
+    vc = r.standard_normal((B, Nmax, 1, d))
+    live = r.random((B, Nmax)) < 0.1
+    kc[:, :, 0, d - 1] = np.where(live, 0.0, -6.0)
+    q[:, :, d - 1] = 6.0
+    mp = Nmax // page
+    pool = B * mp + 3
+    perm = r.permutation(pool)
+    kp = 50.0 * r.standard_normal((pool, page, 1, d))
+    vp = 50.0 * r.standard_normal((pool, page, 1, d))
+    bt = np.full((B, mp), pool + 5, dtype=np.int64)             # unused entries point outside the pool
+    for b in range(B):
+        for x in range(-(-lens[b] // page)):
+            n = min(page, lens[b] - x * page)
+            bt[b, x] = perm[b * mp + x]
+            kp[bt[b, x], :n] = kc[b, x * page:x * page + n]
+            vp[bt[b, x], :n] = vc[b, x * page:x * page + n]
+    return q, kc, vc, kp, vp, bt
+
+
+def test_decode_paged_tau_zero_is_softmax_over_each_sequences_own_keys():
+    lens = [64, 37, 5, 0]
+    q, kc, vc, kp, vp, bt = _paged_inputs(4, 64, 8, 2, 16, lens, 181)
+    dec = orc.decode_paged(q, kp, vp, bt, lens, 0.4, 0.0, 4, 8)
+    for b, n in enumerate(lens):
+        for h in range(2):
+            if n == 0:
+                assert (dec["o"][b, h] == 0).all() and np.isneginf(dec["lse"][b, h])
+                continue
+            e = np.exp(0.4 * kc[b, :n, 0] @ q[b, h])
+            assert np.allclose(dec["o"][b, h], (e / e.sum()) @ vc[b, :n, 0], atol=1e-12)
+            assert abs(dec["lse"][b, h] - math.log(e.sum())) < 1e-12
+    assert np.isneginf(dec["lse_part"][2, :, 1:]).all()            # 5 keys: only the first 16-key split is used
+
+
+@pytest.mark.parametrize("tau", [0.5, 1e-2])
+def test_decode_paged_equals_contiguous_rule_per_sequence(tau):
+    # 128 positions, 4 splits of 32 keys; a sequence of n keys must behave like a contiguous cache of n keys cut
+    # into the same 32-key chunks (L = n), wherever its pages lie in the pool
+    lens = [128, 96, 64, 51]
+    q, kc, vc, kp, vp, bt = _paged_inputs(4, 128, 8, 4, 16, lens, 191)
+    dec = orc.decode_paged(q, kp, vp, bt, lens, 0.5, tau, 4, 8)
+    assert (dec["mask"] == orc.SKIPPED).sum() > 0
+    for b, n in enumerate(lens):
+        S = -(-n // 32)
+        ref = orc.decode(q[b:b + 1], kc[b:b + 1, :n], vc[b:b + 1, :n], 0.5, tau, S, 8)
+        assert orc.lib().mala_oracle_decode_tiles_per_split(n, S, 8) == 4
+        assert np.array_equal(dec["mask"][b, :, :S], ref["mask"][0])
+        assert np.allclose(dec["lse_part"][b, :, :S], ref["lse_part"][0], atol=1e-13)
+        assert np.allclose(dec["o"][b], ref["o"][0], atol=1e-13)
+        assert np.allclose(dec["lse"][b], ref["lse"][0], atol=1e-13)
+        assert (dec["mask"][b, :, S:] == 0).all()
+
+
+def test_decode_paged_does_not_depend_on_where_pages_lie():
+    lens = [80, 33]
+    q, kc, vc, kp, vp, bt = _paged_inputs(2, 96, 8, 2, 16, lens, 201)
+    a = orc.decode_paged(q, kp, vp, bt, lens, 0.5, 0.3, 3, 8)
+    # the same sequences in an orderly pool: sequence b, page x -> pool page b * 6 + x
+    kp2 = np.zeros((12, 16, 1, 8))
+    vp2 = np.zeros((12, 16, 1, 8))
+    bt2 = np.arange(12).reshape(2, 6)
+    for b in range(2):
+        kp2[b * 6:(b + 1) * 6] = kc[b].reshape(6, 16, 1, 8)
+        vp2[b * 6:(b + 1) * 6] = vc[b].reshape(6, 16, 1, 8)
+    c = orc.decode_paged(q, kp2, vp2, bt2, lens, 0.5, 0.3, 3, 8)
+    for key in ("o", "lse", "mask", "lse_part"):
+        assert np.array_equal(a[key], c[key])
