@@ -302,14 +302,16 @@ def decode(q, kcache, vcache, scale: float, tau: float, num_splits: int, Bk: int
     return dict(o=o, lse=lse, mask=mask, crit=crit, o_part=o_part, lse_part=lse_part)
 
 
-def decode_paged(q, kpages, vpages, block_table, seqlens, scale: float, tau: float, num_splits: int, Bk: int):
+def decode_paged(q, kpages, vpages, block_table, seqlens, scale: float, tau: float, num_splits: int, Bk: int,
+                 units=None):
     """Split-KV decode over a paged cache with one length per sequence.
 
     q [B,Hq,d] (or [B,1,Hq,d]); kpages, vpages [num_pages, page_size, Hkv, d]; block_table [B, max_pages]
     (page of the keys page_size*x ..); seqlens [B] (None: every sequence holds max_pages*page_size keys).
     The cache of sequence b is put together page by page and cut off at its length; the decode rule then runs
     on it with L = seqlens[b].  All sequences share one layout of splits over the key positions, the one
-    ``decode`` derives for N_k = max_pages*page_size.  Returns what ``decode`` returns (packed rows).
+    ``decode`` derives for N_k = max_pages*page_size.  ``units``: optional list of (b, h_kv), other entries stay
+    zero.  Returns what ``decode`` returns (packed rows).
     """
     if len(q.shape) == 4:
         q = q[:, 0]
@@ -327,29 +329,30 @@ def decode_paged(q, kpages, vpages, block_table, seqlens, scale: float, tau: flo
     crit = np.full((B, Hkv, num_splits, tps), np.nan)
     o_part = np.zeros((B, Hq, num_splits, d))
     lse_part = np.zeros((B, Hq, num_splits))
-    kp, vp = _np(kpages), _np(vpages)
-    for b in range(B):
+    if units is None:
+        units = [(b, g) for b in range(B) for g in range(Hkv)]
+    for (b, g) in units:
         n = int(min(max(lens[b], 0), Nmax))
         npg = -(-n // page_size)
-        for g in range(Hkv):
-            K = np.ascontiguousarray(np.concatenate([kp[bt[b, x], :, g, :] for x in range(npg)], axis=0)[:n]) \
-                if npg else np.zeros((1, d))
-            V = np.ascontiguousarray(np.concatenate([vp[bt[b, x], :, g, :] for x in range(npg)], axis=0)[:n]) \
-                if npg else np.zeros((1, d))
-            Q = _np(q[b, g * G:(g + 1) * G, :])
-            op = np.zeros((num_splits, G, d))
-            lp = np.zeros((num_splits, G))
-            m = np.zeros((num_splits, tps), dtype=np.uint8)
-            c = np.full((num_splits, tps), np.nan)
-            _ck(lib().mala_oracle_decode_splits_tps(_p(Q), _p(K), _p(V), G, n, d, scale, tau, num_splits, tps, Bk,
-                                                    _p(op), _p(lp), _u8(m), _p(c)), "decode_splits_tps")
-            oo = np.zeros((G, d))
-            ll = np.zeros((G,))
-            _ck(lib().mala_oracle_decode_merge(_p(op), _p(lp), num_splits, G, d, _p(oo), _p(ll)), "decode_merge")
-            o[b, g * G:(g + 1) * G] = oo
-            lse[b, g * G:(g + 1) * G] = ll
-            o_part[b, g * G:(g + 1) * G] = op.transpose(1, 0, 2)
-            lse_part[b, g * G:(g + 1) * G] = lp.T
-            mask[b, g] = m
-            crit[b, g] = c
+        K = np.concatenate([_np(kpages[int(bt[b, x]), :, g, :]) for x in range(npg)], axis=0)[:n] \
+            if npg else np.zeros((1, d))
+        V = np.concatenate([_np(vpages[int(bt[b, x]), :, g, :]) for x in range(npg)], axis=0)[:n] \
+            if npg else np.zeros((1, d))
+        K, V = np.ascontiguousarray(K), np.ascontiguousarray(V)
+        Q = _np(q[b, g * G:(g + 1) * G, :])
+        op = np.zeros((num_splits, G, d))
+        lp = np.zeros((num_splits, G))
+        m = np.zeros((num_splits, tps), dtype=np.uint8)
+        c = np.full((num_splits, tps), np.nan)
+        _ck(lib().mala_oracle_decode_splits_tps(_p(Q), _p(K), _p(V), G, n, d, scale, tau, num_splits, tps, Bk,
+                                                _p(op), _p(lp), _u8(m), _p(c)), "decode_splits_tps")
+        oo = np.zeros((G, d))
+        ll = np.zeros((G,))
+        _ck(lib().mala_oracle_decode_merge(_p(op), _p(lp), num_splits, G, d, _p(oo), _p(ll)), "decode_merge")
+        o[b, g * G:(g + 1) * G] = oo
+        lse[b, g * G:(g + 1) * G] = ll
+        o_part[b, g * G:(g + 1) * G] = op.transpose(1, 0, 2)
+        lse_part[b, g * G:(g + 1) * G] = lp.T
+        mask[b, g] = m
+        crit[b, g] = c
     return dict(o=o, lse=lse, mask=mask, crit=crit, o_part=o_part, lse_part=lse_part)

@@ -21,6 +21,9 @@
 //   warps 4-7  softmax group, thread = key of the tile: per-head maxima and sums by warp shuffles and one small
 //              exchange per tile between the four warps, Eq. 3, P^T -> smem; lazy rescale of O^T
 // K is always streamed; a skipped tile issues no exp, no P, no V load and no PV.
+// The cache may be held in pages (pages of whole tiles, looked up in a block table by the producer, which hands
+// the V tile's coordinates to the UMMA warp) and every sequence may have its own length (which then takes the
+// place of Nk in the item geometry, in L and in the mask of the newest tile).
 #pragma once
 #include "sm100_ptx.cuh"
 

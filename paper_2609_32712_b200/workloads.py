@@ -229,8 +229,9 @@ def paginate(kcache: torch.Tensor, vcache: torch.Tensor, page_size: int, seqlens
     gen.manual_seed(seed)
     perm = torch.randperm(pool, generator=gen)
     lens = [Nk] * B if seqlens is None else [int(x) for x in seqlens]
-    kp = (8.0 * torch.randn((pool, page_size, Hkv, d), generator=gen)).to(kcache.dtype).to(dev)
-    vp = (8.0 * torch.randn((pool, page_size, Hkv, d), generator=gen)).to(vcache.dtype).to(dev)
+    # (one page of junk, repeated: the pool of a full-size cache has 10^9 slots)
+    kp = (8.0 * torch.randn((page_size, Hkv, d), generator=gen)).to(kcache.dtype).to(dev).repeat(pool, 1, 1, 1)
+    vp = (8.0 * torch.randn((page_size, Hkv, d), generator=gen)).to(vcache.dtype).to(dev).repeat(pool, 1, 1, 1)
     bt = torch.full((B, mp), pool + 5, dtype=torch.int32)
     for b in range(B):
         for x in range(-(-lens[b] // page_size)):

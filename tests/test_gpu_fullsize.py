@@ -131,3 +131,33 @@ def test_cfg5_decode_128k(mala, oracle, preset, tau):
         assert tot[0] < tot[1]
     if tau == 0.0:
         assert gm.all()
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+def test_cfg5_decode_128k_paged_variable_lengths(mala, oracle, tau):
+    """cfg5 D held in 256-key pages scattered over a shuffled pool, the eight sequences of different lengths
+    (one key, lengths that end inside a tile, inside a page and inside a split)."""
+    cfg = W.decode_config("cfg5")
+    w = W.make_decode(cfg, preset="D", device="cuda")
+    lens = [131072, 100000, 65536 + 5, 131072, 1, 77777, 131072, 4097]
+    kp, vp, bt, sl = W.paginate(w["kcache"], w["vcache"], 256, seqlens=lens, seed=3)
+    del w["kcache"], w["vcache"]
+    o, lse, st = mala.decode_paged(w["q"], kp, vp, bt, sl, w["scale"], tau, cfg.num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert torch.isfinite(o.float()).all()
+    units = [(0, 0), (1, 3), (2, 5), (4, 2), (7, 7)]
+    ref = oracle.decode_paged(w["q"], kp, vp, bt.cpu().numpy(), lens, w["scale"], tau, cfg.num_splits, 128, units=units)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    G = cfg.Hq // cfg.Hkv
+    for (b, g) in units:
+        for s in range(cfg.num_splits):
+            parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                              tau, lens[b])
+        hs = slice(g * G, (g + 1) * G)
+        parity.check_output(o[b, 0, hs].float().cpu().numpy(), ref["o"][b, hs])
+        assert np.abs(lse[b, hs].cpu().numpy() - ref["lse"][b, hs]).max() <= parity.LSE_ABS
+    legal = sum(-(-n // 128) for n in lens) * cfg.Hkv
+    tot = st.totals.cpu().numpy()
+    assert tot[1] == legal and (tot[0] == legal if tau == 0.0 else tot[0] < legal)
