@@ -61,8 +61,10 @@ static double dot(const double* a, const double* b, int d) {
   return s;
 }
 
-/* Visible-key count L_q (Section 2.1): q + 1 for equal-length causal, N_k otherwise. */
-static double visible_count(int q, int Nk, int causal) { return causal ? (double)(q + 1) : (double)Nk; }
+/* Visible-key count L_q (Section 2.1): the number of keys the query may attend to.  Causal: the queries are
+ * the LAST N_q of N_k positions (off = N_k - N_q >= 0), query row q sits at position q + off and sees the keys
+ * 0 .. q + off, so L_q = q + 1 + off (q + 1 for equal lengths, N_k for the single decode query); otherwise N_k. */
+static double visible_count(int q, int Nk, int causal, int off) { return causal ? (double)(q + 1 + off) : (double)Nk; }
 
 /* theta_q = log(tau / L_q); tau = 0 gives -inf. */
 static double log_threshold(double tau, double L) { return tau > 0.0 ? log(tau / L) : -INFINITY; }
@@ -73,10 +75,10 @@ static double log_threshold(double tau, double L) { return tau > 0.0 ? log(tau /
  * ---------------------------------------------------------------------------------------- */
 int mala_oracle_dense_fwd(const double* Q, const double* K, const double* V, int Nq, int Nk, int d,
                           double scale, int causal, int q_begin, int q_end, double* O, double* lse) {
-  if (causal && Nq != Nk) return -1;
+  if (causal && Nq > Nk) return -1;
 #pragma omp parallel for schedule(dynamic, 16)
   for (int q = q_begin; q < q_end; ++q) {
-    int kmax = causal ? q + 1 : Nk;
+    int kmax = causal ? q + 1 + (Nk - Nq) : Nk;
     double* s = (double*)malloc(sizeof(double) * (size_t)kmax);
     double m = -INFINITY;
     for (int k = 0; k < kmax; ++k) {
@@ -133,11 +135,12 @@ int mala_oracle_dense_bwd(const double* Q, const double* K, const double* V, con
  * O [N,d], lse [N]: rows of the listed blocks are written.  mask, crit: [Tr*Tc], rows of the
  * listed blocks are written (may be NULL).
  * ---------------------------------------------------------------------------------------- */
-int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, int d, double scale, double tau,
+int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale, double tau,
                     int Bq, int Bk, int causal, int n_blocks, const int* blocks, double* O, double* lse,
                     uint8_t* mask, double* crit) {
-  if (N <= 0 || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
-  const int Tr = (N + Bq - 1) / Bq, Tc = (N + Bk - 1) / Bk;
+  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
+  const int off = Nk - N; /* N queries (the last N positions) against Nk keys */
+  const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int nb = blocks ? n_blocks : Tr;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < nb; ++u) {
@@ -151,9 +154,9 @@ int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, in
     double* mt = (double*)malloc(sizeof(double) * rows);
     for (int r = 0; r < rows; ++r) { m[r] = -INFINITY; l[r] = 0.0; }
     for (int j = Tc - 1; j >= 0; --j) { /* descending from the diagonal toward earlier keys */
-      const int k0 = j * Bk, cols = (k0 + Bk <= N ? Bk : N - k0);
+      const int k0 = j * Bk, cols = (k0 + Bk <= Nk ? Bk : Nk - k0);
       /* a tile with no legal key for any row is not visited */
-      if (causal && k0 > q0 + rows - 1) {
+      if (causal && k0 > q0 + rows - 1 + off) {
         if (mask) mask[(size_t)i * Tc + j] = MASK_ILLEGAL;
         if (crit) crit[(size_t)i * Tc + j] = NAN;
         continue;
@@ -167,7 +170,7 @@ int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, in
         for (int c = 0; c < cols; ++c) {
           const int k = k0 + c;
           double s = -INFINITY;
-          if (!causal || k <= q) { s = scale * dot(Q + (size_t)q * d, K + (size_t)k * d, d); legal = 1; }
+          if (!causal || k <= q + off) { s = scale * dot(Q + (size_t)q * d, K + (size_t)k * d, d); legal = 1; }
           S[(size_t)r * Bk + c] = s;
           if (s > mrow) mrow = s;
         }
@@ -176,7 +179,7 @@ int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, in
         double cq;
         if (!legal) cq = -INFINITY;             /* does not constrain retention */
         else if (l[r] == 0.0) cq = INFINITY;    /* nothing retained yet: log-ratio is +inf */
-        else cq = mrow - (m[r] + log(l[r])) - log_threshold(tau, visible_count(q, N, causal));
+        else cq = mrow - (m[r] + log(l[r])) - log_threshold(tau, visible_count(q, Nk, causal, off));
         if (cq > C) C = cq;
       }
       const int retain = !(C < 0.0); /* skip only if every relevant row is strictly below */
@@ -223,9 +226,10 @@ int mala_oracle_bwd_D(const double* O, const double* dO, int N, int d, double* D
  * (both [Bk x Bq], row = key).  Returns 1 if retained; *C_out is the tile criterion
  * max over valid causal entries of (s - lse_q - theta_q). */
 static int bwd_tile(const double* Q, const double* K, const double* V, const double* dO, const double* lse,
-                    const double* D, int N, int d, double scale, double tau, int Bq, int Bk, int causal, int j,
+                    const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal, int j,
                     int i, double* S, double* P, double* dS, double* C_out) {
-  const int k0 = j * Bk, cols_k = (k0 + Bk <= N ? Bk : N - k0);
+  const int off = Nk - N;
+  const int k0 = j * Bk, cols_k = (k0 + Bk <= Nk ? Bk : Nk - k0);
   const int q0 = i * Bq, cols_q = (q0 + Bq <= N ? Bq : N - q0);
   double C = -INFINITY;
   for (int a = 0; a < cols_k; ++a) {
@@ -233,9 +237,9 @@ static int bwd_tile(const double* Q, const double* K, const double* V, const dou
     for (int b = 0; b < cols_q; ++b) {
       const int q = q0 + b;
       double s = -INFINITY;
-      if (!causal || k <= q) {
+      if (!causal || k <= q + off) {
         s = scale * dot(K + (size_t)k * d, Q + (size_t)q * d, d);
-        const double c = s - lse[q] - log_threshold(tau, visible_count(q, N, causal));
+        const double c = s - lse[q] - log_threshold(tau, visible_count(q, Nk, causal, off));
         if (c > C) C = c;
       }
       S[(size_t)a * Bq + b] = s;
@@ -263,16 +267,17 @@ static int bwd_tile(const double* Q, const double* K, const double* V, const dou
  * dQ [N,d] or NULL: contributions of the listed key blocks are ADDED (atomically).
  * mask, crit [Tc*Tr] indexed [j*Tr + i] (may be NULL). */
 int mala_oracle_bwd(const double* Q, const double* K, const double* V, const double* dO, const double* lse,
-                    const double* D, int N, int d, double scale, double tau, int Bq, int Bk, int causal,
+                    const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal,
                     int n_blocks, const int* key_blocks, double* dQ, double* dK, double* dV, uint8_t* mask,
                     double* crit) {
-  if (N <= 0 || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
-  const int Tr = (N + Bq - 1) / Bq, Tc = (N + Bk - 1) / Bk;
+  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
+  const int off = Nk - N;
+  const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int nb = key_blocks ? n_blocks : Tc;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < nb; ++u) {
     const int j = key_blocks ? key_blocks[u] : u;
-    const int k0 = j * Bk, cols_k = (k0 + Bk <= N ? Bk : N - k0);
+    const int k0 = j * Bk, cols_k = (k0 + Bk <= Nk ? Bk : Nk - k0);
     double* S = (double*)malloc(sizeof(double) * (size_t)Bk * Bq);
     double* P = (double*)malloc(sizeof(double) * (size_t)Bk * Bq);
     double* dS = (double*)malloc(sizeof(double) * (size_t)Bk * Bq);
@@ -281,13 +286,13 @@ int mala_oracle_bwd(const double* Q, const double* K, const double* V, const dou
       for (int c = 0; c < d; ++c) { dK[(size_t)(k0 + a) * d + c] = 0.0; dV[(size_t)(k0 + a) * d + c] = 0.0; }
     for (int i = 0; i < Tr; ++i) { /* ascending; legal tiles start at the diagonal */
       const int q0 = i * Bq, cols_q = (q0 + Bq <= N ? Bq : N - q0);
-      if (causal && k0 > q0 + cols_q - 1) { /* no valid causal entry */
+      if (causal && k0 > q0 + cols_q - 1 + off) { /* no valid causal entry */
         if (mask) mask[(size_t)j * Tr + i] = MASK_ILLEGAL;
         if (crit) crit[(size_t)j * Tr + i] = NAN;
         continue;
       }
       double C;
-      const int retain = bwd_tile(Q, K, V, dO, lse, D, N, d, scale, tau, Bq, Bk, causal, j, i, S, P, dS, &C);
+      const int retain = bwd_tile(Q, K, V, dO, lse, D, N, Nk, d, scale, tau, Bq, Bk, causal, j, i, S, P, dS, &C);
       if (mask) mask[(size_t)j * Tr + i] = retain ? MASK_RETAINED : MASK_SKIPPED;
       if (crit) crit[(size_t)j * Tr + i] = C;
       if (!retain) continue;
@@ -320,10 +325,11 @@ int mala_oracle_bwd(const double* Q, const double* K, const double* V, const dou
 /* dQ rows of the listed query blocks of one head: the same tiles as Algorithm 2, gathered per
  * query block (all legal key blocks j), so that sampled blocks can be checked at full size. */
 int mala_oracle_bwd_dq(const double* Q, const double* K, const double* V, const double* dO, const double* lse,
-                       const double* D, int N, int d, double scale, double tau, int Bq, int Bk, int causal,
+                       const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal,
                        int n_blocks, const int* query_blocks, double* dQ) {
-  if (N <= 0 || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
-  const int Tr = (N + Bq - 1) / Bq, Tc = (N + Bk - 1) / Bk;
+  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
+  const int off = Nk - N;
+  const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int nb = query_blocks ? n_blocks : Tr;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < nb; ++u) {
@@ -335,10 +341,10 @@ int mala_oracle_bwd_dq(const double* Q, const double* K, const double* V, const 
     for (int b = 0; b < cols_q; ++b)
       for (int c = 0; c < d; ++c) dQ[(size_t)(q0 + b) * d + c] = 0.0;
     for (int j = 0; j < Tc; ++j) {
-      const int k0 = j * Bk, cols_k = (k0 + Bk <= N ? Bk : N - k0);
-      if (causal && k0 > q0 + cols_q - 1) continue;
+      const int k0 = j * Bk, cols_k = (k0 + Bk <= Nk ? Bk : Nk - k0);
+      if (causal && k0 > q0 + cols_q - 1 + off) continue;
       double C;
-      if (!bwd_tile(Q, K, V, dO, lse, D, N, d, scale, tau, Bq, Bk, causal, j, i, S, P, dS, &C)) continue;
+      if (!bwd_tile(Q, K, V, dO, lse, D, N, Nk, d, scale, tau, Bq, Bk, causal, j, i, S, P, dS, &C)) continue;
       for (int a = 0; a < cols_k; ++a)
         for (int b = 0; b < cols_q; ++b) {
           const double ds = dS[(size_t)a * Bq + b];

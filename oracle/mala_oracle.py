@@ -49,11 +49,11 @@ def lib():
         L.mala_oracle_threads.restype = _ci
         L.mala_oracle_dense_fwd.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _ci, _ci, _ci, _D, _D]
         L.mala_oracle_dense_bwd.argtypes = [_D, _D, _D, _D, _ci, _ci, _cd, _ci, _D, _D, _D]
-        L.mala_oracle_fwd.argtypes = [_D, _D, _D, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D, _D, _U8, _D]
+        L.mala_oracle_fwd.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D, _D, _U8, _D]
         L.mala_oracle_bwd_D.argtypes = [_D, _D, _ci, _ci, _D]
-        L.mala_oracle_bwd.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I,
+        L.mala_oracle_bwd.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I,
                                       _D, _D, _D, _U8, _D]
-        L.mala_oracle_bwd_dq.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D]
+        L.mala_oracle_bwd_dq.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D]
         L.mala_oracle_decode_tiles_per_split.argtypes = [_ci, _ci, _ci]
         L.mala_oracle_decode_splits.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _D, _D, _U8, _D]
         L.mala_oracle_decode_splits_tps.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _D, _D, _U8, _D]
@@ -100,7 +100,8 @@ def _ck(rc: int, what: str):
 
 
 def dense_fwd(q, k, v, scale: float, causal: bool = True):
-    """FullAttn by its definition.  Returns o [B,N,Hq,d], lse [B,Hq,N]."""
+    """FullAttn by its definition (causal with fewer queries than keys: the queries are the last positions).
+    Returns o [B,N,Hq,d], lse [B,Hq,N]."""
     B, N, Hq, d = q.shape
     Hkv = k.shape[2]
     G = Hq // Hkv
@@ -139,12 +140,14 @@ def dense_bwd(q, k, v, do, scale: float, causal: bool = True):
 def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True, units=None):
     """Algorithm 1.  ``units``: optional list of (b, h_q, i) query blocks; rows of other blocks stay NaN.
 
+    q [B,N,Hq,d]; k, v [B,Nk,Hkv,d] with Nk >= N: the queries are the last N of the Nk positions (chunked
+    prefill), query row q sees the keys 0 .. q + Nk - N and L_q = q + 1 + Nk - N.
     Returns dict(o [B,N,Hq,d], lse [B,Hq,N], mask [B,Hq,Tr,Tc] uint8, crit [B,Hq,Tr,Tc]).
     """
     B, N, Hq, d = q.shape
-    Hkv = k.shape[2]
+    Nk, Hkv = k.shape[1], k.shape[2]
     G = Hq // Hkv
-    Tr, Tc = -(-N // Bq), -(-N // Bk)
+    Tr, Tc = -(-N // Bq), -(-Nk // Bk)
     o = np.full((B, N, Hq, d), np.nan)
     lse = np.full((B, Hq, N), np.nan)
     mask = np.zeros((B, Hq, Tr, Tc), dtype=np.uint8)
@@ -164,7 +167,7 @@ def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True
         m = np.zeros((Tr, Tc), dtype=np.uint8)
         c = np.full((Tr, Tc), np.nan)
         bl = np.asarray(blocks, dtype=np.int32) if blocks is not None else None
-        _ck(lib().mala_oracle_fwd(_p(Q), _p(K), _p(V), N, d, scale, tau, Bq, Bk, int(causal),
+        _ck(lib().mala_oracle_fwd(_p(Q), _p(K), _p(V), N, Nk, d, scale, tau, Bq, Bk, int(causal),
                                   0 if bl is None else len(bl), _ip(bl), _p(O), _p(l), _u8(m), _p(c)), "fwd")
         o[b, :, h, :] = O
         lse[b, h] = l
@@ -180,17 +183,17 @@ def bwd(q, k, v, o, do, lse, scale: float, tau: float, Bq: int, Bk: int, causal:
     Full run (both unit lists None): dq, dk, dv complete.  With ``key_units`` = [(b, h_kv, j)] only
     those key blocks are run: their dK/dV rows (summed over the group's query heads) are exact and
     everything else is NaN.  With ``dq_units`` = [(b, h_q, i)] the dQ rows of those query blocks are
-    computed from all their legal key blocks.
+    computed from all their legal key blocks.  Fewer queries than keys: as in ``fwd``.
     Returns dict(dq, dk, dv, mask [B,Hq,Tc,Tr], crit [B,Hq,Tc,Tr]).
     """
     B, N, Hq, d = q.shape
-    Hkv = k.shape[2]
+    Nk, Hkv = k.shape[1], k.shape[2]
     G = Hq // Hkv
-    Tr, Tc = -(-N // Bq), -(-N // Bk)
+    Tr, Tc = -(-N // Bq), -(-Nk // Bk)
     full = key_units is None and dq_units is None
     dq = np.zeros((B, N, Hq, d)) if full else np.full((B, N, Hq, d), np.nan)
-    dk = np.zeros((B, N, Hkv, d)) if full else np.full((B, N, Hkv, d), np.nan)
-    dv = np.zeros((B, N, Hkv, d)) if full else np.full((B, N, Hkv, d), np.nan)
+    dk = np.zeros((B, Nk, Hkv, d)) if full else np.full((B, Nk, Hkv, d), np.nan)
+    dv = np.zeros((B, Nk, Hkv, d)) if full else np.full((B, Nk, Hkv, d), np.nan)
     mask = np.zeros((B, Hq, Tc, Tr), dtype=np.uint8)
     crit = np.full((B, Hq, Tc, Tr), np.nan)
 
@@ -214,17 +217,17 @@ def bwd(q, k, v, o, do, lse, scale: float, tau: float, Bq: int, Bk: int, causal:
         bl = np.asarray(blocks, dtype=np.int32) if blocks is not None else None
         rows = None
         if bl is not None:
-            rows = np.concatenate([np.arange(j * Bk, min(N, (j + 1) * Bk)) for j in bl])
+            rows = np.concatenate([np.arange(j * Bk, min(Nk, (j + 1) * Bk)) for j in bl])
             dk[b, rows, g, :] = 0.0
             dv[b, rows, g, :] = 0.0
         for h in range(g * G, (g + 1) * G):
             Q, K, V, dO, l, D = head_inputs(b, h)
             a = np.zeros((N, d))
-            c = np.zeros((N, d))
-            e = np.zeros((N, d))
+            c = np.zeros((Nk, d))
+            e = np.zeros((Nk, d))
             m = np.zeros((Tc, Tr), dtype=np.uint8)
             cr = np.full((Tc, Tr), np.nan)
-            _ck(lib().mala_oracle_bwd(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, d, scale, tau, Bq, Bk,
+            _ck(lib().mala_oracle_bwd(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, Nk, d, scale, tau, Bq, Bk,
                                       int(causal), 0 if bl is None else len(bl), _ip(bl),
                                       _p(a) if full else None, _p(c), _p(e), _u8(m), _p(cr)), "bwd")
             if full:
@@ -246,7 +249,7 @@ def bwd(q, k, v, o, do, lse, scale: float, tau: float, Bq: int, Bk: int, causal:
             bl = np.asarray(blocks, dtype=np.int32)
             Q, K, V, dO, l, D = head_inputs(b, h)
             a = np.full((N, d), np.nan)
-            _ck(lib().mala_oracle_bwd_dq(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, d, scale, tau, Bq, Bk,
+            _ck(lib().mala_oracle_bwd_dq(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, Nk, d, scale, tau, Bq, Bk,
                                          int(causal), len(bl), _ip(bl), _p(a)), "bwd_dq")
             rows = np.concatenate([np.arange(i * Bq, min(N, (i + 1) * Bq)) for i in bl])
             dq[b, rows, h, :] = a[rows]

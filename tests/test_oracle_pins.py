@@ -554,3 +554,98 @@ def test_decode_paged_does_not_depend_on_where_pages_lie():
     c = orc.decode_paged(q, kp2, vp2, bt2, lens, 0.5, 0.3, 3, 8)
     for key in ("o", "lse", "mask", "lse_part"):
         assert np.array_equal(a[key], c[key])
+
+
+# ------------------------------------------------------------------ fewer queries than keys (chunked prefill)
+@pytest.mark.parametrize("Nq,Nk,Bq,Bk", [(24, 64, 8, 8), (13, 50, 8, 8), (16, 48, 16, 4)])
+def test_chunk_tau_zero_is_softmax_over_the_visible_keys(Nq, Nk, Bq, Bk):
+    # the queries are the last Nq positions: row q attends to the keys 0 .. q + Nk - Nq, nothing else
+    d, scale = 8, 0.4
+    q, k, v = peaky_inputs(Nk, d, 211)
+    qc = q[:, Nk - Nq:]
+    f = orc.fwd(qc, k, v, scale, 0.0, Bq, Bk)
+    for r in range(Nq):
+        vis = r + 1 + Nk - Nq
+        e = np.exp(scale * k[0, :vis, 0] @ qc[0, r, 0])
+        assert np.allclose(f["o"][0, r, 0], (e / e.sum()) @ v[0, :vis, 0], atol=1e-12)
+        assert abs(f["lse"][0, 0, r] - math.log(e.sum())) < 1e-12
+    od, ld = orc.dense_fwd(qc, k, v, scale)
+    assert np.allclose(od, f["o"], atol=1e-12) and np.allclose(ld, f["lse"], atol=1e-12)
+
+
+@pytest.mark.parametrize("tau", [1e-2, 0.5])
+@pytest.mark.parametrize("Nq,Nk,Bq,Bk", [(32, 96, 8, 8), (21, 69, 8, 8), (32, 64, 16, 4)])
+def test_chunk_equals_the_same_rows_of_the_full_run(Nq, Nk, Bq, Bk, tau):
+    # a query block's result depends on its own rows and the keys only, so when the chunk starts on a block
+    # boundary the chunked run must reproduce the last rows of the equal-length run: masks, O, lse and gradients
+    d, scale = 32, 1.0 / math.sqrt(32)
+    off = Nk - Nq
+    assert off % Bq == 0
+    q, k, v = peaky_inputs(Nk, d, 221, Hq=2, Hkv=1, boost=5.0)
+    do = _rng(223).standard_normal(q.shape)
+    full = orc.fwd(q, k, v, scale, tau, Bq, Bk)
+    ch = orc.fwd(q[:, off:], k, v, scale, tau, Bq, Bk)
+    assert (ch["mask"] == orc.SKIPPED).sum() > 0
+    assert np.array_equal(ch["mask"], full["mask"][:, :, off // Bq:])
+    assert np.array_equal(ch["o"], full["o"][:, off:]) and np.array_equal(ch["lse"], full["lse"][:, :, off:])
+    # backward: with dO = 0 on the rows before the chunk those rows contribute nothing (dS = P o (0 - 0))
+    do0 = do.copy()
+    do0[:, :off] = 0.0
+    gf = orc.bwd(q, k, v, full["o"], do0, full["lse"], scale, tau, Bq, Bk)
+    gc = orc.bwd(q[:, off:], k, v, ch["o"], do[:, off:], ch["lse"], scale, tau, Bq, Bk)
+    assert np.array_equal(gc["mask"], gf["mask"][:, :, :, off // Bq:])
+    assert np.allclose(gc["dq"], gf["dq"][:, off:], atol=1e-13)
+    assert np.allclose(gc["dk"], gf["dk"], atol=1e-13) and np.allclose(gc["dv"], gf["dv"], atol=1e-13)
+    assert np.abs(gf["dq"][:, :off]).max() == 0.0
+    # sampled dQ blocks follow the same tiles
+    gd = orc.bwd(q[:, off:], k, v, ch["o"], do[:, off:], ch["lse"], scale, tau, Bq, Bk, dq_units=[(0, 1, 0), (0, 0, 1)])
+    for (h, i) in ((1, 0), (0, 1)):
+        rows = slice(i * Bq, min(Nq, (i + 1) * Bq))
+        assert np.allclose(gd["dq"][0, rows, h], gc["dq"][0, rows, h], atol=1e-13)
+
+
+def test_chunk_of_one_query_is_the_unsplit_decode_rule():
+    # Nq = 1: the single query sees all Nk keys, L = Nk, tiles visited newest first -- the decode rule with one
+    # split and one row
+    Nk, d, scale, tau, Bk = 96, 8, 0.5, 0.5, 8
+    q, kc, vc = _decode_inputs(Nk, d, 1, 231)
+    dec = orc.decode(q, kc, vc, scale, tau, 1, Bk, packed_rows=False)
+    f = orc.fwd(q[:, None, :, :].reshape(1, 1, 1, d), kc, vc, scale, tau, 4, Bk)
+    assert (dec["mask"] == orc.SKIPPED).sum() > 0
+    assert np.array_equal(f["mask"][0, 0, 0], dec["mask"][0, 0, 0])
+    assert np.allclose(f["o"][0, 0, 0], dec["o"][0, 0], atol=1e-13)
+    assert abs(f["lse"][0, 0, 0] - dec["lse"][0, 0]) < 1e-13
+
+
+def test_chunk_offset_inside_a_tile_rows_without_legal_keys_do_not_constrain():
+    # Nk - Nq not a multiple of the tile: the diagonal crosses two key tiles of a query block; brute force
+    Nq, Nk, B_, d, scale, tau = 16, 37, 8, 32, 1.0 / math.sqrt(32), 0.1
+    off = Nk - Nq
+    q, k, v = peaky_inputs(Nk, d, 241, boost=5.0)
+    qc = q[:, off:]
+    f = orc.fwd(qc, k, v, scale, tau, B_, B_)
+    S = scale * (qc[0, :, 0] @ k[0, :, 0].T)
+    for i in range(2):
+        rows = list(range(i * B_, (i + 1) * B_))
+        R = {r: [] for r in rows}
+        for j in reversed(range(-(-Nk // B_))):
+            keys = list(range(j * B_, min(Nk, (j + 1) * B_)))
+            if keys[0] > rows[-1] + off:
+                assert f["mask"][0, 0, i, j] == 0
+                continue
+            skip = True
+            for r in rows:
+                legal = [x for x in keys if x <= r + off]
+                if not legal:
+                    continue
+                Z = sum(math.exp(S[r, x]) for x in R[r])
+                if Z == 0.0 or not (math.exp(max(S[r, x] for x in legal)) / Z < tau / (r + 1 + off)):
+                    skip = False
+            assert f["mask"][0, 0, i, j] == (1 if skip else 2)
+            if not skip:
+                for r in rows:
+                    R[r] += [x for x in keys if x <= r + off]
+        for r in rows:
+            Z = sum(math.exp(S[r, x]) for x in R[r])
+            assert abs(f["lse"][0, 0, r] - math.log(Z)) < 1e-12
+    assert (f["mask"] == orc.SKIPPED).sum() > 0
