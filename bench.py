@@ -178,6 +178,37 @@ class PrefillCase:
         return sum(t.numel() * t.element_size() for t in (self.q, self.k, self.v, self.do))
 
 
+def chunk_leg(cs, Nq, tau, it, peaks):
+    """mala_fwd_chunk / mala_bwd_chunk on the last Nq queries of a prefill case (all keys): latency of the MALA and
+    dense kernels and the tensor-pipe fraction on the tile FLOPs executed."""
+    import torch
+    mala, cc = cs.mala, cs.cfg
+    off = cc.N - Nq
+    q, do = cs.q[:, off:], cs.do[:, off:]
+    o, lse = torch.empty_like(q), torch.empty((cc.B, cc.Hq, Nq), dtype=torch.float32, device=q.device)
+    dq = torch.empty_like(q)
+    row = {}
+    for label, t_ in (("mala", tau), ("dense", 0.0)):
+        f_ms = time_cuda(lambda: mala.fwd_chunk(q, cs.k, cs.v, cs.scale, t_, out=o, lse=lse), 3, it)
+        b_ms = time_cuda(lambda: mala.bwd_chunk(q, cs.k, cs.v, o, do, lse, cs.scale, t_, ws=cs.ws, dq=dq, dk=cs.dk,
+                                                dv=cs.dv), 3, it)
+        row[label] = {"fwd_ms": f_ms, "bwd_ms": b_ms}
+    _, _, fs = mala.fwd_chunk(q, cs.k, cs.v, cs.scale, tau, out=o, lse=lse, stats=True)
+    _, _, _, bs = mala.bwd_chunk(q, cs.k, cs.v, o, do, lse, cs.scale, tau, ws=cs.ws, dq=dq, dk=cs.dk, dv=cs.dv,
+                                 stats=True)
+    torch.cuda.synchronize()
+    (fr, fl), (br, bl) = fs.totals.cpu().tolist(), bs.totals.cpu().tolist()
+    row["fwd_retained_frac"], row["bwd_retained_frac"] = fr / fl, br / bl
+    row["legal_tiles"] = fl
+    row["fwd_tensor_frac_on_executed"] = (fwd_executed_flops(fl, fr, cc.d) / (row["mala"]["fwd_ms"] * 1e-3) / 1e12
+                                          / peaks["tflops_sustained"])
+    row["bwd_tensor_frac_on_executed"] = (bwd_executed_flops(bl, br, cc.d) / (row["mala"]["bwd_ms"] * 1e-3) / 1e12
+                                          / peaks["tflops_sustained"])
+    row["speedup_fwd"] = row["dense"]["fwd_ms"] / row["mala"]["fwd_ms"]
+    row["speedup_bwd"] = row["dense"]["bwd_ms"] / row["mala"]["bwd_ms"]
+    return row
+
+
 def fidelity(cs, taus, it):
     """Work and operator fidelity of MALA against the in-library dense path on one configuration (the protocol
     of Section 5.1 on synthetic states): retained slots per query in forward and backward, omitted softmax mass
@@ -430,6 +461,8 @@ def main():
                                                       / (row["mala"]["bwd_ms"] * 1e-3) / 1e12 / peaks["tflops_sustained"])
                 row["speedup_fwd"] = row["dense"]["fwd_ms"] / row["mala"]["fwd_ms"]
                 row["speedup_bwd"] = row["dense"]["bwd_ms"] / row["mala"]["bwd_ms"]
+                if name == "cfg3":                  # chunked prefill: the last 8192 queries against all 32768 keys
+                    row["chunk_last_8192"] = chunk_leg(cs, 8192, tau, it, peaks)
                 if name == "cfg3" and preset == "R":
                     row["fidelity_vs_dense"] = fidelity(cs, (1e-4, 1e-2, 1.0), it)
                 detail[f"{name}_{preset}"] = row

@@ -84,6 +84,25 @@ int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, cons
              mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d, int causal,
              float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Algorithms 1 and 2 with fewer queries than keys (chunked prefill; cross attention when causal == 0).
+ * q, o, dout, dq [B,Nq,Hq,d]; k, v, dk, dv [B,Nk,Hkv,d]; lse fp32 [B,Hq,Nq].
+ * causal != 0: the queries are the LAST Nq of the Nk positions: query row q attends to the keys 0 .. q + Nk - Nq
+ * and L_q = q + 1 + Nk - Nq, the number of keys it sees (Section 2.1); a query block visits its tiles from its
+ * diagonal toward earlier keys.  The chunk must start on a tile boundary: Nk >= Nq and (Nk - Nq) % 128 == 0,
+ * MALA_ERR_UNSUPPORTED otherwise.  The result equals rows Nk - Nq .. Nk - 1 of the equal-length call on the whole
+ * sequence (for the backward: with dout zero on the earlier rows).
+ * causal == 0: every key legal for every query, L_q = Nk, any Nq and Nk.
+ * Telemetry: fwd retained_per_block [B,Hq,ceil(Nq/128)], tile_bitmask [B,Hq,ceil(Nq/128),ceil(ceil(Nk/128)/32)];
+ * bwd retained_per_block [B,Hq,ceil(Nk/128)], tile_bitmask [B,Hq,ceil(Nk/128),ceil(ceil(Nq/128)/32)].
+ * Workspace of the backward: mala_workspace_bytes(MALA_OP_BWD, B, Hq, Hkv, Nq, d, 0).  Everything else as
+ * mala_fwd / mala_bwd, which are these calls with Nq = Nk = N. */
+int mala_fwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
+                   int Hkv, int Nq, int Nk, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
+                   void* cuda_stream);
+int mala_bwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
+                   mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int Nq, int Nk, int d,
+                   int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Split-KV decode of one new token per sequence ("Fused decoding execution").  q [B,1,Hq,d] (sn is
  * ignored); kcache, vcache [B,Nk,Hkv,d], the newest token's key/value included; o [B,1,Hq,d];
  * lse_opt fp32 [B,Hq] or NULL.  The Hq/Hkv query heads of one KV head are the rows of one tile; the

@@ -172,15 +172,22 @@ int mala_device_status(int* code_out, int clear) {
   return MALA_OK;
 }
 
-int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
-             int Hkv, int N, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
-             void* cuda_stream) {
-  (void)ws; (void)ws_bytes;
+// Lengths of a call with N queries and Nk keys: causal needs the queries to be the last N positions of the Nk,
+// starting on a tile boundary.
+static int check_lengths(int N, int Nk, int causal) {
+  if (N <= 0 || Nk <= 0) return MALA_ERR_INVALID_ARG;
+  if (causal && (Nk < N || (Nk - N) % 128 != 0)) return MALA_ERR_UNSUPPORTED;
+  return MALA_OK;
+}
+
+static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
+                    int Hkv, int N, int Nk, int d, int causal, float scale, float tau, void* cuda_stream) {
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
+  MALA_TRY(check_lengths(N, Nk, causal));
   if (!lse) return MALA_ERR_INVALID_ARG;
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, N, Hq));
-  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, N, Hkv));
-  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, N, Hkv));
+  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, Nk, Hkv));
   MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, N, Hq));
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
@@ -190,8 +197,8 @@ int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const 
 
   CUtensorMap tq, tk, tv;
   if (!make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
-      !make_tensor_map_bnhd(&tk, k.p, B, N, Hkv, d, k.sb, k.sn, k.sh, 128) ||
-      !make_tensor_map_bnhd(&tv, v.p, B, N, Hkv, d, v.sb, v.sn, v.sh, 128))
+      !make_tensor_map_bnhd(&tk, k.p, B, Nk, Hkv, d, k.sb, k.sn, k.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, v.p, B, Nk, Hkv, d, v.sb, v.sn, v.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
   FwdParams p;
@@ -201,7 +208,8 @@ int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const 
   p.bitmask = st ? st->tile_bitmask : nullptr;
   p.totals = st ? (unsigned long long*)st->totals : nullptr;
   p.status = status;
-  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Tr = (N + 127) / 128; p.words = (p.Tr + 31) / 32; p.causal = causal ? 1 : 0;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Tr = (N + 127) / 128; p.causal = causal ? 1 : 0;
+  p.Nk = Nk; p.Tk = (Nk + 127) / 128; p.koff = causal ? (Nk - N) / 128 : 0; p.words = (p.Tk + 31) / 32;
   p.scale_log2 = scale * kLog2e;
   p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
   if (p.bitmask) {
@@ -213,27 +221,56 @@ int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const 
   return dense ? launch_fwd<64, true>(tq, tk, tv, p, stream) : launch_fwd<64, false>(tq, tk, tv, p, stream);
 }
 
-int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
-             mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d, int causal,
-             float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
+             int Hkv, int N, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
+             void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, N, N, d, causal, scale, tau, cuda_stream);
+}
+
+int mala_fwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
+                   int Hkv, int Nq, int Nk, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
+                   void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, cuda_stream);
+}
+
+static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
+                    mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int Nk, int d,
+                    int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
+  MALA_TRY(check_lengths(N, Nk, causal));
   if (!lse || !ws) return MALA_ERR_INVALID_ARG;
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, N, Hq));
-  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, N, Hkv));
-  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, N, Hkv));
+  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, Nk, Hkv));
   MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, N, Hq));
   MALA_TRY(check_view(dout.p, dout.sb, dout.sn, dout.sh, B, N, Hq));
   MALA_TRY(check_view(dq.p, dq.sb, dq.sn, dq.sh, B, N, Hq));
-  MALA_TRY(check_view(dk.p, dk.sb, dk.sn, dk.sh, B, N, Hkv));
-  MALA_TRY(check_view(dv.p, dv.sb, dv.sn, dv.sh, B, N, Hkv));
+  MALA_TRY(check_view(dk.p, dk.sb, dk.sn, dk.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(dv.p, dv.sb, dv.sn, dv.sh, B, Nk, Hkv));
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
   if (ws_bytes < bwd_workspace_bytes(B, Hq, N, d)) return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
   MALA_TRY(device_setup(dev, &status));
-  return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, N, d, causal ? 1 : 0, scale, tau, ws, status,
-                    (cudaStream_t)cuda_stream);
+  return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, N, Nk, d, causal ? 1 : 0, scale, tau, ws,
+                    status, (cudaStream_t)cuda_stream);
+}
+
+int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
+             mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d, int causal,
+             float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, N, N, d, causal, scale, tau, ws, ws_bytes,
+                  cuda_stream);
+}
+
+int mala_bwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
+                   mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int Nq, int Nk, int d,
+                   int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, ws, ws_bytes,
+                  cuda_stream);
 }
 
 int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,

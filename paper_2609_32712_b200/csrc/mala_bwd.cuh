@@ -54,7 +54,8 @@ struct BwdParams {
   uint32_t* bitmask;    // [B,Hq,Tc,words] or null (zero-filled by the host)
   unsigned long long* totals;
   int* status;
-  int B, Hq, Hkv, N, Np, T, words, causal;
+  int B, Hq, Hkv, N, Np, T, words, causal;   // N, Np, T: query rows, padded query rows, query blocks
+  int Nk, Tk, koff;     // keys, key blocks; causal: the queries are the last N positions, koff = (Nk - N) / 128
   float scale, scale_log2;
 };
 
@@ -97,7 +98,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int j = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
-  const int i0 = p.causal ? j : 0;
+  const int i0 = p.causal ? max(j - p.koff, 0) : 0;   // first query block that sees key block j
   const int ni = p.T - i0;
   const int n_tot = G * ni;
   int* status = p.status;
@@ -291,7 +292,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const int qt = (warp - 4) >> 2;                 // column quarter
-    const bool valid_key = (j * 128 + rl) < p.N;
+    const bool valid_key = (j * 128 + rl) < p.Nk;
     const float c2 = p.scale_log2;
     const bool stat_thread = (warp == 4 && lane == 0);
     bool ok = true;
@@ -333,7 +334,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       uint32_t sc[32];
       tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + qt * 32), sc);
       tmem_wait_ld();
-      if (p.causal && i == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
+      if (p.causal && i + p.koff == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
         const uint32_t ninf = 0xff800000u;
         const int c0 = qt * 32;
 #pragma unroll
@@ -383,7 +384,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (stat_thread) {
           ++r_head;
           if (p.bitmask) {
-            uint32_t* bm_row = p.bitmask + ((size_t)(b * p.Hq + hkv * G + hq_n) * p.T + j) * p.words;
+            uint32_t* bm_row = p.bitmask + ((size_t)(b * p.Hq + hkv * G + hq_n) * p.Tk + j) * p.words;
             if ((i >> 5) != bm_word) {
               if (bm_word >= 0) bm_row[bm_word] = bm_bits;
               bm_word = i >> 5;
@@ -456,7 +457,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ++r;
       }
       if (stat_thread && last_of_head) {   // last tile of this query head
-        const size_t row = (size_t)(b * p.Hq + hkv * G + hq_n) * p.T + j;
+        const size_t row = (size_t)(b * p.Hq + hkv * G + hq_n) * p.Tk + j;
         if (p.bitmask && bm_word >= 0) p.bitmask[row * p.words + bm_word] = bm_bits;
         if (p.retained) p.retained[row] = (uint32_t)r_head;
         if (p.totals) {
@@ -585,7 +586,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sn, int64_t o_sh,
                                       const __nv_bfloat16* __restrict__ dout, int64_t d_sb, int64_t d_sn, int64_t d_sh,
                                       const float* __restrict__ lse, float* __restrict__ lse2, float* __restrict__ bq,
-                                      float* __restrict__ Dq, int B, int Hq, int N, int Np, int d, int causal,
+                                      float* __restrict__ Dq, int B, int Hq, int N, int Np, int Nk, int d, int causal,
                                       float log2_tau) {
   const int warps_per_block = blockDim.x >> 5;
   const long long w = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
@@ -611,7 +612,7 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
   for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
   if (lane == 0) {
     const float l2 = lse[((size_t)b * Hq + h) * N + row] * 1.4426950408889634f;
-    const float L = causal ? (float)(row + 1) : (float)N;
+    const float L = causal ? (float)(row + 1 + (Nk - N)) : (float)Nk;   // visible keys
     lse2[w] = l2;
     bq[w] = l2 + (log2_tau - log2f(L));
     Dq[w] = acc;
@@ -674,15 +675,15 @@ inline bool bwd_set_attributes() {
 template <int D, bool kDense>
 inline int bwd_launch_main(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                            const CUtensorMap& tacc, const BwdParams& p, cudaStream_t stream) {
-  dim3 grid(p.T, p.Hkv, p.B);
+  dim3 grid(p.Tk, p.Hkv, p.B);
   mala_bwd_kernel<D, kDense><<<grid, BwdCfg<D>::kThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, tacc, p);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
 inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
-                      mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d,
+                      mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int Nk, int d,
                       int causal, float scale, float tau, void* ws, int* status, cudaStream_t stream) {
-  const int T = (N + 127) / 128, Np = T * 128;
+  const int T = (N + 127) / 128, Np = T * 128, Tk = (Nk + 127) / 128;
   uint8_t* w = (uint8_t*)ws;
   float* acc = (float*)w;
   w += bwd_align256((size_t)B * Hq * Np * d * sizeof(float));
@@ -694,8 +695,8 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   CUtensorMap tq, tk, tv, tdo, tacc;
   if (!make_tensor_map_f32_tiles(&tacc, acc + 64 * d, (uint64_t)B * Hq * T, d / 2, (uint64_t)128 * d * sizeof(float)) ||
       !make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
-      !make_tensor_map_bnhd(&tk, k.p, B, N, Hkv, d, k.sb, k.sn, k.sh, 128) ||
-      !make_tensor_map_bnhd(&tv, v.p, B, N, Hkv, d, v.sb, v.sn, v.sh, 128) ||
+      !make_tensor_map_bnhd(&tk, k.p, B, Nk, Hkv, d, k.sb, k.sn, k.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, v.p, B, Nk, Hkv, d, v.sb, v.sn, v.sh, 128) ||
       !make_tensor_map_bnhd(&tdo, dout.p, B, N, Hq, d, dout.sb, dout.sn, dout.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
@@ -709,9 +710,10 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   p.totals = st ? (unsigned long long*)st->totals : nullptr;
   p.status = status;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Np = Np; p.T = T; p.words = (T + 31) / 32; p.causal = causal;
+  p.Nk = Nk; p.Tk = Tk; p.koff = causal ? (Nk - N) / 128 : 0;
   p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
   if (p.bitmask &&
-      cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * T * p.words * sizeof(uint32_t), stream) != cudaSuccess)
+      cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * Tk * p.words * sizeof(uint32_t), stream) != cudaSuccess)
     return MALA_ERR_CUDA;
 
   {
@@ -720,7 +722,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     const unsigned blocks = (unsigned)((rows + wpb - 1) / wpb);
     bwd_preprocess_kernel<<<blocks, wpb * 32, 0, stream>>>((const __nv_bfloat16*)o.p, o.sb, o.sn, o.sh,
                                                           (const __nv_bfloat16*)dout.p, dout.sb, dout.sn, dout.sh, lse,
-                                                          lse2, bq, Dq, B, Hq, N, Np, d, causal,
+                                                          lse2, bq, Dq, B, Hq, N, Np, Nk, d, causal,
                                                           tau > 0.f ? log2f(tau) : -INFINITY);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }

@@ -30,7 +30,8 @@ struct FwdParams {
   uint32_t* bitmask;             // [B, Hq, Tr, words] or null (zero-filled by the host)
   unsigned long long* totals;    // [2] or null
   int* status;
-  int B, Hq, Hkv, N, Tr, words, causal;
+  int B, Hq, Hkv, N, Tr, words, causal;   // N, Tr: query rows and query blocks
+  int Nk, Tk, koff;              // keys, key blocks; causal: the queries are the last N positions, koff = (Nk - N) / 128
   float scale_log2;              // scale * log2(e)
   float log2_tau;                // log2(tau); unused by the dense kernel
 };
@@ -72,9 +73,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int iA = 2 * c, iB = 2 * c + 1;
   const bool hasB = iB < p.Tr;
   // key steps u = 0 .. U-1 visit key block j0 - u; block X takes part from step first[X] on
-  const int j0 = p.causal ? (hasB ? iB : iA) : (p.Tr - 1);
+  const int j0 = p.causal ? (hasB ? iB : iA) + p.koff : (p.Tk - 1);
   const int U = j0 + 1;
-  const int firstA = p.causal ? (j0 - iA) : 0;       // 1 when B exists (B's diagonal is not legal for A)
+  const int firstA = (p.causal && hasB) ? 1 : 0;     // B's diagonal key block is not legal for A
   int* status = p.status;
 
   if (tid == 0) {
@@ -255,7 +256,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int row = i * 128 + rl;
     const bool valid = row < p.N;
     const float c2 = p.scale_log2;
-    const float Lq = p.causal ? (float)(row + 1) : (float)p.N;
+    const float Lq = p.causal ? (float)(row + 1 + p.koff * 128) : (float)p.Nk;   // visible keys
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f(Lq));
     const uint32_t colS = (uint32_t)x * 128u, colO = 256u + (uint32_t)x * 128u;
     const int first = (x == 0) ? firstA : 0;
@@ -283,7 +284,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tmem_wait_ld();
       if (t == 0) {
         // first visited tile: causal diagonal and / or the ragged end of the key range
-        const int lim = p.causal ? rl : (p.N - 1 - j * 128);
+        const int lim = p.causal ? rl : (p.Nk - 1 - j * 128);
         const uint32_t ninf = 0xff800000u;
 #pragma unroll
         for (int e = 0; e < 32; ++e) {

@@ -49,6 +49,12 @@ def lib():
         L.mala_fwd.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, f, f, vp, sz, vp]
         L.mala_bwd.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, _TOut, _TOut, _TOut, ctypes.POINTER(_Stats),
                                i, i, i, i, i, i, f, f, vp, sz, vp]
+        L.mala_fwd_chunk.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, f, f, vp,
+                                     sz, vp]
+        L.mala_bwd_chunk.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, _TOut, _TOut, _TOut, ctypes.POINTER(_Stats),
+                                     i, i, i, i, i, i, i, f, f, vp, sz, vp]
+        L.mala_fwd_chunk.restype = i
+        L.mala_bwd_chunk.restype = i
         L.mala_decode.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp, sz, vp]
         L.mala_decode_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i,
                                         f, f, i, vp, sz, vp]
@@ -151,6 +157,43 @@ def bwd(q, k, v, o, do, lse, scale: float, tau: float, causal: bool = True, stat
                         ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_bwd")
+    return dq, dk, dv, st
+
+
+def fwd_chunk(q, k, v, scale: float, tau: float, causal: bool = True, stats: bool = False, out=None, lse=None):
+    """mala_fwd_chunk: q [B,Nq,Hq,d] against k, v [B,Nk,Hkv,d] (causal: the queries are the last Nq positions).
+    Returns (o [B,Nq,Hq,d] bf16, lse [B,Hq,Nq] fp32, Stats or None)."""
+    B, Nq, Hq, d = q.shape
+    Nk, Hkv = k.shape[1], k.shape[2]
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq, Nq), dtype=torch.float32, device=q.device) if lse is None else lse
+    Tq, Tk = -(-Nq // 128), -(-Nk // 128)
+    st = Stats((B, Hq, Tq), -(-Tk // 32), q.device) if stats else None
+    rc = lib().mala_fwd_chunk(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TOut), lse.data_ptr(),
+                              ctypes.byref(st.c) if st else None, B, Hq, Hkv, Nq, Nk, d, int(causal), scale, tau,
+                              None, 0, _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_fwd_chunk")
+    return o, lse, st
+
+
+def bwd_chunk(q, k, v, o, do, lse, scale: float, tau: float, causal: bool = True, stats: bool = False, ws=None,
+              dq=None, dk=None, dv=None):
+    """mala_bwd_chunk: returns (dq [B,Nq,Hq,d], dk, dv [B,Nk,Hkv,d], Stats or None)."""
+    B, Nq, Hq, d = q.shape
+    Nk, Hkv = k.shape[1], k.shape[2]
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    Tq, Tk = -(-Nq // 128), -(-Nk // 128)
+    st = Stats((B, Hq, Tk), -(-Tq // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_BWD, B, Hq, Hkv, Nq, d), q.device) if ws is None else ws
+    rc = lib().mala_bwd_chunk(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TIn), _view(do, _TIn),
+                              lse.data_ptr(), _view(dq, _TOut), _view(dk, _TOut), _view(dv, _TOut),
+                              ctypes.byref(st.c) if st else None, B, Hq, Hkv, Nq, Nk, d, int(causal), scale, tau,
+                              ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_bwd_chunk")
     return dq, dk, dv, st
 
 
