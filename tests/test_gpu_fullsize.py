@@ -161,3 +161,55 @@ def test_cfg5_decode_128k_paged_variable_lengths(mala, oracle, tau):
     legal = sum(-(-n // 128) for n in lens) * cfg.Hkv
     tot = st.totals.cpu().numpy()
     assert tot[1] == legal and (tot[0] == legal if tau == 0.0 else tot[0] < legal)
+
+
+@pytest.mark.parametrize("preset,tau", [("R", 1e-4), ("literal", 0.0)])
+def test_cfg3_32k_chunk_of_the_last_8192_queries(mala, oracle, preset, tau):
+    """Chunked prefill at the benchmark's size: the last 8192 queries of cfg3 against all 32768 keys, sampled blocks
+    against the oracle; the forward must also reproduce the rows of the equal-length call bit for bit."""
+    cfg = W.prefill_config("cfg3")
+    w = W.make_prefill(cfg, preset=preset, device="cuda")
+    Nq, off = 8192, cfg.N - 8192
+    q, k, v, do = w["q"][:, off:], w["k"], w["v"], w["do"][:, off:]
+    Tq, Tk, a = Nq // 128, cfg.N // 128, off // 128
+    o, lse, fst = mala.fwd_chunk(q, k, v, w["scale"], tau, stats=True)
+    dq, dk, dv, bst = mala.bwd_chunk(q, k, v, o, do, lse, w["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    o_full, lse_full, _ = mala.fwd(w["q"], k, v, w["scale"], tau)
+    assert torch.equal(o_full[:, off:], o) and torch.equal(lse_full[:, :, off:], lse)
+    fm, bm = fst.mask(Tk), bst.mask(Tq)
+    assert (bm.transpose(2, 3) <= fm).all(), "backward support must be nested in forward support"
+    legal = torch.tril(torch.ones(Tq, Tk, dtype=torch.bool, device=fm.device), diagonal=a)
+    assert not (fm & ~legal).any()
+    if tau == 0.0:
+        assert (fm == legal).all() and (bm.transpose(2, 3) == legal).all()
+    for t in (dq, dk, dv):
+        assert torch.isfinite(t.float()).all()
+    fwd_units = [(0, 0, Tq - 1), (0, 1, 0), (0, 2, 33), (0, 31, 7)]
+    ref = oracle.fwd(q, k, v, w["scale"], tau, 128, 128, units=fwd_units)
+    fmc = fm.cpu().numpy()
+    for (b, h, i) in fwd_units:
+        rows = slice(i * 128, (i + 1) * 128)
+        parity.check_mask(fmc[b, h, i], ref["mask"][b, h, i], ref["crit"][b, h, i], list(range(i + a, -1, -1)), tau,
+                          i * 128 + 1 + off)
+        parity.check_output(o[b, rows, h].float().cpu().numpy(), ref["o"][b, rows, h])
+        assert np.abs(lse[b, h, rows].cpu().numpy() - ref["lse"][b, h, rows]).max() <= parity.LSE_ABS
+    key_units = [(0, 0, Tk - 2), (0, 5, 100), (0, 3, a + 10)]     # after, before and inside the chunk's own positions
+    dq_units = [(0, 6, 40)]
+    g = oracle.bwd(q, k, v, o, do, lse.cpu().numpy(), w["scale"], tau, 128, 128, key_units=key_units,
+                   dq_units=dq_units)
+    bmc = bm.cpu().numpy()
+    G = cfg.Hq // cfg.Hkv
+    for (b, hk, j) in key_units:
+        rows = slice(j * 128, (j + 1) * 128)
+        parity.check_grad(dk[b, rows, hk].float().cpu().numpy(), g["dk"][b, rows, hk], f"dk block {j}")
+        parity.check_grad(dv[b, rows, hk].float().cpu().numpy(), g["dv"][b, rows, hk], f"dv block {j}")
+        for h in range(hk * G, (hk + 1) * G):
+            om, oc = g["mask"][b, h, j], g["crit"][b, h, j]
+            for i in range(Tq):
+                if bool(bmc[b, h, j, i]) != (om[i] == 2):
+                    assert om[i] != 0 and abs(oc[i]) <= parity.MASK_BAND, (h, j, i, oc[i])
+    for (b, h, i) in dq_units:
+        rows = slice(i * 128, (i + 1) * 128)
+        parity.check_grad(dq[b, rows, h].float().cpu().numpy(), g["dq"][b, rows, h], f"dq block {i}")
