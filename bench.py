@@ -502,6 +502,36 @@ def main():
                                           "omitted_mass_max": float((1.0 - torch.exp(lset - lse0)).max()),
                                           "speedup": row["dense"]["us"] / us}
                 row["fidelity_vs_dense"] = fid
+                # fewer, longer splits: a split's normalizer grows with its length, so more of its tiles fall under the
+                # threshold ("Fused decoding execution": the split-local test is the conservative one)
+                sweep = {}
+                for S in (128, 64, 32, 16):
+                    _, _, st = mala.decode(qd, kc, vc, wd["scale"], tau, S, ws=wsd, out=od, stats=True)
+                    ret, leg = st.totals.cpu().tolist()
+                    us = 1e3 * time_cuda(lambda: mala.decode(qd, kc, vc, wd["scale"], tau, S, ws=wsd, out=od,
+                                                              want_lse=False), 25, 100)
+                    need = (leg + ret) * TILE * dcfg.d * 2
+                    sweep[f"splits={S}"] = {"us": us, "retained_frac": ret / leg,
+                                            "rel_l2_o": float((od.float() - o0).norm() / o0.norm()),
+                                            "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                            "speedup": row["dense"]["us"] / us}
+                row["splits_sweep"] = sweep
+                # four new tokens per sequence in one step (mala_decode_multi): 16 rows per KV head, the same bytes
+                q4 = qd.repeat(1, 4, 1, 1).contiguous()
+                o4 = torch.empty_like(q4)
+                ws4 = torch.empty(mala.workspace_bytes(mala.OP_DECODE, dcfg.B * 4, dcfg.Hq, dcfg.Hkv, dcfg.Nk, dcfg.d,
+                                                       dcfg.num_splits), dtype=torch.uint8, device=dev)
+                mt = {}
+                for label, t_ in (("mala", tau), ("dense", 0.0)):
+                    _, _, st = mala.decode_multi(q4, kc, vc, wd["scale"], t_, dcfg.num_splits, ws=ws4, out=o4, stats=True)
+                    ret, leg = st.totals.cpu().tolist()
+                    us = 1e3 * time_cuda(lambda: mala.decode_multi(q4, kc, vc, wd["scale"], t_, dcfg.num_splits, ws=ws4,
+                                                                    out=o4, want_lse=False), 25, 100)
+                    need = (leg + ret) * TILE * dcfg.d * 2
+                    mt[label] = {"us": us, "retained_frac": ret / leg,
+                                 "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+                row["multi_token_4"] = mt
+                del q4, o4, ws4
                 # the same cache in 256-key pages scattered over a shuffled pool (mala_decode_paged)
                 kp, vp, bt, _ = W.paginate(kc, vc, 256, seed=7)
                 pg = {}

@@ -113,6 +113,18 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
                 int B, int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws,
                 size_t ws_bytes, void* cuda_stream);
 
+/* Split-KV decode of Sq new tokens per sequence at once (a verification step of speculative decoding, or a short
+ * chunk).  q, o [B,Sq,Hq,d]; lse_opt fp32 [B,Sq,Hq] or NULL; kcache, vcache [B,Nk,Hkv,d] with the keys and values of
+ * the Sq new tokens already in the last Sq positions.  Token s (0 = oldest) sits at position Nk - Sq + s, attends to
+ * the keys before and at its own position and has L = Nk - Sq + s + 1, the number of keys it sees (Section 2.1).
+ * The Sq * Hq/Hkv rows that share a KV head form one tile (one row that needs a key block retains it for all; a
+ * row that sees no key of a block does not constrain it); requires Sq * Hq/Hkv <= 16 and Sq <= Nk.  Splits,
+ * telemetry and merge as in mala_decode; Sq = 1 is mala_decode.
+ * Workspace: mala_workspace_bytes(MALA_OP_DECODE, B * Sq, Hq, Hkv, Nk, d, num_splits). */
+int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
+                      int B, int Hq, int Hkv, int Nk, int Sq, int d, float scale, float tau, int num_splits, void* ws,
+                      size_t ws_bytes, void* cuda_stream);
+
 /* Split-KV decode over a paged cache with one length per sequence (the serving-side layout of "Fused decoding
  * execution"; the rule itself is the one of mala_decode with L = seqlens[b] for the rows of sequence b).
  * kpages, vpages [num_pages, page_size, Hkv, d] (sb = page stride, sn = key stride, sh = head stride);

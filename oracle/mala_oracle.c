@@ -374,12 +374,26 @@ int mala_oracle_decode_tiles_per_split(int Nk, int num_splits, int Bk) {
 /* The same with the chunk length given (tps tiles of B_k keys per split) instead of derived from N_k: a batch
  * of sequences of different lengths shares one layout of splits over the key positions, and a sequence shorter
  * than a split's first position leaves that split empty.  N_k = 0 is allowed (every split empty). */
+int mala_oracle_decode_splits_rows(const double* Q, const double* K, const double* V, int R, int Nk, int d,
+                                   double scale, double tau, int num_splits, int tps, int Bk, const int* vis,
+                                   double* o_part, double* lse_part, uint8_t* mask, double* crit);
+
 int mala_oracle_decode_splits_tps(const double* Q, const double* K, const double* V, int R, int Nk, int d,
                                   double scale, double tau, int num_splits, int tps, int Bk, double* o_part,
                                   double* lse_part, uint8_t* mask, double* crit) {
+  return mala_oracle_decode_splits_rows(Q, K, V, R, Nk, d, scale, tau, num_splits, tps, Bk, NULL, o_part, lse_part,
+                                        mask, crit);
+}
+
+/* The general form: row r sees the keys 0 .. vis[r]-1 only and has L = vis[r] (vis == NULL: every row sees all
+ * N_k keys).  This is a decode step with several new tokens per sequence, whose keys already sit at the end of the
+ * cache: the token at position x sees x + 1 keys.  A row that sees no key of a tile does not constrain it
+ * (Section 2.2, as for the causal diagonal); a row that has seen no key at all stays (0, -inf). */
+int mala_oracle_decode_splits_rows(const double* Q, const double* K, const double* V, int R, int Nk, int d,
+                                   double scale, double tau, int num_splits, int tps, int Bk, const int* vis,
+                                   double* o_part, double* lse_part, uint8_t* mask, double* crit) {
   if (R <= 0 || Nk < 0 || d <= 0 || num_splits <= 0 || tps <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
   const int chunk = tps * Bk;
-  const double theta = log_threshold(tau, (double)Nk); /* L_0 = N_k, current token included */
 #pragma omp parallel for schedule(dynamic, 1)
   for (int s = 0; s < num_splits; ++s) {
     const int lo = s * chunk, hi = (lo + chunk <= Nk ? lo + chunk : Nk);
@@ -399,14 +413,20 @@ int mala_oracle_decode_splits_tps(const double* Q, const double* K, const double
       const int cols = (k0 + Bk <= hi ? Bk : hi - k0);
       double C = -INFINITY;
       for (int r = 0; r < R; ++r) {
+        const int seen = vis ? vis[r] : Nk; /* keys visible to this row = its L */
         double mrow = -INFINITY;
+        int legal = 0;
         for (int c = 0; c < cols; ++c) {
-          const double sc = scale * dot(Q + (size_t)r * d, K + (size_t)(k0 + c) * d, d);
+          double sc = -INFINITY;
+          if (k0 + c < seen) { sc = scale * dot(Q + (size_t)r * d, K + (size_t)(k0 + c) * d, d); legal = 1; }
           S[(size_t)r * Bk + c] = sc;
           if (sc > mrow) mrow = sc;
         }
         mt[r] = mrow;
-        const double cq = (l[r] == 0.0) ? INFINITY : mrow - (m[r] + log(l[r])) - theta;
+        double cq;
+        if (!legal) cq = -INFINITY;
+        else if (l[r] == 0.0) cq = INFINITY;
+        else cq = mrow - (m[r] + log(l[r])) - log_threshold(tau, (double)seen);
         if (cq > C) C = cq;
       }
       const int retain = !(C < 0.0);
@@ -415,10 +435,12 @@ int mala_oracle_decode_splits_tps(const double* Q, const double* K, const double
       if (!retain) continue;
       for (int r = 0; r < R; ++r) {
         const double mnew = (m[r] > mt[r] ? m[r] : mt[r]);
+        if (mnew == -INFINITY) continue; /* has seen no key yet */
         const double alpha = (m[r] == -INFINITY ? 0.0 : exp(m[r] - mnew));
         double lt = 0.0;
         for (int e = 0; e < d; ++e) acc[(size_t)r * d + e] *= alpha;
         for (int c = 0; c < cols; ++c) {
+          if (S[(size_t)r * Bk + c] == -INFINITY) continue;
           const double p = exp(S[(size_t)r * Bk + c] - mnew);
           lt += p;
           const double* v = V + (size_t)(k0 + c) * d;

@@ -57,10 +57,13 @@ def lib():
         L.mala_oracle_decode_tiles_per_split.argtypes = [_ci, _ci, _ci]
         L.mala_oracle_decode_splits.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _D, _D, _U8, _D]
         L.mala_oracle_decode_splits_tps.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _D, _D, _U8, _D]
+        L.mala_oracle_decode_splits_rows.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _I, _D, _D,
+                                                     _U8, _D]
         L.mala_oracle_decode_merge.argtypes = [_D, _D, _ci, _ci, _ci, _D, _D]
         for f in ("mala_oracle_dense_fwd", "mala_oracle_dense_bwd", "mala_oracle_fwd", "mala_oracle_bwd_D",
                   "mala_oracle_bwd", "mala_oracle_bwd_dq", "mala_oracle_decode_tiles_per_split",
-                  "mala_oracle_decode_splits", "mala_oracle_decode_splits_tps", "mala_oracle_decode_merge"):
+                  "mala_oracle_decode_splits", "mala_oracle_decode_splits_tps", "mala_oracle_decode_splits_rows",
+                  "mala_oracle_decode_merge"):
             getattr(L, f).restype = _ci
         _lib = L
     return _lib
@@ -359,3 +362,43 @@ def decode_paged(q, kpages, vpages, block_table, seqlens, scale: float, tau: flo
         mask[b, g] = m
         crit[b, g] = c
     return dict(o=o, lse=lse, mask=mask, crit=crit, o_part=o_part, lse_part=lse_part)
+
+
+def decode_multi(q, kcache, vcache, scale: float, tau: float, num_splits: int, Bk: int, units=None):
+    """Split-KV decode of Sq new tokens per sequence (their keys and values are the last Sq cache positions).
+
+    q [B,Sq,Hq,d]; caches [B,Nk,Hkv,d].  Token s sits at position Nk - Sq + s, sees the keys up to its own position
+    and has L = Nk - Sq + s + 1.  The Sq * Hq/Hkv rows of a KV head form one tile, row s * G + g.
+    Returns dict(o [B,Sq,Hq,d], lse [B,Sq,Hq], mask [B,Hkv,S,tps], crit, lse_part [B,Sq,Hq,S]).
+    """
+    B, Sq, Hq, d = q.shape
+    Nk, Hkv = kcache.shape[1], kcache.shape[2]
+    G = Hq // Hkv
+    R = Sq * G
+    tps = int(lib().mala_oracle_decode_tiles_per_split(Nk, num_splits, Bk))
+    o = np.zeros((B, Sq, Hq, d))
+    lse = np.zeros((B, Sq, Hq))
+    mask = np.zeros((B, Hkv, num_splits, tps), dtype=np.uint8)
+    crit = np.full((B, Hkv, num_splits, tps), np.nan)
+    lse_part = np.zeros((B, Sq, Hq, num_splits))
+    vis = np.ascontiguousarray(np.repeat(Nk - Sq + 1 + np.arange(Sq), G).astype(np.int32))
+    if units is None:
+        units = [(b, g) for b in range(B) for g in range(Hkv)]
+    for (b, g) in units:
+        K, V = _head(kcache, b, g), _head(vcache, b, g)
+        Q = np.ascontiguousarray(_np(q[b, :, g * G:(g + 1) * G, :]).reshape(R, d))
+        op = np.zeros((num_splits, R, d))
+        lp = np.zeros((num_splits, R))
+        m = np.zeros((num_splits, tps), dtype=np.uint8)
+        c = np.full((num_splits, tps), np.nan)
+        _ck(lib().mala_oracle_decode_splits_rows(_p(Q), _p(K), _p(V), R, Nk, d, scale, tau, num_splits, tps, Bk,
+                                                 _ip(vis), _p(op), _p(lp), _u8(m), _p(c)), "decode_splits_rows")
+        oo = np.zeros((R, d))
+        ll = np.zeros((R,))
+        _ck(lib().mala_oracle_decode_merge(_p(op), _p(lp), num_splits, R, d, _p(oo), _p(ll)), "decode_merge")
+        o[b, :, g * G:(g + 1) * G] = oo.reshape(Sq, G, d)
+        lse[b, :, g * G:(g + 1) * G] = ll.reshape(Sq, G)
+        lse_part[b, :, g * G:(g + 1) * G] = lp.T.reshape(Sq, G, num_splits)
+        mask[b, g] = m
+        crit[b, g] = c
+    return dict(o=o, lse=lse, mask=mask, crit=crit, lse_part=lse_part)

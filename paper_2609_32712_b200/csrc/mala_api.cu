@@ -293,6 +293,26 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
                        (cudaStream_t)cuda_stream);
 }
 
+int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
+                      int B, int Hq, int Hkv, int Nk, int Sq, int d, float scale, float tau, int num_splits, void* ws,
+                      size_t ws_bytes, void* cuda_stream) {
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  if (num_splits <= 0 || Sq <= 0 || !ws) return MALA_ERR_INVALID_ARG;
+  if ((Hq / Hkv) * Sq > 16 || Sq > Nk || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, Sq, Hq));
+  MALA_TRY(check_view(kcache.p, kcache.sb, kcache.sn, kcache.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(vcache.p, vcache.sb, vcache.sn, vcache.sh, B, Nk, Hkv));
+  MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, Sq, Hq));
+  if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
+  if (ws_bytes < decode_workspace_bytes(B * Sq, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  return decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
+                       (cudaStream_t)cuda_stream, nullptr, Sq);
+}
+
 int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* block_table,
                       const int32_t* seqlens, mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq,
                       int Hkv, int num_pages, int page_size, int max_pages_per_seq, int d, float scale, float tau,

@@ -10,13 +10,14 @@
 
 namespace mala {
 
-// lse = log sum_s exp(lse_s), o = sum_s exp(lse_s - lse) o_s; one block per (b, query head), one thread
+// lse = log sum_s exp(lse_s), o = sum_s exp(lse_s - lse) o_s; one block per (b, token, query head), one thread
 // per output column.
 template <int D>
 __global__ void __launch_bounds__(D)
 decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part, __nv_bfloat16* __restrict__ o,
-                    int64_t o_sb, int64_t o_sh, float* __restrict__ lse_out, int Hq, int num_splits) {
-  const int bh = blockIdx.x, b = bh / Hq, h = bh % Hq, c = threadIdx.x;
+                    int64_t o_sb, int64_t o_sn, int64_t o_sh, float* __restrict__ lse_out, int Sq, int Hq,
+                    int num_splits) {
+  const int bh = blockIdx.x, h = bh % Hq, tok = (bh / Hq) % Sq, b = bh / (Hq * Sq), c = threadIdx.x;
   const float* lp = lse_part + (size_t)bh * num_splits;
   float mx = -INFINITY;
   for (int s = 0; s < num_splits; ++s) mx = fmaxf(mx, lp[s]);
@@ -29,22 +30,24 @@ decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ 
     acc += w * o_part[((size_t)bh * num_splits + s) * D + c];
   }
   // (a sequence without keys has no split with mass: its output is 0 and its log-normalizer -inf)
-  o[b * o_sb + h * o_sh + c] = __float2bfloat16(Z > 0.f ? acc / Z : 0.f);
+  o[b * o_sb + tok * o_sn + h * o_sh + c] = __float2bfloat16(Z > 0.f ? acc / Z : 0.f);
   if (lse_out && c == 0) lse_out[bh] = Z > 0.f ? mx + logf(Z) : -INFINITY;
 }
 
 inline size_t decode_align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// (B: sequences x new tokens per sequence)
 inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) {
   return decode_align256((size_t)B * Hq * S * d * sizeof(float)) + decode_align256((size_t)B * Hq * S * sizeof(float));
 }
 
 inline bool decode_set_attributes() {
   bool ok = true;
-#define MALA_DEC_ATTR(DENSE, GP) \
-  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
-  MALA_DEC_ATTR(false, 1) MALA_DEC_ATTR(false, 2) MALA_DEC_ATTR(false, 4) MALA_DEC_ATTR(false, 8) MALA_DEC_ATTR(false, 16)
-  MALA_DEC_ATTR(true, 1) MALA_DEC_ATTR(true, 2) MALA_DEC_ATTR(true, 4) MALA_DEC_ATTR(true, 8) MALA_DEC_ATTR(true, 16)
+#define MALA_DEC_ATTR(DENSE, GP, MULTI) \
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
+#define MALA_DEC_ATTR_GP(GP) MALA_DEC_ATTR(false, GP, false) MALA_DEC_ATTR(true, GP, false) MALA_DEC_ATTR(false, GP, true) MALA_DEC_ATTR(true, GP, true)
+  MALA_DEC_ATTR_GP(1) MALA_DEC_ATTR_GP(2) MALA_DEC_ATTR_GP(4) MALA_DEC_ATTR_GP(8) MALA_DEC_ATTR_GP(16)
+#undef MALA_DEC_ATTR_GP
 #undef MALA_DEC_ATTR
   return ok;
 }
@@ -62,8 +65,10 @@ struct DecPaging {
 inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala_tout o, float* lse_opt,
                                       const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                                       float tau, int num_splits, float* o_part, float* lse_part, int* status,
-                                      cudaStream_t stream, const DecPaging* pg = nullptr) {
+                                      cudaStream_t stream, const DecPaging* pg = nullptr, int Sq = 1) {
   if (d != 128) return MALA_ERR_UNSUPPORTED;
+  const int G = Hq / Hkv;
+  if (Sq < 1 || G * Sq > 16 || Sq > Nk) return MALA_ERR_UNSUPPORTED;
   const bool paged = pg && pg->block_table;
   if (paged && (pg->page_size <= 0 || pg->page_size % 128 != 0 || pg->num_pages <= 0 || pg->bt_stride <= 0))
     return MALA_ERR_UNSUPPORTED;
@@ -72,8 +77,8 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   if ((long long)B * Hkv * num_splits > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
 
   CUtensorMap tq, tk, tv;
-  // q [B,1,Hq,d] viewed with the heads as rows: one 16-row box starting at the group's first head
-  if (!make_tensor_map_bnhd(&tq, q.p, B, Hq, 1, d, q.sb, q.sh, 0, 16) ||
+  // q [B,Sq,Hq,d]: one box of the group's G heads x Sq tokens
+  if (!make_tensor_map_q_rows(&tq, q.p, B, Sq, Hq, d, q.sb, Sq > 1 ? q.sn : 0, q.sh, G) ||
       !make_tensor_map_bnhd(&tk, kc.p, paged ? pg->num_pages : B, paged ? pg->page_size : Nk, Hkv, d, kc.sb, kc.sn,
                             kc.sh, 128) ||
       !make_tensor_map_bnhd(&tv, vc.p, paged ? pg->num_pages : B, paged ? pg->page_size : Nk, Hkv, d, vc.sb, vc.sn,
@@ -90,6 +95,7 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   p.block_table = paged ? pg->block_table : nullptr;
   p.bt_stride = paged ? pg->bt_stride : 0;
   p.tpp = paged ? pg->page_size / 128 : 1;
+  p.Sq = Sq;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Nk = Nk; p.tps = tps; p.num_splits = num_splits; p.words = (tps + 31) / 32;
   p.n_items = B * Hkv * num_splits;
   p.scale_log2 = scale * 1.4426950408889634f;
@@ -103,31 +109,37 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return MALA_ERR_CUDA;
   const int grid = p.n_items < sms ? p.n_items : sms;   // persistent: one CTA per SM
-  const int G = Hq / Hkv;
-#define MALA_DEC_LAUNCH(GP)                                                                                          \
+  const int R = G * Sq;   // rows of a work item
+#define MALA_DEC_LAUNCH2(DENSE, GP)                                                                                  \
   {                                                                                                                  \
-    if (tau == 0.f) mala_decode_split_kernel<true, GP><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
-    else mala_decode_split_kernel<false, GP><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);           \
+    if (Sq > 1) mala_decode_split_kernel<DENSE, GP, true><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    else mala_decode_split_kernel<DENSE, GP, false><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);       \
   }
-  if (G <= 1) MALA_DEC_LAUNCH(1)
-  else if (G <= 2) MALA_DEC_LAUNCH(2)
-  else if (G <= 4) MALA_DEC_LAUNCH(4)
-  else if (G <= 8) MALA_DEC_LAUNCH(8)
+#define MALA_DEC_LAUNCH(GP)            \
+  {                                    \
+    if (tau == 0.f) MALA_DEC_LAUNCH2(true, GP) \
+    else MALA_DEC_LAUNCH2(false, GP)   \
+  }
+  if (R <= 1) MALA_DEC_LAUNCH(1)
+  else if (R <= 2) MALA_DEC_LAUNCH(2)
+  else if (R <= 4) MALA_DEC_LAUNCH(4)
+  else if (R <= 8) MALA_DEC_LAUNCH(8)
   else MALA_DEC_LAUNCH(16)
 #undef MALA_DEC_LAUNCH
+#undef MALA_DEC_LAUNCH2
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
-  decode_merge_kernel<128><<<B * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb, o.sh, lse_opt, Hq,
-                                                       num_splits);
+  decode_merge_kernel<128><<<B * Sq * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
+                                                            Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
 inline int decode_launch(mala_tin q, mala_tin kc, mala_tin vc, mala_tout o, float* lse_opt, const mala_stats* st, int B,
                          int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws, int* status,
-                         cudaStream_t stream, const DecPaging* pg = nullptr) {
+                         cudaStream_t stream, const DecPaging* pg = nullptr, int Sq = 1) {
   float* o_part = (float*)ws;
-  float* lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Hq * num_splits * d * sizeof(float)));
+  float* lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Sq * Hq * num_splits * d * sizeof(float)));
   return decode_launch_with_scratch(q, kc, vc, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, o_part,
-                                    lse_part, status, stream, pg);
+                                    lse_part, status, stream, pg, Sq);
 }
 
 }  // namespace mala

@@ -30,8 +30,8 @@
 namespace mala {
 
 struct DecParams {
-  float* o_part;                 // [B, Hq, num_splits, 128] fp32, normalised per split
-  float* lse_part;               // [B, Hq, num_splits] natural log; -inf for an empty split
+  float* o_part;                 // [B, Sq, Hq, num_splits, 128] fp32, normalised per split
+  float* lse_part;               // [B, Sq, Hq, num_splits] natural log; -inf for an empty split
   uint32_t* retained;            // [B, Hkv, num_splits] or null
   uint32_t* bitmask;             // [B, Hkv, num_splits, words] or null (zero-filled by the host)
   unsigned long long* totals;    // [2] or null
@@ -40,6 +40,7 @@ struct DecParams {
   const int* seqlens;            // [B] keys held by sequence b (<= Nk); L = seqlens[b] for its rows
   const int* block_table;        // [B, bt_stride] page of the tpp consecutive tiles number x*tpp .. x*tpp + tpp - 1
   int bt_stride, tpp;            // tpp: tiles per page (page size / 128)
+  int Sq;                        // new tokens per sequence (the last Sq positions of the cache); rows = Sq * Hq/Hkv
   int B, Hq, Hkv, Nk, tps, num_splits, words, n_items;   // Nk: longest cache the splits are laid out for
   float scale_log2, log2_tau;
 };
@@ -55,9 +56,53 @@ struct DecCfg {
   static constexpr uint32_t kColO = 64;
 };
 
-// GP: the number of packed heads rounded up to a power of two (compile-time, so that the per-head loops of the
-// softmax group unroll without branches)
-template <bool kDense, int GP>
+// Warp-wide reduction of N independent values per lane (N a power of two <= 16) in N-ish shuffles instead of 5 N:
+// while more than one value is left, a lane hands the half of its values that its partner (lane ^ OFF) keeps to that
+// partner and folds the partner's half into the half it keeps; the remaining offsets are plain butterfly steps.
+// Afterwards v[0] holds, in every lane, the reduction over the warp of value number lane >> (5 - log2 N).
+template <int N, int OFF, bool kMax>
+struct RowReduce {
+  static __device__ __forceinline__ void run(float* v, int lane) {
+    if constexpr (OFF > 0) {
+      if constexpr (N > 1) {
+        constexpr int H = N / 2;
+        const bool up = (lane & OFF) != 0;
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+          const float send = up ? v[i] : v[i + H];
+          const float keep = up ? v[i + H] : v[i];
+          const float recv = __shfl_xor_sync(0xffffffffu, send, OFF);
+          v[i] = kMax ? fmaxf(keep, recv) : keep + recv;
+        }
+        RowReduce<H, OFF / 2, kMax>::run(v, lane);
+      } else {
+        const float recv = __shfl_xor_sync(0xffffffffu, v[0], OFF);
+        v[0] = kMax ? fmaxf(v[0], recv) : v[0] + recv;
+        RowReduce<1, OFF / 2, kMax>::run(v, lane);
+      }
+    }
+  }
+};
+
+// N consecutive floats from shared memory (16-byte aligned), as 128-bit loads where N allows
+template <int N>
+__device__ __forceinline__ void lds_row(const float* src, float (&dst)[N]) {
+  if constexpr (N >= 4) {
+#pragma unroll
+    for (int i = 0; i < N; i += 4) {
+      const float4 t = *reinterpret_cast<const float4*>(src + i);
+      dst[i] = t.x; dst[i + 1] = t.y; dst[i + 2] = t.z; dst[i + 3] = t.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; ++i) dst[i] = src[i];
+  }
+}
+
+// GP: the number of packed rows rounded up to a power of two (compile-time, so that the per-row loops of the
+// softmax group unroll without branches).  kMulti: several new tokens per sequence, i.e. rows that see
+// different numbers of keys (one token: every row sees all keys, and the per-row limits fold into scalars).
+template <bool kDense, int GP, bool kMulti>
 __global__ void __launch_bounds__(256, 1)
 mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                          const __grid_constant__ CUtensorMap tmV, const DecParams p) {
@@ -74,13 +119,17 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[4];
   __shared__ int v_row[8], v_outer[8];     // TMA coordinates of the V tile of tile g (ring; written by the producer)
-  __shared__ float xch_max[2][4][16], xch_sum[2][4][16];   // the softmax group's per-tile exchange
+  __shared__ __align__(16) float xch_max[2][4][16], xch_sum[2][4][16];   // the softmax group's per-tile exchange
   __shared__ int early_exit;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.Hq / p.Hkv;
+  const int R = kMulti ? G * p.Sq : G;     // rows of a work item: row s * G + g = token s, head g of the group
   int* status = p.status;
 
+  // the Q tile of an item has R <= 16 rows; the other rows of the two stages are never written: clear them once
+  for (int i = tid; i < 2 * DecCfg::kQBytes / 16; i += DecCfg::kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0u, 0u, 0u, 0u);
+  fence_proxy_async_smem();
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
     for (int s = 0; s < 2; ++s) {
@@ -146,7 +195,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         const int ip = ne & 1;
         ok = mbar_wait(&q_empty[ip], ((ne >> 1) & 1) ^ 1, status);
         if (!ok) break;
-        mbar_arrive_expect_tx(&q_full[ip], DecCfg::kQBytes);
+        mbar_arrive_expect_tx(&q_full[ip], (uint32_t)R * 256u);   // two panels of R rows x 128 bytes
         tma_load_4d(sQ + ip * DecCfg::kQBytes, &tmQ, &q_full[ip], 0, hkv * G, 0, b);
         tma_load_4d(sQ + ip * DecCfg::kQBytes + 2048, &tmQ, &q_full[ip], 64, hkv * G, 0, b);
         for (int t = 0; t < T && ok; ++t, ++g) {
@@ -331,6 +380,19 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     // have the exponent range for it, and moving the reference means waiting until every PV issued so far has
     // retired (their V copies included), which would stall this group for a whole HBM round trip.
     constexpr float kRescaleGap = 60.f;
+    // row q = token tok[q] of the Sq new ones (the last positions of the cache), head q - tok[q] * G of the group:
+    // it sees the keys before position nk - back[q] and its partials lie rowoff[q] rows after the item's first
+    constexpr int kLanesPerRow = 32 / GP;              // after RowReduce, row r sits in lanes r * kLanesPerRow ..
+    const int pub_row = lane / kLanesPerRow;
+    const bool publisher = (lane % kLanesPerRow) == 0;
+    int back[GP];
+    size_t rowoff[GP];
+#pragma unroll
+    for (int q = 0; q < GP; ++q) {
+      const int tok = (kMulti && q < R) ? q / G : 0;
+      back[q] = p.Sq - 1 - tok;
+      rowoff[q] = kMulti ? ((size_t)tok * p.Hq + (size_t)(q - tok * G)) * p.num_splits : (size_t)q * p.num_splits;
+    }
     int g = 0, ne = 0, rg = 0;                     // global tile counter, non-empty item ordinal, retained tiles so far
     uint32_t xc = 0;                               // exchanges so far (buffer xc & 1, barrier phase xc & 1)
     bool ok = true;
@@ -356,50 +418,68 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       if (lane == 0) mbar_arrive(&o_free[pend_ip]);   // the accumulator may take the item after next
 #pragma unroll
       for (int q = 0; q < GP; ++q)
-        if (q < G) p.o_part[(pend_prow0 + (size_t)q * p.num_splits) * 128 + kt] = __uint_as_float(o[q]) / pend_l[q];
+        if (q < R)   // (a row that saw no key of the split: (0, -inf))
+          p.o_part[(pend_prow0 + rowoff[q]) * 128 + kt] =
+              (!kMulti || pend_l[q] > 0.f) ? __uint_as_float(o[q]) / pend_l[q] : 0.f;
       pend = false;
       return true;
     };
     for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
       int b, hkv, split, T, j0, nk;
       geometry(item, b, hkv, split, T, j0, nk);
-      const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)nk));   // L = keys of the sequence
-      const size_t prow0 = ((size_t)b * p.Hq + hkv * G) * p.num_splits + split;   // head q: + q * num_splits
+      // L of a row = the keys it sees: all nk of the sequence for the newest token, one less per token before it
+      int lim[GP];
+      float theta[GP];
+#pragma unroll
+      for (int q = 0; q < GP; ++q) {
+        lim[q] = kMulti ? nk - back[q] : nk;
+        theta[q] = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(lim[q], 1)));
+      }
+      const size_t prow0 = ((size_t)b * p.Sq * p.Hq + hkv * G) * p.num_splits + split;   // row q: + rowoff[q]
       const size_t stat_row = (size_t)(b * p.Hkv + hkv) * p.num_splits + split;
       if (T == 0) {   // empty split: (0, -inf)
-        for (int q = 0; q < G; ++q) p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = 0.f;
-        if (kt < G) p.lse_part[prow0 + (size_t)kt * p.num_splits] = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < GP; ++q)
+          if (q < R) {
+            p.o_part[(prow0 + rowoff[q]) * 128 + kt] = 0.f;
+            if (kt == q) p.lse_part[prow0 + rowoff[q]] = -INFINITY;
+          }
         if (head && p.retained) p.retained[stat_row] = 0u;
         continue;
       }
       const int ip = ne & 1;
       const uint32_t colO = DecCfg::kColO + (uint32_t)ip * 16u;
-      float m_ref[GP], l[GP], lgl[GP], ps_w[GP];   // ps_w: this warp's sums of P of the last retained tile
+      float m_ref[GP], l[GP], lgl[GP];
+      float psum = 0.f;   // this warp's sum of P of the last retained tile, for the row this lane publishes
 #pragma unroll
-      for (int q = 0; q < GP; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; lgl[q] = -INFINITY; ps_w[q] = 0.f; }
+      for (int q = 0; q < GP; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; lgl[q] = -INFINITY; }
       int r = 0;
       bool pending_sum = false;
       uint32_t bm_bits = 0;
       int bm_word = -1;
       uint32_t* bm_row = p.bitmask ? p.bitmask + stat_row * p.words : nullptr;
-      // publishes this warp's (maxima, sums), waits for the group, returns the combined maxima in tmax and adds
-      // the combined sums to l
-      auto exchange = [&](const float (&mx_w)[GP], float (&tmax)[GP]) -> bool {
+      // publishes this warp's (maximum, sum) of row pub_row -- each row by the first lane that holds it after the
+      // warp reduction --, waits for the group, returns the combined maxima in tmax and adds the combined sums to l
+      auto exchange = [&](float mx_row, float (&tmax)[GP]) -> bool {
         const int xb = xc & 1;
-        if (lane == 0) {
-#pragma unroll
-          for (int q = 0; q < GP; ++q) { xch_max[xb][w][q] = mx_w[q]; xch_sum[xb][w][q] = ps_w[q]; }
-          mbar_arrive(&grp_a);
-        }
+        if (publisher) { xch_max[xb][w][pub_row] = mx_row; xch_sum[xb][w][pub_row] = psum; }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&grp_a);
         bool k = mbar_wait(&grp_a, xc & 1, status);
         k = __all_sync(0xffffffffu, k);
         ++xc;
         if (!k) return false;
+        float a0[GP], a1[GP], a2[GP], a3[GP];
+        lds_row<GP>(xch_max[xb][0], a0); lds_row<GP>(xch_max[xb][1], a1);
+        lds_row<GP>(xch_max[xb][2], a2); lds_row<GP>(xch_max[xb][3], a3);
 #pragma unroll
-        for (int q = 0; q < GP; ++q) {
-          tmax[q] = fmaxf(fmaxf(xch_max[xb][0][q], xch_max[xb][1][q]), fmaxf(xch_max[xb][2][q], xch_max[xb][3][q]));
-          if (pending_sum) {
-            l[q] += (xch_sum[xb][0][q] + xch_sum[xb][1][q]) + (xch_sum[xb][2][q] + xch_sum[xb][3][q]);
+        for (int q = 0; q < GP; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
+        if (pending_sum) {
+          lds_row<GP>(xch_sum[xb][0], a0); lds_row<GP>(xch_sum[xb][1], a1);
+          lds_row<GP>(xch_sum[xb][2], a2); lds_row<GP>(xch_sum[xb][3], a3);
+#pragma unroll
+          for (int q = 0; q < GP; ++q) {
+            l[q] += (a0[q] + a1[q]) + (a2[q] + a3[q]);
             lgl[q] = __log2f(l[q]);
           }
         }
@@ -419,22 +499,21 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_free[sb]);     // the scores are in registers
-        const bool key_ok = ((j0 - t) * 128 + kt) < nk;   // only the newest tile of the split can be ragged
+        const int kpos = (j0 - t) * 128 + kt;   // only the newest tile of the sequence has keys that a row does not see
         float x[GP], mx[GP], tmax[GP];
 #pragma unroll
-        for (int q = 0; q < GP; ++q) { x[q] = (key_ok && q < G) ? __uint_as_float(sr[q]) * c2 : -INFINITY; mx[q] = x[q]; }
-#pragma unroll
-        for (int s = 16; s > 0; s >>= 1)   // the reductions of the G heads run interleaved
-#pragma unroll
-          for (int q = 0; q < GP; ++q) mx[q] = fmaxf(mx[q], __shfl_xor_sync(0xffffffffu, mx[q], s));
-        ok = exchange(mx, tmax);
+        for (int q = 0; q < GP; ++q) { x[q] = (kpos < lim[q] && q < R) ? __uint_as_float(sr[q]) * c2 : -INFINITY; mx[q] = x[q]; }
+        RowReduce<GP, 16, true>::run(mx, lane);   // mx[0]: the warp's maximum of row pub_row
+        ok = exchange(mx[0], tmax);
         if (!ok) break;
         // Eq. 3 against the split's partial normalizer: skip iff rowmax - (m + log l) < log(tau / Nk) for every head
         bool retain = true;
         if (!kDense && r > 0) {
           retain = false;
 #pragma unroll
-          for (int q = 0; q < GP; ++q) retain = retain || (q < G && !(((tmax[q] - (m_ref[q] + lgl[q])) - theta) < 0.f));
+          for (int q = 0; q < GP; ++q)   // (a row without a visible key in the tile does not constrain it)
+            retain = retain || (q < R && (!kMulti || tmax[q] > -INFINITY) &&
+                                !(((tmax[q] - (m_ref[q] + lgl[q])) - theta[q]) < 0.f));
         }
         if (!kDense && head) {
           *(volatile int*)&flag[g & 3] = retain ? 1 : 0;
@@ -452,14 +531,14 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         }
         if (r == 0) {
 #pragma unroll
-          for (int q = 0; q < GP; ++q) m_ref[q] = tmax[q];
+          for (int q = 0; q < GP; ++q) m_ref[q] = kMulti ? fmaxf(tmax[q], -1e30f) : tmax[q];   // (finite also for a row that sees no key yet)
         } else {
           float alpha[GP];
           bool resc = false;
 #pragma unroll
           for (int q = 0; q < GP; ++q) {
             alpha[q] = 1.f;
-            if (q < G && tmax[q] > m_ref[q] + kRescaleGap) {   // lazy rescaling: the reference only moves when it has to
+            if (q < R && tmax[q] > m_ref[q] + kRescaleGap) {   // lazy rescaling: the reference only moves when it has to
               alpha[q] = fast_exp2(m_ref[q] - tmax[q]);
               l[q] *= alpha[q];
               lgl[q] = __log2f(l[q]);
@@ -496,28 +575,24 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           const uint32_t col = (uint32_t)(kt & 63);
 #pragma unroll
           for (int q = 0; q < GP; ++q) {
-            ps_w[q] = (q < G) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
-            *reinterpret_cast<__nv_bfloat16*>(dst + sw128_offset((uint32_t)q, col)) = __float2bfloat16_rn(ps_w[q]);
+            x[q] = (q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
+            *reinterpret_cast<__nv_bfloat16*>(dst + sw128_offset((uint32_t)q, col)) = __float2bfloat16_rn(x[q]);
           }
         }
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[ps]);
-        // this warp's per-head sums of the tile (fp32, before the bf16 cast); they travel with the next exchange
-#pragma unroll
-        for (int s = 16; s > 0; s >>= 1)
-#pragma unroll
-          for (int q = 0; q < GP; ++q) ps_w[q] += __shfl_xor_sync(0xffffffffu, ps_w[q], s);
+        // this warp's per-row sums of the tile (fp32, before the bf16 cast); they travel with the next exchange
+        RowReduce<GP, 16, false>::run(x, lane);
+        psum = x[0];
         pending_sum = true;
         ++r;
         ++rg;
       }
       if (!ok) break;
       if (pending_sum) {   // the sums of the last retained tile
-        float none[GP], dummy[GP];
-#pragma unroll
-        for (int q = 0; q < GP; ++q) none[q] = -INFINITY;
-        ok = exchange(none, dummy);
+        float dummy[GP];
+        ok = exchange(-INFINITY, dummy);
         if (!ok) break;
       }
       // the log-normalizer and the telemetry now; O / l (see above) once the item's last PV has retired
@@ -530,7 +605,8 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       for (int q = 0; q < GP; ++q) pend_l[q] = l[q];
 #pragma unroll
       for (int q = 0; q < GP; ++q)
-        if (q < G && kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = (m_ref[q] + lgl[q]) * 0.6931471805599453f;
+        if (q < R && kt == q)
+          p.lse_part[prow0 + rowoff[q]] = (!kMulti || l[q] > 0.f) ? (m_ref[q] + lgl[q]) * 0.6931471805599453f : -INFINITY;
       if (head) {
         if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
         if (p.retained) p.retained[stat_row] = (uint32_t)r;

@@ -44,6 +44,23 @@ inline bool make_tensor_map_bnhd(CUtensorMap* out, const void* base, int B, int 
   return r == CUDA_SUCCESS;
 }
 
+// Tensor map over the bf16 queries of a decode step, [B, S, H, d]: coordinates (c, h, s, b), box = 64 columns x G
+// heads x S tokens, which lands in shared memory as S * G consecutive 128-byte rows (row s * G + g), 128-byte swizzle.
+inline bool make_tensor_map_q_rows(CUtensorMap* out, const void* base, int B, int S, int H, int d, int64_t sb,
+                                   int64_t sn, int64_t sh, int G) {
+  PFN_tensorMapEncodeTiled enc = tensor_map_encoder();
+  if (!enc) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)S, (cuuint64_t)B};
+  auto legal = [&](int64_t s, int n) -> cuuint64_t { return (n == 1 || s <= 0) ? (cuuint64_t)d * 2 : (cuuint64_t)s * 2; };
+  cuuint64_t strides[3] = {legal(sh, H), legal(sn, S), legal(sb, B)};
+  cuuint32_t box[4] = {64u, (cuuint32_t)G, (cuuint32_t)S, 1u};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Tensor map over fp32 tiles: `ntiles` row-major [128 rows x cols] blocks, `tile_stride_bytes` apart, first one at
 // `base`.  Coordinates (col, row, tile), box = 32 columns x 128 rows x 1 tile (128 bytes wide), 128-byte swizzle.
 // Used for TMA reduce-add of fp32 panels.

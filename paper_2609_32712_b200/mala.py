@@ -56,6 +56,9 @@ def lib():
         L.mala_fwd_chunk.restype = i
         L.mala_bwd_chunk.restype = i
         L.mala_decode.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp, sz, vp]
+        L.mala_decode_multi.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, f, f, i,
+                                        vp, sz, vp]
+        L.mala_decode_multi.restype = i
         L.mala_decode_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i,
                                         f, f, i, vp, sz, vp]
         L.mala_decode_paged.restype = i
@@ -213,6 +216,25 @@ def decode(q, kcache, vcache, scale: float, tau: float, num_splits: int, stats: 
                            B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_decode")
+    return o, lse, st
+
+
+def decode_multi(q, kcache, vcache, scale: float, tau: float, num_splits: int, stats: bool = False, ws=None, out=None,
+                 want_lse: bool = True):
+    """mala_decode_multi: q [B,Sq,Hq,d], the Sq new tokens of each sequence (their keys / values are the last Sq
+    positions of the caches).  Returns (o [B,Sq,Hq,d] bf16, lse [B,Sq,Hq] fp32 or None, Stats or None)."""
+    B, Sq, Hq, d = q.shape
+    Nk, Hkv = kcache.shape[1], kcache.shape[2]
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Sq, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    tps = -(-(-(-Nk // num_splits)) // 128)
+    st = Stats((B, Hkv, num_splits), -(-tps // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_DECODE, B * Sq, Hq, Hkv, Nk, d, num_splits), q.device) if ws is None else ws
+    rc = lib().mala_decode_multi(_view(q, _TIn), _view(kcache, _TIn), _view(vcache, _TIn), _view(o, _TOut),
+                                 lse.data_ptr() if lse is not None else None, ctypes.byref(st.c) if st else None,
+                                 B, Hq, Hkv, Nk, Sq, d, scale, tau, num_splits, ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_decode_multi")
     return o, lse, st
 
 

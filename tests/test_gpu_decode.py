@@ -168,3 +168,57 @@ def test_decode_paged_rejects_pages_that_are_not_whole_tiles(mala):
     with pytest.raises(mala.MalaError) as e:
         mala.decode_paged(q, pages, pages, bt, None, 0.1, 0.0, 1)
     assert e.value.code < 0
+
+
+def _run_multi(mala, oracle, w, Sq, tau, num_splits, seed=0):
+    """The decode workload's cache with Sq new tokens: their queries are drawn like the workload's one query."""
+    kc, vc = w["kcache"], w["vcache"]
+    B, Nk, Hkv, d = kc.shape
+    Hq = w["q"].shape[2]
+    G = Hq // Hkv
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(1000 + seed)
+    q = w["q"].float().repeat(1, Sq, 1, 1)
+    q[..., : d - 1] += 0.5 * torch.randn((B, Sq, Hq, d - 1), generator=gen)   # (the last feature keeps the key gate)
+    q = q.to(torch.bfloat16)
+    o, lse, st = mala.decode_multi(q.cuda(), kc.cuda(), vc.cuda(), w["scale"], tau, num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    ref = oracle.decode_multi(q, kc, vc, w["scale"], tau, num_splits, 128)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy(), lse.cpu().numpy()
+    for b in range(B):
+        for g in range(Hkv):
+            for s in range(num_splits):
+                parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                                  tau, Nk - Sq + 1, 128)
+                assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
+    parity.check_output(o_c, ref["o"])
+    assert np.abs(lse_c - ref["lse"]).max() <= parity.LSE_ABS
+    return int((ref["mask"] == 1).sum())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv,Sq", [(1024, 4, 8, 2, 4), (1000, 3, 4, 4, 16), (2050, 4, 4, 2, 5),
+                                             (1027, 2, 6, 2, 4), (640, 5, 2, 1, 8), (4096, 8, 16, 2, 2)])
+def test_decode_multi_literal(mala, oracle, Nk, S, Hq, Hkv, Sq, tau):
+    """Several new tokens per step; (2050, 5) and (1027, 4): the newest key block holds fewer keys than there are
+    new tokens, so its first rows see none of it."""
+    w = W.custom_decode(2, Hq, Hkv, Nk, 128, S, seed=Nk + S + Sq)
+    _run_multi(mala, oracle, w, Sq, tau, S, seed=Sq)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+def test_decode_multi_gated_keys_skip_value_tiles(mala, oracle, tau):
+    w = W.custom_decode(2, 8, 2, 8192, 128, 8, group_types=["diffuse", "peaked"], seed=3, preset="D")
+    assert _run_multi(mala, oracle, w, 4, tau, 8) > 0, "workload must exercise skipping"
+
+
+def test_decode_multi_of_one_token_equals_decode(mala):
+    w = W.custom_decode(2, 8, 2, 4096, 128, 8, group_types=["diffuse", "peaked"], seed=21, preset="D")
+    q, kc, vc = (w[x].cuda() for x in ("q", "kcache", "vcache"))
+    for tau in (0.0, 1e-4):
+        o1, l1, _ = mala.decode(q, kc, vc, w["scale"], tau, 8)
+        o2, l2, _ = mala.decode_multi(q, kc, vc, w["scale"], tau, 8)
+        assert torch.equal(o1, o2) and torch.equal(l1, l2.reshape(l1.shape))

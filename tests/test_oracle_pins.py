@@ -649,3 +649,80 @@ def test_chunk_offset_inside_a_tile_rows_without_legal_keys_do_not_constrain():
             Z = sum(math.exp(S[r, x]) for x in R[r])
             assert abs(f["lse"][0, 0, r] - math.log(Z)) < 1e-12
     assert (f["mask"] == orc.SKIPPED).sum() > 0
+
+
+# ------------------------------------------------------------------ several new tokens per decode step
+def _multi_inputs(Nk, Sq, d, G, seed):
+    r = _rng(seed)
+    q = r.standard_normal((1, Sq, G, d))
+    kc = r.standard_normal((1, Nk, 1, d))
+    vc = r.standard_normal((1, Nk, 1, d))
+    live = r.random(Nk) < 0.1
+    live[-Sq - 2:] = True
+    kc[0, :, 0, d - 1] = np.where(live, 0.0, -6.0)
+    q[0, :, :, d - 1] = 6.0
+    return q, kc, vc
+
+
+@pytest.mark.parametrize("Nk,Sq", [(100, 4), (97, 3), (64, 1)])
+def test_decode_multi_tau_zero_is_softmax_over_each_tokens_visible_keys(Nk, Sq):
+    q, kc, vc = _multi_inputs(Nk, Sq, 8, 2, 251)
+    dec = orc.decode_multi(q, kc, vc, 0.4, 0.0, 3, 8)
+    for s in range(Sq):
+        vis = Nk - Sq + s + 1
+        for h in range(2):
+            e = np.exp(0.4 * kc[0, :vis, 0] @ q[0, s, h])
+            assert np.allclose(dec["o"][0, s, h], (e / e.sum()) @ vc[0, :vis, 0], atol=1e-12)
+            assert abs(dec["lse"][0, s, h] - math.log(e.sum())) < 1e-12
+    if Sq == 1:
+        one = orc.decode(q[:, 0], kc, vc, 0.4, 0.0, 3, 8)
+        assert np.array_equal(one["o"], dec["o"][:, 0]) and np.array_equal(one["lse"], dec["lse"][:, 0])
+
+
+@pytest.mark.parametrize("Nk,Sq,G", [(96, 4, 2), (91, 5, 1), (98, 3, 2)])
+def test_decode_multi_rule_bruteforce_with_per_row_visible_keys(Nk, Sq, G):
+    d, S, Bk, scale, tau = 8, 3, 8, 0.5, 0.5
+    q, kc, vc = _multi_inputs(Nk, Sq, d, G, 261 + Nk)
+    dec = orc.decode_multi(q, kc, vc, scale, tau, S, Bk)
+    tps = dec["mask"].shape[-1]
+    chunk = tps * Bk
+    rows = [(s, g) for s in range(Sq) for g in range(G)]
+    sc = {(s, g): scale * kc[0, :, 0] @ q[0, s, g] for (s, g) in rows}
+    assert (dec["mask"] == orc.SKIPPED).sum() > 0
+    for sp in range(S):
+        kept = {r: [] for r in rows}
+        for t in reversed(range(tps)):
+            keys = [x for x in range(sp * chunk + t * Bk, sp * chunk + (t + 1) * Bk) if x < Nk]
+            if not keys:
+                assert dec["mask"][0, 0, sp, t] == 0
+                continue
+            skip = True
+            for (s, g) in rows:
+                vis = Nk - Sq + s + 1
+                legal = [x for x in keys if x < vis]
+                if not legal:
+                    continue                          # the row sees no key of the tile: it does not constrain it
+                Z = sum(math.exp(sc[(s, g)][x]) for x in kept[(s, g)])
+                if Z == 0.0 or not (math.exp(max(sc[(s, g)][x] for x in legal)) / Z < tau / vis):
+                    skip = False
+            assert dec["mask"][0, 0, sp, t] == (1 if skip else 2)
+            if not skip:
+                for (s, g) in rows:
+                    kept[(s, g)] += [x for x in keys if x < Nk - Sq + s + 1]
+        for (s, g) in rows:
+            Z = sum(math.exp(sc[(s, g)][x]) for x in kept[(s, g)])
+            want = math.log(Z) if Z > 0 else -math.inf
+            got = dec["lse_part"][0, s, g, sp]
+            assert (got == want) if Z == 0 else abs(got - want) < 1e-12
+
+
+def test_decode_multi_one_split_is_the_forward_rule_on_a_chunk_of_the_new_tokens():
+    # the Sq new tokens as one query block of a chunked prefill (one head, one split): same rows, same tiles
+    Nk, Sq, d, Bk, scale, tau = 93, 5, 8, 8, 0.5, 0.5
+    q, kc, vc = _multi_inputs(Nk, Sq, d, 1, 271)
+    dec = orc.decode_multi(q, kc, vc, scale, tau, 1, Bk)
+    f = orc.fwd(q, kc, vc, scale, tau, 8, Bk)           # q [1,Sq,1,d]: the last Sq positions
+    assert (dec["mask"] == orc.SKIPPED).sum() > 0
+    assert np.array_equal(f["mask"][0, 0, 0], dec["mask"][0, 0, 0])
+    assert np.allclose(f["o"][0, :, 0], dec["o"][0, :, 0], atol=1e-13)
+    assert np.allclose(f["lse"][0, 0], dec["lse"][0, :, 0], atol=1e-13)
