@@ -103,6 +103,23 @@ int mala_bwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout
                    mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int Nq, int Nk, int d,
                    int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Algorithms 1 and 2 on B packed sequences of different lengths (self attention, equal query and key lengths per
+ * sequence).  q, o, dout, dq are [1,total,Hq,d] tensors, k, v, dk, dv [1,total,Hkv,d] (sb is ignored); sequence b
+ * holds the rows cu_seqlens[b] .. cu_seqlens[b+1]-1; cu_seqlens: device int32 [B+1], non-decreasing, cu_seqlens[0] = 0,
+ * cu_seqlens[B] = total; max_seqlen >= every length (it sizes the grid and the telemetry).  Every sequence is treated
+ * exactly as a mala_fwd / mala_bwd call on its own rows (its own tile partition, starting at its first row; its own
+ * L_q).  lse: fp32 [Hq,total].  Telemetry as for mala_fwd / mala_bwd with N = max_seqlen (rows of blocks a sequence
+ * does not have stay zero).  Workspace of the backward:
+ * mala_workspace_bytes(MALA_OP_BWD, 1, Hq, Hkv, total + 128 * B, d, 0).  The tile that holds a sequence's last rows
+ * also covers the first rows of the next one: those never reach a result, but they must be finite numbers. */
+int mala_fwd_varlen(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu_seqlens, mala_tout o, float* lse,
+                    const mala_stats* st, int B, int Hq, int Hkv, int total, int max_seqlen, int d, int causal,
+                    float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream);
+int mala_bwd_varlen(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,
+                    const int32_t* cu_seqlens, mala_tout dq, mala_tout dk, mala_tout dv, const mala_stats* st, int B,
+                    int Hq, int Hkv, int total, int max_seqlen, int d, int causal, float scale, float tau, void* ws,
+                    size_t ws_bytes, void* cuda_stream);
+
 /* Split-KV decode of one new token per sequence ("Fused decoding execution").  q [B,1,Hq,d] (sn is
  * ignored); kcache, vcache [B,Nk,Hkv,d], the newest token's key/value included; o [B,1,Hq,d];
  * lse_opt fp32 [B,Hq] or NULL.  The Hq/Hkv query heads of one KV head are the rows of one tile; the

@@ -180,15 +180,18 @@ static int check_lengths(int N, int Nk, int causal) {
   return MALA_OK;
 }
 
+// cu != null: B packed sequences in [1, total, H, d] tensors, N = Nk = the longest one.
 static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
-                    int Hkv, int N, int Nk, int d, int causal, float scale, float tau, void* cuda_stream) {
+                    int Hkv, int N, int Nk, int d, int causal, float scale, float tau, void* cuda_stream,
+                    const int32_t* cu = nullptr, int total = 0) {
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
   MALA_TRY(check_lengths(N, Nk, causal));
   if (!lse) return MALA_ERR_INVALID_ARG;
-  MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, N, Hq));
-  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, Nk, Hkv));
-  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, Nk, Hkv));
-  MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, N, Hq));
+  const int Bt = cu ? 1 : B, Nt = cu ? total : N, Nkt = cu ? total : Nk;   // extents of the tensors
+  MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, Bt, Nt, Hq));
+  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, Bt, Nkt, Hkv));
+  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, Bt, Nkt, Hkv));
+  MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, Bt, Nt, Hq));
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
@@ -196,12 +199,13 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   cudaStream_t stream = (cudaStream_t)cuda_stream;
 
   CUtensorMap tq, tk, tv;
-  if (!make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
-      !make_tensor_map_bnhd(&tk, k.p, B, Nk, Hkv, d, k.sb, k.sn, k.sh, 128) ||
-      !make_tensor_map_bnhd(&tv, v.p, B, Nk, Hkv, d, v.sb, v.sn, v.sh, 128))
+  if (!make_tensor_map_bnhd(&tq, q.p, Bt, Nt, Hq, d, q.sb, q.sn, q.sh, 128) ||
+      !make_tensor_map_bnhd(&tk, k.p, Bt, Nkt, Hkv, d, k.sb, k.sn, k.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, v.p, Bt, Nkt, Hkv, d, v.sb, v.sn, v.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
   FwdParams p;
+  p.cu = cu; p.total = total;
   p.o = (__nv_bfloat16*)o.p; p.o_sb = o.sb; p.o_sn = o.sn; p.o_sh = o.sh;
   p.lse = lse;
   p.retained = st ? st->retained_per_block : nullptr;
@@ -236,11 +240,14 @@ int mala_fwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, 
 }
 
 static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
-                    mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int Nk, int d,
-                    int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
-  MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
-  MALA_TRY(check_lengths(N, Nk, causal));
+                    mala_tout dk, mala_tout dv, const mala_stats* st, int B0, int Hq, int Hkv, int N0, int Nk0, int d,
+                    int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream,
+                    const int32_t* cu = nullptr, int total = 0) {
+  MALA_TRY(check_common(B0, Hq, Hkv, N0, d, scale, tau));
+  MALA_TRY(check_lengths(N0, Nk0, causal));
   if (!lse || !ws) return MALA_ERR_INVALID_ARG;
+  // extents of the tensors and of the workspace (packed sequences: one batch entry of `total` rows)
+  const int B = cu ? 1 : B0, N = cu ? total : N0, Nk = cu ? total : Nk0;
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, N, Hq));
   MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, Nk, Hkv));
   MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, Nk, Hkv));
@@ -250,13 +257,13 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
   MALA_TRY(check_view(dk.p, dk.sb, dk.sn, dk.sh, B, Nk, Hkv));
   MALA_TRY(check_view(dv.p, dv.sb, dv.sn, dv.sh, B, Nk, Hkv));
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-  if (ws_bytes < bwd_workspace_bytes(B, Hq, N, d)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + 128 * B0 : N, d)) return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
   MALA_TRY(device_setup(dev, &status));
-  return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, N, Nk, d, causal ? 1 : 0, scale, tau, ws,
-                    status, (cudaStream_t)cuda_stream);
+  return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B0, Hq, Hkv, N0, Nk0, d, causal ? 1 : 0, scale, tau, ws,
+                    status, (cudaStream_t)cuda_stream, cu, total);
 }
 
 int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
@@ -271,6 +278,31 @@ int mala_bwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout
                    int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
   return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, ws, ws_bytes,
                   cuda_stream);
+}
+
+static int check_packed(const int32_t* cu_seqlens, int B, int total, int max_seqlen) {
+  if (!cu_seqlens || B <= 0 || total <= 0 || max_seqlen <= 0) return MALA_ERR_INVALID_ARG;
+  if ((((uintptr_t)cu_seqlens) & 3) != 0) return MALA_ERR_MISALIGNED;
+  if (max_seqlen > total || (long long)total + 128LL * B > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
+  return MALA_OK;
+}
+
+int mala_fwd_varlen(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu_seqlens, mala_tout o, float* lse,
+                    const mala_stats* st, int B, int Hq, int Hkv, int total, int max_seqlen, int d, int causal,
+                    float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  MALA_TRY(check_packed(cu_seqlens, B, total, max_seqlen));
+  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau, cuda_stream,
+                  cu_seqlens, total);
+}
+
+int mala_bwd_varlen(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,
+                    const int32_t* cu_seqlens, mala_tout dq, mala_tout dk, mala_tout dv, const mala_stats* st, int B,
+                    int Hq, int Hkv, int total, int max_seqlen, int d, int causal, float scale, float tau, void* ws,
+                    size_t ws_bytes, void* cuda_stream) {
+  MALA_TRY(check_packed(cu_seqlens, B, total, max_seqlen));
+  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau,
+                  ws, ws_bytes, cuda_stream, cu_seqlens, total);
 }
 
 int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,

@@ -56,6 +56,11 @@ struct BwdParams {
   int* status;
   int B, Hq, Hkv, N, Np, T, words, causal;   // N, Np, T: query rows, padded query rows, query blocks
   int Nk, Tk, koff;     // keys, key blocks; causal: the queries are the last N positions, koff = (Nk - N) / 128
+  // Packed sequences of different lengths (null: B sequences of N rows each): sequence b holds rows cu[b] ..
+  // cu[b+1]-1 of the [1, total, H, d] tensors.  N, T, Nk, Tk then describe the longest sequence (grid, telemetry
+  // strides); the per-query vectors are [Hq, Np] and the dQ accumulator [Hq, Np, D] with Np >= total + 128 B, where
+  // sequence b owns the rows from (cu[b] + 128 b) / 128 * 128 on (tile-aligned, never overlapping the next one's).
+  const int* cu;
   float scale, scale_log2;
 };
 
@@ -98,8 +103,16 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int j = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
   const int G = p.Hq / p.Hkv;
+  // this sequence: first row in the tensors, rows, blocks, first row in the padded per-head arrays
+  const int row0 = p.cu ? __ldg(p.cu + b) : 0;
+  const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
+  const int Nkeys = p.cu ? Nq : p.Nk;
+  const int T = p.cu ? (Nq + 127) / 128 : p.T;
+  const int bz = p.cu ? 0 : b;                         // outermost TMA coordinate
+  const int prow0 = p.cu ? ((row0 + 128 * b) / 128) * 128 : 0;
+  if (p.cu && j >= T) return;                          // (a sequence shorter than the longest one)
   const int i0 = p.causal ? max(j - p.koff, 0) : 0;   // first query block that sees key block j
-  const int ni = p.T - i0;
+  const int ni = T - i0;
   const int n_tot = G * ni;
   int* status = p.status;
 
@@ -135,27 +148,27 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmDO);
       mbar_arrive_expect_tx(&kv_full, 2 * Cfg::kTileBytes);
       for (int pn = 0; pn < PAN; ++pn) {
-        tma_load_4d(sK + pn * 16384, &tmK, &kv_full, pn * 64, j * 128, hkv, b);
-        tma_load_4d(sV + pn * 16384, &tmV, &kv_full, pn * 64, j * 128, hkv, b);
+        tma_load_4d(sK + pn * 16384, &tmK, &kv_full, pn * 64, row0 + j * 128, hkv, bz);
+        tma_load_4d(sV + pn * 16384, &tmV, &kv_full, pn * 64, row0 + j * 128, hkv, bz);
       }
       bool ok = true;
       int issued = 0;
       int hq = hkv * G, i = i0;   // tile n = (query head, query block), kept by increments: no division per tile
       for (int n = 0; n < n_tot && ok; ++n, ++i) {
-        if (i == p.T) { i = i0; ++hq; }
+        if (i == T) { i = i0; ++hq; }
         const int s = n & 1;
         ok = mbar_wait(&q_empty[s], ((n >> 1) & 1) ^ 1, status);
         if (!ok) break;
         mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, i * 128, hq, b);
+          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128, hq, bz);
         // dO of every tile is fetched ahead, retained or not (the vote comes too late to hide the copy behind it);
         // a skipped tile's stage is handed straight back by the issuer
         ok = mbar_wait(&do_empty[s], ((n >> 1) & 1) ^ 1, status);
         if (!ok) { mbar_wait(&q_full[s], (n >> 1) & 1, status); break; }
         mbar_arrive_expect_tx(&do_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, i * 128, hq, b);
+          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, row0 + i * 128, hq, bz);
         issued = n + 1;
       }
       if (!ok) {
@@ -292,7 +305,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const int qt = (warp - 4) >> 2;                 // column quarter
-    const bool valid_key = (j * 128 + rl) < p.Nk;
+    const bool valid_key = (j * 128 + rl) < Nkeys;
     const float c2 = p.scale_log2;
     const bool stat_thread = (warp == 4 && lane == 0);
     bool ok = true;
@@ -302,7 +315,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     int bm_word = -1;
 
     auto vec_index = [&](int hq_local, int i) -> size_t {
-      return ((size_t)b * p.Hq + hkv * G + hq_local) * p.Np + (size_t)i * 128 + rl;
+      return ((size_t)bz * p.Hq + hkv * G + hq_local) * p.Np + (size_t)prow0 + (size_t)i * 128 + rl;
     };
     // per-query vectors of tile 0 into slot 0 (published by the first column quarter), then a group sync
     if (qt == 0) {
@@ -319,8 +332,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // tile n = (query head hq_n of the group, query block i): kept by increments, no division per tile
     int hq_n = 0, i = i0, slot = 0;
     for (int n = 0; n < n_tot && ok; ++n, ++i, slot = (slot == 2 ? 0 : slot + 1)) {
-      if (i == p.T) { i = i0; ++hq_n; }
-      const bool first_of_head = (i == i0), last_of_head = (i == p.T - 1);
+      if (i == T) { i = i0; ++hq_n; }
+      const bool first_of_head = (i == i0), last_of_head = (i == T - 1);
       // prefetch the per-query vectors of the next tile
       float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
       if (qt == 0 && n + 1 < n_tot) {
@@ -334,6 +347,11 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       uint32_t sc[32];
       tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + qt * 32), sc);
       tmem_wait_ld();
+      if (p.cu && !valid_key) {   // packed sequences: a row past this sequence's end holds the next one's key
+        const uint32_t ninf = 0xff800000u;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) sc[e] = ninf;
+      }
       if (p.causal && i + p.koff == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
         const uint32_t ninf = 0xff800000u;
         const int c0 = qt * 32;
@@ -475,8 +493,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (ok) {
       tc_fence_after();
       const int key = j * 128 + rl;
-      __nv_bfloat16* dvrow = p.dv + (int64_t)b * p.dv_sb + (int64_t)key * p.dv_sn + (int64_t)hkv * p.dv_sh;
-      __nv_bfloat16* dkrow = p.dk + (int64_t)b * p.dk_sb + (int64_t)key * p.dk_sn + (int64_t)hkv * p.dk_sh;
+      __nv_bfloat16* dvrow = p.dv + (int64_t)bz * p.dv_sb + (int64_t)(row0 + key) * p.dv_sn + (int64_t)hkv * p.dv_sh;
+      __nv_bfloat16* dkrow = p.dk + (int64_t)bz * p.dk_sb + (int64_t)(row0 + key) * p.dk_sn + (int64_t)hkv * p.dk_sh;
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
         __nv_bfloat16* out = which ? dkrow : dvrow;
@@ -530,7 +548,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
-      const int tile = (int)(((size_t)b * p.Hq + hq) * p.T + (size_t)i);
+      const int tile = p.cu ? (int)((size_t)hq * (p.Np / 128) + (size_t)(prow0 / 128 + i))
+                            : (int)(((size_t)b * p.Hq + hq) * p.T + (size_t)i);
       uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // D / 64 panels of 16 KB
       uint32_t a[D / 32][32];
 #pragma unroll
@@ -582,26 +601,38 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (warp == 0) tmem_dealloc(tb, 512);
 }
 
-// D = rowsum(O o dO), lse2 = lse * log2(e), bq = lse2 + log2(tau / L_q); one warp per (b, h, row).
+// D = rowsum(O o dO), lse2 = lse * log2(e), bq = lse2 + log2(tau / L_q); one warp per (b, h, row) with row below
+// Npg, the padded length of the (longest) sequence.  Packed sequences (cu != null): the vectors are [Hq, Np] with
+// sequence b's rows from (cu[b] + 128 b) / 128 * 128 on, lse is [Hq, total].
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sn, int64_t o_sh,
                                       const __nv_bfloat16* __restrict__ dout, int64_t d_sb, int64_t d_sn, int64_t d_sh,
                                       const float* __restrict__ lse, float* __restrict__ lse2, float* __restrict__ bq,
                                       float* __restrict__ Dq, int B, int Hq, int N, int Np, int Nk, int d, int causal,
-                                      float log2_tau) {
+                                      float log2_tau, const int* __restrict__ cu, int total_rows, int Npg) {
   const int warps_per_block = blockDim.x >> 5;
-  const long long w = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const long long wi = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  const long long total = (long long)B * Hq * Np;
-  if (w >= total) return;
-  const int row = (int)(w % Np);
-  const int h = (int)((w / Np) % Hq);
-  const int b = (int)(w / ((long long)Np * Hq));
+  const long long total = (long long)B * Hq * Npg;
+  if (wi >= total) return;
+  const int row = (int)(wi % Npg);
+  const int h = (int)((wi / Npg) % Hq);
+  int b = (int)(wi / ((long long)Npg * Hq));
+  long long w = wi;                                  // index into the vectors
+  int row0 = 0;
+  if (cu) {
+    row0 = cu[b];
+    N = cu[b + 1] - row0;
+    Nk = N;
+    if (row >= ((N + 127) / 128) * 128) return;      // beyond this sequence's padded rows
+    w = (long long)h * Np + ((row0 + 128 * b) / 128) * 128 + row;
+    b = 0;
+  }
   if (row >= N) {
     if (lane == 0) { lse2[w] = INFINITY; bq[w] = INFINITY; Dq[w] = 0.f; }
     return;
   }
-  const __nv_bfloat16* op = o + b * o_sb + row * o_sn + h * o_sh;
-  const __nv_bfloat16* dp = dout + b * d_sb + row * d_sn + h * d_sh;
+  const __nv_bfloat16* op = o + b * o_sb + (int64_t)(row0 + row) * o_sn + h * o_sh;
+  const __nv_bfloat16* dp = dout + b * d_sb + (int64_t)(row0 + row) * d_sn + h * d_sh;
   float acc = 0.f;
   for (int c = lane * 2; c < d; c += 64) {
     const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(op + c);
@@ -611,7 +642,7 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
 #pragma unroll
   for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
   if (lane == 0) {
-    const float l2 = lse[((size_t)b * Hq + h) * N + row] * 1.4426950408889634f;
+    const float l2 = lse[cu ? (size_t)h * total_rows + row0 + row : ((size_t)b * Hq + h) * N + row] * 1.4426950408889634f;
     const float L = causal ? (float)(row + 1 + (Nk - N)) : (float)Nk;   // visible keys
     lse2[w] = l2;
     bq[w] = l2 + (log2_tau - log2f(L));
@@ -621,20 +652,32 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
 
 // dq = bf16(scale * acc); one thread per 8 output elements.  The accumulator is tiled (see the file header):
 // consecutive threads take consecutive rows of a tile.
+// (Packed sequences, cu != null: the index runs over (b, h, block i of the longest sequence); the accumulator is
+// [Hq, Np, d] with sequence b's tiles from (cu[b] + 128 b) / 128 on.)
 __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int64_t sb,
-                                      int64_t sn, int64_t sh, int B, int Hq, int N, int Np, int d, float scale) {
+                                      int64_t sn, int64_t sh, int B, int Hq, int N, int Np, int d, float scale,
+                                      const int* __restrict__ cu, int Npg) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = d / 8;
-  const long long total = (long long)B * Hq * Np * per_row;
+  const long long total = (long long)B * Hq * Npg * per_row;
   if (idx >= total) return;
   const int r = (int)(idx % 128);
   const int cg = (int)((idx / 128) % per_row);             // columns 8 cg .. 8 cg + 7
-  const long long tile = idx / (128LL * per_row);          // (b * Hq + h) * (Np / 128) + i
-  const int T = Np / 128;
+  long long tile = idx / (128LL * per_row);                // (b * Hq + h) * (Npg / 128) + i
+  const int T = Npg / 128;
   const int i = (int)(tile % T);
   const int h = (int)((tile / T) % Hq);
-  const int b = (int)(tile / ((long long)T * Hq));
-  const int row = i * 128 + r;
+  int b = (int)(tile / ((long long)T * Hq));
+  int row = i * 128 + r;
+  if (cu) {
+    const int row0 = cu[b];
+    N = cu[b + 1] - row0;
+    if (row >= N) return;
+    tile = (long long)h * (Np / 128) + (row0 + 128 * b) / 128 + i;
+    row += row0;
+    N += row0;
+    b = 0;
+  }
   if (row >= N) return;
   const int half = d / 2;
   const float* base = acc + (size_t)tile * 128 * d;
@@ -658,6 +701,7 @@ __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat
 
 inline size_t bwd_align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// (Packed sequences: B = 1 and N = total rows + 128 x number of sequences.)
 inline size_t bwd_workspace_bytes(int B, int Hq, int N, int d) {
   const size_t Np = (size_t)((N + 127) / 128) * 128;
   return bwd_align256((size_t)B * Hq * Np * d * sizeof(float)) + 3 * bwd_align256((size_t)B * Hq * Np * sizeof(float));
@@ -682,25 +726,32 @@ inline int bwd_launch_main(const CUtensorMap& tq, const CUtensorMap& tk, const C
 
 inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
                       mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int Nk, int d,
-                      int causal, float scale, float tau, void* ws, int* status, cudaStream_t stream) {
-  const int T = (N + 127) / 128, Np = T * 128, Tk = (Nk + 127) / 128;
+                      int causal, float scale, float tau, void* ws, int* status, cudaStream_t stream,
+                      const int* cu = nullptr, int total = 0) {
+  // Packed sequences (cu): N = Nk = the longest sequence; the tensors are [1, total, H, d]; the per-query vectors and
+  // the dQ accumulator are laid out per head over Np = total + 128 B rows (rounded up to a tile).
+  const int T = (N + 127) / 128, Npg = T * 128, Tk = (Nk + 127) / 128;
+  const int Np = cu ? ((total + 128 * B + 127) / 128) * 128 : Npg;
+  const int Bl = cu ? 1 : B;                 // batch extent of the tensors and of the workspace arrays
+  const int Nt = cu ? total : N, Nkt = cu ? total : Nk;   // row extents of the tensors
   uint8_t* w = (uint8_t*)ws;
   float* acc = (float*)w;
-  w += bwd_align256((size_t)B * Hq * Np * d * sizeof(float));
-  const size_t vbytes = bwd_align256((size_t)B * Hq * Np * sizeof(float));
+  w += bwd_align256((size_t)Bl * Hq * Np * d * sizeof(float));
+  const size_t vbytes = bwd_align256((size_t)Bl * Hq * Np * sizeof(float));
   float* lse2 = (float*)w;
   float* bq = (float*)(w + vbytes);
   float* Dq = (float*)(w + 2 * vbytes);
 
   CUtensorMap tq, tk, tv, tdo, tacc;
-  if (!make_tensor_map_f32_tiles(&tacc, acc + 64 * d, (uint64_t)B * Hq * T, d / 2, (uint64_t)128 * d * sizeof(float)) ||
-      !make_tensor_map_bnhd(&tq, q.p, B, N, Hq, d, q.sb, q.sn, q.sh, 128) ||
-      !make_tensor_map_bnhd(&tk, k.p, B, Nk, Hkv, d, k.sb, k.sn, k.sh, 128) ||
-      !make_tensor_map_bnhd(&tv, v.p, B, Nk, Hkv, d, v.sb, v.sn, v.sh, 128) ||
-      !make_tensor_map_bnhd(&tdo, dout.p, B, N, Hq, d, dout.sb, dout.sn, dout.sh, 128))
+  if (!make_tensor_map_f32_tiles(&tacc, acc + 64 * d, (uint64_t)Bl * Hq * (Np / 128), d / 2,
+                                 (uint64_t)128 * d * sizeof(float)) ||
+      !make_tensor_map_bnhd(&tq, q.p, Bl, Nt, Hq, d, q.sb, q.sn, q.sh, 128) ||
+      !make_tensor_map_bnhd(&tk, k.p, Bl, Nkt, Hkv, d, k.sb, k.sn, k.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, v.p, Bl, Nkt, Hkv, d, v.sb, v.sn, v.sh, 128) ||
+      !make_tensor_map_bnhd(&tdo, dout.p, Bl, Nt, Hq, d, dout.sb, dout.sn, dout.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
-  if (cudaMemsetAsync(acc, 0, (size_t)B * Hq * Np * d * sizeof(float), stream) != cudaSuccess) return MALA_ERR_CUDA;
+  if (cudaMemsetAsync(acc, 0, (size_t)Bl * Hq * Np * d * sizeof(float), stream) != cudaSuccess) return MALA_ERR_CUDA;
   BwdParams p;
   p.lse2 = lse2; p.bq = bq; p.Dq = Dq; p.dq_acc = acc;
   p.dk = (__nv_bfloat16*)dk.p; p.dk_sb = dk.sb; p.dk_sn = dk.sn; p.dk_sh = dk.sh;
@@ -711,19 +762,20 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   p.status = status;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Np = Np; p.T = T; p.words = (T + 31) / 32; p.causal = causal;
   p.Nk = Nk; p.Tk = Tk; p.koff = causal ? (Nk - N) / 128 : 0;
+  p.cu = cu;
   p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
   if (p.bitmask &&
       cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * Tk * p.words * sizeof(uint32_t), stream) != cudaSuccess)
     return MALA_ERR_CUDA;
 
   {
-    const long long rows = (long long)B * Hq * Np;
+    const long long rows = (long long)B * Hq * Npg;
     const int wpb = 8;
     const unsigned blocks = (unsigned)((rows + wpb - 1) / wpb);
     bwd_preprocess_kernel<<<blocks, wpb * 32, 0, stream>>>((const __nv_bfloat16*)o.p, o.sb, o.sn, o.sh,
                                                           (const __nv_bfloat16*)dout.p, dout.sb, dout.sn, dout.sh, lse,
                                                           lse2, bq, Dq, B, Hq, N, Np, Nk, d, causal,
-                                                          tau > 0.f ? log2f(tau) : -INFINITY);
+                                                          tau > 0.f ? log2f(tau) : -INFINITY, cu, total, Npg);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   const bool dense = (tau == 0.f);
@@ -732,10 +784,10 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   else rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, tacc, p, stream);
   if (rc != MALA_OK) return rc;
   {
-    const long long total = (long long)B * Hq * Np * (d / 8);
-    const unsigned blocks = (unsigned)((total + 255) / 256);
+    const long long n_out = (long long)B * Hq * Npg * (d / 8);
+    const unsigned blocks = (unsigned)((n_out + 255) / 256);
     bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(acc, (__nv_bfloat16*)dq.p, dq.sb, dq.sn, dq.sh, B, Hq, N, Np, d,
-                                                      scale);
+                                                      scale, cu, Npg);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   return MALA_OK;

@@ -32,6 +32,11 @@ struct FwdParams {
   int* status;
   int B, Hq, Hkv, N, Tr, words, causal;   // N, Tr: query rows and query blocks
   int Nk, Tk, koff;              // keys, key blocks; causal: the queries are the last N positions, koff = (Nk - N) / 128
+  // Packed sequences of different lengths (null: B sequences of N rows each): sequence b holds rows
+  // cu[b] .. cu[b+1]-1 of q, k, v, o (which are then [1, total, H, d] tensors); lse is [Hq, total]; N, Tr, Nk, Tk
+  // above describe the longest sequence (grid, telemetry strides)
+  const int* cu;
+  int total;
   float scale_log2;              // scale * log2(e)
   float log2_tau;                // log2(tau); unused by the dense kernel
 };
@@ -68,12 +73,20 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.Hq / p.Hkv;
   const int b = blockIdx.z, h = blockIdx.y, hkv = h / G;
-  const int npairs = (p.Tr + 1) / 2;
+  // this sequence: first row in the tensors, rows, blocks (packed sequences: equal query and key lengths)
+  const int row0 = p.cu ? __ldg(p.cu + b) : 0;
+  const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
+  const int Nkeys = p.cu ? Nq : p.Nk;
+  const int Tr = p.cu ? (Nq + 127) / 128 : p.Tr;
+  const int Tk = p.cu ? Tr : p.Tk;
+  const int bz = p.cu ? 0 : b;                        // outermost TMA coordinate
+  const int npairs = (Tr + 1) / 2;
+  if ((int)blockIdx.x >= npairs) return;             // (a sequence shorter than the longest one)
   const int c = npairs - 1 - (int)blockIdx.x;        // longest pairs first
   const int iA = 2 * c, iB = 2 * c + 1;
-  const bool hasB = iB < p.Tr;
+  const bool hasB = iB < Tr;
   // key steps u = 0 .. U-1 visit key block j0 - u; block X takes part from step first[X] on
-  const int j0 = p.causal ? (hasB ? iB : iA) + p.koff : (p.Tk - 1);
+  const int j0 = p.causal ? (hasB ? iB : iA) + p.koff : (Tk - 1);
   const int U = j0 + 1;
   const int firstA = (p.causal && hasB) ? 1 : 0;     // B's diagonal key block is not legal for A
   int* status = p.status;
@@ -107,8 +120,8 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
       mbar_arrive_expect_tx(&q_full, (hasB ? 2 : 1) * Cfg::kTileBytes);
       for (int pn = 0; pn < PAN; ++pn) {
-        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, iA * 128, h, b);
-        if (hasB) tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, iB * 128, h, b);
+        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iA * 128, h, bz);
+        if (hasB) tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iB * 128, h, bz);
       }
       int issued = 0, v_issued = 0, s = 0;
       uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
@@ -118,7 +131,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, (j0 - u) * 128, hkv, b);
+          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, row0 + (j0 - u) * 128, hkv, bz);
         issued = u + 1;
         if (++s == KS) { s = 0; par ^= 1; }
         if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
@@ -126,7 +139,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (!ok) break;
           mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
           for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, (j0 - u) * 128, hkv, b);
+            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, row0 + (j0 - u) * 128, hkv, bz);
           v_issued = u + 1;
         }
       }
@@ -212,7 +225,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (leader) {
               mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
               for (int pn = 0; pn < PAN; ++pn)
-                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, (j0 - u) * 128, hkv, b);
+                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, row0 + (j0 - u) * 128, hkv, bz);
             }
             __syncwarp();
           }
@@ -254,9 +267,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const int row = i * 128 + rl;
-    const bool valid = row < p.N;
+    const bool valid = row < Nq;
     const float c2 = p.scale_log2;
-    const float Lq = p.causal ? (float)(row + 1 + p.koff * 128) : (float)p.Nk;   // visible keys
+    const float Lq = p.causal ? (float)(row + 1 + p.koff * 128) : (float)Nkeys;   // visible keys
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f(Lq));
     const uint32_t colS = (uint32_t)x * 128u, colO = 256u + (uint32_t)x * 128u;
     const int first = (x == 0) ? firstA : 0;
@@ -284,7 +297,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tmem_wait_ld();
       if (t == 0) {
         // first visited tile: causal diagonal and / or the ragged end of the key range
-        const int lim = p.causal ? rl : (p.Nk - 1 - j * 128);
+        const int lim = p.causal ? rl : (Nkeys - 1 - j * 128);
         const uint32_t ninf = 0xff800000u;
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
@@ -438,7 +451,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (ok && present_x) {
       tc_fence_after();
       const float inv = 1.f / l;
-      __nv_bfloat16* orow = p.o + (int64_t)b * p.o_sb + (int64_t)row * p.o_sn + (int64_t)h * p.o_sh;
+      __nv_bfloat16* orow = p.o + (int64_t)bz * p.o_sb + (int64_t)(row0 + row) * p.o_sn + (int64_t)h * p.o_sh;
 #pragma unroll
       for (int cc = 0; cc < D / 32; ++cc) {
         uint32_t o[32];
@@ -456,7 +469,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
       }
-      if (valid) p.lse[((size_t)b * p.Hq + h) * p.N + row] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      if (valid)
+        p.lse[p.cu ? (size_t)h * p.total + row0 + row : ((size_t)b * p.Hq + h) * p.N + row] =
+            (m_ref + log2f(l)) * 0.6931471805599453f;
       if (stat_thread) {
         if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
         if (p.retained) p.retained[stat_row] = (uint32_t)r;

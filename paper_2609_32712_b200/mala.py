@@ -55,6 +55,12 @@ def lib():
                                      i, i, i, i, i, i, i, f, f, vp, sz, vp]
         L.mala_fwd_chunk.restype = i
         L.mala_bwd_chunk.restype = i
+        L.mala_fwd_varlen.argtypes = [_TIn, _TIn, _TIn, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, f, f,
+                                      vp, sz, vp]
+        L.mala_bwd_varlen.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, vp, _TOut, _TOut, _TOut, ctypes.POINTER(_Stats),
+                                      i, i, i, i, i, i, i, f, f, vp, sz, vp]
+        L.mala_fwd_varlen.restype = i
+        L.mala_bwd_varlen.restype = i
         L.mala_decode.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp, sz, vp]
         L.mala_decode_multi.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, f, f, i,
                                         vp, sz, vp]
@@ -197,6 +203,43 @@ def bwd_chunk(q, k, v, o, do, lse, scale: float, tau: float, causal: bool = True
                               ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_bwd_chunk")
+    return dq, dk, dv, st
+
+
+def fwd_varlen(q, k, v, cu_seqlens, max_seqlen: int, scale: float, tau: float, causal: bool = True, stats: bool = False):
+    """mala_fwd_varlen: q [1,total,Hq,d], k, v [1,total,Hkv,d] packed sequences; cu_seqlens int32 [B+1] on the device.
+    Returns (o [1,total,Hq,d] bf16, lse [Hq,total] fp32, Stats or None)."""
+    one, total, Hq, d = q.shape
+    assert one == 1 and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    B, Hkv = cu_seqlens.numel() - 1, k.shape[2]
+    o = torch.empty_like(q)
+    lse = torch.empty((Hq, total), dtype=torch.float32, device=q.device)
+    T = -(-max_seqlen // 128)
+    st = Stats((B, Hq, T), -(-T // 32), q.device) if stats else None
+    rc = lib().mala_fwd_varlen(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), cu_seqlens.data_ptr(), _view(o, _TOut),
+                               lse.data_ptr(), ctypes.byref(st.c) if st else None, B, Hq, Hkv, total, max_seqlen, d,
+                               int(causal), scale, tau, None, 0, _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_fwd_varlen")
+    return o, lse, st
+
+
+def bwd_varlen(q, k, v, o, do, lse, cu_seqlens, max_seqlen: int, scale: float, tau: float, causal: bool = True,
+               stats: bool = False, ws=None):
+    """mala_bwd_varlen: returns (dq [1,total,Hq,d], dk, dv [1,total,Hkv,d], Stats or None)."""
+    one, total, Hq, d = q.shape
+    assert one == 1 and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    B, Hkv = cu_seqlens.numel() - 1, k.shape[2]
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    T = -(-max_seqlen // 128)
+    st = Stats((B, Hq, T), -(-T // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_BWD, 1, Hq, Hkv, total + 128 * B, d), q.device) if ws is None else ws
+    rc = lib().mala_bwd_varlen(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TIn), _view(do, _TIn),
+                               lse.data_ptr(), cu_seqlens.data_ptr(), _view(dq, _TOut), _view(dk, _TOut),
+                               _view(dv, _TOut), ctypes.byref(st.c) if st else None, B, Hq, Hkv, total, max_seqlen, d,
+                               int(causal), scale, tau, ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_bwd_varlen")
     return dq, dk, dv, st
 
 

@@ -243,6 +243,18 @@ def paginate(kcache: torch.Tensor, vcache: torch.Tensor, page_size: int, seqlens
     return kp, vp, bt.to(dev), torch.tensor(lens, dtype=torch.int32, device=dev)
 
 
+def pack_sequences(ws):
+    """Packed layout of several single-sequence prefill workloads (each B = 1, same heads): q, k, v, do
+    concatenated along the rows as [1, total, H, d], and cu_seqlens int32 [len(ws) + 1]."""
+    out = {x: torch.cat([w[x] for w in ws], dim=1).contiguous() for x in ("q", "k", "v", "do")}
+    lens = [w["q"].shape[1] for w in ws]
+    cu = [0]
+    for n in lens:
+        cu.append(cu[-1] + n)
+    out.update(cu_seqlens=torch.tensor(cu, dtype=torch.int32, device=out["q"].device), lens=lens, scale=ws[0]["scale"])
+    return out
+
+
 def rademacher_like(t: torch.Tensor, seed: int) -> torch.Tensor:
     """Upstream gradient of +-1 entries (the Rademacher probe of the operator-fidelity protocol, Section 5.1)."""
     gen = torch.Generator(device=t.device)

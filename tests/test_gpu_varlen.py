@@ -1,0 +1,102 @@
+"""GPU parity of mala_fwd_varlen / mala_bwd_varlen (packed sequences of different lengths) against the fp64 oracle,
+which runs every sequence on its own."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_32712_b200 import workloads as W
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mala():
+    from paper_2609_32712_b200 import mala as m
+    m.lib()
+    return m
+
+
+def _run(mala, oracle, lens, Hq, Hkv, d, tau, preset="literal", causal=True, head_types=None):
+    ws = [W.custom_prefill(1, Hq, Hkv, n, d, head_types=head_types, seed=100 + 7 * x + n, preset=preset)
+          for x, n in enumerate(lens)]
+    pk = W.pack_sequences(ws)
+    q, k, v, do, cu = (pk[x].cuda() for x in ("q", "k", "v", "do", "cu_seqlens"))
+    mx = max(lens)
+    o, lse, fst = mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], tau, causal=causal, stats=True)
+    dq, dk, dv, bst = mala.bwd_varlen(q, k, v, o, do, lse, cu, mx, pk["scale"], tau, causal=causal, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    Tm = -(-mx // 128)
+    fm, bm = fst.mask(Tm).cpu().numpy(), bst.mask(Tm).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy()[0], lse.cpu().numpy()
+    dq_c, dk_c, dv_c = (t.float().cpu().numpy()[0] for t in (dq, dk, dv))
+    skipped = legal_f = legal_b = 0
+    for b, (w, n) in enumerate(zip(ws, lens)):
+        r0 = int(pk["cu_seqlens"][b])
+        T = -(-n // 128)
+        ref = oracle.fwd(w["q"], w["k"], w["v"], w["scale"], tau, 128, 128, causal=causal)
+        for h in range(Hq):
+            for i in range(T):
+                order = list(range(i, -1, -1)) if causal else list(range(T - 1, -1, -1))
+                parity.check_mask(fm[b, h, i, :T], ref["mask"][0, h, i], ref["crit"][0, h, i], order, tau,
+                                  i * 128 + 1 if causal else n)
+                assert int(fst.retained[b, h, i]) == int(fm[b, h, i].sum())
+            assert not fm[b, h, T:].any() and not fm[b, h, :, T:].any()
+        parity.check_output(o_c[r0:r0 + n], ref["o"][0])
+        assert np.abs(lse_c[:, r0:r0 + n] - ref["lse"][0]).max() <= parity.LSE_ABS
+        # backward on the GPU's own forward output of this sequence
+        g = oracle.bwd(w["q"], w["k"], w["v"], o[:, r0:r0 + n].float().cpu(), w["do"],
+                       lse[:, r0:r0 + n].cpu().numpy()[None], w["scale"], tau, 128, 128, causal=causal)
+        for h in range(Hq):
+            for j in range(T):
+                om, oc = g["mask"][0, h, j], g["crit"][0, h, j]
+                for i in range(T):
+                    if om[i] == 0:
+                        assert not bm[b, h, j, i]
+                    elif bool(bm[b, h, j, i]) != (om[i] == 2):
+                        assert abs(oc[i]) <= parity.MASK_BAND, (b, h, j, i, oc[i])
+            assert not bm[b, h, T:].any()
+        for got, want, what in ((dq_c, g["dq"], "dq"), (dk_c, g["dk"], "dk"), (dv_c, g["dv"], "dv")):
+            if n == 1 and what != "dv":
+                # one key: p = 1 and dS = p (dP - D) = 0 exactly; the kernel's D comes from the bf16 output
+                assert np.abs(got[r0:r0 + n]).max() <= 1e-2 * np.abs(want).max() + 1e-5
+            else:
+                parity.check_grad(got[r0:r0 + n], want[0], f"{what} seq {b}")
+        skipped += int((ref["mask"] == 1).sum()) + int((g["mask"] == 1).sum())
+        legal_f += int((ref["mask"] > 0).sum())
+        legal_b += int((g["mask"] > 0).sum())
+    assert fst.totals.cpu().numpy()[1] == legal_f and bst.totals.cpu().numpy()[1] == legal_b
+    return skipped
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("lens,Hq,Hkv,d", [([128, 384, 256], 2, 1, 128), ([333, 100, 1, 517], 4, 2, 128),
+                                           ([200, 640, 129], 2, 2, 64), ([700], 2, 1, 128)])
+def test_varlen_literal(mala, oracle, lens, Hq, Hkv, d, tau):
+    _run(mala, oracle, lens, Hq, Hkv, d, tau)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+def test_varlen_skipping_regime(mala, oracle, tau):
+    sk = _run(mala, oracle, [1024, 300, 1500, 777], 4, 2, 128, tau, preset="R",
+              head_types=["diffuse", "peaked", "peaked", "sink"])
+    assert sk > 0, "workload must exercise skipping"
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-2])
+def test_varlen_non_causal(mala, oracle, tau):
+    # every key of the sequence legal: the rows of the next sequence inside a sequence's last tile must be masked
+    _run(mala, oracle, [300, 130, 450], 2, 1, 128, tau, preset="R", causal=False, head_types=["peaked", "diffuse"])
+
+
+def test_varlen_of_equal_lengths_equals_the_batched_call(mala):
+    w = W.custom_prefill(3, 4, 2, 512, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=3, preset="R")
+    q, k, v = (w[x].cuda() for x in ("q", "k", "v"))
+    cu = torch.tensor([0, 512, 1024, 1536], dtype=torch.int32, device="cuda")
+    for tau in (0.0, 1e-4):
+        o, lse, _ = mala.fwd(q, k, v, w["scale"], tau)
+        ov, lv, _ = mala.fwd_varlen(q.reshape(1, 1536, 4, 128), k.reshape(1, 1536, 2, 128), v.reshape(1, 1536, 2, 128),
+                                    cu, 512, w["scale"], tau)
+        assert torch.equal(o.reshape(1, 1536, 4, 128), ov)
+        assert torch.equal(lse.permute(1, 0, 2).reshape(4, 1536), lv)
