@@ -209,6 +209,38 @@ def chunk_leg(cs, Nq, tau, it, peaks):
     return row
 
 
+def varlen_leg(cfg, preset, lens, tau, it, peaks, dev):
+    """mala_fwd_varlen / mala_bwd_varlen on packed sequences with the heads of a prefill configuration: latency of
+    the MALA and dense kernels and the tensor-pipe fraction on the tile FLOPs executed."""
+    import torch
+    from paper_2609_32712_b200 import mala, workloads as W
+    ws = [W.custom_prefill(1, cfg.Hq, cfg.Hkv, n, cfg.d, head_types=cfg.head_types, seed=cfg.seed + 31 * x,
+                           preset=preset, device=dev) for x, n in enumerate(lens)]
+    pk = W.pack_sequences(ws)
+    q, k, v, do, cu = pk["q"], pk["k"], pk["v"], pk["do"], pk["cu_seqlens"]
+    total, mx = sum(lens), max(lens)
+    wsb = torch.empty(mala.workspace_bytes(mala.OP_BWD, 1, cfg.Hq, cfg.Hkv, total + 128 * len(lens), cfg.d),
+                      dtype=torch.uint8, device=dev)
+    row = {"lens": list(lens)}
+    o, lse, _ = mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], tau)
+    for label, t_ in (("mala", tau), ("dense", 0.0)):
+        f_ms = time_cuda(lambda: mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], t_), 3, it)
+        o, lse, _ = mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], t_)
+        b_ms = time_cuda(lambda: mala.bwd_varlen(q, k, v, o, do, lse, cu, mx, pk["scale"], t_, ws=wsb), 3, it)
+        row[label] = {"fwd_ms": f_ms, "bwd_ms": b_ms}
+    o, lse, fs = mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], tau, stats=True)
+    _, _, _, bs = mala.bwd_varlen(q, k, v, o, do, lse, cu, mx, pk["scale"], tau, ws=wsb, stats=True)
+    torch.cuda.synchronize()
+    (fr, fl), (br, bl) = fs.totals.cpu().tolist(), bs.totals.cpu().tolist()
+    row["legal_tiles"] = fl
+    row["fwd_retained_frac"], row["bwd_retained_frac"] = fr / fl, br / bl
+    row["fwd_tensor_frac_on_executed"] = (fwd_executed_flops(fl, fr, cfg.d) / (row["mala"]["fwd_ms"] * 1e-3) / 1e12
+                                          / peaks["tflops_sustained"])
+    row["bwd_tensor_frac_on_executed"] = (bwd_executed_flops(bl, br, cfg.d) / (row["mala"]["bwd_ms"] * 1e-3) / 1e12
+                                          / peaks["tflops_sustained"])
+    return row
+
+
 def fidelity(cs, taus, it):
     """Work and operator fidelity of MALA against the in-library dense path on one configuration (the protocol
     of Section 5.1 on synthetic states): retained slots per query in forward and backward, omitted softmax mass
@@ -463,6 +495,8 @@ def main():
                 row["speedup_bwd"] = row["dense"]["bwd_ms"] / row["mala"]["bwd_ms"]
                 if name == "cfg3":                  # chunked prefill: the last 8192 queries against all 32768 keys
                     row["chunk_last_8192"] = chunk_leg(cs, 8192, tau, it, peaks)
+                if name == "cfg3":                  # the same heads on packed sequences of 16K + 8K + 5000 + 3192 rows
+                    row["varlen_4seq_32768"] = varlen_leg(cc, preset, (16384, 8192, 5000, 3192), tau, it, peaks, dev)
                 if name == "cfg3" and preset == "R":
                     row["fidelity_vs_dense"] = fidelity(cs, (1e-4, 1e-2, 1.0), it)
                 detail[f"{name}_{preset}"] = row
