@@ -442,12 +442,30 @@ def main():
     dev_in = (case.q, case.k, case.v, case.do)
     dev_out = (case.o, case.dq, case.dk, case.dv)
 
+    side = torch.cuda.Stream(device=dev)
+
     def e2e_step():
-        for d_, h_ in zip(dev_in, host_in):
+        # q, k, v in, forward, backward, results out on the caller's stream; the upstream gradient comes in on a
+        # second stream while the forward runs and the forward's output goes out while the backward runs (the
+        # library's calls are asynchronous on the stream they are given, so a caller can overlap its own copies)
+        main = torch.cuda.current_stream()
+        start = main.record_event()
+        for d_, h_ in zip(dev_in[:3], host_in[:3]):
             d_.copy_(h_, non_blocking=True)
-        case.step(tau)
-        for h_, d_ in zip(host_out, dev_out):
+        with torch.cuda.stream(side):
+            side.wait_event(start)                      # the previous step's backward has read dO
+            dev_in[3].copy_(host_in[3], non_blocking=True)
+            do_in = side.record_event()
+        case.fwd(tau)
+        fwd_done = main.record_event()
+        with torch.cuda.stream(side):
+            side.wait_event(fwd_done)
+            host_out[0].copy_(dev_out[0], non_blocking=True)
+        main.wait_event(do_in)
+        case.bwd(tau)
+        for h_, d_ in zip(host_out[1:], dev_out[1:]):
             h_.copy_(d_, non_blocking=True)
+        main.wait_stream(side)
 
     e2e_iters = max(1, min(args.steps, 5))
     e2e_ms = time_cuda(e2e_step, 1, e2e_iters)
