@@ -76,6 +76,36 @@ def test_argument_validation_codes(mala):
         assert f() in (-5, -6)
 
 
+def test_argument_validation_codes_of_the_general_shape_calls(mala):
+    L = mala.lib()
+    buf = ctypes.create_string_buffer(4096)
+    base = (ctypes.addressof(buf) + 255) & ~255
+    tin = lambda: mala._TIn(base, 0, 256, 128)
+    tout = lambda: mala._TOut(base, 0, 256, 128)
+    # chunked prefill: a causal chunk starts on a tile boundary and has no more queries than keys
+    fc = lambda Nq, Nk, causal=1: L.mala_fwd_chunk(tin(), tin(), tin(), tout(), base, None, 1, 2, 2, Nq, Nk, 128, causal,
+                                                   0.1, 1e-4, None, 0, None)
+    assert fc(100, 300) == -2 and fc(512, 256) == -2 and fc(0, 256) == -1
+    bc = lambda Nq, Nk: L.mala_bwd_chunk(tin(), tin(), tin(), tin(), tin(), base, tout(), tout(), tout(), None, 1, 2, 2,
+                                         Nq, Nk, 128, 1, 0.1, 1e-4, base, 1 << 20, None)
+    assert bc(100, 300) == -2 and bc(128, 0) == -1
+    # packed sequences: cu_seqlens required, longest sequence within the total
+    fv = lambda cu, total, mx: L.mala_fwd_varlen(tin(), tin(), tin(), cu, tout(), base, None, 2, 2, 2, total, mx, 128, 1,
+                                                 0.1, 1e-4, None, 0, None)
+    assert fv(None, 256, 128) == -1 and fv(base, 0, 128) == -1 and fv(base, 256, 512) == -2 and fv(base + 2, 256, 128) == -3
+    # several tokens per decode step: at most 16 rows per KV head, no more new tokens than keys
+    dm = lambda Sq, Hq=4, Nk=256: L.mala_decode_multi(tin(), tin(), tin(), tout(), None, None, 1, Hq, 1, Nk, Sq, 128, 0.1,
+                                                      1e-4, 2, base, 1 << 20, None)
+    assert dm(0) == -1 and dm(5) == -2 and dm(2, Hq=16) == -2 and dm(4, Nk=3) == -2
+    # paged decode: pages of whole tiles, a block table
+    dp = lambda page, bt=base: L.mala_decode_paged(tin(), tin(), tin(), bt, None, tout(), None, None, 1, 4, 1, 8, page, 4,
+                                                   128, 0.1, 1e-4, 2, base, 1 << 20, None)
+    assert dp(64) == -2 and dp(200) == -2 and dp(0) == -1 and dp(128, bt=None) == -1 and dp(128, bt=base + 1) == -3
+    # workspace of a decode step with several tokens: as for that many more sequences
+    assert mala.workspace_bytes(mala.OP_DECODE, 8 * 4, 32, 8, 131072, 128, 128) == 4 * mala.workspace_bytes(
+        mala.OP_DECODE, 8, 32, 8, 131072, 128, 128)
+
+
 def test_binding_has_no_cpu_fallback(mala):
     if torch.cuda.is_available():
         pytest.skip("GPU present")
