@@ -18,8 +18,11 @@
 //              the moment its vote is known) and O^T += V^T P^T (as soon as P^T and V are there).  No step waits
 //              for another one's data, so the HBM latency of a V copy that can only be requested after the vote
 //              is hidden behind the tiles that follow.
-//   warps 4-7  softmax group, thread = key of the tile: per-head maxima and sums by warp shuffles and one small
+//   warps 4-7  softmax group, thread = key of the tile: per-row maxima and sums by warp shuffles and one small
 //              exchange per tile between the four warps, Eq. 3, P^T -> smem; lazy rescale of O^T
+//   warps 8-11 second softmax group when the item has eight or more rows: each group takes half of the rows (its
+//              own score columns, P^T rows and O^T columns of the same TMEM lanes); the tile is retained if either
+//              group's rows need it
 // K is always streamed; a skipped tile issues no exp, no P, no V load and no PV.
 // The cache may be held in pages (pages of whole tiles, looked up in a block table by the producer, which hands
 // the V tile's coordinates to the UMMA warp) and every sequence may have its own length (which then takes the
@@ -51,7 +54,7 @@ struct DecCfg {
   static constexpr int kPBytes = 4096;                   // P^T: 16 rows (heads) x 128 keys, two 2 KB panels
   static constexpr int kKStages = 3, kVStages = 3, kPStages = 4, kSStages = 4;
   static constexpr int kSmemBytes = 2 * kQBytes + (kKStages + kVStages) * kTileBytes + kPStages * kPBytes + 1024;
-  static constexpr int kThreads = 256;
+  static constexpr int kThreads = 384;                   // producer, UMMA warp, two idle warps, up to two softmax groups
   static constexpr uint32_t kTmemCols = 128;             // S^T ring 4 x 16, O^T 2 x 16 (item parity)
   static constexpr uint32_t kColO = 64;
 };
@@ -103,10 +106,13 @@ __device__ __forceinline__ void lds_row(const float* src, float (&dst)[N]) {
 // softmax group unroll without branches).  kMulti: several new tokens per sequence, i.e. rows that see
 // different numbers of keys (one token: every row sees all keys, and the per-row limits fold into scalars).
 template <bool kDense, int GP, bool kMulti>
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(384, 1)
 mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                          const __grid_constant__ CUtensorMap tmV, const DecParams p) {
   constexpr int KS = DecCfg::kKStages, VS = DecCfg::kVStages, TB = DecCfg::kTileBytes;
+  constexpr int NG = GP >= 8 ? 2 : 1;      // softmax groups (four warps each)
+  constexpr int GH = GP / NG;              // rows per group
+  constexpr int LDN = NG == 1 ? 16 : GH;   // TMEM columns a softmax thread reads at a time
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                      // [2] item parity
@@ -115,11 +121,11 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   uint8_t* sP = sV + VS * TB;              // [4] P^T ring
 
   __shared__ uint64_t q_full[2], q_empty[2], k_full[KS], k_empty[KS], v_full[VS], v_empty[VS], s_full[4], s_free[4],
-      vote_bar[4], p_full[4], p_free[4], item_done[2], o_free[2], fin_bar, grp_a;
+      vote_bar[4], p_full[4], p_free[4], item_done[2], o_free[2], fin_bar, grp_a[2];
   __shared__ uint32_t tmem_base_s;
-  __shared__ int flag[4];
+  __shared__ int flag[2][4];               // [softmax group][vote ring]
   __shared__ int v_row[8], v_outer[8];     // TMA coordinates of the V tile of tile g (ring; written by the producer)
-  __shared__ __align__(16) float xch_max[2][4][16], xch_sum[2][4][16];   // the softmax group's per-tile exchange
+  __shared__ __align__(16) float xch_max[2][2][4][8], xch_sum[2][2][4][8];   // [buffer][group][warp][row]: per-tile exchange
   __shared__ int early_exit;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -129,21 +135,23 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 
   // the Q tile of an item has R <= 16 rows; the other rows of the two stages are never written: clear them once
   for (int i = tid; i < 2 * DecCfg::kQBytes / 16; i += DecCfg::kThreads) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0u, 0u, 0u, 0u);
+  // likewise the rows R..15 of the P^T ring, so that those columns of O^T stay finite
+  for (int i = tid; i < DecCfg::kPStages * DecCfg::kPBytes / 16; i += DecCfg::kThreads) reinterpret_cast<uint4*>(sP)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async_smem();
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&item_done[s], 1); mbar_init(&o_free[s], 4);
+      mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&item_done[s], 1); mbar_init(&o_free[s], 4 * NG);
+      mbar_init(&grp_a[s], 4);
     }
     for (int s = 0; s < KS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1); }
     for (int s = 0; s < VS; ++s) { mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1); }
     for (int s = 0; s < 4; ++s) {
-      mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4); mbar_init(&vote_bar[s], 1);
-      mbar_init(&p_full[s], 4); mbar_init(&p_free[s], 1);
-      flag[s] = 0;
+      mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4 * NG); mbar_init(&vote_bar[s], NG);
+      mbar_init(&p_full[s], 4 * NG); mbar_init(&p_free[s], 1);
+      flag[0][s] = flag[1][s] = 0;
     }
     mbar_init(&fin_bar, 1);
-    mbar_init(&grp_a, 4);
     mbar_fence_init();
   }
   __syncthreads();
@@ -296,7 +304,8 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             advance(cv);
             progress = true;
           } else if (ready(&vote_bar[cv.g & 3], (cv.g >> 2) & 1)) {
-            const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[cv.g & 3], 0) != 0;
+            const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[0][cv.g & 3] |
+                                                                  (NG > 1 ? *(volatile int*)&flag[1][cv.g & 3] : 0), 0) != 0;
             if (!retain) {
               ret_bits &= ~(1u << (cv.g & 3));
               advance(cv);
@@ -363,35 +372,38 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       mbar_wait_warp(&fin_bar, 0, status);
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
     }
-  } else if (warp >= 4) {
-    // ------------------------------------------------------------------ softmax group: thread = key of the tile
-    // One exchange per tile between the four warps: every warp publishes the per-head maxima of its 32 keys of
-    // this tile together with its per-head sums of P of the previous retained tile; after one group barrier every
-    // thread holds the tile's row maxima and the up-to-date normalizers, evaluates Eq. 3 itself, and goes on.
+  } else if (warp >= 4 && ((warp - 4) >> 2) < NG) {
+    // ------------------------------------------------------------------ softmax groups: thread = key of the tile
+    // A group of four warps handles GH rows (all of them, or half of them each when there are eight or more: the
+    // rows are independent of one another except for the tile's vote).  One exchange per tile between the four
+    // warps of a group: every warp publishes the per-row maxima of its 32 keys of this tile together with its
+    // per-row sums of P of the previous retained tile; after one group barrier every thread holds the tile's row
+    // maxima and the up-to-date normalizers and evaluates Eq. 3 for the group's rows itself.
     const int w = warp & 3;
+    const int grp = (warp - 4) >> 2;               // softmax group
+    const int rb = grp * GH;                       // its first row
     const uint32_t lane_base = (uint32_t)w * 32u;
     const int kt = (int)lane_base + lane;          // key inside the tile; output channel in the epilogue
-    // rows G..15 of the P^T tiles are never written: clear the ring once so that those columns of O^T stay finite
-    for (int i = kt; i < DecCfg::kPStages * DecCfg::kPBytes / 16; i += 128) reinterpret_cast<uint4*>(sP)[i] = make_uint4(0u, 0u, 0u, 0u);
-    fence_proxy_async_smem();
     const float c2 = p.scale_log2;
-    const bool head = (kt == 0);                   // the thread that keeps the telemetry
+    const bool ghead = (kt == 0);                  // the thread that casts the group's vote
+    const bool head = ghead && grp == 0;           // the thread that keeps the telemetry
     // The reference of the exponentials follows the scores only when they exceed it by 2^60: fp32 sums and bf16 P
     // have the exponent range for it, and moving the reference means waiting until every PV issued so far has
     // retired (their V copies included), which would stall this group for a whole HBM round trip.
     constexpr float kRescaleGap = 60.f;
     // row q = token tok[q] of the Sq new ones (the last positions of the cache), head q - tok[q] * G of the group:
     // it sees the keys before position nk - back[q] and its partials lie rowoff[q] rows after the item's first
-    constexpr int kLanesPerRow = 32 / GP;              // after RowReduce, row r sits in lanes r * kLanesPerRow ..
+    constexpr int kLanesPerRow = 32 / GH;              // after RowReduce, row r sits in lanes r * kLanesPerRow ..
     const int pub_row = lane / kLanesPerRow;
     const bool publisher = (lane % kLanesPerRow) == 0;
-    int back[GP];
-    size_t rowoff[GP];
+    int back[GH];
+    size_t rowoff[GH];
 #pragma unroll
-    for (int q = 0; q < GP; ++q) {
-      const int tok = (kMulti && q < R) ? q / G : 0;
+    for (int q = 0; q < GH; ++q) {
+      const int qa = rb + q;                       // row number in the item
+      const int tok = (kMulti && qa < R) ? qa / G : 0;
       back[q] = p.Sq - 1 - tok;
-      rowoff[q] = kMulti ? ((size_t)tok * p.Hq + (size_t)(q - tok * G)) * p.num_splits : (size_t)q * p.num_splits;
+      rowoff[q] = kMulti ? ((size_t)tok * p.Hq + (size_t)(qa - tok * G)) * p.num_splits : (size_t)qa * p.num_splits;
     }
     int g = 0, ne = 0, rg = 0;                     // global tile counter, non-empty item ordinal, retained tiles so far
     uint32_t xc = 0;                               // exchanges so far (buffer xc & 1, barrier phase xc & 1)
@@ -402,23 +414,23 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     bool pend = false;
     int pend_ip = 0, pend_ne = 0;
     size_t pend_prow0 = 0;
-    float pend_l[GP];
+    float pend_l[GH];
 #pragma unroll
-    for (int q = 0; q < GP; ++q) pend_l[q] = 1.f;
+    for (int q = 0; q < GH; ++q) pend_l[q] = 1.f;
     auto flush = [&]() -> bool {
       bool k = mbar_wait(&item_done[pend_ip], (uint32_t)((pend_ne >> 1) & 1), status);
       k = __all_sync(0xffffffffu, k);
       if (!k) return false;
       tc_fence_after();
-      uint32_t o[16];
-      tmem_ld_x16(tmem_addr(tb, lane_base, DecCfg::kColO + (uint32_t)pend_ip * 16u), o);
+      uint32_t o[LDN];
+      tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, DecCfg::kColO + (uint32_t)pend_ip * 16u + (uint32_t)rb), o);
       tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&o_free[pend_ip]);   // the accumulator may take the item after next
 #pragma unroll
-      for (int q = 0; q < GP; ++q)
-        if (q < R)   // (a row that saw no key of the split: (0, -inf))
+      for (int q = 0; q < GH; ++q)
+        if (rb + q < R)   // (a row that saw no key of the split: (0, -inf))
           p.o_part[(pend_prow0 + rowoff[q]) * 128 + kt] =
               (!kMulti || pend_l[q] > 0.f) ? __uint_as_float(o[q]) / pend_l[q] : 0.f;
       pend = false;
@@ -428,10 +440,10 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       int b, hkv, split, T, j0, nk;
       geometry(item, b, hkv, split, T, j0, nk);
       // L of a row = the keys it sees: all nk of the sequence for the newest token, one less per token before it
-      int lim[GP];
-      float theta[GP];
+      int lim[GH];
+      float theta[GH];
 #pragma unroll
-      for (int q = 0; q < GP; ++q) {
+      for (int q = 0; q < GH; ++q) {
         lim[q] = kMulti ? nk - back[q] : nk;
         theta[q] = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(lim[q], 1)));
       }
@@ -439,8 +451,8 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       const size_t stat_row = (size_t)(b * p.Hkv + hkv) * p.num_splits + split;
       if (T == 0) {   // empty split: (0, -inf)
 #pragma unroll
-        for (int q = 0; q < GP; ++q)
-          if (q < R) {
+        for (int q = 0; q < GH; ++q)
+          if (rb + q < R) {
             p.o_part[(prow0 + rowoff[q]) * 128 + kt] = 0.f;
             if (kt == q) p.lse_part[prow0 + rowoff[q]] = -INFINITY;
           }
@@ -449,10 +461,10 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       }
       const int ip = ne & 1;
       const uint32_t colO = DecCfg::kColO + (uint32_t)ip * 16u;
-      float m_ref[GP], l[GP], lgl[GP];
+      float m_ref[GH], l[GH], lgl[GH];
       float psum = 0.f;   // this warp's sum of P of the last retained tile, for the row this lane publishes
 #pragma unroll
-      for (int q = 0; q < GP; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; lgl[q] = -INFINITY; }
+      for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; lgl[q] = -INFINITY; }
       int r = 0;
       bool pending_sum = false;
       uint32_t bm_bits = 0;
@@ -460,25 +472,25 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       uint32_t* bm_row = p.bitmask ? p.bitmask + stat_row * p.words : nullptr;
       // publishes this warp's (maximum, sum) of row pub_row -- each row by the first lane that holds it after the
       // warp reduction --, waits for the group, returns the combined maxima in tmax and adds the combined sums to l
-      auto exchange = [&](float mx_row, float (&tmax)[GP]) -> bool {
+      auto exchange = [&](float mx_row, float (&tmax)[GH]) -> bool {
         const int xb = xc & 1;
-        if (publisher) { xch_max[xb][w][pub_row] = mx_row; xch_sum[xb][w][pub_row] = psum; }
+        if (publisher) { xch_max[xb][grp][w][pub_row] = mx_row; xch_sum[xb][grp][w][pub_row] = psum; }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&grp_a);
-        bool k = mbar_wait(&grp_a, xc & 1, status);
+        if (lane == 0) mbar_arrive(&grp_a[grp]);
+        bool k = mbar_wait(&grp_a[grp], xc & 1, status);
         k = __all_sync(0xffffffffu, k);
         ++xc;
         if (!k) return false;
-        float a0[GP], a1[GP], a2[GP], a3[GP];
-        lds_row<GP>(xch_max[xb][0], a0); lds_row<GP>(xch_max[xb][1], a1);
-        lds_row<GP>(xch_max[xb][2], a2); lds_row<GP>(xch_max[xb][3], a3);
+        float a0[GH], a1[GH], a2[GH], a3[GH];
+        lds_row<GH>(xch_max[xb][grp][0], a0); lds_row<GH>(xch_max[xb][grp][1], a1);
+        lds_row<GH>(xch_max[xb][grp][2], a2); lds_row<GH>(xch_max[xb][grp][3], a3);
 #pragma unroll
-        for (int q = 0; q < GP; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
+        for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
         if (pending_sum) {
-          lds_row<GP>(xch_sum[xb][0], a0); lds_row<GP>(xch_sum[xb][1], a1);
-          lds_row<GP>(xch_sum[xb][2], a2); lds_row<GP>(xch_sum[xb][3], a3);
+          lds_row<GH>(xch_sum[xb][grp][0], a0); lds_row<GH>(xch_sum[xb][grp][1], a1);
+          lds_row<GH>(xch_sum[xb][grp][2], a2); lds_row<GH>(xch_sum[xb][grp][3], a3);
 #pragma unroll
-          for (int q = 0; q < GP; ++q) {
+          for (int q = 0; q < GH; ++q) {
             l[q] += (a0[q] + a1[q]) + (a2[q] + a3[q]);
             lgl[q] = __log2f(l[q]);
           }
@@ -493,17 +505,17 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        uint32_t sr[16];
-        tmem_ld_x16(tmem_addr(tb, lane_base, (uint32_t)sb * 16u), sr);
+        uint32_t sr[LDN];
+        tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, (uint32_t)sb * 16u + (uint32_t)rb), sr);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_free[sb]);     // the scores are in registers
         const int kpos = (j0 - t) * 128 + kt;   // only the newest tile of the sequence has keys that a row does not see
-        float x[GP], mx[GP], tmax[GP];
+        float x[GH], mx[GH], tmax[GH];
 #pragma unroll
-        for (int q = 0; q < GP; ++q) { x[q] = (kpos < lim[q] && q < R) ? __uint_as_float(sr[q]) * c2 : -INFINITY; mx[q] = x[q]; }
-        RowReduce<GP, 16, true>::run(mx, lane);   // mx[0]: the warp's maximum of row pub_row
+        for (int q = 0; q < GH; ++q) { x[q] = (kpos < lim[q] && rb + q < R) ? __uint_as_float(sr[q]) * c2 : -INFINITY; mx[q] = x[q]; }
+        RowReduce<GH, 16, true>::run(mx, lane);   // mx[0]: the warp's maximum of row pub_row
         ok = exchange(mx[0], tmax);
         if (!ok) break;
         // Eq. 3 against the split's partial normalizer: skip iff rowmax - (m + log l) < log(tau / Nk) for every head
@@ -511,13 +523,20 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         if (!kDense && r > 0) {
           retain = false;
 #pragma unroll
-          for (int q = 0; q < GP; ++q)   // (a row without a visible key in the tile does not constrain it)
-            retain = retain || (q < R && (!kMulti || tmax[q] > -INFINITY) &&
+          for (int q = 0; q < GH; ++q)   // (a row without a visible key in the tile does not constrain it)
+            retain = retain || (rb + q < R && (!kMulti || tmax[q] > -INFINITY) &&
                                 !(((tmax[q] - (m_ref[q] + lgl[q])) - theta[q]) < 0.f));
         }
-        if (!kDense && head) {
-          *(volatile int*)&flag[g & 3] = retain ? 1 : 0;
+        if (!kDense && ghead) {
+          *(volatile int*)&flag[grp][g & 3] = retain ? 1 : 0;
           mbar_arrive(&vote_bar[g & 3]);
+        }
+        if (!kDense && NG > 1) {   // the tile is retained if a row of either group needs it
+          ok = mbar_wait(&vote_bar[g & 3], (uint32_t)((g >> 2) & 1), status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          retain = (*(volatile int*)&flag[0][g & 3] | *(volatile int*)&flag[1][g & 3]) != 0;
+          retain = __all_sync(0xffffffffu, retain);
         }
         if (!retain) continue;
         if (head && bm_row) {
@@ -531,14 +550,14 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         }
         if (r == 0) {
 #pragma unroll
-          for (int q = 0; q < GP; ++q) m_ref[q] = kMulti ? fmaxf(tmax[q], -1e30f) : tmax[q];   // (finite also for a row that sees no key yet)
+          for (int q = 0; q < GH; ++q) m_ref[q] = kMulti ? fmaxf(tmax[q], -1e30f) : tmax[q];   // (finite also for a row that sees no key yet)
         } else {
-          float alpha[GP];
+          float alpha[GH];
           bool resc = false;
 #pragma unroll
-          for (int q = 0; q < GP; ++q) {
+          for (int q = 0; q < GH; ++q) {
             alpha[q] = 1.f;
-            if (q < R && tmax[q] > m_ref[q] + kRescaleGap) {   // lazy rescaling: the reference only moves when it has to
+            if (rb + q < R && tmax[q] > m_ref[q] + kRescaleGap) {   // lazy rescaling: the reference only moves when it has to
               alpha[q] = fast_exp2(m_ref[q] - tmax[q]);
               l[q] *= alpha[q];
               lgl[q] = __log2f(l[q]);
@@ -553,12 +572,12 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            uint32_t o[16];
-            tmem_ld_x16(tmem_addr(tb, lane_base, colO), o);
+            uint32_t o[LDN];
+            tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colO + (uint32_t)rb), o);
             tmem_wait_ld();
 #pragma unroll
-            for (int q = 0; q < GP; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
-            tmem_st_x16(tmem_addr(tb, lane_base, colO), o);
+            for (int q = 0; q < GH; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
+            tmem_st_cols<LDN>(tmem_addr(tb, lane_base, colO + (uint32_t)rb), o);
             tmem_wait_st();
             tc_fence_before();
           }
@@ -574,16 +593,16 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           uint8_t* dst = sP + ps * DecCfg::kPBytes + (kt >> 6) * 2048;
           const uint32_t col = (uint32_t)(kt & 63);
 #pragma unroll
-          for (int q = 0; q < GP; ++q) {
-            x[q] = (q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
-            *reinterpret_cast<__nv_bfloat16*>(dst + sw128_offset((uint32_t)q, col)) = __float2bfloat16_rn(x[q]);
+          for (int q = 0; q < GH; ++q) {
+            x[q] = (rb + q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
+            *reinterpret_cast<__nv_bfloat16*>(dst + sw128_offset((uint32_t)(rb + q), col)) = __float2bfloat16_rn(x[q]);
           }
         }
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[ps]);
         // this warp's per-row sums of the tile (fp32, before the bf16 cast); they travel with the next exchange
-        RowReduce<GP, 16, false>::run(x, lane);
+        RowReduce<GH, 16, false>::run(x, lane);
         psum = x[0];
         pending_sum = true;
         ++r;
@@ -591,7 +610,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       }
       if (!ok) break;
       if (pending_sum) {   // the sums of the last retained tile
-        float dummy[GP];
+        float dummy[GH];
         ok = exchange(-INFINITY, dummy);
         if (!ok) break;
       }
@@ -602,10 +621,10 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       pend_ne = ne;
       pend_prow0 = prow0;
 #pragma unroll
-      for (int q = 0; q < GP; ++q) pend_l[q] = l[q];
+      for (int q = 0; q < GH; ++q) pend_l[q] = l[q];
 #pragma unroll
-      for (int q = 0; q < GP; ++q)
-        if (q < R && kt == q)
+      for (int q = 0; q < GH; ++q)
+        if (rb + q < R && kt == q)
           p.lse_part[prow0 + rowoff[q]] = (!kMulti || l[q] > 0.f) ? (m_ref[q] + lgl[q]) * 0.6931471805599453f : -INFINITY;
       if (head) {
         if (bm_row && bm_word >= 0) bm_row[bm_word] = bm_bits;
