@@ -61,6 +61,9 @@ static double dot(const double* a, const double* b, int d) {
   return s;
 }
 
+int mala_oracle_decode_merge(const double* o_part, const double* lse_part, int num_splits, int R, int d,
+                             double* o, double* lse);
+
 /* Visible-key count L_q (Section 2.1): the number of keys the query may attend to.  Causal: the queries are
  * the LAST N_q of N_k positions (off = N_k - N_q >= 0), query row q sits at position q + off and sees the keys
  * 0 .. q + off, so L_q = q + 1 + off (q + 1 for equal lengths, N_k for the single decode query); otherwise N_k. */
@@ -131,16 +134,81 @@ int mala_oracle_dense_bwd(const double* Q, const double* K, const double* V, con
 }
 
 /* ------------------------------------------------------------------------------------------
- * Algorithm 1 (forward) for the listed query blocks of one head (blocks == NULL: all).
+ * Algorithm 1 (forward): the key blocks j_hi, j_hi - 1, ..., j_lo of query block i, in that order, on the
+ * running state m, l, acc (rows of the block).  S, mt: scratch.  mask, crit: [Tr*Tc] or NULL.
+ * ---------------------------------------------------------------------------------------- */
+static void fwd_block_range(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale,
+                            double tau, int Bq, int Bk, int causal, int i, int j_lo, int j_hi, int Tc, double* m,
+                            double* l, double* acc, double* S, double* mt, uint8_t* mask, double* crit) {
+  const int off = Nk - N; /* N queries (the last N positions) against Nk keys */
+  const int q0 = i * Bq, rows = (q0 + Bq <= N ? Bq : N - q0);
+  for (int j = j_hi; j >= j_lo; --j) { /* descending from the diagonal toward earlier keys */
+    const int k0 = j * Bk, cols = (k0 + Bk <= Nk ? Bk : Nk - k0);
+    /* a tile with no legal key for any row is not visited */
+    if (causal && k0 > q0 + rows - 1 + off) {
+      if (mask) mask[(size_t)i * Tc + j] = MASK_ILLEGAL;
+      if (crit) crit[(size_t)i * Tc + j] = NAN;
+      continue;
+    }
+    /* S_ij = Q_i K_j^T with the causal mask (-inf) */
+    double C = -INFINITY;
+    for (int r = 0; r < rows; ++r) {
+      const int q = q0 + r;
+      double mrow = -INFINITY;
+      int legal = 0;
+      for (int c = 0; c < cols; ++c) {
+        const int k = k0 + c;
+        double s = -INFINITY;
+        if (!causal || k <= q + off) { s = scale * dot(Q + (size_t)q * d, K + (size_t)k * d, d); legal = 1; }
+        S[(size_t)r * Bk + c] = s;
+        if (s > mrow) mrow = s;
+      }
+      mt[r] = mrow; /* rowmax(S_ij) */
+      /* row criterion: rowmax - m - log l - log(tau/L), state BEFORE this tile (Eq. 3) */
+      double cq;
+      if (!legal) cq = -INFINITY;             /* does not constrain retention */
+      else if (l[r] == 0.0) cq = INFINITY;    /* nothing retained yet: log-ratio is +inf */
+      else cq = mrow - (m[r] + log(l[r])) - log_threshold(tau, visible_count(q, Nk, causal, off));
+      if (cq > C) C = cq;
+    }
+    const int retain = !(C < 0.0); /* skip only if every relevant row is strictly below */
+    if (mask) mask[(size_t)i * Tc + j] = retain ? MASK_RETAINED : MASK_SKIPPED;
+    if (crit) crit[(size_t)i * Tc + j] = C;
+    if (!retain) continue; /* m, l, O unchanged */
+    /* online-softmax update of every row of the block (Alg. 1, retained branch) */
+    for (int r = 0; r < rows; ++r) {
+      const double mnew = (m[r] > mt[r] ? m[r] : mt[r]);
+      if (mnew == -INFINITY) continue; /* still empty: stays (-inf, 0, 0) */
+      const double alpha = (m[r] == -INFINITY ? 0.0 : exp(m[r] - mnew));
+      double lt = 0.0;
+      for (int c = 0; c < d; ++c) acc[(size_t)r * d + c] *= alpha;
+      for (int c = 0; c < cols; ++c) {
+        const double s = S[(size_t)r * Bk + c];
+        if (s == -INFINITY) continue;
+        const double p = exp(s - mnew);
+        lt += p;
+        const double* v = V + (size_t)(k0 + c) * d;
+        for (int e = 0; e < d; ++e) acc[(size_t)r * d + e] += p * v[e];
+      }
+      l[r] = alpha * l[r] + lt;
+      m[r] = mnew;
+    }
+  }
+}
+
+/* Algorithm 1 for the listed query blocks of one head (blocks == NULL: all).
  * O [N,d], lse [N]: rows of the listed blocks are written.  mask, crit: [Tr*Tc], rows of the
  * listed blocks are written (may be NULL).
- * ---------------------------------------------------------------------------------------- */
-int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale, double tau,
-                    int Bq, int Bk, int causal, int n_blocks, const int* blocks, double* O, double* lse,
-                    uint8_t* mask, double* crit) {
-  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
-  const int off = Nk - N; /* N queries (the last N positions) against Nk keys */
+ * num_splits > 1: the key blocks are cut into num_splits contiguous ranges of ceil(Tc / num_splits) blocks; every
+ * range runs the rule on its own running state (its test sees the range's PARTIAL normalizer, as in "Fused decoding
+ * execution") and the ranges' results (o_s, lse_s) are merged by lse = log sum_s exp(lse_s),
+ * o = sum_s exp(lse_s - lse) o_s.  A range that holds no legal key of a row contributes nothing to it. */
+int mala_oracle_fwd_split(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale,
+                          double tau, int Bq, int Bk, int causal, int num_splits, int n_blocks, const int* blocks,
+                          double* O, double* lse, uint8_t* mask, double* crit) {
+  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || num_splits <= 0 || !(tau >= 0.0)) return -1;
   const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
+  const int tps = (Tc + num_splits - 1) / num_splits;
   const int nb = blocks ? n_blocks : Tr;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < nb; ++u) {
@@ -149,70 +217,40 @@ int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, in
     /* Alg. 1: O_i = 0, l_i = 0, m_i = -inf; L_i from positions */
     double* m = (double*)malloc(sizeof(double) * rows);
     double* l = (double*)malloc(sizeof(double) * rows);
-    double* acc = (double*)calloc((size_t)rows * d, sizeof(double));
+    double* acc = (double*)malloc(sizeof(double) * (size_t)rows * d);
     double* S = (double*)malloc(sizeof(double) * (size_t)rows * Bk);
     double* mt = (double*)malloc(sizeof(double) * rows);
-    for (int r = 0; r < rows; ++r) { m[r] = -INFINITY; l[r] = 0.0; }
-    for (int j = Tc - 1; j >= 0; --j) { /* descending from the diagonal toward earlier keys */
-      const int k0 = j * Bk, cols = (k0 + Bk <= Nk ? Bk : Nk - k0);
-      /* a tile with no legal key for any row is not visited */
-      if (causal && k0 > q0 + rows - 1 + off) {
-        if (mask) mask[(size_t)i * Tc + j] = MASK_ILLEGAL;
-        if (crit) crit[(size_t)i * Tc + j] = NAN;
-        continue;
-      }
-      /* S_ij = Q_i K_j^T with the causal mask (-inf) */
-      double C = -INFINITY;
+    double* o_s = (double*)malloc(sizeof(double) * (size_t)num_splits * rows * d);
+    double* lse_s = (double*)malloc(sizeof(double) * (size_t)num_splits * rows);
+    for (int s = 0; s < num_splits; ++s) {
+      for (int r = 0; r < rows; ++r) { m[r] = -INFINITY; l[r] = 0.0; }
+      memset(acc, 0, sizeof(double) * (size_t)rows * d);
+      const int j_lo = s * tps, j_hi = ((s + 1) * tps < Tc ? (s + 1) * tps : Tc) - 1;
+      fwd_block_range(Q, K, V, N, Nk, d, scale, tau, Bq, Bk, causal, i, j_lo, j_hi, Tc, m, l, acc, S, mt, mask, crit);
+      /* O_i <- diag(l)^-1 O_i,  l_i <- m_i + log l_i */
       for (int r = 0; r < rows; ++r) {
-        const int q = q0 + r;
-        double mrow = -INFINITY;
-        int legal = 0;
-        for (int c = 0; c < cols; ++c) {
-          const int k = k0 + c;
-          double s = -INFINITY;
-          if (!causal || k <= q + off) { s = scale * dot(Q + (size_t)q * d, K + (size_t)k * d, d); legal = 1; }
-          S[(size_t)r * Bk + c] = s;
-          if (s > mrow) mrow = s;
-        }
-        mt[r] = mrow; /* rowmax(S_ij) */
-        /* row criterion: rowmax - m - log l - log(tau/L), state BEFORE this tile (Eq. 3) */
-        double cq;
-        if (!legal) cq = -INFINITY;             /* does not constrain retention */
-        else if (l[r] == 0.0) cq = INFINITY;    /* nothing retained yet: log-ratio is +inf */
-        else cq = mrow - (m[r] + log(l[r])) - log_threshold(tau, visible_count(q, Nk, causal, off));
-        if (cq > C) C = cq;
-      }
-      const int retain = !(C < 0.0); /* skip only if every relevant row is strictly below */
-      if (mask) mask[(size_t)i * Tc + j] = retain ? MASK_RETAINED : MASK_SKIPPED;
-      if (crit) crit[(size_t)i * Tc + j] = C;
-      if (!retain) continue; /* m, l, O unchanged */
-      /* online-softmax update of every row of the block (Alg. 1, retained branch) */
-      for (int r = 0; r < rows; ++r) {
-        const double mnew = (m[r] > mt[r] ? m[r] : mt[r]);
-        if (mnew == -INFINITY) continue; /* still empty: stays (-inf, 0, 0) */
-        const double alpha = (m[r] == -INFINITY ? 0.0 : exp(m[r] - mnew));
-        double lt = 0.0;
-        for (int c = 0; c < d; ++c) acc[(size_t)r * d + c] *= alpha;
-        for (int c = 0; c < cols; ++c) {
-          const double s = S[(size_t)r * Bk + c];
-          if (s == -INFINITY) continue;
-          const double p = exp(s - mnew);
-          lt += p;
-          const double* v = V + (size_t)(k0 + c) * d;
-          for (int e = 0; e < d; ++e) acc[(size_t)r * d + e] += p * v[e];
-        }
-        l[r] = alpha * l[r] + lt;
-        m[r] = mnew;
+        lse_s[(size_t)s * rows + r] = (l[r] == 0.0 ? -INFINITY : m[r] + log(l[r]));
+        for (int c = 0; c < d; ++c)
+          o_s[((size_t)s * rows + r) * d + c] = (l[r] == 0.0 ? 0.0 : acc[(size_t)r * d + c] / l[r]);
       }
     }
-    /* O_i <- diag(l)^-1 O_i,  l_i <- m_i + log l_i */
-    for (int r = 0; r < rows; ++r) {
-      for (int c = 0; c < d; ++c) O[(size_t)(q0 + r) * d + c] = acc[(size_t)r * d + c] / l[r];
-      lse[q0 + r] = m[r] + log(l[r]);
+    if (num_splits == 1) {
+      for (int r = 0; r < rows; ++r) {
+        for (int c = 0; c < d; ++c) O[(size_t)(q0 + r) * d + c] = acc[(size_t)r * d + c] / l[r];
+        lse[q0 + r] = m[r] + log(l[r]);
+      }
+    } else {
+      mala_oracle_decode_merge(o_s, lse_s, num_splits, rows, d, O + (size_t)q0 * d, lse + q0);
     }
-    free(m); free(l); free(acc); free(S); free(mt);
+    free(m); free(l); free(acc); free(S); free(mt); free(o_s); free(lse_s);
   }
   return 0;
+}
+
+int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale, double tau,
+                    int Bq, int Bk, int causal, int n_blocks, const int* blocks, double* O, double* lse,
+                    uint8_t* mask, double* crit) {
+  return mala_oracle_fwd_split(Q, K, V, N, Nk, d, scale, tau, Bq, Bk, causal, 1, n_blocks, blocks, O, lse, mask, crit);
 }
 
 /* D = rowsum(O o dO) (Alg. 2, the term subtracted from dP). */

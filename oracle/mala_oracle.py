@@ -50,6 +50,8 @@ def lib():
         L.mala_oracle_dense_fwd.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _ci, _ci, _ci, _D, _D]
         L.mala_oracle_dense_bwd.argtypes = [_D, _D, _D, _D, _ci, _ci, _cd, _ci, _D, _D, _D]
         L.mala_oracle_fwd.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D, _D, _U8, _D]
+        L.mala_oracle_fwd_split.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _ci, _I, _D, _D, _U8,
+                                            _D]
         L.mala_oracle_bwd_D.argtypes = [_D, _D, _ci, _ci, _D]
         L.mala_oracle_bwd.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I,
                                       _D, _D, _D, _U8, _D]
@@ -60,7 +62,8 @@ def lib():
         L.mala_oracle_decode_splits_rows.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _I, _D, _D,
                                                      _U8, _D]
         L.mala_oracle_decode_merge.argtypes = [_D, _D, _ci, _ci, _ci, _D, _D]
-        for f in ("mala_oracle_dense_fwd", "mala_oracle_dense_bwd", "mala_oracle_fwd", "mala_oracle_bwd_D",
+        for f in ("mala_oracle_dense_fwd", "mala_oracle_dense_bwd", "mala_oracle_fwd", "mala_oracle_fwd_split",
+                  "mala_oracle_bwd_D",
                   "mala_oracle_bwd", "mala_oracle_bwd_dq", "mala_oracle_decode_tiles_per_split",
                   "mala_oracle_decode_splits", "mala_oracle_decode_splits_tps", "mala_oracle_decode_splits_rows",
                   "mala_oracle_decode_merge"):
@@ -140,8 +143,10 @@ def dense_bwd(q, k, v, do, scale: float, causal: bool = True):
     return dq, dk, dv
 
 
-def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True, units=None):
+def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True, units=None, num_splits: int = 1):
     """Algorithm 1.  ``units``: optional list of (b, h_q, i) query blocks; rows of other blocks stay NaN.
+    ``num_splits`` > 1: the key blocks are cut into that many contiguous ranges of ceil(Tc / num_splits) blocks,
+    each range runs the rule on its own state and the results are merged by their log-normalizers.
 
     q [B,N,Hq,d]; k, v [B,Nk,Hkv,d] with Nk >= N: the queries are the last N of the Nk positions (chunked
     prefill), query row q sees the keys 0 .. q + Nk - N and L_q = q + 1 + Nk - N.
@@ -170,8 +175,8 @@ def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True
         m = np.zeros((Tr, Tc), dtype=np.uint8)
         c = np.full((Tr, Tc), np.nan)
         bl = np.asarray(blocks, dtype=np.int32) if blocks is not None else None
-        _ck(lib().mala_oracle_fwd(_p(Q), _p(K), _p(V), N, Nk, d, scale, tau, Bq, Bk, int(causal),
-                                  0 if bl is None else len(bl), _ip(bl), _p(O), _p(l), _u8(m), _p(c)), "fwd")
+        _ck(lib().mala_oracle_fwd_split(_p(Q), _p(K), _p(V), N, Nk, d, scale, tau, Bq, Bk, int(causal), num_splits,
+                                        0 if bl is None else len(bl), _ip(bl), _p(O), _p(l), _u8(m), _p(c)), "fwd")
         o[b, :, h, :] = O
         lse[b, h] = l
         mask[b, h] = m

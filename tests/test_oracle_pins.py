@@ -726,3 +726,70 @@ def test_decode_multi_one_split_is_the_forward_rule_on_a_chunk_of_the_new_tokens
     assert np.array_equal(f["mask"][0, 0, 0], dec["mask"][0, 0, 0])
     assert np.allclose(f["o"][0, :, 0], dec["o"][0, :, 0], atol=1e-13)
     assert np.allclose(f["lse"][0, 0], dec["lse"][0, :, 0], atol=1e-13)
+
+
+# ------------------------------------------------------------------ forward with the key range cut into splits
+@pytest.mark.parametrize("S", [2, 3, 5])
+@pytest.mark.parametrize("Nq,Nk", [(64, 64), (24, 72), (13, 50)])
+def test_fwd_splits_tau_zero_is_dense_for_any_split_count(Nq, Nk, S):
+    d, scale = 8, 0.4
+    q, k, v = peaky_inputs(Nk, d, 281)
+    qc = q[:, Nk - Nq:]
+    f = orc.fwd(qc, k, v, scale, 0.0, 8, 8, num_splits=S)
+    od, ld = orc.dense_fwd(qc, k, v, scale)
+    assert np.allclose(f["o"], od, atol=1e-12) and np.allclose(f["lse"], ld, atol=1e-12)
+    assert not (f["mask"] == orc.SKIPPED).any()
+
+
+def test_fwd_splits_of_one_query_are_the_decode_rule():
+    # one query against 96 keys, 3 ranges of 4 key blocks: exactly split-KV decode of one row
+    Nk, d, scale, tau, Bk, S = 96, 8, 0.5, 0.5, 8, 3
+    q, kc, vc = _decode_inputs(Nk, d, 1, 291)
+    dec = orc.decode(q, kc, vc, scale, tau, S, Bk, packed_rows=False)
+    f = orc.fwd(q.reshape(1, 1, 1, d), kc, vc, scale, tau, 4, Bk, num_splits=S)
+    assert (dec["mask"] == orc.SKIPPED).sum() > 0
+    assert np.array_equal(f["mask"][0, 0, 0], dec["mask"][0, 0].reshape(-1))
+    assert np.allclose(f["o"][0, 0, 0], dec["o"][0, 0], atol=1e-13)
+    assert abs(f["lse"][0, 0, 0] - dec["lse"][0, 0]) < 1e-13
+
+
+@pytest.mark.parametrize("Nq,Nk,S,tau", [(32, 96, 3, 0.1), (21, 69, 2, 0.5), (64, 64, 4, 1e-2)])
+def test_fwd_splits_match_bruteforce_key_sets_per_range(Nq, Nk, S, tau):
+    d, scale, B_ = 32, 1.0 / math.sqrt(32), 8
+    off = Nk - Nq
+    q, k, v = peaky_inputs(Nk, d, 301 + Nk, boost=5.0)
+    qc = q[:, off:]
+    f = orc.fwd(qc, k, v, scale, tau, B_, B_, num_splits=S)
+    Sm = scale * (qc[0, :, 0] @ k[0, :, 0].T)
+    Tc = -(-Nk // B_)
+    tps = -(-Tc // S)
+    assert (f["mask"] == orc.SKIPPED).sum() > 0
+    for i in range(-(-Nq // B_)):
+        rows = list(range(i * B_, min(Nq, (i + 1) * B_)))
+        Z = {r: [] for r in rows}                     # per row: the ranges' normalizers
+        num = {r: np.zeros(d) for r in rows}
+        for s in range(S):
+            R = {r: [] for r in rows}
+            for j in reversed(range(s * tps, min(Tc, (s + 1) * tps))):
+                keys = list(range(j * B_, min(Nk, (j + 1) * B_)))
+                if keys[0] > rows[-1] + off:
+                    assert f["mask"][0, 0, i, j] == 0
+                    continue
+                skip = True
+                for r in rows:
+                    legal = [x for x in keys if x <= r + off]
+                    if not legal:
+                        continue
+                    Zt = sum(math.exp(Sm[r, x]) for x in R[r])
+                    if Zt == 0.0 or not (math.exp(max(Sm[r, x] for x in legal)) / Zt < tau / (r + 1 + off)):
+                        skip = False
+                assert f["mask"][0, 0, i, j] == (1 if skip else 2)
+                if not skip:
+                    for r in rows:
+                        R[r] += [x for x in keys if x <= r + off]
+            for r in rows:                            # merging by the log-normalizers = pooling the retained keys
+                Z[r].append(sum(math.exp(Sm[r, x]) for x in R[r]))
+                num[r] += sum((math.exp(Sm[r, x]) * v[0, x, 0] for x in R[r]), np.zeros(d))
+        for r in rows:
+            assert abs(f["lse"][0, 0, r] - math.log(sum(Z[r]))) < 1e-12
+            assert np.allclose(f["o"][0, r, 0], num[r] / sum(Z[r]), atol=1e-12)
