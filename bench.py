@@ -209,6 +209,36 @@ def chunk_leg(cs, Nq, tau, it, peaks):
     return row
 
 
+def chunk_split_leg(cs, Nq, tau, it):
+    """A short chunk of queries against a long context: mala_fwd_chunk (one CTA per pair of query blocks) against
+    mala_fwd_chunk_split (the keys cut into ranges that run on different SMs), MALA and dense, with the retained
+    fraction of each (the split-local test is the more conservative one)."""
+    import torch
+    mala, cc = cs.mala, cs.cfg
+    q = cs.q[:, cc.N - Nq:]
+    o, lse = torch.empty_like(q), torch.empty((cc.B, cc.Hq, Nq), dtype=torch.float32, device=q.device)
+    row = {}
+    for S in (1, 8, 16, 32):
+        ws = torch.empty(max(256, mala.workspace_bytes(mala.OP_FWD, cc.B, cc.Hq, cc.Hkv, Nq, cc.d, S)), dtype=torch.uint8,
+                         device=q.device)
+        r = {}
+        for label, t_ in (("mala", tau), ("dense", 0.0)):
+            if S == 1:
+                fn = lambda: mala.fwd_chunk(q, cs.k, cs.v, cs.scale, t_, out=o, lse=lse)
+            else:
+                fn = lambda: mala.fwd_chunk_split(q, cs.k, cs.v, cs.scale, t_, S, out=o, lse=lse, ws=ws)
+            r[label + "_ms"] = time_cuda(fn, 3, it)
+        if S == 1:
+            _, _, st = mala.fwd_chunk(q, cs.k, cs.v, cs.scale, tau, out=o, lse=lse, stats=True)
+        else:
+            _, _, st = mala.fwd_chunk_split(q, cs.k, cs.v, cs.scale, tau, S, out=o, lse=lse, ws=ws, stats=True)
+        ret, leg = st.totals.cpu().tolist()
+        r["retained_frac"] = ret / leg
+        row[f"splits={S}"] = r
+        del ws
+    return row
+
+
 def varlen_leg(cfg, preset, lens, tau, it, peaks, dev):
     """mala_fwd_varlen / mala_bwd_varlen on packed sequences with the heads of a prefill configuration: latency of
     the MALA and dense kernels and the tensor-pipe fraction on the tile FLOPs executed."""
@@ -511,6 +541,8 @@ def main():
                                                       / (row["mala"]["bwd_ms"] * 1e-3) / 1e12 / peaks["tflops_sustained"])
                 row["speedup_fwd"] = row["dense"]["fwd_ms"] / row["mala"]["fwd_ms"]
                 row["speedup_bwd"] = row["dense"]["bwd_ms"] / row["mala"]["bwd_ms"]
+                if name == "cfg4":                  # a 1024-query chunk against the 128K context, unsplit and split
+                    row["chunk_last_1024"] = chunk_split_leg(cs, 1024, tau, it)
                 if name == "cfg3":                  # chunked prefill: the last 8192 queries against all 32768 keys
                     row["chunk_last_8192"] = chunk_leg(cs, 8192, tau, it, peaks)
                 if name == "cfg3":                  # the same heads on packed sequences of 16K + 8K + 5000 + 3192 rows

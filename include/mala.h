@@ -103,6 +103,18 @@ int mala_bwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout
                    mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int Nq, int Nk, int d,
                    int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* mala_fwd_chunk with the keys cut into num_splits ranges that run on different SMs: for a short chunk of queries
+ * against a long context (where mala_fwd_chunk has fewer query blocks than the GPU has SMs).  The key blocks
+ * 0 .. ceil(Nk/128)-1 are cut into num_splits contiguous ranges of ceil(ceil(Nk/128)/num_splits) blocks; every range
+ * runs Algorithm 1 on its blocks with its own running state, i.e. its skip test sees the range's PARTIAL normalizer
+ * (the split-local rule of "Fused decoding execution"; more conservative than the unsplit test), and the ranges are
+ * merged by lse = log sum_s exp(lse_s), o = sum_s exp(lse_s - lse) o_s.  num_splits = 1 is mala_fwd_chunk; tau = 0
+ * gives FullAttn for any num_splits.  Telemetry as for mala_fwd_chunk.  ws: device scratch of
+ * mala_workspace_bytes(MALA_OP_FWD, B, Hq, Hkv, Nq, d, num_splits) bytes, 256-byte aligned.  B * num_splits <= 65535. */
+int mala_fwd_chunk_split(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B,
+                         int Hq, int Hkv, int Nq, int Nk, int d, int causal, float scale, float tau, int num_splits,
+                         void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Algorithms 1 and 2 on B packed sequences of different lengths (self attention, equal query and key lengths per
  * sequence).  q, o, dout, dq are [1,total,Hq,d] tensors, k, v, dk, dv [1,total,Hkv,d] (sb is ignored); sequence b
  * holds the rows cu_seqlens[b] .. cu_seqlens[b+1]-1; cu_seqlens: device int32 [B+1], non-decreasing, cu_seqlens[0] = 0,

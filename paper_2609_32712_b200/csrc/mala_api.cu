@@ -110,7 +110,7 @@ static const float kLog2e = 1.4426950408889634f;
 template <int D, bool kDense>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                       cudaStream_t stream) {
-  dim3 grid((p.Tr + 1) / 2, p.Hq, p.B);
+  dim3 grid((p.Tr + 1) / 2, p.Hq, p.B * (p.num_splits > 1 ? p.num_splits : 1));
   mala_fwd_kernel<D, kDense><<<grid, FwdCfg<D, kDense>::kThreads, FwdCfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
@@ -149,7 +149,7 @@ int mala_tile_shape(int op, int d, int* Bq, int* Bk) {
 
 size_t mala_workspace_bytes(int op, int B, int Hq, int Hkv, int N, int d, int num_splits) {
   if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || (d != 64 && d != 128)) return 0;
-  if (op == MALA_OP_FWD) return 256;
+  if (op == MALA_OP_FWD) return num_splits > 1 ? fwd_split_workspace_bytes(B, Hq, N, d, num_splits) : 256;
   if (op == MALA_OP_BWD) return bwd_workspace_bytes(B, Hq, N, d);
   if (op == MALA_OP_DECODE) return num_splits > 0 ? decode_workspace_bytes(B, Hq, d, num_splits) : 0;
   return 0;
@@ -183,7 +183,16 @@ static int check_lengths(int N, int Nk, int causal) {
 // cu != null: B packed sequences in [1, total, H, d] tensors, N = Nk = the longest one.
 static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
                     int Hkv, int N, int Nk, int d, int causal, float scale, float tau, void* cuda_stream,
-                    const int32_t* cu = nullptr, int total = 0) {
+                    const int32_t* cu = nullptr, int total = 0, int num_splits = 1, void* ws = nullptr,
+                    size_t ws_bytes = 0) {
+  if (num_splits < 1) return MALA_ERR_INVALID_ARG;
+  if (num_splits > 1) {
+    if (cu || num_splits > 65535 || (long long)B * num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+    if (!ws) return MALA_ERR_INVALID_ARG;
+    if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
+    if (B > 0 && Hq > 0 && N > 0 && (d == 64 || d == 128) && ws_bytes < fwd_split_workspace_bytes(B, Hq, N, d, num_splits))
+      return MALA_ERR_WORKSPACE_TOO_SMALL;
+  }
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
   MALA_TRY(check_lengths(N, Nk, causal));
   if (!lse) return MALA_ERR_INVALID_ARG;
@@ -206,6 +215,12 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
 
   FwdParams p;
   p.cu = cu; p.total = total;
+  p.num_splits = num_splits;
+  p.tps = ((Nk + 127) / 128 + num_splits - 1) / num_splits;
+  p.o_part = num_splits > 1 ? (float*)ws : nullptr;
+  p.lse_part = num_splits > 1
+                   ? (float*)((uint8_t*)ws + (((size_t)B * Hq * num_splits * N * d * sizeof(float) + 255) & ~(size_t)255))
+                   : nullptr;
   p.o = (__nv_bfloat16*)o.p; p.o_sb = o.sb; p.o_sn = o.sn; p.o_sh = o.sh;
   p.lse = lse;
   p.retained = st ? st->retained_per_block : nullptr;
@@ -220,9 +235,22 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
     if (cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * p.Tr * p.words * sizeof(uint32_t), stream) != cudaSuccess)
       return MALA_ERR_CUDA;
   }
+  if (num_splits > 1 && p.retained &&   // (the ranges add to it)
+      cudaMemsetAsync(p.retained, 0, (size_t)B * Hq * p.Tr * sizeof(uint32_t), stream) != cudaSuccess)
+    return MALA_ERR_CUDA;
   const bool dense = (tau == 0.f);
-  if (d == 128) return dense ? launch_fwd<128, true>(tq, tk, tv, p, stream) : launch_fwd<128, false>(tq, tk, tv, p, stream);
-  return dense ? launch_fwd<64, true>(tq, tk, tv, p, stream) : launch_fwd<64, false>(tq, tk, tv, p, stream);
+  int rc;
+  if (d == 128) rc = dense ? launch_fwd<128, true>(tq, tk, tv, p, stream) : launch_fwd<128, false>(tq, tk, tv, p, stream);
+  else rc = dense ? launch_fwd<64, true>(tq, tk, tv, p, stream) : launch_fwd<64, false>(tq, tk, tv, p, stream);
+  if (rc != MALA_OK || num_splits == 1) return rc;
+  const unsigned rows = (unsigned)((long long)B * Hq * N);
+  if (d == 128)
+    fwd_merge_splits_kernel<128><<<rows, 128, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
+                                                           num_splits, p.tps, p.Tk, p.koff, p.causal);
+  else
+    fwd_merge_splits_kernel<64><<<rows, 64, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
+                                                         num_splits, p.tps, p.Tk, p.koff, p.causal);
+  return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
 int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
@@ -264,6 +292,13 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
   MALA_TRY(device_setup(dev, &status));
   return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B0, Hq, Hkv, N0, Nk0, d, causal ? 1 : 0, scale, tau, ws,
                     status, (cudaStream_t)cuda_stream, cu, total);
+}
+
+int mala_fwd_chunk_split(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B,
+                         int Hq, int Hkv, int Nq, int Nk, int d, int causal, float scale, float tau, int num_splits,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, cuda_stream, nullptr, 0, num_splits,
+                  ws, ws_bytes);
 }
 
 int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,

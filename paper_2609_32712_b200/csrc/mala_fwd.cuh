@@ -37,6 +37,12 @@ struct FwdParams {
   // above describe the longest sequence (grid, telemetry strides)
   const int* cu;
   int total;
+  // Key range cut into num_splits ranges of tps key blocks (num_splits > 1): grid z = b * num_splits + split; a CTA
+  // runs its blocks on the key blocks of its range only and writes the normalised fp32 result and the
+  // log-normalizer of the range; a merge kernel combines the ranges.
+  int num_splits, tps;
+  float* o_part;                 // [B, Hq, num_splits, N, D]
+  float* lse_part;               // [B, Hq, num_splits, N] natural log
   float scale_log2;              // scale * log2(e)
   float log2_tau;                // log2(tau); unused by the dense kernel
 };
@@ -72,7 +78,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.Hq / p.Hkv;
-  const int b = blockIdx.z, h = blockIdx.y, hkv = h / G;
+  const int sp = p.num_splits > 1 ? (int)blockIdx.z % p.num_splits : 0;
+  const int b = p.num_splits > 1 ? (int)blockIdx.z / p.num_splits : (int)blockIdx.z;
+  const int h = blockIdx.y, hkv = h / G;
   // this sequence: first row in the tensors, rows, blocks (packed sequences: equal query and key lengths)
   const int row0 = p.cu ? __ldg(p.cu + b) : 0;
   const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
@@ -83,12 +91,24 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int npairs = (Tr + 1) / 2;
   if ((int)blockIdx.x >= npairs) return;             // (a sequence shorter than the longest one)
   const int c = npairs - 1 - (int)blockIdx.x;        // longest pairs first
-  const int iA = 2 * c, iB = 2 * c + 1;
-  const bool hasB = iB < Tr;
+  int iA = 2 * c, iB = 2 * c + 1;
+  bool hasB = iB < Tr;
+  int dA = p.causal ? iA + p.koff : Tk - 1;          // newest key block with a legal key, per block
+  const int dB = p.causal ? iB + p.koff : Tk - 1;
+  int jlo = 0, jhi = Tk - 1;                         // key blocks of this CTA
+  if (p.num_splits > 1) {
+    jlo = sp * p.tps;
+    jhi = min(Tk, jlo + p.tps) - 1;
+    if (jlo > dA) {                                  // the range holds no legal key of block A
+      if (!hasB || jlo > dB) return;                 // ... nor of block B: nothing to do (the merge knows)
+      iA = iB; dA = dB; hasB = false;                // only B's diagonal block: run B alone
+    }
+  }
   // key steps u = 0 .. U-1 visit key block j0 - u; block X takes part from step first[X] on
-  const int j0 = p.causal ? (hasB ? iB : iA) + p.koff : (Tk - 1);
-  const int U = j0 + 1;
-  const int firstA = (p.causal && hasB) ? 1 : 0;     // B's diagonal key block is not legal for A
+  const int hA = min(dA, jhi), hB = min(dB, jhi);    // first key block each block visits
+  const int j0 = hasB ? hB : hA;
+  const int U = j0 - jlo + 1;
+  const int firstA = hasB ? hB - hA : 0;             // 1 when B's diagonal key block, not legal for A, is in the range
   int* status = p.status;
 
   if (tid == 0) {
@@ -274,6 +294,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t colS = (uint32_t)x * 128u, colO = 256u + (uint32_t)x * 128u;
     const int first = (x == 0) ? firstA : 0;
     const int T = present_x ? (U - first) : 0;       // tiles of this block
+    const bool mask_first = x ? (hB == dB) : (hA == dA);
     float m_ref = -INFINITY, l = 0.f;
     int r = 0;
     bool ok = true;
@@ -295,8 +316,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tmem_ld_x32(tmem_addr(tb, lane_base, colS + 64), s2);
       tmem_ld_x32(tmem_addr(tb, lane_base, colS + 96), s3);
       tmem_wait_ld();
-      if (t == 0) {
-        // first visited tile: causal diagonal and / or the ragged end of the key range
+      if (t == 0 && mask_first) {
+        // first visited tile, when it is the block's newest legal one: causal diagonal and / or the ragged end of
+        // the keys
         const int lim = p.causal ? rl : (Nkeys - 1 - j * 128);
         const uint32_t ninf = 0xff800000u;
 #pragma unroll
@@ -361,7 +383,10 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       if (stat_thread && bm_row) {
         if ((j >> 5) != bm_word) {
-          if (bm_word >= 0) bm_row[bm_word] = bm_bits;
+          if (bm_word >= 0) {
+            if (p.num_splits > 1) atomicOr(&bm_row[bm_word], bm_bits);   // (ranges share words of the row)
+            else bm_row[bm_word] = bm_bits;
+          }
           bm_word = j >> 5;
           bm_bits = 0;
         }
@@ -448,7 +473,34 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       ok = mbar_wait(&fin_bar, 0, status);
       ok = __all_sync(0xffffffffu, ok);
     }
-    if (ok && present_x) {
+    if (ok && present_x && p.num_splits > 1) {
+      // one range of the keys: normalised fp32 partial and the range's log-normalizer
+      tc_fence_after();
+      const float inv = 1.f / l;
+      const size_t prow = (((size_t)b * p.Hq + h) * p.num_splits + sp) * p.N + row;
+#pragma unroll
+      for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t o[32];
+        tmem_ld_x32(tmem_addr(tb, lane_base, colO + cc * 32), o);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            *reinterpret_cast<float4*>(p.o_part + prow * D + cc * 32 + v * 4) =
+                make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
+                            __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
+        }
+      }
+      if (valid) p.lse_part[prow] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      if (stat_thread) {   // several ranges add to the same telemetry rows
+        if (bm_row && bm_word >= 0) atomicOr(&bm_row[bm_word], bm_bits);
+        if (p.retained) atomicAdd(&p.retained[stat_row], (uint32_t)r);
+        if (p.totals) {
+          atomicAdd(&p.totals[0], (unsigned long long)r);
+          atomicAdd(&p.totals[1], (unsigned long long)T);
+        }
+      }
+    } else if (ok && present_x) {
       tc_fence_after();
       const float inv = 1.f / l;
       __nv_bfloat16* orow = p.o + (int64_t)bz * p.o_sb + (int64_t)(row0 + row) * p.o_sn + (int64_t)h * p.o_sh;
@@ -486,6 +538,36 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tb, Cfg::kTmemCols);
+}
+
+// Merge of the key ranges of the split forward: lse = log sum_s exp(lse_s), o = sum_s exp(lse_s - lse) o_s over the
+// ranges that hold a legal key of the row's block (range s does iff s * tps <= the block's newest legal key block).
+// One block of D threads per (b, head, row).
+template <int D>
+__global__ void __launch_bounds__(D)
+fwd_merge_splits_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part,
+                        __nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sn, int64_t o_sh,
+                        float* __restrict__ lse, int Hq, int N, int num_splits, int tps, int Tk, int koff, int causal) {
+  const long long idx = blockIdx.x;
+  const int row = (int)(idx % N), h = (int)((idx / N) % Hq), b = (int)(idx / ((long long)N * Hq)), c = threadIdx.x;
+  const int newest = causal ? row / 128 + koff : Tk - 1;
+  const int ns = min(num_splits, newest / tps + 1);
+  const size_t base = ((size_t)b * Hq + h) * num_splits;
+  float mx = -INFINITY;
+  for (int s = 0; s < ns; ++s) mx = fmaxf(mx, lse_part[(base + s) * N + row]);
+  float Z = 0.f, acc = 0.f;
+  for (int s = 0; s < ns; ++s) {
+    const float w = exp2f((lse_part[(base + s) * N + row] - mx) * 1.4426950408889634f);
+    Z += w;
+    acc += w * o_part[((base + s) * N + row) * D + c];
+  }
+  o[b * o_sb + (int64_t)row * o_sn + h * o_sh + c] = __float2bfloat16(acc / Z);
+  if (c == 0) lse[((size_t)b * Hq + h) * N + row] = mx + logf(Z);
+}
+
+inline size_t fwd_split_workspace_bytes(int B, int Hq, int N, int d, int S) {
+  auto align256 = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  return align256((size_t)B * Hq * S * N * d * sizeof(float)) + align256((size_t)B * Hq * S * N * sizeof(float));
 }
 
 }  // namespace mala

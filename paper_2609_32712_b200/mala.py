@@ -55,6 +55,9 @@ def lib():
                                      i, i, i, i, i, i, i, f, f, vp, sz, vp]
         L.mala_fwd_chunk.restype = i
         L.mala_bwd_chunk.restype = i
+        L.mala_fwd_chunk_split.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, f, f,
+                                           i, vp, sz, vp]
+        L.mala_fwd_chunk_split.restype = i
         L.mala_fwd_varlen.argtypes = [_TIn, _TIn, _TIn, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, f, f,
                                       vp, sz, vp]
         L.mala_bwd_varlen.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, vp, _TOut, _TOut, _TOut, ctypes.POINTER(_Stats),
@@ -183,6 +186,24 @@ def fwd_chunk(q, k, v, scale: float, tau: float, causal: bool = True, stats: boo
                               None, 0, _stream())
     if rc != 0:
         raise MalaError(rc, "mala_fwd_chunk")
+    return o, lse, st
+
+
+def fwd_chunk_split(q, k, v, scale: float, tau: float, num_splits: int, causal: bool = True, stats: bool = False,
+                    out=None, lse=None, ws=None):
+    """mala_fwd_chunk_split: mala_fwd_chunk with the keys cut into num_splits ranges (split-local test, merged)."""
+    B, Nq, Hq, d = q.shape
+    Nk, Hkv = k.shape[1], k.shape[2]
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq, Nq), dtype=torch.float32, device=q.device) if lse is None else lse
+    Tq, Tk = -(-Nq // 128), -(-Nk // 128)
+    st = Stats((B, Hq, Tq), -(-Tk // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_FWD, B, Hq, Hkv, Nq, d, num_splits), q.device) if ws is None else ws
+    rc = lib().mala_fwd_chunk_split(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TOut), lse.data_ptr(),
+                                    ctypes.byref(st.c) if st else None, B, Hq, Hkv, Nq, Nk, d, int(causal), scale, tau,
+                                    num_splits, ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_fwd_chunk_split")
     return o, lse, st
 
 

@@ -122,3 +122,63 @@ def test_chunk_rejects_a_chunk_that_starts_inside_a_tile(mala):
     with pytest.raises(mala.MalaError) as e:
         mala.fwd_chunk(q, kv, kv, 0.1, 0.0)
     assert e.value.code < 0
+
+
+def _run_split(mala, oracle, c, tau, S, causal=True):
+    q, k, v = (c[x].cuda() for x in ("q", "k", "v"))
+    B, Nq, Hq, d = q.shape
+    Nk = k.shape[1]
+    Tq, Tk = -(-Nq // 128), -(-Nk // 128)
+    off = Nk - Nq if causal else 0
+    o, lse, st = mala.fwd_chunk_split(q, k, v, c["scale"], tau, S, causal=causal, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    ref = oracle.fwd(c["q"], c["k"], c["v"], c["scale"], tau, 128, 128, causal=causal, num_splits=S)
+    fm = st.mask(Tk).cpu().numpy()
+    tps = -(-Tk // S)
+    o_c, lse_c = o.float().cpu().numpy(), lse.cpu().numpy()
+    for b in range(B):
+        for h in range(Hq):
+            for i in range(Tq):
+                newest = i + off // 128 if causal else Tk - 1
+                for s in range(S):   # every range is its own run of the rule: its own visiting order and band
+                    js = [j for j in range(min(newest, (s + 1) * tps - 1), s * tps - 1, -1)]
+                    sel = np.zeros(Tk, dtype=bool)
+                    sel[js] = True
+                    parity.check_mask(np.where(sel, fm[b, h, i], False), np.where(sel, ref["mask"][b, h, i], 0),
+                                      ref["crit"][b, h, i], js, tau, i * 128 + 1 + off if causal else Nk)
+                assert int(st.retained[b, h, i]) == int(fm[b, h, i].sum())
+    parity.check_output(o_c, ref["o"])
+    assert np.abs(lse_c - ref["lse"]).max() <= parity.LSE_ABS
+    assert st.totals.cpu().numpy()[1] == int((ref["mask"] > 0).sum())
+    return int((ref["mask"] == 1).sum())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,Nq,d,Hq,Hkv,S", [(1024, 128, 128, 2, 1, 4), (1152, 256, 128, 4, 2, 3), (1000, 232, 128, 2, 2, 8),
+                                              (768, 384, 64, 2, 1, 2), (640, 640, 128, 2, 1, 5), (512, 128, 128, 2, 1, 9)])
+def test_chunk_split_literal(mala, oracle, Nk, Nq, d, Hq, Hkv, S, tau):
+    """Key ranges on different CTAs; (640, 5): equal lengths, ranges of one key block, so that a range can hold only
+    the diagonal block of the second query block of a pair; (512, 9): more ranges than key blocks."""
+    w = W.custom_prefill(2, Hq, Hkv, Nk, d, seed=Nk + Nq + S)
+    _run_split(mala, oracle, _chunk(w, Nq), tau, S)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("Nk,Nq,S", [(4096, 256, 8), (2560, 512, 5)])
+def test_chunk_split_skipping_regime(mala, oracle, Nk, Nq, S, tau):
+    w = W.custom_prefill(1, 4, 2, Nk, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=7, preset="R")
+    assert _run_split(mala, oracle, _chunk(w, Nq), tau, S) > 0, "workload must exercise skipping"
+
+
+def test_chunk_split_non_causal(mala, oracle):
+    w = W.custom_prefill(1, 2, 1, 1100, 128, head_types=["peaked", "diffuse"], seed=5, preset="R")
+    _run_split(mala, oracle, _chunk(w, 200), 1e-2, 3, causal=False)
+
+
+def test_chunk_split_of_one_range_equals_the_unsplit_call(mala):
+    w = W.custom_prefill(1, 4, 2, 1536, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=3, preset="R")
+    q, k, v = (w[x].cuda() for x in ("q", "k", "v"))
+    o1, l1, _ = mala.fwd_chunk(q[:, 1024:], k, v, w["scale"], 1e-4)
+    o2, l2, _ = mala.fwd_chunk_split(q[:, 1024:], k, v, w["scale"], 1e-4, 1)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
