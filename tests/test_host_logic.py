@@ -89,6 +89,12 @@ def test_argument_validation_codes_of_the_general_shape_calls(mala):
     bc = lambda Nq, Nk: L.mala_bwd_chunk(tin(), tin(), tin(), tin(), tin(), base, tout(), tout(), tout(), None, 1, 2, 2,
                                          Nq, Nk, 128, 1, 0.1, 1e-4, base, 1 << 20, None)
     assert bc(100, 300) == -2 and bc(128, 0) == -1
+    # key ranges: a positive count, scratch that is large enough and aligned
+    fs = lambda S, ws=base, n=1 << 20: L.mala_fwd_chunk_split(tin(), tin(), tin(), tout(), base, None, 1, 2, 2, 128, 512, 128,
+                                                              1, 0.1, 1e-4, S, ws, n, None)
+    assert fs(0) == -1 and fs(4, ws=None) == -1 and fs(4, ws=base + 16) == -3 and fs(4, n=64) == -4
+    assert mala.workspace_bytes(mala.OP_FWD, 1, 2, 2, 128, 128, 4) == 2 * 4 * 128 * 128 * 4 + 2 * 4 * 128 * 4
+    assert mala.workspace_bytes(mala.OP_FWD, 1, 2, 2, 128, 128) == 256
     # packed sequences: cu_seqlens required, longest sequence within the total
     fv = lambda cu, total, mx: L.mala_fwd_varlen(tin(), tin(), tin(), cu, tout(), base, None, 2, 2, 2, total, mx, 128, 1,
                                                  0.1, 1e-4, None, 0, None)
