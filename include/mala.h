@@ -155,23 +155,27 @@ int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o,
                       size_t ws_bytes, void* cuda_stream);
 
 /* Split-KV decode over a paged cache with one length per sequence (the serving-side layout of "Fused decoding
- * execution"; the rule itself is the one of mala_decode with L = seqlens[b] for the rows of sequence b).
+ * execution"; the rule itself is the one of mala_decode / mala_decode_multi with seqlens[b] in the place of Nk).
+ * q, o [B,Sq,Hq,d], Sq >= 1 new tokens per sequence whose keys are the last Sq of the sequence's seqlens[b] keys
+ * (Sq * Hq/Hkv <= 16; Sq = 1: sn of q and o is ignored); lse_opt fp32 [B,Sq,Hq] or NULL.
  * kpages, vpages [num_pages, page_size, Hkv, d] (sb = page stride, sn = key stride, sh = head stride);
  * page_size must be a multiple of 128 (MALA_ERR_UNSUPPORTED otherwise).  block_table: device int32
  * [B, max_pages_per_seq]; keys page_size*x .. page_size*(x+1)-1 of sequence b live in page block_table[b][x]
  * (entries beyond the sequence's length are never read; an entry outside [0, num_pages) reads zeros).
  * seqlens: device int32 [B], keys held by each sequence, clamped to [0, max_pages_per_seq*page_size], or NULL
- * if every sequence holds max_pages_per_seq*page_size keys; a sequence without keys gets o = 0, lse = -inf.
+ * if every sequence holds max_pages_per_seq*page_size keys; a token that sees no key (a sequence without keys, or
+ * with fewer keys than new tokens) gets o = 0, lse = -inf.
  * The key positions 0 .. max_pages_per_seq*page_size-1 are cut into num_splits chunks as in mala_decode with
  * Nk = max_pages_per_seq*page_size; splits beyond a sequence's length are empty.  Telemetry shapes as for
  * mala_decode with that Nk.  The values stored in a mapped page beyond the sequence's length must be finite
  * bf16 numbers (a zero-initialised or recycled page is): they never reach the result, but the tile that holds
- * the newest key is multiplied as a whole.  Workspace: mala_workspace_bytes(MALA_OP_DECODE, B, Hq, Hkv,
- * max_pages_per_seq*page_size, d, num_splits).  The library reads block_table and seqlens on the device, on cuda_stream, and keeps neither. */
+ * the newest key is multiplied as a whole.  Workspace: mala_workspace_bytes(MALA_OP_DECODE, B * Sq, Hq, Hkv,
+ * max_pages_per_seq*page_size, d, num_splits).  The library reads block_table and seqlens on the device, on
+ * cuda_stream, and keeps neither. */
 int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* block_table,
                       const int32_t* seqlens, mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq,
-                      int Hkv, int num_pages, int page_size, int max_pages_per_seq, int d, float scale, float tau,
-                      int num_splits, void* ws, size_t ws_bytes, void* cuda_stream);
+                      int Hkv, int num_pages, int page_size, int max_pages_per_seq, int Sq, int d, float scale,
+                      float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Decode for callers that cannot allocate device memory.  (The paper has no counterpart: this entry point
  * exists for integration reasons only and computes exactly what mala_decode computes.)

@@ -317,29 +317,32 @@ def decode_paged(q, kpages, vpages, block_table, seqlens, scale: float, tau: flo
                  units=None):
     """Split-KV decode over a paged cache with one length per sequence.
 
-    q [B,Hq,d] (or [B,1,Hq,d]); kpages, vpages [num_pages, page_size, Hkv, d]; block_table [B, max_pages]
-    (page of the keys page_size*x ..); seqlens [B] (None: every sequence holds max_pages*page_size keys).
-    The cache of sequence b is put together page by page and cut off at its length; the decode rule then runs
-    on it with L = seqlens[b].  All sequences share one layout of splits over the key positions, the one
-    ``decode`` derives for N_k = max_pages*page_size.  ``units``: optional list of (b, h_kv), other entries stay
-    zero.  Returns what ``decode`` returns (packed rows).
+    q [B,Hq,d] or [B,Sq,Hq,d] (Sq new tokens per sequence, whose keys are the last Sq of the sequence's keys);
+    kpages, vpages [num_pages, page_size, Hkv, d]; block_table [B, max_pages] (page of the keys page_size*x ..);
+    seqlens [B] (None: every sequence holds max_pages*page_size keys).
+    The cache of sequence b is put together page by page and cut off at its length n; the decode rule then runs on
+    it: token s sees the keys before position n - Sq + s + 1, which is also its L.  All sequences share one layout of
+    splits over the key positions, the one ``decode`` derives for N_k = max_pages*page_size.  ``units``: optional
+    list of (b, h_kv), other entries stay zero.
+    Returns dict(o [B,Sq,Hq,d] ([B,Hq,d] for a 3-d q), lse, mask [B,Hkv,S,tps], crit, lse_part [B,Sq,Hq,S] / [B,Hq,S]).
     """
-    if len(q.shape) == 4:
-        q = q[:, 0]
-    B, Hq, d = q.shape
+    squeeze = len(q.shape) == 3
+    if squeeze:
+        q = q[:, None]
+    B, Sq, Hq, d = q.shape
     page_size, Hkv = kpages.shape[1], kpages.shape[2]
     G = Hq // Hkv
+    R = Sq * G
     bt = np.asarray(block_table, dtype=np.int64)
     max_pages = bt.shape[1]
     Nmax = max_pages * page_size
     lens = np.full((B,), Nmax, dtype=np.int64) if seqlens is None else np.asarray(seqlens, dtype=np.int64)
     tps = int(lib().mala_oracle_decode_tiles_per_split(Nmax, num_splits, Bk))
-    o = np.zeros((B, Hq, d))
-    lse = np.zeros((B, Hq))
+    o = np.zeros((B, Sq, Hq, d))
+    lse = np.zeros((B, Sq, Hq))
     mask = np.zeros((B, Hkv, num_splits, tps), dtype=np.uint8)
     crit = np.full((B, Hkv, num_splits, tps), np.nan)
-    o_part = np.zeros((B, Hq, num_splits, d))
-    lse_part = np.zeros((B, Hq, num_splits))
+    lse_part = np.zeros((B, Sq, Hq, num_splits))
     if units is None:
         units = [(b, g) for b in range(B) for g in range(Hkv)]
     for (b, g) in units:
@@ -350,23 +353,25 @@ def decode_paged(q, kpages, vpages, block_table, seqlens, scale: float, tau: flo
         V = np.concatenate([_np(vpages[int(bt[b, x]), :, g, :]) for x in range(npg)], axis=0)[:n] \
             if npg else np.zeros((1, d))
         K, V = np.ascontiguousarray(K), np.ascontiguousarray(V)
-        Q = _np(q[b, g * G:(g + 1) * G, :])
-        op = np.zeros((num_splits, G, d))
-        lp = np.zeros((num_splits, G))
+        Q = np.ascontiguousarray(_np(q[b, :, g * G:(g + 1) * G, :]).reshape(R, d))
+        vis = np.ascontiguousarray(np.repeat(n - Sq + 1 + np.arange(Sq), G).astype(np.int32))
+        op = np.zeros((num_splits, R, d))
+        lp = np.zeros((num_splits, R))
         m = np.zeros((num_splits, tps), dtype=np.uint8)
         c = np.full((num_splits, tps), np.nan)
-        _ck(lib().mala_oracle_decode_splits_tps(_p(Q), _p(K), _p(V), G, n, d, scale, tau, num_splits, tps, Bk,
-                                                _p(op), _p(lp), _u8(m), _p(c)), "decode_splits_tps")
-        oo = np.zeros((G, d))
-        ll = np.zeros((G,))
-        _ck(lib().mala_oracle_decode_merge(_p(op), _p(lp), num_splits, G, d, _p(oo), _p(ll)), "decode_merge")
-        o[b, g * G:(g + 1) * G] = oo
-        lse[b, g * G:(g + 1) * G] = ll
-        o_part[b, g * G:(g + 1) * G] = op.transpose(1, 0, 2)
-        lse_part[b, g * G:(g + 1) * G] = lp.T
+        _ck(lib().mala_oracle_decode_splits_rows(_p(Q), _p(K), _p(V), R, n, d, scale, tau, num_splits, tps, Bk,
+                                                 _ip(vis), _p(op), _p(lp), _u8(m), _p(c)), "decode_splits_rows")
+        oo = np.zeros((R, d))
+        ll = np.zeros((R,))
+        _ck(lib().mala_oracle_decode_merge(_p(op), _p(lp), num_splits, R, d, _p(oo), _p(ll)), "decode_merge")
+        o[b, :, g * G:(g + 1) * G] = oo.reshape(Sq, G, d)
+        lse[b, :, g * G:(g + 1) * G] = ll.reshape(Sq, G)
+        lse_part[b, :, g * G:(g + 1) * G] = lp.T.reshape(Sq, G, num_splits)
         mask[b, g] = m
         crit[b, g] = c
-    return dict(o=o, lse=lse, mask=mask, crit=crit, o_part=o_part, lse_part=lse_part)
+    if squeeze:
+        o, lse, lse_part = o[:, 0], lse[:, 0], lse_part[:, 0]
+    return dict(o=o, lse=lse, mask=mask, crit=crit, lse_part=lse_part)
 
 
 def decode_multi(q, kcache, vcache, scale: float, tau: float, num_splits: int, Bk: int, units=None):

@@ -382,21 +382,21 @@ int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o,
 
 int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* block_table,
                       const int32_t* seqlens, mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq,
-                      int Hkv, int num_pages, int page_size, int max_pages_per_seq, int d, float scale, float tau,
-                      int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
-  if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
+                      int Hkv, int num_pages, int page_size, int max_pages_per_seq, int Sq, int d, float scale,
+                      float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || Sq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
   if (page_size % 128 != 0 || (long long)max_pages_per_seq * page_size > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
   const int Nk = max_pages_per_seq * page_size;   // the longest cache a sequence can hold
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
   if (num_splits <= 0 || !ws) return MALA_ERR_INVALID_ARG;
-  if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  if ((Hq / Hkv) * Sq > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
   if ((((uintptr_t)block_table) & 3) != 0 || (((uintptr_t)seqlens) & 3) != 0) return MALA_ERR_MISALIGNED;
-  MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
+  MALA_TRY(check_view(q.p, q.sb, Sq > 1 ? q.sn : 8, q.sh, B, Sq, Hq));
   MALA_TRY(check_view(kpages.p, kpages.sb, kpages.sn, kpages.sh, num_pages, page_size, Hkv));
   MALA_TRY(check_view(vpages.p, vpages.sb, vpages.sn, vpages.sh, num_pages, page_size, Hkv));
-  MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
+  MALA_TRY(check_view(o.p, o.sb, Sq > 1 ? o.sn : 8, o.sh, B, Sq, Hq));
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-  if (ws_bytes < decode_workspace_bytes(B, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < decode_workspace_bytes(B * Sq, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
@@ -405,7 +405,7 @@ int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_
   pg.block_table = block_table; pg.seqlens = seqlens; pg.bt_stride = max_pages_per_seq; pg.page_size = page_size;
   pg.num_pages = num_pages;
   return decode_launch(q, kpages, vpages, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
-                       (cudaStream_t)cuda_stream, &pg);
+                       (cudaStream_t)cuda_stream, &pg, Sq);
 }
 
 int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, int B, int Hq,

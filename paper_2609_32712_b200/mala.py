@@ -68,7 +68,7 @@ def lib():
         L.mala_decode_multi.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, f, f, i,
                                         vp, sz, vp]
         L.mala_decode_multi.restype = i
-        L.mala_decode_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i,
+        L.mala_decode_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, i,
                                         f, f, i, vp, sz, vp]
         L.mala_decode_paged.restype = i
         L.mala_decode_static.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, i, i, i, i, i, f, f, i, vp]
@@ -304,24 +304,24 @@ def decode_multi(q, kcache, vcache, scale: float, tau: float, num_splits: int, s
 
 def decode_paged(q, kpages, vpages, block_table, seqlens, scale: float, tau: float, num_splits: int,
                  stats: bool = False, ws=None, out=None, want_lse: bool = True):
-    """mala_decode_paged: q [B,1,Hq,d]; kpages, vpages [num_pages, page_size, Hkv, d]; block_table int32
-    [B, max_pages_per_seq]; seqlens int32 [B] or None.  Returns (o, lse or None, Stats or None)."""
-    B, one, Hq, d = q.shape
-    assert one == 1
+    """mala_decode_paged: q [B,Sq,Hq,d] (Sq new tokens per sequence); kpages, vpages [num_pages, page_size, Hkv, d];
+    block_table int32 [B, max_pages_per_seq]; seqlens int32 [B] or None.
+    Returns (o [B,Sq,Hq,d], lse [B,Hq] (Sq = 1) or [B,Sq,Hq] or None, Stats or None)."""
+    B, Sq, Hq, d = q.shape
     num_pages, page_size, Hkv = kpages.shape[0], kpages.shape[1], kpages.shape[2]
     assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.shape[0] == B
     assert seqlens is None or (seqlens.dtype == torch.int32 and seqlens.is_contiguous() and seqlens.shape == (B,))
     max_pages = block_table.shape[1]
     Nk = max_pages * page_size
     o = torch.empty_like(q) if out is None else out
-    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    lse = torch.empty((B, Hq) if Sq == 1 else (B, Sq, Hq), dtype=torch.float32, device=q.device) if want_lse else None
     tps = -(-(-(-Nk // num_splits)) // 128)
     st = Stats((B, Hkv, num_splits), -(-tps // 32), q.device) if stats else None
-    ws = _ws(workspace_bytes(OP_DECODE, B, Hq, Hkv, Nk, d, num_splits), q.device) if ws is None else ws
+    ws = _ws(workspace_bytes(OP_DECODE, B * Sq, Hq, Hkv, Nk, d, num_splits), q.device) if ws is None else ws
     rc = lib().mala_decode_paged(_view(q, _TIn), _view(kpages, _TIn), _view(vpages, _TIn), block_table.data_ptr(),
                                  seqlens.data_ptr() if seqlens is not None else None, _view(o, _TOut),
                                  lse.data_ptr() if lse is not None else None, ctypes.byref(st.c) if st else None,
-                                 B, Hq, Hkv, num_pages, page_size, max_pages, d, scale, tau, num_splits,
+                                 B, Hq, Hkv, num_pages, page_size, max_pages, Sq, d, scale, tau, num_splits,
                                  ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_decode_paged")

@@ -102,8 +102,8 @@ def _run_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0):
     torch.cuda.synchronize()
     assert mala.device_status() == 0
     _, Bk = mala.tile_shape(mala.OP_DECODE, d)
-    ref = oracle.decode_paged(w["q"], kp, vp, bt.numpy(), lens.numpy() if seqlens is not None else None, w["scale"],
-                              tau, num_splits, Bk)
+    ref = oracle.decode_paged(w["q"][:, 0], kp, vp, bt.numpy(), lens.numpy() if seqlens is not None else None,
+                              w["scale"], tau, num_splits, Bk)
     tps = ref["mask"].shape[-1]
     gm = st.mask(tps).cpu().numpy()
     o_c, lse_c = o.float().cpu().numpy()[:, 0], lse.cpu().numpy()
@@ -222,3 +222,35 @@ def test_decode_multi_of_one_token_equals_decode(mala):
         o1, l1, _ = mala.decode(q, kc, vc, w["scale"], tau, 8)
         o2, l2, _ = mala.decode_multi(q, kc, vc, w["scale"], tau, 8)
         assert torch.equal(o1, o2) and torch.equal(l1, l2.reshape(l1.shape))
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv,page,Sq,lens", [
+    (2048, 4, 8, 2, 256, 4, [2048, 1000, 129, 3]),     # 16 rows; the last sequence holds fewer keys than new tokens
+    (1536, 3, 4, 2, 128, 3, [1536, 1, 700]),
+])
+def test_decode_paged_with_several_new_tokens(mala, oracle, Nk, S, Hq, Hkv, page, Sq, lens, tau):
+    B = len(lens)
+    w = W.custom_decode(B, Hq, Hkv, Nk, 128, S, group_types=["diffuse", "peaked"], seed=Nk + Sq, preset="D")
+    kp, vp, bt, sl = W.paginate(w["kcache"], w["vcache"], page, seqlens=lens, seed=Sq)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(77)
+    q = w["q"].float().repeat(1, Sq, 1, 1)
+    q[..., :127] += 0.5 * torch.randn((B, Sq, Hq, 127), generator=gen)
+    q = q.to(torch.bfloat16)
+    o, lse, st = mala.decode_paged(q.cuda(), kp.cuda(), vp.cuda(), bt.cuda(), sl.cuda(), w["scale"], tau, S, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    ref = oracle.decode_paged(q, kp, vp, bt.numpy(), lens, w["scale"], tau, S, 128)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    for b in range(B):
+        for g in range(Hkv):
+            for s in range(S):
+                parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                                  tau, max(lens[b] - Sq + 1, 1), 128)
+    o_c, lse_c = o.float().cpu().numpy(), lse.cpu().numpy()
+    parity.check_output(o_c, ref["o"])
+    fin = np.isfinite(ref["lse"])
+    assert np.abs(lse_c[fin] - ref["lse"][fin]).max() <= parity.LSE_ABS
+    assert np.isneginf(lse_c[~fin]).all() and (o_c[~fin] == 0).all()

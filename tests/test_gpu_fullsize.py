@@ -147,7 +147,8 @@ def test_cfg5_decode_128k_paged_variable_lengths(mala, oracle, tau):
     assert mala.device_status() == 0
     assert torch.isfinite(o.float()).all()
     units = [(0, 0), (1, 3), (2, 5), (4, 2), (7, 7)]
-    ref = oracle.decode_paged(w["q"], kp, vp, bt.cpu().numpy(), lens, w["scale"], tau, cfg.num_splits, 128, units=units)
+    ref = oracle.decode_paged(w["q"][:, 0], kp, vp, bt.cpu().numpy(), lens, w["scale"], tau, cfg.num_splits, 128,
+                              units=units)
     tps = ref["mask"].shape[-1]
     gm = st.mask(tps).cpu().numpy()
     G = cfg.Hq // cfg.Hkv

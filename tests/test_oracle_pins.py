@@ -793,3 +793,27 @@ def test_fwd_splits_match_bruteforce_key_sets_per_range(Nq, Nk, S, tau):
         for r in rows:
             assert abs(f["lse"][0, 0, r] - math.log(sum(Z[r]))) < 1e-12
             assert np.allclose(f["o"][0, r, 0], num[r] / sum(Z[r]), atol=1e-12)
+
+
+def test_decode_paged_with_several_new_tokens_per_sequence():
+    # per sequence: the contiguous multi-token rule on its own n keys (same 32-key chunks); a sequence with fewer keys
+    # than new tokens leaves its oldest tokens without any key: (0, -inf)
+    lens = [128, 96, 64, 2]
+    Sq, G, d = 3, 2, 8
+    q1, kc, vc, kp, vp, bt = _paged_inputs(4, 128, d, G, 16, lens, 311)
+    r = _rng(313)
+    q = np.repeat(q1[:, None], Sq, axis=1) + 0.3 * r.standard_normal((4, Sq, G, d))
+    q[..., d - 1] = 6.0
+    dec = orc.decode_paged(q, kp, vp, bt, lens, 0.5, 0.5, 4, 8)
+    assert (dec["mask"] == orc.SKIPPED).sum() > 0
+    for b, n in enumerate(lens[:3]):
+        S = -(-n // 32)
+        ref = orc.decode_multi(q[b:b + 1], kc[b:b + 1, :n], vc[b:b + 1, :n], 0.5, 0.5, S, 8)
+        assert np.array_equal(dec["mask"][b, :, :S], ref["mask"][0])
+        assert np.allclose(dec["o"][b], ref["o"][0], atol=1e-13) and np.allclose(dec["lse"][b], ref["lse"][0], atol=1e-13)
+    # two keys, three new tokens: token 0 sees none, token 1 the first key, token 2 both
+    assert (dec["o"][3, 0] == 0).all() and np.isneginf(dec["lse"][3, 0]).all()
+    for h in range(G):
+        assert np.allclose(dec["o"][3, 1, h], vc[3, 0, 0], atol=1e-12)
+        e = np.exp(0.5 * kc[3, :2, 0] @ q[3, 2, h])
+        assert np.allclose(dec["o"][3, 2, h], (e / e.sum()) @ vc[3, :2, 0], atol=1e-12)
