@@ -423,22 +423,28 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * args.steps + 1)]
-    ev[0].record()
+    # timing hygiene: inputs larger than L2 need no flush; smaller ones (cfg1, cfg2) get L2 overwritten between steps,
+    # outside the per-step events
+    L2_BYTES = 126 << 20
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if case.input_bytes() <= L2_BYTES else None
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     for s in range(args.steps):
+        if flush_buf is not None:
+            flush_buf.fill_(s & 0xff)
+        ev[s][0].record()
         case.fwd(tau)
-        ev[3 * s + 1].record()
+        ev[s][1].record()
         case.bwd(tau)
-        ev[3 * s + 2].record()
-        ev[3 * s + 3].record()
+        ev[s][2].record()
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = ev[0].elapsed_time(ev[3 * args.steps])
-    fwd_ms = sum((ev[3 * s].elapsed_time(ev[3 * s + 1]) for s in range(args.steps))) / args.steps
-    bwd_ms = sum((ev[3 * s + 1].elapsed_time(ev[3 * s + 2]) for s in range(args.steps))) / args.steps
+    fwd_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    bwd_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    # the K steps run back to back on one stream: without a flush this is the elapsed time of the whole region
+    total_ms = ev[0][0].elapsed_time(ev[-1][2]) if flush_buf is None else sum(e[0].elapsed_time(e[2]) for e in ev)
     total_ms = max_over_ranks(total_ms, dev)
     assert mala.device_status() == 0, "a device-side wait expired"
     ms_per_step = total_ms / args.steps
@@ -637,7 +643,10 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{c.name} {args.preset}: causal GQA B={c.B} Hq={c.Hq} Hkv={c.Hkv} N={c.N} d={c.d}, "
                                f"tau={tau}, fwd+bwd per step",
-                   "l2": f"inputs {case.input_bytes() / 1e6:.0f} MB per step exceed the 126 MB L2 (no flush needed)",
+                   "l2": (f"inputs {case.input_bytes() / 1e6:.0f} MB per step exceed the 126 MB L2 (no flush needed)"
+                          if flush_buf is None else
+                          f"inputs {case.input_bytes() / 1e6:.0f} MB per step fit in L2: a 252 MB buffer is written between "
+                          f"steps, outside the timed events"),
                    "parallelism": "replicas (one head slice per GPU, no collective)" if world > 1 else "single GPU"},
         "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
         "fwd_retained_frac": ts["fwd_retained"] / ts["fwd_legal"], "bwd_retained_frac": ts["bwd_retained"] / ts["bwd_legal"],
