@@ -100,3 +100,24 @@ def test_varlen_of_equal_lengths_equals_the_batched_call(mala):
                                     cu, 512, w["scale"], tau)
         assert torch.equal(o.reshape(1, 1536, 4, 128), ov)
         assert torch.equal(lse.permute(1, 0, 2).reshape(4, 1536), lv)
+
+
+def test_varlen_with_an_empty_sequence(mala, oracle):
+    # cu_seqlens = [0, 200, 200, 456]: the second sequence has no rows; the others must come out as if it were not there
+    ws = [W.custom_prefill(1, 2, 1, n, 128, seed=50 + n) for n in (200, 256)]
+    pk = W.pack_sequences(ws)
+    q, k, v, do = (pk[x].cuda() for x in ("q", "k", "v", "do"))
+    cu3 = torch.tensor([0, 200, 200, 456], dtype=torch.int32, device="cuda")
+    cu2 = torch.tensor([0, 200, 456], dtype=torch.int32, device="cuda")
+    for tau in (0.0, 1e-4):
+        o3, l3, _ = mala.fwd_varlen(q, k, v, cu3, 256, pk["scale"], tau)
+        o2, l2, _ = mala.fwd_varlen(q, k, v, cu2, 256, pk["scale"], tau)
+        assert torch.equal(o3, o2) and torch.equal(l3, l2)
+        g3 = mala.bwd_varlen(q, k, v, o3, do, l3, cu3, 256, pk["scale"], tau)
+        g2 = mala.bwd_varlen(q, k, v, o2, do, l2, cu2, 256, pk["scale"], tau)
+        torch.cuda.synchronize()
+        assert mala.device_status() == 0
+        for a, b_ in zip(g3[:3], g2[:3]):
+            assert (a.float() - b_.float()).abs().max() <= 1e-2 * b_.float().abs().max()
+    ref = oracle.fwd(ws[1]["q"], ws[1]["k"], ws[1]["v"], pk["scale"], 1e-4, 128, 128)
+    parity.check_output(o3.float().cpu().numpy()[0, 200:], ref["o"][0])
