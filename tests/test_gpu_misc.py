@@ -115,3 +115,39 @@ def test_binding_reports_errors(mala):
         mala.decode(q64, kv64, kv64, 0.1, 0.0, 2)
     assert e.value.code == -2
     assert mala.device_status() == 0
+
+
+def test_calls_can_be_captured_in_a_cuda_graph(mala):
+    """The library allocates nothing and never synchronises, so a decode step and a forward pass can be captured
+    once and replayed on new inputs written into the same buffers."""
+    wd = W.custom_decode(2, 8, 2, 4096, 128, 8, group_types=["diffuse", "peaked"], seed=31, preset="D")
+    q, kc, vc = (wd[x].cuda() for x in ("q", "kcache", "vcache"))
+    wp = W.custom_prefill(1, 4, 2, 1024, 128, seed=32, preset="R")
+    pq, pk, pv = (wp[x].cuda() for x in ("q", "k", "v"))
+    ws = torch.empty(mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 128, 8), dtype=torch.uint8, device="cuda")
+    o, lse = torch.empty_like(q), torch.empty((2, 8), dtype=torch.float32, device="cuda")
+    po, plse = torch.empty_like(pq), torch.empty((1, 4, 1024), dtype=torch.float32, device="cuda")
+
+    def step():
+        mala.decode(q, kc, vc, wd["scale"], 1e-4, 8, ws=ws, out=o)
+        mala.fwd(pq, pk, pv, wp["scale"], 1e-4, out=po, lse=plse)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):                    # first calls outside the capture (one-time set-up per device)
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    # new inputs in the captured buffers, then replay and compare with direct calls
+    q.copy_(torch.roll(q, 1, dims=2))
+    pq.copy_(torch.roll(pq, 3, dims=1))
+    graph.replay()
+    torch.cuda.synchronize()
+    o_g, po_g, plse_g = o.clone(), po.clone(), plse.clone()
+    o_d, _, _ = mala.decode(q, kc, vc, wd["scale"], 1e-4, 8)
+    po_d, plse_d, _ = mala.fwd(pq, pk, pv, wp["scale"], 1e-4)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert torch.equal(o_g, o_d) and torch.equal(po_g, po_d) and torch.equal(plse_g, plse_d)
