@@ -543,14 +543,17 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int info = *(volatile int*)&dq_info;
       if (info < 0) break;
       const int n = info >> 1, ds = info & 1;
-      ok = mbar_wait(&dq_full, k & 1, status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
+      // (the tile's coordinates while the dQ MMAs are still running: the announcement precedes their completion)
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
       const int tile = p.cu ? (int)((size_t)hq * (p.Np / 128) + (size_t)(prow0 / 128 + i))
                             : (int)(((size_t)b * p.Hq + hq) * p.T + (size_t)i);
       uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // D / 64 panels of 16 KB
+      float* const acc_tile = p.dq_acc + (size_t)tile * (128 * D) + rl * 4;
+      asm volatile("" :: "l"(acc_tile), "l"(stg) : "memory");   // keep the address arithmetic ahead of the wait
+      ok = mbar_wait(&dq_full, k & 1, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
       uint32_t a[D / 32][32];
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + c * 32), a[c]);
@@ -559,7 +562,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(&dq_empty);       // TMEM columns may be reused by the next dP
       {
-        float* acc = p.dq_acc + (size_t)tile * (128 * D) + rl * 4;
+        float* acc = acc_tile;
 #pragma unroll
         for (int c = 0; c < D / 64; ++c)
 #pragma unroll
