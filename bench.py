@@ -134,6 +134,28 @@ def time_cuda(fn, warmup, iters):
     return e0.elapsed_time(e1) / iters
 
 
+def time_alternating(fns, warmup, iters, rounds=2, prep=None):
+    """Average milliseconds per call of each function in `fns` (label -> callable).  The functions are measured in
+    turn over several rounds, so that a clock that drifts under the power cap treats them alike (a kernel timed right
+    after a long backward pass runs a few per cent slower than the same kernel timed first).  `prep` (label ->
+    callable) runs untimed before each of the label's chunks, e.g. the forward pass whose output a backward needs."""
+    import torch
+    for k, f in fns.items():
+        if prep:
+            prep[k]()
+        for _ in range(warmup):
+            f()
+    torch.cuda.synchronize()
+    per = max(1, iters // rounds)
+    tot = {k: 0.0 for k in fns}
+    for _ in range(rounds):
+        for k, f in fns.items():
+            if prep:
+                prep[k]()
+            tot[k] += time_cuda(f, 0, per) * per
+    return {k: v / (per * rounds) for k, v in tot.items()}
+
+
 class PrefillCase:
     """Device-resident inputs, outputs and scratch of one prefill configuration."""
 
@@ -188,11 +210,13 @@ def chunk_leg(cs, Nq, tau, it, peaks):
     o, lse = torch.empty_like(q), torch.empty((cc.B, cc.Hq, Nq), dtype=torch.float32, device=q.device)
     dq = torch.empty_like(q)
     row = {}
-    for label, t_ in (("mala", tau), ("dense", 0.0)):
-        f_ms = time_cuda(lambda: mala.fwd_chunk(q, cs.k, cs.v, cs.scale, t_, out=o, lse=lse), 3, it)
-        b_ms = time_cuda(lambda: mala.bwd_chunk(q, cs.k, cs.v, o, do, lse, cs.scale, t_, ws=cs.ws, dq=dq, dk=cs.dk,
-                                                dv=cs.dv), 3, it)
-        row[label] = {"fwd_ms": f_ms, "bwd_ms": b_ms}
+    taus = {"mala": tau, "dense": 0.0}
+    fwd = {k: (lambda t_=t_: mala.fwd_chunk(q, cs.k, cs.v, cs.scale, t_, out=o, lse=lse)) for k, t_ in taus.items()}
+    bwd = {k: (lambda t_=t_: mala.bwd_chunk(q, cs.k, cs.v, o, do, lse, cs.scale, t_, ws=cs.ws, dq=dq, dk=cs.dk, dv=cs.dv))
+           for k, t_ in taus.items()}
+    f_t, b_t = time_alternating(fwd, 3, it), time_alternating(bwd, 3, it, prep=fwd)
+    for label in taus:
+        row[label] = {"fwd_ms": f_t[label], "bwd_ms": b_t[label]}
     _, _, fs = mala.fwd_chunk(q, cs.k, cs.v, cs.scale, tau, out=o, lse=lse, stats=True)
     _, _, _, bs = mala.bwd_chunk(q, cs.k, cs.v, o, do, lse, cs.scale, tau, ws=cs.ws, dq=dq, dk=cs.dk, dv=cs.dv,
                                  stats=True)
@@ -252,12 +276,14 @@ def varlen_leg(cfg, preset, lens, tau, it, peaks, dev):
     wsb = torch.empty(mala.workspace_bytes(mala.OP_BWD, 1, cfg.Hq, cfg.Hkv, total + 128 * len(lens), cfg.d),
                       dtype=torch.uint8, device=dev)
     row = {"lens": list(lens)}
-    o, lse, _ = mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], tau)
-    for label, t_ in (("mala", tau), ("dense", 0.0)):
-        f_ms = time_cuda(lambda: mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], t_), 3, it)
-        o, lse, _ = mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], t_)
-        b_ms = time_cuda(lambda: mala.bwd_varlen(q, k, v, o, do, lse, cu, mx, pk["scale"], t_, ws=wsb), 3, it)
-        row[label] = {"fwd_ms": f_ms, "bwd_ms": b_ms}
+    taus = {"mala": tau, "dense": 0.0}
+    outs = {lab: mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], t_)[:2] for lab, t_ in taus.items()}
+    fwd = {lab: (lambda t_=t_: mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], t_)) for lab, t_ in taus.items()}
+    bwd = {lab: (lambda t_=t_, lab=lab: mala.bwd_varlen(q, k, v, outs[lab][0], do, outs[lab][1], cu, mx, pk["scale"], t_,
+                                                         ws=wsb)) for lab, t_ in taus.items()}
+    f_t, b_t = time_alternating(fwd, 3, it), time_alternating(bwd, 3, it)
+    for label in taus:
+        row[label] = {"fwd_ms": f_t[label], "bwd_ms": b_t[label]}
     o, lse, fs = mala.fwd_varlen(q, k, v, cu, mx, pk["scale"], tau, stats=True)
     _, _, _, bs = mala.bwd_varlen(q, k, v, o, do, lse, cu, mx, pk["scale"], tau, ws=wsb, stats=True)
     torch.cuda.synchronize()
@@ -383,7 +409,7 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--preset", default="literal", choices=["literal", "R"])
     ap.add_argument("--tau", type=float, default=1e-4)
-    ap.add_argument("--detail-iters", type=int, default=10, help="timed iterations of each detail measurement")
+    ap.add_argument("--detail-iters", type=int, default=20, help="timed iterations of each detail measurement")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-config detail table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -530,9 +556,12 @@ def main():
                 cs = case if (name == args.workload and preset == args.preset) else PrefillCase(name, preset, dev)
                 cc = cs.cfg
                 row = {}
-                for label, t_ in (("mala", tau), ("dense", 0.0)):
-                    f_ms = time_cuda(lambda: cs.fwd(t_), 3, it)
-                    b_ms = time_cuda(lambda: cs.bwd(t_), 3, it)
+                taus = {"mala": tau, "dense": 0.0}
+                f_t = time_alternating({k: (lambda t_=t_: cs.fwd(t_)) for k, t_ in taus.items()}, 3, it)
+                b_t = time_alternating({k: (lambda t_=t_: cs.bwd(t_)) for k, t_ in taus.items()}, 3, it,
+                                       prep={k: (lambda t_=t_: cs.fwd(t_)) for k, t_ in taus.items()})
+                for label in taus:
+                    f_ms, b_ms = f_t[label], b_t[label]
                     row[label] = {"fwd_ms": f_ms, "bwd_ms": b_ms,
                                   "fwd_dense_equiv_tflops": cs.fwd_de / f_ms / 1e9,
                                   "bwd_dense_equiv_tflops": cs.bwd_de / b_ms / 1e9}
