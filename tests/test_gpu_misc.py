@@ -151,3 +151,24 @@ def test_calls_can_be_captured_in_a_cuda_graph(mala):
     torch.cuda.synchronize()
     assert mala.device_status() == 0
     assert torch.equal(o_g, o_d) and torch.equal(po_g, po_d) and torch.equal(plse_g, plse_d)
+
+
+def test_autograd_function_runs_both_algorithms(mala, oracle):
+    from paper_2609_32712_b200.autograd import mala_attention
+    w = W.custom_prefill(1, 4, 2, 640, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=41, preset="R")
+    for tau in (0.0, 1e-4):
+        q, k, v = (w[x].cuda().requires_grad_(True) for x in ("q", "k", "v"))
+        o = mala_attention(q, k, v, tau, scale=w["scale"])
+        (o.float() * w["do"].cuda().float()).sum().backward()
+        o_d, lse_d, _ = mala.fwd(q.detach(), k.detach(), v.detach(), w["scale"], tau)
+        dq, dk, dv, _ = mala.bwd(q.detach(), k.detach(), v.detach(), o_d, w["do"].cuda(), lse_d, w["scale"], tau)
+        assert torch.equal(o.detach(), o_d)
+        for got, want in ((q.grad, dq), (k.grad, dk), (v.grad, dv)):
+            assert (got.float() - want.float()).abs().max() <= 1e-2 * want.float().abs().max()
+    # against the oracle at tau = 0: the exact gradient of dense attention
+    q, k, v = (w[x].cuda().requires_grad_(True) for x in ("q", "k", "v"))
+    mala_attention(q, k, v, 0.0, scale=w["scale"]).backward(w["do"].cuda())
+    gq, gk, gv = oracle.dense_bwd(w["q"], w["k"], w["v"], w["do"], w["scale"])
+    parity.check_grad(q.grad.float().cpu().numpy(), gq, "dq")
+    parity.check_grad(k.grad.float().cpu().numpy(), gk, "dk")
+    parity.check_grad(v.grad.float().cpu().numpy(), gv, "dv")
