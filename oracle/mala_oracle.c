@@ -206,7 +206,7 @@ static void fwd_block_range(const double* Q, const double* K, const double* V, i
 int mala_oracle_fwd_split(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale,
                           double tau, int Bq, int Bk, int causal, int num_splits, int n_blocks, const int* blocks,
                           double* O, double* lse, uint8_t* mask, double* crit) {
-  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || num_splits <= 0 || !(tau >= 0.0)) return -1;
+  if (N <= 0 || (causal && Nk < N) || d <= 0 || Bq <= 0 || Bk <= 0 || num_splits <= 0 || !(tau >= 0.0)) return -1;
   const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int tps = (Tc + num_splits - 1) / num_splits;
   const int nb = blocks ? n_blocks : Tr;
@@ -308,7 +308,7 @@ int mala_oracle_bwd(const double* Q, const double* K, const double* V, const dou
                     const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal,
                     int n_blocks, const int* key_blocks, double* dQ, double* dK, double* dV, uint8_t* mask,
                     double* crit) {
-  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
+  if (N <= 0 || (causal && Nk < N) || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
   const int off = Nk - N;
   const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int nb = key_blocks ? n_blocks : Tc;
@@ -365,7 +365,7 @@ int mala_oracle_bwd(const double* Q, const double* K, const double* V, const dou
 int mala_oracle_bwd_dq(const double* Q, const double* K, const double* V, const double* dO, const double* lse,
                        const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal,
                        int n_blocks, const int* query_blocks, double* dQ) {
-  if (N <= 0 || Nk < N || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
+  if (N <= 0 || (causal && Nk < N) || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
   const int off = Nk - N;
   const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int nb = query_blocks ? n_blocks : Tr;

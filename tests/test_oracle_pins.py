@@ -817,3 +817,21 @@ def test_decode_paged_with_several_new_tokens_per_sequence():
         assert np.allclose(dec["o"][3, 1, h], vc[3, 0, 0], atol=1e-12)
         e = np.exp(0.5 * kc[3, :2, 0] @ q[3, 2, h])
         assert np.allclose(dec["o"][3, 2, h], (e / e.sum()) @ vc[3, :2, 0], atol=1e-12)
+
+
+def test_non_causal_with_more_queries_than_keys_is_plain_softmax():
+    # cross attention: 40 queries, 17 keys, every key legal, L = 17
+    r = _rng(321)
+    q, k, v = r.standard_normal((1, 40, 1, 8)), r.standard_normal((1, 17, 1, 8)), r.standard_normal((1, 17, 1, 8))
+    f = orc.fwd(q, k, v, 0.4, 0.0, 8, 8, causal=False)
+    for i in range(40):
+        e = np.exp(0.4 * k[0, :, 0] @ q[0, i, 0])
+        assert np.allclose(f["o"][0, i, 0], (e / e.sum()) @ v[0, :, 0], atol=1e-12)
+    do = r.standard_normal(q.shape)
+    g = orc.bwd(q, k, v, f["o"], do, f["lse"], 0.4, 0.0, 8, 8, causal=False)
+    P = np.exp(0.4 * q[0, :, 0] @ k[0, :, 0].T - f["lse"][0, 0][:, None])
+    dP = do[0, :, 0] @ v[0, :, 0].T
+    dS = P * (dP - (f["o"][0, :, 0] * do[0, :, 0]).sum(-1)[:, None])
+    assert np.allclose(g["dv"][0, :, 0], P.T @ do[0, :, 0], atol=1e-12)
+    assert np.allclose(g["dq"][0, :, 0], 0.4 * dS @ k[0, :, 0], atol=1e-12)
+    assert np.allclose(g["dk"][0, :, 0], 0.4 * dS.T @ q[0, :, 0], atol=1e-12)
