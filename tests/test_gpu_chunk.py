@@ -95,6 +95,14 @@ def test_chunk_non_causal_any_lengths(mala, oracle, tau):
     _run(mala, oracle, _chunk(w, 200), tau, causal=False)
 
 
+@pytest.mark.parametrize("tau", [0.0, 1e-2])
+def test_chunk_non_causal_more_queries_than_keys(mala, oracle, tau):
+    # cross attention the other way round: 370 queries against 184 keys
+    w = W.custom_prefill(1, 2, 1, 370, 64, head_types=["peaked", "diffuse"], seed=15, preset="R")
+    c = dict(q=w["q"], k=w["k"][:, :184].contiguous(), v=w["v"][:, :184].contiguous(), do=w["do"], scale=w["scale"])
+    _run(mala, oracle, c, tau, causal=False)
+
+
 def test_chunk_equals_rows_of_the_equal_length_call(mala):
     # both entry points on the GPU: the chunk call must give the last rows of the full call (the forward bit for bit)
     w = W.custom_prefill(1, 4, 2, 1536, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=3, preset="R")
