@@ -14,7 +14,7 @@
  *     never frees or retains one.  Tensors are bf16 views [B, N, H, d] given as a base pointer and
  *     element strides (sb, sn, sh); the last dimension is contiguous.  Base pointers must be
  *     16-byte aligned and all strides multiples of 8 elements (16 bytes).
- *   - d is 64 or 128 (the decode calls: 128 only, MALA_ERR_UNSUPPORTED otherwise).  Hq must be a multiple of Hkv; query head h uses key/value head
+ *   - d is 64 or 128.  Hq must be a multiple of Hkv; query head h uses key/value head
  *     h / (Hq / Hkv).  N may be any positive length (the last tile may be ragged).
  *   - scale (> 0, finite) multiplies the fp32 scores; lse is in nats, of the scaled scores, over
  *     the retained set.  tau >= 0, finite.

@@ -44,7 +44,8 @@ inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) {
 inline bool decode_set_attributes() {
   bool ok = true;
 #define MALA_DEC_ATTR(DENSE, GP, MULTI) \
-  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess; \
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
 #define MALA_DEC_ATTR_GP(GP) MALA_DEC_ATTR(false, GP, false) MALA_DEC_ATTR(true, GP, false) MALA_DEC_ATTR(false, GP, true) MALA_DEC_ATTR(true, GP, true)
   MALA_DEC_ATTR_GP(1) MALA_DEC_ATTR_GP(2) MALA_DEC_ATTR_GP(4) MALA_DEC_ATTR_GP(8) MALA_DEC_ATTR_GP(16)
 #undef MALA_DEC_ATTR_GP
@@ -66,7 +67,7 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
                                       const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                                       float tau, int num_splits, float* o_part, float* lse_part, int* status,
                                       cudaStream_t stream, const DecPaging* pg = nullptr, int Sq = 1) {
-  if (d != 128) return MALA_ERR_UNSUPPORTED;
+  if (d != 128 && d != 64) return MALA_ERR_UNSUPPORTED;
   const int G = Hq / Hkv;
   if (Sq < 1 || G * Sq > 16 || Sq > Nk) return MALA_ERR_UNSUPPORTED;
   const bool paged = pg && pg->block_table;
@@ -110,10 +111,15 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
     return MALA_ERR_CUDA;
   const int grid = p.n_items < sms ? p.n_items : sms;   // persistent: one CTA per SM
   const int R = G * Sq;   // rows of a work item
-#define MALA_DEC_LAUNCH2(DENSE, GP)                                                                                  \
+#define MALA_DEC_LAUNCH3(DENSE, GP, MULTI)                                                                           \
   {                                                                                                                  \
-    if (Sq > 1) mala_decode_split_kernel<DENSE, GP, true><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
-    else mala_decode_split_kernel<DENSE, GP, false><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);       \
+    if (d == 128) mala_decode_split_kernel<DENSE, GP, MULTI, 128><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    else mala_decode_split_kernel<DENSE, GP, MULTI, 64><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);           \
+  }
+#define MALA_DEC_LAUNCH2(DENSE, GP)          \
+  {                                          \
+    if (Sq > 1) MALA_DEC_LAUNCH3(DENSE, GP, true) \
+    else MALA_DEC_LAUNCH3(DENSE, GP, false)  \
   }
 #define MALA_DEC_LAUNCH(GP)            \
   {                                    \
@@ -127,8 +133,13 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   else MALA_DEC_LAUNCH(16)
 #undef MALA_DEC_LAUNCH
 #undef MALA_DEC_LAUNCH2
+#undef MALA_DEC_LAUNCH3
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
-  decode_merge_kernel<128><<<B * Sq * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
+  if (d == 128)
+    decode_merge_kernel<128><<<B * Sq * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
+                                                              Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits);
+  else
+    decode_merge_kernel<64><<<B * Sq * Hq, 64, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
                                                             Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }

@@ -105,11 +105,16 @@ __device__ __forceinline__ void lds_row(const float* src, float (&dst)[N]) {
 // GP: the number of packed rows rounded up to a power of two (compile-time, so that the per-row loops of the
 // softmax group unroll without branches).  kMulti: several new tokens per sequence, i.e. rows that see
 // different numbers of keys (one token: every row sees all keys, and the per-row limits fold into scalars).
-template <bool kDense, int GP, bool kMulti>
+// D: head size, 128 or 64.  The shared-memory stages keep their 128-wide size for D = 64 and only their first
+// 64-column panel is filled; O^T is then still accumulated as a 128-row MMA whose rows 64.. (fed from the unfilled
+// half of the V stage) are never read.
+template <bool kDense, int GP, bool kMulti, int D>
 __global__ void __launch_bounds__(384, 1)
 mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                          const __grid_constant__ CUtensorMap tmV, const DecParams p) {
   constexpr int KS = DecCfg::kKStages, VS = DecCfg::kVStages, TB = DecCfg::kTileBytes;
+  constexpr int PAN = D / 64;                    // 64-column panels of a K / V / Q tile
+  constexpr uint32_t kTileTx = 128u * D * 2u;    // bytes one K or V tile copy delivers
   constexpr int NG = GP >= 8 ? 2 : 1;      // softmax groups (four warps each)
   constexpr int GH = GP / NG;              // rows per group
   constexpr int LDN = NG == 1 ? 16 : GH;   // TMEM columns a softmax thread reads at a time
@@ -203,9 +208,10 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         const int ip = ne & 1;
         ok = mbar_wait(&q_empty[ip], ((ne >> 1) & 1) ^ 1, status);
         if (!ok) break;
-        mbar_arrive_expect_tx(&q_full[ip], (uint32_t)R * 256u);   // two panels of R rows x 128 bytes
-        tma_load_4d(sQ + ip * DecCfg::kQBytes, &tmQ, &q_full[ip], 0, hkv * G, 0, b);
-        tma_load_4d(sQ + ip * DecCfg::kQBytes + 2048, &tmQ, &q_full[ip], 64, hkv * G, 0, b);
+        mbar_arrive_expect_tx(&q_full[ip], (uint32_t)R * 128u * PAN);   // panels of R rows x 128 bytes
+#pragma unroll
+        for (int pn = 0; pn < PAN; ++pn)
+          tma_load_4d(sQ + ip * DecCfg::kQBytes + pn * 2048, &tmQ, &q_full[ip], pn * 64, hkv * G, 0, b);
         for (int t = 0; t < T && ok; ++t, ++g) {
           int row, outer;
           tile_coord(b, j0 - t, row, outer);     // (a page lookup is in flight while the slot is waited for)
@@ -215,16 +221,18 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           // tiles behind this one (K ring of three behind the S^T cursor, vote cursor at most four behind that),
           // and it sees the two stores through the K tile's barrier.
           if (!kDense) { v_row[g & 7] = row; v_outer[g & 7] = outer; }
-          mbar_arrive_expect_tx(&k_full[ks], TB);
-          tma_load_4d(sK + ks * TB, &tmK, &k_full[ks], 0, row, hkv, outer);
-          tma_load_4d(sK + ks * TB + 16384, &tmK, &k_full[ks], 64, row, hkv, outer);
+          mbar_arrive_expect_tx(&k_full[ks], kTileTx);
+#pragma unroll
+          for (int pn = 0; pn < PAN; ++pn)
+            tma_load_4d(sK + ks * TB + pn * 16384, &tmK, &k_full[ks], pn * 64, row, hkv, outer);
           if (++ks == KS) { ks = 0; kpar ^= 1; }
           if (kDense) {   // every tile is retained: V follows K
             ok = mbar_wait(&v_empty[vs], vpar, status);
             if (!ok) break;
-            mbar_arrive_expect_tx(&v_full[vs], TB);
-            tma_load_4d(sV + vs * TB, &tmV, &v_full[vs], 0, row, hkv, outer);
-            tma_load_4d(sV + vs * TB + 16384, &tmV, &v_full[vs], 64, row, hkv, outer);
+            mbar_arrive_expect_tx(&v_full[vs], kTileTx);
+#pragma unroll
+            for (int pn = 0; pn < PAN; ++pn)
+              tma_load_4d(sV + vs * TB + pn * 16384, &tmV, &v_full[vs], pn * 64, row, hkv, outer);
             if (++vs == VS) { vs = 0; vpar ^= 1; }
           }
         }
@@ -284,7 +292,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             const uint32_t dS = tmem_addr(tb, 0, (uint32_t)sb * 16u);
             const uint64_t dQ = desc_advance(dQ0, ip * DecCfg::kQBytes), dK = desc_advance(dK0, kc * TB);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)   // K panels lie 16 KB apart, Q panels 2 KB
+            for (int k = 0; k < D / 16; ++k)   // K panels lie 16 KB apart, Q panels 2 KB
               mma_ss(dS, desc_advance(dK, (k >> 2) * 16384 + (k & 3) * 32), desc_advance(dQ, (k >> 2) * 2048 + (k & 3) * 32),
                      idesc_qk, k > 0, leader);
             if (leader) {
@@ -313,9 +321,10 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             } else if (ready(&v_empty[vi], vipar)) {   // V of this tile, on demand
               if (leader) {
                 const int row = *(volatile int*)&v_row[cv.g & 7], outer = *(volatile int*)&v_outer[cv.g & 7];
-                mbar_arrive_expect_tx(&v_full[vi], TB);
-                tma_load_4d(sV + vi * TB, &tmV, &v_full[vi], 0, row, cv.hkv, outer);
-                tma_load_4d(sV + vi * TB + 16384, &tmV, &v_full[vi], 64, row, cv.hkv, outer);
+                mbar_arrive_expect_tx(&v_full[vi], kTileTx);
+#pragma unroll
+                for (int pn = 0; pn < PAN; ++pn)
+                  tma_load_4d(sV + vi * TB + pn * 16384, &tmV, &v_full[vi], pn * 64, row, cv.hkv, outer);
               }
               __syncwarp();
               if (++vi == VS) { vi = 0; vipar ^= 1; }
@@ -430,8 +439,8 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       if (lane == 0) mbar_arrive(&o_free[pend_ip]);   // the accumulator may take the item after next
 #pragma unroll
       for (int q = 0; q < GH; ++q)
-        if (rb + q < R)   // (a row that saw no key of the split: (0, -inf))
-          p.o_part[(pend_prow0 + rowoff[q]) * 128 + kt] =
+        if (rb + q < R && kt < D)   // (a row that saw no key of the split: (0, -inf))
+          p.o_part[(pend_prow0 + rowoff[q]) * D + kt] =
               (!kMulti || pend_l[q] > 0.f) ? __uint_as_float(o[q]) / pend_l[q] : 0.f;
       pend = false;
       return true;
@@ -453,7 +462,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 #pragma unroll
         for (int q = 0; q < GH; ++q)
           if (rb + q < R) {
-            p.o_part[(prow0 + rowoff[q]) * 128 + kt] = 0.f;
+            if (kt < D) p.o_part[(prow0 + rowoff[q]) * D + kt] = 0.f;
             if (kt == q) p.lse_part[prow0 + rowoff[q]] = -INFINITY;
           }
         if (head && p.retained) p.retained[stat_row] = 0u;

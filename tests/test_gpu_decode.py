@@ -254,3 +254,19 @@ def test_decode_paged_with_several_new_tokens(mala, oracle, Nk, S, Hq, Hkv, page
     fin = np.isfinite(ref["lse"])
     assert np.abs(lse_c[fin] - ref["lse"][fin]).max() <= parity.LSE_ABS
     assert np.isneginf(lse_c[~fin]).all() and (o_c[~fin] == 0).all()
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv", [(1024, 4, 8, 2), (1000, 3, 4, 4), (4096, 8, 16, 1), (300, 2, 6, 2)])
+def test_decode_head_size_64(mala, oracle, Nk, S, Hq, Hkv, tau):
+    w = W.custom_decode(2, Hq, Hkv, Nk, 64, S, seed=Nk + S)
+    _run_and_check(mala, oracle, w, tau, S)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+def test_decode_head_size_64_gated_paged_several_tokens(mala, oracle, tau):
+    w = W.custom_decode(2, 8, 2, 8192, 64, 8, group_types=["diffuse", "peaked"], seed=3, preset="D")
+    res = _run_and_check(mala, oracle, w, tau, 8)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+    _run_paged(mala, oracle, w, tau, 8, 256, [8192, 4096 + 77], seed=9)
+    assert _run_multi(mala, oracle, w, 3, tau, 8) > 0
