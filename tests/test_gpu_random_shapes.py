@@ -62,19 +62,19 @@ def test_random_cases(mala, oracle, seed):
         elif kind == "decode":
             Hkv, G = rng.choice([1, 2, 3]), rng.choice([1, 2, 3, 4, 5, 8, 16])
             Nk, S = rng.randint(1, 5000), rng.randint(1, 12)
-            w = W.custom_decode(rng.choice([1, 2, 3]), Hkv * G, Hkv, Nk, 128, S, seed=rng.randint(0, 9999),
+            w = W.custom_decode(rng.choice([1, 2, 3]), Hkv * G, Hkv, Nk, d, S, seed=rng.randint(0, 9999),
                                 preset=rng.choice(["literal", "D"]))
             TD._run_and_check(mala, oracle, w, tau, S)
         elif kind == "paged":
             Hkv, G, page = rng.choice([1, 2]), rng.choice([1, 2, 4, 8]), rng.choice([128, 256, 512])
             Nk, S, B = page * rng.randint(1, 12), rng.randint(1, 8), rng.choice([1, 2, 3])
             lens = [rng.randint(0, Nk) for _ in range(B)]
-            w = W.custom_decode(B, Hkv * G, Hkv, Nk, 128, S, seed=rng.randint(0, 9999), preset=rng.choice(["literal", "D"]))
+            w = W.custom_decode(B, Hkv * G, Hkv, Nk, d, S, seed=rng.randint(0, 9999), preset=rng.choice(["literal", "D"]))
             TD._run_paged(mala, oracle, w, tau, S, page, lens, seed=it)
         else:
             Hkv, G = rng.choice([1, 2]), rng.choice([1, 2, 4])
             Sq = rng.randint(2, 16 // G)
             Nk, S = rng.randint(Sq, 4000), rng.randint(1, 8)
-            w = W.custom_decode(rng.choice([1, 2]), Hkv * G, Hkv, Nk, 128, S, seed=rng.randint(0, 9999),
+            w = W.custom_decode(rng.choice([1, 2]), Hkv * G, Hkv, Nk, d, S, seed=rng.randint(0, 9999),
                                 preset=rng.choice(["literal", "D"]))
             TD._run_multi(mala, oracle, w, Sq, tau, S, seed=it)
