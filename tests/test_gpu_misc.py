@@ -109,10 +109,10 @@ def test_binding_reports_errors(mala):
     with pytest.raises(mala.MalaError) as e:
         mala.fwd(q96, q96, q96, 0.1, 0.0)
     assert e.value.code == -2
-    q64 = torch.zeros(1, 1, 2, 64, dtype=torch.bfloat16, device="cuda")
-    kv64 = torch.zeros(1, 256, 2, 64, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(mala.MalaError) as e:        # decode supports d = 128 only
-        mala.decode(q64, kv64, kv64, 0.1, 0.0, 2)
+    q17 = torch.zeros(1, 1, 34, 128, dtype=torch.bfloat16, device="cuda")
+    kv1 = torch.zeros(1, 256, 2, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(mala.MalaError) as e:        # decode packs at most 16 query heads per KV head
+        mala.decode(q17, kv1, kv1, 0.1, 0.0, 2)
     assert e.value.code == -2
     assert mala.device_status() == 0
 
