@@ -1,4 +1,4 @@
-// Split-KV decode, split kernel ("Fused decoding execution") for sm_100a, head size 128.
+// Split-KV decode, split kernel ("Fused decoding execution") for sm_100a, head size 128 or 64.
 //
 // A work item is one split of one (batch, KV head): the G = Hq/Hkv <= 16 query heads that share the KV head
 // are processed together, L = Nk for every head, the tiles of the split are visited newest first with the
