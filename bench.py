@@ -409,7 +409,10 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--preset", default="literal", choices=["literal", "R"])
     ap.add_argument("--tau", type=float, default=1e-4)
-    ap.add_argument("--detail-iters", type=int, default=20, help="timed iterations of each detail measurement")
+    ap.add_argument("--detail-iters", type=int, default=20,
+                    help="timed iterations of each prefill detail measurement (3 warm-up iterations before them; the "
+                         "paper's protocol of 25 warm-up + 100 timed iterations is what the decode legs use, and "
+                         "--detail-iters 100 gives the prefill legs 100 timed iterations too)")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-config detail table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
