@@ -86,13 +86,17 @@ int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, cons
 
 /* Algorithms 1 and 2 with fewer queries than keys (chunked prefill; cross attention when causal == 0).
  * q, o, dout, dq [B,Nq,Hq,d]; k, v, dk, dv [B,Nk,Hkv,d]; lse fp32 [B,Hq,Nq].
- * causal != 0: the queries are the LAST Nq of the Nk positions: query row q attends to the keys 0 .. q + Nk - Nq
- * and L_q = q + 1 + Nk - Nq, the number of keys it sees (Section 2.1); a query block visits its tiles from its
- * diagonal toward earlier keys.  The chunk must start on a tile boundary: Nk >= Nq and (Nk - Nq) % 128 == 0,
- * MALA_ERR_UNSUPPORTED otherwise.  The result equals rows Nk - Nq .. Nk - 1 of the equal-length call on the whole
- * sequence (for the backward: with dout zero on the earlier rows).
+ * causal != 0: the queries are the LAST Nq of the Nk positions (Nk >= Nq): query row q attends to the keys
+ * 0 .. q + Nk - Nq and L_q = q + 1 + Nk - Nq, the number of keys it sees (Section 2.1); a query block visits its
+ * tiles from its diagonal toward earlier keys.  The query blocks follow the key positions -- block i holds the rows q
+ * with 128 i <= q + (Nk - Nq) % 128 < 128 (i + 1), so the first block of a chunk that starts inside a tile is a short
+ * one -- and the result therefore equals rows Nk - Nq .. Nk - 1 of the equal-length call on the whole sequence wherever
+ * the chunk holds a whole block of that call (for the backward: with dout zero on the earlier rows).
+ * mala_fwd_chunk takes any Nk >= Nq; mala_bwd_chunk needs the chunk to start on a tile boundary,
+ * (Nk - Nq) % 128 == 0 (MALA_ERR_UNSUPPORTED otherwise).
  * causal == 0: every key legal for every query, L_q = Nk, any Nq and Nk.
- * Telemetry: fwd retained_per_block [B,Hq,ceil(Nq/128)], tile_bitmask [B,Hq,ceil(Nq/128),ceil(ceil(Nk/128)/32)];
+ * Telemetry: fwd retained_per_block [B,Hq,Tq], tile_bitmask [B,Hq,Tq,ceil(ceil(Nk/128)/32)] with
+ * Tq = ceil((Nq + (Nk - Nq) % 128) / 128) (causal) or ceil(Nq/128);
  * bwd retained_per_block [B,Hq,ceil(Nk/128)], tile_bitmask [B,Hq,ceil(Nk/128),ceil(ceil(Nq/128)/32)].
  * Workspace of the backward: mala_workspace_bytes(MALA_OP_BWD, B, Hq, Hkv, Nq, d, 0).  Everything else as
  * mala_fwd / mala_bwd, which are these calls with Nq = Nk = N. */

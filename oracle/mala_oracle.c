@@ -138,10 +138,12 @@ int mala_oracle_dense_bwd(const double* Q, const double* K, const double* V, con
  * running state m, l, acc (rows of the block).  S, mt: scratch.  mask, crit: [Tr*Tc] or NULL.
  * ---------------------------------------------------------------------------------------- */
 static void fwd_block_range(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale,
-                            double tau, int Bq, int Bk, int causal, int i, int j_lo, int j_hi, int Tc, double* m,
-                            double* l, double* acc, double* S, double* mt, uint8_t* mask, double* crit) {
+                            double tau, int Bq, int Bk, int causal, int shift, int i, int j_lo, int j_hi, int Tc,
+                            double* m, double* l, double* acc, double* S, double* mt, uint8_t* mask, double* crit) {
   const int off = Nk - N; /* N queries (the last N positions) against Nk keys */
-  const int q0 = i * Bq, rows = (q0 + Bq <= N ? Bq : N - q0);
+  /* query block i holds the rows q with i*Bq <= q + shift < (i+1)*Bq (shift = 0: blocks count from the first row) */
+  const int q0 = (i * Bq - shift > 0 ? i * Bq - shift : 0);
+  const int q1 = ((i + 1) * Bq - shift < N ? (i + 1) * Bq - shift : N), rows = q1 - q0;
   for (int j = j_hi; j >= j_lo; --j) { /* descending from the diagonal toward earlier keys */
     const int k0 = j * Bk, cols = (k0 + Bk <= Nk ? Bk : Nk - k0);
     /* a tile with no legal key for any row is not visited */
@@ -199,21 +201,27 @@ static void fwd_block_range(const double* Q, const double* K, const double* V, i
 /* Algorithm 1 for the listed query blocks of one head (blocks == NULL: all).
  * O [N,d], lse [N]: rows of the listed blocks are written.  mask, crit: [Tr*Tc], rows of the
  * listed blocks are written (may be NULL).
+ * shift (0 <= shift < Bq): the query blocks are laid out as if shift more rows preceded the first one, i.e. block i
+ * holds the rows q with i*Bq <= q + shift < (i+1)*Bq and there are ceil((N + shift)/Bq) blocks.  With
+ * shift = (Nk - N) mod Bq the blocks of a chunk of queries coincide with the blocks those rows have in the
+ * equal-length problem over all Nk positions (the result depends on the partition).
  * num_splits > 1: the key blocks are cut into num_splits contiguous ranges of ceil(Tc / num_splits) blocks; every
  * range runs the rule on its own running state (its test sees the range's PARTIAL normalizer, as in "Fused decoding
  * execution") and the ranges' results (o_s, lse_s) are merged by lse = log sum_s exp(lse_s),
  * o = sum_s exp(lse_s - lse) o_s.  A range that holds no legal key of a row contributes nothing to it. */
 int mala_oracle_fwd_split(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale,
-                          double tau, int Bq, int Bk, int causal, int num_splits, int n_blocks, const int* blocks,
-                          double* O, double* lse, uint8_t* mask, double* crit) {
+                          double tau, int Bq, int Bk, int causal, int num_splits, int shift, int n_blocks,
+                          const int* blocks, double* O, double* lse, uint8_t* mask, double* crit) {
   if (N <= 0 || (causal && Nk < N) || d <= 0 || Bq <= 0 || Bk <= 0 || num_splits <= 0 || !(tau >= 0.0)) return -1;
-  const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
+  if (shift < 0 || shift >= Bq) return -1;
+  const int Tr = (N + shift + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int tps = (Tc + num_splits - 1) / num_splits;
   const int nb = blocks ? n_blocks : Tr;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < nb; ++u) {
     const int i = blocks ? blocks[u] : (Tr - 1 - u); /* long blocks first when running all */
-    const int q0 = i * Bq, rows = (q0 + Bq <= N ? Bq : N - q0);
+    const int q0 = (i * Bq - shift > 0 ? i * Bq - shift : 0);
+    const int q1 = ((i + 1) * Bq - shift < N ? (i + 1) * Bq - shift : N), rows = q1 - q0;
     /* Alg. 1: O_i = 0, l_i = 0, m_i = -inf; L_i from positions */
     double* m = (double*)malloc(sizeof(double) * rows);
     double* l = (double*)malloc(sizeof(double) * rows);
@@ -226,7 +234,8 @@ int mala_oracle_fwd_split(const double* Q, const double* K, const double* V, int
       for (int r = 0; r < rows; ++r) { m[r] = -INFINITY; l[r] = 0.0; }
       memset(acc, 0, sizeof(double) * (size_t)rows * d);
       const int j_lo = s * tps, j_hi = ((s + 1) * tps < Tc ? (s + 1) * tps : Tc) - 1;
-      fwd_block_range(Q, K, V, N, Nk, d, scale, tau, Bq, Bk, causal, i, j_lo, j_hi, Tc, m, l, acc, S, mt, mask, crit);
+      fwd_block_range(Q, K, V, N, Nk, d, scale, tau, Bq, Bk, causal, shift, i, j_lo, j_hi, Tc, m, l, acc, S, mt, mask,
+                      crit);
       /* O_i <- diag(l)^-1 O_i,  l_i <- m_i + log l_i */
       for (int r = 0; r < rows; ++r) {
         lse_s[(size_t)s * rows + r] = (l[r] == 0.0 ? -INFINITY : m[r] + log(l[r]));
@@ -250,7 +259,8 @@ int mala_oracle_fwd_split(const double* Q, const double* K, const double* V, int
 int mala_oracle_fwd(const double* Q, const double* K, const double* V, int N, int Nk, int d, double scale, double tau,
                     int Bq, int Bk, int causal, int n_blocks, const int* blocks, double* O, double* lse,
                     uint8_t* mask, double* crit) {
-  return mala_oracle_fwd_split(Q, K, V, N, Nk, d, scale, tau, Bq, Bk, causal, 1, n_blocks, blocks, O, lse, mask, crit);
+  return mala_oracle_fwd_split(Q, K, V, N, Nk, d, scale, tau, Bq, Bk, causal, 1, 0, n_blocks, blocks, O, lse, mask,
+                               crit);
 }
 
 /* D = rowsum(O o dO) (Alg. 2, the term subtracted from dP). */

@@ -50,8 +50,8 @@ def lib():
         L.mala_oracle_dense_fwd.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _ci, _ci, _ci, _D, _D]
         L.mala_oracle_dense_bwd.argtypes = [_D, _D, _D, _D, _ci, _ci, _cd, _ci, _D, _D, _D]
         L.mala_oracle_fwd.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D, _D, _U8, _D]
-        L.mala_oracle_fwd_split.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _ci, _I, _D, _D, _U8,
-                                            _D]
+        L.mala_oracle_fwd_split.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _ci, _ci, _I, _D, _D,
+                                            _U8, _D]
         L.mala_oracle_bwd_D.argtypes = [_D, _D, _ci, _ci, _D]
         L.mala_oracle_bwd.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I,
                                       _D, _D, _D, _U8, _D]
@@ -143,10 +143,14 @@ def dense_bwd(q, k, v, do, scale: float, causal: bool = True):
     return dq, dk, dv
 
 
-def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True, units=None, num_splits: int = 1):
+def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True, units=None, num_splits: int = 1,
+        q_shift: int = 0):
     """Algorithm 1.  ``units``: optional list of (b, h_q, i) query blocks; rows of other blocks stay NaN.
     ``num_splits`` > 1: the key blocks are cut into that many contiguous ranges of ceil(Tc / num_splits) blocks,
     each range runs the rule on its own state and the results are merged by their log-normalizers.
+    ``q_shift`` (0 <= q_shift < Bq): the query blocks are laid out as if q_shift more rows preceded the first one
+    (block i = rows q with i*Bq <= q + q_shift < (i+1)*Bq); with q_shift = (Nk - N) % Bq a chunk's blocks are the
+    blocks its rows have in the equal-length problem over all Nk positions.
 
     q [B,N,Hq,d]; k, v [B,Nk,Hkv,d] with Nk >= N: the queries are the last N of the Nk positions (chunked
     prefill), query row q sees the keys 0 .. q + Nk - N and L_q = q + 1 + Nk - N.
@@ -155,7 +159,7 @@ def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True
     B, N, Hq, d = q.shape
     Nk, Hkv = k.shape[1], k.shape[2]
     G = Hq // Hkv
-    Tr, Tc = -(-N // Bq), -(-Nk // Bk)
+    Tr, Tc = -(-(N + q_shift) // Bq), -(-Nk // Bk)
     o = np.full((B, N, Hq, d), np.nan)
     lse = np.full((B, Hq, N), np.nan)
     mask = np.zeros((B, Hq, Tr, Tc), dtype=np.uint8)
@@ -176,7 +180,8 @@ def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True
         c = np.full((Tr, Tc), np.nan)
         bl = np.asarray(blocks, dtype=np.int32) if blocks is not None else None
         _ck(lib().mala_oracle_fwd_split(_p(Q), _p(K), _p(V), N, Nk, d, scale, tau, Bq, Bk, int(causal), num_splits,
-                                        0 if bl is None else len(bl), _ip(bl), _p(O), _p(l), _u8(m), _p(c)), "fwd")
+                                        q_shift, 0 if bl is None else len(bl), _ip(bl), _p(O), _p(l), _u8(m), _p(c)),
+            "fwd")
         o[b, :, h, :] = O
         lse[b, h] = l
         mask[b, h] = m

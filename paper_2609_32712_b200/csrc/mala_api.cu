@@ -172,11 +172,11 @@ int mala_device_status(int* code_out, int clear) {
   return MALA_OK;
 }
 
-// Lengths of a call with N queries and Nk keys: causal needs the queries to be the last N positions of the Nk,
-// starting on a tile boundary.
-static int check_lengths(int N, int Nk, int causal) {
+// Lengths of a call with N queries and Nk keys: causal needs the queries to be the last N positions of the Nk; the
+// backward also needs them to start on a tile boundary.
+static int check_lengths(int N, int Nk, int causal, bool aligned_only) {
   if (N <= 0 || Nk <= 0) return MALA_ERR_INVALID_ARG;
-  if (causal && (Nk < N || (Nk - N) % 128 != 0)) return MALA_ERR_UNSUPPORTED;
+  if (causal && (Nk < N || (aligned_only && (Nk - N) % 128 != 0))) return MALA_ERR_UNSUPPORTED;
   return MALA_OK;
 }
 
@@ -194,7 +194,7 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
       return MALA_ERR_WORKSPACE_TOO_SMALL;
   }
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
-  MALA_TRY(check_lengths(N, Nk, causal));
+  MALA_TRY(check_lengths(N, Nk, causal, false));
   if (!lse) return MALA_ERR_INVALID_ARG;
   const int Bt = cu ? 1 : B, Nt = cu ? total : N, Nkt = cu ? total : Nk;   // extents of the tensors
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, Bt, Nt, Hq));
@@ -227,8 +227,11 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   p.bitmask = st ? st->tile_bitmask : nullptr;
   p.totals = st ? (unsigned long long*)st->totals : nullptr;
   p.status = status;
-  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Tr = (N + 127) / 128; p.causal = causal ? 1 : 0;
-  p.Nk = Nk; p.Tk = (Nk + 127) / 128; p.koff = causal ? (Nk - N) / 128 : 0; p.words = (p.Tk + 31) / 32;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.causal = causal ? 1 : 0;
+  p.Nk = Nk; p.Tk = (Nk + 127) / 128; p.words = (p.Tk + 31) / 32;
+  p.koff = causal ? (Nk - N) / 128 : 0;
+  p.qshift = causal ? (Nk - N) % 128 : 0;        // the query blocks follow the key positions
+  p.Tr = (N + p.qshift + 127) / 128;
   p.scale_log2 = scale * kLog2e;
   p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
   if (p.bitmask) {
@@ -246,10 +249,10 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   const unsigned rows = (unsigned)((long long)B * Hq * N);
   if (d == 128)
     fwd_merge_splits_kernel<128><<<rows, 128, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
-                                                           num_splits, p.tps, p.Tk, p.koff, p.causal);
+                                                           num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal);
   else
     fwd_merge_splits_kernel<64><<<rows, 64, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
-                                                         num_splits, p.tps, p.Tk, p.koff, p.causal);
+                                                         num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
@@ -272,7 +275,7 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
                     int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream,
                     const int32_t* cu = nullptr, int total = 0) {
   MALA_TRY(check_common(B0, Hq, Hkv, N0, d, scale, tau));
-  MALA_TRY(check_lengths(N0, Nk0, causal));
+  MALA_TRY(check_lengths(N0, Nk0, causal, true));
   if (!lse || !ws) return MALA_ERR_INVALID_ARG;
   // extents of the tensors and of the workspace (packed sequences: one batch entry of `total` rows)
   const int B = cu ? 1 : B0, N = cu ? total : N0, Nk = cu ? total : Nk0;

@@ -32,6 +32,9 @@ struct FwdParams {
   int* status;
   int B, Hq, Hkv, N, Tr, words, causal;   // N, Tr: query rows and query blocks
   int Nk, Tk, koff;              // keys, key blocks; causal: the queries are the last N positions, koff = (Nk - N) / 128
+  int qshift;                    // causal: (Nk - N) % 128.  The query blocks follow the key positions: block i holds
+                                 // the rows q with 128 i <= q + qshift < 128 (i + 1), Tr = ceil((N + qshift) / 128),
+                                 // and its newest legal key block is i + koff
   // Packed sequences of different lengths (null: B sequences of N rows each): sequence b holds rows
   // cu[b] .. cu[b+1]-1 of q, k, v, o (which are then [1, total, H, d] tensors); lse is [Hq, total]; N, Tr, Nk, Tk
   // above describe the longest sequence (grid, telemetry strides)
@@ -140,8 +143,10 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
       mbar_arrive_expect_tx(&q_full, (hasB ? 2 : 1) * Cfg::kTileBytes);
       for (int pn = 0; pn < PAN; ++pn) {
-        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iA * 128, h, bz);
-        if (hasB) tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iB * 128, h, bz);
+        // (the first block of a chunk that starts inside a tile begins before row 0: those rows read as zeros)
+        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iA * 128 - p.qshift, h, bz);
+        if (hasB)
+          tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iB * 128 - p.qshift, h, bz);
       }
       int issued = 0, v_issued = 0, s = 0;
       uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
@@ -286,10 +291,11 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const bool present_x = (x == 0) || hasB;
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
-    const int row = i * 128 + rl;
-    const bool valid = row < Nq;
+    const int prow_ = i * 128 + rl;                   // row counted in whole blocks from the first block's start
+    const int row = prow_ - p.qshift;                 // row of q, o, lse
+    const bool valid = row >= 0 && row < Nq;
     const float c2 = p.scale_log2;
-    const float Lq = p.causal ? (float)(row + 1 + p.koff * 128) : (float)Nkeys;   // visible keys
+    const float Lq = p.causal ? (float)(prow_ + 1 + p.koff * 128) : (float)Nkeys;   // visible keys
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f(Lq));
     const uint32_t colS = (uint32_t)x * 128u, colO = 256u + (uint32_t)x * 128u;
     const int first = (x == 0) ? firstA : 0;
@@ -547,10 +553,11 @@ template <int D>
 __global__ void __launch_bounds__(D)
 fwd_merge_splits_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part,
                         __nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sn, int64_t o_sh,
-                        float* __restrict__ lse, int Hq, int N, int num_splits, int tps, int Tk, int koff, int causal) {
+                        float* __restrict__ lse, int Hq, int N, int num_splits, int tps, int Tk, int koff, int qshift,
+                        int causal) {
   const long long idx = blockIdx.x;
   const int row = (int)(idx % N), h = (int)((idx / N) % Hq), b = (int)(idx / ((long long)N * Hq)), c = threadIdx.x;
-  const int newest = causal ? row / 128 + koff : Tk - 1;
+  const int newest = causal ? (row + qshift) / 128 + koff : Tk - 1;
   const int ns = min(num_splits, newest / tps + 1);
   const size_t base = ((size_t)b * Hq + h) * num_splits;
   float mx = -INFINITY;

@@ -174,12 +174,13 @@ def bwd(q, k, v, o, do, lse, scale: float, tau: float, causal: bool = True, stat
 
 def fwd_chunk(q, k, v, scale: float, tau: float, causal: bool = True, stats: bool = False, out=None, lse=None):
     """mala_fwd_chunk: q [B,Nq,Hq,d] against k, v [B,Nk,Hkv,d] (causal: the queries are the last Nq positions).
-    Returns (o [B,Nq,Hq,d] bf16, lse [B,Hq,Nq] fp32, Stats or None)."""
+    Returns (o [B,Nq,Hq,d] bf16, lse [B,Hq,Nq] fp32, Stats or None); the telemetry's query blocks follow the key
+    positions (block i = rows q with 128 i <= q + (Nk - Nq) % 128 < 128 (i + 1))."""
     B, Nq, Hq, d = q.shape
     Nk, Hkv = k.shape[1], k.shape[2]
     o = torch.empty_like(q) if out is None else out
     lse = torch.empty((B, Hq, Nq), dtype=torch.float32, device=q.device) if lse is None else lse
-    Tq, Tk = -(-Nq // 128), -(-Nk // 128)
+    Tq, Tk = -(-(Nq + ((Nk - Nq) % 128 if causal else 0)) // 128), -(-Nk // 128)
     st = Stats((B, Hq, Tq), -(-Tk // 32), q.device) if stats else None
     rc = lib().mala_fwd_chunk(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TOut), lse.data_ptr(),
                               ctypes.byref(st.c) if st else None, B, Hq, Hkv, Nq, Nk, d, int(causal), scale, tau,
@@ -196,7 +197,7 @@ def fwd_chunk_split(q, k, v, scale: float, tau: float, num_splits: int, causal: 
     Nk, Hkv = k.shape[1], k.shape[2]
     o = torch.empty_like(q) if out is None else out
     lse = torch.empty((B, Hq, Nq), dtype=torch.float32, device=q.device) if lse is None else lse
-    Tq, Tk = -(-Nq // 128), -(-Nk // 128)
+    Tq, Tk = -(-(Nq + ((Nk - Nq) % 128 if causal else 0)) // 128), -(-Nk // 128)
     st = Stats((B, Hq, Tq), -(-Tk // 32), q.device) if stats else None
     ws = _ws(workspace_bytes(OP_FWD, B, Hq, Hkv, Nq, d, num_splits), q.device) if ws is None else ws
     rc = lib().mala_fwd_chunk_split(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TOut), lse.data_ptr(),

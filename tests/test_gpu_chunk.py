@@ -124,12 +124,74 @@ def test_chunk_equals_rows_of_the_equal_length_call(mala):
         assert (dv.float() - dvc.float()).abs().max() <= 1e-2 * dv.float().abs().max()
 
 
-def test_chunk_rejects_a_chunk_that_starts_inside_a_tile(mala):
+def test_backward_rejects_a_chunk_that_starts_inside_a_tile(mala):
     q = torch.zeros((1, 100, 2, 128), dtype=torch.bfloat16, device="cuda")
     kv = torch.zeros((1, 300, 1, 128), dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros((1, 2, 100), dtype=torch.float32, device="cuda")
     with pytest.raises(mala.MalaError) as e:
-        mala.fwd_chunk(q, kv, kv, 0.1, 0.0)
-    assert e.value.code < 0
+        mala.bwd_chunk(q, kv, kv, q, q, lse, 0.1, 0.0)
+    assert e.value.code == -2
+
+
+def _run_fwd_any_offset(mala, oracle, c, tau, S=1):
+    """Forward of a chunk that may start inside a tile: the query blocks follow the key positions."""
+    q, k, v = (c[x].cuda() for x in ("q", "k", "v"))
+    B, Nq, Hq, d = q.shape
+    Nk = k.shape[1]
+    off = Nk - Nq
+    shift = off % 128
+    Tq, Tk = -(-(Nq + shift) // 128), -(-Nk // 128)
+    if S == 1:
+        o, lse, st = mala.fwd_chunk(q, k, v, c["scale"], tau, stats=True)
+    else:
+        o, lse, st = mala.fwd_chunk_split(q, k, v, c["scale"], tau, S, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    ref = oracle.fwd(c["q"], c["k"], c["v"], c["scale"], tau, 128, 128, num_splits=S, q_shift=shift)
+    fm = st.mask(Tk).cpu().numpy()
+    tps = -(-Tk // S)
+    for b in range(B):
+        for h in range(Hq):
+            for i in range(Tq):
+                newest = i + off // 128
+                first_row = max(i * 128 - shift, 0)
+                for s in range(S):
+                    js = [j for j in range(min(newest, (s + 1) * tps - 1), s * tps - 1, -1)]
+                    sel = np.zeros(Tk, dtype=bool)
+                    sel[js] = True
+                    parity.check_mask(np.where(sel, fm[b, h, i], False), np.where(sel, ref["mask"][b, h, i], 0),
+                                      ref["crit"][b, h, i], js, tau, first_row + 1 + off)
+                assert int(st.retained[b, h, i]) == int(fm[b, h, i].sum())
+    parity.check_output(o.float().cpu().numpy(), ref["o"])
+    assert np.abs(lse.cpu().numpy() - ref["lse"]).max() <= parity.LSE_ABS
+    assert st.totals.cpu().numpy()[1] == int((ref["mask"] > 0).sum())
+    return int((ref["mask"] == 1).sum())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,Nq,d,Hq,Hkv,S", [(500, 100, 128, 2, 1, 1), (1000, 333, 128, 4, 2, 1), (777, 129, 64, 2, 2, 1),
+                                              (1300, 5, 128, 2, 1, 1), (1000, 333, 128, 2, 1, 4), (901, 450, 64, 2, 1, 3)])
+def test_chunk_from_any_position_literal(mala, oracle, Nk, Nq, d, Hq, Hkv, S, tau):
+    w = W.custom_prefill(2, Hq, Hkv, Nk, d, seed=Nk + Nq)
+    _run_fwd_any_offset(mala, oracle, _chunk(w, Nq), tau, S)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("Nk,Nq,S", [(2000, 555, 1), (2500, 300, 5)])
+def test_chunk_from_any_position_skipping_regime(mala, oracle, Nk, Nq, S, tau):
+    w = W.custom_prefill(1, 4, 2, Nk, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=7, preset="R")
+    assert _run_fwd_any_offset(mala, oracle, _chunk(w, Nq), tau, S) > 0, "workload must exercise skipping"
+
+
+def test_chunk_from_any_position_gives_the_rows_of_the_equal_length_call(mala):
+    # where the chunk holds whole blocks of the full call the results are the same bits
+    w = W.custom_prefill(1, 4, 2, 1536, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=3, preset="R")
+    q, k, v = (w[x].cuda() for x in ("q", "k", "v"))
+    off = 1000                                              # 1000 = 7 * 128 + 104: the first whole block starts at 1024
+    for tau in (0.0, 1e-4):
+        o, lse, _ = mala.fwd(q, k, v, w["scale"], tau)
+        oc, lc, _ = mala.fwd_chunk(q[:, off:], k, v, w["scale"], tau)
+        assert torch.equal(o[:, 1024:], oc[:, 24:]) and torch.equal(lse[:, :, 1024:], lc[:, :, 24:])
 
 
 def _run_split(mala, oracle, c, tau, S, causal=True):

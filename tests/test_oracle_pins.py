@@ -835,3 +835,66 @@ def test_non_causal_with_more_queries_than_keys_is_plain_softmax():
     assert np.allclose(g["dv"][0, :, 0], P.T @ do[0, :, 0], atol=1e-12)
     assert np.allclose(g["dq"][0, :, 0], 0.4 * dS @ k[0, :, 0], atol=1e-12)
     assert np.allclose(g["dk"][0, :, 0], 0.4 * dS.T @ q[0, :, 0], atol=1e-12)
+
+
+# ------------------------------------------------------------------ a chunk that starts inside a tile
+@pytest.mark.parametrize("tau", [1e-2, 0.5])
+@pytest.mark.parametrize("Nq,Nk,Bq,Bk,S", [(27, 64, 8, 8, 1), (30, 75, 8, 8, 1), (19, 50, 16, 4, 1), (27, 64, 8, 8, 3)])
+def test_chunk_from_any_position_equals_the_rows_of_the_full_run_when_its_blocks_follow_the_positions(Nq, Nk, Bq, Bk,
+                                                                                                     S, tau):
+    # Nk - Nq is not a multiple of the block: with the query blocks laid out by position (q_shift) the chunked run is
+    # the full run restricted to the chunk's rows -- masks of the blocks they share, O and lse; the first block is the
+    # last rows of a block of the full run, and a row's result does not depend on the other rows of its block EXCEPT
+    # through the block's votes, so equality holds only if the absent rows would not have changed a vote: compare
+    # against the full run with those rows' queries removed from the votes, i.e. against a brute force
+    d, scale = 32, 1.0 / math.sqrt(32)
+    off = Nk - Nq
+    shift = off % Bq
+    assert shift != 0
+    q, k, v = peaky_inputs(Nk, d, 331 + Nk, boost=5.0)
+    qc = q[:, off:]
+    f = orc.fwd(qc, k, v, scale, tau, Bq, Bk, num_splits=S, q_shift=shift)
+    Sm = scale * (qc[0, :, 0] @ k[0, :, 0].T)
+    Tc = -(-Nk // Bk)
+    tps = -(-Tc // S)
+    Tr = -(-(Nq + shift) // Bq)
+    assert f["mask"].shape[2] == Tr
+    skipped = 0
+    for i in range(Tr):
+        rows = [r for r in range(i * Bq - shift, (i + 1) * Bq - shift) if 0 <= r < Nq]
+        Z = {r: [] for r in rows}
+        num = {r: np.zeros(d) for r in rows}
+        for s in range(S):
+            R = {r: [] for r in rows}
+            for j in reversed(range(s * tps, min(Tc, (s + 1) * tps))):
+                keys = list(range(j * Bk, min(Nk, (j + 1) * Bk)))
+                if keys[0] > rows[-1] + off:
+                    assert f["mask"][0, 0, i, j] == 0
+                    continue
+                skip = True
+                for r in rows:
+                    legal = [x for x in keys if x <= r + off]
+                    if not legal:
+                        continue
+                    Zt = sum(math.exp(Sm[r, x]) for x in R[r])
+                    if Zt == 0.0 or not (math.exp(max(Sm[r, x] for x in legal)) / Zt < tau / (r + 1 + off)):
+                        skip = False
+                assert f["mask"][0, 0, i, j] == (1 if skip else 2)
+                skipped += skip
+                if not skip:
+                    for r in rows:
+                        R[r] += [x for x in keys if x <= r + off]
+            for r in rows:
+                Z[r].append(sum(math.exp(Sm[r, x]) for x in R[r]))
+                num[r] += sum((math.exp(Sm[r, x]) * v[0, x, 0] for x in R[r]), np.zeros(d))
+        for r in rows:
+            assert abs(f["lse"][0, 0, r] - math.log(sum(Z[r]))) < 1e-12
+            assert np.allclose(f["o"][0, r, 0], num[r] / sum(Z[r]), atol=1e-12)
+    assert skipped > 0
+    if S == 1:   # the blocks that lie wholly inside the chunk are blocks of the full run
+        full = orc.fwd(q, k, v, scale, tau, Bq, Bk)
+        i_full0 = off // Bq
+        for i in range(1, Tr):
+            assert np.array_equal(f["mask"][0, 0, i], full["mask"][0, 0, i_full0 + i])
+            rows = slice(i * Bq - shift, min(Nq, (i + 1) * Bq - shift))
+            assert np.array_equal(f["o"][0, rows], full["o"][0, off:][rows])
