@@ -493,7 +493,7 @@ def main():
     ach = bwd_exec / (bwd_ms * 1e-3) / 1e12
     # DRAM bytes of one mala_bwd_kernel launch from the committed ncu capture of the same workload
     # (profiles/mala_bwd_kernel_cfg3_literal_tau1e-4.txt: dram__bytes.sum.per_second x gpu__time_duration.sum)
-    traffic = {("cfg3", "literal", 1e-4): 101.539102e9 * 21.446112e-3}.get((args.workload, args.preset, tau))
+    traffic = {("cfg3", "literal", 1e-4): 101.735456e9 * 21.403424e-3}.get((args.workload, args.preset, tau))
     roofline = {"bound": "tensor", "kernel": "mala_bwd_kernel", "achieved": ach, "peak": peaks["tflops_sustained"],
                 "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": traffic,
                 "peak_source": f"{peaks['source']} (bf16 matmul, sustained)",
