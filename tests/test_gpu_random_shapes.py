@@ -55,6 +55,9 @@ def test_random_cases(mala, oracle, seed):
                 TC._run(mala, oracle, c, tau, causal=causal)
             else:
                 TC._run_split(mala, oracle, c, tau, S, causal=causal)
+                if causal and Nk > Nq + 1:   # the forward also from a position inside a tile, unsplit and split
+                    c2 = TC._chunk(w, Nq + rng.randint(1, min(127, Nk - Nq)))
+                    TC._run_fwd_any_offset(mala, oracle, c2, tau, rng.choice([1, S]))
         elif kind == "varlen":
             Hq, Hkv = _heads(rng)
             lens = [rng.randint(1, 600) for _ in range(rng.randint(1, 4))]
