@@ -684,6 +684,17 @@ def main():
                                  "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
                 row["paged_256"] = pg
                 del kp, vp, bt
+                # ... and in 16-key pages (a tile is then put together from eight pages)
+                kp, vp, bt, _ = W.paginate(kc, vc, 16, seed=7)
+                pg = {}
+                for label, t_ in (("mala", tau), ("dense", 0.0)):
+                    us = 1e3 * time_cuda(lambda: mala.decode_paged(qd, kp, vp, bt, None, wd["scale"], t_, dcfg.num_splits,
+                                                                    ws=wsd, out=od, want_lse=False), 25, 100)
+                    need = row[label]["needed_gb"] * 1e9
+                    pg[label] = {"us": us, "achieved_gbs": need / (us * 1e-6) / 1e9,
+                                 "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+                row["paged_16"] = pg
+                del kp, vp, bt
             detail[f"cfg5_{preset}"] = row
             del wd, qd, kc, vc, wsd
             torch.cuda.empty_cache()

@@ -163,7 +163,8 @@ int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o,
  * q, o [B,Sq,Hq,d], Sq >= 1 new tokens per sequence whose keys are the last Sq of the sequence's seqlens[b] keys
  * (Sq * Hq/Hkv <= 16; Sq = 1: sn of q and o is ignored); lse_opt fp32 [B,Sq,Hq] or NULL.
  * kpages, vpages [num_pages, page_size, Hkv, d] (sb = page stride, sn = key stride, sh = head stride);
- * page_size must be a multiple of 128 (MALA_ERR_UNSUPPORTED otherwise).  block_table: device int32
+ * page_size is a multiple of 128, or 8, 16, 32 or 64 (a 128-key tile is then fetched as several copies, which costs
+ * throughput; MALA_ERR_UNSUPPORTED for any other size).  block_table: device int32
  * [B, max_pages_per_seq]; keys page_size*x .. page_size*(x+1)-1 of sequence b live in page block_table[b][x]
  * (entries beyond the sequence's length are never read; an entry outside [0, num_pages) reads zeros).
  * seqlens: device int32 [B], keys held by each sequence, clamped to [0, max_pages_per_seq*page_size], or NULL

@@ -388,7 +388,9 @@ int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_
                       int Hkv, int num_pages, int page_size, int max_pages_per_seq, int Sq, int d, float scale,
                       float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
   if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || Sq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
-  if (page_size % 128 != 0 || (long long)max_pages_per_seq * page_size > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
+  if (page_size < 8 || (page_size % 128 != 0 && 128 % page_size != 0) ||
+      (long long)max_pages_per_seq * page_size > 0x7fffffffLL)
+    return MALA_ERR_UNSUPPORTED;
   const int Nk = max_pages_per_seq * page_size;   // the longest cache a sequence can hold
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
   if (num_splits <= 0 || !ws) return MALA_ERR_INVALID_ARG;

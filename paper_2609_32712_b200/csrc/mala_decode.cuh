@@ -71,8 +71,11 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   const int G = Hq / Hkv;
   if (Sq < 1 || G * Sq > 16 || Sq > Nk) return MALA_ERR_UNSUPPORTED;
   const bool paged = pg && pg->block_table;
-  if (paged && (pg->page_size <= 0 || pg->page_size % 128 != 0 || pg->num_pages <= 0 || pg->bt_stride <= 0))
+  // pages of whole tiles, or 8, 16, 32 or 64 keys (a tile is then put together from several pages)
+  if (paged && (pg->page_size < 8 || (pg->page_size % 128 != 0 && 128 % pg->page_size != 0) || pg->num_pages <= 0 ||
+                pg->bt_stride <= 0))
     return MALA_ERR_UNSUPPORTED;
+  const int box_rows = paged && pg->page_size < 128 ? pg->page_size : 128;
   const int per = (Nk + num_splits - 1) / num_splits;
   const int tps = (per + 127) / 128;
   if ((long long)B * Hkv * num_splits > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
@@ -81,9 +84,9 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   // q [B,Sq,Hq,d]: one box of the group's G heads x Sq tokens
   if (!make_tensor_map_q_rows(&tq, q.p, B, Sq, Hq, d, q.sb, Sq > 1 ? q.sn : 0, q.sh, G) ||
       !make_tensor_map_bnhd(&tk, kc.p, paged ? pg->num_pages : B, paged ? pg->page_size : Nk, Hkv, d, kc.sb, kc.sn,
-                            kc.sh, 128) ||
+                            kc.sh, box_rows) ||
       !make_tensor_map_bnhd(&tv, vc.p, paged ? pg->num_pages : B, paged ? pg->page_size : Nk, Hkv, d, vc.sb, vc.sn,
-                            vc.sh, 128))
+                            vc.sh, box_rows))
     return MALA_ERR_TENSOR_MAP;
 
   DecParams p;
@@ -95,7 +98,9 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   p.seqlens = pg ? pg->seqlens : nullptr;
   p.block_table = paged ? pg->block_table : nullptr;
   p.bt_stride = paged ? pg->bt_stride : 0;
-  p.tpp = paged ? pg->page_size / 128 : 1;
+  p.tpp = paged && pg->page_size >= 128 ? pg->page_size / 128 : 1;
+  p.ppt = 128 / box_rows;
+  p.prows = box_rows;
   p.Sq = Sq;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Nk = Nk; p.tps = tps; p.num_splits = num_splits; p.words = (tps + 31) / 32;
   p.n_items = B * Hkv * num_splits;

@@ -42,7 +42,10 @@ struct DecParams {
   // Paged / variable-length caches (both null for one contiguous cache of Nk keys per sequence):
   const int* seqlens;            // [B] keys held by sequence b (<= Nk); L = seqlens[b] for its rows
   const int* block_table;        // [B, bt_stride] page of the tpp consecutive tiles number x*tpp .. x*tpp + tpp - 1
-  int bt_stride, tpp;            // tpp: tiles per page (page size / 128)
+  int bt_stride, tpp;            // tpp: tiles per page (page size / 128; 1 for smaller pages)
+  int ppt, prows;                // pages per tile and keys per page when a page is smaller than a tile (else 1, 128):
+                                 // a tile is then fetched as ppt copies of prows rows, block_table holds one entry
+                                 // per page
   int Sq;                        // new tokens per sequence (the last Sq positions of the cache); rows = Sq * Hq/Hkv
   int B, Hq, Hkv, Nk, tps, num_splits, words, n_items;   // Nk: longest cache the splits are laid out for
   float scale_log2, log2_tau;
@@ -129,7 +132,8 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       vote_bar[4], p_full[4], p_free[4], item_done[2], o_free[2], fin_bar, grp_a[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[2][4];               // [softmax group][vote ring]
-  __shared__ int v_row[8], v_outer[8];     // TMA coordinates of the V tile of tile g (ring; written by the producer)
+  __shared__ int v_row[8], v_outer[8];     // TMA coordinates of the V tile of tile g (ring; written by the producer;
+                                           // pages smaller than a tile: sequence and key block instead)
   __shared__ __align__(16) float xch_max[2][2][4][8], xch_sum[2][2][4][8];   // [buffer][group][warp][row]: per-tile exchange
   __shared__ int early_exit;
 
@@ -180,7 +184,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     T = hi > lo ? (hi - lo + 127) / 128 : 0;
     j0 = lo / 128 + T - 1;
   };
-  // TMA coordinates (key row, outermost index) of key block jt of sequence b
+  // TMA coordinates (key row, outermost index) of key block jt of sequence b, one copy per tile
   auto tile_coord = [&](int b, int jt, int& row, int& outer) {
     if (p.block_table) {
       const int pg = jt / p.tpp;
@@ -189,6 +193,19 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     } else {
       outer = b;
       row = jt * 128;
+    }
+  };
+  // Pages smaller than a tile (ppt > 1): the tile is put together from ppt copies of prows rows, copy c from page
+  // jt * ppt + c of the sequence (a table entry past the last page reads as "no page": zeros).
+  auto small_page = [&](int b, int jt, int c) -> int {
+    const int pg = jt * p.ppt + c;
+    return pg < p.bt_stride ? __ldg(p.block_table + (size_t)b * p.bt_stride + pg) : -1;
+  };
+  auto load_tile_small = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int b, int jt, int hkv) {
+    for (int c = 0; c < p.ppt; ++c) {
+      const int outer = small_page(b, jt, c);
+#pragma unroll
+      for (int pn = 0; pn < PAN; ++pn) tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, outer);
     }
   };
 
@@ -213,8 +230,9 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         for (int pn = 0; pn < PAN; ++pn)
           tma_load_4d(sQ + ip * DecCfg::kQBytes + pn * 2048, &tmQ, &q_full[ip], pn * 64, hkv * G, 0, b);
         for (int t = 0; t < T && ok; ++t, ++g) {
-          int row, outer;
-          tile_coord(b, j0 - t, row, outer);     // (a page lookup is in flight while the slot is waited for)
+          const bool small = p.ppt > 1;
+          int row = j0 - t, outer = b;           // (pages smaller than a tile: looked up copy by copy)
+          if (!small) tile_coord(b, j0 - t, row, outer);   // (a page lookup is in flight while the slot is waited for)
           ok = mbar_wait(&k_empty[ks], kpar, status);
           if (!ok) break;
           // The UMMA warp requests V of tile g from these coordinates after the vote.  It cannot be more than six
@@ -222,17 +240,21 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           // and it sees the two stores through the K tile's barrier.
           if (!kDense) { v_row[g & 7] = row; v_outer[g & 7] = outer; }
           mbar_arrive_expect_tx(&k_full[ks], kTileTx);
+          if (small) load_tile_small(sK + ks * TB, &tmK, &k_full[ks], b, j0 - t, hkv);
+          else
 #pragma unroll
-          for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sK + ks * TB + pn * 16384, &tmK, &k_full[ks], pn * 64, row, hkv, outer);
+            for (int pn = 0; pn < PAN; ++pn)
+              tma_load_4d(sK + ks * TB + pn * 16384, &tmK, &k_full[ks], pn * 64, row, hkv, outer);
           if (++ks == KS) { ks = 0; kpar ^= 1; }
           if (kDense) {   // every tile is retained: V follows K
             ok = mbar_wait(&v_empty[vs], vpar, status);
             if (!ok) break;
             mbar_arrive_expect_tx(&v_full[vs], kTileTx);
+            if (small) load_tile_small(sV + vs * TB, &tmV, &v_full[vs], b, j0 - t, hkv);
+            else
 #pragma unroll
-            for (int pn = 0; pn < PAN; ++pn)
-              tma_load_4d(sV + vs * TB + pn * 16384, &tmV, &v_full[vs], pn * 64, row, hkv, outer);
+              for (int pn = 0; pn < PAN; ++pn)
+                tma_load_4d(sV + vs * TB + pn * 16384, &tmV, &v_full[vs], pn * 64, row, hkv, outer);
             if (++vs == VS) { vs = 0; vpar ^= 1; }
           }
         }
@@ -322,9 +344,11 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
               if (leader) {
                 const int row = *(volatile int*)&v_row[cv.g & 7], outer = *(volatile int*)&v_outer[cv.g & 7];
                 mbar_arrive_expect_tx(&v_full[vi], kTileTx);
+                if (p.ppt > 1) load_tile_small(sV + vi * TB, &tmV, &v_full[vi], outer, row, cv.hkv);
+                else
 #pragma unroll
-                for (int pn = 0; pn < PAN; ++pn)
-                  tma_load_4d(sV + vi * TB + pn * 16384, &tmV, &v_full[vi], pn * 64, row, cv.hkv, outer);
+                  for (int pn = 0; pn < PAN; ++pn)
+                    tma_load_4d(sV + vi * TB + pn * 16384, &tmV, &v_full[vi], pn * 64, row, cv.hkv, outer);
               }
               __syncwarp();
               if (++vi == VS) { vi = 0; vipar ^= 1; }

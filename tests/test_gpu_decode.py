@@ -161,9 +161,21 @@ def test_decode_paged_identity_table_equals_contiguous_call(mala):
         assert torch.equal(s1.retained, s2.retained)
 
 
-def test_decode_paged_rejects_pages_that_are_not_whole_tiles(mala):
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv,page,lens", [
+    (1024, 4, 8, 2, 16, [1024, 500, 17]),              # 16-key pages: eight copies per tile
+    (2048, 4, 4, 1, 64, [2048, 1000, 129, 0]),
+    (1520, 3, 4, 2, 32, [1520, 33]),                   # the positions end inside a tile: table entries past the last page
+    (4096, 16, 16, 2, 8, [4096, 2047]),
+])
+def test_decode_paged_with_pages_smaller_than_a_tile(mala, oracle, Nk, S, Hq, Hkv, page, lens, tau):
+    w = W.custom_decode(len(lens), Hq, Hkv, Nk, 128, S, group_types=["diffuse", "peaked"], seed=Nk + page, preset="D")
+    _run_paged(mala, oracle, w, tau, S, page, lens, seed=page)
+
+
+def test_decode_paged_rejects_pages_that_do_not_tile(mala):
     q = torch.zeros((1, 1, 4, 128), dtype=torch.bfloat16, device="cuda")
-    pages = torch.zeros((4, 64, 1, 128), dtype=torch.bfloat16, device="cuda")
+    pages = torch.zeros((4, 48, 1, 128), dtype=torch.bfloat16, device="cuda")
     bt = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
     with pytest.raises(mala.MalaError) as e:
         mala.decode_paged(q, pages, pages, bt, None, 0.1, 0.0, 1)

@@ -103,10 +103,11 @@ def test_argument_validation_codes_of_the_general_shape_calls(mala):
     dm = lambda Sq, Hq=4, Nk=256: L.mala_decode_multi(tin(), tin(), tin(), tout(), None, None, 1, Hq, 1, Nk, Sq, 128, 0.1,
                                                       1e-4, 2, base, 1 << 20, None)
     assert dm(0) == -1 and dm(5) == -2 and dm(2, Hq=16) == -2 and dm(4, Nk=3) == -2
-    # paged decode: pages of whole tiles, a block table
+    # paged decode: pages of whole tiles or of 8, 16, 32, 64 keys, a block table
     dp = lambda page, bt=base, Sq=1: L.mala_decode_paged(tin(), tin(), tin(), bt, None, tout(), None, None, 1, 4, 1, 8,
                                                          page, 4, Sq, 128, 0.1, 1e-4, 2, base, 1 << 20, None)
-    assert dp(64) == -2 and dp(200) == -2 and dp(0) == -1 and dp(128, bt=None) == -1 and dp(128, bt=base + 1) == -3
+    assert dp(48) == -2 and dp(200) == -2 and dp(4) == -2 and dp(0) == -1 and dp(128, bt=None) == -1
+    assert dp(128, bt=base + 1) == -3 and dp(16, bt=base + 1) == -3
     assert dp(128, Sq=0) == -1 and dp(128, Sq=5) == -2
     # workspace of a decode step with several tokens: as for that many more sequences
     assert mala.workspace_bytes(mala.OP_DECODE, 8 * 4, 32, 8, 131072, 128, 128) == 4 * mala.workspace_bytes(
