@@ -136,6 +136,19 @@ int mala_bwd_varlen(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
                     int Hq, int Hkv, int total, int max_seqlen, int d, int causal, float scale, float tau, void* ws,
                     size_t ws_bytes, void* cuda_stream);
 
+/* Algorithm 1 on B packed sequences each of which has more keys than queries -- a batch of prefill chunks behind
+ * cached prefixes.  q, o [1,total_q,Hq,d] with sequence b in rows cu_seqlens_q[b] .. cu_seqlens_q[b+1]-1; k, v
+ * [1,total_k,Hkv,d] with its keys in rows cu_seqlens_k[b] .. cu_seqlens_k[b+1]-1 (both device int32 [B+1]).  Every
+ * sequence is treated exactly as a mala_fwd_chunk call on its own rows: causal != 0 puts its queries at its last
+ * positions (it must not have more queries than keys: such a sequence is left untouched), its query blocks follow its
+ * key positions, L_q is the number of keys the row sees; causal == 0: every key of the sequence legal, L = its number
+ * of keys.  max_seqlen_q / max_seqlen_k >= every length.  lse fp32 [Hq,total_q].  Telemetry as for mala_fwd_chunk
+ * with Tq = ceil((max_seqlen_q + 127) / 128) and ceil(max_seqlen_k / 128) key blocks. */
+int mala_fwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,
+                           mala_tout o, float* lse, const mala_stats* st, int B, int Hq, int Hkv, int total_q,
+                           int total_k, int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau,
+                           void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Split-KV decode of one new token per sequence ("Fused decoding execution").  q [B,1,Hq,d] (sn is
  * ignored); kcache, vcache [B,Nk,Hkv,d], the newest token's key/value included; o [B,1,Hq,d];
  * lse_opt fp32 [B,Hq] or NULL.  The Hq/Hkv query heads of one KV head are the rows of one tile; the

@@ -184,7 +184,7 @@ static int check_lengths(int N, int Nk, int causal, bool aligned_only) {
 static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
                     int Hkv, int N, int Nk, int d, int causal, float scale, float tau, void* cuda_stream,
                     const int32_t* cu = nullptr, int total = 0, int num_splits = 1, void* ws = nullptr,
-                    size_t ws_bytes = 0) {
+                    size_t ws_bytes = 0, const int32_t* cu_k = nullptr, int total_k = 0) {
   if (num_splits < 1) return MALA_ERR_INVALID_ARG;
   if (num_splits > 1) {
     if (cu || num_splits > 65535 || (long long)B * num_splits > 65535) return MALA_ERR_UNSUPPORTED;
@@ -196,7 +196,7 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
   MALA_TRY(check_lengths(N, Nk, causal, false));
   if (!lse) return MALA_ERR_INVALID_ARG;
-  const int Bt = cu ? 1 : B, Nt = cu ? total : N, Nkt = cu ? total : Nk;   // extents of the tensors
+  const int Bt = cu ? 1 : B, Nt = cu ? total : N, Nkt = cu ? (cu_k ? total_k : total) : Nk;   // extents of the tensors
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, Bt, Nt, Hq));
   MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, Bt, Nkt, Hkv));
   MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, Bt, Nkt, Hkv));
@@ -214,7 +214,7 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
     return MALA_ERR_TENSOR_MAP;
 
   FwdParams p;
-  p.cu = cu; p.total = total;
+  p.cu = cu; p.total = total; p.cu_k = cu_k;
   p.num_splits = num_splits;
   p.tps = ((Nk + 127) / 128 + num_splits - 1) / num_splits;
   p.o_part = num_splits > 1 ? (float*)ws : nullptr;
@@ -232,6 +232,10 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   p.koff = causal ? (Nk - N) / 128 : 0;
   p.qshift = causal ? (Nk - N) % 128 : 0;        // the query blocks follow the key positions
   p.Tr = (N + p.qshift + 127) / 128;
+  if (cu_k) {   // per sequence on the device; the grid and the telemetry are laid out for the longest ones
+    p.koff = 0; p.qshift = 0;
+    p.Tr = (N + 127 + 127) / 128;
+  }
   p.scale_log2 = scale * kLog2e;
   p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
   if (p.bitmask) {
@@ -332,6 +336,18 @@ int mala_fwd_varlen(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu_seqlen
   MALA_TRY(check_packed(cu_seqlens, B, total, max_seqlen));
   return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau, cuda_stream,
                   cu_seqlens, total);
+}
+
+int mala_fwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,
+                           mala_tout o, float* lse, const mala_stats* st, int B, int Hq, int Hkv, int total_q,
+                           int total_k, int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau,
+                           void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  MALA_TRY(check_packed(cu_seqlens_q, B, total_q, max_seqlen_q));
+  MALA_TRY(check_packed(cu_seqlens_k, B, total_k, max_seqlen_k));
+  if (causal && max_seqlen_k < max_seqlen_q) return MALA_ERR_UNSUPPORTED;
+  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen_q, max_seqlen_k, d, causal, scale, tau, cuda_stream,
+                  cu_seqlens_q, total_q, 1, nullptr, 0, cu_seqlens_k, total_k);
 }
 
 int mala_bwd_varlen(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,

@@ -40,6 +40,9 @@ struct FwdParams {
   // above describe the longest sequence (grid, telemetry strides)
   const int* cu;
   int total;
+  const int* cu_k;               // packed sequences whose keys are longer than their queries (a cached prefix): the keys
+                                 // of sequence b are rows cu_k[b] .. cu_k[b+1]-1 of k, v; its queries are the last
+                                 // positions (null: keys as queries)
   // Key range cut into num_splits ranges of tps key blocks (num_splits > 1): grid z = b * num_splits + split; a CTA
   // runs its blocks on the key blocks of its range only and writes the normalised fp32 result and the
   // log-normalizer of the range; a merge kernel combines the ranges.
@@ -84,20 +87,24 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int sp = p.num_splits > 1 ? (int)blockIdx.z % p.num_splits : 0;
   const int b = p.num_splits > 1 ? (int)blockIdx.z / p.num_splits : (int)blockIdx.z;
   const int h = blockIdx.y, hkv = h / G;
-  // this sequence: first row in the tensors, rows, blocks (packed sequences: equal query and key lengths)
+  // this sequence: first rows in the tensors, rows, keys, blocks
   const int row0 = p.cu ? __ldg(p.cu + b) : 0;
   const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
-  const int Nkeys = p.cu ? Nq : p.Nk;
-  const int Tr = p.cu ? (Nq + 127) / 128 : p.Tr;
-  const int Tk = p.cu ? Tr : p.Tk;
+  const int krow0 = p.cu_k ? __ldg(p.cu_k + b) : row0;
+  const int Nkeys = p.cu_k ? __ldg(p.cu_k + b + 1) - krow0 : (p.cu ? Nq : p.Nk);
+  if (p.cu_k && p.causal && Nkeys < Nq) return;       // (not defined: more queries than keys)
+  const int koff = p.cu_k ? (p.causal ? (Nkeys - Nq) / 128 : 0) : p.koff;
+  const int qshift = p.cu_k ? (p.causal ? (Nkeys - Nq) % 128 : 0) : p.qshift;
+  const int Tr = p.cu ? (Nq + qshift + 127) / 128 : p.Tr;
+  const int Tk = p.cu ? (Nkeys + 127) / 128 : p.Tk;
   const int bz = p.cu ? 0 : b;                        // outermost TMA coordinate
   const int npairs = (Tr + 1) / 2;
   if ((int)blockIdx.x >= npairs) return;             // (a sequence shorter than the longest one)
   const int c = npairs - 1 - (int)blockIdx.x;        // longest pairs first
   int iA = 2 * c, iB = 2 * c + 1;
   bool hasB = iB < Tr;
-  int dA = p.causal ? iA + p.koff : Tk - 1;          // newest key block with a legal key, per block
-  const int dB = p.causal ? iB + p.koff : Tk - 1;
+  int dA = p.causal ? iA + koff : Tk - 1;            // newest key block with a legal key, per block
+  const int dB = p.causal ? iB + koff : Tk - 1;
   int jlo = 0, jhi = Tk - 1;                         // key blocks of this CTA
   if (p.num_splits > 1) {
     jlo = sp * p.tps;
@@ -144,9 +151,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_arrive_expect_tx(&q_full, (hasB ? 2 : 1) * Cfg::kTileBytes);
       for (int pn = 0; pn < PAN; ++pn) {
         // (the first block of a chunk that starts inside a tile begins before row 0: those rows read as zeros)
-        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iA * 128 - p.qshift, h, bz);
+        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iA * 128 - qshift, h, bz);
         if (hasB)
-          tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iB * 128 - p.qshift, h, bz);
+          tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iB * 128 - qshift, h, bz);
       }
       int issued = 0, v_issued = 0, s = 0;
       uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
@@ -156,7 +163,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, row0 + (j0 - u) * 128, hkv, bz);
+          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, krow0 + (j0 - u) * 128, hkv, bz);
         issued = u + 1;
         if (++s == KS) { s = 0; par ^= 1; }
         if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
@@ -164,7 +171,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (!ok) break;
           mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
           for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, row0 + (j0 - u) * 128, hkv, bz);
+            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow0 + (j0 - u) * 128, hkv, bz);
           v_issued = u + 1;
         }
       }
@@ -250,7 +257,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             if (leader) {
               mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
               for (int pn = 0; pn < PAN; ++pn)
-                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, row0 + (j0 - u) * 128, hkv, bz);
+                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, krow0 + (j0 - u) * 128, hkv, bz);
             }
             __syncwarp();
           }
@@ -292,10 +299,10 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const int prow_ = i * 128 + rl;                   // row counted in whole blocks from the first block's start
-    const int row = prow_ - p.qshift;                 // row of q, o, lse
+    const int row = prow_ - qshift;                   // row of q, o, lse
     const bool valid = row >= 0 && row < Nq;
     const float c2 = p.scale_log2;
-    const float Lq = p.causal ? (float)(prow_ + 1 + p.koff * 128) : (float)Nkeys;   // visible keys
+    const float Lq = p.causal ? (float)(prow_ + 1 + koff * 128) : (float)Nkeys;   // visible keys
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f(Lq));
     const uint32_t colS = (uint32_t)x * 128u, colO = 256u + (uint32_t)x * 128u;
     const int first = (x == 0) ? firstA : 0;

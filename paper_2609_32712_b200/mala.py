@@ -62,6 +62,9 @@ def lib():
                                       vp, sz, vp]
         L.mala_bwd_varlen.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, vp, _TOut, _TOut, _TOut, ctypes.POINTER(_Stats),
                                       i, i, i, i, i, i, i, f, f, vp, sz, vp]
+        L.mala_fwd_varlen_prefix.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i,
+                                             i, i, i, f, f, vp, sz, vp]
+        L.mala_fwd_varlen_prefix.restype = i
         L.mala_fwd_varlen.restype = i
         L.mala_bwd_varlen.restype = i
         L.mala_decode.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp, sz, vp]
@@ -243,6 +246,26 @@ def fwd_varlen(q, k, v, cu_seqlens, max_seqlen: int, scale: float, tau: float, c
                                int(causal), scale, tau, None, 0, _stream())
     if rc != 0:
         raise MalaError(rc, "mala_fwd_varlen")
+    return o, lse, st
+
+
+def fwd_varlen_prefix(q, k, v, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int, scale: float, tau: float,
+                      causal: bool = True, stats: bool = False):
+    """mala_fwd_varlen_prefix: packed q [1,total_q,Hq,d] against packed k, v [1,total_k,Hkv,d], every sequence with at
+    least as many keys as queries.  Returns (o, lse [Hq,total_q], Stats or None)."""
+    one, total_q, Hq, d = q.shape
+    total_k, Hkv = k.shape[1], k.shape[2]
+    B = cu_seqlens_q.numel() - 1
+    o = torch.empty_like(q)
+    lse = torch.empty((Hq, total_q), dtype=torch.float32, device=q.device)
+    Tq, Tk = -(-(max_seqlen_q + 127) // 128), -(-max_seqlen_k // 128)
+    st = Stats((B, Hq, Tq), -(-Tk // 32), q.device) if stats else None
+    rc = lib().mala_fwd_varlen_prefix(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), cu_seqlens_q.data_ptr(),
+                                      cu_seqlens_k.data_ptr(), _view(o, _TOut), lse.data_ptr(),
+                                      ctypes.byref(st.c) if st else None, B, Hq, Hkv, total_q, total_k, max_seqlen_q,
+                                      max_seqlen_k, d, int(causal), scale, tau, None, 0, _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_fwd_varlen_prefix")
     return o, lse, st
 
 

@@ -121,3 +121,47 @@ def test_varlen_with_an_empty_sequence(mala, oracle):
             assert (a.float() - b_.float()).abs().max() <= 1e-2 * b_.float().abs().max()
     ref = oracle.fwd(ws[1]["q"], ws[1]["k"], ws[1]["v"], pk["scale"], 1e-4, 128, 128)
     parity.check_output(o3.float().cpu().numpy()[0, 200:], ref["o"][0])
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("causal", [True, False])
+def test_varlen_with_cached_prefixes(mala, oracle, tau, causal):
+    """Packed prefill chunks behind prefixes of different lengths (chunks that start inside a tile included): every
+    sequence against the oracle's chunk rule with its query blocks laid out by position."""
+    Hq, Hkv, d = 4, 2, 128
+    nk = [900, 128, 517, 300, 64]
+    nq = [260, 128, 100, 1, 64]                       # prefix lengths 640, 0, 417, 299, 0
+    ws = [W.custom_prefill(1, Hq, Hkv, n, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=60 + x, preset="R")
+          for x, n in enumerate(nk)]
+    q = torch.cat([w["q"][:, n - m:] for w, n, m in zip(ws, nk, nq)], dim=1).contiguous()
+    k = torch.cat([w["k"] for w in ws], dim=1).contiguous()
+    v = torch.cat([w["v"] for w in ws], dim=1).contiguous()
+    cq = torch.tensor(np.concatenate([[0], np.cumsum(nq)]), dtype=torch.int32)
+    ck = torch.tensor(np.concatenate([[0], np.cumsum(nk)]), dtype=torch.int32)
+    o, lse, st = mala.fwd_varlen_prefix(q.cuda(), k.cuda(), v.cuda(), cq.cuda(), ck.cuda(), max(nq), max(nk),
+                                        ws[0]["scale"], tau, causal=causal, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    Tkm = -(-max(nk) // 128)
+    fm = st.mask(Tkm).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy()[0], lse.cpu().numpy()
+    legal = skipped = 0
+    for b, (w, n, m) in enumerate(zip(ws, nk, nq)):
+        off = n - m
+        shift = off % 128 if causal else 0
+        ref = oracle.fwd(w["q"][:, n - m:], w["k"], w["v"], w["scale"], tau, 128, 128, causal=causal, q_shift=shift)
+        Tq, Tk = ref["mask"].shape[2], ref["mask"].shape[3]
+        r0 = int(cq[b])
+        for h in range(Hq):
+            for i in range(Tq):
+                order = list(range(i + off // 128, -1, -1)) if causal else list(range(Tk - 1, -1, -1))
+                parity.check_mask(fm[b, h, i, :Tk], ref["mask"][0, h, i], ref["crit"][0, h, i], order, tau,
+                                  max(i * 128 - shift, 0) + 1 + off if causal else n)
+            assert not fm[b, h, Tq:].any() and not fm[b, h, :, Tk:].any()
+        parity.check_output(o_c[r0:r0 + m], ref["o"][0])
+        assert np.abs(lse_c[:, r0:r0 + m] - ref["lse"][0]).max() <= parity.LSE_ABS
+        legal += int((ref["mask"] > 0).sum())
+        skipped += int((ref["mask"] == 1).sum())
+    assert st.totals.cpu().numpy()[1] == legal
+    if tau > 0 and causal:
+        assert skipped > 0

@@ -99,6 +99,9 @@ def test_argument_validation_codes_of_the_general_shape_calls(mala):
     fv = lambda cu, total, mx: L.mala_fwd_varlen(tin(), tin(), tin(), cu, tout(), base, None, 2, 2, 2, total, mx, 128, 1,
                                                  0.1, 1e-4, None, 0, None)
     assert fv(None, 256, 128) == -1 and fv(base, 0, 128) == -1 and fv(base, 256, 512) == -2 and fv(base + 2, 256, 128) == -3
+    fp = lambda cq, ck, mq=128, mk=256: L.mala_fwd_varlen_prefix(tin(), tin(), tin(), cq, ck, tout(), base, None, 2, 2, 2, 256,
+                                                                 512, mq, mk, 128, 1, 0.1, 1e-4, None, 0, None)
+    assert fp(None, base) == -1 and fp(base, None) == -1 and fp(base, base, mq=256, mk=128) == -2
     # several tokens per decode step: at most 16 rows per KV head, no more new tokens than keys
     dm = lambda Sq, Hq=4, Nk=256: L.mala_decode_multi(tin(), tin(), tin(), tout(), None, None, 1, Hq, 1, Nk, Sq, 128, 0.1,
                                                       1e-4, 2, base, 1 << 20, None)
