@@ -149,6 +149,19 @@ int mala_fwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu
                            int total_k, int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau,
                            void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* mala_fwd_varlen_prefix with the keys and values held in pages: a batch of prefill chunks behind prefixes that
+ * live in a paged cache (the chunks' own keys and values already written to their pages).  q, o [1,total_q,Hq,d]
+ * packed by cu_seqlens_q (device int32 [B+1]); kpages, vpages [num_pages, page_size, Hkv, d] with page_size a multiple
+ * of 128; block_table device int32 [B, max_pages_per_seq] (keys page_size*x .. of sequence b in page
+ * block_table[b][x]); seqlens_k device int32 [B], the keys sequence b holds, its queries being its last positions
+ * (a sequence with no keys, or with fewer keys than queries when causal != 0, is left untouched).  Slots of a mapped
+ * page beyond the sequence's length must hold finite numbers.  Everything else as mala_fwd_varlen_prefix with
+ * max_seqlen_k = max_pages_per_seq * page_size. */
+int mala_fwd_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* cu_seqlens_q, const int32_t* block_table,
+                   const int32_t* seqlens_k, mala_tout o, float* lse, const mala_stats* st, int B, int Hq, int Hkv,
+                   int total_q, int max_seqlen_q, int num_pages, int page_size, int max_pages_per_seq, int d, int causal,
+                   float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Split-KV decode of one new token per sequence ("Fused decoding execution").  q [B,1,Hq,d] (sn is
  * ignored); kcache, vcache [B,Nk,Hkv,d], the newest token's key/value included; o [B,1,Hq,d];
  * lse_opt fp32 [B,Hq] or NULL.  The Hq/Hkv query heads of one KV head are the rows of one tile; the

@@ -180,11 +180,19 @@ static int check_lengths(int N, int Nk, int causal, bool aligned_only) {
   return MALA_OK;
 }
 
+// Keys and values in pages for the forward: k, v are [num_pages, page_size, Hkv, d].
+struct FwdPaging {
+  const int32_t* block_table;
+  const int32_t* seqlens_k;
+  int num_pages, page_size, max_pages_per_seq;
+};
+
 // cu != null: B packed sequences in [1, total, H, d] tensors, N = Nk = the longest one.
 static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
                     int Hkv, int N, int Nk, int d, int causal, float scale, float tau, void* cuda_stream,
                     const int32_t* cu = nullptr, int total = 0, int num_splits = 1, void* ws = nullptr,
-                    size_t ws_bytes = 0, const int32_t* cu_k = nullptr, int total_k = 0) {
+                    size_t ws_bytes = 0, const int32_t* cu_k = nullptr, int total_k = 0,
+                    const FwdPaging* pg = nullptr) {
   if (num_splits < 1) return MALA_ERR_INVALID_ARG;
   if (num_splits > 1) {
     if (cu || num_splits > 65535 || (long long)B * num_splits > 65535) return MALA_ERR_UNSUPPORTED;
@@ -198,8 +206,8 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   if (!lse) return MALA_ERR_INVALID_ARG;
   const int Bt = cu ? 1 : B, Nt = cu ? total : N, Nkt = cu ? (cu_k ? total_k : total) : Nk;   // extents of the tensors
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, Bt, Nt, Hq));
-  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, Bt, Nkt, Hkv));
-  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, Bt, Nkt, Hkv));
+  MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv));
+  MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv));
   MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, Bt, Nt, Hq));
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
@@ -209,12 +217,16 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
 
   CUtensorMap tq, tk, tv;
   if (!make_tensor_map_bnhd(&tq, q.p, Bt, Nt, Hq, d, q.sb, q.sn, q.sh, 128) ||
-      !make_tensor_map_bnhd(&tk, k.p, Bt, Nkt, Hkv, d, k.sb, k.sn, k.sh, 128) ||
-      !make_tensor_map_bnhd(&tv, v.p, Bt, Nkt, Hkv, d, v.sb, v.sn, v.sh, 128))
+      !make_tensor_map_bnhd(&tk, k.p, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv, d, k.sb, k.sn, k.sh, 128) ||
+      !make_tensor_map_bnhd(&tv, v.p, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv, d, v.sb, v.sn, v.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
   FwdParams p;
   p.cu = cu; p.total = total; p.cu_k = cu_k;
+  p.block_table = pg ? pg->block_table : nullptr;
+  p.seqlens_k = pg ? pg->seqlens_k : nullptr;
+  p.bt_stride = pg ? pg->max_pages_per_seq : 0;
+  p.tpp = pg ? pg->page_size / 128 : 1;
   p.num_splits = num_splits;
   p.tps = ((Nk + 127) / 128 + num_splits - 1) / num_splits;
   p.o_part = num_splits > 1 ? (float*)ws : nullptr;
@@ -232,7 +244,7 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   p.koff = causal ? (Nk - N) / 128 : 0;
   p.qshift = causal ? (Nk - N) % 128 : 0;        // the query blocks follow the key positions
   p.Tr = (N + p.qshift + 127) / 128;
-  if (cu_k) {   // per sequence on the device; the grid and the telemetry are laid out for the longest ones
+  if (cu_k || pg) {   // per sequence on the device; the grid and the telemetry are laid out for the longest ones
     p.koff = 0; p.qshift = 0;
     p.Tr = (N + 127 + 127) / 128;
   }
@@ -348,6 +360,24 @@ int mala_fwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu
   if (causal && max_seqlen_k < max_seqlen_q) return MALA_ERR_UNSUPPORTED;
   return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen_q, max_seqlen_k, d, causal, scale, tau, cuda_stream,
                   cu_seqlens_q, total_q, 1, nullptr, 0, cu_seqlens_k, total_k);
+}
+
+int mala_fwd_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* cu_seqlens_q, const int32_t* block_table,
+                   const int32_t* seqlens_k, mala_tout o, float* lse, const mala_stats* st, int B, int Hq, int Hkv,
+                   int total_q, int max_seqlen_q, int num_pages, int page_size, int max_pages_per_seq, int d, int causal,
+                   float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  MALA_TRY(check_packed(cu_seqlens_q, B, total_q, max_seqlen_q));
+  if (!block_table || !seqlens_k || num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0) return MALA_ERR_INVALID_ARG;
+  if ((((uintptr_t)block_table) & 3) != 0 || (((uintptr_t)seqlens_k) & 3) != 0) return MALA_ERR_MISALIGNED;
+  if (page_size % 128 != 0 || (long long)max_pages_per_seq * page_size > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
+  const int max_k = max_pages_per_seq * page_size;
+  if (causal && max_k < max_seqlen_q) return MALA_ERR_UNSUPPORTED;
+  FwdPaging pg;
+  pg.block_table = block_table; pg.seqlens_k = seqlens_k; pg.num_pages = num_pages; pg.page_size = page_size;
+  pg.max_pages_per_seq = max_pages_per_seq;
+  return fwd_impl(q, kpages, vpages, o, lse, st, B, Hq, Hkv, max_seqlen_q, max_k, d, causal, scale, tau, cuda_stream,
+                  cu_seqlens_q, total_q, 1, nullptr, 0, nullptr, 0, &pg);
 }
 
 int mala_bwd_varlen(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,

@@ -40,6 +40,12 @@ struct FwdParams {
   // above describe the longest sequence (grid, telemetry strides)
   const int* cu;
   int total;
+  // Keys and values in pages (null: not paged): k, v are [num_pages, page_size, Hkv, D] with page_size a multiple of
+  // 128; keys 128 x .. of sequence b lie in page block_table[b * bt_stride + x / tpp]; it has seqlens_k[b] keys and
+  // its queries (packed, cu) are its last positions
+  const int* block_table;
+  const int* seqlens_k;
+  int bt_stride, tpp;
   const int* cu_k;               // packed sequences whose keys are longer than their queries (a cached prefix): the keys
                                  // of sequence b are rows cu_k[b] .. cu_k[b+1]-1 of k, v; its queries are the last
                                  // positions (null: keys as queries)
@@ -90,11 +96,24 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // this sequence: first rows in the tensors, rows, keys, blocks
   const int row0 = p.cu ? __ldg(p.cu + b) : 0;
   const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
+  const bool own_keys = p.cu_k || p.block_table;      // the sequence's key count differs from its query count
   const int krow0 = p.cu_k ? __ldg(p.cu_k + b) : row0;
-  const int Nkeys = p.cu_k ? __ldg(p.cu_k + b + 1) - krow0 : (p.cu ? Nq : p.Nk);
-  if (p.cu_k && p.causal && Nkeys < Nq) return;       // (not defined: more queries than keys)
-  const int koff = p.cu_k ? (p.causal ? (Nkeys - Nq) / 128 : 0) : p.koff;
-  const int qshift = p.cu_k ? (p.causal ? (Nkeys - Nq) % 128 : 0) : p.qshift;
+  const int Nkeys = p.block_table ? __ldg(p.seqlens_k + b)
+                                  : (p.cu_k ? __ldg(p.cu_k + b + 1) - krow0 : (p.cu ? Nq : p.Nk));
+  if (own_keys && (Nkeys <= 0 || (p.causal && Nkeys < Nq))) return;   // (not defined: no keys, more queries than keys)
+  const int koff = own_keys ? (p.causal ? (Nkeys - Nq) / 128 : 0) : p.koff;
+  const int qshift = own_keys ? (p.causal ? (Nkeys - Nq) % 128 : 0) : p.qshift;
+  // TMA coordinates (key row, outermost index) of key block jt
+  auto key_coord = [&](int jt, int& row, int& outer) {
+    if (p.block_table) {
+      const int pg = jt / p.tpp;
+      outer = __ldg(p.block_table + (size_t)b * p.bt_stride + pg);
+      row = (jt - pg * p.tpp) * 128;
+    } else {
+      outer = p.cu ? 0 : b;
+      row = krow0 + jt * 128;
+    }
+  };
   const int Tr = p.cu ? (Nq + qshift + 127) / 128 : p.Tr;
   const int Tk = p.cu ? (Nkeys + 127) / 128 : p.Tk;
   const int bz = p.cu ? 0 : b;                        // outermost TMA coordinate
@@ -159,11 +178,13 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
       bool ok = true;
       for (int u = 0; u < U && ok; ++u) {
+        int krow, kouter;
+        key_coord(j0 - u, krow, kouter);   // (a page lookup is in flight while the stage is waited for)
         ok = mbar_wait(&k_empty[s], par, status);
         if (!ok) break;
         mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, krow0 + (j0 - u) * 128, hkv, bz);
+          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, krow, hkv, kouter);
         issued = u + 1;
         if (++s == KS) { s = 0; par ^= 1; }
         if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
@@ -171,7 +192,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (!ok) break;
           mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
           for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow0 + (j0 - u) * 128, hkv, bz);
+            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow, hkv, kouter);
           v_issued = u + 1;
         }
       }
@@ -255,9 +276,11 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             ok = mbar_wait_warp(&v_empty[x], (r & 1) ^ 1, status);
             if (!ok) break;
             if (leader) {
+              int vrow, vouter;
+              key_coord(j0 - u, vrow, vouter);
               mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
               for (int pn = 0; pn < PAN; ++pn)
-                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, krow0 + (j0 - u) * 128, hkv, bz);
+                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, vrow, hkv, vouter);
             }
             __syncwarp();
           }

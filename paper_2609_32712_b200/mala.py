@@ -65,6 +65,9 @@ def lib():
         L.mala_fwd_varlen_prefix.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i,
                                              i, i, i, f, f, vp, sz, vp]
         L.mala_fwd_varlen_prefix.restype = i
+        L.mala_fwd_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, i,
+                                     i, i, f, f, vp, sz, vp]
+        L.mala_fwd_paged.restype = i
         L.mala_fwd_varlen.restype = i
         L.mala_bwd_varlen.restype = i
         L.mala_decode.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp, sz, vp]
@@ -266,6 +269,26 @@ def fwd_varlen_prefix(q, k, v, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, ma
                                       max_seqlen_k, d, int(causal), scale, tau, None, 0, _stream())
     if rc != 0:
         raise MalaError(rc, "mala_fwd_varlen_prefix")
+    return o, lse, st
+
+
+def fwd_paged(q, kpages, vpages, cu_seqlens_q, block_table, seqlens_k, max_seqlen_q: int, scale: float, tau: float,
+              causal: bool = True, stats: bool = False):
+    """mala_fwd_paged: packed q [1,total_q,Hq,d] against keys / values in pages [num_pages, page_size, Hkv, d]
+    (block_table int32 [B, max_pages], seqlens_k int32 [B]).  Returns (o, lse [Hq,total_q], Stats or None)."""
+    one, total_q, Hq, d = q.shape
+    num_pages, page_size, Hkv = kpages.shape[0], kpages.shape[1], kpages.shape[2]
+    B, max_pages = block_table.shape
+    o = torch.empty_like(q)
+    lse = torch.empty((Hq, total_q), dtype=torch.float32, device=q.device)
+    Tq, Tk = -(-(max_seqlen_q + 127) // 128), -(-(max_pages * page_size) // 128)
+    st = Stats((B, Hq, Tq), -(-Tk // 32), q.device) if stats else None
+    rc = lib().mala_fwd_paged(_view(q, _TIn), _view(kpages, _TIn), _view(vpages, _TIn), cu_seqlens_q.data_ptr(),
+                              block_table.data_ptr(), seqlens_k.data_ptr(), _view(o, _TOut), lse.data_ptr(),
+                              ctypes.byref(st.c) if st else None, B, Hq, Hkv, total_q, max_seqlen_q, num_pages,
+                              page_size, max_pages, d, int(causal), scale, tau, None, 0, _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_fwd_paged")
     return o, lse, st
 
 

@@ -165,3 +165,42 @@ def test_varlen_with_cached_prefixes(mala, oracle, tau, causal):
     assert st.totals.cpu().numpy()[1] == legal
     if tau > 0 and causal:
         assert skipped > 0
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("page", [128, 256])
+def test_prefill_chunks_against_a_paged_cache(mala, oracle, tau, page):
+    """Packed prefill chunks whose keys and values (prefix and chunk) lie in pages scattered over a shuffled pool."""
+    Hq, Hkv, d = 4, 2, 128
+    nk = [900, 128, 517, 300]
+    nq = [260, 128, 100, 1]
+    ws = [W.custom_prefill(1, Hq, Hkv, n, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=70 + x, preset="R")
+          for x, n in enumerate(nk)]
+    Nmax = -(-max(nk) // page) * page
+    kc = torch.zeros((len(nk), Nmax, Hkv, d), dtype=torch.bfloat16)
+    vc = torch.zeros_like(kc)
+    for b, (w, n) in enumerate(zip(ws, nk)):
+        kc[b, :n], vc[b, :n] = w["k"][0], w["v"][0]
+    kp, vp, bt, sl = W.paginate(kc, vc, page, seqlens=nk, seed=page)
+    q = torch.cat([w["q"][:, n - m:] for w, n, m in zip(ws, nk, nq)], dim=1).contiguous()
+    cq = torch.tensor(np.concatenate([[0], np.cumsum(nq)]), dtype=torch.int32)
+    o, lse, st = mala.fwd_paged(q.cuda(), kp.cuda(), vp.cuda(), cq.cuda(), bt.cuda(), sl.cuda(), max(nq), ws[0]["scale"],
+                                tau, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    fm = st.mask(Nmax // 128).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy()[0], lse.cpu().numpy()
+    legal = 0
+    for b, (w, n, m) in enumerate(zip(ws, nk, nq)):
+        off = n - m
+        ref = oracle.fwd(w["q"][:, n - m:], w["k"], w["v"], w["scale"], tau, 128, 128, q_shift=off % 128)
+        Tq, Tk = ref["mask"].shape[2], ref["mask"].shape[3]
+        r0 = int(cq[b])
+        for h in range(Hq):
+            for i in range(Tq):
+                parity.check_mask(fm[b, h, i, :Tk], ref["mask"][0, h, i], ref["crit"][0, h, i],
+                                  list(range(i + off // 128, -1, -1)), tau, max(i * 128 - off % 128, 0) + 1 + off)
+        parity.check_output(o_c[r0:r0 + m], ref["o"][0])
+        assert np.abs(lse_c[:, r0:r0 + m] - ref["lse"][0]).max() <= parity.LSE_ABS
+        legal += int((ref["mask"] > 0).sum())
+    assert st.totals.cpu().numpy()[1] == legal

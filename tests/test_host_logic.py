@@ -102,6 +102,9 @@ def test_argument_validation_codes_of_the_general_shape_calls(mala):
     fp = lambda cq, ck, mq=128, mk=256: L.mala_fwd_varlen_prefix(tin(), tin(), tin(), cq, ck, tout(), base, None, 2, 2, 2, 256,
                                                                  512, mq, mk, 128, 1, 0.1, 1e-4, None, 0, None)
     assert fp(None, base) == -1 and fp(base, None) == -1 and fp(base, base, mq=256, mk=128) == -2
+    fg = lambda page=128, bt=base, sl=base: L.mala_fwd_paged(tin(), tin(), tin(), base, bt, sl, tout(), base, None, 2, 2, 2, 256,
+                                                             128, 8, page, 4, 128, 1, 0.1, 1e-4, None, 0, None)
+    assert fg(page=64) == -2 and fg(bt=None) == -1 and fg(sl=None) == -1 and fg(bt=base + 2) == -3
     # several tokens per decode step: at most 16 rows per KV head, no more new tokens than keys
     dm = lambda Sq, Hq=4, Nk=256: L.mala_decode_multi(tin(), tin(), tin(), tout(), None, None, 1, Hq, 1, Nk, Sq, 128, 0.1,
                                                       1e-4, 2, base, 1 << 20, None)
