@@ -297,6 +297,48 @@ def varlen_leg(cfg, preset, lens, tau, it, peaks, dev):
     return row
 
 
+def serving_prefill_leg(cfg, preset, tau, it, peaks, dev):
+    """A serving-style prefill batch with the heads of a prefill configuration: eight sequences, a 2048-token chunk each
+    behind prefixes of 0 ... 30720 tokens, packed (mala_fwd_varlen_prefix) and against a paged cache (mala_fwd_paged,
+    256-key pages in a shuffled pool): latency of the MALA and dense kernels, tensor-pipe fraction on executed work."""
+    import torch
+    from paper_2609_32712_b200 import mala, workloads as W
+    prefixes, chunk = (30720, 16384, 8192, 4096, 2048, 1000, 300, 0), 2048
+    nk = [p_ + chunk for p_ in prefixes]
+    ws = [W.custom_prefill(1, cfg.Hq, cfg.Hkv, n, cfg.d, head_types=cfg.head_types, seed=cfg.seed + 17 * x, preset=preset,
+                           device=dev) for x, n in enumerate(nk)]
+    q = torch.cat([w["q"][:, n - chunk:] for w, n in zip(ws, nk)], dim=1).contiguous()
+    k = torch.cat([w["k"] for w in ws], dim=1).contiguous()
+    v = torch.cat([w["v"] for w in ws], dim=1).contiguous()
+    cq = torch.tensor([chunk * x for x in range(len(nk) + 1)], dtype=torch.int32, device=dev)
+    ck = torch.tensor([0] + list(torch.tensor(nk).cumsum(0)), dtype=torch.int32, device=dev)
+    scale = ws[0]["scale"]
+    Nmax = -(-max(nk) // 256) * 256
+    kc = torch.zeros((len(nk), Nmax, cfg.Hkv, cfg.d), dtype=torch.bfloat16, device=dev)
+    vc = torch.zeros_like(kc)
+    for b, (w, n) in enumerate(zip(ws, nk)):
+        kc[b, :n], vc[b, :n] = w["k"][0], w["v"][0]
+    kp, vp, bt, sl = W.paginate(kc, vc, 256, seqlens=nk, seed=11)
+    del kc, vc, ws
+    row = {"prefixes": list(prefixes), "chunk": chunk}
+    taus = {"mala": tau, "dense": 0.0}
+    packed = time_alternating({lab: (lambda t_=t_: mala.fwd_varlen_prefix(q, k, v, cq, ck, chunk, max(nk), scale, t_))
+                               for lab, t_ in taus.items()}, 3, it)
+    paged = time_alternating({lab: (lambda t_=t_: mala.fwd_paged(q, kp, vp, cq, bt, sl, chunk, scale, t_))
+                              for lab, t_ in taus.items()}, 3, it)
+    _, _, st = mala.fwd_varlen_prefix(q, k, v, cq, ck, chunk, max(nk), scale, tau, stats=True)
+    torch.cuda.synchronize()
+    ret, leg = st.totals.cpu().tolist()
+    for lab in taus:
+        row[lab] = {"packed_ms": packed[lab], "paged_ms": paged[lab]}
+    row["legal_tiles"], row["retained_frac"] = leg, ret / leg
+    row["tensor_frac_on_executed"] = (fwd_executed_flops(leg, ret, cfg.d) / (packed["mala"] * 1e-3) / 1e12
+                                      / peaks["tflops_sustained"])
+    row["dense_tensor_frac"] = (fwd_executed_flops(leg, leg, cfg.d) / (packed["dense"] * 1e-3) / 1e12
+                                / peaks["tflops_sustained"])
+    return row
+
+
 def fidelity(cs, taus, it):
     """Work and operator fidelity of MALA against the in-library dense path on one configuration (the protocol
     of Section 5.1 on synthetic states): retained slots per query in forward and backward, omitted softmax mass
@@ -604,6 +646,8 @@ def main():
                     row["chunk_last_8192"] = chunk_leg(cs, 8192, tau, it, peaks)
                 if name == "cfg3":                  # the same heads on packed sequences of 16K + 8K + 5000 + 3192 rows
                     row["varlen_4seq_32768"] = varlen_leg(cc, preset, (16384, 8192, 5000, 3192), tau, it, peaks, dev)
+                if name == "cfg3":                  # a serving-style batch of prefill chunks behind cached prefixes
+                    row["serving_prefill_8x2048"] = serving_prefill_leg(cc, preset, tau, it, peaks, dev)
                 if name == "cfg3" and preset == "R":
                     row["fidelity_vs_dense"] = fidelity(cs, (1e-4, 1e-2, 1.0), it)
                 detail[f"{name}_{preset}"] = row
