@@ -271,14 +271,16 @@ int mala_oracle_bwd_D(const double* O, const double* dO, int N, int d, double* D
 
 /* One backward tile (key block j, query block i) of Algorithm 2.  Computes S_ji = K_j Q_i^T with
  * the causal mask, the offline test of Eq. 4 against the saved lse, and, if retained, P and dS
- * (both [Bk x Bq], row = key).  Returns 1 if retained; *C_out is the tile criterion
- * max over valid causal entries of (s - lse_q - theta_q). */
+ * (both [Bk x Bq], row = key, column b = query q0 + b).  Returns 1 if retained; *C_out is the tile
+ * criterion max over valid causal entries of (s - lse_q - theta_q).
+ * shift: query block i holds the rows q with i*Bq <= q + shift < (i+1)*Bq, as in the forward pass. */
 static int bwd_tile(const double* Q, const double* K, const double* V, const double* dO, const double* lse,
-                    const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal, int j,
-                    int i, double* S, double* P, double* dS, double* C_out) {
+                    const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal, int shift,
+                    int j, int i, double* S, double* P, double* dS, double* C_out) {
   const int off = Nk - N;
   const int k0 = j * Bk, cols_k = (k0 + Bk <= Nk ? Bk : Nk - k0);
-  const int q0 = i * Bq, cols_q = (q0 + Bq <= N ? Bq : N - q0);
+  const int q0 = (i * Bq - shift > 0 ? i * Bq - shift : 0);
+  const int q1 = ((i + 1) * Bq - shift < N ? (i + 1) * Bq - shift : N), cols_q = q1 - q0;
   double C = -INFINITY;
   for (int a = 0; a < cols_k; ++a) {
     const int k = k0 + a;
@@ -313,14 +315,16 @@ static int bwd_tile(const double* Q, const double* K, const double* V, const dou
 /* Algorithm 2 for the listed key blocks of one query head (key_blocks == NULL: all).
  * dK, dV [N,d]: rows of the listed key blocks are overwritten with this head's contribution.
  * dQ [N,d] or NULL: contributions of the listed key blocks are ADDED (atomically).
- * mask, crit [Tc*Tr] indexed [j*Tr + i] (may be NULL). */
+ * mask, crit [Tc*Tr] indexed [j*Tr + i] (may be NULL); Tr = ceil((N + shift)/Bq), shift as in the
+ * forward pass (0 <= shift < Bq). */
 int mala_oracle_bwd(const double* Q, const double* K, const double* V, const double* dO, const double* lse,
                     const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal,
-                    int n_blocks, const int* key_blocks, double* dQ, double* dK, double* dV, uint8_t* mask,
+                    int shift, int n_blocks, const int* key_blocks, double* dQ, double* dK, double* dV, uint8_t* mask,
                     double* crit) {
   if (N <= 0 || (causal && Nk < N) || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
+  if (shift < 0 || shift >= Bq) return -1;
   const int off = Nk - N;
-  const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
+  const int Tr = (N + shift + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int nb = key_blocks ? n_blocks : Tc;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < nb; ++u) {
@@ -333,14 +337,15 @@ int mala_oracle_bwd(const double* Q, const double* K, const double* V, const dou
     for (int a = 0; a < cols_k; ++a)
       for (int c = 0; c < d; ++c) { dK[(size_t)(k0 + a) * d + c] = 0.0; dV[(size_t)(k0 + a) * d + c] = 0.0; }
     for (int i = 0; i < Tr; ++i) { /* ascending; legal tiles start at the diagonal */
-      const int q0 = i * Bq, cols_q = (q0 + Bq <= N ? Bq : N - q0);
+      const int q0 = (i * Bq - shift > 0 ? i * Bq - shift : 0);
+      const int q1 = ((i + 1) * Bq - shift < N ? (i + 1) * Bq - shift : N), cols_q = q1 - q0;
       if (causal && k0 > q0 + cols_q - 1 + off) { /* no valid causal entry */
         if (mask) mask[(size_t)j * Tr + i] = MASK_ILLEGAL;
         if (crit) crit[(size_t)j * Tr + i] = NAN;
         continue;
       }
       double C;
-      const int retain = bwd_tile(Q, K, V, dO, lse, D, N, Nk, d, scale, tau, Bq, Bk, causal, j, i, S, P, dS, &C);
+      const int retain = bwd_tile(Q, K, V, dO, lse, D, N, Nk, d, scale, tau, Bq, Bk, causal, shift, j, i, S, P, dS, &C);
       if (mask) mask[(size_t)j * Tr + i] = retain ? MASK_RETAINED : MASK_SKIPPED;
       if (crit) crit[(size_t)j * Tr + i] = C;
       if (!retain) continue;
@@ -374,15 +379,17 @@ int mala_oracle_bwd(const double* Q, const double* K, const double* V, const dou
  * query block (all legal key blocks j), so that sampled blocks can be checked at full size. */
 int mala_oracle_bwd_dq(const double* Q, const double* K, const double* V, const double* dO, const double* lse,
                        const double* D, int N, int Nk, int d, double scale, double tau, int Bq, int Bk, int causal,
-                       int n_blocks, const int* query_blocks, double* dQ) {
+                       int shift, int n_blocks, const int* query_blocks, double* dQ) {
   if (N <= 0 || (causal && Nk < N) || d <= 0 || Bq <= 0 || Bk <= 0 || !(tau >= 0.0)) return -1;
+  if (shift < 0 || shift >= Bq) return -1;
   const int off = Nk - N;
-  const int Tr = (N + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
+  const int Tr = (N + shift + Bq - 1) / Bq, Tc = (Nk + Bk - 1) / Bk;
   const int nb = query_blocks ? n_blocks : Tr;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < nb; ++u) {
     const int i = query_blocks ? query_blocks[u] : (Tr - 1 - u);
-    const int q0 = i * Bq, cols_q = (q0 + Bq <= N ? Bq : N - q0);
+    const int q0 = (i * Bq - shift > 0 ? i * Bq - shift : 0);
+    const int q1 = ((i + 1) * Bq - shift < N ? (i + 1) * Bq - shift : N), cols_q = q1 - q0;
     double* S = (double*)malloc(sizeof(double) * (size_t)Bk * Bq);
     double* P = (double*)malloc(sizeof(double) * (size_t)Bk * Bq);
     double* dS = (double*)malloc(sizeof(double) * (size_t)Bk * Bq);
@@ -392,7 +399,7 @@ int mala_oracle_bwd_dq(const double* Q, const double* K, const double* V, const 
       const int k0 = j * Bk, cols_k = (k0 + Bk <= Nk ? Bk : Nk - k0);
       if (causal && k0 > q0 + cols_q - 1 + off) continue;
       double C;
-      if (!bwd_tile(Q, K, V, dO, lse, D, N, Nk, d, scale, tau, Bq, Bk, causal, j, i, S, P, dS, &C)) continue;
+      if (!bwd_tile(Q, K, V, dO, lse, D, N, Nk, d, scale, tau, Bq, Bk, causal, shift, j, i, S, P, dS, &C)) continue;
       for (int a = 0; a < cols_k; ++a)
         for (int b = 0; b < cols_q; ++b) {
           const double ds = dS[(size_t)a * Bq + b];

@@ -53,9 +53,10 @@ def lib():
         L.mala_oracle_fwd_split.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _ci, _ci, _I, _D, _D,
                                             _U8, _D]
         L.mala_oracle_bwd_D.argtypes = [_D, _D, _ci, _ci, _D]
-        L.mala_oracle_bwd.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I,
+        L.mala_oracle_bwd.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _ci, _I,
                                       _D, _D, _D, _U8, _D]
-        L.mala_oracle_bwd_dq.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _I, _D]
+        L.mala_oracle_bwd_dq.argtypes = [_D, _D, _D, _D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _ci, _ci, _I,
+                                         _D]
         L.mala_oracle_decode_tiles_per_split.argtypes = [_ci, _ci, _ci]
         L.mala_oracle_decode_splits.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _D, _D, _U8, _D]
         L.mala_oracle_decode_splits_tps.argtypes = [_D, _D, _D, _ci, _ci, _ci, _cd, _cd, _ci, _ci, _ci, _D, _D, _U8, _D]
@@ -190,19 +191,20 @@ def fwd(q, k, v, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True
 
 
 def bwd(q, k, v, o, do, lse, scale: float, tau: float, Bq: int, Bk: int, causal: bool = True,
-        key_units=None, dq_units=None):
+        key_units=None, dq_units=None, q_shift: int = 0):
     """Algorithm 2 with the given forward output ``o`` and saved ``lse``.
 
     Full run (both unit lists None): dq, dk, dv complete.  With ``key_units`` = [(b, h_kv, j)] only
     those key blocks are run: their dK/dV rows (summed over the group's query heads) are exact and
     everything else is NaN.  With ``dq_units`` = [(b, h_q, i)] the dQ rows of those query blocks are
-    computed from all their legal key blocks.  Fewer queries than keys: as in ``fwd``.
+    computed from all their legal key blocks.  Fewer queries than keys and ``q_shift``: as in ``fwd``
+    (query block i = rows q with i*Bq <= q + q_shift < (i+1)*Bq; Tr = ceil((N + q_shift)/Bq)).
     Returns dict(dq, dk, dv, mask [B,Hq,Tc,Tr], crit [B,Hq,Tc,Tr]).
     """
     B, N, Hq, d = q.shape
     Nk, Hkv = k.shape[1], k.shape[2]
     G = Hq // Hkv
-    Tr, Tc = -(-N // Bq), -(-Nk // Bk)
+    Tr, Tc = -(-(N + q_shift) // Bq), -(-Nk // Bk)
     full = key_units is None and dq_units is None
     dq = np.zeros((B, N, Hq, d)) if full else np.full((B, N, Hq, d), np.nan)
     dk = np.zeros((B, Nk, Hkv, d)) if full else np.full((B, Nk, Hkv, d), np.nan)
@@ -241,7 +243,7 @@ def bwd(q, k, v, o, do, lse, scale: float, tau: float, Bq: int, Bk: int, causal:
             m = np.zeros((Tc, Tr), dtype=np.uint8)
             cr = np.full((Tc, Tr), np.nan)
             _ck(lib().mala_oracle_bwd(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, Nk, d, scale, tau, Bq, Bk,
-                                      int(causal), 0 if bl is None else len(bl), _ip(bl),
+                                      int(causal), q_shift, 0 if bl is None else len(bl), _ip(bl),
                                       _p(a) if full else None, _p(c), _p(e), _u8(m), _p(cr)), "bwd")
             if full:
                 dq[b, :, h, :] = a
@@ -263,8 +265,8 @@ def bwd(q, k, v, o, do, lse, scale: float, tau: float, Bq: int, Bk: int, causal:
             Q, K, V, dO, l, D = head_inputs(b, h)
             a = np.full((N, d), np.nan)
             _ck(lib().mala_oracle_bwd_dq(_p(Q), _p(K), _p(V), _p(dO), _p(l), _p(D), N, Nk, d, scale, tau, Bq, Bk,
-                                         int(causal), len(bl), _ip(bl), _p(a)), "bwd_dq")
-            rows = np.concatenate([np.arange(i * Bq, min(N, (i + 1) * Bq)) for i in bl])
+                                         int(causal), q_shift, len(bl), _ip(bl), _p(a)), "bwd_dq")
+            rows = np.concatenate([np.arange(max(0, i * Bq - q_shift), min(N, (i + 1) * Bq - q_shift)) for i in bl])
             dq[b, rows, h, :] = a[rows]
     return dict(dq=dq, dk=dk, dv=dv, mask=mask, crit=crit)
 

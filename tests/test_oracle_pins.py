@@ -87,22 +87,24 @@ def brute_mala_fwd(Q, K, V, scale, tau, Bq, Bk):
     return O, lse, mask
 
 
-def brute_mala_bwd(Q, K, V, dO, O, lse, scale, tau, Bq, Bk):
+def brute_mala_bwd(Q, K, V, dO, O, lse, scale, tau, Bq, Bk, shift=0):
     """Eq. 4 per tile with the saved lse, then the attention-backward equations restricted to the
-    retained tiles, written with whole-matrix products."""
-    N = Q.shape[0]
+    retained tiles, written with whole-matrix products.  The queries are the last rows of the keys' positions;
+    query block i holds the rows q with i*Bq <= q + shift < (i+1)*Bq."""
+    N, Nk = Q.shape[0], K.shape[0]
+    off = Nk - N
     S = scale * (Q @ K.T)                                       # [q, k]
-    Tr, Tc = -(-N // Bq), -(-N // Bk)
+    Tr, Tc = -(-(N + shift) // Bq), -(-Nk // Bk)
     mask = np.zeros((Tc, Tr), dtype=np.uint8)
-    keep = np.zeros((N, N), dtype=bool)
+    keep = np.zeros((N, Nk), dtype=bool)
     for j in range(Tc):
         for i in range(Tr):
-            qs = range(i * Bq, min(N, (i + 1) * Bq))
-            ks = range(j * Bk, min(N, (j + 1) * Bk))
-            ent = [(q, k) for q in qs for k in ks if k <= q]
+            qs = range(max(0, i * Bq - shift), min(N, (i + 1) * Bq - shift))
+            ks = range(j * Bk, min(Nk, (j + 1) * Bk))
+            ent = [(q, k) for q in qs for k in ks if k <= q + off]
             if not ent:
                 continue
-            skip = all(math.exp(S[q, k] - lse[q]) < tau / (q + 1) for (q, k) in ent)
+            skip = all(math.exp(S[q, k] - lse[q]) < tau / (q + 1 + off) for (q, k) in ent)
             mask[j, i] = 1 if skip else 2
             if not skip:
                 for (q, k) in ent:
@@ -898,3 +900,39 @@ def test_chunk_from_any_position_equals_the_rows_of_the_full_run_when_its_blocks
             assert np.array_equal(f["mask"][0, 0, i], full["mask"][0, 0, i_full0 + i])
             rows = slice(i * Bq - shift, min(Nq, (i + 1) * Bq - shift))
             assert np.array_equal(f["o"][0, rows], full["o"][0, off:][rows])
+
+
+@pytest.mark.parametrize("tau", [1e-2, 0.5])
+@pytest.mark.parametrize("Nq,Nk,Bq,Bk", [(27, 64, 8, 8), (30, 75, 8, 8), (19, 50, 16, 4), (24, 64, 8, 8)])
+def test_bwd_of_a_chunk_from_any_position_matches_bruteforce(Nq, Nk, Bq, Bk, tau):
+    # the offline rule on a chunk whose query blocks follow the positions (q_shift = (Nk - Nq) mod Bq): every tile
+    # decision and the three gradients against a brute force over entries, and the tile decisions of every query
+    # block the chunk holds completely against the backward pass of the whole sequence with the same lse
+    d, scale = 32, 1.0 / math.sqrt(32)
+    off = Nk - Nq
+    shift = off % Bq
+    q, k, v = peaky_inputs(Nk, d, 431 + Nk, boost=5.0)
+    do = _rng(432).standard_normal(q.shape)
+    qc, doc = q[:, off:], do[:, off:]
+    f = orc.fwd(qc, k, v, scale, tau, Bq, Bk, q_shift=shift)
+    g = orc.bwd(qc, k, v, f["o"], doc, f["lse"], scale, tau, Bq, Bk, q_shift=shift)
+    dQ, dK, dV, M = brute_mala_bwd(qc[0, :, 0], k[0, :, 0], v[0, :, 0], doc[0, :, 0], f["o"][0, :, 0], f["lse"][0, 0],
+                                   scale, tau, Bq, Bk, shift=shift)
+    assert (g["mask"][0, 0] == M).all() and (M == 1).any()
+    assert np.allclose(g["dq"][0, :, 0], dQ, atol=1e-11)
+    assert np.allclose(g["dk"][0, :, 0], dK, atol=1e-11)
+    assert np.allclose(g["dv"][0, :, 0], dV, atol=1e-11)
+    # whole sequence, its lse rows replaced by the chunk's: the blocks they share decide alike
+    ff = orc.fwd(q, k, v, scale, tau, Bq, Bk)
+    lse = ff["lse"].copy()
+    lse[:, :, off:] = f["lse"]
+    gg = orc.bwd(q, k, v, ff["o"], do, lse, scale, tau, Bq, Bk)
+    i_first = off // Bq + (1 if shift else 0)                   # first block of the whole run made of chunk rows only
+    assert np.array_equal(g["mask"][0, 0][:, i_first - off // Bq:], gg["mask"][0, 0][:, i_first:])
+    # dq_units / key_units take the same blocks
+    part = orc.bwd(qc, k, v, f["o"], doc, f["lse"], scale, tau, Bq, Bk, key_units=[(0, 0, 1)], dq_units=[(0, 0, 0), (0, 0, 2)],
+                   q_shift=shift)
+    r0 = slice(0, Bq - shift)
+    r2 = slice(2 * Bq - shift, min(Nq, 3 * Bq - shift))
+    assert np.allclose(part["dq"][0, r0, 0], dQ[r0], atol=1e-11) and np.allclose(part["dq"][0, r2, 0], dQ[r2], atol=1e-11)
+    assert np.allclose(part["dk"][0, Bk:2 * Bk, 0], dK[Bk:2 * Bk], atol=1e-11)
