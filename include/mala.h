@@ -92,13 +92,13 @@ int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, cons
  * with 128 i <= q + (Nk - Nq) % 128 < 128 (i + 1), so the first block of a chunk that starts inside a tile is a short
  * one -- and the result therefore equals rows Nk - Nq .. Nk - 1 of the equal-length call on the whole sequence wherever
  * the chunk holds a whole block of that call (for the backward: with dout zero on the earlier rows).
- * mala_fwd_chunk takes any Nk >= Nq; mala_bwd_chunk needs the chunk to start on a tile boundary,
- * (Nk - Nq) % 128 == 0 (MALA_ERR_UNSUPPORTED otherwise).
+ * Both calls take any Nk >= Nq.
  * causal == 0: every key legal for every query, L_q = Nk, any Nq and Nk.
  * Telemetry: fwd retained_per_block [B,Hq,Tq], tile_bitmask [B,Hq,Tq,ceil(ceil(Nk/128)/32)] with
  * Tq = ceil((Nq + (Nk - Nq) % 128) / 128) (causal) or ceil(Nq/128);
- * bwd retained_per_block [B,Hq,ceil(Nk/128)], tile_bitmask [B,Hq,ceil(Nk/128),ceil(ceil(Nq/128)/32)].
- * Workspace of the backward: mala_workspace_bytes(MALA_OP_BWD, B, Hq, Hkv, Nq, d, 0).  Everything else as
+ * bwd retained_per_block [B,Hq,ceil(Nk/128)], tile_bitmask [B,Hq,ceil(Nk/128),ceil(Tq/32)].
+ * Workspace of the backward: mala_workspace_bytes(MALA_OP_BWD, B, Hq, Hkv, Nq + (Nk - Nq) % 128, d, 0) when causal
+ * (the accumulator holds whole query blocks), mala_workspace_bytes(MALA_OP_BWD, B, Hq, Hkv, Nq, d, 0) otherwise.  Everything else as
  * mala_fwd / mala_bwd, which are these calls with Nq = Nk = N. */
 int mala_fwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
                    int Hkv, int Nq, int Nk, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,

@@ -172,11 +172,10 @@ int mala_device_status(int* code_out, int clear) {
   return MALA_OK;
 }
 
-// Lengths of a call with N queries and Nk keys: causal needs the queries to be the last N positions of the Nk; the
-// backward also needs them to start on a tile boundary.
-static int check_lengths(int N, int Nk, int causal, bool aligned_only) {
+// Lengths of a call with N queries and Nk keys: causal needs the queries to be the last N positions of the Nk.
+static int check_lengths(int N, int Nk, int causal) {
   if (N <= 0 || Nk <= 0) return MALA_ERR_INVALID_ARG;
-  if (causal && (Nk < N || (aligned_only && (Nk - N) % 128 != 0))) return MALA_ERR_UNSUPPORTED;
+  if (causal && Nk < N) return MALA_ERR_UNSUPPORTED;
   return MALA_OK;
 }
 
@@ -202,7 +201,7 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
       return MALA_ERR_WORKSPACE_TOO_SMALL;
   }
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
-  MALA_TRY(check_lengths(N, Nk, causal, false));
+  MALA_TRY(check_lengths(N, Nk, causal));
   if (!lse) return MALA_ERR_INVALID_ARG;
   const int Bt = cu ? 1 : B, Nt = cu ? total : N, Nkt = cu ? (cu_k ? total_k : total) : Nk;   // extents of the tensors
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, Bt, Nt, Hq));
@@ -291,7 +290,7 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
                     int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream,
                     const int32_t* cu = nullptr, int total = 0) {
   MALA_TRY(check_common(B0, Hq, Hkv, N0, d, scale, tau));
-  MALA_TRY(check_lengths(N0, Nk0, causal, true));
+  MALA_TRY(check_lengths(N0, Nk0, causal));
   if (!lse || !ws) return MALA_ERR_INVALID_ARG;
   // extents of the tensors and of the workspace (packed sequences: one batch entry of `total` rows)
   const int B = cu ? 1 : B0, N = cu ? total : N0, Nk = cu ? total : Nk0;
@@ -304,7 +303,9 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
   MALA_TRY(check_view(dk.p, dk.sb, dk.sn, dk.sh, B, Nk, Hkv));
   MALA_TRY(check_view(dv.p, dv.sb, dv.sn, dv.sh, B, Nk, Hkv));
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + 128 * B0 : N, d)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  // (a causal chunk that starts inside a tile: the query blocks follow the positions, (Nk - N) % 128 more rows)
+  const int pad_rows = (causal && !cu) ? (Nk0 - N0) % 128 : 0;
+  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + 128 * B0 : N + pad_rows, d)) return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;

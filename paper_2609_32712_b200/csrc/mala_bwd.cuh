@@ -56,6 +56,11 @@ struct BwdParams {
   int* status;
   int B, Hq, Hkv, N, Np, T, words, causal;   // N, Np, T: query rows, padded query rows, query blocks
   int Nk, Tk, koff;     // keys, key blocks; causal: the queries are the last N positions, koff = (Nk - N) / 128
+  // Causal with (Nk - N) % 128 = qshift != 0: the query blocks follow the positions, block i = the rows q with
+  // 128 i <= q + qshift < 128 (i + 1); T and Np count those blocks, and the per-query vectors and the dQ
+  // accumulator are indexed by q + qshift.  The first block's missing rows load as zeros (rows before the tensor)
+  // and carry lse = +inf like the rows past the end, so they neither vote nor contribute.
+  int qshift;
   // Packed sequences of different lengths (null: B sequences of N rows each): sequence b holds rows cu[b] ..
   // cu[b+1]-1 of the [1, total, H, d] tensors.  N, T, Nk, Tk then describe the longest sequence (grid, telemetry
   // strides); the per-query vectors are [Hq, Np] and the dQ accumulator [Hq, Np, D] with Np >= total + 128 B, where
@@ -161,14 +166,14 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128, hq, bz);
+          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128 - p.qshift, hq, bz);
         // dO of every tile is fetched ahead, retained or not (the vote comes too late to hide the copy behind it);
         // a skipped tile's stage is handed straight back by the issuer
         ok = mbar_wait(&do_empty[s], ((n >> 1) & 1) ^ 1, status);
         if (!ok) { mbar_wait(&q_full[s], (n >> 1) & 1, status); break; }
         mbar_arrive_expect_tx(&do_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, row0 + i * 128, hq, bz);
+          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, row0 + i * 128 - p.qshift, hq, bz);
         issued = n + 1;
       }
       if (!ok) {
@@ -605,22 +610,24 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 }
 
 // D = rowsum(O o dO), lse2 = lse * log2(e), bq = lse2 + log2(tau / L_q); one warp per (b, h, row) with row below
-// Npg, the padded length of the (longest) sequence.  Packed sequences (cu != null): the vectors are [Hq, Np] with
+// Npg, the padded length of the (longest) sequence; entry `row` describes query row - qshift (qshift != 0 only
+// without cu).  Packed sequences (cu != null): the vectors are [Hq, Np] with
 // sequence b's rows from (cu[b] + 128 b) / 128 * 128 on, lse is [Hq, total].
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sn, int64_t o_sh,
                                       const __nv_bfloat16* __restrict__ dout, int64_t d_sb, int64_t d_sn, int64_t d_sh,
                                       const float* __restrict__ lse, float* __restrict__ lse2, float* __restrict__ bq,
                                       float* __restrict__ Dq, int B, int Hq, int N, int Np, int Nk, int d, int causal,
-                                      float log2_tau, const int* __restrict__ cu, int total_rows, int Npg) {
+                                      float log2_tau, const int* __restrict__ cu, int total_rows, int Npg, int qshift) {
   const int warps_per_block = blockDim.x >> 5;
   const long long wi = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   const long long total = (long long)B * Hq * Npg;
   if (wi >= total) return;
-  const int row = (int)(wi % Npg);
+  int row = (int)(wi % Npg);
   const int h = (int)((wi / Npg) % Hq);
   int b = (int)(wi / ((long long)Npg * Hq));
   long long w = wi;                                  // index into the vectors
+  row -= qshift;                                     // the query this entry describes
   int row0 = 0;
   if (cu) {
     row0 = cu[b];
@@ -630,7 +637,7 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
     w = (long long)h * Np + ((row0 + 128 * b) / 128) * 128 + row;
     b = 0;
   }
-  if (row >= N) {
+  if (row < 0 || row >= N) {
     if (lane == 0) { lse2[w] = INFINITY; bq[w] = INFINITY; Dq[w] = 0.f; }
     return;
   }
@@ -659,7 +666,7 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
 // [Hq, Np, d] with sequence b's tiles from (cu[b] + 128 b) / 128 on.)
 __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int64_t sb,
                                       int64_t sn, int64_t sh, int B, int Hq, int N, int Np, int d, float scale,
-                                      const int* __restrict__ cu, int Npg) {
+                                      const int* __restrict__ cu, int Npg, int qshift) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = d / 8;
   const long long total = (long long)B * Hq * Npg * per_row;
@@ -671,7 +678,7 @@ __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat
   const int i = (int)(tile % T);
   const int h = (int)((tile / T) % Hq);
   int b = (int)(tile / ((long long)T * Hq));
-  int row = i * 128 + r;
+  int row = i * 128 + r - qshift;                          // (qshift != 0 only without cu)
   if (cu) {
     const int row0 = cu[b];
     N = cu[b + 1] - row0;
@@ -681,7 +688,7 @@ __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat
     N += row0;
     b = 0;
   }
-  if (row >= N) return;
+  if (row < 0 || row >= N) return;
   const int half = d / 2;
   const float* base = acc + (size_t)tile * 128 * d;
   float4 x, y;
@@ -733,7 +740,8 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
                       const int* cu = nullptr, int total = 0) {
   // Packed sequences (cu): N = Nk = the longest sequence; the tensors are [1, total, H, d]; the per-query vectors and
   // the dQ accumulator are laid out per head over Np = total + 128 B rows (rounded up to a tile).
-  const int T = (N + 127) / 128, Npg = T * 128, Tk = (Nk + 127) / 128;
+  const int qshift = (causal && !cu) ? (Nk - N) % 128 : 0;
+  const int T = (N + qshift + 127) / 128, Npg = T * 128, Tk = (Nk + 127) / 128;
   const int Np = cu ? ((total + 128 * B + 127) / 128) * 128 : Npg;
   const int Bl = cu ? 1 : B;                 // batch extent of the tensors and of the workspace arrays
   const int Nt = cu ? total : N, Nkt = cu ? total : Nk;   // row extents of the tensors
@@ -764,7 +772,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   p.totals = st ? (unsigned long long*)st->totals : nullptr;
   p.status = status;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Np = Np; p.T = T; p.words = (T + 31) / 32; p.causal = causal;
-  p.Nk = Nk; p.Tk = Tk; p.koff = causal ? (Nk - N) / 128 : 0;
+  p.Nk = Nk; p.Tk = Tk; p.koff = causal ? (Nk - N) / 128 : 0; p.qshift = qshift;
   p.cu = cu;
   p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
   if (p.bitmask &&
@@ -778,7 +786,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     bwd_preprocess_kernel<<<blocks, wpb * 32, 0, stream>>>((const __nv_bfloat16*)o.p, o.sb, o.sn, o.sh,
                                                           (const __nv_bfloat16*)dout.p, dout.sb, dout.sn, dout.sh, lse,
                                                           lse2, bq, Dq, B, Hq, N, Np, Nk, d, causal,
-                                                          tau > 0.f ? log2f(tau) : -INFINITY, cu, total, Npg);
+                                                          tau > 0.f ? log2f(tau) : -INFINITY, cu, total, Npg, qshift);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   const bool dense = (tau == 0.f);
@@ -790,7 +798,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     const long long n_out = (long long)B * Hq * Npg * (d / 8);
     const unsigned blocks = (unsigned)((n_out + 255) / 256);
     bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(acc, (__nv_bfloat16*)dq.p, dq.sb, dq.sn, dq.sh, B, Hq, N, Np, d,
-                                                      scale, cu, Npg);
+                                                      scale, cu, Npg, qshift);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   return MALA_OK;

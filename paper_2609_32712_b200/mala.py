@@ -222,9 +222,10 @@ def bwd_chunk(q, k, v, o, do, lse, scale: float, tau: float, causal: bool = True
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
-    Tq, Tk = -(-Nq // 128), -(-Nk // 128)
+    shift = (Nk - Nq) % 128 if causal and Nk >= Nq else 0     # query blocks follow the positions
+    Tq, Tk = -(-(Nq + shift) // 128), -(-Nk // 128)
     st = Stats((B, Hq, Tk), -(-Tq // 32), q.device) if stats else None
-    ws = _ws(workspace_bytes(OP_BWD, B, Hq, Hkv, Nq, d), q.device) if ws is None else ws
+    ws = _ws(workspace_bytes(OP_BWD, B, Hq, Hkv, Nq + shift, d), q.device) if ws is None else ws
     rc = lib().mala_bwd_chunk(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TIn), _view(do, _TIn),
                               lse.data_ptr(), _view(dq, _TOut), _view(dk, _TOut), _view(dv, _TOut),
                               ctypes.byref(st.c) if st else None, B, Hq, Hkv, Nq, Nk, d, int(causal), scale, tau,

@@ -124,13 +124,72 @@ def test_chunk_equals_rows_of_the_equal_length_call(mala):
         assert (dv.float() - dvc.float()).abs().max() <= 1e-2 * dv.float().abs().max()
 
 
-def test_backward_rejects_a_chunk_that_starts_inside_a_tile(mala):
-    q = torch.zeros((1, 100, 2, 128), dtype=torch.bfloat16, device="cuda")
-    kv = torch.zeros((1, 300, 1, 128), dtype=torch.bfloat16, device="cuda")
-    lse = torch.zeros((1, 2, 100), dtype=torch.float32, device="cuda")
-    with pytest.raises(mala.MalaError) as e:
-        mala.bwd_chunk(q, kv, kv, q, q, lse, 0.1, 0.0)
-    assert e.value.code == -2
+def _run_bwd_any_offset(mala, oracle, c, tau):
+    """Backward of a chunk that may start inside a tile, on the GPU's own forward output."""
+    q, k, v, do = (c[x].cuda() for x in ("q", "k", "v", "do"))
+    B, Nq, Hq, d = q.shape
+    Nk = k.shape[1]
+    shift = (Nk - Nq) % 128
+    Tq, Tk = -(-(Nq + shift) // 128), -(-Nk // 128)
+    o, lse, fst = mala.fwd_chunk(q, k, v, c["scale"], tau, stats=True)
+    dq, dk, dv, bst = mala.bwd_chunk(q, k, v, o, do, lse, c["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    rb = oracle.bwd(c["q"], c["k"], c["v"], o.float().cpu(), c["do"], lse.cpu().numpy(), c["scale"], tau, 128, 128,
+                    q_shift=shift)
+    bm = bst.mask(Tq).cpu().numpy()                      # [B,Hq,Tk,Tq]
+    assert rb["mask"].shape == bm.shape
+    for b in range(B):
+        for h in range(Hq):
+            for j in range(Tk):
+                om, oc = rb["mask"][b, h, j], rb["crit"][b, h, j]
+                for i in range(Tq):
+                    if om[i] == 0:
+                        assert not bm[b, h, j, i]
+                    elif bool(bm[b, h, j, i]) != (om[i] == 2):
+                        assert abs(oc[i]) <= parity.MASK_BAND, (b, h, j, i, oc[i])
+                assert int(bst.retained[b, h, j]) == int(bm[b, h, j].sum())
+    parity.check_grad(dq.float().cpu().numpy(), rb["dq"], "dq")
+    parity.check_grad(dk.float().cpu().numpy(), rb["dk"], "dk")
+    parity.check_grad(dv.float().cpu().numpy(), rb["dv"], "dv")
+    assert (bm.transpose(0, 1, 3, 2) <= fst.mask(Tk).cpu().numpy()).all()        # nesting
+    assert bst.totals.cpu().numpy()[1] == int((rb["mask"] > 0).sum())
+    return int((rb["mask"] == 1).sum())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,Nq,d,Hq,Hkv", [(500, 100, 128, 2, 1), (1000, 333, 128, 4, 2), (777, 129, 64, 2, 2),
+                                            (1300, 5, 128, 2, 1), (640, 639, 128, 2, 1)])
+def test_chunk_backward_from_any_position_literal(mala, oracle, Nk, Nq, d, Hq, Hkv, tau):
+    w = W.custom_prefill(2, Hq, Hkv, Nk, d, seed=Nk + Nq)
+    _run_bwd_any_offset(mala, oracle, _chunk(w, Nq), tau)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("Nk,Nq,d", [(2000, 555, 128), (2500, 1300, 64)])
+def test_chunk_backward_from_any_position_skipping_regime(mala, oracle, Nk, Nq, d, tau):
+    w = W.custom_prefill(1, 4, 2, Nk, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=9, preset="R")
+    assert _run_bwd_any_offset(mala, oracle, _chunk(w, Nq), tau) > 0, "workload must exercise skipping"
+
+
+def test_chunk_backward_from_any_position_gives_the_rows_of_the_equal_length_call(mala):
+    w = W.custom_prefill(1, 4, 2, 1536, 128, head_types=["diffuse", "peaked", "peaked", "sink"], seed=3, preset="R")
+    q, k, v, do = (w[x].cuda() for x in ("q", "k", "v", "do"))
+    off = 1000
+    for tau in (0.0, 1e-4):
+        o, lse, _ = mala.fwd(q, k, v, w["scale"], tau)
+        do0 = do.clone()
+        do0[:, :off] = 0
+        dq, dk, dv, _ = mala.bwd(q, k, v, o, do0, lse, w["scale"], tau)
+        dqc, dkc, dvc, _ = mala.bwd_chunk(q[:, off:], k, v, o[:, off:], do[:, off:], lse[:, :, off:].contiguous(),
+                                          w["scale"], tau)
+        # the chunk's first block lacks the rows before `off`; with dout zero there they contribute nothing, but they
+        # vote in the whole call: compare from the first whole block on for dQ, and dK / dV within the tolerance that
+        # a tile retained by one call and skipped by the other leaves (entries below tau / L_q)
+        first = 1024 - off
+        assert (dq[:, 1024:].float() - dqc[:, first:].float()).abs().max() <= 1e-2 * dqc.float().abs().max()
+        assert (dk.float() - dkc.float()).abs().max() <= 1e-2 * dk.float().abs().max()
+        assert (dv.float() - dvc.float()).abs().max() <= 1e-2 * dv.float().abs().max()
 
 
 def _run_fwd_any_offset(mala, oracle, c, tau, S=1):

@@ -82,13 +82,13 @@ def test_argument_validation_codes_of_the_general_shape_calls(mala):
     base = (ctypes.addressof(buf) + 255) & ~255
     tin = lambda: mala._TIn(base, 0, 256, 128)
     tout = lambda: mala._TOut(base, 0, 256, 128)
-    # chunked prefill: a causal chunk has no more queries than keys; only the backward needs it to start on a tile boundary
+    # chunked prefill: a causal chunk has no more queries than keys and may start anywhere
     fc = lambda Nq, Nk, causal=1: L.mala_fwd_chunk(tin(), tin(), tin(), tout(), base, None, 1, 2, 2, Nq, Nk, 128, causal,
                                                    0.1, 1e-4, None, 0, None)
     assert fc(512, 256) == -2 and fc(0, 256) == -1 and fc(100, 300) != -2
     bc = lambda Nq, Nk: L.mala_bwd_chunk(tin(), tin(), tin(), tin(), tin(), base, tout(), tout(), tout(), None, 1, 2, 2,
                                          Nq, Nk, 128, 1, 0.1, 1e-4, base, 1 << 20, None)
-    assert bc(100, 300) == -2 and bc(128, 0) == -1
+    assert bc(512, 256) == -2 and bc(128, 0) == -1 and bc(100, 300) != -2
     # key ranges: a positive count, scratch that is large enough and aligned
     fs = lambda S, ws=base, n=1 << 20: L.mala_fwd_chunk_split(tin(), tin(), tin(), tout(), base, None, 1, 2, 2, 128, 512, 128,
                                                               1, 0.1, 1e-4, S, ws, n, None)
