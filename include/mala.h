@@ -14,8 +14,9 @@
  *     never frees or retains one.  Tensors are bf16 views [B, N, H, d] given as a base pointer and
  *     element strides (sb, sn, sh); the last dimension is contiguous.  Base pointers must be
  *     16-byte aligned and all strides multiples of 8 elements (16 bytes).
- *   - d is 64 or 128.  Hq must be a multiple of Hkv; query head h uses key/value head
- *     h / (Hq / Hkv).  N may be any positive length (the last tile may be ragged).
+ *   - d is a multiple of 8 between 8 and 128.  The kernels exist for 64 and 128 columns; another head size runs
+ *     on the next of the two at that size's cost (the missing columns are read as zeros and never stored).
+ *     Hq must be a multiple of Hkv; query head h uses key/value head h / (Hq / Hkv).  N may be any positive length (the last tile may be ragged).
  *   - scale (> 0, finite) multiplies the fp32 scores; lse is in nats, of the scaled scores, over
  *     the retained set.  tau >= 0, finite.
  *   - Tile partition: mala_tile_shape() reports it; forward and backward use the same partition.

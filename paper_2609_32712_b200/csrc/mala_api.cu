@@ -92,7 +92,7 @@ static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float
   if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0) return MALA_ERR_INVALID_ARG;
   if (!(tau >= 0.f) || !isfinite(tau)) return MALA_ERR_INVALID_ARG;
   if (!(scale > 0.f) || !isfinite(scale)) return MALA_ERR_INVALID_ARG;
-  if (d != 64 && d != 128) return MALA_ERR_UNSUPPORTED;
+  if (!head_size_ok(d)) return MALA_ERR_UNSUPPORTED;
   if (Hq % Hkv != 0) return MALA_ERR_UNSUPPORTED;
   if (B > 65535 || Hq > 65535) return MALA_ERR_UNSUPPORTED;
   return MALA_OK;
@@ -141,17 +141,18 @@ const char* mala_strerror(int code) {
 
 int mala_tile_shape(int op, int d, int* Bq, int* Bk) {
   if (!Bq || !Bk) return MALA_ERR_INVALID_ARG;
-  if (d != 64 && d != 128) return MALA_ERR_UNSUPPORTED;
+  if (!head_size_ok(d)) return MALA_ERR_UNSUPPORTED;
   if (op == MALA_OP_FWD || op == MALA_OP_BWD) { *Bq = 128; *Bk = 128; return MALA_OK; }
   if (op == MALA_OP_DECODE) { *Bq = 0; *Bk = 128; return MALA_OK; }
   return MALA_ERR_UNSUPPORTED;
 }
 
 size_t mala_workspace_bytes(int op, int B, int Hq, int Hkv, int N, int d, int num_splits) {
-  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || (d != 64 && d != 128)) return 0;
-  if (op == MALA_OP_FWD) return num_splits > 1 ? fwd_split_workspace_bytes(B, Hq, N, d, num_splits) : 256;
-  if (op == MALA_OP_BWD) return bwd_workspace_bytes(B, Hq, N, d);
-  if (op == MALA_OP_DECODE) return num_splits > 0 ? decode_workspace_bytes(B, Hq, d, num_splits) : 0;
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || !head_size_ok(d)) return 0;
+  const int D = padded_head_size(d);
+  if (op == MALA_OP_FWD) return num_splits > 1 ? fwd_split_workspace_bytes(B, Hq, N, D, num_splits) : 256;
+  if (op == MALA_OP_BWD) return bwd_workspace_bytes(B, Hq, N, D);
+  if (op == MALA_OP_DECODE) return num_splits > 0 ? decode_workspace_bytes(B, Hq, D, num_splits) : 0;
   return 0;
 }
 
@@ -197,7 +198,8 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
     if (cu || num_splits > 65535 || (long long)B * num_splits > 65535) return MALA_ERR_UNSUPPORTED;
     if (!ws) return MALA_ERR_INVALID_ARG;
     if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-    if (B > 0 && Hq > 0 && N > 0 && (d == 64 || d == 128) && ws_bytes < fwd_split_workspace_bytes(B, Hq, N, d, num_splits))
+    if (B > 0 && Hq > 0 && N > 0 && head_size_ok(d) &&
+        ws_bytes < fwd_split_workspace_bytes(B, Hq, N, padded_head_size(d), num_splits))
       return MALA_ERR_WORKSPACE_TOO_SMALL;
   }
   MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
@@ -220,7 +222,9 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
       !make_tensor_map_bnhd(&tv, v.p, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv, d, v.sb, v.sn, v.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
+  const int D = padded_head_size(d);
   FwdParams p;
+  p.d = d;
   p.cu = cu; p.total = total; p.cu_k = cu_k;
   p.block_table = pg ? pg->block_table : nullptr;
   p.seqlens_k = pg ? pg->seqlens_k : nullptr;
@@ -230,7 +234,7 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   p.tps = ((Nk + 127) / 128 + num_splits - 1) / num_splits;
   p.o_part = num_splits > 1 ? (float*)ws : nullptr;
   p.lse_part = num_splits > 1
-                   ? (float*)((uint8_t*)ws + (((size_t)B * Hq * num_splits * N * d * sizeof(float) + 255) & ~(size_t)255))
+                   ? (float*)((uint8_t*)ws + (((size_t)B * Hq * num_splits * N * D * sizeof(float) + 255) & ~(size_t)255))
                    : nullptr;
   p.o = (__nv_bfloat16*)o.p; p.o_sb = o.sb; p.o_sn = o.sn; p.o_sh = o.sh;
   p.lse = lse;
@@ -258,16 +262,16 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
     return MALA_ERR_CUDA;
   const bool dense = (tau == 0.f);
   int rc;
-  if (d == 128) rc = dense ? launch_fwd<128, true>(tq, tk, tv, p, stream) : launch_fwd<128, false>(tq, tk, tv, p, stream);
+  if (D == 128) rc = dense ? launch_fwd<128, true>(tq, tk, tv, p, stream) : launch_fwd<128, false>(tq, tk, tv, p, stream);
   else rc = dense ? launch_fwd<64, true>(tq, tk, tv, p, stream) : launch_fwd<64, false>(tq, tk, tv, p, stream);
   if (rc != MALA_OK || num_splits == 1) return rc;
   const unsigned rows = (unsigned)((long long)B * Hq * N);
-  if (d == 128)
+  if (D == 128)
     fwd_merge_splits_kernel<128><<<rows, 128, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
-                                                           num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal);
+                                                           num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal, d);
   else
     fwd_merge_splits_kernel<64><<<rows, 64, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
-                                                         num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal);
+                                                         num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal, d);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
@@ -305,7 +309,8 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
   // (a causal chunk that starts inside a tile: the query blocks follow the positions, (Nk - N) % 128 more rows)
   const int pad_rows = (causal && !cu) ? (Nk0 - N0) % 128 : 0;
-  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + 128 * B0 : N + pad_rows, d)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + 128 * B0 : N + pad_rows, padded_head_size(d)))
+    return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
@@ -401,7 +406,7 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
   MALA_TRY(check_view(vcache.p, vcache.sb, vcache.sn, vcache.sh, B, Nk, Hkv));
   MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-  if (ws_bytes < decode_workspace_bytes(B, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < decode_workspace_bytes(B, Hq, padded_head_size(d), num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
@@ -421,7 +426,7 @@ int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o,
   MALA_TRY(check_view(vcache.p, vcache.sb, vcache.sn, vcache.sh, B, Nk, Hkv));
   MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, Sq, Hq));
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-  if (ws_bytes < decode_workspace_bytes(B * Sq, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < decode_workspace_bytes(B * Sq, Hq, padded_head_size(d), num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
@@ -448,7 +453,7 @@ int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_
   MALA_TRY(check_view(vpages.p, vpages.sb, vpages.sn, vpages.sh, num_pages, page_size, Hkv));
   MALA_TRY(check_view(o.p, o.sb, Sq > 1 ? o.sn : 8, o.sh, B, Sq, Hq));
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-  if (ws_bytes < decode_workspace_bytes(B * Sq, Hq, d, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  if (ws_bytes < decode_workspace_bytes(B * Sq, Hq, padded_head_size(d), num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
@@ -469,7 +474,7 @@ int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o
   MALA_TRY(check_view(kcache.p, kcache.sb, kcache.sn, kcache.sh, B, Nk, Hkv));
   MALA_TRY(check_view(vcache.p, vcache.sb, vcache.sn, vcache.sh, B, Nk, Hkv));
   MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
-  if (decode_workspace_bytes(B, Hq, d, num_splits) > (size_t)MALA_STATIC_SCRATCH_BYTES)
+  if (decode_workspace_bytes(B, Hq, padded_head_size(d), num_splits) > (size_t)MALA_STATIC_SCRATCH_BYTES)
     return MALA_ERR_STATIC_SCRATCH_EXCEEDED;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
@@ -478,7 +483,7 @@ int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o
   unsigned char* scratch = nullptr;
   MALA_TRY(static_scratch_address(dev, &scratch));
   float* o_part = (float*)scratch;
-  float* lse_part = (float*)(scratch + decode_align256((size_t)B * Hq * num_splits * d * sizeof(float)));
+  float* lse_part = (float*)(scratch + decode_align256((size_t)B * Hq * num_splits * padded_head_size(d) * sizeof(float)));
   // every (batch, head, split) entry of both arrays is written by the split kernel (empty splits
   // included) before the merge reads it, so nothing left over from an earlier call is ever read
   return decode_launch_with_scratch(q, kcache, vcache, o, lse_opt, nullptr, B, Hq, Hkv, Nk, d, scale, tau, num_splits,

@@ -61,6 +61,7 @@ struct BwdParams {
   // accumulator are indexed by q + qshift.  The first block's missing rows load as zeros (rows before the tensor)
   // and carry lse = +inf like the rows past the end, so they neither vote nor contribute.
   int qshift;
+  int d;                // head size of the tensors (<= D; columns d .. D-1 are zeros and never stored)
   // Packed sequences of different lengths (null: B sequences of N rows each): sequence b holds rows cu[b] ..
   // cu[b+1]-1 of the [1, total, H, d] tensors.  N, T, Nk, Tk then describe the longest sequence (grid, telemetry
   // strides); the per-query vectors are [Hq, Np] and the dQ accumulator [Hq, Np, D] with Np >= total + 128 B, where
@@ -523,7 +524,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
               w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * f, __uint_as_float(o[8 * v + 3]) * f);
               w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * f, __uint_as_float(o[8 * v + 5]) * f);
               w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * f, __uint_as_float(o[8 * v + 7]) * f);
-              *reinterpret_cast<uint4*>(out + c * 32 + v * 8) = w;
+              if (c * 32 + v * 8 < p.d) *reinterpret_cast<uint4*>(out + c * 32 + v * 8) = w;
             }
           }
         }
@@ -666,7 +667,8 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
 // [Hq, Np, d] with sequence b's tiles from (cu[b] + 128 b) / 128 on.)
 __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int64_t sb,
                                       int64_t sn, int64_t sh, int B, int Hq, int N, int Np, int d, float scale,
-                                      const int* __restrict__ cu, int Npg, int qshift) {
+                                      const int* __restrict__ cu, int Npg, int qshift, int d_out) {
+  // d: columns of the accumulator (the padded head size); d_out <= d: columns of dq
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = d / 8;
   const long long total = (long long)B * Hq * Npg * per_row;
@@ -688,7 +690,7 @@ __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat
     N += row0;
     b = 0;
   }
-  if (row < 0 || row >= N) return;
+  if (row < 0 || row >= N || cg * 8 >= d_out) return;
   const int half = d / 2;
   const float* base = acc + (size_t)tile * 128 * d;
   float4 x, y;
@@ -712,7 +714,7 @@ __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat
 inline size_t bwd_align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // (Packed sequences: B = 1 and N = total rows + 128 x number of sequences.)
-inline size_t bwd_workspace_bytes(int B, int Hq, int N, int d) {
+inline size_t bwd_workspace_bytes(int B, int Hq, int N, int d) {   // d: the padded head size
   const size_t Np = (size_t)((N + 127) / 128) * 128;
   return bwd_align256((size_t)B * Hq * Np * d * sizeof(float)) + 3 * bwd_align256((size_t)B * Hq * Np * sizeof(float));
 }
@@ -740,6 +742,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
                       const int* cu = nullptr, int total = 0) {
   // Packed sequences (cu): N = Nk = the longest sequence; the tensors are [1, total, H, d]; the per-query vectors and
   // the dQ accumulator are laid out per head over Np = total + 128 B rows (rounded up to a tile).
+  const int D = padded_head_size(d);         // columns of the kernels and of the dQ accumulator
   const int qshift = (causal && !cu) ? (Nk - N) % 128 : 0;
   const int T = (N + qshift + 127) / 128, Npg = T * 128, Tk = (Nk + 127) / 128;
   const int Np = cu ? ((total + 128 * B + 127) / 128) * 128 : Npg;
@@ -747,22 +750,22 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   const int Nt = cu ? total : N, Nkt = cu ? total : Nk;   // row extents of the tensors
   uint8_t* w = (uint8_t*)ws;
   float* acc = (float*)w;
-  w += bwd_align256((size_t)Bl * Hq * Np * d * sizeof(float));
+  w += bwd_align256((size_t)Bl * Hq * Np * D * sizeof(float));
   const size_t vbytes = bwd_align256((size_t)Bl * Hq * Np * sizeof(float));
   float* lse2 = (float*)w;
   float* bq = (float*)(w + vbytes);
   float* Dq = (float*)(w + 2 * vbytes);
 
   CUtensorMap tq, tk, tv, tdo, tacc;
-  if (!make_tensor_map_f32_tiles(&tacc, acc + 64 * d, (uint64_t)Bl * Hq * (Np / 128), d / 2,
-                                 (uint64_t)128 * d * sizeof(float)) ||
+  if (!make_tensor_map_f32_tiles(&tacc, acc + 64 * D, (uint64_t)Bl * Hq * (Np / 128), D / 2,
+                                 (uint64_t)128 * D * sizeof(float)) ||
       !make_tensor_map_bnhd(&tq, q.p, Bl, Nt, Hq, d, q.sb, q.sn, q.sh, 128) ||
       !make_tensor_map_bnhd(&tk, k.p, Bl, Nkt, Hkv, d, k.sb, k.sn, k.sh, 128) ||
       !make_tensor_map_bnhd(&tv, v.p, Bl, Nkt, Hkv, d, v.sb, v.sn, v.sh, 128) ||
       !make_tensor_map_bnhd(&tdo, dout.p, Bl, Nt, Hq, d, dout.sb, dout.sn, dout.sh, 128))
     return MALA_ERR_TENSOR_MAP;
 
-  if (cudaMemsetAsync(acc, 0, (size_t)Bl * Hq * Np * d * sizeof(float), stream) != cudaSuccess) return MALA_ERR_CUDA;
+  if (cudaMemsetAsync(acc, 0, (size_t)Bl * Hq * Np * D * sizeof(float), stream) != cudaSuccess) return MALA_ERR_CUDA;
   BwdParams p;
   p.lse2 = lse2; p.bq = bq; p.Dq = Dq; p.dq_acc = acc;
   p.dk = (__nv_bfloat16*)dk.p; p.dk_sb = dk.sb; p.dk_sn = dk.sn; p.dk_sh = dk.sh;
@@ -773,7 +776,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   p.status = status;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Np = Np; p.T = T; p.words = (T + 31) / 32; p.causal = causal;
   p.Nk = Nk; p.Tk = Tk; p.koff = causal ? (Nk - N) / 128 : 0; p.qshift = qshift;
-  p.cu = cu;
+  p.cu = cu; p.d = d;
   p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
   if (p.bitmask &&
       cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * Tk * p.words * sizeof(uint32_t), stream) != cudaSuccess)
@@ -791,14 +794,14 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   }
   const bool dense = (tau == 0.f);
   int rc;
-  if (d == 128) rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, tacc, p, stream);
+  if (D == 128) rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, tacc, p, stream);
   else rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, tacc, p, stream);
   if (rc != MALA_OK) return rc;
   {
-    const long long n_out = (long long)B * Hq * Npg * (d / 8);
+    const long long n_out = (long long)B * Hq * Npg * (D / 8);
     const unsigned blocks = (unsigned)((n_out + 255) / 256);
-    bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(acc, (__nv_bfloat16*)dq.p, dq.sb, dq.sn, dq.sh, B, Hq, N, Np, d,
-                                                      scale, cu, Npg, qshift);
+    bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(acc, (__nv_bfloat16*)dq.p, dq.sb, dq.sn, dq.sh, B, Hq, N, Np, D,
+                                                      scale, cu, Npg, qshift, d);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   return MALA_OK;

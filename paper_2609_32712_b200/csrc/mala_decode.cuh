@@ -16,7 +16,7 @@ template <int D>
 __global__ void __launch_bounds__(D)
 decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part, __nv_bfloat16* __restrict__ o,
                     int64_t o_sb, int64_t o_sn, int64_t o_sh, float* __restrict__ lse_out, int Sq, int Hq,
-                    int num_splits) {
+                    int num_splits, int d) {   // d <= D: columns of o
   const int bh = blockIdx.x, h = bh % Hq, tok = (bh / Hq) % Sq, b = bh / (Hq * Sq), c = threadIdx.x;
   const float* lp = lse_part + (size_t)bh * num_splits;
   float mx = -INFINITY;
@@ -30,14 +30,14 @@ decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ 
     acc += w * o_part[((size_t)bh * num_splits + s) * D + c];
   }
   // (a sequence without keys has no split with mass: its output is 0 and its log-normalizer -inf)
-  o[b * o_sb + tok * o_sn + h * o_sh + c] = __float2bfloat16(Z > 0.f ? acc / Z : 0.f);
+  if (c < d) o[b * o_sb + tok * o_sn + h * o_sh + c] = __float2bfloat16(Z > 0.f ? acc / Z : 0.f);
   if (lse_out && c == 0) lse_out[bh] = Z > 0.f ? mx + logf(Z) : -INFINITY;
 }
 
 inline size_t decode_align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // (B: sequences x new tokens per sequence)
-inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) {
+inline size_t decode_workspace_bytes(int B, int Hq, int d, int S) {   // d: the padded head size
   return decode_align256((size_t)B * Hq * S * d * sizeof(float)) + decode_align256((size_t)B * Hq * S * sizeof(float));
 }
 
@@ -67,7 +67,8 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
                                       const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                                       float tau, int num_splits, float* o_part, float* lse_part, int* status,
                                       cudaStream_t stream, const DecPaging* pg = nullptr, int Sq = 1) {
-  if (d != 128 && d != 64) return MALA_ERR_UNSUPPORTED;
+  if (!head_size_ok(d)) return MALA_ERR_UNSUPPORTED;
+  const int D = padded_head_size(d);
   const int G = Hq / Hkv;
   if (Sq < 1 || G * Sq > 16 || Sq > Nk) return MALA_ERR_UNSUPPORTED;
   const bool paged = pg && pg->block_table;
@@ -118,7 +119,7 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   const int R = G * Sq;   // rows of a work item
 #define MALA_DEC_LAUNCH3(DENSE, GP, MULTI)                                                                           \
   {                                                                                                                  \
-    if (d == 128) mala_decode_split_kernel<DENSE, GP, MULTI, 128><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    if (D == 128) mala_decode_split_kernel<DENSE, GP, MULTI, 128><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
     else mala_decode_split_kernel<DENSE, GP, MULTI, 64><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);           \
   }
 #define MALA_DEC_LAUNCH2(DENSE, GP)          \
@@ -140,12 +141,12 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
 #undef MALA_DEC_LAUNCH2
 #undef MALA_DEC_LAUNCH3
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
-  if (d == 128)
+  if (D == 128)
     decode_merge_kernel<128><<<B * Sq * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
-                                                              Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits);
+                                                              Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits, d);
   else
     decode_merge_kernel<64><<<B * Sq * Hq, 64, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
-                                                            Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits);
+                                                            Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits, d);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
@@ -153,7 +154,8 @@ inline int decode_launch(mala_tin q, mala_tin kc, mala_tin vc, mala_tout o, floa
                          int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws, int* status,
                          cudaStream_t stream, const DecPaging* pg = nullptr, int Sq = 1) {
   float* o_part = (float*)ws;
-  float* lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Sq * Hq * num_splits * d * sizeof(float)));
+  float* lse_part =
+      (float*)((uint8_t*)ws + decode_align256((size_t)B * Sq * Hq * num_splits * padded_head_size(d) * sizeof(float)));
   return decode_launch_with_scratch(q, kc, vc, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, o_part,
                                     lse_part, status, stream, pg, Sq);
 }

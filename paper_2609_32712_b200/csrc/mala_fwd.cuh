@@ -54,6 +54,7 @@ struct FwdParams {
   // log-normalizer of the range; a merge kernel combines the ranges.
   int num_splits, tps;
   float* o_part;                 // [B, Hq, num_splits, N, D]
+  int d;                         // head size of the tensors (<= D; the columns d .. D-1 are zeros and never stored)
   float* lse_part;               // [B, Hq, num_splits, N] natural log
   float scale_log2;              // scale * log2(e)
   float log2_tau;                // log2(tau); unused by the dense kernel
@@ -522,7 +523,8 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (valid) {
 #pragma unroll
           for (int v = 0; v < 8; ++v)
-            *reinterpret_cast<float4*>(p.o_part + prow * D + cc * 32 + v * 4) =
+            if (cc * 32 + v * 4 < p.d)
+              *reinterpret_cast<float4*>(p.o_part + prow * D + cc * 32 + v * 4) =
                 make_float4(__uint_as_float(o[4 * v]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
                             __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
         }
@@ -553,7 +555,7 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
             w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
             w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + cc * 32 + v * 8) = w;
+            if (cc * 32 + v * 8 < p.d) *reinterpret_cast<uint4*>(orow + cc * 32 + v * 8) = w;
           }
         }
       }
@@ -584,7 +586,7 @@ __global__ void __launch_bounds__(D)
 fwd_merge_splits_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part,
                         __nv_bfloat16* __restrict__ o, int64_t o_sb, int64_t o_sn, int64_t o_sh,
                         float* __restrict__ lse, int Hq, int N, int num_splits, int tps, int Tk, int koff, int qshift,
-                        int causal) {
+                        int causal, int d) {
   const long long idx = blockIdx.x;
   const int row = (int)(idx % N), h = (int)((idx / N) % Hq), b = (int)(idx / ((long long)N * Hq)), c = threadIdx.x;
   const int newest = causal ? (row + qshift) / 128 + koff : Tk - 1;
@@ -596,13 +598,14 @@ fwd_merge_splits_kernel(const float* __restrict__ o_part, const float* __restric
   for (int s = 0; s < ns; ++s) {
     const float w = exp2f((lse_part[(base + s) * N + row] - mx) * 1.4426950408889634f);
     Z += w;
-    acc += w * o_part[((base + s) * N + row) * D + c];
+    if (c < d) acc += w * o_part[((base + s) * N + row) * D + c];
   }
-  o[b * o_sb + (int64_t)row * o_sn + h * o_sh + c] = __float2bfloat16(acc / Z);
+  if (c < d) o[b * o_sb + (int64_t)row * o_sn + h * o_sh + c] = __float2bfloat16(acc / Z);
   if (c == 0) lse[((size_t)b * Hq + h) * N + row] = mx + logf(Z);
 }
 
-inline size_t fwd_split_workspace_bytes(int B, int Hq, int N, int d, int S) {
+inline size_t fwd_split_workspace_bytes(int B, int Hq, int N, int D, int S) {   // D: padded head size
+  const int d = D;
   auto align256 = [](size_t x) { return (x + 255) & ~(size_t)255; };
   return align256((size_t)B * Hq * S * N * d * sizeof(float)) + align256((size_t)B * Hq * S * N * sizeof(float));
 }

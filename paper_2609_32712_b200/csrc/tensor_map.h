@@ -28,6 +28,12 @@ inline PFN_tensorMapEncodeTiled tensor_map_encoder() {
 // Tensor map over a bf16 [B, N, H, d] view: coordinates (c, n, h, b), box = 64 columns x box_rows rows,
 // 128-byte swizzle, out-of-range rows read as zero.  Returns false if the driver rejects it
 // (base not 16-byte aligned, a stride not a multiple of 16 bytes, ...).
+// Head sizes: any multiple of 8 up to 128.  The kernels are built for D = 64 and D = 128 columns; a smaller head runs
+// on the next of the two with the missing columns read as zeros (TMA fills what lies beyond the tensor map's inner
+// extent d) and never stored.
+inline bool head_size_ok(int d) { return d >= 8 && d <= 128 && d % 8 == 0; }
+inline int padded_head_size(int d) { return d <= 64 ? 64 : 128; }
+
 inline bool make_tensor_map_bnhd(CUtensorMap* out, const void* base, int B, int N, int H, int d, int64_t sb,
                                  int64_t sn, int64_t sh, int box_rows) {
   PFN_tensorMapEncodeTiled enc = tensor_map_encoder();

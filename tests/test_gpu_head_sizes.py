@@ -1,0 +1,96 @@
+"""Head sizes other than 64 and 128 (any multiple of 8 up to 128): every entry point against the oracle.  The kernels
+run them on the next of their two column counts with the missing columns read as zeros, so what these cases guard is
+that nothing beyond column d is stored and that the zero columns change no result."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_32712_b200 import workloads as W
+from tests import parity
+from tests.test_gpu_chunk import _chunk, _run, _run_bwd_any_offset, _run_fwd_any_offset, _run_split
+from tests.test_gpu_decode import _run_and_check, _run_multi, _run_paged
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mala():
+    from paper_2609_32712_b200 import mala as m
+    m.lib()
+    return m
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("d,N,Hq,Hkv", [(96, 640, 4, 2), (80, 500, 2, 1), (32, 700, 2, 2), (8, 300, 2, 1), (120, 257, 2, 1),
+                                        (40, 384, 4, 1)])
+def test_forward_and_backward_literal(mala, oracle, d, N, Hq, Hkv, tau):
+    w = W.custom_prefill(2, Hq, Hkv, N, d, seed=d + N)
+    _run(mala, oracle, _chunk(w, N), tau)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("d", [96, 48])
+def test_forward_and_backward_skipping_regime(mala, oracle, d, tau):
+    w = W.custom_prefill(1, 4, 2, 2048, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=d, preset="R")
+    assert _run(mala, oracle, _chunk(w, 2048), tau) > 0, "workload must exercise skipping"
+
+
+@pytest.mark.parametrize("d", [96, 24])
+def test_chunks_and_key_ranges(mala, oracle, d):
+    w = W.custom_prefill(1, 4, 2, 1500, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=d + 1, preset="R")
+    _run(mala, oracle, _chunk(w, 348), 1e-4)                      # starts on a tile boundary
+    _run_fwd_any_offset(mala, oracle, _chunk(w, 333), 1e-4)
+    _run_fwd_any_offset(mala, oracle, _chunk(w, 333), 1e-4, S=3)
+    _run_bwd_any_offset(mala, oracle, _chunk(w, 333), 1e-4)
+    _run_split(mala, oracle, _chunk(w, 220), 1e-4, 4)
+    _run(mala, oracle, _chunk(w, 200), 1e-2, causal=False)
+
+
+def test_nothing_is_stored_beyond_the_head_size(mala):
+    # outputs are views of wider buffers filled with a sentinel: the columns past d must keep it
+    d, dw, N = 96, 128, 400
+    w = W.custom_prefill(1, 2, 1, N, d, seed=5)
+    q, k, v, do = (w[x].cuda() for x in ("q", "k", "v", "do"))
+
+    def wide(like):
+        buf = torch.full(like.shape[:-1] + (dw,), 7.0, dtype=torch.bfloat16, device="cuda")
+        return buf, buf[..., :d]
+
+    ob, o = wide(q)
+    mala.fwd(q, k, v, w["scale"], 1e-4, out=o)
+    lse = mala.fwd(q, k, v, w["scale"], 1e-4)[1]
+    (dqb, dq), (dkb, dk), (dvb, dv) = wide(q), wide(k), wide(v)
+    mala.bwd(q, k, v, o, do, lse, w["scale"], 1e-4, dq=dq, dk=dk, dv=dv)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    for buf in (ob, dqb, dkb, dvb):
+        assert (buf[..., d:] == 7.0).all() and not (buf[..., :d] == 7.0).all()
+    o2, _, _ = mala.fwd(q, k, v, w["scale"], 1e-4)
+    assert torch.equal(o2, o)
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("d,Nk,S,Hq,Hkv", [(96, 1024, 4, 8, 2), (80, 1000, 3, 8, 4), (32, 4096, 8, 16, 1), (8, 300, 2, 6, 2),
+                                           (120, 2048, 4, 3, 1)])
+def test_decode_literal(mala, oracle, d, Nk, S, Hq, Hkv, tau):
+    w = W.custom_decode(2, Hq, Hkv, Nk, d, S, seed=Nk + d)
+    _run_and_check(mala, oracle, w, tau, S)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("d", [96, 40])
+def test_decode_gated_paged_several_tokens(mala, oracle, d, tau):
+    w = W.custom_decode(2, 8, 2, 8192, d, 8, group_types=["diffuse", "peaked"], seed=3 + d, preset="D")
+    res = _run_and_check(mala, oracle, w, tau, 8)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+    _run_paged(mala, oracle, w, tau, 8, 256, [8192, 4096 + 77], seed=9)
+    _run_paged(mala, oracle, w, tau, 8, 16, [8192, 1000], seed=10)
+    assert _run_multi(mala, oracle, w, 3, tau, 8) > 0
+
+
+def test_head_sizes_that_are_refused(mala):
+    for d in (4, 100, 136, 256):
+        q = torch.zeros(1, 256, 2, d, dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(mala.MalaError) as e:
+            mala.fwd(q, q, q, 0.1, 0.0)
+        assert e.value.code in (-2, -3)

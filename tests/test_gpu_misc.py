@@ -105,9 +105,9 @@ def test_binding_reports_errors(mala):
     with pytest.raises(mala.MalaError) as e:
         mala.fwd(q, q, q, 0.1, -1.0)
     assert e.value.code == -1
-    q96 = torch.zeros(1, 256, 2, 96, dtype=torch.bfloat16, device="cuda")
+    q256 = torch.zeros(1, 256, 2, 256, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(mala.MalaError) as e:
-        mala.fwd(q96, q96, q96, 0.1, 0.0)
+        mala.fwd(q256, q256, q256, 0.1, 0.0)
     assert e.value.code == -2
     q17 = torch.zeros(1, 1, 34, 128, dtype=torch.bfloat16, device="cuda")
     kv1 = torch.zeros(1, 256, 2, 128, dtype=torch.bfloat16, device="cuda")

@@ -41,9 +41,12 @@ def test_host_only_queries(mala):
     assert mala.tile_shape(mala.OP_BWD, 64) == (128, 128)
     assert mala.tile_shape(mala.OP_DECODE, 128) == (0, 128)
     with pytest.raises(mala.MalaError):
-        mala.tile_shape(mala.OP_FWD, 96)
+        mala.tile_shape(mala.OP_FWD, 256)
     # backward scratch: fp32 dQ accumulator + three fp32 per-row vectors, rows padded to whole tiles
     assert mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 64) == 2 * 1024 * 64 * 4 + 3 * 2 * 1024 * 4
+    # (head sizes between the two kernel widths take the wider one's scratch)
+    assert mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 96) == mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 128)
+    assert mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 40, 8) == mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 64, 8)
     assert mala.workspace_bytes(mala.OP_DECODE, 8, 32, 8, 131072, 128, 128) == 8 * 32 * 128 * 128 * 4 + 8 * 32 * 128 * 4
     assert mala.workspace_bytes(mala.OP_DECODE, 8, 32, 8, 131072, 128, 0) == 0
     assert mala.lib().mala_strerror(-4).decode() == "workspace too small"
@@ -61,7 +64,7 @@ def test_argument_validation_codes(mala):
     assert f(B=0) == -1 and f(N=-3) == -1
     assert f(tau=-1.0) == -1 and f(tau=float("nan")) == -1 and f(scale=0.0) == -1 and f(scale=float("inf")) == -1
     assert f(lse=None) == -1
-    assert f(d=96) == -2 and f(Hq=3, Hkv=2) == -2
+    assert f(d=256) == -2 and f(d=100) == -2 and f(d=0) == -2 and f(Hq=3, Hkv=2) == -2
     assert f(q=tin(off=2)) == -3 and f(q=tin(sn=130)) == -3
     # decode: too many packed heads, bad split count
     g = lambda **kw: L.mala_decode(tin(), tin(), tin(), tout(), None, None, 1, kw.get("Hq", 4), kw.get("Hkv", 1), 256,
