@@ -28,11 +28,20 @@ def _heads(rng):
 
 @pytest.mark.parametrize("seed", [2, 3, 4])
 def test_random_cases(mala, oracle, seed):
+    _sweep(mala, oracle, seed, [64, 128], 40)
+
+
+@pytest.mark.parametrize("seed", [5, 6])
+def test_random_cases_any_head_size(mala, oracle, seed):
+    _sweep(mala, oracle, seed, list(range(8, 129, 8)), 40)
+
+
+def _sweep(mala, oracle, seed, head_sizes, n):
     rng = random.Random(seed)
-    for it in range(40):
+    for it in range(n):
         kind = rng.choice(["fwdbwd", "chunk", "split", "varlen", "decode", "paged", "multi"])
         tau = rng.choice([0.0, 1e-5, 1e-4, 1e-2, 1.0])
-        d = rng.choice([64, 128])
+        d = rng.choice(head_sizes)
         preset = rng.choice(["literal", "R"])
         if kind == "fwdbwd":
             Hq, Hkv = _heads(rng)
@@ -58,6 +67,8 @@ def test_random_cases(mala, oracle, seed):
                 if causal and Nk > Nq + 1:   # the forward also from a position inside a tile, unsplit and split
                     c2 = TC._chunk(w, Nq + rng.randint(1, min(127, Nk - Nq)))
                     TC._run_fwd_any_offset(mala, oracle, c2, tau, rng.choice([1, S]))
+                    if len(head_sizes) > 2:   # (the newer sweep: the backward from that position as well)
+                        TC._run_bwd_any_offset(mala, oracle, c2, tau)
         elif kind == "varlen":
             Hq, Hkv = _heads(rng)
             lens = [rng.randint(1, 600) for _ in range(rng.randint(1, 4))]
