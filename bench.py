@@ -690,13 +690,14 @@ def main():
                 # fewer, longer splits: a split's normalizer grows with its length, so more of its tiles fall under the
                 # threshold ("Fused decoding execution": the split-local test is the conservative one)
                 sweep = {}
-                for S in (128, 64, 32, 16):
+                S_auto = mala.decode_suggest_splits(dcfg.B, dcfg.Hkv, dcfg.Nk)
+                for S in sorted({128, 64, 32, 16, S_auto}, reverse=True):
                     _, _, st = mala.decode(qd, kc, vc, wd["scale"], tau, S, ws=wsd, out=od, stats=True)
                     ret, leg = st.totals.cpu().tolist()
                     us = 1e3 * time_cuda(lambda: mala.decode(qd, kc, vc, wd["scale"], tau, S, ws=wsd, out=od,
                                                               want_lse=False), 25, 100)
                     need = (leg + ret) * TILE * dcfg.d * 2
-                    sweep[f"splits={S}"] = {"us": us, "retained_frac": ret / leg,
+                    sweep[f"splits={S}" + (" (suggested)" if S == S_auto else "")] = {"us": us, "retained_frac": ret / leg,
                                             "rel_l2_o": float((od.float() - o0).norm() / o0.norm()),
                                             "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
                                             "speedup": row["dense"]["us"] / us}

@@ -237,6 +237,17 @@ int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_
 int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, int B, int Hq,
                        int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* cuda_stream);
 
+/* A split count for mala_decode and its variants (host only; nothing is launched).  The skip test of a split sees
+ * only that split's partial normalizer ("Fused decoding execution"), so it passes more often the longer the split:
+ * the best count is the SMALLEST one that still spreads the B * Hkv * num_splits work items evenly over the SMs.
+ * Items differ in how many tiles they retain, so an SM needs several of them to even that out.
+ * Returned: the smallest S with at least six items per SM and at least two tiles per split (without the first
+ * condition where the two cannot both hold) whose longest per-SM queue, ceil(B*Hkv*S / sm_count) items of
+ * ceil(ceil(Nk/128) / S) tiles each, is within 4 % of the shortest such queue any admissible S gives.
+ * Nk: the (longest) cache length; sm_count <= 0: the current device's SM count is used.
+ * Returns the count (>= 1) or a negative MALA_ERR_* code. */
+int mala_decode_suggest_splits(int B, int Hkv, int Nk, int sm_count);
+
 /* Scratch bytes needed by one call of `op` (MALA_OP_*); N is Nk for decode; num_splits is ignored
  * for fwd / bwd.  Returns 0 for unsupported arguments. */
 size_t mala_workspace_bytes(int op, int B, int Hq, int Hkv, int N, int d, int num_splits);

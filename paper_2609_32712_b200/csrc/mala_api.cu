@@ -139,6 +139,27 @@ const char* mala_strerror(int code) {
   }
 }
 
+int mala_decode_suggest_splits(int B, int Hkv, int Nk, int sm_count) {
+  if (B <= 0 || Hkv <= 0 || Nk <= 0) return MALA_ERR_INVALID_ARG;
+  if (sm_count <= 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+      return MALA_ERR_CUDA;
+  }
+  const long long T = (Nk + 127) / 128, groups = (long long)B * Hkv;
+  auto queue = [&](long long S) { return ((groups * S + sm_count - 1) / sm_count) * ((T + S - 1) / S); };
+  long long hi = T / 2 > 1 ? T / 2 : 1;                       // at least two tiles per split
+  if (hi > 65535) hi = 65535;
+  long long lo = (6LL * sm_count + groups - 1) / groups;       // at least six items per SM ...
+  if (lo > hi) lo = 1;                                         // ... where the cache is long enough for that
+  long long best = queue(lo);
+  for (long long S = lo + 1; S <= hi; ++S) best = queue(S) < best ? queue(S) : best;
+  for (long long S = lo; S <= hi; ++S)
+    if (queue(S) * 100 <= best * 104) return (int)S;
+  return (int)lo;
+}
+
 int mala_tile_shape(int op, int d, int* Bq, int* Bk) {
   if (!Bq || !Bk) return MALA_ERR_INVALID_ARG;
   if (!head_size_ok(d)) return MALA_ERR_UNSUPPORTED;

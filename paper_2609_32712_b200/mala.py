@@ -82,6 +82,8 @@ def lib():
         L.mala_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
         L.mala_workspace_bytes.restype = sz
         L.mala_tile_shape.argtypes = [i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
+        L.mala_decode_suggest_splits.argtypes = [i, i, i, i]
+        L.mala_decode_suggest_splits.restype = i
         L.mala_device_status.argtypes = [ctypes.POINTER(i), i]
         L.mala_strerror.argtypes = [i]
         L.mala_strerror.restype = ctypes.c_char_p
@@ -107,6 +109,14 @@ def tile_shape(op: int, d: int):
     if rc != 0:
         raise MalaError(rc, "mala_tile_shape")
     return bq.value, bk.value
+
+
+def decode_suggest_splits(B: int, Hkv: int, Nk: int, sm_count: int = 0) -> int:
+    """mala_decode_suggest_splits: the smallest split count that still fills the SMs evenly."""
+    rc = int(lib().mala_decode_suggest_splits(B, Hkv, Nk, sm_count))
+    if rc < 0:
+        raise MalaError(rc, "mala_decode_suggest_splits")
+    return rc
 
 
 def workspace_bytes(op: int, B: int, Hq: int, Hkv: int, N: int, d: int, num_splits: int = 0) -> int:

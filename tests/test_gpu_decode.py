@@ -71,6 +71,14 @@ def test_decode_gated_keys_skip_value_tiles(mala, oracle, Nk, S, tau):
     assert res["totals"][1] == res["retained"] + res["skipped"]
 
 
+def test_decode_with_the_suggested_split_count(mala, oracle):
+    w = W.custom_decode(2, 8, 2, 20000, 128, 1, group_types=["diffuse", "peaked"], seed=77, preset="D")
+    S = mala.decode_suggest_splits(2, 2, 20000)              # SM count of the current device
+    assert 1 <= S <= 157 // 2
+    assert S == mala.decode_suggest_splits(2, 2, 20000, torch.cuda.get_device_properties(0).multi_processor_count)
+    _run_and_check(mala, oracle, w, 1e-4, S)
+
+
 def test_decode_tau_zero_is_split_invariant(mala):
     w = W.custom_decode(1, 8, 2, 4096, 128, 4, seed=11)
     q, kc, vc = (w[x].cuda() for x in ("q", "kcache", "vcache"))

@@ -50,6 +50,21 @@ def test_host_only_queries(mala):
     assert mala.workspace_bytes(mala.OP_DECODE, 8, 32, 8, 131072, 128, 128) == 8 * 32 * 128 * 128 * 4 + 8 * 32 * 128 * 4
     assert mala.workspace_bytes(mala.OP_DECODE, 8, 32, 8, 131072, 128, 0) == 0
     assert mala.lib().mala_strerror(-4).decode() == "workspace too small"
+    # split count for decode: the smallest one that fills the SMs evenly (queue = items per SM x tiles per item)
+    # with at least six items per SM and two tiles per split
+    T = 1024
+    queue = lambda S, groups=64, sms=148: -(-groups * S // sms) * -(-T // S)
+    S = mala.decode_suggest_splits(8, 8, 131072, 148)
+    lo = -(-6 * 148 // 64)
+    best = min(queue(x) for x in range(lo, T // 2 + 1))
+    assert S >= lo and queue(S) * 100 <= best * 104 and all(queue(x) * 100 > best * 104 for x in range(lo, S))
+    assert S == 16                                                        # 1024 items: seven per SM, 64 tiles each
+    assert mala.decode_suggest_splits(1024, 8, 4096, 148) == 1            # enough sequences: no split needed
+    assert mala.decode_suggest_splits(1, 1, 100, 148) == 1                # one tile cannot be split
+    assert mala.decode_suggest_splits(1, 1, 131072, 148) in range(128, 149)   # one head: about one split per SM
+    assert mala.decode_suggest_splits(2, 8, 1024, 148) <= 4               # short cache: two tiles per split at least
+    with pytest.raises(mala.MalaError):
+        mala.decode_suggest_splits(0, 8, 4096, 148)
 
 
 def test_argument_validation_codes(mala):
