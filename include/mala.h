@@ -150,6 +150,19 @@ int mala_fwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu
                            int total_k, int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau,
                            void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Algorithm 2 for mala_fwd_varlen_prefix: every sequence is treated exactly as a mala_bwd_chunk call on its own
+ * rows, with the query blocks following its key positions as in the forward call.  o, dout, dq like q; dk, dv like k;
+ * lse fp32 [Hq,total_q] as the forward call wrote it.  A sequence without queries (or, causal != 0, with more queries
+ * than keys) gets zero dk / dv rows (and zero dq rows).  Telemetry as for mala_bwd_chunk with ceil(max_seqlen_k / 128)
+ * key blocks and Tq = ceil((max_seqlen_q + 127) / 128).  Workspace:
+ * mala_workspace_bytes(MALA_OP_BWD, 1, Hq, Hkv, total_q + 384 * B, d, 0).  As for the other packed calls, the tiles at
+ * a sequence's ends also cover rows of its neighbours, which must be finite numbers. */
+int mala_bwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,
+                           const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k, mala_tout dq, mala_tout dk,
+                           mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int total_q, int total_k,
+                           int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau, void* ws,
+                           size_t ws_bytes, void* cuda_stream);
+
 /* mala_fwd_varlen_prefix with the keys and values held in pages: a batch of prefill chunks behind prefixes that
  * live in a paged cache (the chunks' own keys and values already written to their pages).  q, o [1,total_q,Hq,d]
  * packed by cu_seqlens_q (device int32 [B+1]); kpages, vpages [num_pages, page_size, Hkv, d] with page_size a multiple

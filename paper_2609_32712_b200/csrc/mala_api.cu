@@ -313,12 +313,12 @@ int mala_fwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, 
 static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
                     mala_tout dk, mala_tout dv, const mala_stats* st, int B0, int Hq, int Hkv, int N0, int Nk0, int d,
                     int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream,
-                    const int32_t* cu = nullptr, int total = 0) {
+                    const int32_t* cu = nullptr, int total = 0, const int32_t* cu_k = nullptr, int total_k = 0) {
   MALA_TRY(check_common(B0, Hq, Hkv, N0, d, scale, tau));
   MALA_TRY(check_lengths(N0, Nk0, causal));
   if (!lse || !ws) return MALA_ERR_INVALID_ARG;
   // extents of the tensors and of the workspace (packed sequences: one batch entry of `total` rows)
-  const int B = cu ? 1 : B0, N = cu ? total : N0, Nk = cu ? total : Nk0;
+  const int B = cu ? 1 : B0, N = cu ? total : N0, Nk = cu ? (cu_k ? total_k : total) : Nk0;
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, N, Hq));
   MALA_TRY(check_view(k.p, k.sb, k.sn, k.sh, B, Nk, Hkv));
   MALA_TRY(check_view(v.p, v.sb, v.sn, v.sh, B, Nk, Hkv));
@@ -330,14 +330,14 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
   // (a causal chunk that starts inside a tile: the query blocks follow the positions, (Nk - N) % 128 more rows)
   const int pad_rows = (causal && !cu) ? (Nk0 - N0) % 128 : 0;
-  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + 128 * B0 : N + pad_rows, padded_head_size(d)))
+  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + (cu_k ? 384 : 128) * B0 : N + pad_rows, padded_head_size(d)))
     return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
   MALA_TRY(device_setup(dev, &status));
   return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B0, Hq, Hkv, N0, Nk0, d, causal ? 1 : 0, scale, tau, ws,
-                    status, (cudaStream_t)cuda_stream, cu, total);
+                    status, (cudaStream_t)cuda_stream, cu, total, cu_k, total_k);
 }
 
 int mala_fwd_chunk_split(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B,
@@ -414,6 +414,19 @@ int mala_bwd_varlen(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
   MALA_TRY(check_packed(cu_seqlens, B, total, max_seqlen));
   return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau,
                   ws, ws_bytes, cuda_stream, cu_seqlens, total);
+}
+
+int mala_bwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,
+                           const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k, mala_tout dq, mala_tout dk,
+                           mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int total_q, int total_k,
+                           int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau, void* ws,
+                           size_t ws_bytes, void* cuda_stream) {
+  MALA_TRY(check_packed(cu_seqlens_q, B, total_q, max_seqlen_q));
+  MALA_TRY(check_packed(cu_seqlens_k, B, total_k, max_seqlen_k));
+  if ((long long)total_q + 384LL * B > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
+  if (causal && max_seqlen_k < max_seqlen_q) return MALA_ERR_UNSUPPORTED;
+  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, max_seqlen_q, max_seqlen_k, d, causal, scale, tau,
+                  ws, ws_bytes, cuda_stream, cu_seqlens_q, total_q, cu_seqlens_k, total_k);
 }
 
 int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,

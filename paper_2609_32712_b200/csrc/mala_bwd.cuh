@@ -67,6 +67,10 @@ struct BwdParams {
   // strides); the per-query vectors are [Hq, Np] and the dQ accumulator [Hq, Np, D] with Np >= total + 128 B, where
   // sequence b owns the rows from (cu[b] + 128 b) / 128 * 128 on (tile-aligned, never overlapping the next one's).
   const int* cu;
+  // Packed sequences with more keys than queries (null: keys packed like the queries): sequence b's keys are rows
+  // cu_k[b] .. cu_k[b+1]-1 of k, v, dk, dv; koff and qshift are then derived per sequence, and sequence b owns the
+  // padded rows from (cu[b] + 384 b) / 128 * 128 on (a short first block and a ragged last one each need a tile more).
+  const int* cu_k;
   float scale, scale_log2;
 };
 
@@ -112,12 +116,26 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // this sequence: first row in the tensors, rows, blocks, first row in the padded per-head arrays
   const int row0 = p.cu ? __ldg(p.cu + b) : 0;
   const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
-  const int Nkeys = p.cu ? Nq : p.Nk;
-  const int T = p.cu ? (Nq + 127) / 128 : p.T;
+  const int krow0 = p.cu_k ? __ldg(p.cu_k + b) : row0;
+  const int Nkeys = p.cu_k ? __ldg(p.cu_k + b + 1) - krow0 : (p.cu ? Nq : p.Nk);
+  const int koff = p.cu_k ? (p.causal ? (Nkeys - Nq) / 128 : 0) : p.koff;
+  const int qshift = p.cu_k ? (p.causal ? (Nkeys - Nq) % 128 : 0) : p.qshift;
+  const int T = p.cu ? (Nq + qshift + 127) / 128 : p.T;
   const int bz = p.cu ? 0 : b;                         // outermost TMA coordinate
-  const int prow0 = p.cu ? ((row0 + 128 * b) / 128) * 128 : 0;
-  if (p.cu && j >= T) return;                          // (a sequence shorter than the longest one)
-  const int i0 = p.causal ? max(j - p.koff, 0) : 0;   // first query block that sees key block j
+  const int prow0 = p.cu ? ((row0 + (p.cu_k ? 384 : 128) * b) / 128) * 128 : 0;
+  if (p.cu && j >= (Nkeys + 127) / 128) return;        // (a sequence shorter than the longest one)
+  if (p.cu_k && (Nq <= 0 || (p.causal && Nkeys < Nq))) {
+    // keys without queries (or lengths the call does not allow): their gradients are zero
+    for (int x = threadIdx.x; x < 128 * (p.d / 8); x += blockDim.x) {
+      const int key = j * 128 + x / (p.d / 8), c = (x % (p.d / 8)) * 8;
+      if (key < Nkeys) {
+        *reinterpret_cast<uint4*>(p.dk + (int64_t)(krow0 + key) * p.dk_sn + (int64_t)hkv * p.dk_sh + c) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(p.dv + (int64_t)(krow0 + key) * p.dv_sn + (int64_t)hkv * p.dv_sh + c) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    return;
+  }
+  const int i0 = p.causal ? max(j - koff, 0) : 0;      // first query block that sees key block j
   const int ni = T - i0;
   const int n_tot = G * ni;
   int* status = p.status;
@@ -154,8 +172,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); tma_prefetch_desc(&tmDO);
       mbar_arrive_expect_tx(&kv_full, 2 * Cfg::kTileBytes);
       for (int pn = 0; pn < PAN; ++pn) {
-        tma_load_4d(sK + pn * 16384, &tmK, &kv_full, pn * 64, row0 + j * 128, hkv, bz);
-        tma_load_4d(sV + pn * 16384, &tmV, &kv_full, pn * 64, row0 + j * 128, hkv, bz);
+        tma_load_4d(sK + pn * 16384, &tmK, &kv_full, pn * 64, krow0 + j * 128, hkv, bz);
+        tma_load_4d(sV + pn * 16384, &tmV, &kv_full, pn * 64, krow0 + j * 128, hkv, bz);
       }
       bool ok = true;
       int issued = 0;
@@ -167,14 +185,14 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128 - p.qshift, hq, bz);
+          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128 - qshift, hq, bz);
         // dO of every tile is fetched ahead, retained or not (the vote comes too late to hide the copy behind it);
         // a skipped tile's stage is handed straight back by the issuer
         ok = mbar_wait(&do_empty[s], ((n >> 1) & 1) ^ 1, status);
         if (!ok) { mbar_wait(&q_full[s], (n >> 1) & 1, status); break; }
         mbar_arrive_expect_tx(&do_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, row0 + i * 128 - p.qshift, hq, bz);
+          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, row0 + i * 128 - qshift, hq, bz);
         issued = n + 1;
       }
       if (!ok) {
@@ -358,7 +376,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
         for (int e = 0; e < 32; ++e) sc[e] = ninf;
       }
-      if (p.causal && i + p.koff == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
+      if (p.causal && i + koff == j) {   // diagonal tile: entry (key rl, query col) is legal iff rl <= col
         const uint32_t ninf = 0xff800000u;
         const int c0 = qt * 32;
 #pragma unroll
@@ -499,8 +517,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (ok) {
       tc_fence_after();
       const int key = j * 128 + rl;
-      __nv_bfloat16* dvrow = p.dv + (int64_t)bz * p.dv_sb + (int64_t)(row0 + key) * p.dv_sn + (int64_t)hkv * p.dv_sh;
-      __nv_bfloat16* dkrow = p.dk + (int64_t)bz * p.dk_sb + (int64_t)(row0 + key) * p.dk_sn + (int64_t)hkv * p.dk_sh;
+      __nv_bfloat16* dvrow = p.dv + (int64_t)bz * p.dv_sb + (int64_t)(krow0 + key) * p.dv_sn + (int64_t)hkv * p.dv_sh;
+      __nv_bfloat16* dkrow = p.dk + (int64_t)bz * p.dk_sb + (int64_t)(krow0 + key) * p.dk_sn + (int64_t)hkv * p.dk_sh;
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
         __nv_bfloat16* out = which ? dkrow : dvrow;
@@ -618,7 +636,8 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
                                       const __nv_bfloat16* __restrict__ dout, int64_t d_sb, int64_t d_sn, int64_t d_sh,
                                       const float* __restrict__ lse, float* __restrict__ lse2, float* __restrict__ bq,
                                       float* __restrict__ Dq, int B, int Hq, int N, int Np, int Nk, int d, int causal,
-                                      float log2_tau, const int* __restrict__ cu, int total_rows, int Npg, int qshift) {
+                                      float log2_tau, const int* __restrict__ cu, int total_rows, int Npg, int qshift,
+                                      const int* __restrict__ cu_k) {
   const int warps_per_block = blockDim.x >> 5;
   const long long wi = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -628,16 +647,17 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
   const int h = (int)((wi / Npg) % Hq);
   int b = (int)(wi / ((long long)Npg * Hq));
   long long w = wi;                                  // index into the vectors
-  row -= qshift;                                     // the query this entry describes
   int row0 = 0;
   if (cu) {
     row0 = cu[b];
     N = cu[b + 1] - row0;
-    Nk = N;
-    if (row >= ((N + 127) / 128) * 128) return;      // beyond this sequence's padded rows
-    w = (long long)h * Np + ((row0 + 128 * b) / 128) * 128 + row;
+    Nk = cu_k ? cu_k[b + 1] - cu_k[b] : N;
+    if (cu_k) qshift = (causal && Nk >= N) ? (Nk - N) % 128 : 0;   // (per sequence)
+    if (row >= ((N + qshift + 127) / 128) * 128) return;           // beyond this sequence's padded rows
+    w = (long long)h * Np + ((row0 + (cu_k ? 384 : 128) * b) / 128) * 128 + row;
     b = 0;
   }
+  row -= qshift;                                     // the query this entry describes
   if (row < 0 || row >= N) {
     if (lane == 0) { lse2[w] = INFINITY; bq[w] = INFINITY; Dq[w] = 0.f; }
     return;
@@ -667,7 +687,8 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ o, int64
 // [Hq, Np, d] with sequence b's tiles from (cu[b] + 128 b) / 128 on.)
 __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int64_t sb,
                                       int64_t sn, int64_t sh, int B, int Hq, int N, int Np, int d, float scale,
-                                      const int* __restrict__ cu, int Npg, int qshift, int d_out) {
+                                      const int* __restrict__ cu, int Npg, int qshift, int d_out,
+                                      const int* __restrict__ cu_k, int causal) {
   // d: columns of the accumulator (the padded head size); d_out <= d: columns of dq
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int per_row = d / 8;
@@ -680,12 +701,20 @@ __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat
   const int i = (int)(tile % T);
   const int h = (int)((tile / T) % Hq);
   int b = (int)(tile / ((long long)T * Hq));
-  int row = i * 128 + r - qshift;                          // (qshift != 0 only without cu)
+  int row = i * 128 + r;
   if (cu) {
     const int row0 = cu[b];
     N = cu[b + 1] - row0;
-    if (row >= N) return;
-    tile = (long long)h * (Np / 128) + (row0 + 128 * b) / 128 + i;
+    if (cu_k) {
+      const int Nk = cu_k[b + 1] - cu_k[b];
+      qshift = (causal && Nk >= N) ? (Nk - N) % 128 : 0;   // (per sequence)
+    }
+  }
+  row -= qshift;
+  if (cu) {
+    const int row0 = cu[b];
+    if (row < 0 || row >= N) return;
+    tile = (long long)h * (Np / 128) + (row0 + (cu_k ? 384 : 128) * b) / 128 + i;
     row += row0;
     N += row0;
     b = 0;
@@ -739,15 +768,16 @@ inline int bwd_launch_main(const CUtensorMap& tq, const CUtensorMap& tk, const C
 inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
                       mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int Nk, int d,
                       int causal, float scale, float tau, void* ws, int* status, cudaStream_t stream,
-                      const int* cu = nullptr, int total = 0) {
+                      const int* cu = nullptr, int total = 0, const int* cu_k = nullptr, int total_k = 0) {
   // Packed sequences (cu): N = Nk = the longest sequence; the tensors are [1, total, H, d]; the per-query vectors and
   // the dQ accumulator are laid out per head over Np = total + 128 B rows (rounded up to a tile).
   const int D = padded_head_size(d);         // columns of the kernels and of the dQ accumulator
   const int qshift = (causal && !cu) ? (Nk - N) % 128 : 0;
-  const int T = (N + qshift + 127) / 128, Npg = T * 128, Tk = (Nk + 127) / 128;
-  const int Np = cu ? ((total + 128 * B + 127) / 128) * 128 : Npg;
+  // (cu_k: every sequence has its own shift below 128, so the longest one may span a block more than its rows fill)
+  const int T = (N + (cu_k ? 127 : qshift) + 127) / 128, Npg = T * 128, Tk = (Nk + 127) / 128;
+  const int Np = cu ? ((total + (cu_k ? 384 : 128) * B + 127) / 128) * 128 : Npg;
   const int Bl = cu ? 1 : B;                 // batch extent of the tensors and of the workspace arrays
-  const int Nt = cu ? total : N, Nkt = cu ? total : Nk;   // row extents of the tensors
+  const int Nt = cu ? total : N, Nkt = cu ? (cu_k ? total_k : total) : Nk;   // row extents of the tensors
   uint8_t* w = (uint8_t*)ws;
   float* acc = (float*)w;
   w += bwd_align256((size_t)Bl * Hq * Np * D * sizeof(float));
@@ -776,7 +806,8 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   p.status = status;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.N = N; p.Np = Np; p.T = T; p.words = (T + 31) / 32; p.causal = causal;
   p.Nk = Nk; p.Tk = Tk; p.koff = causal ? (Nk - N) / 128 : 0; p.qshift = qshift;
-  p.cu = cu; p.d = d;
+  p.cu = cu; p.cu_k = cu_k; p.d = d;
+  if (cu_k) { p.koff = 0; p.qshift = 0; }    // per sequence, on the device
   p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
   if (p.bitmask &&
       cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * Tk * p.words * sizeof(uint32_t), stream) != cudaSuccess)
@@ -789,7 +820,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     bwd_preprocess_kernel<<<blocks, wpb * 32, 0, stream>>>((const __nv_bfloat16*)o.p, o.sb, o.sn, o.sh,
                                                           (const __nv_bfloat16*)dout.p, dout.sb, dout.sn, dout.sh, lse,
                                                           lse2, bq, Dq, B, Hq, N, Np, Nk, d, causal,
-                                                          tau > 0.f ? log2f(tau) : -INFINITY, cu, total, Npg, qshift);
+                                                          tau > 0.f ? log2f(tau) : -INFINITY, cu, total, Npg, qshift, cu_k);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   const bool dense = (tau == 0.f);
@@ -801,7 +832,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     const long long n_out = (long long)B * Hq * Npg * (D / 8);
     const unsigned blocks = (unsigned)((n_out + 255) / 256);
     bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(acc, (__nv_bfloat16*)dq.p, dq.sb, dq.sn, dq.sh, B, Hq, N, Np, D,
-                                                      scale, cu, Npg, qshift, d);
+                                                      scale, cu, Npg, qshift, d, cu_k, causal);
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   return MALA_OK;

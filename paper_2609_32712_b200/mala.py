@@ -65,6 +65,9 @@ def lib():
         L.mala_fwd_varlen_prefix.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i,
                                              i, i, i, f, f, vp, sz, vp]
         L.mala_fwd_varlen_prefix.restype = i
+        L.mala_bwd_varlen_prefix.argtypes = [_TIn, _TIn, _TIn, _TIn, _TIn, vp, vp, vp, _TOut, _TOut, _TOut,
+                                             ctypes.POINTER(_Stats), i, i, i, i, i, i, i, i, i, f, f, vp, sz, vp]
+        L.mala_bwd_varlen_prefix.restype = i
         L.mala_fwd_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, i,
                                      i, i, f, f, vp, sz, vp]
         L.mala_fwd_paged.restype = i
@@ -319,6 +322,28 @@ def bwd_varlen(q, k, v, o, do, lse, cu_seqlens, max_seqlen: int, scale: float, t
                                int(causal), scale, tau, ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_bwd_varlen")
+    return dq, dk, dv, st
+
+
+def bwd_varlen_prefix(q, k, v, o, do, lse, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int,
+                      scale: float, tau: float, causal: bool = True, stats: bool = False, ws=None):
+    """mala_bwd_varlen_prefix: returns (dq [1,total_q,Hq,d], dk, dv [1,total_k,Hkv,d], Stats or None)."""
+    one, total_q, Hq, d = q.shape
+    total_k, Hkv = k.shape[1], k.shape[2]
+    for cu in (cu_seqlens_q, cu_seqlens_k):
+        assert cu.dtype == torch.int32 and cu.is_contiguous()
+    B = cu_seqlens_q.numel() - 1
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    Tq, Tk = -(-(max_seqlen_q + 127) // 128), -(-max_seqlen_k // 128)
+    st = Stats((B, Hq, Tk), -(-Tq // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_BWD, 1, Hq, Hkv, total_q + 384 * B, d), q.device) if ws is None else ws
+    rc = lib().mala_bwd_varlen_prefix(_view(q, _TIn), _view(k, _TIn), _view(v, _TIn), _view(o, _TIn), _view(do, _TIn),
+                                      lse.data_ptr(), cu_seqlens_q.data_ptr(), cu_seqlens_k.data_ptr(),
+                                      _view(dq, _TOut), _view(dk, _TOut), _view(dv, _TOut),
+                                      ctypes.byref(st.c) if st else None, B, Hq, Hkv, total_q, total_k, max_seqlen_q,
+                                      max_seqlen_k, d, int(causal), scale, tau, ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_bwd_varlen_prefix")
     return dq, dk, dv, st
 
 

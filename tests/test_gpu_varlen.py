@@ -165,6 +165,66 @@ def test_varlen_with_cached_prefixes(mala, oracle, tau, causal):
     assert st.totals.cpu().numpy()[1] == legal
     if tau > 0 and causal:
         assert skipped > 0
+    # backward on the GPU's own forward output: every sequence against the oracle's chunk backward
+    do = torch.cat([w["do"][:, n - m:] for w, n, m in zip(ws, nk, nq)], dim=1).contiguous()
+    dq, dk, dv, bst = mala.bwd_varlen_prefix(q.cuda(), k.cuda(), v.cuda(), o, do.cuda(), lse, cq.cuda(), ck.cuda(),
+                                             max(nq), max(nk), ws[0]["scale"], tau, causal=causal, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    Tqm = -(-(max(nq) + 127) // 128)
+    bm = bst.mask(Tqm).cpu().numpy()                     # [B,Hq,Tkm,Tqm]
+    legal_b = 0
+    for b, (w, n, m) in enumerate(zip(ws, nk, nq)):
+        shift = (n - m) % 128 if causal else 0
+        r0, k0 = int(cq[b]), int(ck[b])
+        rb = oracle.bwd(w["q"][:, n - m:], w["k"], w["v"], o[:, r0:r0 + m].float().cpu(), w["do"][:, n - m:],
+                        lse_c[None, :, r0:r0 + m], w["scale"], tau, 128, 128, causal=causal, q_shift=shift)
+        Tk, Tq = rb["mask"].shape[2], rb["mask"].shape[3]
+        for h in range(Hq):
+            for j in range(Tk):
+                om, oc = rb["mask"][0, h, j], rb["crit"][0, h, j]
+                for i in range(Tq):
+                    if om[i] == 0:
+                        assert not bm[b, h, j, i]
+                    elif bool(bm[b, h, j, i]) != (om[i] == 2):
+                        assert abs(oc[i]) <= parity.MASK_BAND, (b, h, j, i, oc[i])
+            assert not bm[b, h, Tk:].any() and not bm[b, h, :, Tq:].any()
+        if m > 1:
+            parity.check_grad(dq[0, r0:r0 + m].float().cpu().numpy(), rb["dq"][0], "dq")
+        else:     # (a single query: its gradient may be exactly zero, see the packed test above)
+            assert np.abs(dq[0, r0:r0 + m].float().cpu().numpy() - rb["dq"][0]).max() <= 1e-2 * max(np.abs(rb["dq"]).max(), 1e-3)
+        parity.check_grad(dk[0, k0:k0 + n].float().cpu().numpy(), rb["dk"][0], "dk")
+        parity.check_grad(dv[0, k0:k0 + n].float().cpu().numpy(), rb["dv"][0], "dv")
+        legal_b += int((rb["mask"] > 0).sum())
+    assert bst.totals.cpu().numpy()[1] == legal_b
+
+
+def test_varlen_prefix_backward_sequences_without_queries_get_zero_gradients(mala):
+    Hq, Hkv, d = 2, 1, 64
+    nk, nq = [300, 200, 140], [100, 0, 140]
+    w = W.custom_prefill(1, Hq, Hkv, sum(nk), d, seed=88)
+    q = w["q"][:, :sum(nq)].contiguous().cuda()
+    do = w["do"][:, :sum(nq)].contiguous().cuda()
+    k, v = w["k"].cuda(), w["v"].cuda()
+    cq = torch.tensor(np.concatenate([[0], np.cumsum(nq)]), dtype=torch.int32).cuda()
+    ck = torch.tensor(np.concatenate([[0], np.cumsum(nk)]), dtype=torch.int32).cuda()
+    o, lse, _ = mala.fwd_varlen_prefix(q, k, v, cq, ck, max(nq), max(nk), w["scale"], 1e-4)
+    dq, dk, dv, _ = mala.bwd_varlen_prefix(q, k, v, o, do, lse, cq, ck, max(nq), max(nk), w["scale"], 1e-4)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert (dk[0, 300:500] == 0).all() and (dv[0, 300:500] == 0).all()
+    assert dk[0, :300].float().abs().max() > 0 and dk[0, 500:].float().abs().max() > 0
+    # the neighbours are what separate calls give
+    for b, (r0, k0) in enumerate([(0, 0), (100, 300), (100, 500)]):
+        if nq[b] == 0:
+            continue
+        qs, ks, vs = q[:, r0:r0 + nq[b]], k[:, k0:k0 + nk[b]], v[:, k0:k0 + nk[b]]
+        o1, l1, _ = mala.fwd_chunk(qs.contiguous(), ks.contiguous(), vs.contiguous(), w["scale"], 1e-4)
+        g = mala.bwd_chunk(qs.contiguous(), ks.contiguous(), vs.contiguous(), o1, do[:, r0:r0 + nq[b]].contiguous(), l1,
+                           w["scale"], 1e-4)
+        assert torch.equal(o1, o[:, r0:r0 + nq[b]])
+        assert torch.equal(g[1], dk[:, k0:k0 + nk[b]]) and torch.equal(g[2], dv[:, k0:k0 + nk[b]])
+        assert (g[0].float() - dq[:, r0:r0 + nq[b]].float()).abs().max() <= 1e-2 * g[0].float().abs().max()
 
 
 @pytest.mark.parametrize("tau", [0.0, 1e-4])

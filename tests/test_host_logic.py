@@ -120,6 +120,11 @@ def test_argument_validation_codes_of_the_general_shape_calls(mala):
     fp = lambda cq, ck, mq=128, mk=256: L.mala_fwd_varlen_prefix(tin(), tin(), tin(), cq, ck, tout(), base, None, 2, 2, 2, 256,
                                                                  512, mq, mk, 128, 1, 0.1, 1e-4, None, 0, None)
     assert fp(None, base) == -1 and fp(base, None) == -1 and fp(base, base, mq=256, mk=128) == -2
+    bp = lambda cq, ck, mq=128, mk=256, n=1 << 30: L.mala_bwd_varlen_prefix(
+        tin(), tin(), tin(), tin(), tin(), base, cq, ck, tout(), tout(), tout(), None, 2, 2, 2, 256, 512, mq, mk, 128, 1, 0.1,
+        1e-4, base, n, None)
+    assert bp(None, base) == -1 and bp(base, None) == -1 and bp(base, base, mq=256, mk=128) == -2
+    assert bp(base, base, n=1024) == -4        # scratch for total_q + 384 B rows
     fg = lambda page=128, bt=base, sl=base: L.mala_fwd_paged(tin(), tin(), tin(), base, bt, sl, tout(), base, None, 2, 2, 2, 256,
                                                              128, 8, page, 4, 128, 1, 0.1, 1e-4, None, 0, None)
     assert fg(page=64) == -2 and fg(bt=None) == -1 and fg(sl=None) == -1 and fg(bt=base + 2) == -3
