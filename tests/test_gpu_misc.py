@@ -172,3 +172,38 @@ def test_autograd_function_runs_both_algorithms(mala, oracle):
     parity.check_grad(q.grad.float().cpu().numpy(), gq, "dq")
     parity.check_grad(k.grad.float().cpu().numpy(), gk, "dk")
     parity.check_grad(v.grad.float().cpu().numpy(), gv, "dv")
+
+
+def test_autograd_functions_for_chunks_and_packed_sequences(mala):
+    from paper_2609_32712_b200.autograd import mala_attention, mala_attention_packed
+    w = W.custom_prefill(1, 4, 2, 900, 96, head_types=["diffuse", "peaked", "peaked", "sink"], seed=43, preset="R")
+    tau, Nq = 1e-4, 333
+    # a chunk of queries from a position inside a tile
+    q = w["q"][:, 900 - Nq:].cuda().requires_grad_(True)
+    k, v = (w[x].cuda().requires_grad_(True) for x in ("k", "v"))
+    do = w["do"][:, 900 - Nq:].cuda()
+    o = mala_attention(q, k, v, tau, scale=w["scale"])
+    o.backward(do)
+    o_d, lse_d, _ = mala.fwd_chunk(q.detach(), k.detach(), v.detach(), w["scale"], tau)
+    dq, dk, dv, _ = mala.bwd_chunk(q.detach(), k.detach(), v.detach(), o_d, do, lse_d, w["scale"], tau)
+    assert torch.equal(o.detach(), o_d) and torch.equal(k.grad, dk) and torch.equal(v.grad, dv)
+    assert (q.grad.float() - dq.float()).abs().max() <= 1e-2 * dq.float().abs().max()
+    # two packed sequences, the second behind a prefix
+    nq, nk = [200, 100], [200, 700]
+    qp = torch.cat([w["q"][:, :200], w["q"][:, 800:900]], dim=1).contiguous().cuda().requires_grad_(True)
+    kp = torch.cat([w["k"][:, :200], w["k"][:, 200:900]], dim=1).contiguous().cuda().requires_grad_(True)
+    vp = torch.cat([w["v"][:, :200], w["v"][:, 200:900]], dim=1).contiguous().cuda().requires_grad_(True)
+    dop = torch.cat([w["do"][:, :200], w["do"][:, 800:900]], dim=1).contiguous().cuda()
+    cq = torch.tensor([0, 200, 300], dtype=torch.int32, device="cuda")
+    ck = torch.tensor([0, 200, 900], dtype=torch.int32, device="cuda")
+    op = mala_attention_packed(qp, kp, vp, cq, ck, max(nq), max(nk), tau, scale=w["scale"])
+    op.backward(dop)
+    for b in range(2):
+        qs = qp.detach()[:, int(cq[b]):int(cq[b + 1])].contiguous()
+        ks, vs = (t.detach()[:, int(ck[b]):int(ck[b + 1])].contiguous() for t in (kp, vp))
+        o1, l1, _ = mala.fwd_chunk(qs, ks, vs, w["scale"], tau)
+        g = mala.bwd_chunk(qs, ks, vs, o1, dop[:, int(cq[b]):int(cq[b + 1])].contiguous(), l1, w["scale"], tau)
+        assert torch.equal(o1, op.detach()[:, int(cq[b]):int(cq[b + 1])])
+        assert torch.equal(g[1], kp.grad[:, int(ck[b]):int(ck[b + 1])]) and torch.equal(g[2], vp.grad[:, int(ck[b]):int(ck[b + 1])])
+        assert (g[0].float() - qp.grad[:, int(cq[b]):int(cq[b + 1])].float()).abs().max() <= 1e-2 * g[0].float().abs().max()
+    assert mala.device_status() == 0
