@@ -936,3 +936,42 @@ def test_bwd_of_a_chunk_from_any_position_matches_bruteforce(Nq, Nk, Bq, Bk, tau
     r2 = slice(2 * Bq - shift, min(Nq, 3 * Bq - shift))
     assert np.allclose(part["dq"][0, r0, 0], dQ[r0], atol=1e-11) and np.allclose(part["dq"][0, r2, 0], dQ[r2], atol=1e-11)
     assert np.allclose(part["dk"][0, Bk:2 * Bk, 0], dK[Bk:2 * Bk], atol=1e-11)
+
+
+# ------------------------------------------------------------------ matched-work diagnostics (analysis on the oracle)
+def test_matched_work_controls():
+    from oracle import matched_work as mw
+    B, N, Hq, Hkv, d, Bq, Bk, tau = 3, 96, 4, 2, 16, 8, 8, 0.3
+    q, k, v = peaky_inputs(N, d, 501, Hq=Hq, Hkv=Hkv, B=B, boost=3.0)
+    q[:, :, 0] *= 0.3                                            # one diffuse head: the heads' counts differ
+    scale = 1.0 / math.sqrt(d)
+    res = mw.matched_work(q, k, v, scale, tau, Bq, Bk)
+    f = orc.fwd(q, k, v, scale, tau, Bq, Bk)
+    assert res["tiles"] == int((f["mask"] == orc.RETAINED).sum()) and (f["mask"] == orc.SKIPPED).sum() > 0
+    # MALA's omitted mass from the tile masses of the dense softmax = 1 - exp(lse_screened - lse_reference)
+    _, lse_ref = orc.dense_fwd(q, k, v, scale)
+    om = 1.0 - np.exp(f["lse"] - lse_ref)                        # [B,Hq,N]
+    assert np.allclose(res["mala_per_block"], om.reshape(B, Hq, N // Bq, Bq).mean(axis=3), atol=1e-12)
+    assert 0 < res["mala"] <= tau / (1 + tau)
+    # every policy spends exactly MALA's number of tiles
+    for p_ in ("per_instance", "static", "position_only"):
+        assert int(res["budgets"][p_].sum()) == res["tiles"]
+    # with MALA's own count per decision, keeping the heaviest tiles cannot omit more (block sums) than MALA does
+    assert (res["per_instance_per_block"] <= res["mala_per_block"] + 1e-12).all()
+    assert res["per_instance"] <= res["mala"] and res["per_instance"] <= res["static"] + 1e-12
+    # brute force of the per-instance control on one decision
+    b, h, i = 1, 2, 7
+    S = scale * (q[b, :, h] @ k[b, :, h // 2].T)
+    S[np.triu_indices(N, 1)] = -np.inf
+    P = np.exp(S - S.max(axis=1, keepdims=True))
+    P /= P.sum(axis=1, keepdims=True)
+    rows = P[i * Bq:(i + 1) * Bq]
+    mass = [rows[:, j * Bk:(j + 1) * Bk].sum() for j in range(i + 1)]
+    n = int((f["mask"][b, h, i] == orc.RETAINED).sum())
+    best = sorted(mass, reverse=True)[:n]
+    assert abs(res["per_instance_per_block"][b, h, i] - (1.0 - sum(best) / Bq)) < 1e-12
+    # tau = 0: nothing omitted by anyone; one batch entry: the static control is the per-instance one
+    z = mw.matched_work(q, k, v, scale, 0.0, Bq, Bk)
+    assert max(abs(z[p_]) for p_ in ("mala", "per_instance", "static", "position_only")) < 1e-12
+    one = mw.matched_work(q[:1], k[:1], v[:1], scale, tau, Bq, Bk)
+    assert np.array_equal(one["budgets"]["static"], one["budgets"]["per_instance"])
