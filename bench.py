@@ -297,6 +297,34 @@ def varlen_leg(cfg, preset, lens, tau, it, peaks, dev):
     return row
 
 
+def head_size_leg(cfg, preset, d, tau, it, peaks, dev):
+    """The configuration's shapes with another head size (it runs on the next wider kernel, with zero-filled columns):
+    latency of the MALA and dense kernels and the tensor-pipe fraction counted on the d columns that carry data."""
+    import torch
+    from paper_2609_32712_b200 import mala, workloads as W
+    w = W.custom_prefill(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, d, head_types=cfg.head_types, seed=cfg.seed, preset=preset, device=dev)
+    q, k, v, do = w["q"], w["k"], w["v"], w["do"]
+    wsb = torch.empty(mala.workspace_bytes(mala.OP_BWD, cfg.B, cfg.Hq, cfg.Hkv, cfg.N, d), dtype=torch.uint8, device=dev)
+    taus = {"mala": tau, "dense": 0.0}
+    outs = {lab: mala.fwd(q, k, v, w["scale"], t_)[:2] for lab, t_ in taus.items()}
+    fwd = {lab: (lambda t_=t_: mala.fwd(q, k, v, w["scale"], t_)) for lab, t_ in taus.items()}
+    bwd = {lab: (lambda t_=t_, lab=lab: mala.bwd(q, k, v, outs[lab][0], do, outs[lab][1], w["scale"], t_, ws=wsb))
+           for lab, t_ in taus.items()}
+    f_t, b_t = time_alternating(fwd, 3, it), time_alternating(bwd, 3, it)
+    row = {"d": d}
+    for label in taus:
+        row[label] = {"fwd_ms": f_t[label], "bwd_ms": b_t[label]}
+    _, _, fs = mala.fwd(q, k, v, w["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    fr, fl = fs.totals.cpu().tolist()
+    row["fwd_retained_frac"] = fr / fl
+    row["dense_fwd_tensor_frac_on_d_columns"] = (fwd_executed_flops(fl, fl, d) / (f_t["dense"] * 1e-3) / 1e12
+                                                 / peaks["tflops_sustained"])
+    row["dense_bwd_tensor_frac_on_d_columns"] = (bwd_executed_flops(fl, fl, d) / (b_t["dense"] * 1e-3) / 1e12
+                                                 / peaks["tflops_sustained"])
+    return row
+
+
 def serving_prefill_leg(cfg, preset, tau, it, peaks, dev):
     """A serving-style prefill batch with the heads of a prefill configuration: eight sequences, a 2048-token chunk each
     behind prefixes of 0 ... 30720 tokens, packed (mala_fwd_varlen_prefix) and against a paged cache (mala_fwd_paged,
@@ -648,6 +676,8 @@ def main():
                     row["varlen_4seq_32768"] = varlen_leg(cc, preset, (16384, 8192, 5000, 3192), tau, it, peaks, dev)
                 if name == "cfg3":                  # a serving-style batch of prefill chunks behind cached prefixes
                     row["serving_prefill_8x2048"] = serving_prefill_leg(cc, preset, tau, it, peaks, dev)
+                if name == "cfg3":                  # the same shapes with 96-column heads (run on the 128-column kernels)
+                    row["head_size_96"] = head_size_leg(cc, preset, 96, tau, it, peaks, dev)
                 if name == "cfg3" and preset == "R":
                     row["fidelity_vs_dense"] = fidelity(cs, (1e-4, 1e-2, 1.0), it)
                 detail[f"{name}_{preset}"] = row
