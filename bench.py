@@ -328,7 +328,7 @@ def head_size_leg(cfg, preset, d, tau, it, peaks, dev):
 def serving_prefill_leg(cfg, preset, tau, it, peaks, dev):
     """A serving-style prefill batch with the heads of a prefill configuration: eight sequences, a 2048-token chunk each
     behind prefixes of 0 ... 30720 tokens, packed (mala_fwd_varlen_prefix) and against a paged cache (mala_fwd_paged,
-    256-key pages in a shuffled pool): latency of the MALA and dense kernels, tensor-pipe fraction on executed work."""
+    256-key and 16-key pages in a shuffled pool): latency of the MALA and dense kernels, tensor-pipe fraction on executed work."""
     import torch
     from paper_2609_32712_b200 import mala, workloads as W
     prefixes, chunk = (30720, 16384, 8192, 4096, 2048, 1000, 300, 0), 2048
@@ -347,6 +347,7 @@ def serving_prefill_leg(cfg, preset, tau, it, peaks, dev):
     for b, (w, n) in enumerate(zip(ws, nk)):
         kc[b, :n], vc[b, :n] = w["k"][0], w["v"][0]
     kp, vp, bt, sl = W.paginate(kc, vc, 256, seqlens=nk, seed=11)
+    kp16, vp16, bt16, sl16 = W.paginate(kc, vc, 16, seqlens=nk, seed=12)
     del kc, vc, ws
     row = {"prefixes": list(prefixes), "chunk": chunk}
     taus = {"mala": tau, "dense": 0.0}
@@ -354,11 +355,13 @@ def serving_prefill_leg(cfg, preset, tau, it, peaks, dev):
                                for lab, t_ in taus.items()}, 3, it)
     paged = time_alternating({lab: (lambda t_=t_: mala.fwd_paged(q, kp, vp, cq, bt, sl, chunk, scale, t_))
                               for lab, t_ in taus.items()}, 3, it)
+    paged16 = time_alternating({lab: (lambda t_=t_: mala.fwd_paged(q, kp16, vp16, cq, bt16, sl16, chunk, scale, t_))
+                                for lab, t_ in taus.items()}, 3, it)
     _, _, st = mala.fwd_varlen_prefix(q, k, v, cq, ck, chunk, max(nk), scale, tau, stats=True)
     torch.cuda.synchronize()
     ret, leg = st.totals.cpu().tolist()
     for lab in taus:
-        row[lab] = {"packed_ms": packed[lab], "paged_ms": paged[lab]}
+        row[lab] = {"packed_ms": packed[lab], "paged_ms": paged[lab], "paged_16key_pages_ms": paged16[lab]}
     row["legal_tiles"], row["retained_frac"] = leg, ret / leg
     row["tensor_frac_on_executed"] = (fwd_executed_flops(leg, ret, cfg.d) / (packed["mala"] * 1e-3) / 1e12
                                       / peaks["tflops_sustained"])

@@ -166,7 +166,8 @@ int mala_bwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_
 /* mala_fwd_varlen_prefix with the keys and values held in pages: a batch of prefill chunks behind prefixes that
  * live in a paged cache (the chunks' own keys and values already written to their pages).  q, o [1,total_q,Hq,d]
  * packed by cu_seqlens_q (device int32 [B+1]); kpages, vpages [num_pages, page_size, Hkv, d] with page_size a multiple
- * of 128; block_table device int32 [B, max_pages_per_seq] (keys page_size*x .. of sequence b in page
+ * of 128, or 8, 16, 32 or 64 (a tile is then put together from 128 / page_size pages, each with its own table
+ * lookup, at reduced throughput); block_table device int32 [B, max_pages_per_seq] (keys page_size*x .. of sequence b in page
  * block_table[b][x]); seqlens_k device int32 [B], the keys sequence b holds, its queries being its last positions
  * (a sequence with no keys, or with fewer keys than queries when causal != 0, is left untouched).  Slots of a mapped
  * page beyond the sequence's length must hold finite numbers.  Everything else as mala_fwd_varlen_prefix with

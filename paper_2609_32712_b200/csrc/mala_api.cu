@@ -67,6 +67,10 @@ static int device_setup(int dev, int** status_out) {
     ok = ok && set_smem(mala_fwd_kernel<128, false>, FwdCfg<128, false>::kSmemBytes);
     ok = ok && set_smem(mala_fwd_kernel<64, false>, FwdCfg<64, false>::kSmemBytes);
     ok = ok && set_smem(mala_fwd_kernel<64, true>, FwdCfg<64, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<128, true, true>, FwdCfg<128, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<128, false, true>, FwdCfg<128, false>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<64, false, true>, FwdCfg<64, false>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<64, true, true>, FwdCfg<64, true>::kSmemBytes);
     ok = ok && bwd_set_attributes();
     ok = ok && decode_set_attributes();
     if (!ok) return MALA_ERR_CUDA;
@@ -111,7 +115,10 @@ template <int D, bool kDense>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                       cudaStream_t stream) {
   dim3 grid((p.Tr + 1) / 2, p.Hq, p.B * (p.num_splits > 1 ? p.num_splits : 1));
-  mala_fwd_kernel<D, kDense><<<grid, FwdCfg<D, kDense>::kThreads, FwdCfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
+  if (p.ppt > 1)
+    mala_fwd_kernel<D, kDense, true><<<grid, FwdCfg<D, kDense>::kThreads, FwdCfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
+  else
+    mala_fwd_kernel<D, kDense><<<grid, FwdCfg<D, kDense>::kThreads, FwdCfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
@@ -238,9 +245,10 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   cudaStream_t stream = (cudaStream_t)cuda_stream;
 
   CUtensorMap tq, tk, tv;
+  const int box_rows = (pg && pg->page_size < 128) ? pg->page_size : 128;   // pages smaller than a tile: one copy per page
   if (!make_tensor_map_bnhd(&tq, q.p, Bt, Nt, Hq, d, q.sb, q.sn, q.sh, 128) ||
-      !make_tensor_map_bnhd(&tk, k.p, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv, d, k.sb, k.sn, k.sh, 128) ||
-      !make_tensor_map_bnhd(&tv, v.p, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv, d, v.sb, v.sn, v.sh, 128))
+      !make_tensor_map_bnhd(&tk, k.p, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv, d, k.sb, k.sn, k.sh, box_rows) ||
+      !make_tensor_map_bnhd(&tv, v.p, pg ? pg->num_pages : Bt, pg ? pg->page_size : Nkt, Hkv, d, v.sb, v.sn, v.sh, box_rows))
     return MALA_ERR_TENSOR_MAP;
 
   const int D = padded_head_size(d);
@@ -250,7 +258,8 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
   p.block_table = pg ? pg->block_table : nullptr;
   p.seqlens_k = pg ? pg->seqlens_k : nullptr;
   p.bt_stride = pg ? pg->max_pages_per_seq : 0;
-  p.tpp = pg ? pg->page_size / 128 : 1;
+  p.tpp = (pg && pg->page_size >= 128) ? pg->page_size / 128 : 1;
+  p.ppt = 128 / box_rows; p.prows = box_rows;
   p.num_splits = num_splits;
   p.tps = ((Nk + 127) / 128 + num_splits - 1) / num_splits;
   p.o_part = num_splits > 1 ? (float*)ws : nullptr;
@@ -397,7 +406,10 @@ int mala_fwd_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* 
   MALA_TRY(check_packed(cu_seqlens_q, B, total_q, max_seqlen_q));
   if (!block_table || !seqlens_k || num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0) return MALA_ERR_INVALID_ARG;
   if ((((uintptr_t)block_table) & 3) != 0 || (((uintptr_t)seqlens_k) & 3) != 0) return MALA_ERR_MISALIGNED;
-  if (page_size % 128 != 0 || (long long)max_pages_per_seq * page_size > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
+  // pages of whole tiles, or 8, 16, 32 or 64 keys (a tile is then put together from several pages)
+  if (page_size < 8 || (page_size % 128 != 0 && 128 % page_size != 0) ||
+      (long long)max_pages_per_seq * page_size > 0x7fffffffLL)
+    return MALA_ERR_UNSUPPORTED;
   const int max_k = max_pages_per_seq * page_size;
   if (causal && max_k < max_seqlen_q) return MALA_ERR_UNSUPPORTED;
   FwdPaging pg;

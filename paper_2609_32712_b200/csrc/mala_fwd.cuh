@@ -46,6 +46,10 @@ struct FwdParams {
   const int* block_table;
   const int* seqlens_k;
   int bt_stride, tpp;
+  // Pages smaller than a tile (8, 16, 32 or 64 keys): ppt = 128 / page_size copies of prows = page_size rows make
+  // up a tile, copy c of key block x from page block_table[b * bt_stride + x * ppt + c] (tpp = 1 then; a table
+  // entry past the row's end reads as "no page": zeros).  ppt = 1 otherwise.
+  int ppt, prows;
   const int* cu_k;               // packed sequences whose keys are longer than their queries (a cached prefix): the keys
                                  // of sequence b are rows cu_k[b] .. cu_k[b+1]-1 of k, v; its queries are the last
                                  // positions (null: keys as queries)
@@ -71,7 +75,9 @@ struct FwdCfg {
   static constexpr uint32_t kTmemCols = 512;
 };
 
-template <int D, bool kDense>
+// kSmall: the keys and values lie in pages smaller than a tile (a kernel of its own, so that the copy loop with its
+// table lookups costs the other layouts nothing).
+template <int D, bool kDense, bool kSmall = false>
 __global__ void __launch_bounds__(384, 1)
 mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const FwdParams p) {
@@ -115,6 +121,15 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       row = krow0 + jt * 128;
     }
   };
+  auto load_tile_small = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int jt) {
+    for (int c = 0; c < p.ppt; ++c) {
+      const int pg = jt * p.ppt + c;
+      const int outer = pg < p.bt_stride ? __ldg(p.block_table + (size_t)b * p.bt_stride + pg) : -1;
+#pragma unroll
+      for (int pn = 0; pn < D / 64; ++pn) tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, outer);
+    }
+  };
+  constexpr bool small_pages = kSmall;
   const int Tr = p.cu ? (Nq + qshift + 127) / 128 : p.Tr;
   const int Tk = p.cu ? (Nkeys + 127) / 128 : p.Tk;
   const int bz = p.cu ? 0 : b;                        // outermost TMA coordinate
@@ -179,21 +194,25 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
       bool ok = true;
       for (int u = 0; u < U && ok; ++u) {
-        int krow, kouter;
-        key_coord(j0 - u, krow, kouter);   // (a page lookup is in flight while the stage is waited for)
+        int krow = 0, kouter = 0;
+        if (!small_pages) key_coord(j0 - u, krow, kouter);   // (a page lookup is in flight while the stage is waited for)
         ok = mbar_wait(&k_empty[s], par, status);
         if (!ok) break;
         mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
-        for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, krow, hkv, kouter);
+        if (small_pages) load_tile_small(sK + s * Cfg::kTileBytes, &tmK, &k_full[s], j0 - u);
+        else
+          for (int pn = 0; pn < PAN; ++pn)
+            tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, krow, hkv, kouter);
         issued = u + 1;
         if (++s == KS) { s = 0; par ^= 1; }
         if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
           ok = mbar_wait(&v_empty[u & 1], ((u >> 1) & 1) ^ 1, status);
           if (!ok) break;
           mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
-          for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow, hkv, kouter);
+          if (small_pages) load_tile_small(sV + (u & 1) * Cfg::kTileBytes, &tmV, &v_full[u & 1], j0 - u);
+          else
+            for (int pn = 0; pn < PAN; ++pn)
+              tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow, hkv, kouter);
           v_issued = u + 1;
         }
       }
@@ -277,11 +296,15 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             ok = mbar_wait_warp(&v_empty[x], (r & 1) ^ 1, status);
             if (!ok) break;
             if (leader) {
-              int vrow, vouter;
-              key_coord(j0 - u, vrow, vouter);
               mbar_arrive_expect_tx(&v_full[x], Cfg::kTileBytes);
-              for (int pn = 0; pn < PAN; ++pn)
-                tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, vrow, hkv, vouter);
+              if (small_pages) {
+                load_tile_small(sV + x * Cfg::kTileBytes, &tmV, &v_full[x], j0 - u);
+              } else {
+                int vrow, vouter;
+                key_coord(j0 - u, vrow, vouter);
+                for (int pn = 0; pn < PAN; ++pn)
+                  tma_load_4d(sV + x * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[x], pn * 64, vrow, hkv, vouter);
+              }
             }
             __syncwarp();
           }

@@ -228,7 +228,7 @@ def test_varlen_prefix_backward_sequences_without_queries_get_zero_gradients(mal
 
 
 @pytest.mark.parametrize("tau", [0.0, 1e-4])
-@pytest.mark.parametrize("page", [128, 256])
+@pytest.mark.parametrize("page", [128, 256, 16, 64])
 def test_prefill_chunks_against_a_paged_cache(mala, oracle, tau, page):
     """Packed prefill chunks whose keys and values (prefix and chunk) lie in pages scattered over a shuffled pool."""
     Hq, Hkv, d = 4, 2, 128
@@ -248,7 +248,7 @@ def test_prefill_chunks_against_a_paged_cache(mala, oracle, tau, page):
                                 tau, stats=True)
     torch.cuda.synchronize()
     assert mala.device_status() == 0
-    fm = st.mask(Nmax // 128).cpu().numpy()
+    fm = st.mask(-(-Nmax // 128)).cpu().numpy()
     o_c, lse_c = o.float().cpu().numpy()[0], lse.cpu().numpy()
     legal = 0
     for b, (w, n, m) in enumerate(zip(ws, nk, nq)):

@@ -127,7 +127,7 @@ def test_argument_validation_codes_of_the_general_shape_calls(mala):
     assert bp(base, base, n=1024) == -4        # scratch for total_q + 384 B rows
     fg = lambda page=128, bt=base, sl=base: L.mala_fwd_paged(tin(), tin(), tin(), base, bt, sl, tout(), base, None, 2, 2, 2, 256,
                                                              128, 8, page, 4, 128, 1, 0.1, 1e-4, None, 0, None)
-    assert fg(page=64) == -2 and fg(bt=None) == -1 and fg(sl=None) == -1 and fg(bt=base + 2) == -3
+    assert fg(page=48) == -2 and fg(page=4) == -2 and fg(bt=None) == -1 and fg(sl=None) == -1 and fg(bt=base + 2) == -3
     # several tokens per decode step: at most 16 rows per KV head, no more new tokens than keys
     dm = lambda Sq, Hq=4, Nk=256: L.mala_decode_multi(tin(), tin(), tin(), tout(), None, None, 1, Hq, 1, Nk, Sq, 128, 0.1,
                                                       1e-4, 2, base, 1 << 20, None)
