@@ -201,15 +201,58 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     const int pg = jt * p.ppt + c;
     return pg < p.bt_stride ? __ldg(p.block_table + (size_t)b * p.bt_stride + pg) : -1;
   };
-  auto load_tile_small = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int b, int jt, int hkv) {
-    for (int c = 0; c < p.ppt; ++c) {
-      const int outer = small_page(b, jt, c);
-#pragma unroll
-      for (int pn = 0; pn < PAN; ++pn) tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, outer);
-    }
+
+  // The copies of a tile are issued by a whole converged warp: lane x issues copy x / PAN of panel x % PAN, so the
+  // table lookups are one coalesced load and the copies are issued side by side (one lane alone cannot issue 16 to 32 copies per tile in a
+  // tile's HBM time).  The barrier's expect_tx has been posted by then.
+  auto load_tile_small_warp = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int b, int jt, int hkv) {
+    const int c = lane / PAN, pn = lane % PAN;
+    if (c < p.ppt) tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, small_page(b, jt, c));
   };
 
-  if (warp == 0) {
+  if (warp == 0 && p.ppt > 1) {
+    // ------------------------------------------------------------------ TMA producer, pages smaller than a tile:
+    // the loop of the producer below, run by all 32 lanes (waits and counters warp-uniform)
+    if (lane == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); }
+    int ne = 0, g = 0, ks = 0, vs = 0;
+    uint32_t kpar = 1, vpar = 1;
+    bool ok = true;
+    for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+      int b, hkv, split, T, j0, nk;
+      geometry(item, b, hkv, split, T, j0, nk);
+      if (T == 0) continue;
+      const int ip = ne & 1;
+      ok = mbar_wait_warp(&q_empty[ip], ((ne >> 1) & 1) ^ 1, status);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_arrive_expect_tx(&q_full[ip], (uint32_t)R * 128u * PAN);
+#pragma unroll
+        for (int pn = 0; pn < PAN; ++pn)
+          tma_load_4d(sQ + ip * DecCfg::kQBytes + pn * 2048, &tmQ, &q_full[ip], pn * 64, hkv * G, 0, b);
+      }
+      for (int t = 0; t < T && ok; ++t, ++g) {
+        ok = mbar_wait_warp(&k_empty[ks], kpar, status);
+        if (!ok) break;
+        if (lane == 0) {
+          if (!kDense) { v_row[g & 7] = j0 - t; v_outer[g & 7] = b; }
+          mbar_arrive_expect_tx(&k_full[ks], kTileTx);
+        }
+        __syncwarp();
+        load_tile_small_warp(sK + ks * TB, &tmK, &k_full[ks], b, j0 - t, hkv);
+        if (++ks == KS) { ks = 0; kpar ^= 1; }
+        if (kDense) {   // every tile is retained: V follows K
+          ok = mbar_wait_warp(&v_empty[vs], vpar, status);
+          if (!ok) break;
+          if (lane == 0) mbar_arrive_expect_tx(&v_full[vs], kTileTx);
+          __syncwarp();
+          load_tile_small_warp(sV + vs * TB, &tmV, &v_full[vs], b, j0 - t, hkv);
+          if (++vs == VS) { vs = 0; vpar ^= 1; }
+        }
+      }
+      ++ne;
+    }
+    if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -230,9 +273,8 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         for (int pn = 0; pn < PAN; ++pn)
           tma_load_4d(sQ + ip * DecCfg::kQBytes + pn * 2048, &tmQ, &q_full[ip], pn * 64, hkv * G, 0, b);
         for (int t = 0; t < T && ok; ++t, ++g) {
-          const bool small = p.ppt > 1;
-          int row = j0 - t, outer = b;           // (pages smaller than a tile: looked up copy by copy)
-          if (!small) tile_coord(b, j0 - t, row, outer);   // (a page lookup is in flight while the slot is waited for)
+          int row, outer;
+          tile_coord(b, j0 - t, row, outer);     // (a page lookup is in flight while the slot is waited for)
           ok = mbar_wait(&k_empty[ks], kpar, status);
           if (!ok) break;
           // The UMMA warp requests V of tile g from these coordinates after the vote.  It cannot be more than six
@@ -240,21 +282,17 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           // and it sees the two stores through the K tile's barrier.
           if (!kDense) { v_row[g & 7] = row; v_outer[g & 7] = outer; }
           mbar_arrive_expect_tx(&k_full[ks], kTileTx);
-          if (small) load_tile_small(sK + ks * TB, &tmK, &k_full[ks], b, j0 - t, hkv);
-          else
 #pragma unroll
-            for (int pn = 0; pn < PAN; ++pn)
-              tma_load_4d(sK + ks * TB + pn * 16384, &tmK, &k_full[ks], pn * 64, row, hkv, outer);
+          for (int pn = 0; pn < PAN; ++pn)
+            tma_load_4d(sK + ks * TB + pn * 16384, &tmK, &k_full[ks], pn * 64, row, hkv, outer);
           if (++ks == KS) { ks = 0; kpar ^= 1; }
           if (kDense) {   // every tile is retained: V follows K
             ok = mbar_wait(&v_empty[vs], vpar, status);
             if (!ok) break;
             mbar_arrive_expect_tx(&v_full[vs], kTileTx);
-            if (small) load_tile_small(sV + vs * TB, &tmV, &v_full[vs], b, j0 - t, hkv);
-            else
 #pragma unroll
-              for (int pn = 0; pn < PAN; ++pn)
-                tma_load_4d(sV + vs * TB + pn * 16384, &tmV, &v_full[vs], pn * 64, row, hkv, outer);
+            for (int pn = 0; pn < PAN; ++pn)
+              tma_load_4d(sV + vs * TB + pn * 16384, &tmV, &v_full[vs], pn * 64, row, hkv, outer);
             if (++vs == VS) { vs = 0; vpar ^= 1; }
           }
         }
@@ -344,11 +382,18 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
               if (leader) {
                 const int row = *(volatile int*)&v_row[cv.g & 7], outer = *(volatile int*)&v_outer[cv.g & 7];
                 mbar_arrive_expect_tx(&v_full[vi], kTileTx);
-                if (p.ppt > 1) load_tile_small(sV + vi * TB, &tmV, &v_full[vi], outer, row, cv.hkv);
-                else
+                if (p.ppt > 1) {   // (one lane, copy after copy: this warp's time belongs to the MMAs)
+                  for (int c = 0; c < p.ppt; ++c) {
+                    const int pgid = small_page(outer, row, c);
+#pragma unroll
+                    for (int pn = 0; pn < PAN; ++pn)
+                      tma_load_4d(sV + vi * TB + pn * 16384 + c * p.prows * 128, &tmV, &v_full[vi], pn * 64, 0, cv.hkv, pgid);
+                  }
+                } else {
 #pragma unroll
                   for (int pn = 0; pn < PAN; ++pn)
                     tma_load_4d(sV + vi * TB + pn * 16384, &tmV, &v_full[vi], pn * 64, row, cv.hkv, outer);
+                }
               }
               __syncwarp();
               if (++vi == VS) { vi = 0; vipar ^= 1; }
