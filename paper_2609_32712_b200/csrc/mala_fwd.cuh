@@ -179,7 +179,53 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (warp < 4) {
   // warps 0-3 (producer, issuers) need few registers; the two softmax warpgroups take the rest
   reg_dealloc<72>();
-  if (warp == 0) {
+  if (warp == 0 && kSmall) {
+    // ------------------------------------------------------------------ TMA producer, pages smaller than a tile:
+    // the loop of the producer below run by all 32 lanes (waits and counters warp-uniform); lane x issues copy
+    // x / PAN of panel x % PAN of a tile, so the table lookups are one coalesced load and the copies are issued side
+    // by side instead of one after the other
+    auto load_tile_small_warp = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int jt) {
+      const int c = lane / PAN, pn = lane % PAN, pg = jt * p.ppt + c;
+      if (c < p.ppt) {
+        const int outer = pg < p.bt_stride ? __ldg(p.block_table + (size_t)b * p.bt_stride + pg) : -1;
+        tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, outer);
+      }
+    };
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+      mbar_arrive_expect_tx(&q_full, (hasB ? 2 : 1) * Cfg::kTileBytes);
+      for (int pn = 0; pn < PAN; ++pn) {
+        tma_load_4d(sQ + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iA * 128 - qshift, h, bz);
+        if (hasB)
+          tma_load_4d(sQ + Cfg::kTileBytes + pn * 16384, &tmQ, &q_full, pn * 64, row0 + iB * 128 - qshift, h, bz);
+      }
+    }
+    int issued = 0, v_issued = 0, s = 0;
+    uint32_t par = 1;
+    bool ok = true;
+    for (int u = 0; u < U && ok; ++u) {
+      ok = mbar_wait_warp(&k_empty[s], par, status);
+      if (!ok) break;
+      if (lane == 0) mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
+      __syncwarp();
+      load_tile_small_warp(sK + s * Cfg::kTileBytes, &tmK, &k_full[s], j0 - u);
+      issued = u + 1;
+      if (++s == KS) { s = 0; par ^= 1; }
+      if (kDense) {
+        ok = mbar_wait_warp(&v_empty[u & 1], ((u >> 1) & 1) ^ 1, status);
+        if (!ok) break;
+        if (lane == 0) mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
+        __syncwarp();
+        load_tile_small_warp(sV + (u & 1) * Cfg::kTileBytes, &tmV, &v_full[u & 1], j0 - u);
+        v_issued = u + 1;
+      }
+    }
+    if (!ok && lane == 0) {
+      mbar_wait(&q_full, 0, status);
+      for (int u = (issued > KS ? issued - KS : 0); u < issued; ++u) mbar_wait(&k_full[u % KS], (u / KS) & 1, status);
+      for (int u = (v_issued > 2 ? v_issued - 2 : 0); u < v_issued; ++u) mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
+    }
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer: Q_A, Q_B, K ring
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -194,25 +240,21 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       uint32_t par = 1;                 // parity of the "empty" phase to wait for (first pass: free)
       bool ok = true;
       for (int u = 0; u < U && ok; ++u) {
-        int krow = 0, kouter = 0;
-        if (!small_pages) key_coord(j0 - u, krow, kouter);   // (a page lookup is in flight while the stage is waited for)
+        int krow, kouter;
+        key_coord(j0 - u, krow, kouter);   // (a page lookup is in flight while the stage is waited for)
         ok = mbar_wait(&k_empty[s], par, status);
         if (!ok) break;
         mbar_arrive_expect_tx(&k_full[s], Cfg::kTileBytes);
-        if (small_pages) load_tile_small(sK + s * Cfg::kTileBytes, &tmK, &k_full[s], j0 - u);
-        else
-          for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, krow, hkv, kouter);
+        for (int pn = 0; pn < PAN; ++pn)
+          tma_load_4d(sK + s * Cfg::kTileBytes + pn * 16384, &tmK, &k_full[s], pn * 64, krow, hkv, kouter);
         issued = u + 1;
         if (++s == KS) { s = 0; par ^= 1; }
         if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
           ok = mbar_wait(&v_empty[u & 1], ((u >> 1) & 1) ^ 1, status);
           if (!ok) break;
           mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
-          if (small_pages) load_tile_small(sV + (u & 1) * Cfg::kTileBytes, &tmV, &v_full[u & 1], j0 - u);
-          else
-            for (int pn = 0; pn < PAN; ++pn)
-              tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow, hkv, kouter);
+          for (int pn = 0; pn < PAN; ++pn)
+            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow, hkv, kouter);
           v_issued = u + 1;
         }
       }
