@@ -228,10 +228,10 @@ def test_varlen_prefix_backward_sequences_without_queries_get_zero_gradients(mal
 
 
 @pytest.mark.parametrize("tau", [0.0, 1e-4])
-@pytest.mark.parametrize("page", [128, 256, 16, 64])
-def test_prefill_chunks_against_a_paged_cache(mala, oracle, tau, page):
+@pytest.mark.parametrize("page,d", [(128, 128), (256, 128), (16, 128), (64, 128), (8, 64), (32, 96), (128, 40)])
+def test_prefill_chunks_against_a_paged_cache(mala, oracle, tau, page, d):
     """Packed prefill chunks whose keys and values (prefix and chunk) lie in pages scattered over a shuffled pool."""
-    Hq, Hkv, d = 4, 2, 128
+    Hq, Hkv = 4, 2
     nk = [900, 128, 517, 300]
     nq = [260, 128, 100, 1]
     ws = [W.custom_prefill(1, Hq, Hkv, n, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=70 + x, preset="R")
