@@ -578,7 +578,9 @@ def main():
     # The step's inputs lie in pinned host memory, one contiguous block per KV-head group (the unit the path shards
     # by), and its results go back to pinned host memory.  The groups are independent, so the step is pipelined over
     # them through the library's own calls: group g + 1 is copied in and group g - 1 copied out while group g runs
-    # forward and backward (three streams; the calls are asynchronous on the stream they are given).
+    # forward and backward (three streams; the calls are asynchronous on the stream they are given).  A group's
+    # forward waits only for its q, k, v (dO follows behind them) and its output goes back while its backward runs,
+    # which shortens the pipeline's fill and drain.
     G = c.Hq // c.Hkv
     groups = []
     for g in range(c.Hkv):
@@ -599,20 +601,27 @@ def main():
         with torch.cuda.stream(cin):
             cin.wait_event(start)                       # the previous step has read these buffers
             for gr in groups:
-                for d_, h_ in zip(gr["d_in"], gr["h_in"]):
+                for d_, h_ in zip(gr["d_in"][:3], gr["h_in"][:3]):
                     d_.copy_(h_, non_blocking=True)
-                ready.append(cin.record_event())
+                ev_qkv = cin.record_event()
+                gr["d_in"][3].copy_(gr["h_in"][3], non_blocking=True)
+                ready.append((ev_qkv, cin.record_event()))
         cout.wait_event(start)
-        for gr, ev_in in zip(groups, ready):
+        for gr, (ev_qkv, ev_do) in zip(groups, ready):
             q_, k_, v_, do_ = gr["d_in"]
             o_, dq_, dk_, dv_ = gr["d_out"]
-            main.wait_event(ev_in)
+            main.wait_event(ev_qkv)
             mala.fwd(q_, k_, v_, case.scale, tau, out=o_, lse=g_lse, ws=g_ws)
+            fwd_done = main.record_event()
+            with torch.cuda.stream(cout):
+                cout.wait_event(fwd_done)
+                gr["h_out"][0].copy_(o_, non_blocking=True)
+            main.wait_event(ev_do)
             mala.bwd(q_, k_, v_, o_, do_, g_lse, case.scale, tau, ws=g_ws, dq=dq_, dk=dk_, dv=dv_)
             done = main.record_event()
             with torch.cuda.stream(cout):
                 cout.wait_event(done)
-                for h_, d_ in zip(gr["h_out"], gr["d_out"]):
+                for h_, d_ in zip(gr["h_out"][1:], gr["d_out"][1:]):
                     h_.copy_(d_, non_blocking=True)
         main.wait_stream(cout)
         main.wait_stream(cin)
