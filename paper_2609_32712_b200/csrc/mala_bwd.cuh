@@ -6,11 +6,8 @@
 //                           for every query head of the group and every query block i >= j (ascending)
 //                           S^T = K_j Q_i^T is recomputed on tensor cores and tested against the saved
 //                           lse (Eq. 4).  Only retained tiles run dP^T = V dO^T, P^T,
-//                           dS^T = P^T o (dP^T - D), dV += P^T dO, dK += dS^T Q, dQ_i += dS K_j.
-//                           In a run of skipped tiles the next tile's scores are issued into a second TMEM
-//                           region before the current tile's vote is known, Q(n+2) is requested the moment
-//                           vote(n) is known, and no dO is loaded (dO is fetched ahead only behind a retained
-//                           tile, on demand for a retained tile behind a skipped one).
+//                           dS^T = P^T o (dP^T - D), dV += P^T dO, dK += dS^T Q, dQ_i += dS K_j
+//                           (dO is fetched ahead for every tile: the vote comes too late to hide the copy).
 //                           dK, dV accumulate in TMEM; dQ tiles are added to an fp32 accumulator in
 //                           global memory, one half of the columns by vector reductions from registers
 //                           (red.global.add.v4.f32), the other half by TMA reduce-add from shared memory.
@@ -24,7 +21,7 @@
 //   bwd_convert_dq_kernel : dq = bf16(scale * accumulator), back in row-major order.
 //
 // Warp roles of the main kernel (768 threads; registers are re-split between the warpgroups):
-//   warp 0       TMA producer (K_j, V_j once; Q ring; dO ring; the MALA kernel's producer follows the votes)
+//   warp 0       TMA producer (K_j, V_j once; Q ring; dO ring)
 //   warp 1       UMMA warp (all 32 lanes run the issue loop, one elected lane issues); warps 2-3 idle
 //   warps 4-19   score group, four threads per key row (32 query columns each): reads S^T once, applies
 //                Eq. 4 and votes; retained tiles: P^T -> TMEM (A operand of dV), then, with P^T still in
@@ -43,10 +40,6 @@
 #include "../../include/mala.h"
 #include "sm100_ptx.cuh"
 #include "tensor_map.h"
-
-#ifndef MALA_BWD_CHEAP_BOUND
-#define MALA_BWD_CHEAP_BOUND 1
-#endif
 
 namespace mala {
 
@@ -90,7 +83,7 @@ struct BwdCfg {
   // have consumed it (D = 128); for D = 64 a dO stage is too small, so two separate dS stages follow.
   static constexpr int kSmemBytes = 6 * kTileBytes + (D == 128 ? 0 : 2 * kDsBytes) + 1024;
   static constexpr int kThreads = 768;
-  static constexpr uint32_t kColDV = 256, kColDK = 384;   // columns 0..255: two regions for S^T / P^T and dP^T / dS^T / dQ
+  static constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
 };
 
 template <int D, bool kDense>
@@ -109,14 +102,11 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   // dS^T stages, [2 halves][128 key rows][64 q] bf16, 128B swizzle
   uint8_t* sDS = (D == 128) ? sDO : sDO + 2 * Cfg::kTileBytes;
 
-  __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full[2], vote_bar[2], p_full, dp_full,
-      ds_full, dst_full, dv_done, dq_full, dq_empty, dq_info_bar, fin_bar, stg_full, ds_free, vec_full[4], vec_empty[4];
-  __shared__ __align__(16) float vec[4][3][128];   // [tile & 3][lse2 | bq | Dq][query column], filled by warp 2
-  __shared__ int stat_r_head, stat_word;            // telemetry state of the one thread that writes it
-  __shared__ uint32_t stat_bits;
-  __shared__ float vmin[4][4];                     // [tile & 3][column quarter]: smallest bq of the quarter's 32 columns
+  __shared__ uint64_t kv_full, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, vote_bar[2], p_full, dp_full,
+      ds_full, dst_full, dv_done, dq_full, dq_empty, dq_info_bar, grp_bar, fin_bar, stg_full, ds_free;
+  __shared__ __align__(16) float vec[3][3][128];   // [slot][lse2 | bq | Dq][query column]
   __shared__ uint32_t tmem_base_s;
-  __shared__ int flag[4];
+  __shared__ int flag[3];
   __shared__ int dq_info;
   __shared__ int early_exit;
 
@@ -158,12 +148,11 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       mbar_init(&do_full[s], 1); mbar_init(&do_empty[s], 1);
       mbar_init(&vote_bar[s], 16);
     }
-    mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1); mbar_init(&p_full, 16); mbar_init(&dp_full, 1); mbar_init(&ds_full, 16); mbar_init(&dst_full, 16);
-    mbar_init(&dv_done, 1); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
+    mbar_init(&s_full, 1); mbar_init(&p_full, 16); mbar_init(&dp_full, 1); mbar_init(&ds_full, 16); mbar_init(&dst_full, 16);
+    mbar_init(&dv_done, 1); mbar_init(&grp_bar, 16); mbar_init(&dq_full, 1); mbar_init(&dq_empty, 4); mbar_init(&dq_info_bar, 1);
     mbar_init(&fin_bar, 1);
     mbar_init(&stg_full, 4); mbar_init(&ds_free, 1);
-    for (int s = 0; s < 4; ++s) { mbar_init(&vec_full[s], 1); mbar_init(&vec_empty[s], 16); }
-    flag[0] = flag[1] = flag[2] = flag[3] = 0;
+    flag[0] = flag[1] = flag[2] = 0;
     dq_info = -1;
     mbar_fence_init();
   }
@@ -175,9 +164,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
 
-  // register split (setmaxnreg): 4 x 48 + 16 x 72 + 4 x 144 = 24 x 80 (no spills in any role at these sizes)
   if (warp < 4) {
-  reg_dealloc<48>();
+  reg_dealloc<40>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -187,122 +175,33 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tma_load_4d(sK + pn * 16384, &tmK, &kv_full, pn * 64, krow0 + j * 128, hkv, bz);
         tma_load_4d(sV + pn * 16384, &tmV, &kv_full, pn * 64, krow0 + j * 128, hkv, bz);
       }
-      // Shared-memory stages: Q ring of two (tile n in stage n & 1), dO ring of two (tile n's dO, when it is
-      // fetched at all, in stage n & 1).  The dense kernel fetches Q and dO of every tile ahead.  The MALA kernel
-      // follows the votes itself: Q(n+2) is requested the moment vote(n) is known (a skipped tile's stage is free
-      // then: every score warp has read the scores, so the MMAs that read Q have retired); dO is fetched ahead only
-      // for a tile whose predecessor was retained (a one-bit predictor) and on demand, after the vote, for a
-      // retained tile that was not predicted -- a run of skipped tiles loads no dO at all.  A dO that was fetched
-      // ahead for a tile that is then skipped is never handed to anyone: the producer itself waits for it to land
-      // before it reuses the stage.
       bool ok = true;
-      // per-stage state, 16 bits per stage in one register (this warp runs on 40 registers):
-      //   bit 0 parity of the Q copies issued, bit 1 a Q copy was issued, bit 2 parity of the q_empty phases consumed,
-      //   bit 3 the stage's last tile was retained (wait for q_empty before reuse), bit 4 parity of the dO copies
-      //   issued, bit 5 a dO copy was issued, bit 6 parity of the do_empty phases consumed,
-      //   bits 7-8 the stage's last dO copy: 0 none / released, 1 used by a retained tile, 2 orphan
-      uint32_t st = 0;
-      auto push_q = [&](int n, int hq_, int i_) -> bool {
-        const int s = n & 1, sh = s * 16;
-        if ((st >> sh) & 8u) {
-          if (!mbar_wait(&q_empty[s], (st >> (sh + 2)) & 1u, status)) return false;
-          st ^= 4u << sh;
-          st &= ~(8u << sh);
-        }
+      int issued = 0;
+      int hq = hkv * G, i = i0;   // tile n = (query head, query block), kept by increments: no division per tile
+      for (int n = 0; n < n_tot && ok; ++n, ++i) {
+        if (i == T) { i = i0; ++hq; }
+        const int s = n & 1;
+        ok = mbar_wait(&q_empty[s], ((n >> 1) & 1) ^ 1, status);
+        if (!ok) break;
         mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i_ * 128 - qshift, hq_, bz);
-        st = (st ^ (1u << sh)) | (2u << sh);
-        return true;
-      };
-      auto push_do = [&](int n, int hq_, int i_) -> bool {
-        const int s = n & 1, sh = s * 16;
-        const uint32_t kind = (st >> (sh + 7)) & 3u;
-        if (kind == 1u) {
-          if (!mbar_wait(&do_empty[s], (st >> (sh + 6)) & 1u, status)) return false;
-          st ^= 64u << sh;
-        } else if (kind == 2u) {   // (the parity of the last copy's phase is the complement of the running parity)
-          if (!mbar_wait(&do_full[s], ((st >> (sh + 4)) & 1u) ^ 1u, status)) return false;
-        }
-        st &= ~(0x180u << sh);
+          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128 - qshift, hq, bz);
+        // dO of every tile is fetched ahead, retained or not (the vote comes too late to hide the copy behind it);
+        // a skipped tile's stage is handed straight back by the issuer
+        ok = mbar_wait(&do_empty[s], ((n >> 1) & 1) ^ 1, status);
+        if (!ok) { mbar_wait(&q_full[s], (n >> 1) & 1, status); break; }
         mbar_arrive_expect_tx(&do_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, row0 + i_ * 128 - qshift, hq_, bz);
-        st = (st ^ (16u << sh)) | (32u << sh);
-        return true;
-      };
-      // tile n = (query head, query block), kept by increments: no division per tile
-      int hq = hkv * G, i = i0;
-      auto next_tile = [&](int& hq_, int& i_) { if (++i_ == T) { i_ = i0; ++hq_; } };
-      if (kDense) {
-        for (int n = 0; n < n_tot && ok; ++n) {
-          if (n >= 2) st |= (8u | 0x80u) << ((n & 1) * 16);   // both stages' previous tiles were retained ones
-          ok = push_q(n, hq, i) && push_do(n, hq, i);
-          next_tile(hq, i);
-        }
-      } else {
-        ok = push_q(0, hq, i) && push_do(0, hq, i);
-        if (ok && n_tot > 1) { int h1 = hq, i1 = i; next_tile(h1, i1); ok = push_q(1, h1, i1); }
-        bool pref = true;                    // dO of the current tile was fetched ahead
-        for (int n = 0; n < n_tot && ok; ++n) {
-          const int s = n & 1, sh = s * 16;
-          ok = mbar_wait(&vote_bar[s], (n >> 1) & 1, status);
-          if (!ok) break;
-          const bool retain = (*(volatile int*)&flag[n & 3]) != 0;
-          int h1 = hq, i1 = i;
-          next_tile(h1, i1);
-          if (retain) {
-            if (!pref) ok = push_do(n, hq, i);   // (still sees what the stage's PREVIOUS copy was)
-            // tile n now holds both its stages until dK(n) (Q) and the end of its dQ drain (dO)
-            st = (st & ~(0x180u << sh)) | ((8u | 0x80u) << sh);
-            if (ok && n + 1 < n_tot) ok = push_do(n + 1, h1, i1);
-          } else if (pref) {
-            st = (st & ~(0x180u << sh)) | (0x100u << sh);   // fetched ahead in vain: an orphan
-          }
-          hq = h1; i = i1;
-          if (ok && n + 2 < n_tot) { next_tile(h1, i1); ok = push_q(n + 2, h1, i1); }
-          pref = retain;
+          tma_load_4d(sDO + s * Cfg::kTileBytes + pn * 16384, &tmDO, &do_full[s], pn * 64, row0 + i * 128 - qshift, hq, bz);
+        issued = n + 1;
+      }
+      if (!ok) {
+        mbar_wait(&kv_full, 0, status);
+        for (int n = (issued > 2 ? issued - 2 : 0); n < issued; ++n) {
+          mbar_wait(&q_full[n & 1], (n >> 1) & 1, status);
+          mbar_wait(&do_full[n & 1], (n >> 1) & 1, status);
         }
       }
-      // every copy this thread issued has landed before the CTA may exit (the ones nobody consumed: orphans, and
-      // everything still in flight after a failed wait)
-      if (!ok) mbar_wait(&kv_full, 0, status);
-      for (int s = 0; s < 2; ++s) {
-        const uint32_t x = st >> (s * 16);
-        if (!ok && (x & 2u)) mbar_wait(&q_full[s], (x & 1u) ^ 1u, status);
-        if ((!ok || ((x >> 7) & 3u) == 2u) && (x & 32u)) mbar_wait(&do_full[s], ((x >> 4) & 1u) ^ 1u, status);
-      }
-    }
-  } else if (warp == 2) {
-    // ------------------------------------------------------------------ per-query vectors
-    // lse2, the test offset bq and D of the 128 queries of every tile, into a ring of four shared-memory slots, well
-    // ahead of the score group (which reads them as broadcast float4s); for the MALA kernel also the smallest bq of
-    // each 32-column quarter.  Lane l carries queries 4 l .. 4 l + 3.
-    bool ok = true;
-    int hq_l = 0, i = i0;
-    for (int m = 0; m < n_tot && ok; ++m) {
-      const int slot = m & 3;
-      if (m >= 4) {   // every score warp has left tile m - 4
-        ok = mbar_wait_warp(&vec_empty[slot], ((m >> 2) & 1) ^ 1, status);
-        if (!ok) break;
-      }
-      const size_t x = ((size_t)bz * p.Hq + hkv * G + hq_l) * p.Np + (size_t)prow0 + (size_t)i * 128 + lane * 4;
-      const float4 a = *reinterpret_cast<const float4*>(p.lse2 + x);
-      const float4 bqv = *reinterpret_cast<const float4*>(p.bq + x);
-      const float4 dd = *reinterpret_cast<const float4*>(p.Dq + x);
-      *reinterpret_cast<float4*>(&vec[slot][0][lane * 4]) = a;
-      *reinterpret_cast<float4*>(&vec[slot][1][lane * 4]) = bqv;
-      *reinterpret_cast<float4*>(&vec[slot][2][lane * 4]) = dd;
-      if (!kDense) {
-        float mn = fminf(fminf(bqv.x, bqv.y), fminf(bqv.z, bqv.w));
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1));
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2));
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 4));
-        if ((lane & 7) == 0) vmin[slot][lane >> 3] = mn;
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&vec_full[slot]);
-      if (++i == T) { i = i0; ++hq_l; }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
@@ -324,64 +223,35 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint64_t dDSm0 = make_smem_desc(smem_u32(sDS), 16384, 1024);  // dS^T stage 0 as MN-major A (dQ)
       bool ok = mbar_wait_warp(&kv_full, 0, status);
       int r = 0;   // retained tiles so far
-      // The 256 TMEM columns that are not dK / dV form two regions of 128.  A retained tile has its scores (then
-      // P^T) in one region and dP^T / dS^T / dQ in the other.  In a run of skipped tiles the scores alternate
-      // between the regions: when tile n-1 was skipped, S^T(n+1) is issued into the region tile n does NOT use
-      // before vote(n) is known, so the tensor pipe works on the next scores while the score group reads and
-      // votes on the current ones.  If tile n then turns out to be retained, its dP^T needs that region: the
-      // speculative scores are abandoned (dP^T follows them in tensor-pipe order and overwrites them) and
-      // S^T(n+1) is issued again after dV(n), as in a run of retained tiles.
-      uint32_t reg_v = 0;          // region of S^T(n) (the dense kernel never leaves region 0)
-#define MALA_BWD_REG (kDense ? 0u : reg_v)
-      bool prev_retain = true;     // (tile -1 counts as retained: no speculation before the first vote)
-      bool pref = true;            // dO(n) was fetched ahead (mirror of the producer's rule)
-      bool dq_pending = false;     // the last retained tile's dQ may still sit in the other region
-      int df_cnt0 = 0, df_cnt1 = 0;   // dO copies into each stage so far (mirror of the producer's count)
-      auto issue_qk = [&](int n, uint32_t rg) -> bool {
+      auto issue_qk = [&](int n) -> bool {
         const int s = n & 1;
         if (!mbar_wait_warp(&q_full[s], (n >> 1) & 1, status)) return false;
         tc_fence_after();
         const uint64_t dQk = desc_advance(dQk0, s * Cfg::kTileBytes);
-        const uint32_t tS = tmem_addr(tb, 0, rg * 128u);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-          mma_ss(tS, desc_advance(dKk, off), desc_advance(dQk, off), idesc_s, k > 0, leader);
+          mma_ss(tmem_addr(tb, 0, Cfg::kColS), desc_advance(dKk, off), desc_advance(dQk, off), idesc_s, k > 0, leader);
         }
-        if (leader) tc_commit(&s_full[rg]);
+        if (leader) tc_commit(&s_full);
         return true;
       };
-      if (ok) ok = issue_qk(0, 0);
+      if (ok) ok = issue_qk(0);
       for (int n = 0; n < n_tot && ok; ++n) {
         const int s = n & 1;
-        const bool has_next = n + 1 < n_tot;
-        const bool spec = !kDense && !prev_retain && has_next;
-        if (spec) {
-          if (dq_pending) {   // the other region may still hold the dQ tile of the last retained tile
-            ok = mbar_wait_warp(&dq_empty, (r - 1) & 1, status);
-            if (!ok) break;
-            dq_pending = false;
-          }
-          ok = issue_qk(n + 1, MALA_BWD_REG ^ 1u);
-          if (!ok) break;
-        }
         bool retain = true;
         if (!kDense) {
-          ok = mbar_wait_warp(&vote_bar[s], (n >> 1) & 1, status);
+          ok = mbar_wait_warp(&vote_bar[n & 1], (n >> 1) & 1, status);
           if (!ok) break;
-          retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[n & 3], 0) != 0;
+          retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[n % 3], 0) != 0;
         }
         const int ds = s;       // dO stage (the dS^T / dQ staging of the tile reuses it)
         if (retain) {
-          const uint32_t reg = MALA_BWD_REG;
-          const uint32_t colS = reg * 128u, colDP = (reg ^ 1u) * 128u;
-          if (dq_pending) {   // the dQ tile of the previous retained tile (aliased with dP) has been read out
+          if (r > 0) {   // the dQ tile of the previous retained tile (aliased with dP) has been read out
             ok = mbar_wait_warp(&dq_empty, (r - 1) & 1, status);
             if (!ok) break;
           }
-          const int dfc = kDense ? (n >> 1) : (ds ? df_cnt1 : df_cnt0);
-          if (!kDense) { if (ds) ++df_cnt1; else ++df_cnt0; }
-          ok = mbar_wait_warp(&do_full[ds], dfc & 1, status);
+          ok = mbar_wait_warp(&do_full[ds], (n >> 1) & 1, status);
           if (!ok) break;
           tc_fence_after();
           const uint64_t dDOk = desc_advance(dDOk0, ds * Cfg::kTileBytes);
@@ -390,7 +260,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {   // dP^T = V dO^T
             const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
-            mma_ss(tmem_addr(tb, 0, colDP), desc_advance(dVk, off), desc_advance(dDOk, off), idesc_s, k > 0, leader);
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dVk, off), desc_advance(dDOk, off), idesc_s, k > 0, leader);
           }
           if (leader) tc_commit(&dp_full);
           ok = mbar_wait_warp(&p_full, r & 1, status);
@@ -398,12 +268,14 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < 8; ++k)   // dV += P^T dO
-            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, colS + (k >> 1) * 32 + (k & 1) * 8),
+            mma_ts(tmem_addr(tb, 0, Cfg::kColDV), tmem_addr(tb, 0, Cfg::kColS + (k >> 1) * 32 + (k & 1) * 8),
                    desc_advance(dDOm, k * 2048), idesc_dv, k > 0 ? 1u : acc0, leader);
           if (leader) tc_commit(&dv_done);
-          // the score region is free once dV has been issued (the score group keeps P^T in registers):
-          // recompute the next tile's scores while dS is being formed
-          if (has_next) { ok = issue_qk(n + 1, reg); if (!ok) break; }
+        }
+        // the score buffer is free once dV has been issued (the score group keeps P^T in registers):
+        // recompute the next tile's scores while dS is being formed
+        if (n + 1 < n_tot) { ok = issue_qk(n + 1); if (!ok) break; }
+        if (retain) {
           ok = mbar_wait_warp(&dst_full, r & 1, status);
           if (!ok) break;
           tc_fence_after();
@@ -412,7 +284,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           const uint32_t acc1 = r > 0 ? 1u : 0u;
 #pragma unroll
           for (int k = 0; k < 8; ++k)     // dK += dS^T Q, dS^T read from TMEM (the dP columns)
-            mma_ts(tmem_addr(tb, 0, Cfg::kColDK), tmem_addr(tb, 0, colDP + (k >> 1) * 32 + (k & 1) * 8),
+            mma_ts(tmem_addr(tb, 0, Cfg::kColDK), tmem_addr(tb, 0, Cfg::kColDP + (k >> 1) * 32 + (k & 1) * 8),
                    desc_advance(dQm, k * 2048), idesc_dv, k > 0 ? 1u : acc1, leader);
           if (leader) tc_commit(&q_empty[s]);
           ok = mbar_wait_warp(&ds_full, r & 1, status);   // the shared-memory copy of dS^T
@@ -420,25 +292,21 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < 8; ++k)     // dQ_i tile = dS K_j, into the dP columns (after dK has read dS^T from them)
-            mma_ss(tmem_addr(tb, 0, colDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
+            mma_ss(tmem_addr(tb, 0, Cfg::kColDP), desc_advance(dDSm, k * 2048), desc_advance(dKm, k * 2048), idesc_dq,
                    k > 0, leader);
           if (leader) {
-            *(volatile int*)&dq_info = n * 4 + ds * 2 + (int)(reg ^ 1u);
+            *(volatile int*)&dq_info = n * 2 + ds;
             mbar_arrive(&dq_info_bar);
             tc_commit(&dq_full);
             tc_commit(&ds_free);   // dS^T has been consumed: the dQ group may stage the dQ tile in that stage
           }
           ++r;
-          dq_pending = true;
         } else {
-          // skipped tile: nothing to hand back (the producer follows the votes itself); a dO that was fetched
-          // ahead for it only counts as a use of its stage
-          if (pref) { if (ds) ++df_cnt1; else ++df_cnt0; }
-          if (spec) reg_v ^= 1u;                 // the next scores are already (being) formed in the other region
-          else if (has_next) { ok = issue_qk(n + 1, MALA_BWD_REG); if (!ok) break; }
+          // skipped tile: Q and the dO fetched ahead (once it has landed) go back to their rings
+          ok = mbar_wait_warp(&do_full[ds], (n >> 1) & 1, status);
+          if (!ok) break;
+          if (leader) { mbar_arrive(&q_empty[s]); mbar_arrive(&do_empty[ds]); }
         }
-        pref = retain;
-        prev_retain = retain;
       }
       // tell the dQ group that nothing more will come, then wait for every MMA to retire
       __syncwarp();
@@ -449,7 +317,6 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_commit(&fin_bar);
       }
       mbar_wait_warp(&fin_bar, 0, status);
-#undef MALA_BWD_REG
     }
   }
   } else if (warp < 20) {
@@ -467,27 +334,42 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const bool stat_thread = (warp == 4 && lane == 0);
     bool ok = true;
     int r = 0;
+    int r_head = 0;
+    uint32_t bm_bits = 0;
+    int bm_word = -1;
+
+    auto vec_index = [&](int hq_local, int i) -> size_t {
+      return ((size_t)bz * p.Hq + hkv * G + hq_local) * p.Np + (size_t)prow0 + (size_t)i * 128 + rl;
+    };
+    // per-query vectors of tile 0 into slot 0 (published by the first column quarter), then a group sync
+    if (qt == 0) {
+      const size_t x = vec_index(0, i0);
+      vec[0][0][rl] = p.lse2[x];
+      vec[0][1][rl] = p.bq[x];
+      vec[0][2][rl] = p.Dq[x];
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&grp_bar);
+    ok = mbar_wait(&grp_bar, 0, status);
+    ok = __all_sync(0xffffffffu, ok);
 
     // tile n = (query head hq_n of the group, query block i): kept by increments, no division per tile
-    int hq_n = 0, i = i0;
-    // mirror of the issuer's bookkeeping: the region that holds S^T(n), and how many score tiles each region has
-    // been given so far (speculative ones that were abandoned included)
-    // (one register: bit 0 = region, bit 1 = previous tile retained, bits 2 / 3 = parity of the count of region 0 / 1)
-    uint32_t rs = 2u;
-    for (int n = 0; n < n_tot && ok; ++n, ++i) {
+    int hq_n = 0, i = i0, slot = 0;
+    for (int n = 0; n < n_tot && ok; ++n, ++i, slot = (slot == 2 ? 0 : slot + 1)) {
       if (i == T) { i = i0; ++hq_n; }
-      const int slot = n & 3;
       const bool first_of_head = (i == i0), last_of_head = (i == T - 1);
-      const uint32_t reg = kDense ? 0u : (rs & 1u);
-      const uint32_t colS = reg * 128u, colDP = (reg ^ 1u) * 128u;
-      ok = mbar_wait(&s_full[reg], kDense ? (uint32_t)(n & 1) : ((rs >> (2 + reg)) & 1u), status);
-      if (!kDense) rs ^= 4u << reg;
-      if (ok) ok = mbar_wait(&vec_full[slot], (n >> 2) & 1, status);   // this tile's per-query vectors (long there)
+      // prefetch the per-query vectors of the next tile
+      float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
+      if (qt == 0 && n + 1 < n_tot) {
+        const size_t x = last_of_head ? vec_index(hq_n + 1, i0) : vec_index(hq_n, i + 1);
+        nx0 = p.lse2[x]; nx1 = p.bq[x]; nx2 = p.Dq[x];
+      }
+      ok = mbar_wait(&s_full, n & 1, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       uint32_t sc[32];
-      tmem_ld_x32(tmem_addr(tb, lane_base, colS + qt * 32), sc);
+      tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColS + qt * 32), sc);
       tmem_wait_ld();
       if (p.cu && !valid_key) {   // packed sequences: a row past this sequence's end holds the next one's key
         const uint32_t ninf = 0xff800000u;
@@ -501,41 +383,31 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         for (int e = 0; e < 32; ++e)
           if (c0 + e < rl) sc[e] = ninf;
       }
-      // Eq. 4 (MALA only): skip iff s - lse_q < log(tau / L_q) on every valid entry.
-      // A bound is tried first: max_e (s_e c2 - bq_e) <= (max_e s_e) c2 - min_e bq_e (c2 > 0, and
-      // fma is monotone in each argument, so the inequality holds for the rounded values too); when the bound is
-      // negative for every thread of the warp, none of them can vote and the exact maximum is not needed -- half the
-      // instructions and no shared-memory reads on the path that a run of skipped tiles repeats.
+      // Eq. 4 (MALA only): skip iff s - lse_q < log(tau / L_q) on every valid entry
       float crit = -INFINITY;
-      bool need_exact = !kDense;
-      if (!kDense && MALA_BWD_CHEAP_BOUND) {   // (no branch on per-thread state around the vote: the warp stays converged)
-        float m0 = __uint_as_float(sc[0]), m1 = __uint_as_float(sc[1]);   // two chains, two registers
-#pragma unroll
-        for (int e = 0; e < 7; ++e) {
-          m0 = max3(m0, __uint_as_float(sc[2 + 4 * e]), __uint_as_float(sc[3 + 4 * e]));
-          m1 = max3(m1, __uint_as_float(sc[4 + 4 * e]), __uint_as_float(sc[5 + 4 * e]));
-        }
-        const float mx = max3(m0, m1, fmaxf(__uint_as_float(sc[30]), __uint_as_float(sc[31])));
-        need_exact = __any_sync(0xffffffffu, valid_key && !(fmaf(mx, c2, -vmin[slot][qt]) < 0.f));
-      }
-      if (need_exact) {
+      if (!kDense) {
         const float4* bb = reinterpret_cast<const float4*>(vec[slot][1]) + qt * 8;
-        float c0 = -INFINITY, c1 = -INFINITY;   // two chains of three-input maxima
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const float4 x0 = bb[e];
-          c0 = max3(c0, fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y));
-          c1 = max3(c1, fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w));
+          crit = fmaxf(crit, fmaxf(fmaxf(fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y)),
+                                   fmaxf(fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w))));
         }
-        crit = fmaxf(c0, c1);
+      }
+      // publish the next tile's vectors.  Slot (n+1) % 3 was last read in tile n-2, which every warp has left:
+      // the scores of tile n only exist because all 16 warps delivered P^T of tile n-1, after their tile n-2.
+      // The readers in tile n+1 see the values through the chain arrive (P^T / vote) -> UMMA warp -> scores.
+      if (qt == 0) {
+        const int ns = (slot == 2 ? 0 : slot + 1);
+        vec[ns][0][rl] = nx0; vec[ns][1][rl] = nx1; vec[ns][2][rl] = nx2;
       }
       bool retain = true;
       if (!kDense) {
         const bool vote = valid_key && !(crit < 0.f);
         const bool any = __any_sync(0xffffffffu, vote);
         if (lane == 0) {
-          if (any) *(volatile int*)&flag[n & 3] = 1;
-          if (warp == 4) *(volatile int*)&flag[(n + 1) & 3] = 0;
+          if (any) *(volatile int*)&flag[slot] = 1;
+          if (warp == 4) *(volatile int*)&flag[slot == 2 ? 0 : slot + 1] = 0;
           tc_fence_before();
           mbar_arrive(&vote_bar[n & 1]);
         }
@@ -545,29 +417,22 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           ok = mbar_wait(&vote_bar[n & 1], (n >> 1) & 1, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          retain = (*(volatile int*)&flag[n & 3]) != 0;
+          retain = (*(volatile int*)&flag[slot]) != 0;
         }
       }
       if (!kDense) retain = __all_sync(0xffffffffu, retain);   // same value in every lane: the branch below is uniform
-      // where the next scores will be (see the issuer): they were issued ahead into the other region iff the
-      // previous tile was skipped; a retained tile abandons them and has them issued again into its own region
-      {
-        const bool spec = !kDense && !(rs & 2u) && (n + 1 < n_tot);
-        rs = retain ? (rs | 2u) : (rs & ~2u);
-        if (spec) rs ^= retain ? (8u >> reg) : 1u;
-      }
-      if (stat_thread && first_of_head) { stat_r_head = 0; stat_bits = 0; stat_word = -1; }
+      if (stat_thread && first_of_head) { r_head = 0; bm_bits = 0; bm_word = -1; }
       if (retain) {
         if (stat_thread) {
-          ++stat_r_head;
+          ++r_head;
           if (p.bitmask) {
             uint32_t* bm_row = p.bitmask + ((size_t)(b * p.Hq + hkv * G + hq_n) * p.Tk + j) * p.words;
-            if ((i >> 5) != stat_word) {
-              if (stat_word >= 0) bm_row[stat_word] = stat_bits;
-              stat_word = i >> 5;
-              stat_bits = 0;
+            if ((i >> 5) != bm_word) {
+              if (bm_word >= 0) bm_row[bm_word] = bm_bits;
+              bm_word = i >> 5;
+              bm_bits = 0;
             }
-            stat_bits |= 1u << (i & 31);
+            bm_bits |= 1u << (i & 31);
           }
         }
         // P^T = exp2(s * c2 - lse2_q) (bf16), written over S^T in TMEM as the A operand of dV
@@ -585,7 +450,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             pk[2 * e + 1] = pack_bf16x2(p2, p3);
           }
         }
-        tmem_st_x16(tmem_addr(tb, lane_base, colS + qt * 32), pk);
+        tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColS + qt * 32), pk);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -599,7 +464,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         uint32_t w[16];
         {
           uint32_t dp[32];
-          tmem_ld_x32(tmem_addr(tb, lane_base, colDP + qt * 32), dp);
+          tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + qt * 32), dp);
           tmem_wait_ld();
           const float4* dd = reinterpret_cast<const float4*>(vec[slot][2]) + qt * 8;
 #pragma unroll
@@ -613,7 +478,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
         // dS^T also goes to TMEM, over this thread's own (already consumed) dP^T columns: A operand of dK
-        tmem_st_x16(tmem_addr(tb, lane_base, colDP + qt * 32), w);
+        tmem_st_x16(tmem_addr(tb, lane_base, Cfg::kColDP + qt * 32), w);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -633,14 +498,12 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (lane == 0) mbar_arrive(&ds_full);
         ++r;
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&vec_empty[slot]);   // this warp has read the tile's vectors for the last time
       if (stat_thread && last_of_head) {   // last tile of this query head
         const size_t row = (size_t)(b * p.Hq + hkv * G + hq_n) * p.Tk + j;
-        if (p.bitmask && stat_word >= 0) p.bitmask[row * p.words + stat_word] = stat_bits;
-        if (p.retained) p.retained[row] = (uint32_t)stat_r_head;
+        if (p.bitmask && bm_word >= 0) p.bitmask[row * p.words + bm_word] = bm_bits;
+        if (p.retained) p.retained[row] = (uint32_t)r_head;
         if (p.totals) {
-          atomicAdd(&p.totals[0], (unsigned long long)stat_r_head);
+          atomicAdd(&p.totals[0], (unsigned long long)r_head);
           atomicAdd(&p.totals[1], (unsigned long long)ni);
         }
       }
@@ -692,7 +555,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // registers; the others are staged as 32-column swizzled panels in the tile's dS^T stage -- free once
     // dQ has retired -- and added by TMA reduce-add; the stage goes back to the dO ring when the TMA has
     // read it.
-    reg_alloc<144>();
+    reg_alloc<152>();
     const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
     const int rl = (int)lane_base + lane;
     const bool elected = (warp == 20 && lane == 0);
@@ -703,8 +566,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (!ok) break;
       const int info = *(volatile int*)&dq_info;
       if (info < 0) break;
-      const int n = info >> 2, ds = (info >> 1) & 1;
-      const uint32_t colDQ = kDense ? 128u : (uint32_t)(info & 1) * 128u;   // the region that holds this tile's dQ
+      const int n = info >> 1, ds = info & 1;
       // (the tile's coordinates while the dQ MMAs are still running: the announcement precedes their completion)
       const int hq = hkv * G + n / ni, i = i0 + n % ni;
       const int tile = p.cu ? (int)((size_t)hq * (p.Np / 128) + (size_t)(prow0 / 128 + i))
@@ -718,7 +580,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       tc_fence_after();
       uint32_t a[D / 32][32];
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) tmem_ld_x32(tmem_addr(tb, lane_base, colDQ + c * 32), a[c]);
+      for (int c = 0; c < D / 32; ++c) tmem_ld_x32(tmem_addr(tb, lane_base, Cfg::kColDP + c * 32), a[c]);
       tmem_wait_ld();
       tc_fence_before();
       __syncwarp();

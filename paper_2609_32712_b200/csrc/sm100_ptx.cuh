@@ -259,21 +259,6 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-// minimum of a float over the 32 lanes of a converged warp (no NaNs): one integer reduction on keys whose signed
-// order is the order of the floats
-__device__ __forceinline__ float warp_min_f32(float x) {
-  int k = __float_as_int(x);
-  k ^= (k >> 31) & 0x7fffffff;
-  k = __reduce_min_sync(0xffffffffu, k);
-  k ^= (k >> 31) & 0x7fffffff;
-  return __int_as_float(k);
-}
-// maximum of three values in one instruction (sm_100)
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float r;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-  return r;
-}
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
