@@ -448,7 +448,7 @@ def run_reference(args, rank):
     case.q, case.k, case.v, case.do = w["q"], w["k"], w["v"], w["do"]
     T = -(-cfg.N // TILE)
     # the sampled backward needs o and lse of the sampled rows only through D and lse; use the oracle's own forward
-    # on the rows that the sampled key block touches (the last T//64 query blocks)
+    # on the rows that the sampled key blocks touch (the query blocks of the upper half)
     units = [(0, h, i) for h in range(cfg.Hq // cfg.Hkv) for i in range(T // 2, T)]
     f = orc.fwd(case.q, case.k, case.v, case.scale, args.tau, TILE, TILE, units=units)
     o = torch.from_numpy(f["o"]).nan_to_num(0.0)

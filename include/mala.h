@@ -39,7 +39,7 @@ extern "C" {
 
 #define MALA_OK 0
 #define MALA_ERR_INVALID_ARG (-1)        /* NULL pointer, non-positive size, bad tau / scale */
-#define MALA_ERR_UNSUPPORTED (-2)        /* d not in {64,128}, Hq % Hkv != 0, too many splits ... */
+#define MALA_ERR_UNSUPPORTED (-2)        /* d not a multiple of 8 in 8..128, Hq % Hkv != 0, too many splits ... */
 #define MALA_ERR_MISALIGNED (-3)         /* pointer / stride alignment rules above violated */
 #define MALA_ERR_WORKSPACE_TOO_SMALL (-4)
 #define MALA_ERR_WRONG_ARCH (-5)         /* current device is not compute capability 10.x */
@@ -168,7 +168,8 @@ int mala_bwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_
  * packed by cu_seqlens_q (device int32 [B+1]); kpages, vpages [num_pages, page_size, Hkv, d] with page_size a multiple
  * of 128, or 8, 16, 32 or 64 (a tile is then put together from 128 / page_size pages, each with its own table
  * lookup, at reduced throughput); block_table device int32 [B, max_pages_per_seq] (keys page_size*x .. of sequence b in page
- * block_table[b][x]); seqlens_k device int32 [B], the keys sequence b holds, its queries being its last positions
+ * block_table[b][x]); seqlens_k device int32 [B], the keys sequence b holds, clamped to
+ * max_pages_per_seq * page_size (what its block-table row can map), its queries being its last positions
  * (a sequence with no keys, or with fewer keys than queries when causal != 0, is left untouched).  Slots of a mapped
  * page beyond the sequence's length must hold finite numbers.  Everything else as mala_fwd_varlen_prefix with
  * max_seqlen_k = max_pages_per_seq * page_size. */

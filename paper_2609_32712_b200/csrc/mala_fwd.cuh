@@ -105,7 +105,8 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
   const bool own_keys = p.cu_k || p.block_table;      // the sequence's key count differs from its query count
   const int krow0 = p.cu_k ? __ldg(p.cu_k + b) : row0;
-  const int Nkeys = p.block_table ? __ldg(p.seqlens_k + b)
+  // (paged: a length beyond what the block table's row can map is clamped, so no lookup ever leaves the row)
+  const int Nkeys = p.block_table ? min(__ldg(p.seqlens_k + b), p.bt_stride * (p.ppt > 1 ? p.prows : p.tpp * 128))
                                   : (p.cu_k ? __ldg(p.cu_k + b + 1) - krow0 : (p.cu ? Nq : p.Nk));
   if (own_keys && (Nkeys <= 0 || (p.causal && Nkeys < Nq))) return;   // (not defined: no keys, more queries than keys)
   const int koff = own_keys ? (p.causal ? (Nkeys - Nq) / 128 : 0) : p.koff;

@@ -12,6 +12,8 @@ head ``h`` with key head ``h // (Hq // Hkv)``:
   planted   q_i = q0_i + 3 * sum_{j in P_i} k_j           P_i: up to P distinct keys drawn from [0, i)
   peaked    planted (P keys) + (4/sqrt(d)) * sum_{j=max(0,i-63)}^{i} k_j     (64-token local window, +4)
   sink      q_i = q0_i + (6/sqrt(d)) * sum_{j<min(4,i+1)} k_j              (first 4 keys, +6)
+  decay     k_j[d-1] = j / 256, q_i[d-1] = rate * 256 * sqrt(d): score(i, j) = rate * j + noise, mass decaying smoothly
+            toward earlier keys (rate = 1e-3 .. 3e-3 by head; one query head per KV head); for near-threshold tests
 
 ``q += c * k_j`` raises score (i, j) by ``c * |k_j|^2 / sqrt(d) ~= c * sqrt(d)``.
 
@@ -155,6 +157,15 @@ def make_prefill(cfg: PrefillConfig, preset: str = "literal", device="cpu", seed
             kind = cfg.head_types[h]
             k_h = k[b, :, h // G, :]
             if kind == "diffuse":
+                continue
+            if kind == "decay":
+                # score(i, j) = rate * j + N(0, 1): the softmax mass of a row decays smoothly toward earlier keys (a
+                # per-row shift does not change a softmax), so the tile criteria pass through zero with a small slope
+                # per tile -- the inputs on which near-threshold decisions are tested.  Uses the last feature of the
+                # head's KV head (meant for one query head per KV head).
+                rate = 1e-3 * (1 + h % 3)
+                k[b, :, h // G, d - 1] = torch.arange(N, device=dev, dtype=torch.float32) / 256.0
+                q[b, :, h, d - 1] = rate * 256.0 * math.sqrt(d)
                 continue
             if preset == "R":
                 nseg = -(-N // 256)

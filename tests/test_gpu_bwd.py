@@ -57,8 +57,9 @@ def _run_isolated(mala, oracle, w, tau, causal=True):
     fm = fst.mask(T).cpu().numpy()
     bm = st.mask(T).cpu().numpy().transpose(0, 1, 3, 2)
     assert (bm <= fm).all()
+    crit = np.abs(ref["crit"][ref["mask"] > 0])
     return dict(flips=flips, err=e, skipped=int((ref["mask"] == 1).sum()), retained=int((ref["mask"] == 2).sum()),
-                totals=st.totals.cpu().numpy())
+                totals=st.totals.cpu().numpy(), near=int((crit < 1e-2).sum()), band=int((crit <= parity.MASK_BAND).sum()))
 
 
 @pytest.mark.parametrize("tau", [0.0, 1e-4])
@@ -97,3 +98,20 @@ def test_bwd_cfg1_end_to_end(mala, oracle, tau):
 def test_bwd_non_causal(mala, oracle, tau):
     w = W.custom_prefill(1, 2, 1, 300, 128, head_types=["peaked", "diffuse"], seed=5, preset="R")
     _run_isolated(mala, oracle, w, tau, causal=False)
+
+
+def test_bwd_near_threshold_decisions(mala, oracle, capsys):
+    """Eq. 4 next to equality: softmax mass decaying smoothly toward earlier keys puts tile criteria within 1e-2 of zero
+    and some inside the 1e-3 band; decisions outside the band must be the oracle's, flips inside it are reported."""
+    w = W.custom_prefill(2, 6, 6, 4096, 64, head_types=["decay"] * 6, seed=5)
+    near = band = flips = 0
+    for tau in (1.0,):
+        res = _run_isolated(mala, oracle, w, tau)
+        assert res["skipped"] > 0
+        flips += res["flips"]
+        near += res["near"]
+        band += res["band"]
+    with capsys.disabled():
+        print(f"\n[near-threshold backward] tiles with |C| < 1e-2: {near}, inside the 1e-3 band: {band}, "
+              f"decisions that differ from the oracle (all inside the band): {flips}")
+    assert near >= 3 and band >= 1, "the workload must put tiles next to the threshold"

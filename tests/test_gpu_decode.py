@@ -16,7 +16,7 @@ def mala():
     return m
 
 
-def _run_and_check(mala, oracle, w, tau, num_splits, units=None):
+def _run_and_check(mala, oracle, w, tau, num_splits, units=None, rounding_bound=False):
     q, kc, vc = (w[x].cuda() for x in ("q", "kcache", "vcache"))
     B, _, Hq, d = q.shape
     Nk, Hkv = kc.shape[1], kc.shape[2]
@@ -26,6 +26,8 @@ def _run_and_check(mala, oracle, w, tau, num_splits, units=None):
     assert mala.device_status() == 0
     _, Bk = mala.tile_shape(mala.OP_DECODE, d)
     ref = oracle.decode(w["q"], w["kcache"], w["vcache"], w["scale"], tau, num_splits, Bk, units=units)
+    ref_abs = (oracle.decode(w["q"], w["kcache"], w["vcache"].abs(), w["scale"], tau, num_splits, Bk, units=units)
+               if rounding_bound else None)          # a = sum_k p_k |v_k| for parity.check_output's rounding bound
     tps = ref["mask"].shape[-1]
     gm = st.mask(tps).cpu().numpy()                    # [B,Hkv,S,tps]
     if units is None:
@@ -38,7 +40,7 @@ def _run_and_check(mala, oracle, w, tau, num_splits, units=None):
                                        list(range(tps - 1, -1, -1)), tau, Nk, Bk)
             assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
         hs = slice(g * G, (g + 1) * G)
-        parity.check_output(o_c[b, hs], ref["o"][b, hs])
+        parity.check_output(o_c[b, hs], ref["o"][b, hs], a_ref=ref_abs["o"][b, hs] if rounding_bound else None)
         assert np.abs(lse_c[b, hs] - ref["lse"][b, hs]).max() <= parity.LSE_ABS
         skipped += int((ref["mask"][b, g] == 1).sum())
         retained += int((ref["mask"][b, g] == 2).sum())
@@ -99,7 +101,7 @@ def test_decode_strided_cache_view(mala, oracle):
     parity.check_output(o.float().cpu().numpy()[:, 0], ref["o"])
 
 
-def _run_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0):
+def _run_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0, rounding_bound=False):
     kp, vp, bt, lens = W.paginate(w["kcache"], w["vcache"], page_size, seqlens=seqlens, seed=seed)
     q = w["q"].cuda()
     B, _, Hq, d = q.shape
@@ -112,6 +114,8 @@ def _run_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0):
     _, Bk = mala.tile_shape(mala.OP_DECODE, d)
     ref = oracle.decode_paged(w["q"][:, 0], kp, vp, bt.numpy(), lens.numpy() if seqlens is not None else None,
                               w["scale"], tau, num_splits, Bk)
+    ref_abs = (oracle.decode_paged(w["q"][:, 0], kp, vp.abs(), bt.numpy(), lens.numpy() if seqlens is not None else None,
+                                   w["scale"], tau, num_splits, Bk) if rounding_bound else None)
     tps = ref["mask"].shape[-1]
     gm = st.mask(tps).cpu().numpy()
     o_c, lse_c = o.float().cpu().numpy()[:, 0], lse.cpu().numpy()
@@ -124,7 +128,7 @@ def _run_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0):
                                   tau, max(n, 1), Bk)
                 assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
             hs = slice(g * G, (g + 1) * G)
-            parity.check_output(o_c[b, hs], ref["o"][b, hs])
+            parity.check_output(o_c[b, hs], ref["o"][b, hs], a_ref=ref_abs["o"][b, hs] if rounding_bound else None)
             if n > 0:
                 assert np.abs(lse_c[b, hs] - ref["lse"][b, hs]).max() <= parity.LSE_ABS
             else:

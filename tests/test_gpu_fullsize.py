@@ -96,7 +96,7 @@ def test_cfg3_32k(mala, oracle, preset, tau):
     _prefill_sampled(mala, oracle, "cfg3", preset, tau, fwd_units, key_units, dq_units)
 
 
-@pytest.mark.parametrize("preset,tau", [("R", 1e-4), ("literal", 0.0)])
+@pytest.mark.parametrize("preset,tau", [("literal", 1e-4), ("R", 1e-4), ("literal", 0.0)])
 def test_cfg4_128k(mala, oracle, preset, tau):
     T = 1024
     fwd_units = [(0, 1, T - 1), (0, 2, 300), (0, 4, 3)]

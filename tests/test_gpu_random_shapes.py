@@ -1,5 +1,12 @@
 """Seeded sweep over randomly drawn shapes, head layouts, tolerances and presets for every entry point, each case
-checked against the fp64 oracle by the helpers of the other GPU test files."""
+checked against the fp64 oracle by the helpers of the other GPU test files.
+
+The draws on which the absolute output limits (max-abs 2e-2, mean-abs 2e-3) do not hold are kept as named cases at the
+end of the file.  They are of two kinds: outputs of magnitude 4-5 (the bf16 spacing of the OUTPUT alone is 0.031 there),
+and decode calls with one query head per KV head whose softmax sits on one key, where the mean is taken over that one
+head's few dozen outputs of magnitude ~1.  Both are checked against the rounding model of the kernels instead
+(parity.check_output with a_ref: |o_gpu - o| <= 2^-8 (|o| + sum_k p_k |v_k|) element by element, the absolute max-abs
+limit wherever |o| <= 3), at the drawn tolerance and at tau = 0, where the dense kernel must show the same error."""
 import random
 
 import pytest
@@ -26,12 +33,12 @@ def _heads(rng):
     return hkv * g, hkv
 
 
-@pytest.mark.parametrize("seed", [2, 3, 4])
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 4, 11])
 def test_random_cases(mala, oracle, seed):
     _sweep(mala, oracle, seed, [64, 128], 40)
 
 
-@pytest.mark.parametrize("seed", [5, 6])
+@pytest.mark.parametrize("seed", [0, 1, 5, 6])
 def test_random_cases_any_head_size(mala, oracle, seed):
     _sweep(mala, oracle, seed, list(range(8, 129, 8)), 40)
 
@@ -78,13 +85,14 @@ def _sweep(mala, oracle, seed, head_sizes, n):
             Nk, S = rng.randint(1, 5000), rng.randint(1, 12)
             w = W.custom_decode(rng.choice([1, 2, 3]), Hkv * G, Hkv, Nk, d, S, seed=rng.randint(0, 9999),
                                 preset=rng.choice(["literal", "D"]))
-            TD._run_and_check(mala, oracle, w, tau, S)
+            # (one query row per KV head: the mean error is then a mean over ONE head's d outputs, see the file header)
+            TD._run_and_check(mala, oracle, w, tau, S, rounding_bound=(G == 1))
         elif kind == "paged":
             Hkv, G, page = rng.choice([1, 2]), rng.choice([1, 2, 4, 8]), rng.choice([128, 256, 512])
             Nk, S, B = page * rng.randint(1, 12), rng.randint(1, 8), rng.choice([1, 2, 3])
             lens = [rng.randint(0, Nk) for _ in range(B)]
             w = W.custom_decode(B, Hkv * G, Hkv, Nk, d, S, seed=rng.randint(0, 9999), preset=rng.choice(["literal", "D"]))
-            TD._run_paged(mala, oracle, w, tau, S, page, lens, seed=it)
+            TD._run_paged(mala, oracle, w, tau, S, page, lens, seed=it, rounding_bound=(G == 1))
         else:
             Hkv, G = rng.choice([1, 2]), rng.choice([1, 2, 4])
             Sq = rng.randint(2, 16 // G)
@@ -92,3 +100,44 @@ def _sweep(mala, oracle, seed, head_sizes, n):
             w = W.custom_decode(rng.choice([1, 2]), Hkv * G, Hkv, Nk, d, S, seed=rng.randint(0, 9999),
                                 preset=rng.choice(["literal", "D"]))
             TD._run_multi(mala, oracle, w, Sq, tau, S, seed=it)
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# Named draws outside the absolute limits (found by the sweep above over more seeds), checked against the rounding model
+
+LARGE_OUTPUT_PREFILL = [(28, 200), (6, 200), (2, 333)]     # (seed, N): d = 64 "planted" heads, |o| up to 4.5 - 5.0
+
+
+@pytest.mark.parametrize("seed,N", LARGE_OUTPUT_PREFILL)
+def test_named_large_outputs_follow_the_bf16_rounding_model(mala, oracle, seed, N):
+    w = W.custom_prefill(1, 2, 2, N, 64, head_types=["planted", "planted"], seed=seed)
+    res = {tau: TF._run_and_check(mala, oracle, w, tau, rounding_bound=True) for tau in (1e-4, 0.0)}
+    assert res[1e-4]["o_absmax"] > 4.4, "the case is here for its large outputs"
+    # the dense kernel (tau = 0) shows the same error on the same inputs: a rounding effect, not an effect of the rule
+    assert res[0.0]["max_err"] >= 0.5 * res[1e-4]["max_err"]
+    assert res[1e-4]["max_err"] <= parity_bound_at(res[1e-4]["o_absmax"])
+
+
+def parity_bound_at(o_absmax):
+    """Largest error the rounding model allows for an output of this magnitude whose softmax sits on one key."""
+    from tests import parity
+    return parity.BF16_U * 2.0 * o_absmax * 1.02 + 1e-5
+
+
+SINGLE_HEAD_DECODE = [
+    dict(kind="decode", B=3, Hkv=3, G=1, Nk=4123, S=1, d=64, seed=6177, preset="literal", tau=0.01),
+    dict(kind="decode", B=3, Hkv=3, G=1, Nk=3926, S=4, d=56, seed=1000, preset="literal", tau=0.0),
+    dict(kind="paged", B=2, Hkv=2, G=1, Nk=4096, S=2, d=64, seed=9384, preset="literal", tau=0.0, page=512,
+         lens=[247, 4095], page_seed=20),
+]
+
+
+@pytest.mark.parametrize("case", SINGLE_HEAD_DECODE, ids=lambda c: f"{c['kind']}-seed{c['seed']}")
+def test_named_single_head_decode_follows_the_bf16_rounding_model(mala, oracle, case):
+    c = case
+    w = W.custom_decode(c["B"], c["Hkv"] * c["G"], c["Hkv"], c["Nk"], c["d"], c["S"], seed=c["seed"], preset=c["preset"])
+    for tau in sorted({c["tau"], 0.0}):          # the drawn tolerance and the dense kernel
+        if c["kind"] == "decode":
+            TD._run_and_check(mala, oracle, w, tau, c["S"], rounding_bound=True)
+        else:
+            TD._run_paged(mala, oracle, w, tau, c["S"], c["page"], c["lens"], seed=c["page_seed"], rounding_bound=True)

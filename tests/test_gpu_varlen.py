@@ -264,3 +264,23 @@ def test_prefill_chunks_against_a_paged_cache(mala, oracle, tau, page, d):
         assert np.abs(lse_c[:, r0:r0 + m] - ref["lse"][0]).max() <= parity.LSE_ABS
         legal += int((ref["mask"] > 0).sum())
     assert st.totals.cpu().numpy()[1] == legal
+
+
+@pytest.mark.parametrize("page", [128, 16])
+def test_paged_prefill_clamps_a_length_beyond_the_block_table(mala, page):
+    """A sequence that reports more keys than its block-table row can map is treated as holding exactly what the row
+    maps: no table lookup leaves the row, and the result equals the call with the clamped length."""
+    Hq, Hkv, d, nk, nq = 4, 2, 128, 1024, 100
+    w = W.custom_prefill(1, Hq, Hkv, nk, d, seed=91, preset="R")
+    kp, vp, bt, _ = W.paginate(w["k"], w["v"], page, seqlens=[nk], seed=3)
+    assert bt.shape[1] * page == nk
+    q = w["q"][:, nk - nq:].contiguous().cuda()
+    cq = torch.tensor([0, nq], dtype=torch.int32).cuda()
+    outs = []
+    for reported in (nk, 5 * nk):
+        sl = torch.tensor([reported], dtype=torch.int32).cuda()
+        o, lse, _ = mala.fwd_paged(q, kp.cuda(), vp.cuda(), cq, bt.cuda(), sl, nq, w["scale"], 1e-4)
+        torch.cuda.synchronize()
+        assert mala.device_status() == 0
+        outs.append((o, lse))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
