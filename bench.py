@@ -11,6 +11,10 @@ MALA and dense kernels on cfg3 / cfg4 (literal and paper-regime "R" inputs), dec
 figures (retained slots, omitted mass, relative L2 against the dense path) at tau = 1e-4, 1e-2 and 1.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py --only fwd|bwd|decode --workload cfg2 --preset R --tau 1e-4 --iters 3
+      (a few launches of one operator and nothing else: the small fixed command profiler captures are taken on)
+  python bench.py --workload tp8 [--preset S --tau 1] (under torchrun --nproc-per-node 8: one tensor-parallel rank's
+      head slice of the paper's 128K operator benchmark per GPU, timed as the synchronized wall clock of the group)
 """
 from __future__ import annotations
 
@@ -53,6 +57,31 @@ def load_peaks():
         return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
                     source="measured")
     return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+def load_dram_traffic(workload, preset, tau):
+    """DRAM bytes of one launch of the dominant kernel on (workload, preset, tau), from the table kept beside the ncu
+    summaries it was read from (profiles/dram_traffic.txt); None where no capture exists."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None, None
+    with open(path) as f:
+        for line in f:
+            t = line.split()
+            if len(t) >= 6 and not line.startswith("#") and t[0] == workload and t[1] == preset and float(t[2]) == tau:
+                return float(t[4]), t[5]
+    return None, None
+
+
+def clk_per_tile(mala_ms, dense_ms, retained, legal, sm_mhz, n_sm=148):
+    """SM clocks one SM spends per retained and per skipped tile: the dense kernel's time over all legal tiles gives
+    the retained figure, the MALA kernel's time minus the retained share of the dense time the skipped one."""
+    if not sm_mhz or legal <= 0:
+        return None, None
+    per_ret = dense_ms * 1e-3 * sm_mhz * 1e6 * n_sm / legal
+    skipped = legal - retained
+    per_skip = ((mala_ms - retained / legal * dense_ms) * 1e-3 * sm_mhz * 1e6 * n_sm / skipped) if skipped > 0 else None
+    return per_ret, per_skip
 
 
 class ClockSampler:
@@ -370,6 +399,35 @@ def serving_prefill_leg(cfg, preset, tau, it, peaks, dev):
     return row
 
 
+def head_type_leg(cs, tau, it):
+    """Per head type of a prefill case (one query head of each KV group, run as a multi-head call on strided views):
+    retained fraction and latency of the MALA and dense kernels, so that the skip path's throughput can be read for
+    the sparse head types alone."""
+    import torch
+    mala, cc = cs.mala, cs.cfg
+    G = cc.Hq // cc.Hkv
+    rows = {}
+    for t in range(G):
+        q, do = cs.q[:, :, t::G], cs.do[:, :, t::G]                 # head h = G g + t of every group g: its own KV head
+        o, dq = torch.empty_like(q), torch.empty_like(q)
+        lse = torch.empty((cc.B, cc.Hkv, cc.N), dtype=torch.float32, device=q.device)
+        taus = {"mala": tau, "dense": 0.0}
+        fwd = {k_: (lambda t_=t_: mala.fwd(q, cs.k, cs.v, cs.scale, t_, out=o, lse=lse)) for k_, t_ in taus.items()}
+        bwd = {k_: (lambda t_=t_: mala.bwd(q, cs.k, cs.v, o, do, lse, cs.scale, t_, ws=cs.ws, dq=dq, dk=cs.dk, dv=cs.dv))
+               for k_, t_ in taus.items()}
+        f_t, b_t = time_alternating(fwd, 3, it), time_alternating(bwd, 3, it, prep=fwd)
+        _, _, fs = mala.fwd(q, cs.k, cs.v, cs.scale, tau, out=o, lse=lse, stats=True)
+        _, _, _, bs = mala.bwd(q, cs.k, cs.v, o, do, lse, cs.scale, tau, ws=cs.ws, dq=dq, dk=cs.dk, dv=cs.dv, stats=True)
+        torch.cuda.synchronize()
+        (fr, fl), (br, bl) = fs.totals.cpu().tolist(), bs.totals.cpu().tolist()
+        kind = cc.head_types[t] if cs.preset == "literal" else ("diffuse" if (cc.head_types[t] == "diffuse" and cs.preset == "R") else "anchor+retrieval")
+        rows[f"type{t}:{kind}"] = {"heads": cc.Hkv, "fwd_retained_frac": fr / fl, "bwd_retained_frac": br / bl,
+                                   "fwd_ms": f_t["mala"], "bwd_ms": b_t["mala"], "dense_fwd_ms": f_t["dense"],
+                                   "dense_bwd_ms": b_t["dense"], "speedup_fwd": f_t["dense"] / f_t["mala"],
+                                   "speedup_bwd": b_t["dense"] / b_t["mala"]}
+    return rows
+
+
 def fidelity(cs, taus, it):
     """Work and operator fidelity of MALA against the in-library dense path on one configuration (the protocol
     of Section 5.1 on synthetic states): retained slots per query in forward and backward, omitted softmax mass
@@ -442,10 +500,13 @@ def run_reference(args, rank):
     class Host:
         pass
     cfg = W.prefill_config(args.workload)
-    w = W.make_prefill(cfg, preset=args.preset, device="cpu")
+    # the inputs of the GPU arm: drawn by the same generator on the same kind of device (a CUDA generator where the
+    # box has a GPU, which it does wherever the GPU arm runs), then moved to the host
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = W.make_prefill(cfg, preset=args.preset, device=gen_dev)
     case = Host()
     case.cfg, case.preset, case.scale = cfg, args.preset, w["scale"]
-    case.q, case.k, case.v, case.do = w["q"], w["k"], w["v"], w["do"]
+    case.q, case.k, case.v, case.do = (w[x].cpu() for x in ("q", "k", "v", "do"))
     T = -(-cfg.N // TILE)
     # the sampled backward needs o and lse of the sampled rows only through D and lse; use the oracle's own forward
     # on the rows that the sampled key blocks touch (the query blocks of the upper half)
@@ -466,11 +527,36 @@ def run_reference(args, rank):
         "impl": "reference", "metric": "mala_fwd_bwd_dense_equiv_tflops", "value": val, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{args.workload} {args.preset} tau={args.tau}", "sample": what},
+        "config": {"workload": f"{args.workload} {args.preset} tau={args.tau}", "sample": what,
+                   "inputs": f"seeded generator on {gen_dev} (the GPU arm's tensors), moved to the host"},
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": what},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
+
+
+def run_only(args, dev):
+    """--only: a few launches of one operator on one synthetic configuration, nothing else."""
+    import dataclasses
+    import torch
+    from paper_2609_32712_b200 import mala, workloads as W
+    if args.only == "decode":
+        cfg = dataclasses.replace(W.decode_config("cfg5"), B=args.decode_batch)
+        w = W.make_decode(cfg, preset=args.preset if args.preset in ("literal", "D") else "literal", device=dev)
+        for _ in range(args.iters):
+            mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], args.tau, cfg.num_splits)
+    else:
+        cfg = W.prefill_config(args.workload)
+        w = W.make_prefill(cfg, preset=args.preset, device=dev)
+        o, lse, _ = mala.fwd(w["q"], w["k"], w["v"], w["scale"], args.tau)
+        for _ in range(args.iters):
+            if args.only == "fwd":
+                mala.fwd(w["q"], w["k"], w["v"], w["scale"], args.tau, out=o, lse=lse)
+            else:
+                mala.bwd(w["q"], w["k"], w["v"], o, w["do"], lse, w["scale"], args.tau)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    print("ok")
 
 
 def main():
@@ -479,13 +565,19 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mala", choices=["mala", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
-    ap.add_argument("--preset", default="literal", choices=["literal", "R"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "tp8"])
+    ap.add_argument("--preset", default="literal", choices=["literal", "R", "S", "D"])
+    ap.add_argument("--only", default=None, choices=["fwd", "bwd", "decode"],
+                    help="run a few launches of one operator on --workload / --preset / --tau and exit (no timing table, "
+                         "no CPU leg): the command that profiler captures are taken on")
+    ap.add_argument("--iters", type=int, default=3, help="launches of --only")
+    ap.add_argument("--decode-batch", type=int, default=2, help="batch size of --only decode (cfg5 shapes otherwise)")
     ap.add_argument("--tau", type=float, default=1e-4)
-    ap.add_argument("--detail-iters", type=int, default=20,
-                    help="timed iterations of each prefill detail measurement (3 warm-up iterations before them; the "
-                         "paper's protocol of 25 warm-up + 100 timed iterations is what the decode legs use, and "
-                         "--detail-iters 100 gives the prefill legs 100 timed iterations too)")
+    ap.add_argument("--detail-iters", type=int, default=None,
+                    help="timed iterations of every prefill detail measurement, after 3 warm-up iterations.  Default: the "
+                         "MALA / dense rows of cfg3 and cfg4 use the paper's protocol (25 warm-up + 100 timed iterations, "
+                         "as the decode rows always do) and the secondary rows (chunks, packed sequences, head types "
+                         "...) 3 + 20; config.protocol in the output says which")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-config detail table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -511,6 +603,10 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     warmup = max(args.warmup, 3)
     peaks = load_peaks()
+
+    if args.only:
+        run_only(args, dev)
+        return
 
     # ---------------------------------------------------------------- main timed region (inputs in HBM)
     case = PrefillCase(args.workload, args.preset, dev, seed_offset=rank)
@@ -553,6 +649,30 @@ def main():
     step_flops = case.fwd_de + case.bwd_de
     value = whole_job_value(step_flops, world, ms_per_step)
 
+    # The paper's operator benchmark: one tensor-parallel rank's head slice per GPU, timed as the synchronized wall
+    # clock of the group (the slowest rank), the dense kernels on the same inputs beside it
+    tp8 = None
+    if args.workload == "tp8":
+        def group_ms(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            t = time_cuda(fn, 0, max(args.steps, 5))
+            return max_over_ranks(t, dev)
+        case.fwd(0.0)
+        d_f, d_b = group_ms(lambda: case.fwd(0.0)), group_ms(lambda: case.bwd(0.0))
+        case.fwd(tau)
+        m_f, m_b = group_ms(lambda: case.fwd(tau)), group_ms(lambda: case.bwd(tau))
+        tp8 = {"ranks": world, "slice": f"Hq={c.Hq} Hkv={c.Hkv} N={c.N} d={c.d} per rank, preset {args.preset}, tau={tau}",
+               "timing": "synchronized wall clock of the group: CUDA events per rank, maximum over the ranks",
+               "mala": {"fwd_ms": m_f, "bwd_ms": m_b}, "dense": {"fwd_ms": d_f, "bwd_ms": d_b},
+               "speedup_fwd": d_f / m_f, "speedup_bwd": d_b / m_b,
+               "paper_context": "8 x H100, TP = 8, tau = 1, about 1024 retained slots per query on the authors' model: "
+                                "forward 2.2x, backward 3.0x, decode 1.6x over FullAttn (other hardware and inputs; "
+                                "context, not a target)"}
+
     if rank != 0:
         if world > 1:
             dist.barrier()
@@ -564,11 +684,11 @@ def main():
     bwd_exec = bwd_executed_flops(ts["bwd_legal"], ts["bwd_retained"], c.d)
     fwd_exec = fwd_executed_flops(ts["fwd_legal"], ts["fwd_retained"], c.d)
     ach = bwd_exec / (bwd_ms * 1e-3) / 1e12
-    # DRAM bytes of one mala_bwd_kernel launch from the committed ncu capture of the same workload
-    # (profiles/mala_bwd_kernel_cfg3_literal_tau1e-4.txt: dram__bytes.sum.per_second x gpu__time_duration.sum)
-    traffic = {("cfg3", "literal", 1e-4): 101.735456e9 * 21.403424e-3}.get((args.workload, args.preset, tau))
+    # DRAM bytes of one mala_bwd_kernel launch: from the table of committed ncu captures, null where none exists
+    traffic, traffic_src = load_dram_traffic(args.workload, args.preset, tau)
     roofline = {"bound": "tensor", "kernel": "mala_bwd_kernel", "achieved": ach, "peak": peaks["tflops_sustained"],
                 "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": traffic,
+                "traffic_source": traffic_src,
                 "peak_source": f"{peaks['source']} (bf16 matmul, sustained)",
                 "note": "duration = whole mala_bwd call (preprocess + main + dQ convert), so frac is a lower bound",
                 "fwd": {"kernel": "mala_fwd_kernel", "achieved": fwd_exec / (fwd_ms * 1e-3) / 1e12,
@@ -654,16 +774,20 @@ def main():
     # ---------------------------------------------------------------- detail: MALA vs dense, per config
     detail = {}
     if world == 1 and not args.no_detail:
-        it = args.detail_iters
+        it = args.detail_iters if args.detail_iters else 20                    # secondary rows
+        main_w, main_it = (3, args.detail_iters) if args.detail_iters else (25, 100)   # MALA / dense rows
         for name in ("cfg3", "cfg4"):
-            for preset in ("literal", "R"):
+            for preset in ("literal", "R", "S"):
                 cs = case if (name == args.workload and preset == args.preset) else PrefillCase(name, preset, dev)
                 cc = cs.cfg
                 row = {}
                 taus = {"mala": tau, "dense": 0.0}
-                f_t = time_alternating({k: (lambda t_=t_: cs.fwd(t_)) for k, t_ in taus.items()}, 3, it)
-                b_t = time_alternating({k: (lambda t_=t_: cs.bwd(t_)) for k, t_ in taus.items()}, 3, it,
+                smp = ClockSampler(local_rank)
+                smp.start()
+                f_t = time_alternating({k: (lambda t_=t_: cs.fwd(t_)) for k, t_ in taus.items()}, main_w, main_it)
+                b_t = time_alternating({k: (lambda t_=t_: cs.bwd(t_)) for k, t_ in taus.items()}, main_w, main_it,
                                        prep={k: (lambda t_=t_: cs.fwd(t_)) for k, t_ in taus.items()})
+                mhz = smp.stop().get("sm_mhz")
                 for label in taus:
                     f_ms, b_ms = f_t[label], b_t[label]
                     row[label] = {"fwd_ms": f_ms, "bwd_ms": b_ms,
@@ -680,6 +804,21 @@ def main():
                                                       / (row["mala"]["bwd_ms"] * 1e-3) / 1e12 / peaks["tflops_sustained"])
                 row["speedup_fwd"] = row["dense"]["fwd_ms"] / row["mala"]["fwd_ms"]
                 row["speedup_bwd"] = row["dense"]["bwd_ms"] / row["mala"]["bwd_ms"]
+                # SM clocks per tile and SM (time x sampled median SM clock / tiles): a retained tile from the dense
+                # kernel, a skipped one from what the MALA kernel takes beyond the retained share of the dense time
+                n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+                fr, fs_ = clk_per_tile(f_t["mala"], f_t["dense"], st["fwd_retained"], st["fwd_legal"], mhz, n_sm)
+                br, bs_ = clk_per_tile(b_t["mala"], b_t["dense"], st["bwd_retained"], st["bwd_legal"], mhz, n_sm)
+                row["clk_per_retained_tile"] = {"fwd": fr, "bwd": br}
+                row["clk_per_skipped_tile"] = {"fwd": fs_, "bwd": bs_}
+                row["sm_mhz_during_row"] = mhz
+                if preset in ("R", "S"):             # per head type: where the retained tiles are, and what each type costs
+                    row["by_head_type"] = head_type_leg(cs, tau, it)
+                if preset == "S":                    # (this repository's addition, like R: every head sparse)
+                    detail[f"{name}_{preset}"] = row
+                    del cs
+                    torch.cuda.empty_cache()
+                    continue
                 if name == "cfg4":                  # a 1024-query chunk against the 128K context, unsplit and split
                     row["chunk_last_1024"] = chunk_split_leg(cs, 1024, tau, it)
                 if name == "cfg3":                  # chunked prefill: the last 8192 queries against all 32768 keys
@@ -796,12 +935,20 @@ def main():
                           if flush_buf is None else
                           f"inputs {case.input_bytes() / 1e6:.0f} MB per step fit in L2: a 252 MB buffer is written between "
                           f"steps, outside the timed events"),
+                   "protocol": ("main timed region: --warmup / --steps; detail rows: cfg3 / cfg4 MALA and dense kernels "
+                                + ("25 warm-up + 100 timed iterations" if not args.detail_iters else
+                                   f"3 warm-up + {args.detail_iters} timed iterations")
+                                + ", in turn over two rounds; secondary rows (chunks, packed sequences, serving batch, "
+                                  "head sizes, head types, fidelity) 3 + "
+                                + str(args.detail_iters if args.detail_iters else 20) + "; decode rows 25 + 100"),
                    "parallelism": "replicas (one head slice per GPU, no collective)" if world > 1 else "single GPU"},
         "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
         "fwd_retained_frac": ts["fwd_retained"] / ts["fwd_legal"], "bwd_retained_frac": ts["bwd_retained"] / ts["bwd_legal"],
         "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * args.steps,   # (timed region: fwd + 3 backward kernels per step)
         "roofline": roofline, "cpu_baseline": cpu_baseline, "detail": detail,
     }
+    if tp8 is not None:
+        out["tp8"] = tp8
     print(json.dumps(out))
     if world > 1:
         dist.barrier()

@@ -275,6 +275,17 @@ int mala_tile_shape(int op, int d, int* Bq, int* Bk);
  * clear != 0, resets it.  Synchronises the device.  HOST pointer. */
 int mala_device_status(int* code_out, int clear);
 
+/* ---- Test support (not part of the operator) ------------------------------------------------------------------
+ * Every wait inside the kernels is bounded (Conventions, last item).  This call makes one such wait run out on
+ * purpose, in the only way that harms nothing: it launches a single small thread block whose one waiting thread
+ * polls, with the kernels' own wait routine, a barrier that nobody ever arrives on, gives up after limit_cycles
+ * clock cycles (1 .. 1e8; the kernels themselves use about 2 s), records MALA_ERR_DEVICE_TIMEOUT in the device's
+ * status word and returns through the normal exit.  Nothing faults, traps or waits without a limit.  Afterwards
+ * mala_device_status reports the code, and every later launch of this library on the device returns at once
+ * without touching its outputs until the word is cleared (mala_device_status with clear != 0).
+ * Asynchronous on cuda_stream; MALA_OK or a negative MALA_ERR_* code (MALA_ERR_INVALID_ARG for a limit out of range). */
+int mala_test_expire_wait(long long limit_cycles, void* cuda_stream);
+
 const char* mala_strerror(int code);
 int mala_version(void);
 

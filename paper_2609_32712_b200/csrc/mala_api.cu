@@ -15,6 +15,16 @@ namespace mala {
 // Sticky per-device status word written by kernels whose bounded waits expire.
 __device__ int g_mala_status;
 
+// The kernels' bounded wait on a barrier that nobody arrives on (test support, see mala_test_expire_wait): the wait
+// gives up after limit_cycles, records the time-out in the status word and the kernel leaves through its normal exit.
+__global__ void expire_wait_kernel(int* status, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); mbar_fence_init(); }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(&bar, 0, status, limit_cycles);
+  __syncthreads();
+}
+
 static std::mutex g_mu;
 static int* g_status_ptr[64];
 static bool g_attr_done[64];
@@ -199,6 +209,16 @@ int mala_device_status(int* code_out, int clear) {
     if (cudaMemcpy(status, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return MALA_ERR_CUDA;
   }
   return MALA_OK;
+}
+
+int mala_test_expire_wait(long long limit_cycles, void* cuda_stream) {
+  if (limit_cycles <= 0 || limit_cycles > 100000000LL) return MALA_ERR_INVALID_ARG;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  expire_wait_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(status, limit_cycles);
+  return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
 // Lengths of a call with N queries and Nk keys: causal needs the queries to be the last N positions of the Nk.

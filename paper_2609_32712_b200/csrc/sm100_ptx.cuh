@@ -53,14 +53,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait for the phase with the given parity.  Returns false after kWaitLimitCycles, or as
 // soon as another thread of the grid has recorded an error; the status word is then non-zero.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status,
+                                          long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t it = 0;
   while (!mbar_try_wait(bar, parity)) {
     if (((++it) & 0xff) == 0) {
       if (*(volatile int*)status != 0) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         atomicCAS(status, 0, kDevTimeout);
         return false;
       }

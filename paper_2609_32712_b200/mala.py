@@ -82,6 +82,8 @@ def lib():
         L.mala_decode_paged.restype = i
         L.mala_decode_static.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, i, i, i, i, i, f, f, i, vp]
         L.mala_decode_static.restype = i
+        L.mala_test_expire_wait.argtypes = [ctypes.c_longlong, vp]
+        L.mala_test_expire_wait.restype = i
         L.mala_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
         L.mala_workspace_bytes.restype = sz
         L.mala_tile_shape.argtypes = [i, i, ctypes.POINTER(i), ctypes.POINTER(i)]
@@ -132,6 +134,13 @@ def device_status(clear: bool = True) -> int:
     if rc != 0:
         raise MalaError(rc, "mala_device_status")
     return code.value
+
+
+def test_expire_wait(limit_cycles: int = 100000) -> None:
+    """mala_test_expire_wait: makes one bounded device-side wait run out (test support)."""
+    rc = lib().mala_test_expire_wait(limit_cycles, _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_test_expire_wait")
 
 
 class Stats:

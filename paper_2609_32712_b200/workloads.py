@@ -23,6 +23,10 @@ tiles): every K row is rescaled to norm sqrt(d); non-diffuse heads use
 ``[0, 256 seg)`` (none for seg 0): a self anchor plus two retrieval keys shared by 256 consecutive
 queries.
 
+Preset ``"S"`` (this repository's addition as well): preset "R" with EVERY head built that way, the diffuse ones
+included -- no head retains everything, which puts the whole configuration at the sparsity the paper reports for
+trained models (about 1000 retained key slots per query).
+
 Preset ``"D"`` (decode): the last feature gates keys -- ``k_j[d-1] = 0`` for live keys and ``-19``
 otherwise, ``q[d-1] = 19`` for non-diffuse KV groups; live keys are one 128-key tile per 1024-key
 chunk (tile ``(5 * chunk + 3) mod 8``) plus the newest 128 keys.
@@ -78,7 +82,7 @@ def _mix4(n: int) -> List[str]:
 
 
 def prefill_config(name: str) -> PrefillConfig:
-    """The four prefill configurations of the benchmark definition, by name ``cfg1`` .. ``cfg4``."""
+    """The four prefill configurations of the benchmark definition, by name ``cfg1`` .. ``cfg4``, and ``tp8``."""
     if name == "cfg1":
         return PrefillConfig("cfg1", 1, 2, 2, 1024, 64, ["planted"] * 2, planted=4, seed=1)
     if name == "cfg2":
@@ -87,6 +91,10 @@ def prefill_config(name: str) -> PrefillConfig:
         return PrefillConfig("cfg3", 1, 32, 8, 32768, 128, _mix4(32), taus=[0.0, 1e-4], seed=3)
     if name == "cfg4":
         return PrefillConfig("cfg4", 1, 8, 2, 131072, 128, _mix4(8), taus=[0.0, 1e-4], seed=4)
+    if name == "tp8":
+        # one tensor-parallel rank's slice of the paper's operator benchmark (64 query / 8 KV heads over 8 ranks):
+        # 8 query heads on 1 KV head, 131072 tokens, head size 128; the 32K configuration's head mix
+        return PrefillConfig("tp8", 1, 8, 1, 131072, 128, _mix4(8), taus=[0.0, 1e-4, 1.0], seed=6)
     raise KeyError(name)
 
 
@@ -147,7 +155,7 @@ def make_prefill(cfg: PrefillConfig, preset: str = "literal", device="cpu", seed
     k = _randn((B, N, Hkv, d), gen, dev)
     v = _randn((B, N, Hkv, d), gen, dev)
     do = _randn((B, N, Hq, d), gen, dev)
-    if preset == "R":
+    if preset in ("R", "S"):
         k = k * (math.sqrt(d) / k.norm(dim=-1, keepdim=True))
     elif preset != "literal":
         raise KeyError(preset)
@@ -156,7 +164,7 @@ def make_prefill(cfg: PrefillConfig, preset: str = "literal", device="cpu", seed
         for h in range(Hq):
             kind = cfg.head_types[h]
             k_h = k[b, :, h // G, :]
-            if kind == "diffuse":
+            if kind == "diffuse" and preset != "S":
                 continue
             if kind == "decay":
                 # score(i, j) = rate * j + N(0, 1): the softmax mass of a row decays smoothly toward earlier keys (a
@@ -167,7 +175,7 @@ def make_prefill(cfg: PrefillConfig, preset: str = "literal", device="cpu", seed
                 k[b, :, h // G, d - 1] = torch.arange(N, device=dev, dtype=torch.float32) / 256.0
                 q[b, :, h, d - 1] = rate * 256.0 * math.sqrt(d)
                 continue
-            if preset == "R":
+            if preset in ("R", "S"):
                 nseg = -(-N // 256)
                 u = torch.rand((nseg, 2), generator=gen, device=dev, dtype=torch.float64)
                 seg = torch.arange(nseg, device=dev, dtype=torch.float64)

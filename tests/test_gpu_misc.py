@@ -207,3 +207,34 @@ def test_autograd_functions_for_chunks_and_packed_sequences(mala):
         assert torch.equal(g[1], kp.grad[:, int(ck[b]):int(ck[b + 1])]) and torch.equal(g[2], vp.grad[:, int(ck[b]):int(ck[b + 1])])
         assert (g[0].float() - qp.grad[:, int(cq[b]):int(cq[b + 1])].float()).abs().max() <= 1e-2 * g[0].float().abs().max()
     assert mala.device_status() == 0
+
+
+def test_an_expired_device_wait_is_reported_and_later_launches_do_nothing_until_cleared(mala, oracle):
+    """The time-out path of the kernels' bounded waits, made to run out in the one harmless way: a single small block
+    waits (with a short limit) on a barrier nobody arrives on and gives up.  Nothing faults, traps or hangs."""
+    w = W.custom_prefill(1, 2, 1, 256, 128, seed=4, preset="R")
+    q, k, v = (w[x].cuda() for x in ("q", "k", "v"))
+    assert mala.device_status() == 0
+    try:
+        mala.test_expire_wait(100000)
+        torch.cuda.synchronize()
+        assert mala.device_status(clear=False) == -8                    # MALA_ERR_DEVICE_TIMEOUT, sticky
+        assert mala.lib().mala_strerror(-8).decode() == "bounded device-side wait expired"
+        # a launch while the word is set returns at once and leaves its outputs alone
+        o = torch.full_like(q, 7.0)
+        lse = torch.full((1, 2, 256), 7.0, dtype=torch.float32, device="cuda")
+        mala.fwd(q, k, v, w["scale"], 1e-4, out=o, lse=lse)
+        torch.cuda.synchronize()
+        assert (o == 7.0).all() and (lse == 7.0).all()
+        assert mala.device_status(clear=False) == -8
+    finally:
+        mala.device_status(clear=True)                                   # read and clear
+    assert mala.device_status() == 0
+    # ... and afterwards the same call computes the right result
+    o, lse, _ = mala.fwd(q, k, v, w["scale"], 1e-4)
+    torch.cuda.synchronize()
+    ref = oracle.fwd(w["q"], w["k"], w["v"], w["scale"], 1e-4, 128, 128)
+    parity.check_output(o.float().cpu().numpy(), ref["o"])
+    assert np.abs(lse.cpu().numpy() - ref["lse"]).max() <= parity.LSE_ABS
+    with pytest.raises(mala.MalaError):
+        mala.test_expire_wait(0)
