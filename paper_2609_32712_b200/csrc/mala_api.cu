@@ -359,14 +359,14 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
   if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
   // (a causal chunk that starts inside a tile: the query blocks follow the positions, (Nk - N) % 128 more rows)
   const int pad_rows = (causal && !cu) ? (Nk0 - N0) % 128 : 0;
-  if (ws_bytes < bwd_workspace_bytes(B, Hq, cu ? total + (cu_k ? 384 : 128) * B0 : N + pad_rows, padded_head_size(d)))
+  if (ws_bytes < bwd_base_workspace_bytes(B, Hq, cu ? total + (cu_k ? 384 : 128) * B0 : N + pad_rows, padded_head_size(d)))
     return MALA_ERR_WORKSPACE_TOO_SMALL;
   int dev = 0;
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
   MALA_TRY(device_setup(dev, &status));
   return bwd_launch(q, k, v, o, dout, lse, dq, dk, dv, st, B0, Hq, Hkv, N0, Nk0, d, causal ? 1 : 0, scale, tau, ws,
-                    status, (cudaStream_t)cuda_stream, cu, total, cu_k, total_k);
+                    ws_bytes, status, (cudaStream_t)cuda_stream, cu, total, cu_k, total_k);
 }
 
 int mala_fwd_chunk_split(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B,

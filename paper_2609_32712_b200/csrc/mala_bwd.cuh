@@ -41,6 +41,10 @@
 #include "sm100_ptx.cuh"
 #include "tensor_map.h"
 
+#ifndef MALA_BWD_TWO_PASS
+#define MALA_BWD_TWO_PASS 1
+#endif
+
 namespace mala {
 
 struct BwdParams {
@@ -71,6 +75,9 @@ struct BwdParams {
   // cu_k[b] .. cu_k[b+1]-1 of k, v, dk, dv; koff and qshift are then derived per sequence, and sequence b owns the
   // padded rows from (cu[b] + 384 b) / 128 * 128 on (a short first block and a ragged last one each need a tile more).
   const int* cu_k;
+  // List mode (second pass behind mala_bwd_scout_kernel): the masks of the retained tiles, rows padded to wpad words
+  const uint32_t* list_mask;   // [B,Hq,Tk,wpad]
+  int wpad;
   float scale, scale_log2;
 };
 
@@ -86,7 +93,32 @@ struct BwdCfg {
   static constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
 };
 
-template <int D, bool kDense>
+// Walks the set bits of the G mask rows of a CTA (query heads of the group, then query blocks, ascending): the tile
+// sequence of the list mode.  Every role keeps its own copy and advances it in step with its tile counter.
+struct ListIter {
+  const uint32_t* m;
+  int wpad, G, h, w;
+  uint32_t bits;
+  __device__ __forceinline__ void init(const uint32_t* mask, int wpad_, int G_) {
+    m = mask; wpad = wpad_; G = G_; h = 0; w = 0; bits = mask[0];
+  }
+  __device__ __forceinline__ bool next(int& h_out, int& i_out) {
+    while (bits == 0u) {
+      if (++w == wpad) { w = 0; if (++h == G) return false; }
+      bits = m[h * wpad + w];
+    }
+    i_out = w * 32 + __ffs(bits) - 1;
+    bits &= bits - 1u;
+    h_out = h;
+    return true;
+  }
+};
+
+constexpr int kBwdListWords = 4096;   // mask words of one CTA's G rows held in shared memory (list mode)
+
+// kList (with kDense): the tiles are those of the mask rows in p.list_mask, all of them retained: no test, no votes,
+// the dense tile pipeline on a sparse tile sequence.
+template <int D, bool kDense, bool kList = false>
 __global__ void __launch_bounds__(768, 1)
 mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDO,
@@ -135,10 +167,38 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     return;
   }
+  static_assert(!kList || kDense, "the list mode runs the dense tile pipeline");
+  __shared__ uint32_t lmask[kList ? kBwdListWords : 1];
+  __shared__ int list_total;
   const int i0 = p.causal ? max(j - koff, 0) : 0;      // first query block that sees key block j
   const int ni = T - i0;
-  const int n_tot = G * ni;
+  int n_tot = G * ni;
   int* status = p.status;
+  if (kList) {
+    // the masks of this CTA's G rows into shared memory, and the number of tiles they hold
+    if (tid == 0) list_total = 0;
+    __syncthreads();
+    int cnt = 0;
+    for (int x = tid; x < G * p.wpad; x += blockDim.x) {
+      const uint32_t wv = __ldg(p.list_mask + (((size_t)b * p.Hq + (size_t)hkv * G + x / p.wpad) * p.Tk + j) * p.wpad + x % p.wpad);
+      lmask[x] = wv;
+      cnt += __popc(wv);
+    }
+    for (int sft = 16; sft > 0; sft >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, sft);
+    if (lane == 0 && cnt) atomicAdd(&list_total, cnt);
+    __syncthreads();
+    n_tot = list_total;
+    if (n_tot == 0) {   // nothing retained in this key block: zero gradients
+      for (int x = threadIdx.x; x < 128 * (p.d / 8); x += blockDim.x) {
+        const int key = j * 128 + x / (p.d / 8), c = (x % (p.d / 8)) * 8;
+        if (key < Nkeys) {
+          *reinterpret_cast<uint4*>(p.dk + (int64_t)bz * p.dk_sb + (int64_t)(krow0 + key) * p.dk_sn + (int64_t)hkv * p.dk_sh + c) = make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(p.dv + (int64_t)bz * p.dv_sb + (int64_t)(krow0 + key) * p.dv_sn + (int64_t)hkv * p.dv_sh + c) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      return;
+    }
+  }
 
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
@@ -178,8 +238,11 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       bool ok = true;
       int issued = 0;
       int hq = hkv * G, i = i0;   // tile n = (query head, query block), kept by increments: no division per tile
+      ListIter it;
+      if (kList) it.init(lmask, p.wpad, G);
       for (int n = 0; n < n_tot && ok; ++n, ++i) {
-        if (i == T) { i = i0; ++hq; }
+        if (kList) { int hl; it.next(hl, i); hq = hkv * G + hl; }
+        else if (i == T) { i = i0; ++hq; }
         const int s = n & 1;
         ok = mbar_wait(&q_empty[s], ((n >> 1) & 1) ^ 1, status);
         if (!ok) break;
@@ -341,9 +404,14 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     auto vec_index = [&](int hq_local, int i) -> size_t {
       return ((size_t)bz * p.Hq + hkv * G + hq_local) * p.Np + (size_t)prow0 + (size_t)i * 128 + rl;
     };
+    // (list mode: the tile sequence comes from the masks; one tile of look-ahead for the vectors' prefetch)
+    ListIter it;
+    int h_nx = 0, i_nx = i0;
+    bool have_nx = true;
+    if (kList) { it.init(lmask, p.wpad, G); have_nx = it.next(h_nx, i_nx); }
     // per-query vectors of tile 0 into slot 0 (published by the first column quarter), then a group sync
     if (qt == 0) {
-      const size_t x = vec_index(0, i0);
+      const size_t x = vec_index(kList ? h_nx : 0, kList ? i_nx : i0);
       vec[0][0][rl] = p.lse2[x];
       vec[0][1][rl] = p.bq[x];
       vec[0][2][rl] = p.Dq[x];
@@ -356,12 +424,13 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // tile n = (query head hq_n of the group, query block i): kept by increments, no division per tile
     int hq_n = 0, i = i0, slot = 0;
     for (int n = 0; n < n_tot && ok; ++n, ++i, slot = (slot == 2 ? 0 : slot + 1)) {
-      if (i == T) { i = i0; ++hq_n; }
-      const bool first_of_head = (i == i0), last_of_head = (i == T - 1);
+      if (kList) { hq_n = h_nx; i = i_nx; have_nx = it.next(h_nx, i_nx); }
+      else if (i == T) { i = i0; ++hq_n; }
+      const bool first_of_head = !kList && (i == i0), last_of_head = !kList && (i == T - 1);
       // prefetch the per-query vectors of the next tile
       float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
       if (qt == 0 && n + 1 < n_tot) {
-        const size_t x = last_of_head ? vec_index(hq_n + 1, i0) : vec_index(hq_n, i + 1);
+        const size_t x = kList ? vec_index(h_nx, i_nx) : (last_of_head ? vec_index(hq_n + 1, i0) : vec_index(hq_n, i + 1));
         nx0 = p.lse2[x]; nx1 = p.bq[x]; nx2 = p.Dq[x];
       }
       ok = mbar_wait(&s_full, n & 1, status);
@@ -560,6 +629,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const int rl = (int)lane_base + lane;
     const bool elected = (warp == 20 && lane == 0);
     if (elected) tma_prefetch_desc(&tmAcc);
+    ListIter it;
+    if (kList) it.init(lmask, p.wpad, G);
     for (int k = 0;; ++k) {
       bool ok = mbar_wait(&dq_info_bar, k & 1, status);
       ok = __all_sync(0xffffffffu, ok);
@@ -568,7 +639,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (info < 0) break;
       const int n = info >> 1, ds = info & 1;
       // (the tile's coordinates while the dQ MMAs are still running: the announcement precedes their completion)
-      const int hq = hkv * G + n / ni, i = i0 + n % ni;
+      int hq = hkv * G + n / ni, i = i0 + n % ni;
+      if (kList) { int hl; it.next(hl, i); hq = hkv * G + hl; }   // (every tile of the list is announced, in order)
       const int tile = p.cu ? (int)((size_t)hq * (p.Np / 128) + (size_t)(prow0 / 128 + i))
                             : (int)(((size_t)b * p.Hq + hq) * p.T + (size_t)i);
       uint8_t* stg = sDS + ds * Cfg::kDsBytes;     // D / 64 panels of 16 KB
@@ -740,12 +812,29 @@ __global__ void bwd_convert_dq_kernel(const float* __restrict__ acc, __nv_bfloat
   *reinterpret_cast<uint4*>(dq + b * sb + row * sn + h * sh + cg * 8) = w;
 }
 
+}  // namespace mala
+#include "mala_bwd_scout.cuh"
+namespace mala {
+
 inline size_t bwd_align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// Two-pass backward (tau > 0): words per mask row (padded to four) and bytes of the masks + row counts of a call with
+// T query blocks and Tk key blocks
+inline int bwd_mask_wpad(int T) { return (((T + 31) / 32) + 3) & ~3; }
+inline size_t bwd_list_bytes(int B, int Hq, int T, int Tk) {
+  return bwd_align256((size_t)B * Hq * Tk * bwd_mask_wpad(T) * sizeof(uint32_t)) + bwd_align256((size_t)B * Hq * Tk * sizeof(uint32_t));
+}
+
 // (Packed sequences: B = 1 and N = total rows + 128 x number of sequences.)
-inline size_t bwd_workspace_bytes(int B, int Hq, int N, int d) {   // d: the padded head size
+inline size_t bwd_base_workspace_bytes(int B, int Hq, int N, int d) {   // d: the padded head size
   const size_t Np = (size_t)((N + 127) / 128) * 128;
   return bwd_align256((size_t)B * Hq * Np * d * sizeof(float)) + 3 * bwd_align256((size_t)B * Hq * Np * sizeof(float));
+}
+// What mala_workspace_bytes reports: the base scratch plus the masks of the two-pass path for as many key blocks as
+// query blocks (a call with more key blocks than that takes the two-pass path only if it is given room for them).
+inline size_t bwd_workspace_bytes(int B, int Hq, int N, int d) {
+  const int T = (N + 127) / 128;
+  return bwd_base_workspace_bytes(B, Hq, N, d) + bwd_list_bytes(B, Hq, T, T);
 }
 
 inline bool bwd_set_attributes() {
@@ -754,20 +843,31 @@ inline bool bwd_set_attributes() {
   ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes) == cudaSuccess;
   ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_kernel<64, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_scout_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoutCfg<128>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_bwd_scout_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoutCfg<64>::kSmemBytes) == cudaSuccess;
   return ok;
 }
 
-template <int D, bool kDense>
+template <int D, bool kDense, bool kList = false>
 inline int bwd_launch_main(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                            const CUtensorMap& tacc, const BwdParams& p, cudaStream_t stream) {
   dim3 grid(p.Tk, p.Hkv, p.B);
-  mala_bwd_kernel<D, kDense><<<grid, BwdCfg<D>::kThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, tacc, p);
+  mala_bwd_kernel<D, kDense, kList><<<grid, BwdCfg<D>::kThreads, BwdCfg<D>::kSmemBytes, stream>>>(tq, tk, tv, tdo, tacc, p);
+  return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
+}
+
+template <int D>
+inline int bwd_launch_scout(const CUtensorMap& tq, const CUtensorMap& tk, const ScoutParams& sp, cudaStream_t stream) {
+  dim3 grid((sp.Tk + 1) / 2, sp.Hkv, sp.B);
+  mala_bwd_scout_kernel<D><<<grid, ScoutCfg<D>::kThreads, ScoutCfg<D>::kSmemBytes, stream>>>(tq, tk, sp);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 
 inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
                       mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int Nk, int d,
-                      int causal, float scale, float tau, void* ws, int* status, cudaStream_t stream,
+                      int causal, float scale, float tau, void* ws, size_t ws_bytes, int* status, cudaStream_t stream,
                       const int* cu = nullptr, int total = 0, const int* cu_k = nullptr, int total_k = 0) {
   // Packed sequences (cu): N = Nk = the longest sequence; the tensors are [1, total, H, d]; the per-query vectors and
   // the dQ accumulator are laid out per head over Np = total + 128 B rows (rounded up to a tile).
@@ -809,6 +909,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   p.cu = cu; p.cu_k = cu_k; p.d = d;
   if (cu_k) { p.koff = 0; p.qshift = 0; }    // per sequence, on the device
   p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
+  p.list_mask = nullptr; p.wpad = 0;
   if (p.bitmask &&
       cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * Tk * p.words * sizeof(uint32_t), stream) != cudaSuccess)
     return MALA_ERR_CUDA;
@@ -824,9 +925,37 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   }
   const bool dense = (tau == 0.f);
+  // tau > 0: two passes where their limits hold and the workspace has room for the masks -- the test of every legal
+  // tile first (mala_bwd_scout_kernel), then the dense tile pipeline on the retained tiles only; otherwise the one-pass
+  // kernel that tests and works tile by tile.
+  const int wpad = bwd_mask_wpad(T);
+  const size_t base_bytes = bwd_align256((size_t)Bl * Hq * Np * D * sizeof(float)) + 3 * vbytes;
+  const bool two_pass = !dense && MALA_BWD_TWO_PASS && (Hq / Hkv) * wpad <= kBwdListWords && T <= 32 * ScoutCfg<128>::kMaskWords &&
+                        ws_bytes >= base_bytes + bwd_list_bytes(B, Hq, T, Tk);
   int rc;
-  if (D == 128) rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, tacc, p, stream);
-  else rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, tacc, p, stream);
+  if (two_pass) {
+    uint8_t* lw = (uint8_t*)ws + base_bytes;
+    ScoutParams sp;
+    sp.bq = bq;
+    sp.mask = (uint32_t*)lw;
+    sp.row_count = (uint32_t*)(lw + bwd_align256((size_t)B * Hq * Tk * wpad * sizeof(uint32_t)));
+    sp.tel_retained = p.retained; sp.tel_bitmask = p.bitmask; sp.totals = p.totals;
+    sp.status = status;
+    sp.B = B; sp.Hq = Hq; sp.Hkv = Hkv; sp.N = N; sp.Np = Np; sp.T = T; sp.words = p.words; sp.wpad = wpad; sp.causal = causal;
+    sp.Nk = Nk; sp.Tk = Tk; sp.koff = p.koff; sp.qshift = p.qshift; sp.cu = cu; sp.cu_k = cu_k;
+    sp.scale_log2 = p.scale_log2;
+    rc = (D == 128) ? bwd_launch_scout<128>(tq, tk, sp, stream) : bwd_launch_scout<64>(tq, tk, sp, stream);
+    if (rc != MALA_OK) return rc;
+    BwdParams pl = p;
+    pl.retained = nullptr; pl.bitmask = nullptr; pl.totals = nullptr;   // (the first pass wrote the telemetry)
+    pl.list_mask = sp.mask; pl.wpad = wpad;
+    rc = (D == 128) ? bwd_launch_main<128, true, true>(tq, tk, tv, tdo, tacc, pl, stream)
+                    : bwd_launch_main<64, true, true>(tq, tk, tv, tdo, tacc, pl, stream);
+  } else if (D == 128) {
+    rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, tacc, p, stream);
+  } else {
+    rc = dense ? bwd_launch_main<64, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<64, false>(tq, tk, tv, tdo, tacc, p, stream);
+  }
   if (rc != MALA_OK) return rc;
   {
     const long long n_out = (long long)B * Hq * Npg * (D / 8);

@@ -1,0 +1,316 @@
+// First pass of the MALA backward (Algorithm 2): the offline test of Eq. 4 for every legal tile, and nothing else.
+//
+// The backward test of a tile depends only on its scores and on the saved log-normalizers, not on any other tile, so
+// the retained support of a key block can be found before any gradient work starts.  This kernel does that at the rate
+// the tensor pipe forms the scores: one CTA per (pair of key blocks, KV head, batch) keeps both K tiles in shared
+// memory (a Q tile then feeds two score tiles: at one key block per CTA the kernel was bound by the delivery of the Q
+// tiles, 32 KB per tile from L2), streams the Q tiles of the group's query heads through a ring of four stages, forms
+// S^T = K_j Q_i^T into one of four TMEM buffers, and four warpgroups -- one per buffer -- read their buffer and test it
+// while the next three score tiles are in flight.  Nothing waits for a vote: a warp that finds a retained entry sets the tile's bit in a shared-memory copy of
+// the row's mask, and the row is written out when the head's last tile has been tested.  The second pass
+// (mala_bwd_kernel in its list mode) then visits the retained tiles only and runs the dense tile pipeline on them.
+//
+// Output, per (batch, query head, key block j): the row's mask (bit i set iff tile (j, i) is retained; rows padded to
+// a multiple of four words) and its number of set bits.
+//
+// Warp roles (640 threads): warp 0 TMA producer (K_j once, Q ring), warp 1 UMMA issuer, warp 2 per-query test offsets
+// (bq = lse2 + log2(tau / L_q) of the tile's 128 queries into a ring of four shared-memory slots, with the minimum of
+// each 32-column chunk), warps 4-19 the four test groups (thread = key row).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "../../include/mala.h"
+#include "sm100_ptx.cuh"
+#include "tensor_map.h"
+
+namespace mala {
+
+struct ScoutParams {
+  const float* bq;            // [B,Hq,Np] lse2 + log2(tau / L_q); +inf on padding rows
+  uint32_t* mask;             // [B,Hq,Tk,wpad] (packed sequences: B entries as well)
+  uint32_t* row_count;        // [B,Hq,Tk]
+  uint32_t* tel_retained;     // telemetry (may be null): [B,Hq,Tk]
+  uint32_t* tel_bitmask;      // telemetry (may be null): [B,Hq,Tk,words], zero-filled by the host
+  unsigned long long* totals; // telemetry (may be null)
+  int* status;
+  int B, Hq, Hkv, N, Np, T, words, wpad, causal;
+  int Nk, Tk, koff, qshift;
+  const int* cu;
+  const int* cu_k;
+  float scale_log2;
+};
+
+template <int D>
+struct ScoutCfg {
+  static constexpr int kPanels = D / 64;
+  static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kStages = 4;
+  static constexpr int kSmemBytes = (2 + kStages) * kTileBytes + 1024;   // K of two key blocks, Q ring
+  static constexpr int kThreads = 640;
+  static constexpr int kMaskWords = 256;     // words of one row's mask held in shared memory (query blocks / 32)
+};
+
+template <int D>
+__global__ void __launch_bounds__(640, 1)
+mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                      const ScoutParams p) {
+  using Cfg = ScoutCfg<D>;
+  constexpr int PAN = Cfg::kPanels;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sK = smem;                          // key blocks ja, jb
+  uint8_t* sQ = sK + 2 * Cfg::kTileBytes;      // 4 stages
+
+  __shared__ uint64_t k_full, q_full[4], q_empty[4], s_full[4], s_empty[4], vec_full[4], vec_empty[4], fin_bar;
+  __shared__ __align__(16) float vec[4][128];  // [sub-tile & 3][query column]: bq
+  __shared__ float vmin[4][4];                 // [sub-tile & 3][32-column chunk]: smallest bq of the chunk
+  __shared__ uint32_t rowmask[2][2][Cfg::kMaskWords];   // [head parity][key block of the pair][word]
+  __shared__ uint32_t row_pop[2][2];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int early_exit;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ja = 2 * (int)blockIdx.x, jb = ja + 1, hkv = blockIdx.y, b = blockIdx.z;
+  const int G = p.Hq / p.Hkv;
+  // this sequence (the geometry of mala_bwd_kernel)
+  const int row0 = p.cu ? __ldg(p.cu + b) : 0;
+  const int Nq = p.cu ? __ldg(p.cu + b + 1) - row0 : p.N;
+  const int krow0 = p.cu_k ? __ldg(p.cu_k + b) : row0;
+  const int Nkeys = p.cu_k ? __ldg(p.cu_k + b + 1) - krow0 : (p.cu ? Nq : p.Nk);
+  const int koff = p.cu_k ? (p.causal ? (Nkeys - Nq) / 128 : 0) : p.koff;
+  const int qshift = p.cu_k ? (p.causal ? (Nkeys - Nq) % 128 : 0) : p.qshift;
+  const int T = p.cu ? (Nq + qshift + 127) / 128 : p.T;
+  const int bz = p.cu ? 0 : b;
+  const int prow0 = p.cu ? ((row0 + (p.cu_k ? 384 : 128) * b) / 128) * 128 : 0;
+  const int Tk_seq = p.cu ? (Nkeys + 127) / 128 : p.Tk;                      // key blocks of this sequence
+  const bool none = p.cu_k && (Nq <= 0 || (p.causal && Nkeys < Nq));         // (no defined tile at all)
+  const bool has_a = !none && ja < Tk_seq, has_b = !none && jb < Tk_seq;
+  // Q tiles i0a .. T-1 of every head; the second key block's tile exists from i0b on
+  const int i0a = p.causal ? max(ja - koff, 0) : 0;
+  const int i0b = has_b ? (p.causal ? max(jb - koff, 0) : 0) : T;
+  const int ni = has_a ? T - i0a : 0;
+  const int n_tot = G * ni;                                                   // Q tiles of this CTA
+  const size_t out_row0 = ((size_t)b * p.Hq + (size_t)hkv * G) * p.Tk;        // + h * Tk + j
+  int* status = p.status;
+  if (n_tot <= 0) {   // key blocks without queries: empty rows
+    for (int kb = 0; kb < 2; ++kb) {
+      const int j = ja + kb;
+      if (j >= p.Tk) continue;
+      for (int x = tid; x < G * p.wpad; x += blockDim.x)
+        p.mask[(out_row0 + (size_t)(x / p.wpad) * p.Tk + j) * p.wpad + x % p.wpad] = 0u;
+      if (tid < G) {
+        p.row_count[out_row0 + (size_t)tid * p.Tk + j] = 0u;
+        if (p.tel_retained) p.tel_retained[out_row0 + (size_t)tid * p.Tk + j] = 0u;
+      }
+    }
+    return;
+  }
+
+  if (tid == 0) {
+    early_exit = (*(volatile int*)status != 0);
+    mbar_init(&k_full, 1);
+    for (int s = 0; s < 4; ++s) {
+      mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 4);
+      mbar_init(&vec_full[s], 1); mbar_init(&vec_empty[s], 4);
+    }
+    mbar_init(&fin_bar, 1);
+    row_pop[0][0] = row_pop[0][1] = row_pop[1][0] = row_pop[1][1] = 0u;
+    mbar_fence_init();
+  }
+  for (int x = tid; x < 4 * Cfg::kMaskWords; x += blockDim.x) rowmask[0][0][x] = 0u;
+  __syncthreads();
+  if (early_exit) return;
+  if (warp == 0) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tb = tmem_base_s;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
+      mbar_arrive_expect_tx(&k_full, (has_b ? 2 : 1) * Cfg::kTileBytes);
+      for (int pn = 0; pn < PAN; ++pn) {
+        tma_load_4d(sK + pn * 16384, &tmK, &k_full, pn * 64, krow0 + ja * 128, hkv, bz);
+        if (has_b) tma_load_4d(sK + Cfg::kTileBytes + pn * 16384, &tmK, &k_full, pn * 64, krow0 + jb * 128, hkv, bz);
+      }
+      bool ok = true;
+      int hq = hkv * G, i = i0a;
+      for (int n = 0; n < n_tot && ok; ++n) {
+        const int s = n & 3;
+        ok = mbar_wait(&q_empty[s], ((n >> 2) & 1) ^ 1, status);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
+        for (int pn = 0; pn < PAN; ++pn)
+          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128 - qshift, hq, bz);
+        if (++i == T) { i = i0a; ++hq; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer (warp-uniform issue loop)
+    // Q tile n feeds one score tile per key block of the pair (the second one only where it is legal); score tile m
+    // goes to TMEM buffer m & 3
+    const uint32_t leader = elect_one();
+    constexpr uint32_t idesc = make_idesc_bf16(128, 128, false, false);
+    const uint64_t dKa = make_smem_desc(smem_u32(sK), 16, 1024);
+    const uint64_t dKb = make_smem_desc(smem_u32(sK + Cfg::kTileBytes), 16, 1024);
+    const uint64_t dQ0 = make_smem_desc(smem_u32(sQ), 16, 1024);
+    bool ok = mbar_wait_warp(&k_full, 0, status);
+    int m = 0, i = i0a;
+    for (int n = 0; n < n_tot && ok; ++n) {
+      const int s = n & 3;
+      ok = mbar_wait_warp(&q_full[s], (n >> 2) & 1, status);
+      if (!ok) break;
+      const uint64_t dQ = desc_advance(dQ0, s * Cfg::kTileBytes);
+      const int nsub = (i >= i0b) ? 2 : 1;
+      for (int kb = 0; kb < nsub && ok; ++kb, ++m) {
+        const int buf = m & 3;
+        ok = mbar_wait_warp(&s_empty[buf], ((m >> 2) & 1) ^ 1, status);   // the buffer's previous tile has been read
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t dK = kb ? dKb : dKa;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t off = (k >> 2) * 16384 + (k & 3) * 32;
+          mma_ss(tmem_addr(tb, 0, buf * 128), desc_advance(dK, off), desc_advance(dQ, off), idesc, k > 0, leader);
+        }
+        if (leader) tc_commit(&s_full[buf]);
+      }
+      if (leader) tc_commit(&q_empty[s]);
+      if (++i == T) i = i0a;
+    }
+    __syncwarp();
+    if (leader) tc_commit(&fin_bar);
+    mbar_wait_warp(&fin_bar, 0, status);
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ test offsets of every score tile's 128 queries
+    bool ok = true;
+    int hq_l = 0, i = i0a, m = 0;
+    for (int n = 0; n < n_tot && ok; ++n) {
+      const size_t x = ((size_t)bz * p.Hq + hkv * G + hq_l) * p.Np + (size_t)prow0 + (size_t)i * 128 + lane * 4;
+      const float4 v = *reinterpret_cast<const float4*>(p.bq + x);
+      float mn = fminf(fminf(v.x, v.y), fminf(v.z, v.w));
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1));
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2));
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 4));
+      const int nsub = (i >= i0b) ? 2 : 1;
+      for (int kb = 0; kb < nsub && ok; ++kb, ++m) {   // (one slot per score tile: both key blocks get their copy)
+        const int s = m & 3;
+        ok = mbar_wait_warp(&vec_empty[s], ((m >> 2) & 1) ^ 1, status);
+        if (!ok) break;
+        *reinterpret_cast<float4*>(&vec[s][lane * 4]) = v;
+        if ((lane & 7) == 0) vmin[s][lane >> 3] = mn;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&vec_full[s]);
+      }
+      if (++i == T) { i = i0a; ++hq_l; }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ test groups: group g takes the score tiles m = g mod 4
+    const int g = (warp - 4) >> 2;
+    const uint32_t lane_base = (uint32_t)(warp & 3) * 32u;
+    const int rl = (int)lane_base + lane;
+    const float c2 = p.scale_log2;
+    const int st = tid - 128;                      // 0 .. 511 among the test threads
+    bool ok = true;
+    int use = 0;                                   // score tiles this group has taken (parity of its barriers)
+    int m = 0;
+    for (int h = 0; h < G; ++h) {
+      for (int i = i0a; i < T; ++i) {
+        const int nsub = (i >= i0b) ? 2 : 1;
+        for (int kb = 0; kb < nsub; ++kb, ++m) {
+          if ((m & 3) != g || !ok) continue;
+          const int j = ja + kb;
+          const bool valid_key = (j * 128 + rl) < Nkeys;
+          ok = mbar_wait(&s_full[g], use & 1, status);
+          if (ok) ok = mbar_wait(&vec_full[g], use & 1, status);
+          ok = __all_sync(0xffffffffu, ok);
+          ++use;
+          if (!ok) continue;
+          tc_fence_after();
+          const bool diag = p.causal && (i + koff == j);
+          bool vote = false;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t sc[32];
+            tmem_ld_x32(tmem_addr(tb, lane_base, g * 128 + c * 32), sc);
+            tmem_wait_ld();
+            if (diag) {   // entry (key rl, query col) is legal iff rl <= col
+              const uint32_t ninf = 0xff800000u;
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (c * 32 + e < rl) sc[e] = ninf;
+            }
+            // bound first: max_e (s_e c2 - bq_e) <= (max_e s_e) c2 - min_e bq_e (c2 > 0; fma is monotone in each argument)
+            float m0 = __uint_as_float(sc[0]), m1 = __uint_as_float(sc[1]);
+#pragma unroll
+            for (int e = 0; e < 7; ++e) {
+              m0 = max3(m0, __uint_as_float(sc[2 + 4 * e]), __uint_as_float(sc[3 + 4 * e]));
+              m1 = max3(m1, __uint_as_float(sc[4 + 4 * e]), __uint_as_float(sc[5 + 4 * e]));
+            }
+            const float mx = max3(m0, m1, fmaxf(__uint_as_float(sc[30]), __uint_as_float(sc[31])));
+            const bool cand = valid_key && !(fmaf(mx, c2, -vmin[g][c]) < 0.f);
+            if (__any_sync(0xffffffffu, cand)) {
+              const float4* bb = reinterpret_cast<const float4*>(vec[g]) + c * 8;
+              float c0 = -INFINITY, c1 = -INFINITY;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float4 x0 = bb[e];
+                c0 = max3(c0, fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y));
+                c1 = max3(c1, fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w));
+              }
+              vote = vote || (valid_key && !(fmaxf(c0, c1) < 0.f));
+            }
+            // (one retaining entry decides the tile: the other chunks need not be read)
+            if (__any_sync(0xffffffffu, vote)) break;
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(&s_empty[g]);
+            mbar_arrive(&vec_empty[g]);
+          }
+          if (__any_sync(0xffffffffu, vote) && lane == 0) atomicOr(&rowmask[h & 1][kb][i >> 5], 1u << (i & 31));
+        }
+      }
+      // the head's rows are complete when all sixteen warps have passed their last tile of it
+      // (a warp whose wait failed keeps taking part in the barriers: the others must not be left waiting at one)
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      for (int kb = 0; kb < 2; ++kb) {
+        if (ja + kb >= p.Tk) continue;
+        uint32_t* rm = rowmask[h & 1][kb];
+        const size_t orow = out_row0 + (size_t)h * p.Tk + ja + kb;
+        uint32_t pop = 0;
+        for (int x = st; x < p.wpad; x += 512) {
+          const uint32_t wv = x < Cfg::kMaskWords ? rm[x] : 0u;
+          p.mask[orow * p.wpad + x] = wv;
+          if (p.tel_bitmask && x < p.words) p.tel_bitmask[orow * p.words + x] = wv;
+          pop += __popc(wv);
+          if (x < Cfg::kMaskWords) rm[x] = 0u;      // (next written two heads on, behind another barrier)
+        }
+        for (int sft = 16; sft > 0; sft >>= 1) pop += __shfl_xor_sync(0xffffffffu, pop, sft);
+        if (lane == 0 && pop) atomicAdd(&row_pop[h & 1][kb], pop);
+      }
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      if (st < 2 && ja + st < p.Tk) {
+        const uint32_t cnt = row_pop[h & 1][st];
+        row_pop[h & 1][st] = 0u;
+        const size_t orow = out_row0 + (size_t)h * p.Tk + ja + st;
+        p.row_count[orow] = cnt;
+        if (p.tel_retained) p.tel_retained[orow] = cnt;
+        const int legal = st ? max(T - i0b, 0) : ni;
+        if (p.totals && (st == 0 || has_b)) {
+          atomicAdd(&p.totals[0], (unsigned long long)cnt);
+          atomicAdd(&p.totals[1], (unsigned long long)legal);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+}  // namespace mala

@@ -43,7 +43,7 @@ def test_host_only_queries(mala):
     with pytest.raises(mala.MalaError):
         mala.tile_shape(mala.OP_FWD, 256)
     # backward scratch: fp32 dQ accumulator + three fp32 per-row vectors, rows padded to whole tiles
-    assert mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 64) == 2 * 1024 * 64 * 4 + 3 * 2 * 1024 * 4
+    assert mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 64) == 2 * 1024 * 64 * 4 + 3 * 2 * 1024 * 4 + 256 + 256
     # (head sizes between the two kernel widths take the wider one's scratch)
     assert mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 96) == mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 128)
     assert mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 40, 8) == mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 64, 8)
