@@ -44,6 +44,9 @@
 #ifndef MALA_BWD_TWO_PASS
 #define MALA_BWD_TWO_PASS 1
 #endif
+#ifndef MALA_BWD_SAMPLE
+#define MALA_BWD_SAMPLE 1
+#endif
 
 namespace mala {
 
@@ -78,6 +81,10 @@ struct BwdParams {
   // List mode (second pass behind mala_bwd_scout_kernel): the masks of the retained tiles, rows padded to wpad words
   const uint32_t* list_mask;   // [B,Hq,Tk,wpad]
   int wpad;
+  // One-pass kernel behind the first pass: only the heads whose row count is kScoutDirectRow are handled, and dK, dV
+  // are added to what the list-mode launch stored
+  const uint32_t* sel_rows;    // [B,Hq,Tk] or null (all heads)
+  int accum_dkv;
   float scale, scale_log2;
 };
 
@@ -200,6 +207,18 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   }
 
+  // the query heads of the group this CTA handles: all of them, or (one-pass kernel behind the first pass) those whose
+  // rows the first pass left alone
+  __shared__ int hsel[16];
+  __shared__ int nsel_s;
+  if (warp == 0) {   // (one row flag per lane)
+    bool mine = lane < G && lane < 16;
+    if (!kList && !kDense && p.sel_rows)
+      mine = mine && __ldg(p.sel_rows + ((size_t)b * p.Hq + (size_t)hkv * G + lane) * p.Tk + j) == 0xffffffffu;
+    const uint32_t m = __ballot_sync(0xffffffffu, mine);
+    if (mine) hsel[__popc(m & ((1u << lane) - 1u))] = lane;
+    if (lane == 0) nsel_s = __popc(m);
+  }
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
     mbar_init(&kv_full, 1);
@@ -217,7 +236,8 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     mbar_fence_init();
   }
   __syncthreads();
-  if (early_exit) return;
+  if (early_exit || nsel_s == 0) return;
+  if (!kList && !kDense) n_tot = nsel_s * ni;
   if (warp == 0) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
@@ -237,12 +257,13 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       bool ok = true;
       int issued = 0;
-      int hq = hkv * G, i = i0;   // tile n = (query head, query block), kept by increments: no division per tile
+      int hk = 0, i = i0;   // tile n = (hk-th handled query head, query block), kept by increments: no division per tile
       ListIter it;
       if (kList) it.init(lmask, p.wpad, G);
       for (int n = 0; n < n_tot && ok; ++n, ++i) {
-        if (kList) { int hl; it.next(hl, i); hq = hkv * G + hl; }
-        else if (i == T) { i = i0; ++hq; }
+        if (kList) it.next(hk, i);
+        else if (i == T) { i = i0; ++hk; }
+        const int hq = hkv * G + (kList ? hk : hsel[hk]);
         const int s = n & 1;
         ok = mbar_wait(&q_empty[s], ((n >> 1) & 1) ^ 1, status);
         if (!ok) break;
@@ -411,7 +432,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     if (kList) { it.init(lmask, p.wpad, G); have_nx = it.next(h_nx, i_nx); }
     // per-query vectors of tile 0 into slot 0 (published by the first column quarter), then a group sync
     if (qt == 0) {
-      const size_t x = vec_index(kList ? h_nx : 0, kList ? i_nx : i0);
+      const size_t x = vec_index(kList ? h_nx : hsel[0], kList ? i_nx : i0);
       vec[0][0][rl] = p.lse2[x];
       vec[0][1][rl] = p.bq[x];
       vec[0][2][rl] = p.Dq[x];
@@ -422,7 +443,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     ok = __all_sync(0xffffffffu, ok);
 
     // tile n = (query head hq_n of the group, query block i): kept by increments, no division per tile
-    int hq_n = 0, i = i0, slot = 0;
+    int hq_n = 0, i = i0, slot = 0;   // (hq_n: index into the handled heads; list mode: the head itself)
     for (int n = 0; n < n_tot && ok; ++n, ++i, slot = (slot == 2 ? 0 : slot + 1)) {
       if (kList) { hq_n = h_nx; i = i_nx; have_nx = it.next(h_nx, i_nx); }
       else if (i == T) { i = i0; ++hq_n; }
@@ -430,7 +451,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // prefetch the per-query vectors of the next tile
       float nx0 = 0.f, nx1 = 0.f, nx2 = 0.f;
       if (qt == 0 && n + 1 < n_tot) {
-        const size_t x = kList ? vec_index(h_nx, i_nx) : (last_of_head ? vec_index(hq_n + 1, i0) : vec_index(hq_n, i + 1));
+        const size_t x = kList ? vec_index(h_nx, i_nx) : (last_of_head ? vec_index(hsel[hq_n + 1], i0) : vec_index(hsel[hq_n], i + 1));
         nx0 = p.lse2[x]; nx1 = p.bq[x]; nx2 = p.Dq[x];
       }
       ok = mbar_wait(&s_full, n & 1, status);
@@ -495,7 +516,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (stat_thread) {
           ++r_head;
           if (p.bitmask) {
-            uint32_t* bm_row = p.bitmask + ((size_t)(b * p.Hq + hkv * G + hq_n) * p.Tk + j) * p.words;
+            uint32_t* bm_row = p.bitmask + ((size_t)(b * p.Hq + hkv * G + hsel[hq_n]) * p.Tk + j) * p.words;
             if ((i >> 5) != bm_word) {
               if (bm_word >= 0) bm_row[bm_word] = bm_bits;
               bm_word = i >> 5;
@@ -568,7 +589,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         ++r;
       }
       if (stat_thread && last_of_head) {   // last tile of this query head
-        const size_t row = (size_t)(b * p.Hq + hkv * G + hq_n) * p.Tk + j;
+        const size_t row = (size_t)(b * p.Hq + hkv * G + hsel[hq_n]) * p.Tk + j;
         if (p.bitmask && bm_word >= 0) p.bitmask[row * p.words + bm_word] = bm_bits;
         if (p.retained) p.retained[row] = (uint32_t)r_head;
         if (p.totals) {
@@ -611,6 +632,16 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
               w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * f, __uint_as_float(o[8 * v + 3]) * f);
               w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * f, __uint_as_float(o[8 * v + 5]) * f);
               w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * f, __uint_as_float(o[8 * v + 7]) * f);
+              if (!kDense && p.accum_dkv && c * 32 + v * 8 < p.d) {   // add to what the list-mode launch stored for the other heads
+                const uint4 pv = *reinterpret_cast<const uint4*>(out + c * 32 + v * 8);
+                const uint32_t pr[4] = {pv.x, pv.y, pv.z, pv.w};
+                uint32_t nw[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  nw[e] = pack_bf16x2(__uint_as_float(o[8 * v + 2 * e]) * f + __uint_as_float(pr[e] << 16),
+                                      __uint_as_float(o[8 * v + 2 * e + 1]) * f + __uint_as_float(pr[e] & 0xffff0000u));
+                w = make_uint4(nw[0], nw[1], nw[2], nw[3]);
+              }
               if (c * 32 + v * 8 < p.d) *reinterpret_cast<uint4*>(out + c * 32 + v * 8) = w;
             }
           }
@@ -639,7 +670,7 @@ mala_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       if (info < 0) break;
       const int n = info >> 1, ds = info & 1;
       // (the tile's coordinates while the dQ MMAs are still running: the announcement precedes their completion)
-      int hq = hkv * G + n / ni, i = i0 + n % ni;
+      int hq = hkv * G + hsel[n / ni], i = i0 + n % ni;
       if (kList) { int hl; it.next(hl, i); hq = hkv * G + hl; }   // (every tile of the list is announced, in order)
       const int tile = p.cu ? (int)((size_t)hq * (p.Np / 128) + (size_t)(prow0 / 128 + i))
                             : (int)(((size_t)b * p.Hq + hq) * p.T + (size_t)i);
@@ -909,7 +940,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   p.cu = cu; p.cu_k = cu_k; p.d = d;
   if (cu_k) { p.koff = 0; p.qshift = 0; }    // per sequence, on the device
   p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
-  p.list_mask = nullptr; p.wpad = 0;
+  p.list_mask = nullptr; p.wpad = 0; p.sel_rows = nullptr; p.accum_dkv = 0;
   if (p.bitmask &&
       cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hq * Tk * p.words * sizeof(uint32_t), stream) != cudaSuccess)
     return MALA_ERR_CUDA;
@@ -930,7 +961,7 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
   // kernel that tests and works tile by tile.
   const int wpad = bwd_mask_wpad(T);
   const size_t base_bytes = bwd_align256((size_t)Bl * Hq * Np * D * sizeof(float)) + 3 * vbytes;
-  const bool two_pass = !dense && MALA_BWD_TWO_PASS && (Hq / Hkv) * wpad <= kBwdListWords && T <= 32 * ScoutCfg<128>::kMaskWords &&
+  const bool two_pass = !dense && MALA_BWD_TWO_PASS && (Hq / Hkv) * 2 * wpad <= kScoutMaskWords && (Hq / Hkv) <= 16 &&
                         ws_bytes >= base_bytes + bwd_list_bytes(B, Hq, T, Tk);
   int rc;
   if (two_pass) {
@@ -944,13 +975,21 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     sp.B = B; sp.Hq = Hq; sp.Hkv = Hkv; sp.N = N; sp.Np = Np; sp.T = T; sp.words = p.words; sp.wpad = wpad; sp.causal = causal;
     sp.Nk = Nk; sp.Tk = Tk; sp.koff = p.koff; sp.qshift = p.qshift; sp.cu = cu; sp.cu_k = cu_k;
     sp.scale_log2 = p.scale_log2;
+    sp.sample = MALA_BWD_SAMPLE;
     rc = (D == 128) ? bwd_launch_scout<128>(tq, tk, sp, stream) : bwd_launch_scout<64>(tq, tk, sp, stream);
     if (rc != MALA_OK) return rc;
     BwdParams pl = p;
-    pl.retained = nullptr; pl.bitmask = nullptr; pl.totals = nullptr;   // (the first pass wrote the telemetry)
+    pl.retained = nullptr; pl.bitmask = nullptr; pl.totals = nullptr;   // (the first pass wrote the telemetry of these rows)
     pl.list_mask = sp.mask; pl.wpad = wpad;
     rc = (D == 128) ? bwd_launch_main<128, true, true>(tq, tk, tv, tdo, tacc, pl, stream)
                     : bwd_launch_main<64, true, true>(tq, tk, tv, tdo, tacc, pl, stream);
+    if (rc != MALA_OK) return rc;
+    if (sp.sample) {   // the rows the first pass left alone: tested and worked tile by tile, added to the stored dK, dV
+      BwdParams pd = p;
+      pd.sel_rows = sp.row_count; pd.accum_dkv = 1;
+      rc = (D == 128) ? bwd_launch_main<128, false>(tq, tk, tv, tdo, tacc, pd, stream)
+                      : bwd_launch_main<64, false>(tq, tk, tv, tdo, tacc, pd, stream);
+    }
   } else if (D == 128) {
     rc = dense ? bwd_launch_main<128, true>(tq, tk, tv, tdo, tacc, p, stream) : bwd_launch_main<128, false>(tq, tk, tv, tdo, tacc, p, stream);
   } else {

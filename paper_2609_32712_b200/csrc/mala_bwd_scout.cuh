@@ -10,8 +10,14 @@
 // the row's mask, and the row is written out when the head's last tile has been tested.  The second pass
 // (mala_bwd_kernel in its list mode) then visits the retained tiles only and runs the dense tile pipeline on them.
 //
+// Rows that retain everything gain nothing from a first pass (their scores would be formed twice), so the rows of a
+// CTA are sampled first: every eighth tile of every head.  A head whose sampled tiles are all retained, for both key
+// blocks of the pair, is left to the one-pass kernel (mala_bwd_kernel without the list, restricted to such heads), which
+// tests and works tile by tile; only the other heads are tested in full here.
+//
 // Output, per (batch, query head, key block j): the row's mask (bit i set iff tile (j, i) is retained; rows padded to
-// a multiple of four words) and its number of set bits.
+// a multiple of four words) and its number of set bits, or an empty mask and the count kScoutDirectRow for a row that
+// is left to the one-pass kernel.
 //
 // Warp roles (640 threads): warp 0 TMA producer (K_j once, Q ring), warp 1 UMMA issuer, warp 2 per-query test offsets
 // (bq = lse2 + log2(tau / L_q) of the tile's 128 queries into a ring of four shared-memory slots, with the minimum of
@@ -25,6 +31,11 @@
 
 namespace mala {
 
+constexpr uint32_t kScoutDirectRow = 0xffffffffu;   // row_count of a row left to the one-pass kernel
+constexpr int kScoutMaskWords = 4096;               // mask words of one CTA (G heads x 2 key blocks x wpad) in shared memory
+constexpr int kScoutSampleStride = 8;               // every eighth tile of a row is sampled first ...
+constexpr int kScoutSampleMinTiles = 32;            // ... in rows of at least this many tiles
+
 struct ScoutParams {
   const float* bq;            // [B,Hq,Np] lse2 + log2(tau / L_q); +inf on padding rows
   uint32_t* mask;             // [B,Hq,Tk,wpad] (packed sequences: B entries as well)
@@ -37,6 +48,7 @@ struct ScoutParams {
   int Nk, Tk, koff, qshift;
   const int* cu;
   const int* cu_k;
+  int sample;                 // sample the rows first and leave the ones that retain everything to the one-pass kernel
   float scale_log2;
 };
 
@@ -47,8 +59,29 @@ struct ScoutCfg {
   static constexpr int kStages = 4;
   static constexpr int kSmemBytes = (2 + kStages) * kTileBytes + 1024;   // K of two key blocks, Q ring
   static constexpr int kThreads = 640;
-  static constexpr int kMaskWords = 256;     // words of one row's mask held in shared memory (query blocks / 32)
 };
+
+// The tile sequence of a CTA, the same for every role: the sampled tiles of all heads, then -- once the sampled votes
+// have decided which heads are left to the one-pass kernel (`sync` returns after dflag[] has been written) -- the other
+// tiles of the other heads.  body(h, i) handles Q tile i of head h; both return false to stop.
+template <class Body, class Sync>
+__device__ __forceinline__ bool scout_for_each_tile(int G, int i0a, int T, bool sampling, const volatile int* dflag,
+                                                    Body body, Sync sync) {
+  if (sampling) {
+    for (int h = 0; h < G; ++h)
+      for (int i = i0a; i < T; i += kScoutSampleStride)
+        if (!body(h, i)) return false;
+    if (!sync()) return false;
+  }
+  for (int h = 0; h < G; ++h) {
+    if (sampling && dflag[h]) continue;
+    for (int i = i0a; i < T; ++i) {
+      if (sampling && ((i - i0a) % kScoutSampleStride) == 0) continue;
+      if (!body(h, i)) return false;
+    }
+  }
+  return true;
+}
 
 template <int D>
 __global__ void __launch_bounds__(640, 1)
@@ -61,11 +94,11 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint8_t* sK = smem;                          // key blocks ja, jb
   uint8_t* sQ = sK + 2 * Cfg::kTileBytes;      // 4 stages
 
-  __shared__ uint64_t k_full, q_full[4], q_empty[4], s_full[4], s_empty[4], vec_full[4], vec_empty[4], fin_bar;
-  __shared__ __align__(16) float vec[4][128];  // [sub-tile & 3][query column]: bq
-  __shared__ float vmin[4][4];                 // [sub-tile & 3][32-column chunk]: smallest bq of the chunk
-  __shared__ uint32_t rowmask[2][2][Cfg::kMaskWords];   // [head parity][key block of the pair][word]
-  __shared__ uint32_t row_pop[2][2];
+  __shared__ uint64_t k_full, q_full[4], q_empty[4], s_full[4], s_empty[4], vec_full[4], vec_empty[4], fin_bar, phase_bar;
+  __shared__ __align__(16) float vec[4][128];  // [score tile & 3][query column]: bq
+  __shared__ float vmin[4][4];                 // [score tile & 3][32-column chunk]: smallest bq of the chunk
+  __shared__ uint32_t rowmask[kScoutMaskWords];   // [head][key block of the pair][wpad]
+  __shared__ int dflag[16];                    // head is left to the one-pass kernel
   __shared__ uint32_t tmem_base_s;
   __shared__ int early_exit;
 
@@ -89,15 +122,16 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   const int i0a = p.causal ? max(ja - koff, 0) : 0;
   const int i0b = has_b ? (p.causal ? max(jb - koff, 0) : 0) : T;
   const int ni = has_a ? T - i0a : 0;
-  const int n_tot = G * ni;                                                   // Q tiles of this CTA
+  const bool sampling = p.sample && ni >= kScoutSampleMinTiles;
   const size_t out_row0 = ((size_t)b * p.Hq + (size_t)hkv * G) * p.Tk;        // + h * Tk + j
+  const int wpad = p.wpad;
   int* status = p.status;
-  if (n_tot <= 0) {   // key blocks without queries: empty rows
+  if (ni <= 0) {   // key blocks without queries: empty rows
     for (int kb = 0; kb < 2; ++kb) {
       const int j = ja + kb;
       if (j >= p.Tk) continue;
-      for (int x = tid; x < G * p.wpad; x += blockDim.x)
-        p.mask[(out_row0 + (size_t)(x / p.wpad) * p.Tk + j) * p.wpad + x % p.wpad] = 0u;
+      for (int x = tid; x < G * wpad; x += blockDim.x)
+        p.mask[(out_row0 + (size_t)(x / wpad) * p.Tk + j) * wpad + x % wpad] = 0u;
       if (tid < G) {
         p.row_count[out_row0 + (size_t)tid * p.Tk + j] = 0u;
         if (p.tel_retained) p.tel_retained[out_row0 + (size_t)tid * p.Tk + j] = 0u;
@@ -113,11 +147,11 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 4);
       mbar_init(&vec_full[s], 1); mbar_init(&vec_empty[s], 4);
     }
-    mbar_init(&fin_bar, 1);
-    row_pop[0][0] = row_pop[0][1] = row_pop[1][0] = row_pop[1][1] = 0u;
+    mbar_init(&fin_bar, 1); mbar_init(&phase_bar, 1);
     mbar_fence_init();
   }
-  for (int x = tid; x < 4 * Cfg::kMaskWords; x += blockDim.x) rowmask[0][0][x] = 0u;
+  for (int x = tid; x < G * 2 * wpad; x += blockDim.x) rowmask[x] = 0u;
+  if (tid < 16) dflag[tid] = 0;
   __syncthreads();
   if (early_exit) return;
   if (warp == 0) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
@@ -125,6 +159,8 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
+  // (the roles that run ahead of the tests wait here, between the sampled tiles and the others, for the decisions)
+  auto wait_decisions = [&]() -> bool { return mbar_wait(&phase_bar, 0, status); };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -135,17 +171,16 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         tma_load_4d(sK + pn * 16384, &tmK, &k_full, pn * 64, krow0 + ja * 128, hkv, bz);
         if (has_b) tma_load_4d(sK + Cfg::kTileBytes + pn * 16384, &tmK, &k_full, pn * 64, krow0 + jb * 128, hkv, bz);
       }
-      bool ok = true;
-      int hq = hkv * G, i = i0a;
-      for (int n = 0; n < n_tot && ok; ++n) {
+      int n = 0;
+      scout_for_each_tile(G, i0a, T, sampling, dflag, [&](int h, int i) -> bool {
         const int s = n & 3;
-        ok = mbar_wait(&q_empty[s], ((n >> 2) & 1) ^ 1, status);
-        if (!ok) break;
+        if (!mbar_wait(&q_empty[s], ((n >> 2) & 1) ^ 1, status)) return false;
         mbar_arrive_expect_tx(&q_full[s], Cfg::kTileBytes);
         for (int pn = 0; pn < PAN; ++pn)
-          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128 - qshift, hq, bz);
-        if (++i == T) { i = i0a; ++hq; }
-      }
+          tma_load_4d(sQ + s * Cfg::kTileBytes + pn * 16384, &tmQ, &q_full[s], pn * 64, row0 + i * 128 - qshift, hkv * G + h, bz);
+        ++n;
+        return true;
+      }, wait_decisions);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer (warp-uniform issue loop)
@@ -157,17 +192,15 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const uint64_t dKb = make_smem_desc(smem_u32(sK + Cfg::kTileBytes), 16, 1024);
     const uint64_t dQ0 = make_smem_desc(smem_u32(sQ), 16, 1024);
     bool ok = mbar_wait_warp(&k_full, 0, status);
-    int m = 0, i = i0a;
-    for (int n = 0; n < n_tot && ok; ++n) {
+    int n = 0, m = 0;
+    if (ok) scout_for_each_tile(G, i0a, T, sampling, dflag, [&](int h, int i) -> bool {
       const int s = n & 3;
-      ok = mbar_wait_warp(&q_full[s], (n >> 2) & 1, status);
-      if (!ok) break;
+      if (!mbar_wait_warp(&q_full[s], (n >> 2) & 1, status)) return false;
       const uint64_t dQ = desc_advance(dQ0, s * Cfg::kTileBytes);
       const int nsub = (i >= i0b) ? 2 : 1;
-      for (int kb = 0; kb < nsub && ok; ++kb, ++m) {
+      for (int kb = 0; kb < nsub; ++kb, ++m) {
         const int buf = m & 3;
-        ok = mbar_wait_warp(&s_empty[buf], ((m >> 2) & 1) ^ 1, status);   // the buffer's previous tile has been read
-        if (!ok) break;
+        if (!mbar_wait_warp(&s_empty[buf], ((m >> 2) & 1) ^ 1, status)) return false;   // the buffer's previous tile has been read
         tc_fence_after();
         const uint64_t dK = kb ? dKb : dKa;
 #pragma unroll
@@ -178,34 +211,33 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (leader) tc_commit(&s_full[buf]);
       }
       if (leader) tc_commit(&q_empty[s]);
-      if (++i == T) i = i0a;
-    }
+      ++n;
+      return true;
+    }, [&]() -> bool { return mbar_wait_warp(&phase_bar, 0, status); });
     __syncwarp();
     if (leader) tc_commit(&fin_bar);
     mbar_wait_warp(&fin_bar, 0, status);
   } else if (warp == 2) {
     // ------------------------------------------------------------------ test offsets of every score tile's 128 queries
-    bool ok = true;
-    int hq_l = 0, i = i0a, m = 0;
-    for (int n = 0; n < n_tot && ok; ++n) {
-      const size_t x = ((size_t)bz * p.Hq + hkv * G + hq_l) * p.Np + (size_t)prow0 + (size_t)i * 128 + lane * 4;
+    int m = 0;
+    scout_for_each_tile(G, i0a, T, sampling, dflag, [&](int h, int i) -> bool {
+      const size_t x = ((size_t)bz * p.Hq + hkv * G + h) * p.Np + (size_t)prow0 + (size_t)i * 128 + lane * 4;
       const float4 v = *reinterpret_cast<const float4*>(p.bq + x);
       float mn = fminf(fminf(v.x, v.y), fminf(v.z, v.w));
       mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1));
       mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2));
       mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 4));
       const int nsub = (i >= i0b) ? 2 : 1;
-      for (int kb = 0; kb < nsub && ok; ++kb, ++m) {   // (one slot per score tile: both key blocks get their copy)
+      for (int kb = 0; kb < nsub; ++kb, ++m) {   // (one slot per score tile: both key blocks get their copy)
         const int s = m & 3;
-        ok = mbar_wait_warp(&vec_empty[s], ((m >> 2) & 1) ^ 1, status);
-        if (!ok) break;
+        if (!mbar_wait_warp(&vec_empty[s], ((m >> 2) & 1) ^ 1, status)) return false;
         *reinterpret_cast<float4*>(&vec[s][lane * 4]) = v;
         if ((lane & 7) == 0) vmin[s][lane >> 3] = mn;
         __syncwarp();
         if (lane == 0) mbar_arrive(&vec_full[s]);
       }
-      if (++i == T) { i = i0a; ++hq_l; }
-    }
+      return true;
+    }, [&]() -> bool { return mbar_wait_warp(&phase_bar, 0, status); });
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ test groups: group g takes the score tiles m = g mod 4
     const int g = (warp - 4) >> 2;
@@ -213,96 +245,105 @@ mala_bwd_scout_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const int rl = (int)lane_base + lane;
     const float c2 = p.scale_log2;
     const int st = tid - 128;                      // 0 .. 511 among the test threads
-    bool ok = true;
+    bool ok = true;                                // (a warp whose wait failed goes on through the barriers below)
     int use = 0;                                   // score tiles this group has taken (parity of its barriers)
     int m = 0;
-    for (int h = 0; h < G; ++h) {
-      for (int i = i0a; i < T; ++i) {
-        const int nsub = (i >= i0b) ? 2 : 1;
-        for (int kb = 0; kb < nsub; ++kb, ++m) {
-          if ((m & 3) != g || !ok) continue;
-          const int j = ja + kb;
-          const bool valid_key = (j * 128 + rl) < Nkeys;
-          ok = mbar_wait(&s_full[g], use & 1, status);
-          if (ok) ok = mbar_wait(&vec_full[g], use & 1, status);
-          ok = __all_sync(0xffffffffu, ok);
-          ++use;
-          if (!ok) continue;
-          tc_fence_after();
-          const bool diag = p.causal && (i + koff == j);
-          bool vote = false;
+    scout_for_each_tile(G, i0a, T, sampling, dflag, [&](int h, int i) -> bool {
+      const int nsub = (i >= i0b) ? 2 : 1;
+      for (int kb = 0; kb < nsub; ++kb, ++m) {
+        if ((m & 3) != g || !ok) continue;
+        const int j = ja + kb;
+        const bool valid_key = (j * 128 + rl) < Nkeys;
+        ok = mbar_wait(&s_full[g], use & 1, status);
+        if (ok) ok = mbar_wait(&vec_full[g], use & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+        ++use;
+        if (!ok) continue;
+        tc_fence_after();
+        const bool diag = p.causal && (i + koff == j);
+        bool vote = false;
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            uint32_t sc[32];
-            tmem_ld_x32(tmem_addr(tb, lane_base, g * 128 + c * 32), sc);
-            tmem_wait_ld();
-            if (diag) {   // entry (key rl, query col) is legal iff rl <= col
-              const uint32_t ninf = 0xff800000u;
+        for (int c = 0; c < 4; ++c) {
+          uint32_t sc[32];
+          tmem_ld_x32(tmem_addr(tb, lane_base, g * 128 + c * 32), sc);
+          tmem_wait_ld();
+          if (diag) {   // entry (key rl, query col) is legal iff rl <= col
+            const uint32_t ninf = 0xff800000u;
 #pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (c * 32 + e < rl) sc[e] = ninf;
-            }
-            // bound first: max_e (s_e c2 - bq_e) <= (max_e s_e) c2 - min_e bq_e (c2 > 0; fma is monotone in each argument)
-            float m0 = __uint_as_float(sc[0]), m1 = __uint_as_float(sc[1]);
-#pragma unroll
-            for (int e = 0; e < 7; ++e) {
-              m0 = max3(m0, __uint_as_float(sc[2 + 4 * e]), __uint_as_float(sc[3 + 4 * e]));
-              m1 = max3(m1, __uint_as_float(sc[4 + 4 * e]), __uint_as_float(sc[5 + 4 * e]));
-            }
-            const float mx = max3(m0, m1, fmaxf(__uint_as_float(sc[30]), __uint_as_float(sc[31])));
-            const bool cand = valid_key && !(fmaf(mx, c2, -vmin[g][c]) < 0.f);
-            if (__any_sync(0xffffffffu, cand)) {
-              const float4* bb = reinterpret_cast<const float4*>(vec[g]) + c * 8;
-              float c0 = -INFINITY, c1 = -INFINITY;
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const float4 x0 = bb[e];
-                c0 = max3(c0, fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y));
-                c1 = max3(c1, fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w));
-              }
-              vote = vote || (valid_key && !(fmaxf(c0, c1) < 0.f));
-            }
-            // (one retaining entry decides the tile: the other chunks need not be read)
-            if (__any_sync(0xffffffffu, vote)) break;
+            for (int e = 0; e < 32; ++e)
+              if (c * 32 + e < rl) sc[e] = ninf;
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(&s_empty[g]);
-            mbar_arrive(&vec_empty[g]);
+          // bound first: max_e (s_e c2 - bq_e) <= (max_e s_e) c2 - min_e bq_e (c2 > 0; fma is monotone in each argument)
+          float m0 = __uint_as_float(sc[0]), m1 = __uint_as_float(sc[1]);
+#pragma unroll
+          for (int e = 0; e < 7; ++e) {
+            m0 = max3(m0, __uint_as_float(sc[2 + 4 * e]), __uint_as_float(sc[3 + 4 * e]));
+            m1 = max3(m1, __uint_as_float(sc[4 + 4 * e]), __uint_as_float(sc[5 + 4 * e]));
           }
-          if (__any_sync(0xffffffffu, vote) && lane == 0) atomicOr(&rowmask[h & 1][kb][i >> 5], 1u << (i & 31));
+          const float mx = max3(m0, m1, fmaxf(__uint_as_float(sc[30]), __uint_as_float(sc[31])));
+          const bool cand = valid_key && !(fmaf(mx, c2, -vmin[g][c]) < 0.f);
+          if (__any_sync(0xffffffffu, cand)) {
+            const float4* bb = reinterpret_cast<const float4*>(vec[g]) + c * 8;
+            float c0 = -INFINITY, c1 = -INFINITY;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float4 x0 = bb[e];
+              c0 = max3(c0, fmaf(__uint_as_float(sc[4 * e + 0]), c2, -x0.x), fmaf(__uint_as_float(sc[4 * e + 1]), c2, -x0.y));
+              c1 = max3(c1, fmaf(__uint_as_float(sc[4 * e + 2]), c2, -x0.z), fmaf(__uint_as_float(sc[4 * e + 3]), c2, -x0.w));
+            }
+            vote = vote || (valid_key && !(fmaxf(c0, c1) < 0.f));
+          }
+          // (one retaining entry decides the tile: the other chunks need not be read)
+          if (__any_sync(0xffffffffu, vote)) break;
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&s_empty[g]);
+          mbar_arrive(&vec_empty[g]);
+        }
+        if (__any_sync(0xffffffffu, vote) && lane == 0) atomicOr(&rowmask[(h * 2 + kb) * wpad + (i >> 5)], 1u << (i & 31));
       }
-      // the head's rows are complete when all sixteen warps have passed their last tile of it
-      // (a warp whose wait failed keeps taking part in the barriers: the others must not be left waiting at one)
+      return true;
+    }, [&]() -> bool {
+      // all sampled tiles have been tested once the sixteen warps meet here: a head whose samples are all retained,
+      // for both key blocks, is left to the one-pass kernel
       asm volatile("bar.sync 1, 512;" ::: "memory");
-      for (int kb = 0; kb < 2; ++kb) {
-        if (ja + kb >= p.Tk) continue;
-        uint32_t* rm = rowmask[h & 1][kb];
-        const size_t orow = out_row0 + (size_t)h * p.Tk + ja + kb;
-        uint32_t pop = 0;
-        for (int x = st; x < p.wpad; x += 512) {
-          const uint32_t wv = x < Cfg::kMaskWords ? rm[x] : 0u;
-          p.mask[orow * p.wpad + x] = wv;
-          if (p.tel_bitmask && x < p.words) p.tel_bitmask[orow * p.words + x] = wv;
-          pop += __popc(wv);
-          if (x < Cfg::kMaskWords) rm[x] = 0u;      // (next written two heads on, behind another barrier)
-        }
-        for (int sft = 16; sft > 0; sft >>= 1) pop += __shfl_xor_sync(0xffffffffu, pop, sft);
-        if (lane == 0 && pop) atomicAdd(&row_pop[h & 1][kb], pop);
+      if (st < G) {
+        int got = 0;
+        for (int x = 0; x < 2 * wpad; ++x) got += __popc(rowmask[st * 2 * wpad + x]);
+        int want = 0;
+        for (int i = i0a; i < T; i += kScoutSampleStride) want += (i >= i0b) ? 2 : 1;
+        dflag[st] = (got == want);
       }
       asm volatile("bar.sync 1, 512;" ::: "memory");
-      if (st < 2 && ja + st < p.Tk) {
-        const uint32_t cnt = row_pop[h & 1][st];
-        row_pop[h & 1][st] = 0u;
-        const size_t orow = out_row0 + (size_t)h * p.Tk + ja + st;
-        p.row_count[orow] = cnt;
-        if (p.tel_retained) p.tel_retained[orow] = cnt;
-        const int legal = st ? max(T - i0b, 0) : ni;
-        if (p.totals && (st == 0 || has_b)) {
-          atomicAdd(&p.totals[0], (unsigned long long)cnt);
-          atomicAdd(&p.totals[1], (unsigned long long)legal);
+      if (st == 0) mbar_arrive(&phase_bar);
+      return true;
+    });
+    // every tile has been tested once the sixteen warps meet here: the rows go out
+    asm volatile("bar.sync 1, 512;" ::: "memory");
+    for (int r = (st >> 5); r < G * 2; r += 16) {           // one warp per row
+      const int h = r >> 1, kb = r & 1, j = ja + kb;
+      if (j >= p.Tk) continue;
+      const bool direct = sampling && dflag[h] != 0;
+      const size_t orow = out_row0 + (size_t)h * p.Tk + j;
+      uint32_t pop = 0;
+      for (int x = lane; x < wpad; x += 32) {
+        const uint32_t wv = direct ? 0u : rowmask[r * wpad + x];
+        p.mask[orow * wpad + x] = wv;
+        if (!direct && p.tel_bitmask && x < p.words) p.tel_bitmask[orow * p.words + x] = wv;
+        pop += __popc(wv);
+      }
+      for (int sft = 16; sft > 0; sft >>= 1) pop += __shfl_xor_sync(0xffffffffu, pop, sft);
+      if (lane == 0) {
+        p.row_count[orow] = direct ? kScoutDirectRow : pop;
+        const bool present = kb ? has_b : true;
+        if (!direct) {
+          if (p.tel_retained) p.tel_retained[orow] = pop;
+          if (p.totals && present) {
+            atomicAdd(&p.totals[0], (unsigned long long)pop);
+            atomicAdd(&p.totals[1], (unsigned long long)(kb ? max(T - i0b, 0) : ni));
+          }
         }
       }
     }
