@@ -976,7 +976,9 @@ inline int bwd_launch(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin d
     sp.Nk = Nk; sp.Tk = Tk; sp.koff = p.koff; sp.qshift = p.qshift; sp.cu = cu; sp.cu_k = cu_k;
     sp.scale_log2 = p.scale_log2;
     sp.sample = MALA_BWD_SAMPLE;
-    rc = (D == 128) ? bwd_launch_scout<128>(tq, tk, sp, stream) : bwd_launch_scout<64>(tq, tk, sp, stream);
+    CUtensorMap tq2;   // the queries again, in boxes of two tiles
+    if (!make_tensor_map_bnhd(&tq2, q.p, Bl, Nt, Hq, d, q.sb, q.sn, q.sh, 256)) return MALA_ERR_TENSOR_MAP;
+    rc = (D == 128) ? bwd_launch_scout<128>(tq2, tk, sp, stream) : bwd_launch_scout<64>(tq2, tk, sp, stream);
     if (rc != MALA_OK) return rc;
     BwdParams pl = p;
     pl.retained = nullptr; pl.bitmask = nullptr; pl.totals = nullptr;   // (the first pass wrote the telemetry of these rows)
