@@ -432,22 +432,18 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           if (e + 96 > lim) s3[e] = ninf;
         }
       }
-      float mx[8];
+      // row maximum of the 128 scores: four chains of three-input maxima (half the instructions of pairwise maxima)
+      float mx[4];
+      mx[0] = __uint_as_float(s0[0]); mx[1] = __uint_as_float(s1[0]); mx[2] = __uint_as_float(s2[0]); mx[3] = __uint_as_float(s3[0]);
 #pragma unroll
-      for (int q = 0; q < 8; ++q) mx[q] = -INFINITY;
-#pragma unroll
-      for (int e = 0; e < 32; e += 4) {   // eight independent chains
-        mx[0] = fmaxf(mx[0], fmaxf(__uint_as_float(s0[e]), __uint_as_float(s0[e + 1])));
-        mx[1] = fmaxf(mx[1], fmaxf(__uint_as_float(s0[e + 2]), __uint_as_float(s0[e + 3])));
-        mx[2] = fmaxf(mx[2], fmaxf(__uint_as_float(s1[e]), __uint_as_float(s1[e + 1])));
-        mx[3] = fmaxf(mx[3], fmaxf(__uint_as_float(s1[e + 2]), __uint_as_float(s1[e + 3])));
-        mx[4] = fmaxf(mx[4], fmaxf(__uint_as_float(s2[e]), __uint_as_float(s2[e + 1])));
-        mx[5] = fmaxf(mx[5], fmaxf(__uint_as_float(s2[e + 2]), __uint_as_float(s2[e + 3])));
-        mx[6] = fmaxf(mx[6], fmaxf(__uint_as_float(s3[e]), __uint_as_float(s3[e + 1])));
-        mx[7] = fmaxf(mx[7], fmaxf(__uint_as_float(s3[e + 2]), __uint_as_float(s3[e + 3])));
+      for (int e = 1; e < 31; e += 2) {
+        mx[0] = max3(mx[0], __uint_as_float(s0[e]), __uint_as_float(s0[e + 1]));
+        mx[1] = max3(mx[1], __uint_as_float(s1[e]), __uint_as_float(s1[e + 1]));
+        mx[2] = max3(mx[2], __uint_as_float(s2[e]), __uint_as_float(s2[e + 1]));
+        mx[3] = max3(mx[3], __uint_as_float(s3[e]), __uint_as_float(s3[e + 1]));
       }
       // row maximum of the scaled scores, log2 domain
-      const float mt = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * c2;
+      const float mt = fmaxf(max3(mx[0], mx[1], __uint_as_float(s0[31])), max3(mx[2], mx[3], fmaxf(fmaxf(__uint_as_float(s1[31]), __uint_as_float(s2[31])), __uint_as_float(s3[31])))) * c2;
       bool retain = true;
       if (!kDense) {
         // Eq. 3: skip iff rowmax - (m + log l) < log(tau / L) for every valid row
