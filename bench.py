@@ -11,7 +11,7 @@ MALA and dense kernels on cfg3 / cfg4 (literal and paper-regime "R" inputs), dec
 figures (retained slots, omitted mass, relative L2 against the dense path) at tau = 1e-4, 1e-2 and 1.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-  python bench.py --only fwd|bwd|decode --workload cfg2 --preset R --tau 1e-4 --iters 3
+  python bench.py --only fwd|bwd|decode|decode8 --workload cfg2 --preset R --tau 1e-4 --iters 3
       (a few launches of one operator and nothing else: the small fixed command profiler captures are taken on)
   python bench.py --workload tp8 [--preset S --tau 1] (under torchrun --nproc-per-node 8: one tensor-parallel rank's
       head slice of the paper's 128K operator benchmark per GPU, timed as the synchronized wall clock of the group)
@@ -540,11 +540,17 @@ def run_only(args, dev):
     import dataclasses
     import torch
     from paper_2609_32712_b200 import mala, workloads as W
-    if args.only == "decode":
+    if args.only in ("decode", "decode8"):
         cfg = dataclasses.replace(W.decode_config("cfg5"), B=args.decode_batch)
         w = W.make_decode(cfg, preset=args.preset if args.preset in ("literal", "D") else "literal", device=dev)
+        if args.only == "decode8":
+            k8, ks8, _ = W.quantize_cache_e4m3(w["kcache"])
+            v8, vs8, _ = W.quantize_cache_e4m3(w["vcache"])
         for _ in range(args.iters):
-            mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], args.tau, cfg.num_splits)
+            if args.only == "decode8":
+                mala.decode_fp8(w["q"], k8, v8, ks8, vs8, w["scale"], args.tau, cfg.num_splits)
+            else:
+                mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], args.tau, cfg.num_splits)
     else:
         cfg = W.prefill_config(args.workload)
         w = W.make_prefill(cfg, preset=args.preset, device=dev)
@@ -567,7 +573,7 @@ def main():
     ap.add_argument("--impl", default="mala", choices=["mala", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "tp8"])
     ap.add_argument("--preset", default="literal", choices=["literal", "R", "S", "D"])
-    ap.add_argument("--only", default=None, choices=["fwd", "bwd", "decode"],
+    ap.add_argument("--only", default=None, choices=["fwd", "bwd", "decode", "decode8"],
                     help="run a few launches of one operator on --workload / --preset / --tau and exit (no timing table, "
                          "no CPU leg): the command that profiler captures are taken on")
     ap.add_argument("--iters", type=int, default=3, help="launches of --only")
@@ -855,6 +861,25 @@ def main():
                               "achieved_gbs": need / (us * 1e-6) / 1e9,
                               "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
             row["speedup"] = row["dense"]["us"] / row["mala"]["us"]
+            # the same cache stored as e4m3 with one scale per 128-key tile (mala_decode_fp8): half the bytes
+            k8, ks8, _ = W.quantize_cache_e4m3(kc)
+            v8, vs8, _ = W.quantize_cache_e4m3(vc)
+            f8 = {}
+            for label, t_ in (("mala", tau), ("dense", 0.0)):
+                us = 1e3 * time_cuda(lambda: mala.decode_fp8(qd, k8, v8, ks8, vs8, wd["scale"], t_, dcfg.num_splits, ws=wsd,
+                                                              out=od, want_lse=False), 25, 100)
+                o8, _, st = mala.decode_fp8(qd, k8, v8, ks8, vs8, wd["scale"], t_, dcfg.num_splits, ws=wsd, stats=True)
+                torch.cuda.synchronize()
+                ret, leg = st.totals.cpu().tolist()
+                need = (leg + ret) * TILE * dcfg.d              # one byte per element
+                o16, _, _ = mala.decode(qd, kc, vc, wd["scale"], t_, dcfg.num_splits)
+                f8[label] = {"us": us, "retained_frac": ret / leg, "needed_gb": need / 1e9,
+                             "achieved_gbs": need / (us * 1e-6) / 1e9,
+                             "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                             "speedup_vs_bf16_cache": row[label]["us"] / us,
+                             "rel_l2_o_vs_bf16_cache": float((o8.float() - o16.float()).norm() / o16.float().norm())}
+            row["e4m3_cache"] = f8
+            del k8, v8, ks8, vs8
             if preset == "D":                       # work and fidelity against the dense decode, tau up to 1
                 o0, lse0, _ = mala.decode(qd, kc, vc, wd["scale"], 0.0, dcfg.num_splits, ws=wsd)
                 o0, fid = o0.float(), {}

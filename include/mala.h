@@ -188,6 +188,19 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
                 int B, int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws,
                 size_t ws_bytes, void* cuda_stream);
 
+/* mala_decode over an 8-bit KV cache: the same operator ("Fused decoding execution"; the paper keeps the cache intact,
+ * and so does this call -- only the storage type differs) on keys and values stored as e4m3 with one fp32 scale per
+ * (sequence, KV head, 128-key tile):
+ *     k[b, n, h, :] = kscale[b, h, n / 128] * e4m3(kcache8[b, n, h, :]),   v likewise with vscale.
+ * The result is that of mala_decode on those dequantised values (the step streams half the bytes).
+ * kcache8, vcache8: 8-bit [B,Nk,Hkv,d] views, strides in ELEMENTS (= bytes), multiples of 16; kscale, vscale: device
+ * fp32 [B,Hkv,ceil(Nk/128)].  d a multiple of 16, at most 128; Hq/Hkv <= 4 (MALA_ERR_UNSUPPORTED otherwise).  q, o,
+ * lse_opt, telemetry, splits and merge as in mala_decode.
+ * Workspace: mala_workspace_bytes(MALA_OP_DECODE, B, Hq, Hkv, Nk, 128, num_splits). */
+int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float* kscale, const float* vscale,
+                    mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
+                    float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Split-KV decode of Sq new tokens per sequence at once (a verification step of speculative decoding, or a short
  * chunk).  q, o [B,Sq,Hq,d]; lse_opt fp32 [B,Sq,Hq] or NULL; kcache, vcache [B,Nk,Hkv,d] with the keys and values of
  * the Sq new tokens already in the last Sq positions.  Token s (0 = oldest) sits at position Nk - Sq + s, attends to

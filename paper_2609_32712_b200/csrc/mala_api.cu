@@ -211,6 +211,12 @@ int mala_device_status(int* code_out, int clear) {
   return MALA_OK;
 }
 
+#ifdef MALA_F8_TRACE
+int mala_f8_trace(long long* out) {
+  return cudaMemcpyFromSymbol(out, mala::f8_trace, sizeof(long long) * 64 * 16) == cudaSuccess ? 0 : -1;
+}
+#endif
+
 int mala_test_expire_wait(long long limit_cycles, void* cuda_stream) {
   if (limit_cycles <= 0 || limit_cycles > 100000000LL) return MALA_ERR_INVALID_ARG;
   int dev = 0;
@@ -479,6 +485,34 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
   MALA_TRY(device_setup(dev, &status));
   return decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
                        (cudaStream_t)cuda_stream);
+}
+
+int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float* kscale, const float* vscale,
+                    mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
+                    float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  if (num_splits <= 0 || !ws || !kscale || !vscale) return MALA_ERR_INVALID_ARG;
+  if (Hq / Hkv > 4 || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
+  // 8-bit views: strides in elements = bytes, multiples of 16
+  auto check8 = [&](const mala_tin& t) -> int {
+    if (!t.p) return MALA_ERR_INVALID_ARG;
+    if (!aligned16(t.p)) return MALA_ERR_MISALIGNED;
+    if ((B > 1 && t.sb % 16) || (Nk > 1 && t.sn % 16) || (Hkv > 1 && t.sh % 16)) return MALA_ERR_MISALIGNED;
+    if ((B > 1 && t.sb <= 0) || (Nk > 1 && t.sn <= 0) || (Hkv > 1 && t.sh <= 0)) return MALA_ERR_INVALID_ARG;
+    return MALA_OK;
+  };
+  MALA_TRY(check8(kcache8));
+  MALA_TRY(check8(vcache8));
+  MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
+  if ((((uintptr_t)ws) & 255) != 0 || (((uintptr_t)kscale) & 3) != 0 || (((uintptr_t)vscale) & 3) != 0) return MALA_ERR_MISALIGNED;
+  if (ws_bytes < decode_workspace_bytes(B, Hq, 128, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  return decode_fp8_launch(q, kcache8, vcache8, kscale, vscale, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits,
+                           ws, status, (cudaStream_t)cuda_stream);
 }
 
 int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,

@@ -6,6 +6,7 @@
 
 #include "../../include/mala.h"
 #include "mala_decode_split.cuh"
+#include "mala_decode_fp8.cuh"
 #include "tensor_map.h"
 
 namespace mala {
@@ -48,6 +49,10 @@ inline bool decode_set_attributes() {
   ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
 #define MALA_DEC_ATTR_GP(GP) MALA_DEC_ATTR(false, GP, false) MALA_DEC_ATTR(true, GP, false) MALA_DEC_ATTR(false, GP, true) MALA_DEC_ATTR(true, GP, true)
   MALA_DEC_ATTR_GP(1) MALA_DEC_ATTR_GP(2) MALA_DEC_ATTR_GP(4) MALA_DEC_ATTR_GP(8) MALA_DEC_ATTR_GP(16)
+#define MALA_F8_ATTR(DENSE, GP) \
+  ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg::kSmemBytes) == cudaSuccess;
+  MALA_F8_ATTR(false, 1) MALA_F8_ATTR(true, 1) MALA_F8_ATTR(false, 2) MALA_F8_ATTR(true, 2) MALA_F8_ATTR(false, 4) MALA_F8_ATTR(true, 4)
+#undef MALA_F8_ATTR
 #undef MALA_DEC_ATTR_GP
 #undef MALA_DEC_ATTR
   return ok;
@@ -147,6 +152,54 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   else
     decode_merge_kernel<64><<<B * Sq * Hq, 64, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
                                                             Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits, d);
+  return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
+}
+
+// Decode over an e4m3 cache with one fp32 scale per (sequence, KV head, 128-key tile): kc / vc are 8-bit [B,Nk,Hkv,d]
+// views (strides in elements), kscale / vscale fp32 [B,Hkv,ceil(Nk/128)].  Up to four query heads per KV head.
+inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* kscale, const float* vscale, mala_tout o,
+                             float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
+                             float tau, int num_splits, void* ws, int* status, cudaStream_t stream) {
+  const int G = Hq / Hkv;
+  if (G > 4 || d % 16 != 0 || d > 128 || d < 16) return MALA_ERR_UNSUPPORTED;
+  const int per = (Nk + num_splits - 1) / num_splits;
+  const int tps = (per + 127) / 128;
+  if ((long long)B * Hkv * num_splits > 0x7fffffffLL || (long long)B * Hkv * ((Nk + 127) / 128) > 0x7fffffffLL)
+    return MALA_ERR_UNSUPPORTED;
+  CUtensorMap tq, tk, tv;
+  if (!make_tensor_map_q_rows(&tq, q.p, B, 1, Hq, d, q.sb, 0, q.sh, G) ||
+      !make_tensor_map_u8_bnhd(&tk, kc.p, B, Nk, Hkv, d, kc.sb, kc.sn, kc.sh) ||
+      !make_tensor_map_u8_bnhd(&tv, vc.p, B, Nk, Hkv, d, vc.sb, vc.sn, vc.sh))
+    return MALA_ERR_TENSOR_MAP;
+  DecF8Params p;
+  p.o_part = (float*)ws;
+  p.lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Hq * num_splits * 128 * sizeof(float)));
+  p.retained = st ? st->retained_per_block : nullptr;
+  p.bitmask = st ? st->tile_bitmask : nullptr;
+  p.totals = st ? (unsigned long long*)st->totals : nullptr;
+  p.status = status;
+  p.kscale = kscale; p.vscale = vscale;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Nk = Nk; p.tps = tps; p.num_splits = num_splits; p.words = (tps + 31) / 32;
+  p.n_items = B * Hkv * num_splits; p.nt = (Nk + 127) / 128;
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
+  if (p.bitmask &&
+      cudaMemsetAsync(p.bitmask, 0, (size_t)B * Hkv * num_splits * p.words * sizeof(uint32_t), stream) != cudaSuccess)
+    return MALA_ERR_CUDA;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return MALA_ERR_CUDA;
+  const int grid = p.n_items < sms ? p.n_items : sms;
+#define MALA_F8_LAUNCH(DENSE, GP) mala_decode_fp8_kernel<DENSE, GP><<<grid, DecF8Cfg::kThreads, DecF8Cfg::kSmemBytes, stream>>>(tq, tk, tv, p)
+  const bool dense = (tau == 0.f);
+  if (G <= 1) { if (dense) MALA_F8_LAUNCH(true, 1); else MALA_F8_LAUNCH(false, 1); }
+  else if (G <= 2) { if (dense) MALA_F8_LAUNCH(true, 2); else MALA_F8_LAUNCH(false, 2); }
+  else { if (dense) MALA_F8_LAUNCH(true, 4); else MALA_F8_LAUNCH(false, 4); }
+#undef MALA_F8_LAUNCH
+  if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
+  decode_merge_kernel<128><<<B * Hq, 128, 0, stream>>>(p.o_part, p.lse_part, (__nv_bfloat16*)o.p, o.sb, 0, o.sh, lse_opt, 1,
+                                                      Hq, num_splits, d);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 

@@ -50,6 +50,23 @@ inline bool make_tensor_map_bnhd(CUtensorMap* out, const void* base, int B, int 
   return r == CUDA_SUCCESS;
 }
 
+// Tensor map over an 8-bit [B, N, H, d] view (strides in elements = bytes): coordinates (c, n, h, b), box = 128 columns
+// x 128 rows (one 16 KB tile), 128-byte swizzle; columns beyond d and rows beyond N read as zero.
+inline bool make_tensor_map_u8_bnhd(CUtensorMap* out, const void* base, int B, int N, int H, int d, int64_t sb,
+                                    int64_t sn, int64_t sh) {
+  PFN_tensorMapEncodeTiled enc = tensor_map_encoder();
+  if (!enc) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+  auto legal = [&](int64_t s, int n) -> cuuint64_t { return (n == 1 || s <= 0) ? (cuuint64_t)((d + 15) / 16 * 16) : (cuuint64_t)s; };
+  cuuint64_t strides[3] = {legal(sn, N), legal(sh, H), legal(sb, B)};
+  cuuint32_t box[4] = {128u, 128u, 1u, 1u};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Tensor map over the bf16 queries of a decode step, [B, S, H, d]: coordinates (c, h, s, b), box = 64 columns x G
 // heads x S tokens, which lands in shared memory as S * G consecutive 128-byte rows (row s * G + g), 128-byte swizzle.
 inline bool make_tensor_map_q_rows(CUtensorMap* out, const void* base, int B, int S, int H, int d, int64_t sb,

@@ -80,6 +80,9 @@ def lib():
         L.mala_decode_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, i, i,
                                         f, f, i, vp, sz, vp]
         L.mala_decode_paged.restype = i
+        L.mala_decode_fp8.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp,
+                                      sz, vp]
+        L.mala_decode_fp8.restype = i
         L.mala_decode_static.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, i, i, i, i, i, f, f, i, vp]
         L.mala_decode_static.restype = i
         L.mala_test_expire_wait.argtypes = [ctypes.c_longlong, vp]
@@ -372,6 +375,35 @@ def decode(q, kcache, vcache, scale: float, tau: float, num_splits: int, stats: 
                            B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_decode")
+    return o, lse, st
+
+
+def _view8(t: torch.Tensor):
+    assert t.dtype in (torch.uint8, torch.float8_e4m3fn) and t.dim() == 4 and t.stride(3) == 1, \
+        "expects 8-bit [B,N,H,d], last dim contiguous"
+    return _TIn(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def decode_fp8(q, kcache8, vcache8, kscale, vscale, scale: float, tau: float, num_splits: int, stats: bool = False,
+               ws=None, out=None, want_lse: bool = True):
+    """mala_decode_fp8: q [B,1,Hq,d] bf16; kcache8, vcache8 e4m3 codes [B,Nk,Hkv,d] (uint8 or float8_e4m3fn);
+    kscale, vscale fp32 [B,Hkv,ceil(Nk/128)].  Returns (o [B,1,Hq,d] bf16, lse [B,Hq] fp32 or None, Stats or None)."""
+    B, one, Hq, d = q.shape
+    assert one == 1
+    Nk, Hkv = kcache8.shape[1], kcache8.shape[2]
+    assert kscale.dtype == torch.float32 and kscale.is_contiguous() and tuple(kscale.shape) == (B, Hkv, -(-Nk // 128))
+    assert vscale.dtype == torch.float32 and vscale.is_contiguous() and tuple(vscale.shape) == (B, Hkv, -(-Nk // 128))
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    tps = -(-(-(-Nk // num_splits)) // 128)
+    st = Stats((B, Hkv, num_splits), -(-tps // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_DECODE, B, Hq, Hkv, Nk, 128, num_splits), q.device) if ws is None else ws
+    rc = lib().mala_decode_fp8(_view(q, _TIn), _view8(kcache8), _view8(vcache8), kscale.data_ptr(), vscale.data_ptr(),
+                               _view(o, _TOut), lse.data_ptr() if lse is not None else None,
+                               ctypes.byref(st.c) if st else None, B, Hq, Hkv, Nk, d, scale, tau, num_splits,
+                               ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_decode_fp8")
     return o, lse, st
 
 

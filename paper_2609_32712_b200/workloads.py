@@ -297,3 +297,21 @@ def custom_decode(B, Hq, Hkv, Nk, d, num_splits, group_types=None, seed=0, prese
     cfg = DecodeConfig(f"custom_dec_B{B}_H{Hq}_{Hkv}_N{Nk}_d{d}", B, Hq, Hkv, Nk, d, num_splits, list(group_types),
                        seed=seed)
     return make_decode(cfg, preset=preset, device=device)
+
+
+def quantize_cache_e4m3(x: torch.Tensor, tile: int = 128):
+    """8-bit storage of a KV cache [B, Nk, Hkv, d]: e4m3 values with one fp32 scale per (sequence, KV head, tile of
+    128 keys), scale = largest magnitude of the tile / 448 (the largest e4m3 value).  Returns (codes uint8
+    [B,Nk,Hkv,d], scales fp32 [B,Hkv,ceil(Nk/tile)], dequantised fp32 [B,Nk,Hkv,d] = scale * e4m3(code), the values an
+    8-bit decode call works on and its oracle is given)."""
+    B, Nk, Hkv, d = x.shape
+    nt = -(-Nk // tile)
+    xf = torch.zeros((B, nt * tile, Hkv, d), dtype=torch.float32, device=x.device)
+    xf[:, :Nk] = x.float()
+    t = xf.view(B, nt, tile, Hkv, d)
+    amax = t.abs().amax(dim=(2, 4))                                   # [B, nt, Hkv]
+    scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+    codes = (t / scale[:, :, None, :, None]).clamp(-448.0, 448.0).to(torch.float8_e4m3fn)
+    deq = (codes.float() * scale[:, :, None, :, None]).view(B, nt * tile, Hkv, d)[:, :Nk].contiguous()
+    codes = codes.view(B, nt * tile, Hkv, d)[:, :Nk].contiguous().view(torch.uint8)
+    return codes, scale.permute(0, 2, 1).contiguous(), deq

@@ -294,3 +294,59 @@ def test_decode_head_size_64_gated_paged_several_tokens(mala, oracle, tau):
     assert res["skipped"] > 0, "workload must exercise skipping"
     _run_paged(mala, oracle, w, tau, 8, 256, [8192, 4096 + 77], seed=9)
     assert _run_multi(mala, oracle, w, 3, tau, 8) > 0
+
+
+def _run_fp8(mala, oracle, w, tau, num_splits):
+    """mala_decode_fp8 on the e4m3 codes of a cache against the oracle on the dequantised values (the oracle has no
+    8-bit arithmetic of its own: it is handed scale * e4m3(code) as fp32)."""
+    k8, ks, kd = W.quantize_cache_e4m3(w["kcache"])
+    v8, vs, vd = W.quantize_cache_e4m3(w["vcache"])
+    q = w["q"].cuda()
+    B, _, Hq, d = q.shape
+    Nk, Hkv = k8.shape[1], k8.shape[2]
+    G = Hq // Hkv
+    o, lse, st = mala.decode_fp8(q, k8.cuda(), v8.cuda(), ks.cuda(), vs.cuda(), w["scale"], tau, num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    ref = oracle.decode(w["q"], kd, vd, w["scale"], tau, num_splits, 128)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy()[:, 0], lse.cpu().numpy()
+    skipped = retained = 0
+    for b in range(B):
+        for g in range(Hkv):
+            for s in range(num_splits):
+                parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                                  tau, Nk, 128)
+                assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
+            hs = slice(g * G, (g + 1) * G)
+            parity.check_output(o_c[b, hs], ref["o"][b, hs])
+            assert np.abs(lse_c[b, hs] - ref["lse"][b, hs]).max() <= parity.LSE_ABS
+            skipped += int((ref["mask"][b, g] == 1).sum())
+            retained += int((ref["mask"][b, g] == 2).sum())
+    return dict(skipped=skipped, retained=retained, totals=st.totals.cpu().numpy())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv,d", [(128, 1, 4, 1, 128), (1024, 4, 8, 2, 128), (1000, 3, 4, 4, 128), (4096, 8, 2, 1, 128),
+                                            (700, 8, 2, 1, 64), (2100, 5, 6, 2, 96), (8192, 64, 8, 2, 128)])
+def test_decode_fp8_cache_literal(mala, oracle, Nk, S, Hq, Hkv, d, tau):
+    w = W.custom_decode(2, Hq, Hkv, Nk, d, S, seed=Nk + S)
+    _run_fp8(mala, oracle, w, tau, S)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("Nk,S", [(8192, 8), (5000, 4)])
+def test_decode_fp8_cache_skips_value_tiles(mala, oracle, Nk, S, tau):
+    w = W.custom_decode(2, 8, 2, Nk, 128, S, group_types=["diffuse", "peaked"], seed=3, preset="D")
+    res = _run_fp8(mala, oracle, w, tau, S)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+    assert res["totals"][1] == res["retained"] + res["skipped"]
+
+
+def test_decode_fp8_refuses_what_it_does_not_support(mala):
+    w = W.custom_decode(1, 8, 1, 256, 128, 1, seed=1)
+    k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
+    with pytest.raises(mala.MalaError) as e:     # eight query heads per KV head
+        mala.decode_fp8(w["q"].cuda(), k8.cuda(), k8.cuda(), ks.cuda(), ks.cuda(), w["scale"], 0.0, 1)
+    assert e.value.code == -2
