@@ -212,6 +212,9 @@ int mala_device_status(int* code_out, int clear) {
 }
 
 #ifdef MALA_F8_TRACE
+int mala_f8_fail(int* out) {
+  return cudaMemcpyFromSymbol(out, mala::f8_fail, sizeof(int) * 24) == cudaSuccess ? 0 : -1;
+}
 int mala_f8_trace(long long* out) {
   return cudaMemcpyFromSymbol(out, mala::f8_trace, sizeof(long long) * 64 * 16) == cudaSuccess ? 0 : -1;
 }
