@@ -211,15 +211,6 @@ int mala_device_status(int* code_out, int clear) {
   return MALA_OK;
 }
 
-#ifdef MALA_F8_TRACE
-int mala_f8_fail(int* out) {
-  return cudaMemcpyFromSymbol(out, mala::f8_fail, sizeof(int) * 24) == cudaSuccess ? 0 : -1;
-}
-int mala_f8_trace(long long* out) {
-  return cudaMemcpyFromSymbol(out, mala::f8_trace, sizeof(long long) * 64 * 16) == cudaSuccess ? 0 : -1;
-}
-#endif
-
 int mala_test_expire_wait(long long limit_cycles, void* cuda_stream) {
   if (limit_cycles <= 0 || limit_cycles > 100000000LL) return MALA_ERR_INVALID_ARG;
   int dev = 0;

@@ -26,15 +26,19 @@
 //
 // At one byte per element a tile arrives twice as fast as in the bf16 kernels, faster than one softmax group can
 // take tiles one after the other (its per-tile chain of TMEM load, two cross-warp reductions, exponentials and the
-// P^T store is latency, not throughput).  Two softmax groups therefore take alternate tiles of a work item, each with
-// its own references, normalizer, P^T slots and O^T accumulator (two online-softmax streams, merged when the item is
-// written out).  Everything a tile needs is computed without the item's state -- its row maxima, its probabilities
-// against the group's own references, their sums -- except the skip test of Eq. 3, which needs the normalizer after
-// the tile before it.  That test, the update of the normalizer and the vote are a short section the groups pass
-// through in tile order (a ring of "turn" barriers); in it a group combines its own (m, l) with the other group's
-// published pair.  The probabilities of a tile that turns out to be skipped were computed for nothing (a few
-// exponentials per thread); its P^T slot is simply reused.  A tile that needs a reference raised takes the slow
-// order instead (decision first, then the rescaling, then the probabilities).
+// P^T store is latency, not throughput).  Two softmax groups therefore take alternate tiles (by the CTA's running tile
+// count, so that a group's consecutive tiles are never further apart than the rings of four are deep), each with its
+// own references, normalizer, P^T slots and O^T accumulator: two online-softmax streams per work item, merged when
+// the item is written out.  Everything a tile needs is computed without the item's state -- its row maxima, its
+// probabilities against the group's own references, their sums -- except the skip test of Eq. 3, which needs the
+// normalizer after the tile before it.  That test is the "turn" of a tile, and turns are taken in tile order (a ring
+// of barriers): one thread of the group waits for the turn before, combines its stream's log-sum-exp with the other
+// group's published one (all that the test needs), decides, publishes and hands the turn on -- a few dozen
+// instructions of one thread -- and the rest of the group picks the decision up behind it.  The probabilities of a
+// tile that turns out to be skipped were computed for nothing (a few exponentials per thread); its P^T slot is
+// simply reused.  A tile that needs a reference raised takes the slow order instead (decision first, then the
+// rescaling, then the probabilities, the turn held meanwhile).  The dense kernel (tau = 0) has no decision to take
+// and its groups run unordered.
 //
 // Every warp that issues asynchronous work walks the CTA's tiles in order and blocks on exactly what its next
 // instruction needs (a warp that polls the barriers of several jobs in one loop, sleeping in between, reacts to each
@@ -43,8 +47,10 @@
 //   warp 1       converts an item's queries, issues S^T of every tile
 //   warp 2       MALA kernel: takes the votes in tile order, requests the raw V copy of a retained tile
 //   warp 3       issues O^T += V8^T P8^T of every retained tile
-//   warps 4-7    softmax group A: even tiles of an item (thread = key of the tile); writes the item's partial output
-//   warps 8-11   softmax group B: odd tiles
+//   warps 4-7    softmax group 0 (thread = key of the tile), up to four packed query heads
+//   warps 8-11   softmax group 1
+//   warps 12-15  epilogue group (thread = output channel): merges the streams of a finished item, writes its partial
+//                output and log-sum-exp, hands the item's state slot and accumulators back
 #pragma once
 #include <cuda_fp16.h>
 
@@ -52,32 +58,6 @@
 #include "sm100_ptx.cuh"
 
 namespace mala {
-
-#if defined(MALA_F8_TRACE) && !defined(MALA_F8_NOTR)
-__device__ long long f8_trace[64 * 16];
-#define F8TR(slot, g) do { if (blockIdx.x == 0 && (g) >= 64 && (g) < 128 && (threadIdx.x & 31) == 0) f8_trace[((g) - 64) * 16 + (slot)] = clock64(); } while (0)
-#else
-#ifdef MALA_F8_TRACE
-__device__ long long f8_trace[64 * 16];
-#endif
-#define F8TR(slot, g) do {} while (0)
-#endif
-
-#ifdef MALA_F8_TRACE
-__device__ int f8_fail[24];
-__device__ __forceinline__ bool f8_note(bool ok, int line) {
-  if (!ok) {
-    atomicCAS(&f8_fail[0], 0, (int)blockIdx.x + 1);
-    if (*(volatile int*)&f8_fail[0] == (int)blockIdx.x + 1) atomicCAS(&f8_fail[4 + (threadIdx.x >> 5)], 0, line);
-  }
-  return ok;
-}
-#define MWAIT(line, ...) f8_note(mbar_wait(__VA_ARGS__), line)
-#define MWAITW(line, ...) f8_note(mbar_wait_warp(__VA_ARGS__), line)
-#else
-#define MWAIT(line, ...) mbar_wait(__VA_ARGS__)
-#define MWAITW(line, ...) mbar_wait_warp(__VA_ARGS__)
-#endif
 
 struct DecF8Params {
   float* o_part;                 // [B, Hq, num_splits, 128] fp32, normalised per split
@@ -103,7 +83,8 @@ struct DecF8Cfg {
   static constexpr int kQ8Bytes = 2048;                  // 16 rows x 128 e4m3
   static constexpr int kP8Bytes = 2048;                  // 16 rows x 128 e4m3
   static constexpr int kGroups = MALA_F8_GROUPS;         // softmax groups: group n takes tiles n, n + kGroups, .. of an item
-  static constexpr int kPSlots = 2 * kGroups;
+  static constexpr int kPPerGroup = 4;                   // P8^T slots of a group: how far it may run ahead of its PVs
+  static constexpr int kPSlots = kPPerGroup * kGroups;
   static constexpr int kSmemBytes = 2 * kStages * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPSlots * kP8Bytes + 1024;
   static constexpr int kThreads = 128 * (2 + kGroups);   // issuing warps, softmax groups, epilogue group
   static constexpr uint32_t kColO = 64;                  // S^T ring 4 x 16, then O^T 2 x kGroups x 16 (item parity, group)
@@ -143,7 +124,7 @@ __global__ void __launch_bounds__(DecF8Cfg::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
   using Cfg = DecF8Cfg;
-  constexpr int RB = Cfg::kRawBytes, NS = Cfg::kStages, NG = Cfg::kGroups;
+  constexpr int RB = Cfg::kRawBytes, NS = Cfg::kStages, NG = Cfg::kGroups, PP = Cfg::kPPerGroup;
   constexpr int GH = GP;                   // rows of a softmax group
   constexpr int LDN = 16;
   constexpr float kPScale = 64.f;          // P' of the key that sets the reference
@@ -155,17 +136,18 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint8_t* sVr = sKr + NS * RB;            // [6] raw V
   uint8_t* sQ = sVr + NS * RB;             // [2] item parity, bf16 as copied
   uint8_t* sQ8 = sQ + 2 * Cfg::kQBytes;    // [2] item parity: rows h = q1, 4 + h = q2, rest zero
-  uint8_t* sP = sQ8 + 2 * Cfg::kQ8Bytes;   // [2 NG] P8^T slots (2 group + n & 1): rows h = p1, 4 + h = p2, rest zero
+  uint8_t* sP = sQ8 + 2 * Cfg::kQ8Bytes;   // [4 NG] P8^T slots (4 group + n % 4): rows h = p1, 4 + h = p2, rest zero
 
   __shared__ uint64_t qr_full[2], q_empty[2], kr_full[NS], kr_empty[NS], v_full[NS], v_empty[NS], s_full[4], s_free[4],
-      vote_bar[4], vote_read[4], turn_done[4], p_full[2 * NG], p_free[2 * NG], item_done[2], o_free[2], fin_bar,
-      grp_bar[NG], ret_full[8], ret_free[8];
+      vote_bar[4], vote_read[4], turn_done[4], p_full[PP * NG], p_free[PP * NG], item_done[2], o_free[2], fin_bar,
+      grp_bar[NG], dec_bar[NG], ret_full[8], ret_free[8];
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[4];
   __shared__ int ret_ring[8];              // decision of tile g at g & 7 (vote warp -> PV warp)
   __shared__ float q_inv[8][4];            // 2^-k of the rows of non-empty item number n, at n & 7
   __shared__ __align__(16) float xch[NG][2][4][8];         // [group][buffer][warp][row]
   __shared__ __align__(16) float st_m[2][NG][4], st_l[2][NG][4], st_y[2][NG][4];   // [item parity][group][row]: (m, l, yref)
+  __shared__ __align__(16) float st_a[2][NG][4];           // ... and m + log2 l, all that the other groups' turns need
   __shared__ int st_r[2][NG];                              // ... and retained tiles of the group in the item
   __shared__ int early_exit;
 
@@ -182,18 +164,22 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     for (int s = 0; s < 2; ++s) {
       mbar_init(&qr_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&item_done[s], 1); mbar_init(&o_free[s], 4);
     }
-    for (int s = 0; s < NG; ++s) mbar_init(&grp_bar[s], 4);
-    for (int s = 0; s < 2 * NG; ++s) { mbar_init(&p_full[s], 4); mbar_init(&p_free[s], 1); }
+    for (int s = 0; s < NG; ++s) { mbar_init(&grp_bar[s], 4); mbar_init(&dec_bar[s], 1); }
+    for (int s = 0; s < PP * NG; ++s) { mbar_init(&p_full[s], 4); mbar_init(&p_free[s], 1); }
     for (int s = 0; s < NS; ++s) {
       mbar_init(&kr_full[s], 1); mbar_init(&kr_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
     }
     for (int s = 0; s < 4; ++s) {
       mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4); mbar_init(&vote_bar[s], 1); mbar_init(&vote_read[s], 1);
-      mbar_init(&turn_done[s], 4);
+      mbar_init(&turn_done[s], 1);
       flag[s] = 0;
     }
     for (int s = 0; s < 8; ++s) { mbar_init(&ret_full[s], 1); mbar_init(&ret_free[s], 1); }
     mbar_init(&fin_bar, 1);
+    for (int i = 0; i < 2 * NG * 4; ++i) {
+      (&st_l[0][0][0])[i] = 0.f; (&st_m[0][0][0])[i] = -INFINITY; (&st_y[0][0][0])[i] = 0.f; (&st_a[0][0][0])[i] = -INFINITY;
+    }
+    for (int i = 0; i < 2 * NG; ++i) (&st_r[0][0])[i] = 0;
     mbar_fence_init();
   }
   __syncthreads();
@@ -227,7 +213,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         geometry(item, b, hkv, split, T, j0);
         if (T == 0) continue;
         const int ip = ne & 1;
-        ok = MWAIT(__LINE__, &q_empty[ip], ((ne >> 1) & 1) ^ 1, status);
+        ok = mbar_wait(&q_empty[ip], ((ne >> 1) & 1) ^ 1, status);
         if (!ok) break;
         mbar_arrive_expect_tx(&qr_full[ip], (uint32_t)R * 128u * 2u);   // two panels of R rows x 128 bytes
         for (int pn = 0; pn < 2; ++pn)
@@ -235,13 +221,12 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int t = 0; t < T && ok; ++t, ++g) {
           const int s = g % NS;
           const uint32_t ph = (uint32_t)((g / NS) & 1);
-          ok = MWAIT(__LINE__, &kr_empty[s], ph ^ 1u, status);
+          ok = mbar_wait(&kr_empty[s], ph ^ 1u, status);
           if (!ok) break;
-          F8TR(0, g);
           mbar_arrive_expect_tx(&kr_full[s], RB);
           tma_load_4d(sKr + s * RB, &tmK, &kr_full[s], 0, (j0 - t) * 128, hkv, b);
           if (kDense) {   // every tile is retained: V follows K
-            ok = MWAIT(__LINE__, &v_empty[s], ph ^ 1u, status);
+            ok = mbar_wait(&v_empty[s], ph ^ 1u, status);
             if (!ok) break;
             mbar_arrive_expect_tx(&v_full[s], RB);
             tma_load_4d(sVr + s * RB, &tmV, &v_full[s], 0, (j0 - t) * 128, hkv, b);
@@ -279,18 +264,15 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       for (; c.valid && ok; advance(c)) {
         const int ip = c.ne & 1, sb = c.g & 3, kc = c.g % NS;
         if (c.g >= 4) {
-          ok = MWAITW(__LINE__, &s_free[sb], (uint32_t)(((c.g >> 2) - 1) & 1), status);
-#ifdef MALA_F8_TRACE
-          if (!ok && lane == 0 && f8_fail[0] == (int)blockIdx.x + 1) { f8_fail[20] = c.g; f8_fail[21] = c.item; f8_fail[22] = c.t; }
-#endif
+          ok = mbar_wait_warp(&s_free[sb], (uint32_t)(((c.g >> 2) - 1) & 1), status);
           // (the vote of the tile that had this slot has been read: its flag may be overwritten)
-          if (!kDense && ok) ok = MWAITW(__LINE__, &vote_read[sb], (uint32_t)(((c.g >> 2) - 1) & 1), status);
+          if (!kDense && ok) ok = mbar_wait_warp(&vote_read[sb], (uint32_t)(((c.g >> 2) - 1) & 1), status);
         }
         if (ok && c.t == 0) {
           // the item's queries have landed (which the producer requested once the MMAs of the item two before had
           // read this slot): row qh (128 bf16 in two 64-column panels, lane = four consecutive columns) becomes
           // rows qh and 4 + qh of the e4m3 operand
-          ok = MWAITW(__LINE__, &qr_full[ip], (uint32_t)((c.ne >> 1) & 1), status);
+          ok = mbar_wait_warp(&qr_full[ip], (uint32_t)((c.ne >> 1) & 1), status);
           if (!ok) break;
           const uint8_t* qraw = sQ + ip * Cfg::kQBytes;
           uint8_t* q8 = sQ8 + ip * Cfg::kQ8Bytes;
@@ -316,10 +298,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           fence_proxy_async_smem();
           __syncwarp();
         }
-        if (ok) ok = MWAITW(__LINE__, &kr_full[kc], (uint32_t)((c.g / NS) & 1), status);
+        if (ok) ok = mbar_wait_warp(&kr_full[kc], (uint32_t)((c.g / NS) & 1), status);
         if (!ok) break;
         tc_fence_after();
-        F8TR(1, c.g);
         const uint32_t dS = tmem_addr(tb, 0, (uint32_t)sb * 16u);
         const uint64_t dQ = desc_advance(dQ0, ip * Cfg::kQ8Bytes), dK = desc_advance(dK0, kc * RB);
 #pragma unroll
@@ -337,15 +318,15 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (!kDense) {
         int nv = 0;                              // raw V copies requested -- ring slot nv % 6
         for (; c.valid && ok; advance(c)) {
-          ok = MWAITW(__LINE__, &vote_bar[c.g & 3], (uint32_t)((c.g >> 2) & 1), status);
-          if (ok && c.g >= 8) ok = MWAITW(__LINE__, &ret_free[c.g & 7], (uint32_t)(((c.g >> 3) - 1) & 1), status);
+          ok = mbar_wait_warp(&vote_bar[c.g & 3], (uint32_t)((c.g >> 2) & 1), status);
+          if (ok && c.g >= 8) ok = mbar_wait_warp(&ret_free[c.g & 7], (uint32_t)(((c.g >> 3) - 1) & 1), status);
           if (!ok) break;
           const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[c.g & 3], 0) != 0;
           __syncwarp();
           if (leader) mbar_arrive(&vote_read[c.g & 3]);
           if (retain) {
             const int vs = nv % NS;
-            if (nv >= NS) ok = MWAITW(__LINE__, &v_empty[vs], (uint32_t)(((nv / NS) - 1) & 1), status);
+            if (nv >= NS) ok = mbar_wait_warp(&v_empty[vs], (uint32_t)(((nv / NS) - 1) & 1), status);
             if (!ok) break;
             if (leader) {
               mbar_arrive_expect_tx(&v_full[vs], RB);
@@ -366,14 +347,14 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const uint64_t dV0 = make_smem_desc(smem_u32(sVr), 16384, 1024);   // V tile read MN-major (M = channel)
       const uint64_t dP0 = make_smem_desc(smem_u32(sP), 16, 1024);
       int npv = 0;                               // PVs issued so far: raw V stage npv % 6
-      int npv_g[NG], r_item_g[NG];               // ... per softmax group (P8^T slot 2 group + (n & 1)), and of the current item
+      int npv_g[NG], r_item_g[NG];               // ... per softmax group (P8^T slot 4 group + n % 4), and of the current item
 #pragma unroll
       for (int i = 0; i < NG; ++i) { npv_g[i] = 0; r_item_g[i] = 0; }
       int r_item = 0;
       for (; c.valid && ok; advance(c)) {
         bool retain = true;
         if (!kDense) {
-          ok = MWAITW(__LINE__, &ret_full[c.g & 7], (uint32_t)((c.g >> 3) & 1), status);
+          ok = mbar_wait_warp(&ret_full[c.g & 7], (uint32_t)((c.g >> 3) & 1), status);
           if (!ok) break;
           retain = __shfl_sync(0xffffffffu, *(volatile int*)&ret_ring[c.g & 7], 0) != 0;
           __syncwarp();
@@ -385,14 +366,13 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           int n_g = 0, ri_g = 0;
 #pragma unroll
           for (int i = 0; i < NG; ++i) if (i == gp) { n_g = npv_g[i]; ri_g = r_item_g[i]; }
-          const int ps = 2 * gp + (n_g & 1), vc = npv % NS;
-          ok = MWAITW(__LINE__, &p_full[ps], (uint32_t)((n_g >> 1) & 1), status);
-          if (ok) ok = MWAITW(__LINE__, &v_full[vc], (uint32_t)((npv / NS) & 1), status);
+          const int ps = PP * gp + (n_g % PP), vc = npv % NS;
+          ok = mbar_wait_warp(&p_full[ps], (uint32_t)((n_g / PP) & 1), status);
+          if (ok) ok = mbar_wait_warp(&v_full[vc], (uint32_t)((npv / NS) & 1), status);
           if (ok && r_item == 0 && c.ne >= 2)
-            ok = MWAITW(__LINE__, &o_free[ip], (uint32_t)(((c.ne >> 1) - 1) & 1), status);
+            ok = mbar_wait_warp(&o_free[ip], (uint32_t)(((c.ne >> 1) - 1) & 1), status);
           if (!ok) break;
           tc_fence_after();
-          F8TR(2, c.g);
           const uint32_t dO = tmem_addr(tb, 0, Cfg::kColO + (uint32_t)(ip * NG + gp) * 16u);
           const uint64_t dV = desc_advance(dV0, vc * RB), dP = desc_advance(dP0, ps * Cfg::kP8Bytes);
           const uint32_t acc0 = ri_g > 0 ? 1u : 0u;
@@ -415,7 +395,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       if (leader) tc_commit(&fin_bar);
       __syncwarp();
-      MWAITW(__LINE__, &fin_bar, 0, status);
+      mbar_wait_warp(&fin_bar, 0, status);
     }
     if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
   } else if (warp >= 4 + 4 * NG) {
@@ -444,7 +424,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         continue;
       }
       const int ip = ne & 1;
-      ok = MWAIT(__LINE__, &item_done[ip], (uint32_t)((ne >> 1) & 1), status);
+      ok = mbar_wait(&item_done[ip], (uint32_t)((ne >> 1) & 1), status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -478,7 +458,15 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
       }
       tc_fence_before();
-      __syncwarp();
+      __syncwarp();   // (every lane has read the state)
+      if (head) {     // the slot starts the item after next empty
+#pragma unroll
+        for (int s2 = 0; s2 < NG; ++s2) {
+#pragma unroll
+          for (int q = 0; q < GH; ++q) { st_l[ip][s2][q] = 0.f; st_a[ip][s2][q] = -INFINITY; }
+          *(volatile int*)&st_r[ip][s2] = 0;
+        }
+      }
       if (lane == 0) mbar_arrive(&o_free[ip]);
 #pragma unroll
       for (int q = 0; q < GH; ++q)
@@ -510,7 +498,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const bool publisher = (lane % kLanesPerRow) == 0;
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(p.Nk, 1)));
     int ne = 0, g0 = 0;                          // non-empty items so far, tiles of those items
-    int rg = 0;                                  // retained tiles of this group so far: P8^T slot 2 grp + (rg & 1)
+    int rg = 0;                                  // retained tiles of this group so far: P8^T slot 4 grp + rg % 4
+    int nt_own = 0;                              // tiles of this group so far (phase of its decision barrier)
     uint32_t xc = 0;                             // exchanges of this group so far (buffer and barrier phase xc & 1)
     bool ok = true;
     // one value per (warp, row) to all threads of the group
@@ -519,7 +508,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       if (publisher) xch[grp][xb][w][pub_row] = mine;
       __syncwarp();
       if (lane == 0) mbar_arrive(&grp_bar[grp]);
-      bool k = MWAIT(__LINE__, &grp_bar[grp], xc & 1, status);
+      bool k = mbar_wait(&grp_bar[grp], xc & 1, status);
       k = __all_sync(0xffffffffu, k);
       ++xc;
       if (!k) return false;
@@ -544,11 +533,11 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const int ip = ne & 1;
       const uint32_t colO = Cfg::kColO + (uint32_t)(ip * NG + grp) * 16u;
       uint32_t* bm_row = p.bitmask ? p.bitmask + stat_row * p.words : nullptr;
-      float m_ref[GH], l[GH], yref[GH], c2q[GH];
+      float m_ref[GH], l[GH], yref[GH], c2q[GH], a_own[GH];
 #pragma unroll
-      for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; c2q[q] = c2; }
+      for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; c2q[q] = c2; a_own[q] = -INFINITY; }
       int r = 0;                                 // tiles of the item this group has retained
-      bool have_q = false;
+      bool have_q = false, have_slot = false;
       for (int t = (grp + NG - g0 % NG) % NG; t < T; t += NG) {
         const int g = g0 + t;
         if (first) {
@@ -575,13 +564,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
         }
         const int sb = g & 3;
-        ok = MWAIT(__LINE__, &s_full[sb], (uint32_t)((g >> 2) & 1), status);
+        ok = mbar_wait(&s_full[sb], (uint32_t)((g >> 2) & 1), status);
         ok = __all_sync(0xffffffffu, ok);
-#ifdef MALA_F8_TRACE
-        if (!ok && w == 0 && lane == 0 && f8_fail[0] == (int)blockIdx.x + 1) { f8_fail[16 + grp] = g; f8_fail[12 + grp] = item; }
-#endif
         if (!ok) break;
-        if (w == 0) F8TR(3, g);
         tc_fence_after();
         uint32_t sr[LDN];
         tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, (uint32_t)sb * 16u), sr);
@@ -595,51 +580,27 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           have_q = true;
         }
         const int kpos = (j0 - t) * 128 + kt;
-        float x[GH], tmax[GH];
-        {
-          float mx[GH], a0[GH], a1[GH], a2[GH], a3[GH];
+        float x[GH], tmax[GH], psum[GH];
 #pragma unroll
-          for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
-            x[q] = (kpos < p.Nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
-            mx[q] = x[q];
-          }
-          if (w == 0) F8TR(11, g);
-          RowReduce<GH, 16, true>::run(mx, lane);
-          if (w == 0) F8TR(12, g);
-          ok = exchange(mx[0], a0, a1, a2, a3);
-          if (!ok) break;
-#pragma unroll
-          for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
+        for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
+          x[q] = (kpos < p.Nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
+          psum[q] = 0.f;
         }
-        if (w == 0) F8TR(4, g);
-        // probabilities against the group's references, ahead of the decision, unless a reference has to be raised
-        bool fast = true;
-        if (r == 0) {
-#pragma unroll
-          for (int q = 0; q < GH; ++q) { m_ref[q] = tmax[q]; yref[q] = tmax[q] + lv; }   // (nothing accumulated yet)
-        } else {
-#pragma unroll
-          for (int q = 0; q < GH; ++q)
-            fast = fast && !(q < R && (tmax[q] + lv > yref[q] + kPGap || tmax[q] > m_ref[q] + kMGap));
-        }
-        float psum[GH];
-#pragma unroll
-        for (int q = 0; q < GH; ++q) psum[q] = 0.f;
-        const int ps = 2 * grp + (rg & 1);
-        auto probabilities = [&]() -> bool {     // P8^T of this tile into slot ps, psum[] = its row sums
-          if (rg >= 2) {
-            bool k = MWAIT(__LINE__, &p_free[ps], (uint32_t)(((rg >> 1) - 1) & 1), status);
+        const int ps = PP * grp + (rg % PP);
+        // P8^T of this tile into slot ps against the group's references; e[] = the unrounded exp2(x - m)
+        auto store_p = [&](float (&e)[GH]) -> bool {
+          if (rg >= PP) {
+            bool k = mbar_wait(&p_free[ps], (uint32_t)(((rg / PP) - 1) & 1), status);
             k = __all_sync(0xffffffffu, k);
             if (!k) return false;
           }
-          float e[GH], pp[GH], a0[GH], a1[GH], a2[GH], a3[GH];
+          float pp[GH];
 #pragma unroll
           for (int q = 0; q < GH; ++q) {
             e[q] = (q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
             // P' = 64 exp2(x + lv - yref) = e * 64 exp2(m + lv - yref): the tile's V scale rides on the probability
             pp[q] = (q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
           }
-          if (w == 0) F8TR(10, g);
           uint8_t* dst = sP + ps * Cfg::kP8Bytes;
           const uint32_t chunk = (uint32_t)kt >> 4, within = (uint32_t)kt & 15u;
           if constexpr (GH == 1) {
@@ -656,51 +617,56 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               dst[(q + 5) * 128 + ((chunk ^ (uint32_t)(q + 5)) << 4) + within] = (uint8_t)(s01.y >> 8);
             }
           }
-          if (w == 0) F8TR(7, g);
           fence_proxy_async_smem();
-          if (w == 0) F8TR(8, g);
+          return true;
+        };
+        // ... and its row sums over the group
+        auto probabilities = [&]() -> bool {
+          float e[GH], a0[GH], a1[GH], a2[GH], a3[GH];
+          if (!store_p(e)) return false;
           RowReduce<GH, 16, false>::run(e, lane);
-          if (w == 0) F8TR(9, g);
           if (!exchange(e[0], a0, a1, a2, a3)) return false;
 #pragma unroll
           for (int q = 0; q < GH; ++q) psum[q] = (a0[q] + a1[q]) + (a2[q] + a3[q]);
           return true;
         };
-        if (fast) { ok = probabilities(); if (!ok) break; }
-        if (w == 0) F8TR(5, g);
-        // ---- the turn of tile g: Eq. 3 against the normalizer after tile g - 1, the groups' two streams combined
-        if (g > 0) {
-          ok = MWAIT(__LINE__, &turn_done[(g - 1) & 3], (uint32_t)(((g - 1) >> 2) & 1), status);
-          ok = __all_sync(0xffffffffu, ok);
+        // The row maxima first; then the probabilities against the group's references, ahead of the decision, unless
+        // a maximum is too far above a reference (they are then formed on the slow path, after the decision).
+        bool fast = true;
+        {
+          float mx[GH], a0[GH], a1[GH], a2[GH], a3[GH];
+#pragma unroll
+          for (int q = 0; q < GH; ++q) mx[q] = x[q];
+          RowReduce<GH, 16, true>::run(mx, lane);
+          ok = exchange(mx[0], a0, a1, a2, a3);
           if (!ok) break;
+#pragma unroll
+          for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
         }
-        if (w == 0) F8TR(13, g);
-        bool retain = true;
-        if (!kDense && t > 0) {
-          float M[GH], L[GH];
+        if (r == 0) {
 #pragma unroll
-          for (int q = 0; q < GH; ++q) { M[q] = r > 0 ? m_ref[q] : -INFINITY; L[q] = r > 0 ? l[q] : 0.f; }
-#pragma unroll
-          for (int o2 = 1; o2 < NG; ++o2) {       // the other groups' streams as published at their last turns
-            const int og = (grp + o2) % NG;
-            float mo[GH], lo[GH];
-            lds_row<GH>(st_m[ip][og], mo);
-            lds_row<GH>(st_l[ip][og], lo);
-#pragma unroll
-            for (int q = 0; q < GH; ++q)
-              if (lo[q] > 0.f) {
-                const float Mn = fmaxf(M[q], mo[q]);
-                L[q] = L[q] * fast_exp2(M[q] - Mn) + lo[q] * fast_exp2(mo[q] - Mn);   // (0 * exp2(-inf) = 0)
-                M[q] = Mn;
-              }
-          }
-          retain = false;
+          for (int q = 0; q < GH; ++q) { m_ref[q] = tmax[q]; yref[q] = tmax[q] + lv; }   // (nothing accumulated yet)
+        } else {
 #pragma unroll
           for (int q = 0; q < GH; ++q)
-            retain = retain || (q < R && !(((tmax[q] - (M[q] + __log2f(L[q]))) - theta) < 0.f));
+            fast = fast && !(q < R && (tmax[q] + lv > yref[q] + kPGap || tmax[q] > m_ref[q] + kMGap));
         }
-        if (retain && !fast) {
-          // raise the references first: this group's O^T (its earlier PVs have to be complete) and l follow
+        if (fast) { ok = probabilities(); if (!ok) break; }
+        // ---- the turn of tile g.  Eq. 3 needs the normalizer after tile g - 1: the streams of all groups as published
+        // at their last turns.  One thread of the group (its head) takes the turn -- waits for the turn before, decides,
+        // publishes the group's new state and hands the turn on -- so that the chain from tile to tile is a few dozen
+        // instructions of one thread; the others pick the decision up behind it.
+        if (!have_slot) {   // the item's state slot is that of the item two before, which has to have been written out
+          if (ne >= 2) {
+            ok = mbar_wait(&o_free[ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          have_slot = true;
+        }
+        // raises the references to this tile's maxima: l follows here, this group's O^T (whose earlier PVs have to be
+        // complete) in TMEM; then the probabilities against the new references
+        auto slow_probabilities = [&]() -> bool {
           float alpha[GH];
           bool touch = false;
 #pragma unroll
@@ -716,9 +682,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
           }
           if (touch) {
-            ok = MWAIT(__LINE__, &p_free[2 * grp + ((rg - 1) & 1)], (uint32_t)(((rg - 1) >> 1) & 1), status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            bool k = mbar_wait(&p_free[PP * grp + ((rg - 1) % PP)], (uint32_t)(((rg - 1) / PP) & 1), status);
+            k = __all_sync(0xffffffffu, k);
+            if (!k) return false;
             tc_fence_after();
             uint32_t o[LDN];
             tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colO), o);
@@ -732,47 +698,104 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             tmem_wait_st();
             tc_fence_before();
           }
-          ok = probabilities();
-          if (!ok) break;
-        }
-        if (retain) {
+          return probabilities();
+        };
+        // the group's state after this tile, for the other groups' turns and the write-out
+        auto publish = [&](int r_new) {
+#pragma unroll
+          for (int q = 0; q < GH; ++q) { st_m[ip][grp][q] = m_ref[q]; st_l[ip][grp][q] = l[q]; st_y[ip][grp][q] = yref[q]; }
+          *(volatile int*)&st_r[ip][grp] = r_new;
+        };
+        bool retain = true;
+        if (kDense) {
+          // no decision to take, hence no order between the groups: the state only serves the write-out
+          if (!fast) { ok = slow_probabilities(); if (!ok) break; }
 #pragma unroll
           for (int q = 0; q < GH; ++q) l[q] += psum[q];
           ++r;
-        }
-        if (t == 0 && ne >= 2) {   // the state slot is that of the item two before, which has to have been written out
-          ok = MWAIT(__LINE__, &o_free[ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
-        // (the state is published before the tile's P8^T or vote is handed on: what follows from either -- the PV, the
-        // item's completion, its write-out -- then sees it)
-        if (head) {
+          if (head) publish(r);
+        } else {
+          bool handed_on = false;
+          if (head) {
+            // everything that does not need the other groups is ready before the wait: this stream's log-sum-exp
+            // before the tile (a_own) and after it, should it be retained (psum is known on the fast path)
+            float a_ret[GH];
 #pragma unroll
-          for (int q = 0; q < GH; ++q) { st_m[ip][grp][q] = m_ref[q]; st_l[ip][grp][q] = l[q]; st_y[ip][grp][q] = yref[q]; }
-          *(volatile int*)&st_r[ip][grp] = r;
-          if (t == 0) {   // the other groups have seen nothing of this item yet
+            for (int q = 0; q < GH; ++q) a_ret[q] = m_ref[q] + __log2f(l[q] + psum[q]);
+            if (g > 0) ok = mbar_wait(&turn_done[(g - 1) & 3], (uint32_t)(((g - 1) >> 2) & 1), status);
+            if (ok) {
+              if (t > 0) {
+                float lse[GH];
 #pragma unroll
-            for (int o2 = 1; o2 < NG; ++o2) {
-              const int og = (grp + o2) % NG;
+                for (int q = 0; q < GH; ++q) lse[q] = a_own[q];
 #pragma unroll
-              for (int q = 0; q < GH; ++q) { st_m[ip][og][q] = -INFINITY; st_l[ip][og][q] = 0.f; st_y[ip][og][q] = 0.f; }
-              *(volatile int*)&st_r[ip][og] = 0;
+                for (int o2 = 1; o2 < NG; ++o2) {
+                  float ao[GH];
+                  lds_row<GH>(st_a[ip][(grp + o2) % NG], ao);
+#pragma unroll
+                  for (int q = 0; q < GH; ++q) {   // log2(2^lse + 2^ao); a stream without a tile is at -inf
+                    const float M = fmaxf(lse[q], ao[q]), d = fminf(lse[q], ao[q]) - M;
+                    lse[q] = M + __log2f(1.f + fast_exp2(d));
+                  }
+                }
+                retain = false;
+#pragma unroll
+                for (int q = 0; q < GH; ++q) retain = retain || (q < R && !(((tmax[q] - lse[q]) - theta) < 0.f));
+              }
+              *(volatile int*)&flag[g & 3] = retain ? 1 : 0;
+              if (fast || !retain) {   // the stream's new log-sum-exp is known: the turn is handed on at once
+#pragma unroll
+                for (int q = 0; q < GH; ++q) st_a[ip][grp][q] = retain ? a_ret[q] : a_own[q];
+                mbar_arrive(&turn_done[g & 3]);
+                if (retain) {
+#pragma unroll
+                  for (int q = 0; q < GH; ++q) l[q] += psum[q];
+                }
+                publish(r + (retain ? 1 : 0));
+                mbar_arrive(&vote_bar[g & 3]);
+                handed_on = true;
+              }
+              mbar_arrive(&dec_bar[grp]);
             }
           }
-          if (!kDense) {
-            *(volatile int*)&flag[g & 3] = retain ? 1 : 0;
+          ok = __all_sync(0xffffffffu, ok);
+          if (ok && !head) ok = mbar_wait(&dec_bar[grp], (uint32_t)(nt_own & 1), status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          retain = *(volatile int*)&flag[g & 3] != 0;
+          if (retain && !fast) {   // (every thread of the group; the head keeps the turn until the state is known)
+            ok = slow_probabilities();
+            if (!ok) break;
+          }
+          if (retain) {
+            if (!(head && handed_on)) {
+#pragma unroll
+              for (int q = 0; q < GH; ++q) l[q] += psum[q];
+            }
+            ++r;
+          }
+          // this stream's log-sum-exp after the tile (all threads keep it; the head's copy is the one that is used)
+          if (retain) {
+#pragma unroll
+            for (int q = 0; q < GH; ++q) a_own[q] = m_ref[q] + __log2f(l[q]);
+          }
+          if (head && !handed_on) {
+#pragma unroll
+            for (int q = 0; q < GH; ++q) st_a[ip][grp][q] = a_own[q];
+            mbar_arrive(&turn_done[g & 3]);
+            publish(r);
             mbar_arrive(&vote_bar[g & 3]);
           }
-          if (retain && bm_row) atomicOr(bm_row + ((T - 1 - t) >> 5), 1u << ((T - 1 - t) & 31));
         }
+        ++nt_own;
+        if (head && retain && bm_row) atomicOr(bm_row + ((T - 1 - t) >> 5), 1u << ((T - 1 - t) & 31));
+        // (the state was published before the tile's P8^T is handed on: the PV, the item's completion and its write-out
+        // follow from the arrivals below)
         __syncwarp();
         if (retain) {
           ++rg;
           if (lane == 0) mbar_arrive(&p_full[ps]);
         }
-        if (lane == 0) mbar_arrive(&turn_done[g & 3]);
-        if (w == 0) F8TR(6, g);
       }
       if (!ok) break;
       ++ne;

@@ -296,9 +296,11 @@ def test_decode_head_size_64_gated_paged_several_tokens(mala, oracle, tau):
     assert _run_multi(mala, oracle, w, 3, tau, 8) > 0
 
 
-def _run_fp8(mala, oracle, w, tau, num_splits):
+def _run_fp8(mala, oracle, w, tau, num_splits, rounding_bound=False):
     """mala_decode_fp8 on the e4m3 codes of a cache against the oracle on the dequantised values (the oracle has no
-    8-bit arithmetic of its own: it is handed scale * e4m3(code) as fp32)."""
+    8-bit arithmetic of its own: it is handed scale * e4m3(code) as fp32).  rounding_bound: outputs are compared by
+    parity.check_output's rounding model (a probability enters the PV product with a relative error of 2^-9, as in the
+    bf16 kernels, here as the sum of two e4m3 numbers; the output is cast to bf16)."""
     k8, ks, kd = W.quantize_cache_e4m3(w["kcache"])
     v8, vs, vd = W.quantize_cache_e4m3(w["vcache"])
     q = w["q"].cuda()
@@ -309,6 +311,7 @@ def _run_fp8(mala, oracle, w, tau, num_splits):
     torch.cuda.synchronize()
     assert mala.device_status() == 0
     ref = oracle.decode(w["q"], kd, vd, w["scale"], tau, num_splits, 128)
+    ref_abs = oracle.decode(w["q"], kd, vd.abs(), w["scale"], tau, num_splits, 128) if rounding_bound else None
     tps = ref["mask"].shape[-1]
     gm = st.mask(tps).cpu().numpy()
     o_c, lse_c = o.float().cpu().numpy()[:, 0], lse.cpu().numpy()
@@ -320,7 +323,7 @@ def _run_fp8(mala, oracle, w, tau, num_splits):
                                   tau, Nk, 128)
                 assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
             hs = slice(g * G, (g + 1) * G)
-            parity.check_output(o_c[b, hs], ref["o"][b, hs])
+            parity.check_output(o_c[b, hs], ref["o"][b, hs], a_ref=ref_abs["o"][b, hs] if rounding_bound else None)
             assert np.abs(lse_c[b, hs] - ref["lse"][b, hs]).max() <= parity.LSE_ABS
             skipped += int((ref["mask"][b, g] == 1).sum())
             retained += int((ref["mask"][b, g] == 2).sum())
@@ -341,6 +344,16 @@ def test_decode_fp8_cache_skips_value_tiles(mala, oracle, Nk, S, tau):
     w = W.custom_decode(2, 8, 2, Nk, 128, S, group_types=["diffuse", "peaked"], seed=3, preset="D")
     res = _run_fp8(mala, oracle, w, tau, S)
     assert res["skipped"] > 0, "workload must exercise skipping"
+    assert res["totals"][1] == res["retained"] + res["skipped"]
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("B,Nk,S,Hq,Hkv", [(40, 3000, 5, 8, 8), (24, 1500, 7, 16, 4), (64, 700, 3, 4, 2)])
+def test_decode_fp8_cache_many_work_items_per_cta(mala, oracle, B, Nk, S, Hq, Hkv, tau):
+    """More (sequence, KV head, split) items than SMs, with one to five tiles each: every CTA walks several items, the
+    softmax groups change places from item to item and the state slots and accumulators are handed back and reused."""
+    w = W.custom_decode(B, Hq, Hkv, Nk, 128, S, seed=B + Nk, preset="D" if tau > 0 else "literal")
+    res = _run_fp8(mala, oracle, w, tau, S, rounding_bound=True)
     assert res["totals"][1] == res["retained"] + res["skipped"]
 
 
