@@ -458,7 +458,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
       }
       tc_fence_before();
-      __syncwarp();   // (every lane has read the state)
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // every thread of the group has read the item's state
       if (head) {     // the slot starts the item after next empty
 #pragma unroll
         for (int s2 = 0; s2 < NG; ++s2) {

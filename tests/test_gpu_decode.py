@@ -357,6 +357,24 @@ def test_decode_fp8_cache_many_work_items_per_cta(mala, oracle, B, Nk, S, Hq, Hk
     assert res["totals"][1] == res["retained"] + res["skipped"]
 
 
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+def test_decode_fp8_repeated_launches_give_identical_bits(mala, tau):
+    """Several work items per CTA, eight tiles each, launched many times: the result does not depend on how the groups
+    of a CTA happen to interleave (no atomics on the data path, every hand-over through a barrier)."""
+    w = W.custom_decode(8, 32, 8, 16384, 128, 16, seed=9, preset="D", device="cuda")
+    k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
+    v8, vs, _ = W.quantize_cache_e4m3(w["vcache"])
+    first = None
+    for _ in range(40):
+        o, lse, _ = mala.decode_fp8(w["q"], k8, v8, ks, vs, w["scale"], tau, 16)
+        if first is None:
+            first = (o.clone(), lse.clone())
+            assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+        else:
+            assert torch.equal(o, first[0]) and torch.equal(lse, first[1])
+    assert mala.device_status() == 0
+
+
 def test_decode_fp8_refuses_what_it_does_not_support(mala):
     w = W.custom_decode(1, 8, 1, 256, 128, 1, seed=1)
     k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
