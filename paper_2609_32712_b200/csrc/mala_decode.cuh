@@ -181,6 +181,8 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
   p.kscale = kscale; p.vscale = vscale;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Nk = Nk; p.tps = tps; p.num_splits = num_splits; p.words = (tps + 31) / 32;
   p.n_items = B * Hkv * num_splits; p.nt = (Nk + 127) / 128;
+  p.by_splits.set((uint32_t)num_splits);
+  p.by_hkv.set((uint32_t)Hkv);
   p.scale_log2 = scale * 1.4426950408889634f;
   p.log2_tau = tau > 0.f ? log2f(tau) : -INFINITY;
   if (p.bitmask &&

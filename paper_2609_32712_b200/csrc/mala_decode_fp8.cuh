@@ -59,6 +59,25 @@
 
 namespace mala {
 
+// Division of a 32-bit number by a divisor known at launch, as a multiplication and shifts (every thread of the
+// softmax groups works out which sequence, KV head and split a work item is; hardware has no integer divide, and the
+// few dozen dependent instructions of an emulated one sit on the per-tile chain of those threads).
+struct FastDiv {
+  uint32_t d, mul, sh;
+  __host__ void set(uint32_t divisor) {
+    d = divisor;
+    uint32_t l = 0;
+    while ((1ull << l) < divisor) ++l;
+    sh = l;
+    mul = (uint32_t)(((1ull << 32) * ((1ull << l) - divisor)) / divisor + 1);
+  }
+  __device__ __forceinline__ uint32_t div(uint32_t n) const {
+    if (d == 1u) return n;
+    const uint32_t t = __umulhi(mul, n);
+    return (t + ((n - t) >> 1)) >> (sh - 1u);
+  }
+};
+
 struct DecF8Params {
   float* o_part;                 // [B, Hq, num_splits, 128] fp32, normalised per split
   float* lse_part;               // [B, Hq, num_splits] natural log; -inf for an empty split
@@ -70,11 +89,8 @@ struct DecF8Params {
   const float* vscale;           // [B, Hkv, nt]
   int B, Hq, Hkv, Nk, tps, num_splits, words, n_items, nt;
   float scale_log2, log2_tau;
+  FastDiv by_splits, by_hkv;
 };
-
-#ifndef MALA_F8_GROUPS
-#define MALA_F8_GROUPS 2
-#endif
 
 struct DecF8Cfg {
   static constexpr int kRawBytes = 128 * 128;            // one e4m3 tile
@@ -82,7 +98,7 @@ struct DecF8Cfg {
   static constexpr int kQBytes = 4096;                   // 16 rows x 128 bf16, as copied
   static constexpr int kQ8Bytes = 2048;                  // 16 rows x 128 e4m3
   static constexpr int kP8Bytes = 2048;                  // 16 rows x 128 e4m3
-  static constexpr int kGroups = MALA_F8_GROUPS;         // softmax groups: group n takes tiles n, n + kGroups, .. of an item
+  static constexpr int kGroups = 2;                      // softmax groups (at most three: the rings of four)
   static constexpr int kPPerGroup = 4;                   // P8^T slots of a group: how far it may run ahead of its PVs
   static constexpr int kPSlots = kPPerGroup * kGroups;
   static constexpr int kSmemBytes = 2 * kStages * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPSlots * kP8Bytes + 1024;
@@ -191,10 +207,10 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const uint32_t tb = tmem_base_s;
 
   auto geometry = [&](int item, int& b, int& hkv, int& split, int& T, int& j0) {
-    split = item % p.num_splits;
-    const int bh = item / p.num_splits;
-    hkv = bh % p.Hkv;
-    b = bh / p.Hkv;
+    const int bh = (int)p.by_splits.div((uint32_t)item);
+    split = item - bh * p.num_splits;
+    b = (int)p.by_hkv.div((uint32_t)bh);
+    hkv = bh - b * p.Hkv;
     const int lo = split * p.tps * 128;
     const int hi = min(p.Nk, lo + p.tps * 128);
     T = hi > lo ? (hi - lo + 127) / 128 : 0;
