@@ -861,23 +861,30 @@ def main():
                               "achieved_gbs": need / (us * 1e-6) / 1e9,
                               "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
             row["speedup"] = row["dense"]["us"] / row["mala"]["us"]
-            # the same cache stored as e4m3 with one scale per 128-key tile (mala_decode_fp8): half the bytes
+            # the same cache stored as e4m3 with one scale per 128-key tile (mala_decode_fp8): half the bytes.  Two
+            # layouts of the same [B,Nk,Hkv,d] view: key-major (a key's heads adjacent, the layout of the bf16 rows) and
+            # head-major (a head's keys adjacent: a tile is then one contiguous 16 KB run instead of 128-byte pieces)
             k8, ks8, _ = W.quantize_cache_e4m3(kc)
             v8, vs8, _ = W.quantize_cache_e4m3(vc)
+            head_major = lambda x: x.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
             f8 = {}
-            for label, t_ in (("mala", tau), ("dense", 0.0)):
-                us = 1e3 * time_cuda(lambda: mala.decode_fp8(qd, k8, v8, ks8, vs8, wd["scale"], t_, dcfg.num_splits, ws=wsd,
-                                                              out=od, want_lse=False), 25, 100)
-                o8, _, st = mala.decode_fp8(qd, k8, v8, ks8, vs8, wd["scale"], t_, dcfg.num_splits, ws=wsd, stats=True)
-                torch.cuda.synchronize()
-                ret, leg = st.totals.cpu().tolist()
-                need = (leg + ret) * TILE * dcfg.d              # one byte per element
-                o16, _, _ = mala.decode(qd, kc, vc, wd["scale"], t_, dcfg.num_splits)
-                f8[label] = {"us": us, "retained_frac": ret / leg, "needed_gb": need / 1e9,
-                             "achieved_gbs": need / (us * 1e-6) / 1e9,
-                             "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                             "speedup_vs_bf16_cache": row[label]["us"] / us,
-                             "rel_l2_o_vs_bf16_cache": float((o8.float() - o16.float()).norm() / o16.float().norm())}
+            for layout, (ka, va) in (("key_major", (k8, v8)), ("head_major", (head_major(k8), head_major(v8)))):
+                lay = {}
+                for label, t_ in (("mala", tau), ("dense", 0.0)):
+                    us = 1e3 * time_cuda(lambda: mala.decode_fp8(qd, ka, va, ks8, vs8, wd["scale"], t_, dcfg.num_splits,
+                                                                  ws=wsd, out=od, want_lse=False), 25, 100)
+                    o8, _, st = mala.decode_fp8(qd, ka, va, ks8, vs8, wd["scale"], t_, dcfg.num_splits, ws=wsd, stats=True)
+                    torch.cuda.synchronize()
+                    ret, leg = st.totals.cpu().tolist()
+                    need = (leg + ret) * TILE * dcfg.d              # one byte per element
+                    o16, _, _ = mala.decode(qd, kc, vc, wd["scale"], t_, dcfg.num_splits)
+                    lay[label] = {"us": us, "retained_frac": ret / leg, "needed_gb": need / 1e9,
+                                  "achieved_gbs": need / (us * 1e-6) / 1e9,
+                                  "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                  "speedup_vs_bf16_cache": row[label]["us"] / us,
+                                  "rel_l2_o_vs_bf16_cache": float((o8.float() - o16.float()).norm() / o16.float().norm())}
+                f8[layout] = lay
+                del ka, va
             row["e4m3_cache"] = f8
             del k8, v8, ks8, vs8
             if preset == "D":                       # work and fidelity against the dense decode, tau up to 1

@@ -92,14 +92,17 @@ struct DecF8Params {
   FastDiv by_splits, by_hkv;
 };
 
+// NG_: softmax groups -- two for the MALA kernel (their turns couple them; a third only adds to the chain), three for
+// the dense kernel (unordered groups; at most three: the rings of four)
+template <int NG_>
 struct DecF8Cfg {
   static constexpr int kRawBytes = 128 * 128;            // one e4m3 tile
   static constexpr int kStages = 6;                      // raw K ring, raw V ring
   static constexpr int kQBytes = 4096;                   // 16 rows x 128 bf16, as copied
   static constexpr int kQ8Bytes = 2048;                  // 16 rows x 128 e4m3
   static constexpr int kP8Bytes = 2048;                  // 16 rows x 128 e4m3
-  static constexpr int kGroups = 2;                      // softmax groups (at most three: the rings of four)
-  static constexpr int kPPerGroup = 4;                   // P8^T slots of a group: how far it may run ahead of its PVs
+  static constexpr int kGroups = NG_;
+  static constexpr int kPPerGroup = kGroups == 2 ? 4 : 2;                   // P8^T slots of a group: how far it may run ahead of its PVs
   static constexpr int kPSlots = kPPerGroup * kGroups;
   static constexpr int kSmemBytes = 2 * kStages * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPSlots * kP8Bytes + 1024;
   static constexpr int kThreads = 128 * (2 + kGroups);   // issuing warps, softmax groups, epilogue group
@@ -135,11 +138,11 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
   return make_uint2(lead, f32x2_to_e4m3x2((a - back.x) * 16.f, (b - back.y) * 16.f));
 }
 
-template <bool kDense, int GP>
-__global__ void __launch_bounds__(DecF8Cfg::kThreads, 1)
+template <bool kDense, int GP, int NG_ = (kDense ? 3 : 2)>
+__global__ void __launch_bounds__(DecF8Cfg<NG_>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
-  using Cfg = DecF8Cfg;
+  using Cfg = DecF8Cfg<NG_>;
   constexpr int RB = Cfg::kRawBytes, NS = Cfg::kStages, NG = Cfg::kGroups, PP = Cfg::kPPerGroup;
   constexpr int GH = GP;                   // rows of a softmax group
   constexpr int LDN = 16;

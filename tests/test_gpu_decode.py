@@ -375,6 +375,19 @@ def test_decode_fp8_repeated_launches_give_identical_bits(mala, tau):
     assert mala.device_status() == 0
 
 
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+def test_decode_fp8_head_major_cache_view(mala, tau):
+    """The cache views are strided: a head-major [B,Hkv,Nk,d] cache passed as its [B,Nk,Hkv,d] view gives the bits of
+    the key-major one."""
+    w = W.custom_decode(2, 8, 2, 3000, 128, 5, seed=4, preset="D", device="cuda")
+    k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
+    v8, vs, _ = W.quantize_cache_e4m3(w["vcache"])
+    hm = lambda x: x.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    o0, l0, _ = mala.decode_fp8(w["q"], k8, v8, ks, vs, w["scale"], tau, 5)
+    o1, l1, _ = mala.decode_fp8(w["q"], hm(k8), hm(v8), ks, vs, w["scale"], tau, 5)
+    assert torch.equal(o0, o1) and torch.equal(l0, l1)
+
+
 def test_decode_fp8_refuses_what_it_does_not_support(mala):
     w = W.custom_decode(1, 8, 1, 256, 128, 1, seed=1)
     k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
