@@ -17,7 +17,7 @@
 //                   heads per KV head), products of e4m3 values are exact in the fp32 accumulator, and a softmax
 //                   thread forms (S[h] + S[4 + h] / 16) * scale * kscale / 2^k.
 //   O^T += V8^T P8^T  V8 is read MN-major.  A probability enters as P' = 64 exp2(y - yref) with y = x + log2(vscale)
-//                   the score of the key weighted by its V tile's scale and yref a running reference of the stream
+//                   the score of the key weighted by its V tile's scale and yref a running reference of the item
 //                   (so the tile's scale rides on P', inside e4m3's narrow range whatever its magnitude), split as
 //                   p1 = e4m3(P'), p2 = e4m3(16 (P' - p1)): relative error 2^-9 for P' >= 2^-6, absolute 2^-14 below
 //                   (2^-20 of the largest probability).  yref is raised, and O^T rescaled, whenever a tile's largest
@@ -25,32 +25,25 @@
 //                   is summed in fp32 from the unrounded exp2(x - m), with its own reference m.
 //
 // At one byte per element a tile arrives twice as fast as in the bf16 kernels, faster than one softmax group can
-// take tiles one after the other (its per-tile chain of TMEM load, two cross-warp reductions, exponentials and the
-// P^T store is latency, not throughput).  Two softmax groups therefore take alternate tiles (by the CTA's running tile
-// count, so that a group's consecutive tiles are never further apart than the rings of four are deep), each with its
-// own references, normalizer, P^T slots and O^T accumulator: two online-softmax streams per work item, merged when
-// the item is written out.  Everything a tile needs is computed without the item's state -- its row maxima, its
-// probabilities against the group's own references, their sums -- except the skip test of Eq. 3, which needs the
-// normalizer after the tile before it.  That test is the "turn" of a tile, and turns are taken in tile order (a ring
-// of barriers): one thread of the group waits for the turn before, combines its stream's log-sum-exp with the other
-// group's published one (all that the test needs), decides, publishes and hands the turn on -- a few dozen
-// instructions of one thread -- and the rest of the group picks the decision up behind it.  The probabilities of a
-// tile that turns out to be skipped were computed for nothing (a few exponentials per thread); its P^T slot is
-// simply reused.  A tile that needs a reference raised takes the slow order instead (decision first, then the
-// rescaling, then the probabilities, the turn held meanwhile).  The dense kernel (tau = 0) has no decision to take
-// and its groups run unordered.
+// take tiles one after the other: its per-tile chain (TMEM load, a cross-warp maximum, the Eq. 3 test, exponentials,
+// the P^T store, a cross-warp sum) is latency, not throughput, and Eq. 3 makes it sequential within a work item.  So
+// a CTA runs NG independent pipelines ("streams") side by side, each the whole of what the bf16 kernel's CTA is: its
+// own rings of raw K and V tiles, S^T ring, P^T slots, accumulators, its own issuing warps and its own softmax group
+// walking one work item at a time, tile by tile, with the item's state in registers.  The CTA's work items go to
+// the streams in turn.  Nothing is shared between the streams but the SM, so none ever waits for another.  An item's
+// partial output is written by an epilogue group once its last PV has completed, so that no softmax group stalls at
+// an item boundary.
 //
-// Every warp that issues asynchronous work walks the CTA's tiles in order and blocks on exactly what its next
-// instruction needs (a warp that polls the barriers of several jobs in one loop, sleeping in between, reacts to each
-// event a loop iteration late, which at this rate is slower than the tiles arrive):
-//   warp 0       TMA producer (Q, raw K ring of six; dense kernel: raw V ring of six)
-//   warp 1       converts an item's queries, issues S^T of every tile
-//   warp 2       MALA kernel: takes the votes in tile order, requests the raw V copy of a retained tile
-//   warp 3       issues O^T += V8^T P8^T of every retained tile
-//   warps 4-7    softmax group 0 (thread = key of the tile), up to four packed query heads
-//   warps 8-11   softmax group 1
-//   warps 12-15  epilogue group (thread = output channel): merges the streams of a finished item, writes its partial
-//                output and log-sum-exp, hands the item's state slot and accumulators back
+// Every warp that issues asynchronous work has one job, walks its stream's tiles in order and blocks on exactly what
+// its next instruction needs (a warp that polls the barriers of several jobs in one loop, sleeping in between,
+// reacts to each event a loop iteration late, which at this rate is slower than the tiles arrive).  Per stream k:
+//   warp k            TMA producer (Q, raw K ring; dense kernel: raw V ring)
+//   warp NG + k       converts an item's queries, issues S^T of every tile
+//   warp 2NG + k      MALA kernel: takes the votes in order, requests the raw V copy of a retained tile
+//   warp 3NG + k      issues O^T += V8^T P8^T of every retained tile
+//   warps 4NG + 4k .. softmax group (thread = key of the tile), up to four packed query heads
+// and for all streams
+//   last four warps   epilogue group (thread = output channel)
 #pragma once
 #include <cuda_fp16.h>
 
@@ -59,9 +52,9 @@
 
 namespace mala {
 
-// Division of a 32-bit number by a divisor known at launch, as a multiplication and shifts (every thread of the
-// softmax groups works out which sequence, KV head and split a work item is; hardware has no integer divide, and the
-// few dozen dependent instructions of an emulated one sit on the per-tile chain of those threads).
+// Division of a 32-bit number by a divisor known at launch, as a multiplication and shifts (every role works out for
+// itself which sequence, KV head and split a work item is; hardware has no integer divide, and the few dozen
+// dependent instructions of an emulated one would sit on the per-tile chain of the softmax threads).
 struct FastDiv {
   uint32_t d, mul, sh;
   __host__ void set(uint32_t divisor) {
@@ -92,22 +85,21 @@ struct DecF8Params {
   FastDiv by_splits, by_hkv;
 };
 
-// NG_: softmax groups -- two for the MALA kernel (their turns couple them; a third only adds to the chain), three for
-// the dense kernel (unordered groups; at most three: the rings of four)
+// NG_: streams
 template <int NG_>
 struct DecF8Cfg {
   static constexpr int kRawBytes = 128 * 128;            // one e4m3 tile
-  static constexpr int kStages = 6;                      // raw K ring, raw V ring
-  static constexpr int kQBytes = 4096;                   // 16 rows x 128 bf16, as copied
-  static constexpr int kQ8Bytes = 2048;                  // 16 rows x 128 e4m3
-  static constexpr int kP8Bytes = 2048;                  // 16 rows x 128 e4m3
   static constexpr int kGroups = NG_;
-  static constexpr int kPPerGroup = kGroups == 2 ? 4 : 2;                   // P8^T slots of a group: how far it may run ahead of its PVs
-  static constexpr int kPSlots = kPPerGroup * kGroups;
-  static constexpr int kSmemBytes = 2 * kStages * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPSlots * kP8Bytes + 1024;
-  static constexpr int kThreads = 128 * (2 + kGroups);   // issuing warps, softmax groups, epilogue group
-  static constexpr uint32_t kColO = 64;                  // S^T ring 4 x 16, then O^T 2 x kGroups x 16 (item parity, group)
-  static constexpr uint32_t kTmemCols = (kColO + 2 * kGroups * 16) <= 128 ? 128 : 256;
+  static constexpr int kStages = 6 / NG_;                // raw K ring, raw V ring of a stream
+  static constexpr int kQBytes = 1024;                   // landing buffer of an item's queries as copied: 4 rows x 128 bf16
+  static constexpr int kQ8Bytes = 2048;                  // 16 rows x 128 e4m3, one per item parity
+  static constexpr int kP8Bytes = 2048;                  // 16 rows x 128 e4m3
+  static constexpr int kPPerGroup = 4;                   // P8^T slots of a stream: how far its softmax group may run ahead of its PVs
+  static constexpr int kStreamBytes = 2 * kStages * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPPerGroup * kP8Bytes;
+  static constexpr int kSmemBytes = kGroups * kStreamBytes + 1024;
+  static constexpr int kThreads = 32 * (4 * kGroups) + 128 * kGroups + 128;   // issuing warps, softmax groups, epilogue group
+  static constexpr uint32_t kColsPerStream = 96;         // S^T ring 4 x 16, O^T 2 x 16 (item parity)
+  static constexpr uint32_t kTmemCols = kGroups * kColsPerStream <= 128 ? 128 : 256;
 };
 
 // Instruction descriptor of tcgen05.mma kind::f8f6f4 with e4m3 A and B (format 0), fp32 accumulate
@@ -138,36 +130,35 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
   return make_uint2(lead, f32x2_to_e4m3x2((a - back.x) * 16.f, (b - back.y) * 16.f));
 }
 
-template <bool kDense, int GP, int NG_ = (kDense ? 3 : 2)>
+// The CTA's tile sequence.  Its non-empty work items (blockIdx.x, + gridDim.x, ..) are handed to the NG streams in
+// order, each stream taking the next one when it has finished its own; the tiles of the streams' current items are
+// interleaved round-robin.  pos counts the tiles of the sequence (ring slots are pos % depth).  The state is a few
+// integers and depends on tile counts only, so every role keeps its own copy in step.
+template <bool kDense, int GP, int NG_ = 2>
 __global__ void __launch_bounds__(DecF8Cfg<NG_>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
   using Cfg = DecF8Cfg<NG_>;
   constexpr int RB = Cfg::kRawBytes, NS = Cfg::kStages, NG = Cfg::kGroups, PP = Cfg::kPPerGroup;
   constexpr int GH = GP;                   // rows of a softmax group
-  constexpr int LDN = 16;
+  constexpr int LDN = 8;                   // S^T / O^T columns a thread reads (leading parts 0..3, remainders 4..7)
   constexpr float kPScale = 64.f;          // P' of the key that sets the reference
   constexpr float kPGap = 2.8f;            // log2(448 / 64), rounded down: how far y may pass yref
   constexpr float kMGap = 60.f;            // ... and x the normalizer's reference (fp32)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* sKr = smem;                     // [6] raw K
-  uint8_t* sVr = sKr + NS * RB;            // [6] raw V
-  uint8_t* sQ = sVr + NS * RB;             // [2] item parity, bf16 as copied
-  uint8_t* sQ8 = sQ + 2 * Cfg::kQBytes;    // [2] item parity: rows h = q1, 4 + h = q2, rest zero
-  uint8_t* sP = sQ8 + 2 * Cfg::kQ8Bytes;   // [4 NG] P8^T slots (4 group + n % 4): rows h = p1, 4 + h = p2, rest zero
 
-  __shared__ uint64_t qr_full[2], q_empty[2], kr_full[NS], kr_empty[NS], v_full[NS], v_empty[NS], s_full[4], s_free[4],
-      vote_bar[4], vote_read[4], turn_done[4], p_full[PP * NG], p_free[PP * NG], item_done[2], o_free[2], fin_bar,
-      grp_bar[NG], dec_bar[NG], ret_full[8], ret_free[8];
+  // per stream
+  __shared__ uint64_t qr_full[NG][2], qr_free[NG][2], q8_free[NG][2], kr_full[NG][NS], kr_empty[NG][NS], v_full[NG][NS],
+      v_empty[NG][NS], s_full[NG][4], s_free[NG][4], vote_bar[NG][4], vote_read[NG][4], p_full[NG][PP], p_free[NG][PP],
+      item_done[NG][2], st_full[NG][2], o_free[NG][2], grp_bar[NG], ret_full[NG][8], ret_free[NG][8], fin_bar[NG];
   __shared__ uint32_t tmem_base_s;
-  __shared__ int flag[4];
-  __shared__ int ret_ring[8];              // decision of tile g at g & 7 (vote warp -> PV warp)
-  __shared__ float q_inv[8][4];            // 2^-k of the rows of non-empty item number n, at n & 7
-  __shared__ __align__(16) float xch[NG][2][4][8];         // [group][buffer][warp][row]
-  __shared__ __align__(16) float st_m[2][NG][4], st_l[2][NG][4], st_y[2][NG][4];   // [item parity][group][row]: (m, l, yref)
-  __shared__ __align__(16) float st_a[2][NG][4];           // ... and m + log2 l, all that the other groups' turns need
-  __shared__ int st_r[2][NG];                              // ... and retained tiles of the group in the item
+  __shared__ int flag[NG][4];
+  __shared__ int ret_ring[NG][8];          // decision of the stream's tile g at g & 7 (vote warp -> PV warp)
+  __shared__ float q_inv[NG][2][4];        // 2^-k of the query rows of a stream's item
+  __shared__ __align__(16) float xch[NG][2][4][4];         // [stream][buffer][warp][row]
+  __shared__ __align__(16) float st_m[NG][2][4], st_l[NG][2][4], st_y[NG][2][4];   // a finished item's (m, l, yref)
+  __shared__ int st_r[NG][2];                              // ... and its retained tiles
   __shared__ int early_exit;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -175,30 +166,37 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const int R = G;
   int* status = p.status;
 
-  for (int i = tid; i < (2 * Cfg::kQ8Bytes + Cfg::kPSlots * Cfg::kP8Bytes) / 16; i += Cfg::kThreads)
-    reinterpret_cast<uint4*>(sQ8)[i] = make_uint4(0u, 0u, 0u, 0u);
+  // the stream's part of shared memory
+  auto stream_base = [&](int k) -> uint8_t* { return smem + k * Cfg::kStreamBytes; };
+  // [NS] raw K | [NS] raw V | [2] Q8 (item parity) | [PP] P8^T | [2] Q landing buffers
+  auto sKr_of = [&](int k) -> uint8_t* { return stream_base(k); };
+  auto sVr_of = [&](int k) -> uint8_t* { return stream_base(k) + NS * RB; };
+  auto sQ8_of = [&](int k) -> uint8_t* { return stream_base(k) + 2 * NS * RB; };
+  auto sP_of = [&](int k) -> uint8_t* { return stream_base(k) + 2 * NS * RB + 2 * Cfg::kQ8Bytes; };
+  auto sQ_of = [&](int k) -> uint8_t* { return stream_base(k) + 2 * NS * RB + 2 * Cfg::kQ8Bytes + PP * Cfg::kP8Bytes; };
+
+  for (int k = 0; k < NG; ++k)   // Q8 and P8^T rows that are never written stay zero
+    for (int i = tid; i < (2 * Cfg::kQ8Bytes + PP * Cfg::kP8Bytes) / 16; i += Cfg::kThreads)
+      reinterpret_cast<uint4*>(sQ8_of(k))[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_proxy_async_smem();
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&qr_full[s], 1); mbar_init(&q_empty[s], 1); mbar_init(&item_done[s], 1); mbar_init(&o_free[s], 4);
+    for (int k = 0; k < NG; ++k) {
+      mbar_init(&grp_bar[k], 4); mbar_init(&fin_bar[k], 1);
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(&qr_full[k][i], 1); mbar_init(&qr_free[k][i], 1); mbar_init(&q8_free[k][i], 1);
+        mbar_init(&item_done[k][i], 1); mbar_init(&st_full[k][i], 1); mbar_init(&o_free[k][i], 4);
+      }
+      for (int s = 0; s < PP; ++s) { mbar_init(&p_full[k][s], 4); mbar_init(&p_free[k][s], 1); }
+      for (int s = 0; s < NS; ++s) {
+        mbar_init(&kr_full[k][s], 1); mbar_init(&kr_empty[k][s], 1); mbar_init(&v_full[k][s], 1); mbar_init(&v_empty[k][s], 1);
+      }
+      for (int s = 0; s < 4; ++s) {
+        mbar_init(&s_full[k][s], 1); mbar_init(&s_free[k][s], 4); mbar_init(&vote_bar[k][s], 1); mbar_init(&vote_read[k][s], 1);
+        flag[k][s] = 0;
+      }
+      for (int s = 0; s < 8; ++s) { mbar_init(&ret_full[k][s], 1); mbar_init(&ret_free[k][s], 1); }
     }
-    for (int s = 0; s < NG; ++s) { mbar_init(&grp_bar[s], 4); mbar_init(&dec_bar[s], 1); }
-    for (int s = 0; s < PP * NG; ++s) { mbar_init(&p_full[s], 4); mbar_init(&p_free[s], 1); }
-    for (int s = 0; s < NS; ++s) {
-      mbar_init(&kr_full[s], 1); mbar_init(&kr_empty[s], 1); mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
-    }
-    for (int s = 0; s < 4; ++s) {
-      mbar_init(&s_full[s], 1); mbar_init(&s_free[s], 4); mbar_init(&vote_bar[s], 1); mbar_init(&vote_read[s], 1);
-      mbar_init(&turn_done[s], 1);
-      flag[s] = 0;
-    }
-    for (int s = 0; s < 8; ++s) { mbar_init(&ret_full[s], 1); mbar_init(&ret_free[s], 1); }
-    mbar_init(&fin_bar, 1);
-    for (int i = 0; i < 2 * NG * 4; ++i) {
-      (&st_l[0][0][0])[i] = 0.f; (&st_m[0][0][0])[i] = -INFINITY; (&st_y[0][0][0])[i] = 0.f; (&st_a[0][0][0])[i] = -INFINITY;
-    }
-    for (int i = 0; i < 2 * NG; ++i) (&st_r[0][0])[i] = 0;
     mbar_fence_init();
   }
   __syncthreads();
@@ -209,230 +207,238 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
 
-  auto geometry = [&](int item, int& b, int& hkv, int& split, int& T, int& j0) {
+  // tiles, sequence, KV head, split and newest tile of a work item
+  auto tiles_of = [&](int item) -> int {
+    const int split = item - (int)p.by_splits.div((uint32_t)item) * p.num_splits;
+    const int lo = split * p.tps * 128;
+    const int hi = min(p.Nk, lo + p.tps * 128);
+    return hi > lo ? (hi - lo + 127) >> 7 : 0;
+  };
+  auto geometry = [&](int item, int& b, int& hkv, int& split, int& j0, int T) {
     const int bh = (int)p.by_splits.div((uint32_t)item);
     split = item - bh * p.num_splits;
     b = (int)p.by_hkv.div((uint32_t)bh);
     hkv = bh - b * p.Hkv;
-    const int lo = split * p.tps * 128;
-    const int hi = min(p.Nk, lo + p.tps * 128);
-    T = hi > lo ? (hi - lo + 127) / 128 : 0;
-    j0 = lo / 128 + T - 1;
+    j0 = split * p.tps + T - 1;
   };
   auto scale_index = [&](int b, int hkv, int jt) -> int { return (b * p.Hkv + hkv) * p.nt + jt; };
+  // the CTA's work items are blockIdx.x, + gridDim.x, ..; stream k takes the k-th, (k + NG)-th, .. of them
+  const int item_step = NG * (int)gridDim.x;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-      int ne = 0, g = 0;
-      bool ok = true;
-      for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-        int b, hkv, split, T, j0;
-        geometry(item, b, hkv, split, T, j0);
-        if (T == 0) continue;
-        const int ip = ne & 1;
-        ok = mbar_wait(&q_empty[ip], ((ne >> 1) & 1) ^ 1, status);
-        if (!ok) break;
-        mbar_arrive_expect_tx(&qr_full[ip], (uint32_t)R * 128u * 2u);   // two panels of R rows x 128 bytes
-        for (int pn = 0; pn < 2; ++pn)
-          tma_load_4d(sQ + ip * Cfg::kQBytes + pn * 2048, &tmQ, &qr_full[ip], pn * 64, hkv * G, 0, b);
-        for (int t = 0; t < T && ok; ++t, ++g) {
-          const int s = g % NS;
-          const uint32_t ph = (uint32_t)((g / NS) & 1);
-          ok = mbar_wait(&kr_empty[s], ph ^ 1u, status);
-          if (!ok) break;
-          mbar_arrive_expect_tx(&kr_full[s], RB);
-          tma_load_4d(sKr + s * RB, &tmK, &kr_full[s], 0, (j0 - t) * 128, hkv, b);
-          if (kDense) {   // every tile is retained: V follows K
-            ok = mbar_wait(&v_empty[s], ph ^ 1u, status);
-            if (!ok) break;
-            mbar_arrive_expect_tx(&v_full[s], RB);
-            tma_load_4d(sVr + s * RB, &tmV, &v_full[s], 0, (j0 - t) * 128, hkv, b);
-          }
-        }
-        ++ne;
-      }
-      if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
-    }
-  } else if (warp <= 3) {
-    // ------------------------------------------------------------------ the three issuing warps
+  if (warp < 4 * NG) {
+    // ------------------------------------------------------------------ the issuing warps of stream k
+    const int job = warp / NG, k = warp - job * NG;
+    const int item0 = (int)blockIdx.x + k * (int)gridDim.x;
+    uint8_t* sKr = sKr_of(k);
+    uint8_t* sVr = sVr_of(k);
+    uint8_t* sQ8 = sQ8_of(k);
+    uint8_t* sP = sP_of(k);
+    uint8_t* sQ = sQ_of(k);
+    const uint32_t tS = tmem_addr(tb, 0, (uint32_t)k * Cfg::kColsPerStream);          // S^T ring of the stream
+    const uint32_t tO = tmem_addr(tb, 0, (uint32_t)k * Cfg::kColsPerStream + 64u);    // its two accumulators
     const uint32_t leader = elect_one();
-    struct Cur { int item, ne, t, T, b, hkv, j0, g; bool valid; };
-    auto first_item = [&](Cur& c, int from, int ne, int g) {
-      c.valid = false;
-      c.g = g;
-      for (int item = from; item < p.n_items; item += gridDim.x) {
-        int b, hkv, split, T, j0;
-        geometry(item, b, hkv, split, T, j0);
-        if (T > 0) { c.item = item; c.ne = ne; c.t = 0; c.T = T; c.b = b; c.hkv = hkv; c.j0 = j0; c.valid = true; return; }
-      }
-    };
-    auto advance = [&](Cur& c) {
-      if (c.t + 1 < c.T) { ++c.t; ++c.g; return; }
-      first_item(c, c.item + gridDim.x, c.ne + 1, c.g + 1);
-    };
-    Cur c;
-    first_item(c, blockIdx.x, 0, 0);
     bool ok = true;
-    if (warp == 1) {
+    if (job == 0) {
+      // ---- TMA producer
+      if (lane == 0) {
+        tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+        int ne = 0, g = 0;
+        for (int item = item0; item < p.n_items && ok; item += item_step) {
+          const int T = tiles_of(item);
+          if (T == 0) continue;
+          int b, hkv, split, j0;
+          geometry(item, b, hkv, split, j0, T);
+          const int qs = ne & 1;
+          if (ne >= 2) ok = mbar_wait(&qr_free[k][qs], (uint32_t)(((ne >> 1) - 1) & 1), status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&qr_full[k][qs], (uint32_t)R * 128u * 2u);   // two panels of R rows x 128 bytes
+          for (int pn = 0; pn < 2; ++pn)
+            tma_load_4d(sQ + qs * Cfg::kQBytes + pn * 512, &tmQ, &qr_full[k][qs], pn * 64, hkv * G, 0, b);
+          for (int t = 0; t < T && ok; ++t, ++g) {
+            const int s = g % NS;
+            const uint32_t ph = (uint32_t)((g / NS) & 1);
+            ok = mbar_wait(&kr_empty[k][s], ph ^ 1u, status);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&kr_full[k][s], RB);
+            tma_load_4d(sKr + s * RB, &tmK, &kr_full[k][s], 0, (j0 - t) * 128, hkv, b);
+            if (kDense) {   // every tile is retained: V follows K
+              ok = mbar_wait(&v_empty[k][s], ph ^ 1u, status);
+              if (!ok) break;
+              mbar_arrive_expect_tx(&v_full[k][s], RB);
+              tma_load_4d(sVr + s * RB, &tmV, &v_full[k][s], 0, (j0 - t) * 128, hkv, b);
+            }
+          }
+          ++ne;
+        }
+      }
+    } else if (job == 1) {
       // ---- Q of an item -> two e4m3 rows per head; S^T = K8 Q8^T of every tile
       constexpr uint32_t idesc_qk = make_idesc_e4m3(128, 16, false, false);
       const uint64_t dQ0 = make_smem_desc(smem_u32(sQ8), 16, 1024);
       const uint64_t dK0 = make_smem_desc(smem_u32(sKr), 16, 1024);
-      for (; c.valid && ok; advance(c)) {
-        const int ip = c.ne & 1, sb = c.g & 3, kc = c.g % NS;
-        if (c.g >= 4) {
-          ok = mbar_wait_warp(&s_free[sb], (uint32_t)(((c.g >> 2) - 1) & 1), status);
-          // (the vote of the tile that had this slot has been read: its flag may be overwritten)
-          if (!kDense && ok) ok = mbar_wait_warp(&vote_read[sb], (uint32_t)(((c.g >> 2) - 1) & 1), status);
-        }
-        if (ok && c.t == 0) {
-          // the item's queries have landed (which the producer requested once the MMAs of the item two before had
-          // read this slot): row qh (128 bf16 in two 64-column panels, lane = four consecutive columns) becomes
-          // rows qh and 4 + qh of the e4m3 operand
-          ok = mbar_wait_warp(&qr_full[ip], (uint32_t)((c.ne >> 1) & 1), status);
-          if (!ok) break;
-          const uint8_t* qraw = sQ + ip * Cfg::kQBytes;
-          uint8_t* q8 = sQ8 + ip * Cfg::kQ8Bytes;
-          for (int qh = 0; qh < R; ++qh) {
-            const int e0 = lane * 4;
-            const uint8_t* src = qraw + (e0 >> 6) * 2048 + qh * 128 + (((((e0 & 63) >> 3)) ^ (qh & 7)) << 4) + (e0 & 7) * 2;
-            const uint2 w2 = *reinterpret_cast<const uint2*>(src);
-            float a[4] = {__uint_as_float(w2.x << 16), __uint_as_float(w2.x & 0xffff0000u), __uint_as_float(w2.y << 16),
-                          __uint_as_float(w2.y & 0xffff0000u)};
-            float mx = fmaxf(fmaxf(fabsf(a[0]), fabsf(a[1])), fmaxf(fabsf(a[2]), fabsf(a[3])));
+      int ne = 0, g = 0;
+      for (int item = item0; item < p.n_items && ok; item += item_step) {
+        const int T = tiles_of(item);
+        if (T == 0) continue;
+        const int ip = ne & 1;
+        uint8_t* q8 = sQ8 + ip * Cfg::kQ8Bytes;
+        // the item's queries have landed: row qh (128 bf16 in two 64-column panels, rows qh and 4 + qh of the
+        // landing atom; lane = four consecutive columns) becomes rows qh and 4 + qh of the e4m3 operand, once the
+        // MMAs of the item that had the operand's slot before have read it
+        ok = mbar_wait_warp(&qr_full[k][ip], (uint32_t)((ne >> 1) & 1), status);
+        if (ok && ne >= 2) ok = mbar_wait_warp(&q8_free[k][ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
+        if (!ok) break;
+        for (int qh = 0; qh < R; ++qh) {
+          const int e0 = lane * 4;
+          const int prow = qh + 4 * (e0 >> 6);
+          const uint8_t* src = sQ + ip * Cfg::kQBytes + prow * 128 + (((((e0 & 63) >> 3)) ^ prow) << 4) + (e0 & 7) * 2;
+          const uint2 w2 = *reinterpret_cast<const uint2*>(src);
+          float a[4] = {__uint_as_float(w2.x << 16), __uint_as_float(w2.x & 0xffff0000u), __uint_as_float(w2.y << 16),
+                        __uint_as_float(w2.y & 0xffff0000u)};
+          float mx = fmaxf(fmaxf(fabsf(a[0]), fabsf(a[1])), fmaxf(fabsf(a[2]), fabsf(a[3])));
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            // 2^k brings the row's largest magnitude into [128, 256)  (k = 0 for a zero row; kept inside fp32's exponents)
-            const int ef = (int)((__float_as_uint(mx) >> 23) & 0xffu);
-            const int k = ef == 0 ? 0 : min(max(134 - ef, -100), 100);
-            const float up = __uint_as_float((uint32_t)(k + 127) << 23), down = __uint_as_float((uint32_t)(127 - k) << 23);
-            const uint2 s01 = split_e4m3x2(a[0] * up, a[1] * up), s23 = split_e4m3x2(a[2] * up, a[3] * up);
-            const int r2 = 4 + qh;
-            *reinterpret_cast<uint32_t*>(q8 + qh * 128 + (((e0 >> 4) ^ (qh & 7)) << 4) + (e0 & 15)) = s01.x | (s23.x << 16);
-            *reinterpret_cast<uint32_t*>(q8 + r2 * 128 + (((e0 >> 4) ^ (r2 & 7)) << 4) + (e0 & 15)) = s01.y | (s23.y << 16);
-            if (lane == 0) q_inv[c.ne & 7][qh] = down;
+          for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+          // 2^k brings the row's largest magnitude into [128, 256)  (k = 0 for a zero row; kept inside fp32's exponents)
+          const int ef = (int)((__float_as_uint(mx) >> 23) & 0xffu);
+          const int kk = ef == 0 ? 0 : min(max(134 - ef, -100), 100);
+          const float up = __uint_as_float((uint32_t)(kk + 127) << 23), down = __uint_as_float((uint32_t)(127 - kk) << 23);
+          const uint2 s01 = split_e4m3x2(a[0] * up, a[1] * up), s23 = split_e4m3x2(a[2] * up, a[3] * up);
+          const int r2 = 4 + qh;
+          *reinterpret_cast<uint32_t*>(q8 + qh * 128 + (((e0 >> 4) ^ (qh & 7)) << 4) + (e0 & 15)) = s01.x | (s23.x << 16);
+          *reinterpret_cast<uint32_t*>(q8 + r2 * 128 + (((e0 >> 4) ^ (r2 & 7)) << 4) + (e0 & 15)) = s01.y | (s23.y << 16);
+          if (lane == 0) q_inv[k][ip][qh] = down;
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (leader) mbar_arrive(&qr_free[k][ip]);
+        const uint64_t dQ = desc_advance(dQ0, ip * Cfg::kQ8Bytes);
+        for (int t = 0; t < T && ok; ++t, ++g) {
+          const int sb = g & 3, kc = g % NS;
+          if (g >= 4) {
+            ok = mbar_wait_warp(&s_free[k][sb], (uint32_t)(((g >> 2) - 1) & 1), status);
+            // (the vote of the tile that had this slot has been read: its flag may be overwritten)
+            if (!kDense && ok) ok = mbar_wait_warp(&vote_read[k][sb], (uint32_t)(((g >> 2) - 1) & 1), status);
           }
-          fence_proxy_async_smem();
+          if (ok) ok = mbar_wait_warp(&kr_full[k][kc], (uint32_t)((g / NS) & 1), status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t dS = tS + (uint32_t)sb * 16u;
+          const uint64_t dK = desc_advance(dK0, kc * RB);
+#pragma unroll
+          for (int kq = 0; kq < 4; ++kq)     // 32 e4m3 elements of the head size per instruction
+            mma_ss_f8(dS, desc_advance(dK, kq * 32), desc_advance(dQ, kq * 32), idesc_qk, kq > 0, leader);
+          if (leader) {
+            tc_commit(&kr_empty[k][kc]);
+            tc_commit(&s_full[k][sb]);
+            if (t == T - 1) tc_commit(&q8_free[k][ip]);
+          }
           __syncwarp();
         }
-        if (ok) ok = mbar_wait_warp(&kr_full[kc], (uint32_t)((c.g / NS) & 1), status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t dS = tmem_addr(tb, 0, (uint32_t)sb * 16u);
-        const uint64_t dQ = desc_advance(dQ0, ip * Cfg::kQ8Bytes), dK = desc_advance(dK0, kc * RB);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)     // 32 e4m3 elements of the head size per instruction
-          mma_ss_f8(dS, desc_advance(dK, k * 32), desc_advance(dQ, k * 32), idesc_qk, k > 0, leader);
-        if (leader) {
-          tc_commit(&kr_empty[kc]);
-          tc_commit(&s_full[sb]);
-          if (c.t == c.T - 1) tc_commit(&q_empty[ip]);
-        }
-        __syncwarp();
+        ++ne;
       }
-    } else if (warp == 2) {
+    } else if (job == 2) {
       // ---- the votes (MALA kernel): a retained tile's raw V copy is requested, the decision is passed on
       if (!kDense) {
-        int nv = 0;                              // raw V copies requested -- ring slot nv % 6
-        for (; c.valid && ok; advance(c)) {
-          ok = mbar_wait_warp(&vote_bar[c.g & 3], (uint32_t)((c.g >> 2) & 1), status);
-          if (ok && c.g >= 8) ok = mbar_wait_warp(&ret_free[c.g & 7], (uint32_t)(((c.g >> 3) - 1) & 1), status);
-          if (!ok) break;
-          const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[c.g & 3], 0) != 0;
-          __syncwarp();
-          if (leader) mbar_arrive(&vote_read[c.g & 3]);
-          if (retain) {
-            const int vs = nv % NS;
-            if (nv >= NS) ok = mbar_wait_warp(&v_empty[vs], (uint32_t)(((nv / NS) - 1) & 1), status);
+        int g = 0, nv = 0;                       // tiles so far; raw V copies requested -- ring slot nv % NS
+        for (int item = item0; item < p.n_items && ok; item += item_step) {
+          const int T = tiles_of(item);
+          if (T == 0) continue;
+          int b, hkv, split, j0;
+          geometry(item, b, hkv, split, j0, T);
+          for (int t = 0; t < T && ok; ++t, ++g) {
+            ok = mbar_wait_warp(&vote_bar[k][g & 3], (uint32_t)((g >> 2) & 1), status);
+            if (ok && g >= 8) ok = mbar_wait_warp(&ret_free[k][g & 7], (uint32_t)(((g >> 3) - 1) & 1), status);
             if (!ok) break;
-            if (leader) {
-              mbar_arrive_expect_tx(&v_full[vs], RB);
-              tma_load_4d(sVr + vs * RB, &tmV, &v_full[vs], 0, (c.j0 - c.t) * 128, c.hkv, c.b);
+            const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[k][g & 3], 0) != 0;
+            __syncwarp();
+            if (leader) mbar_arrive(&vote_read[k][g & 3]);
+            if (retain) {
+              const int vs = nv % NS;
+              if (nv >= NS) ok = mbar_wait_warp(&v_empty[k][vs], (uint32_t)(((nv / NS) - 1) & 1), status);
+              if (!ok) break;
+              if (leader) {
+                mbar_arrive_expect_tx(&v_full[k][vs], RB);
+                tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, (j0 - t) * 128, hkv, b);
+              }
+              ++nv;
             }
-            ++nv;
+            if (leader) {
+              *(volatile int*)&ret_ring[k][g & 7] = retain ? 1 : 0;
+              mbar_arrive(&ret_full[k][g & 7]);
+            }
+            __syncwarp();
           }
-          if (leader) {
-            *(volatile int*)&ret_ring[c.g & 7] = retain ? 1 : 0;
-            mbar_arrive(&ret_full[c.g & 7]);
-          }
-          __syncwarp();
         }
       }
     } else {
-      // ---- O^T += V8^T P8^T of every retained tile, into the accumulator of the tile's softmax group
+      // ---- O^T += V8^T P8^T of every retained tile, into the accumulator of the item
       constexpr uint32_t idesc_pv = make_idesc_e4m3(128, 16, true, false);
       const uint64_t dV0 = make_smem_desc(smem_u32(sVr), 16384, 1024);   // V tile read MN-major (M = channel)
       const uint64_t dP0 = make_smem_desc(smem_u32(sP), 16, 1024);
-      int npv = 0;                               // PVs issued so far: raw V stage npv % 6
-      int npv_g[NG], r_item_g[NG];               // ... per softmax group (P8^T slot 4 group + n % 4), and of the current item
+      int ne = 0, g = 0, npv = 0;                // items, tiles, PVs so far: raw V stage npv % NS, P8^T slot npv % PP
+      for (int item = item0; item < p.n_items && ok; item += item_step) {
+        const int T = tiles_of(item);
+        if (T == 0) continue;
+        const int ip = ne & 1;
+        int r_item = 0;
+        for (int t = 0; t < T && ok; ++t, ++g) {
+          bool retain = true;
+          if (!kDense) {
+            ok = mbar_wait_warp(&ret_full[k][g & 7], (uint32_t)((g >> 3) & 1), status);
+            if (!ok) break;
+            retain = __shfl_sync(0xffffffffu, *(volatile int*)&ret_ring[k][g & 7], 0) != 0;
+            __syncwarp();
+            if (leader) mbar_arrive(&ret_free[k][g & 7]);
+          }
+          if (retain) {
+            const int ps = npv % PP, vc = npv % NS;
+            ok = mbar_wait_warp(&p_full[k][ps], (uint32_t)((npv / PP) & 1), status);
+            if (ok) ok = mbar_wait_warp(&v_full[k][vc], (uint32_t)((npv / NS) & 1), status);
+            // (the accumulator is that of the item two before, which has to have been written out)
+            if (ok && r_item == 0 && ne >= 2) ok = mbar_wait_warp(&o_free[k][ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t dO = tO + (uint32_t)ip * 16u;
+            const uint64_t dV = desc_advance(dV0, vc * RB), dP = desc_advance(dP0, ps * Cfg::kP8Bytes);
+            const uint32_t acc0 = r_item > 0 ? 1u : 0u;
 #pragma unroll
-      for (int i = 0; i < NG; ++i) { npv_g[i] = 0; r_item_g[i] = 0; }
-      int r_item = 0;
-      for (; c.valid && ok; advance(c)) {
-        bool retain = true;
-        if (!kDense) {
-          ok = mbar_wait_warp(&ret_full[c.g & 7], (uint32_t)((c.g >> 3) & 1), status);
-          if (!ok) break;
-          retain = __shfl_sync(0xffffffffu, *(volatile int*)&ret_ring[c.g & 7], 0) != 0;
+            for (int kq = 0; kq < 4; ++kq)     // 32 keys per instruction: 32 rows of the V tile, 32 bytes of a P8^T row
+              mma_ss_f8(dO, desc_advance(dV, kq * 4096), desc_advance(dP, kq * 32), idesc_pv, kq > 0 ? 1u : acc0, leader);
+            if (leader) { tc_commit(&v_empty[k][vc]); tc_commit(&p_free[k][ps]); }
+            ++npv;
+            ++r_item;
+          }
+          if (t == T - 1 && leader) tc_commit(&item_done[k][ip]);
           __syncwarp();
-          if (leader) mbar_arrive(&ret_free[c.g & 7]);
         }
-        const int ip = c.ne & 1;
-        if (retain) {
-          const int gp = c.g % NG;               // the softmax group of this tile
-          int n_g = 0, ri_g = 0;
-#pragma unroll
-          for (int i = 0; i < NG; ++i) if (i == gp) { n_g = npv_g[i]; ri_g = r_item_g[i]; }
-          const int ps = PP * gp + (n_g % PP), vc = npv % NS;
-          ok = mbar_wait_warp(&p_full[ps], (uint32_t)((n_g / PP) & 1), status);
-          if (ok) ok = mbar_wait_warp(&v_full[vc], (uint32_t)((npv / NS) & 1), status);
-          if (ok && r_item == 0 && c.ne >= 2)
-            ok = mbar_wait_warp(&o_free[ip], (uint32_t)(((c.ne >> 1) - 1) & 1), status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t dO = tmem_addr(tb, 0, Cfg::kColO + (uint32_t)(ip * NG + gp) * 16u);
-          const uint64_t dV = desc_advance(dV0, vc * RB), dP = desc_advance(dP0, ps * Cfg::kP8Bytes);
-          const uint32_t acc0 = ri_g > 0 ? 1u : 0u;
-#pragma unroll
-          for (int k = 0; k < 4; ++k)     // 32 keys per instruction: 32 rows of the V tile, 32 bytes of a P8^T row
-            mma_ss_f8(dO, desc_advance(dV, k * 4096), desc_advance(dP, k * 32), idesc_pv, k > 0 ? 1u : acc0, leader);
-          if (leader) { tc_commit(&v_empty[vc]); tc_commit(&p_free[ps]); }
-          ++npv;
-          ++r_item;
-#pragma unroll
-          for (int i = 0; i < NG; ++i) if (i == gp) { ++npv_g[i]; ++r_item_g[i]; }
-        }
-        if (c.t == c.T - 1) {
-          if (leader) tc_commit(&item_done[ip]);
-          r_item = 0;
-#pragma unroll
-          for (int i = 0; i < NG; ++i) r_item_g[i] = 0;
-        }
-        __syncwarp();
+        ++ne;
       }
-      if (leader) tc_commit(&fin_bar);
+      if (leader) tc_commit(&fin_bar[k]);
       __syncwarp();
-      mbar_wait_warp(&fin_bar, 0, status);
+      mbar_wait_warp(&fin_bar[k], 0, status);
     }
     if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
-  } else if (warp >= 4 + 4 * NG) {
+  } else if (warp >= 8 * NG) {
     // ------------------------------------------------------------------ epilogue group: thread = output channel
-    // An item is written out when its last PV has completed: the groups' streams (m, l, yref, O^T) are merged, the
-    // split's partial output and log-sum-exp stored, and the item's state slot and accumulators handed back.
+    // An item is written out when its last PV has completed and its stream has left its state: the partial output,
+    // normalised by the split's own normalizer, and the log-sum-exp are stored and the item's accumulator and state
+    // slot handed back.  The CTA's items are taken in their order, i.e. the streams in turn.
     const int w = warp & 3;
     const uint32_t lane_base = (uint32_t)w * 32u;
     const int kt = (int)lane_base + lane;
     const bool head = (kt == 0);
-    int ne = 0;
+    int ne_k[NG];
+#pragma unroll
+    for (int i = 0; i < NG; ++i) ne_k[i] = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-      int b, hkv, split, T, j0;
-      geometry(item, b, hkv, split, T, j0);
+    int k = 0;
+    for (int item = (int)blockIdx.x; item < p.n_items && ok; item += (int)gridDim.x, k = (k + 1 == NG) ? 0 : k + 1) {
+      const int T = tiles_of(item);
+      int b, hkv, split, j0;
+      geometry(item, b, hkv, split, j0, T);
       const size_t prow0 = ((size_t)b * p.Hq + hkv * G) * p.num_splits + split;
       const size_t stat_row = (size_t)(b * p.Hkv + hkv) * p.num_splits + split;
-      if (T == 0) {
+      if (T == 0) {   // a split without keys: (0, -inf)
 #pragma unroll
         for (int q = 0; q < GH; ++q)
           if (q < R) {
@@ -442,56 +448,32 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (head && p.retained) p.retained[stat_row] = 0u;
         continue;
       }
+      int ne = 0;
+#pragma unroll
+      for (int i = 0; i < NG; ++i) if (i == k) { ne = ne_k[i]; ++ne_k[i]; }
       const int ip = ne & 1;
-      ok = mbar_wait(&item_done[ip], (uint32_t)((ne >> 1) & 1), status);
+      ok = mbar_wait(&item_done[k][ip], (uint32_t)((ne >> 1) & 1), status);
+      ok = ok && mbar_wait(&st_full[k][ip], (uint32_t)((ne >> 1) & 1), status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      float M[GH], L[GH], num[GH];
-#pragma unroll
-      for (int q = 0; q < GH; ++q) { M[q] = -INFINITY; L[q] = 0.f; num[q] = 0.f; }
-      int r_all = 0;
-#pragma unroll
-      for (int s2 = 0; s2 < NG; ++s2) {
-        float ms[GH], ls[GH];
-        lds_row<GH>(st_m[ip][s2], ms);
-        lds_row<GH>(st_l[ip][s2], ls);
-#pragma unroll
-        for (int q = 0; q < GH; ++q) M[q] = fmaxf(M[q], ls[q] > 0.f ? ms[q] : -INFINITY);
-        r_all += *(volatile int*)&st_r[ip][s2];
-      }
-#pragma unroll
-      for (int s2 = 0; s2 < NG; ++s2) {
-        float ms[GH], ls[GH], ys[GH];
-        lds_row<GH>(st_m[ip][s2], ms);
-        lds_row<GH>(st_l[ip][s2], ls);
-        lds_row<GH>(st_y[ip][s2], ys);
-        uint32_t o[LDN];
-        tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, Cfg::kColO + (uint32_t)(ip * NG + s2) * 16u), o);
-        tmem_wait_ld();
-#pragma unroll
-        for (int q = 0; q < GH; ++q)
-          if (ls[q] > 0.f) {   // (the accumulator of a group that retained nothing was never written)
-            L[q] += ls[q] * fast_exp2(ms[q] - M[q]);
-            num[q] += fmaf(__uint_as_float(o[4 + q]), 0.0625f, __uint_as_float(o[q])) * fast_exp2(ys[q] - M[q]);
-          }
-      }
+      float ms[GH], ls[GH], ys[GH];
+      lds_row<GH>(st_m[k][ip], ms);
+      lds_row<GH>(st_l[k][ip], ls);
+      lds_row<GH>(st_y[k][ip], ys);
+      const int r_all = *(volatile int*)&st_r[k][ip];
+      uint32_t o[LDN];
+      tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, (uint32_t)k * Cfg::kColsPerStream + 64u + (uint32_t)ip * 16u), o);
+      tmem_wait_ld();
       tc_fence_before();
-      asm volatile("bar.sync 1, 128;" ::: "memory");   // every thread of the group has read the item's state
-      if (head) {     // the slot starts the item after next empty
-#pragma unroll
-        for (int s2 = 0; s2 < NG; ++s2) {
-#pragma unroll
-          for (int q = 0; q < GH; ++q) { st_l[ip][s2][q] = 0.f; st_a[ip][s2][q] = -INFINITY; }
-          *(volatile int*)&st_r[ip][s2] = 0;
-        }
-      }
-      if (lane == 0) mbar_arrive(&o_free[ip]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&o_free[k][ip]);
 #pragma unroll
       for (int q = 0; q < GH; ++q)
-        if (q < R) {
-          p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = num[q] / (L[q] * kPScale);
-          if (kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = (M[q] + __log2f(L[q])) * 0.6931471805599453f;
+        if (q < R) {   // O^T is in units of 2^yref / 64, l in units of 2^m
+          const float num = fmaf(__uint_as_float(o[4 + q]), 0.0625f, __uint_as_float(o[q])) * fast_exp2(ys[q] - ms[q]);
+          p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = num / (ls[q] * kPScale);
+          if (kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = (ms[q] + __log2f(ls[q])) * 0.6931471805599453f;
         }
       if (head) {
         if (p.retained) p.retained[stat_row] = (uint32_t)r_all;
@@ -500,13 +482,13 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           atomicAdd(&p.totals[1], (unsigned long long)T);
         }
       }
-      ++ne;
     }
   } else {
-    // ------------------------------------------------------------------ softmax groups: thread = key of the tile
-    // Group n takes the CTA's tiles n, n + NG, .. (counted through all its items, so that a group's consecutive
-    // tiles are never further apart than the rings of four are deep).
-    const int grp = (warp - 4) >> 2;
+    // ------------------------------------------------------------------ softmax group of stream k: thread = key of the tile
+    const int k = (warp - 4 * NG) >> 2;
+    const int item0 = (int)blockIdx.x + k * (int)gridDim.x;
+    uint8_t* sP = sP_of(k);
+    const uint32_t colS = (uint32_t)k * Cfg::kColsPerStream, colO0 = colS + 64u;
     const int w = warp & 3;
     const uint32_t lane_base = (uint32_t)w * 32u;
     const int kt = (int)lane_base + lane;
@@ -516,27 +498,26 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const int pub_row = lane / kLanesPerRow;
     const bool publisher = (lane % kLanesPerRow) == 0;
     const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(p.Nk, 1)));
-    int ne = 0, g0 = 0;                          // non-empty items so far, tiles of those items
-    int rg = 0;                                  // retained tiles of this group so far: P8^T slot 4 grp + rg % 4
-    int nt_own = 0;                              // tiles of this group so far (phase of its decision barrier)
-    uint32_t xc = 0;                             // exchanges of this group so far (buffer and barrier phase xc & 1)
+    int ne = 0, g = 0;                           // items and tiles of this stream so far
+    int rg = 0;                                  // retained tiles so far: P8^T slot rg % PP
+    uint32_t xc = 0;                             // exchanges so far (buffer and barrier phase xc & 1)
     bool ok = true;
     // one value per (warp, row) to all threads of the group
     auto exchange = [&](float mine, float (&a0)[GH], float (&a1)[GH], float (&a2)[GH], float (&a3)[GH]) -> bool {
       const int xb = xc & 1;
-      if (publisher) xch[grp][xb][w][pub_row] = mine;
+      if (publisher) xch[k][xb][w][pub_row] = mine;
       __syncwarp();
-      if (lane == 0) mbar_arrive(&grp_bar[grp]);
-      bool k = mbar_wait(&grp_bar[grp], xc & 1, status);
-      k = __all_sync(0xffffffffu, k);
+      if (lane == 0) mbar_arrive(&grp_bar[k]);
+      bool kk = mbar_wait(&grp_bar[k], xc & 1, status);
+      kk = __all_sync(0xffffffffu, kk);
       ++xc;
-      if (!k) return false;
-      lds_row<GH>(xch[grp][xb][0], a0); lds_row<GH>(xch[grp][xb][1], a1);
-      lds_row<GH>(xch[grp][xb][2], a2); lds_row<GH>(xch[grp][xb][3], a3);
+      if (!kk) return false;
+      lds_row<GH>(xch[k][xb][0], a0); lds_row<GH>(xch[k][xb][1], a1);
+      lds_row<GH>(xch[k][xb][2], a2); lds_row<GH>(xch[k][xb][3], a3);
       return true;
     };
-    // scales of the tile this group takes next (requested while the one before it is processed; loaded straight
-    // into the registers they are used from)
+    // scales of the tile after this one (requested while this one is processed; loaded straight into the registers
+    // they are used from -- a copy would wait for the load at once)
     auto ld_scale = [&](const float* base, int idx) -> float {
       float v;
       asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(base + idx));
@@ -544,154 +525,99 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     };
     float ks_nx = 1.f, vs_nx = 1.f;
     bool first = true;
-    for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-      int b, hkv, split, T, j0;
-      geometry(item, b, hkv, split, T, j0);
-      const size_t stat_row = (size_t)(b * p.Hkv + hkv) * p.num_splits + split;
+    for (int item = item0; item < p.n_items && ok; item += item_step) {
+      const int T = tiles_of(item);
       if (T == 0) continue;
+      int b, hkv, split, j0;
+      geometry(item, b, hkv, split, j0, T);
       const int ip = ne & 1;
-      const uint32_t colO = Cfg::kColO + (uint32_t)(ip * NG + grp) * 16u;
-      uint32_t* bm_row = p.bitmask ? p.bitmask + stat_row * p.words : nullptr;
-      float m_ref[GH], l[GH], yref[GH], c2q[GH], a_own[GH];
-#pragma unroll
-      for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; c2q[q] = c2; a_own[q] = -INFINITY; }
-      int r = 0;                                 // tiles of the item this group has retained
-      bool have_q = false, have_slot = false;
-      for (int t = (grp + NG - g0 % NG) % NG; t < T; t += NG) {
-        const int g = g0 + t;
-        if (first) {
-          ks_nx = ld_scale(p.kscale, scale_index(b, hkv, j0 - t));
-          vs_nx = ld_scale(p.vscale, scale_index(b, hkv, j0 - t));
-          first = false;
+      const uint32_t colO = colO0 + (uint32_t)ip * 16u;
+      uint32_t* bm_row = p.bitmask ? p.bitmask + ((size_t)(b * p.Hkv + hkv) * p.num_splits + split) * p.words : nullptr;
+      // the first tile of the stream's next non-empty item (for the look-ahead at this item's last tile)
+      int nidx = -1;
+      for (int it2 = item + item_step; it2 < p.n_items; it2 += item_step) {
+        const int T2 = tiles_of(it2);
+        if (T2 > 0) {
+          int b2, h2, s2, j2;
+          geometry(it2, b2, h2, s2, j2, T2);
+          nidx = scale_index(b2, h2, j2);
+          break;
         }
+      }
+      if (first) {
+        ks_nx = ld_scale(p.kscale, scale_index(b, hkv, j0));
+        vs_nx = ld_scale(p.vscale, scale_index(b, hkv, j0));
+        first = false;
+      }
+      int r = 0;                                 // tiles of the item retained so far
+      float m_ref[GH], l[GH], yref[GH], lgl[GH], c2q[GH];
+#pragma unroll
+      for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; lgl[q] = -INFINITY; c2q[q] = c2; }
+      for (int t = 0; t < T; ++t, ++g) {
         const float ks = ks_nx, lv = __log2f(vs_nx);
-        if (t + NG < T) {
-          ks_nx = ld_scale(p.kscale, scale_index(b, hkv, j0 - t - NG));
-          vs_nx = ld_scale(p.vscale, scale_index(b, hkv, j0 - t - NG));
-        } else {   // the group's first tile in the next item that has one
-          int g0n = g0 + T;
-          for (int it2 = item + gridDim.x; it2 < p.n_items; it2 += gridDim.x) {
-            int b2, h2, s2, T2, j2;
-            geometry(it2, b2, h2, s2, T2, j2);
-            const int t2 = (grp + NG - g0n % NG) % NG;
-            if (t2 < T2) {
-              ks_nx = ld_scale(p.kscale, scale_index(b2, h2, j2 - t2));
-              vs_nx = ld_scale(p.vscale, scale_index(b2, h2, j2 - t2));
-              break;
-            }
-            g0n += T2;
-          }
+        if (t + 1 < T) {
+          ks_nx = ld_scale(p.kscale, scale_index(b, hkv, j0 - t - 1));
+          vs_nx = ld_scale(p.vscale, scale_index(b, hkv, j0 - t - 1));
+        } else if (nidx >= 0) {
+          ks_nx = ld_scale(p.kscale, nidx);
+          vs_nx = ld_scale(p.vscale, nidx);
         }
         const int sb = g & 3;
-        ok = mbar_wait(&s_full[sb], (uint32_t)((g >> 2) & 1), status);
+        ok = mbar_wait(&s_full[k][sb], (uint32_t)((g >> 2) & 1), status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
         uint32_t sr[LDN];
-        tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, (uint32_t)sb * 16u), sr);
+        tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colS + (uint32_t)sb * 16u), sr);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&s_free[sb]);
-        if (!have_q) {
+        if (lane == 0) mbar_arrive(&s_free[k][sb]);
+        if (t == 0) {
 #pragma unroll
-          for (int q = 0; q < GH; ++q) c2q[q] = c2 * *(volatile float*)&q_inv[ne & 7][q];
-          have_q = true;
+          for (int q = 0; q < GH; ++q) c2q[q] = c2 * *(volatile float*)&q_inv[k][ip][q];
         }
         const int kpos = (j0 - t) * 128 + kt;
-        float x[GH], tmax[GH], psum[GH];
-#pragma unroll
-        for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
-          x[q] = (kpos < p.Nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
-          psum[q] = 0.f;
-        }
-        const int ps = PP * grp + (rg % PP);
-        // P8^T of this tile into slot ps against the group's references; e[] = the unrounded exp2(x - m)
-        auto store_p = [&](float (&e)[GH]) -> bool {
-          if (rg >= PP) {
-            bool k = mbar_wait(&p_free[ps], (uint32_t)(((rg / PP) - 1) & 1), status);
-            k = __all_sync(0xffffffffu, k);
-            if (!k) return false;
-          }
-          float pp[GH];
-#pragma unroll
-          for (int q = 0; q < GH; ++q) {
-            e[q] = (q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
-            // P' = 64 exp2(x + lv - yref) = e * 64 exp2(m + lv - yref): the tile's V scale rides on the probability
-            pp[q] = (q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
-          }
-          uint8_t* dst = sP + ps * Cfg::kP8Bytes;
-          const uint32_t chunk = (uint32_t)kt >> 4, within = (uint32_t)kt & 15u;
-          if constexpr (GH == 1) {
-            const uint2 s0 = split_e4m3x2(pp[0], 0.f);
-            dst[0 * 128 + ((chunk ^ 0u) << 4) + within] = (uint8_t)s0.x;
-            dst[4 * 128 + ((chunk ^ 4u) << 4) + within] = (uint8_t)s0.y;
-          } else {
-#pragma unroll
-            for (int q = 0; q < GH; q += 2) {
-              const uint2 s01 = split_e4m3x2(pp[q], pp[q + 1]);
-              dst[(q + 0) * 128 + ((chunk ^ (uint32_t)(q + 0)) << 4) + within] = (uint8_t)s01.x;
-              dst[(q + 1) * 128 + ((chunk ^ (uint32_t)(q + 1)) << 4) + within] = (uint8_t)(s01.x >> 8);
-              dst[(q + 4) * 128 + ((chunk ^ (uint32_t)(q + 4)) << 4) + within] = (uint8_t)s01.y;
-              dst[(q + 5) * 128 + ((chunk ^ (uint32_t)(q + 5)) << 4) + within] = (uint8_t)(s01.y >> 8);
-            }
-          }
-          fence_proxy_async_smem();
-          return true;
-        };
-        // ... and its row sums over the group
-        auto probabilities = [&]() -> bool {
-          float e[GH], a0[GH], a1[GH], a2[GH], a3[GH];
-          if (!store_p(e)) return false;
-          RowReduce<GH, 16, false>::run(e, lane);
-          if (!exchange(e[0], a0, a1, a2, a3)) return false;
-#pragma unroll
-          for (int q = 0; q < GH; ++q) psum[q] = (a0[q] + a1[q]) + (a2[q] + a3[q]);
-          return true;
-        };
-        // The row maxima first; then the probabilities against the group's references, ahead of the decision, unless
-        // a maximum is too far above a reference (they are then formed on the slow path, after the decision).
-        bool fast = true;
+        float x[GH], tmax[GH];
         {
           float mx[GH], a0[GH], a1[GH], a2[GH], a3[GH];
 #pragma unroll
-          for (int q = 0; q < GH; ++q) mx[q] = x[q];
+          for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
+            x[q] = (kpos < p.Nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
+            mx[q] = x[q];
+          }
           RowReduce<GH, 16, true>::run(mx, lane);
           ok = exchange(mx[0], a0, a1, a2, a3);
           if (!ok) break;
 #pragma unroll
           for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
         }
+        // Eq. 3 against the split's partial normalizer: skip iff rowmax - (m + log l) < log(tau / Nk) for every head
+        bool retain = true;
+        if (!kDense && r > 0) {
+          retain = false;
+#pragma unroll
+          for (int q = 0; q < GH; ++q) retain = retain || (q < R && !(((tmax[q] - (m_ref[q] + lgl[q])) - theta) < 0.f));
+        }
+        if (!kDense && head) {
+          *(volatile int*)&flag[k][g & 3] = retain ? 1 : 0;
+          mbar_arrive(&vote_bar[k][g & 3]);
+        }
+        if (!retain) continue;
+        if (head && bm_row) atomicOr(bm_row + ((T - 1 - t) >> 5), 1u << ((T - 1 - t) & 31));
+        const int ps = rg % PP;
         if (r == 0) {
 #pragma unroll
           for (int q = 0; q < GH; ++q) { m_ref[q] = tmax[q]; yref[q] = tmax[q] + lv; }   // (nothing accumulated yet)
         } else {
-#pragma unroll
-          for (int q = 0; q < GH; ++q)
-            fast = fast && !(q < R && (tmax[q] + lv > yref[q] + kPGap || tmax[q] > m_ref[q] + kMGap));
-        }
-        if (fast) { ok = probabilities(); if (!ok) break; }
-        // ---- the turn of tile g.  Eq. 3 needs the normalizer after tile g - 1: the streams of all groups as published
-        // at their last turns.  One thread of the group (its head) takes the turn -- waits for the turn before, decides,
-        // publishes the group's new state and hands the turn on -- so that the chain from tile to tile is a few dozen
-        // instructions of one thread; the others pick the decision up behind it.
-        if (!have_slot) {   // the item's state slot is that of the item two before, which has to have been written out
-          if (ne >= 2) {
-            ok = mbar_wait(&o_free[ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-          }
-          have_slot = true;
-        }
-        // raises the references to this tile's maxima: l follows here, this group's O^T (whose earlier PVs have to be
-        // complete) in TMEM; then the probabilities against the new references
-        auto slow_probabilities = [&]() -> bool {
+          // a maximum too far above a reference: the reference is raised, l follows here and O^T (whose earlier PVs
+          // have to be complete) in TMEM
           float alpha[GH];
           bool touch = false;
 #pragma unroll
           for (int q = 0; q < GH; ++q) {
             alpha[q] = 1.f;
-            if (q < R) {
+            if (q < R && (tmax[q] + lv > yref[q] + kPGap || tmax[q] > m_ref[q] + kMGap)) {
               const float mn = fmaxf(m_ref[q], tmax[q]), yn = fmaxf(yref[q], tmax[q] + lv);
               l[q] *= fast_exp2(m_ref[q] - mn);
               alpha[q] = fast_exp2(yref[q] - yn);
@@ -701,9 +627,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             }
           }
           if (touch) {
-            bool k = mbar_wait(&p_free[PP * grp + ((rg - 1) % PP)], (uint32_t)(((rg - 1) / PP) & 1), status);
-            k = __all_sync(0xffffffffu, k);
-            if (!k) return false;
+            ok = mbar_wait(&p_free[k][(rg - 1) % PP], (uint32_t)(((rg - 1) / PP) & 1), status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
             tc_fence_after();
             uint32_t o[LDN];
             tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colO), o);
@@ -717,108 +643,68 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             tmem_wait_st();
             tc_fence_before();
           }
-          return probabilities();
-        };
-        // the group's state after this tile, for the other groups' turns and the write-out
-        auto publish = [&](int r_new) {
-#pragma unroll
-          for (int q = 0; q < GH; ++q) { st_m[ip][grp][q] = m_ref[q]; st_l[ip][grp][q] = l[q]; st_y[ip][grp][q] = yref[q]; }
-          *(volatile int*)&st_r[ip][grp] = r_new;
-        };
-        bool retain = true;
-        if (kDense) {
-          // no decision to take, hence no order between the groups: the state only serves the write-out
-          if (!fast) { ok = slow_probabilities(); if (!ok) break; }
-#pragma unroll
-          for (int q = 0; q < GH; ++q) l[q] += psum[q];
-          ++r;
-          if (head) publish(r);
-        } else {
-          bool handed_on = false;
-          if (head) {
-            // everything that does not need the other groups is ready before the wait: this stream's log-sum-exp
-            // before the tile (a_own) and after it, should it be retained (psum is known on the fast path)
-            float a_ret[GH];
-#pragma unroll
-            for (int q = 0; q < GH; ++q) a_ret[q] = m_ref[q] + __log2f(l[q] + psum[q]);
-            if (g > 0) ok = mbar_wait(&turn_done[(g - 1) & 3], (uint32_t)(((g - 1) >> 2) & 1), status);
-            if (ok) {
-              if (t > 0) {
-                float lse[GH];
-#pragma unroll
-                for (int q = 0; q < GH; ++q) lse[q] = a_own[q];
-#pragma unroll
-                for (int o2 = 1; o2 < NG; ++o2) {
-                  float ao[GH];
-                  lds_row<GH>(st_a[ip][(grp + o2) % NG], ao);
-#pragma unroll
-                  for (int q = 0; q < GH; ++q) {   // log2(2^lse + 2^ao); a stream without a tile is at -inf
-                    const float M = fmaxf(lse[q], ao[q]), d = fminf(lse[q], ao[q]) - M;
-                    lse[q] = M + __log2f(1.f + fast_exp2(d));
-                  }
-                }
-                retain = false;
-#pragma unroll
-                for (int q = 0; q < GH; ++q) retain = retain || (q < R && !(((tmax[q] - lse[q]) - theta) < 0.f));
-              }
-              *(volatile int*)&flag[g & 3] = retain ? 1 : 0;
-              if (fast || !retain) {   // the stream's new log-sum-exp is known: the turn is handed on at once
-#pragma unroll
-                for (int q = 0; q < GH; ++q) st_a[ip][grp][q] = retain ? a_ret[q] : a_own[q];
-                mbar_arrive(&turn_done[g & 3]);
-                if (retain) {
-#pragma unroll
-                  for (int q = 0; q < GH; ++q) l[q] += psum[q];
-                }
-                publish(r + (retain ? 1 : 0));
-                mbar_arrive(&vote_bar[g & 3]);
-                handed_on = true;
-              }
-              mbar_arrive(&dec_bar[grp]);
-            }
-          }
-          ok = __all_sync(0xffffffffu, ok);
-          if (ok && !head) ok = mbar_wait(&dec_bar[grp], (uint32_t)(nt_own & 1), status);
+        }
+        if (rg >= PP) {
+          ok = mbar_wait(&p_free[k][ps], (uint32_t)(((rg / PP) - 1) & 1), status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          retain = *(volatile int*)&flag[g & 3] != 0;
-          if (retain && !fast) {   // (every thread of the group; the head keeps the turn until the state is known)
-            ok = slow_probabilities();
-            if (!ok) break;
-          }
-          if (retain) {
-            if (!(head && handed_on)) {
+        }
+        float e[GH], pp[GH];
 #pragma unroll
-              for (int q = 0; q < GH; ++q) l[q] += psum[q];
-            }
-            ++r;
-          }
-          // this stream's log-sum-exp after the tile (all threads keep it; the head's copy is the one that is used)
-          if (retain) {
+        for (int q = 0; q < GH; ++q) {
+          e[q] = (q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
+          // P' = 64 exp2(x + lv - yref) = e * 64 exp2(m + lv - yref): the tile's V scale rides on the probability
+          pp[q] = (q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
+        }
+        uint8_t* dst = sP + ps * Cfg::kP8Bytes;
+        const uint32_t chunk = (uint32_t)kt >> 4, within = (uint32_t)kt & 15u;
+        if constexpr (GH == 1) {
+          const uint2 s0 = split_e4m3x2(pp[0], 0.f);
+          dst[0 * 128 + ((chunk ^ 0u) << 4) + within] = (uint8_t)s0.x;
+          dst[4 * 128 + ((chunk ^ 4u) << 4) + within] = (uint8_t)s0.y;
+        } else {
 #pragma unroll
-            for (int q = 0; q < GH; ++q) a_own[q] = m_ref[q] + __log2f(l[q]);
-          }
-          if (head && !handed_on) {
-#pragma unroll
-            for (int q = 0; q < GH; ++q) st_a[ip][grp][q] = a_own[q];
-            mbar_arrive(&turn_done[g & 3]);
-            publish(r);
-            mbar_arrive(&vote_bar[g & 3]);
+          for (int q = 0; q < GH; q += 2) {
+            const uint2 s01 = split_e4m3x2(pp[q], pp[q + 1]);
+            dst[(q + 0) * 128 + ((chunk ^ (uint32_t)(q + 0)) << 4) + within] = (uint8_t)s01.x;
+            dst[(q + 1) * 128 + ((chunk ^ (uint32_t)(q + 1)) << 4) + within] = (uint8_t)(s01.x >> 8);
+            dst[(q + 4) * 128 + ((chunk ^ (uint32_t)(q + 4)) << 4) + within] = (uint8_t)s01.y;
+            dst[(q + 5) * 128 + ((chunk ^ (uint32_t)(q + 5)) << 4) + within] = (uint8_t)(s01.y >> 8);
           }
         }
-        ++nt_own;
-        if (head && retain && bm_row) atomicOr(bm_row + ((T - 1 - t) >> 5), 1u << ((T - 1 - t) & 31));
-        // (the state was published before the tile's P8^T is handed on: the PV, the item's completion and its write-out
-        // follow from the arrivals below)
+        fence_proxy_async_smem();
         __syncwarp();
-        if (retain) {
-          ++rg;
-          if (lane == 0) mbar_arrive(&p_full[ps]);
+        if (lane == 0) mbar_arrive(&p_full[k][ps]);
+        {
+          float a0[GH], a1[GH], a2[GH], a3[GH];
+          RowReduce<GH, 16, false>::run(e, lane);
+          ok = exchange(e[0], a0, a1, a2, a3);
+          if (!ok) break;
+#pragma unroll
+          for (int q = 0; q < GH; ++q) {
+            l[q] += (a0[q] + a1[q]) + (a2[q] + a3[q]);
+            lgl[q] = __log2f(l[q]);
+          }
         }
+        ++r;
+        ++rg;
       }
       if (!ok) break;
+      // The item's state for its write-out; the slot is that of the stream's item two before, which has to have been
+      // written out.  Only the thread that writes the state waits for that: the write-out of THIS item, which follows
+      // the arrival below, completes the same barrier again, and a thread that looked at it only then would take the
+      // phase it waits for to be still outstanding.
+      if (head) {
+        if (ne >= 2) ok = mbar_wait(&o_free[k][ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
+        if (ok) {
+#pragma unroll
+          for (int q = 0; q < GH; ++q) { st_m[k][ip][q] = m_ref[q]; st_l[k][ip][q] = l[q]; st_y[k][ip][q] = yref[q]; }
+          *(volatile int*)&st_r[k][ip] = r;
+          mbar_arrive(&st_full[k][ip]);
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);
       ++ne;
-      g0 += T;
     }
   }
 
