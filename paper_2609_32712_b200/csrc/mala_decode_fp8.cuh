@@ -207,18 +207,21 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   tc_fence_after();
   const uint32_t tb = tmem_base_s;
 
-  // tiles, sequence, KV head, split and newest tile of a work item
+  // Tiles, sequence, KV head, split and newest tile of a work item.  The KV head is the fastest index of an item's
+  // number: the CTAs that run side by side then read the same keys of a key-major cache, each its own head's 128
+  // bytes of every key's row, and the row is fetched from memory once, not once per head.
   auto tiles_of = [&](int item) -> int {
-    const int split = item - (int)p.by_splits.div((uint32_t)item) * p.num_splits;
+    const int bs = (int)p.by_hkv.div((uint32_t)item);
+    const int split = bs - (int)p.by_splits.div((uint32_t)bs) * p.num_splits;
     const int lo = split * p.tps * 128;
     const int hi = min(p.Nk, lo + p.tps * 128);
     return hi > lo ? (hi - lo + 127) >> 7 : 0;
   };
   auto geometry = [&](int item, int& b, int& hkv, int& split, int& j0, int T) {
-    const int bh = (int)p.by_splits.div((uint32_t)item);
-    split = item - bh * p.num_splits;
-    b = (int)p.by_hkv.div((uint32_t)bh);
-    hkv = bh - b * p.Hkv;
+    const int bs = (int)p.by_hkv.div((uint32_t)item);
+    hkv = item - bs * p.Hkv;
+    b = (int)p.by_splits.div((uint32_t)bs);
+    split = bs - b * p.num_splits;
     j0 = split * p.tps + T - 1;
   };
   auto scale_index = [&](int b, int hkv, int jt) -> int { return (b * p.Hkv + hkv) * p.nt + jt; };
