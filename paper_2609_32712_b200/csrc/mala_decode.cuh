@@ -50,7 +50,7 @@ inline bool decode_set_attributes() {
 #define MALA_DEC_ATTR_GP(GP) MALA_DEC_ATTR(false, GP, false) MALA_DEC_ATTR(true, GP, false) MALA_DEC_ATTR(false, GP, true) MALA_DEC_ATTR(true, GP, true)
   MALA_DEC_ATTR_GP(1) MALA_DEC_ATTR_GP(2) MALA_DEC_ATTR_GP(4) MALA_DEC_ATTR_GP(8) MALA_DEC_ATTR_GP(16)
 #define MALA_F8_ATTR(DENSE, GP) \
-  ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess;
   MALA_F8_ATTR(false, 1) MALA_F8_ATTR(true, 1) MALA_F8_ATTR(false, 2) MALA_F8_ATTR(true, 2) MALA_F8_ATTR(false, 4) MALA_F8_ATTR(true, 4)
 #undef MALA_F8_ATTR
 #undef MALA_DEC_ATTR_GP
@@ -193,7 +193,7 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return MALA_ERR_CUDA;
   const int grid = p.n_items < sms ? p.n_items : sms;
-#define MALA_F8_LAUNCH(DENSE, GP) mala_decode_fp8_kernel<DENSE, GP><<<grid, DecF8Cfg<2>::kThreads, DecF8Cfg<2>::kSmemBytes, stream>>>(tq, tk, tv, p)
+#define MALA_F8_LAUNCH(DENSE, GP) mala_decode_fp8_kernel<DENSE, GP><<<grid, DecF8Cfg<2, DENSE>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p)
   const bool dense = (tau == 0.f);
   if (G <= 1) { if (dense) MALA_F8_LAUNCH(true, 1); else MALA_F8_LAUNCH(false, 1); }
   else if (G <= 2) { if (dense) MALA_F8_LAUNCH(true, 2); else MALA_F8_LAUNCH(false, 2); }

@@ -85,17 +85,20 @@ struct DecF8Params {
   FastDiv by_splits, by_hkv;
 };
 
-// NG_: streams
-template <int NG_>
+// NG_: streams (two: a third, with the registers moved from the issuing warps to the softmax groups and rings of two
+// stages, gained the MALA kernel 4% and the dense kernel nothing).  kDense_: the dense kernel requests V with K and splits a stream's six stages evenly; the MALA kernel
+// requests V only after a tile's vote, a memory latency before its PV, and gives the V ring the larger share.
+template <int NG_, bool kDense_>
 struct DecF8Cfg {
   static constexpr int kRawBytes = 128 * 128;            // one e4m3 tile
   static constexpr int kGroups = NG_;
-  static constexpr int kStages = 6 / NG_;                // raw K ring, raw V ring of a stream
+  static constexpr int kKStages = kDense_ ? 3 : 2;       // raw K ring of a stream
+  static constexpr int kVStages = kDense_ ? 3 : 4;       // raw V ring
   static constexpr int kQBytes = 1024;                   // landing buffer of an item's queries as copied: 4 rows x 128 bf16
   static constexpr int kQ8Bytes = 2048;                  // 16 rows x 128 e4m3, one per item parity
   static constexpr int kP8Bytes = 2048;                  // 16 rows x 128 e4m3
   static constexpr int kPPerGroup = 4;                   // P8^T slots of a stream: how far its softmax group may run ahead of its PVs
-  static constexpr int kStreamBytes = 2 * kStages * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPPerGroup * kP8Bytes;
+  static constexpr int kStreamBytes = (kKStages + kVStages) * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPPerGroup * kP8Bytes;
   static constexpr int kSmemBytes = kGroups * kStreamBytes + 1024;
   static constexpr int kThreads = 32 * (4 * kGroups) + 128 * kGroups + 128;   // issuing warps, softmax groups, epilogue group
   static constexpr uint32_t kColsPerStream = 96;         // S^T ring 4 x 16, O^T 2 x 16 (item parity)
@@ -135,11 +138,12 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
 // interleaved round-robin.  pos counts the tiles of the sequence (ring slots are pos % depth).  The state is a few
 // integers and depends on tile counts only, so every role keeps its own copy in step.
 template <bool kDense, int GP, int NG_ = 2>
-__global__ void __launch_bounds__(DecF8Cfg<NG_>::kThreads, 1)
+__global__ void __launch_bounds__(DecF8Cfg<NG_, kDense>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
-  using Cfg = DecF8Cfg<NG_>;
-  constexpr int RB = Cfg::kRawBytes, NS = Cfg::kStages, NG = Cfg::kGroups, PP = Cfg::kPPerGroup;
+  using Cfg = DecF8Cfg<NG_, kDense>;
+  constexpr int RB = Cfg::kRawBytes, NK = Cfg::kKStages, NV = Cfg::kVStages, NG = Cfg::kGroups, PP = Cfg::kPPerGroup;
+  static_assert(!kDense || NK == NV, "the dense producer walks both rings with one index");
   constexpr int GH = GP;                   // rows of a softmax group
   constexpr int LDN = 8;                   // S^T / O^T columns a thread reads (leading parts 0..3, remainders 4..7)
   constexpr float kPScale = 64.f;          // P' of the key that sets the reference
@@ -149,8 +153,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   // per stream
-  __shared__ uint64_t qr_full[NG][2], qr_free[NG][2], q8_free[NG][2], kr_full[NG][NS], kr_empty[NG][NS], v_full[NG][NS],
-      v_empty[NG][NS], s_full[NG][4], s_free[NG][4], vote_bar[NG][4], vote_read[NG][4], p_full[NG][PP], p_free[NG][PP],
+  __shared__ uint64_t qr_full[NG][2], qr_free[NG][2], q8_free[NG][2], kr_full[NG][NK], kr_empty[NG][NK], v_full[NG][NV],
+      v_empty[NG][NV], s_full[NG][4], s_free[NG][4], vote_bar[NG][4], vote_read[NG][4], p_full[NG][PP], p_free[NG][PP],
       item_done[NG][2], st_full[NG][2], o_free[NG][2], grp_bar[NG], ret_full[NG][8], ret_free[NG][8], fin_bar[NG];
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[NG][4];
@@ -168,12 +172,12 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
   // the stream's part of shared memory
   auto stream_base = [&](int k) -> uint8_t* { return smem + k * Cfg::kStreamBytes; };
-  // [NS] raw K | [NS] raw V | [2] Q8 (item parity) | [PP] P8^T | [2] Q landing buffers
+  // [NK] raw K | [NV] raw V | [2] Q8 (item parity) | [PP] P8^T | [2] Q landing buffers
   auto sKr_of = [&](int k) -> uint8_t* { return stream_base(k); };
-  auto sVr_of = [&](int k) -> uint8_t* { return stream_base(k) + NS * RB; };
-  auto sQ8_of = [&](int k) -> uint8_t* { return stream_base(k) + 2 * NS * RB; };
-  auto sP_of = [&](int k) -> uint8_t* { return stream_base(k) + 2 * NS * RB + 2 * Cfg::kQ8Bytes; };
-  auto sQ_of = [&](int k) -> uint8_t* { return stream_base(k) + 2 * NS * RB + 2 * Cfg::kQ8Bytes + PP * Cfg::kP8Bytes; };
+  auto sVr_of = [&](int k) -> uint8_t* { return stream_base(k) + NK * RB; };
+  auto sQ8_of = [&](int k) -> uint8_t* { return stream_base(k) + (NK + NV) * RB; };
+  auto sP_of = [&](int k) -> uint8_t* { return stream_base(k) + (NK + NV) * RB + 2 * Cfg::kQ8Bytes; };
+  auto sQ_of = [&](int k) -> uint8_t* { return stream_base(k) + (NK + NV) * RB + 2 * Cfg::kQ8Bytes + PP * Cfg::kP8Bytes; };
 
   for (int k = 0; k < NG; ++k)   // Q8 and P8^T rows that are never written stay zero
     for (int i = tid; i < (2 * Cfg::kQ8Bytes + PP * Cfg::kP8Bytes) / 16; i += Cfg::kThreads)
@@ -188,9 +192,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         mbar_init(&item_done[k][i], 1); mbar_init(&st_full[k][i], 1); mbar_init(&o_free[k][i], 4);
       }
       for (int s = 0; s < PP; ++s) { mbar_init(&p_full[k][s], 4); mbar_init(&p_free[k][s], 1); }
-      for (int s = 0; s < NS; ++s) {
-        mbar_init(&kr_full[k][s], 1); mbar_init(&kr_empty[k][s], 1); mbar_init(&v_full[k][s], 1); mbar_init(&v_empty[k][s], 1);
-      }
+      for (int s = 0; s < NK; ++s) { mbar_init(&kr_full[k][s], 1); mbar_init(&kr_empty[k][s], 1); }
+      for (int s = 0; s < NV; ++s) { mbar_init(&v_full[k][s], 1); mbar_init(&v_empty[k][s], 1); }
       for (int s = 0; s < 4; ++s) {
         mbar_init(&s_full[k][s], 1); mbar_init(&s_free[k][s], 4); mbar_init(&vote_bar[k][s], 1); mbar_init(&vote_read[k][s], 1);
         flag[k][s] = 0;
@@ -258,8 +261,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           for (int pn = 0; pn < 2; ++pn)
             tma_load_4d(sQ + qs * Cfg::kQBytes + pn * 512, &tmQ, &qr_full[k][qs], pn * 64, hkv * G, 0, b);
           for (int t = 0; t < T && ok; ++t, ++g) {
-            const int s = g % NS;
-            const uint32_t ph = (uint32_t)((g / NS) & 1);
+            const int s = g % NK;
+            const uint32_t ph = (uint32_t)((g / NK) & 1);
             ok = mbar_wait(&kr_empty[k][s], ph ^ 1u, status);
             if (!ok) break;
             mbar_arrive_expect_tx(&kr_full[k][s], RB);
@@ -316,13 +319,13 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (leader) mbar_arrive(&qr_free[k][ip]);
         const uint64_t dQ = desc_advance(dQ0, ip * Cfg::kQ8Bytes);
         for (int t = 0; t < T && ok; ++t, ++g) {
-          const int sb = g & 3, kc = g % NS;
+          const int sb = g & 3, kc = g % NK;
           if (g >= 4) {
             ok = mbar_wait_warp(&s_free[k][sb], (uint32_t)(((g >> 2) - 1) & 1), status);
             // (the vote of the tile that had this slot has been read: its flag may be overwritten)
             if (!kDense && ok) ok = mbar_wait_warp(&vote_read[k][sb], (uint32_t)(((g >> 2) - 1) & 1), status);
           }
-          if (ok) ok = mbar_wait_warp(&kr_full[k][kc], (uint32_t)((g / NS) & 1), status);
+          if (ok) ok = mbar_wait_warp(&kr_full[k][kc], (uint32_t)((g / NK) & 1), status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t dS = tS + (uint32_t)sb * 16u;
@@ -342,7 +345,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     } else if (job == 2) {
       // ---- the votes (MALA kernel): a retained tile's raw V copy is requested, the decision is passed on
       if (!kDense) {
-        int g = 0, nv = 0;                       // tiles so far; raw V copies requested -- ring slot nv % NS
+        int g = 0, nv = 0;                       // tiles so far; raw V copies requested -- ring slot nv % NV
         for (int item = item0; item < p.n_items && ok; item += item_step) {
           const int T = tiles_of(item);
           if (T == 0) continue;
@@ -356,8 +359,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             __syncwarp();
             if (leader) mbar_arrive(&vote_read[k][g & 3]);
             if (retain) {
-              const int vs = nv % NS;
-              if (nv >= NS) ok = mbar_wait_warp(&v_empty[k][vs], (uint32_t)(((nv / NS) - 1) & 1), status);
+              const int vs = nv % NV;
+              if (nv >= NV) ok = mbar_wait_warp(&v_empty[k][vs], (uint32_t)(((nv / NV) - 1) & 1), status);
               if (!ok) break;
               if (leader) {
                 mbar_arrive_expect_tx(&v_full[k][vs], RB);
@@ -378,7 +381,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       constexpr uint32_t idesc_pv = make_idesc_e4m3(128, 16, true, false);
       const uint64_t dV0 = make_smem_desc(smem_u32(sVr), 16384, 1024);   // V tile read MN-major (M = channel)
       const uint64_t dP0 = make_smem_desc(smem_u32(sP), 16, 1024);
-      int ne = 0, g = 0, npv = 0;                // items, tiles, PVs so far: raw V stage npv % NS, P8^T slot npv % PP
+      int ne = 0, g = 0, npv = 0;                // items, tiles, PVs so far: raw V stage npv % NV, P8^T slot npv % PP
       for (int item = item0; item < p.n_items && ok; item += item_step) {
         const int T = tiles_of(item);
         if (T == 0) continue;
@@ -394,9 +397,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             if (leader) mbar_arrive(&ret_free[k][g & 7]);
           }
           if (retain) {
-            const int ps = npv % PP, vc = npv % NS;
+            const int ps = npv % PP, vc = npv % NV;
             ok = mbar_wait_warp(&p_full[k][ps], (uint32_t)((npv / PP) & 1), status);
-            if (ok) ok = mbar_wait_warp(&v_full[k][vc], (uint32_t)((npv / NS) & 1), status);
+            if (ok) ok = mbar_wait_warp(&v_full[k][vc], (uint32_t)((npv / NV) & 1), status);
             // (the accumulator is that of the item two before, which has to have been written out)
             if (ok && r_item == 0 && ne >= 2) ok = mbar_wait_warp(&o_free[k][ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
             if (!ok) break;
