@@ -160,7 +160,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __shared__ int flag[NG][4];
   __shared__ int ret_ring[NG][8];          // decision of the stream's tile g at g & 7 (vote warp -> PV warp)
   __shared__ float q_inv[NG][2][4];        // 2^-k of the query rows of a stream's item
-  __shared__ __align__(16) float xch[NG][2][4][4];         // [stream][buffer][warp][row]
+  __shared__ __align__(16) float xch[NG][2][4][8];         // [stream][buffer][warp][row maxima 0..3, row sums 4..7]
   __shared__ __align__(16) float st_m[NG][2][4], st_l[NG][2][4], st_y[NG][2][4];   // a finished item's (m, l, yref)
   __shared__ int st_r[NG][2];                              // ... and its retained tiles
   __shared__ int early_exit;
@@ -508,18 +508,35 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     int rg = 0;                                  // retained tiles so far: P8^T slot rg % PP
     uint32_t xc = 0;                             // exchanges so far (buffer and barrier phase xc & 1)
     bool ok = true;
-    // one value per (warp, row) to all threads of the group
-    auto exchange = [&](float mine, float (&a0)[GH], float (&a1)[GH], float (&a2)[GH], float (&a3)[GH]) -> bool {
+    // The one exchange of a tile between the four warps: each warp's row maxima of this tile and its row sums of
+    // the last retained tile (which the test of this tile needs in the normalizer).  Returns the maxima in tmax and
+    // adds the sums to l.
+    float psum_w = 0.f;                          // this warp's sum of row pub_row, last retained tile
+    bool pending_sum = false;
+    auto exchange = [&](float mx_w, float (&tmax)[GH], float (&l)[GH], float (&lgl)[GH]) -> bool {
       const int xb = xc & 1;
-      if (publisher) xch[k][xb][w][pub_row] = mine;
+      if (publisher) { xch[k][xb][w][pub_row] = mx_w; xch[k][xb][w][4 + pub_row] = psum_w; }
       __syncwarp();
       if (lane == 0) mbar_arrive(&grp_bar[k]);
       bool kk = mbar_wait(&grp_bar[k], xc & 1, status);
       kk = __all_sync(0xffffffffu, kk);
       ++xc;
       if (!kk) return false;
+      float a0[GH], a1[GH], a2[GH], a3[GH];
       lds_row<GH>(xch[k][xb][0], a0); lds_row<GH>(xch[k][xb][1], a1);
       lds_row<GH>(xch[k][xb][2], a2); lds_row<GH>(xch[k][xb][3], a3);
+#pragma unroll
+      for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
+      if (pending_sum) {
+        lds_row<GH>(xch[k][xb][0] + 4, a0); lds_row<GH>(xch[k][xb][1] + 4, a1);
+        lds_row<GH>(xch[k][xb][2] + 4, a2); lds_row<GH>(xch[k][xb][3] + 4, a3);
+#pragma unroll
+        for (int q = 0; q < GH; ++q) {
+          l[q] += (a0[q] + a1[q]) + (a2[q] + a3[q]);
+          lgl[q] = __log2f(l[q]);
+        }
+        pending_sum = false;
+      }
       return true;
     };
     // scales of the tile after this one (requested while this one is processed; loaded straight into the registers
@@ -586,17 +603,15 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int kpos = (j0 - t) * 128 + kt;
         float x[GH], tmax[GH];
         {
-          float mx[GH], a0[GH], a1[GH], a2[GH], a3[GH];
+          float mx[GH];
 #pragma unroll
           for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
             x[q] = (kpos < p.Nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
             mx[q] = x[q];
           }
           RowReduce<GH, 16, true>::run(mx, lane);
-          ok = exchange(mx[0], a0, a1, a2, a3);
+          ok = exchange(mx[0], tmax, l, lgl);
           if (!ok) break;
-#pragma unroll
-          for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
         }
         // Eq. 3 against the split's partial normalizer: skip iff rowmax - (m + log l) < log(tau / Nk) for every head
         bool retain = true;
@@ -681,21 +696,18 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[k][ps]);
-        {
-          float a0[GH], a1[GH], a2[GH], a3[GH];
-          RowReduce<GH, 16, false>::run(e, lane);
-          ok = exchange(e[0], a0, a1, a2, a3);
-          if (!ok) break;
-#pragma unroll
-          for (int q = 0; q < GH; ++q) {
-            l[q] += (a0[q] + a1[q]) + (a2[q] + a3[q]);
-            lgl[q] = __log2f(l[q]);
-          }
-        }
+        RowReduce<GH, 16, false>::run(e, lane);   // (the sums cross the group with the next tile's maxima)
+        psum_w = e[0];
+        pending_sum = true;
         ++r;
         ++rg;
       }
       if (!ok) break;
+      if (pending_sum) {   // the last retained tile's sums
+        float unused[GH];
+        ok = exchange(-INFINITY, unused, l, lgl);
+        if (!ok) break;
+      }
       // The item's state for its write-out; the slot is that of the stream's item two before, which has to have been
       // written out.  Only the thread that writes the state waits for that: the write-out of THIS item, which follows
       // the arrival below, completes the same barrier again, and a thread that looked at it only then would take the
