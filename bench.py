@@ -60,8 +60,8 @@ def load_peaks():
 
 
 def load_dram_traffic(workload, preset, tau):
-    """DRAM bytes of one launch of the dominant kernel on (workload, preset, tau), from the table kept beside the ncu
-    summaries it was read from (profiles/dram_traffic.txt); None where no capture exists."""
+    """DRAM bytes of the backward's main kernels for one call on (workload, preset, tau), from the table kept beside the
+    ncu summaries it was read from (profiles/dram_traffic.txt); None where no capture exists."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if not os.path.exists(path):
         return None, None
@@ -690,13 +690,16 @@ def main():
     bwd_exec = bwd_executed_flops(ts["bwd_legal"], ts["bwd_retained"], c.d)
     fwd_exec = fwd_executed_flops(ts["fwd_legal"], ts["fwd_retained"], c.d)
     ach = bwd_exec / (bwd_ms * 1e-3) / 1e12
-    # DRAM bytes of one mala_bwd_kernel launch: from the table of committed ncu captures, null where none exists
+    # DRAM bytes of the main kernels of one mala_bwd call (at tau > 0: first pass, list pass, one-pass kernel on the rows
+    # left to it): from the table of committed ncu captures, null where none exists
     traffic, traffic_src = load_dram_traffic(args.workload, args.preset, tau)
     roofline = {"bound": "tensor", "kernel": "mala_bwd_kernel", "achieved": ach, "peak": peaks["tflops_sustained"],
                 "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": traffic,
                 "traffic_source": traffic_src,
                 "peak_source": f"{peaks['source']} (bf16 matmul, sustained)",
-                "note": "duration = whole mala_bwd call (preprocess + main + dQ convert), so frac is a lower bound",
+                "note": "duration = whole mala_bwd call (preprocess + main kernels + dQ convert; at tau > 0 the main "
+                        "kernels are the first pass that tests every legal tile, the pass over its retained tiles and "
+                        "the one-pass kernel on the rows left to it), so frac is a lower bound",
                 "fwd": {"kernel": "mala_fwd_kernel", "achieved": fwd_exec / (fwd_ms * 1e-3) / 1e12,
                         "frac": fwd_exec / (fwd_ms * 1e-3) / 1e12 / peaks["tflops_sustained"]}}
 
@@ -976,7 +979,7 @@ def main():
                    "parallelism": "replicas (one head slice per GPU, no collective)" if world > 1 else "single GPU"},
         "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
         "fwd_retained_frac": ts["fwd_retained"] / ts["fwd_legal"], "bwd_retained_frac": ts["bwd_retained"] / ts["bwd_legal"],
-        "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * args.steps,   # (timed region: fwd + 3 backward kernels per step)
+        "clocks": clocks, "e2e": e2e, "gpu_launches": (6 if tau > 0 else 4) * args.steps,   # (timed region per step: fwd + preprocess, main kernel(s) -- three at tau > 0 -- and dQ convert of the backward)
         "roofline": roofline, "cpu_baseline": cpu_baseline, "detail": detail,
     }
     if tp8 is not None:
