@@ -141,3 +141,22 @@ def test_named_single_head_decode_follows_the_bf16_rounding_model(mala, oracle, 
             TD._run_and_check(mala, oracle, w, tau, c["S"], rounding_bound=True)
         else:
             TD._run_paged(mala, oracle, w, tau, c["S"], c["page"], c["lens"], seed=c["page_seed"], rounding_bound=True)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_random_cases_decode_over_an_e4m3_cache(mala, oracle, seed):
+    """Randomly drawn decode calls over an 8-bit cache: group sizes 1, 2, 4, head sizes in multiples of 16, cache lengths
+    and split counts that give work items of zero to a dozen tiles (several items per CTA, empty trailing splits),
+    every tolerance, both presets.  Outputs by the rounding model (single heads and large outputs occur)."""
+    rng = random.Random(1000 + seed)
+    for _ in range(12):
+        hkv, g = rng.choice([1, 2, 3, 5]), rng.choice([1, 2, 4])
+        d = rng.choice([16, 32, 64, 80, 96, 128])
+        B = rng.choice([1, 2, 3, 7])
+        Nk = rng.choice([rng.randint(1, 300), rng.randint(300, 3000), rng.randint(3000, 12000)])
+        S = rng.choice([1, 2, 3, 5, 8, 16, 33])
+        tau = rng.choice([0.0, 1e-5, 1e-4, 1e-2, 1.0])
+        preset = rng.choice(["literal", "D"])
+        w = W.custom_decode(B, hkv * g, hkv, Nk, d, S, seed=rng.randint(0, 10**6), preset=preset)
+        res = TD._run_fp8(mala, oracle, w, tau, S, rounding_bound=True)
+        assert res["totals"][1] == res["retained"] + res["skipped"], (B, hkv, g, d, Nk, S, tau, preset)
