@@ -378,9 +378,10 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
     } else {
       // ---- O^T += V8^T P8^T of every retained tile, into the accumulator of the item
-      constexpr uint32_t idesc_pv = make_idesc_e4m3(128, 16, true, false);
+      constexpr uint32_t idesc_pv = make_idesc_e4m3(128, 16, true, true);
       const uint64_t dV0 = make_smem_desc(smem_u32(sVr), 16384, 1024);   // V tile read MN-major (M = channel)
-      const uint64_t dP0 = make_smem_desc(smem_u32(sP), 16, 1024);
+      // P8^T read MN-major too, without swizzle: 16 bytes (the 16 columns) per key, core matrices of 8 keys 128 bytes apart
+      const uint64_t dP0 = make_smem_desc(smem_u32(sP), 128, 128) & ~((uint64_t)7 << 61);
       int ne = 0, g = 0, npv = 0;                // items, tiles, PVs so far: raw V stage npv % NV, P8^T slot npv % PP
       for (int item = item0; item < p.n_items && ok; item += item_step) {
         const int T = tiles_of(item);
@@ -409,7 +410,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             const uint32_t acc0 = r_item > 0 ? 1u : 0u;
 #pragma unroll
             for (int kq = 0; kq < 4; ++kq)     // 32 keys per instruction: 32 rows of the V tile, 32 bytes of a P8^T row
-              mma_ss_f8(dO, desc_advance(dV, kq * 4096), desc_advance(dP, kq * 32), idesc_pv, kq > 0 ? 1u : acc0, leader);
+              mma_ss_f8(dO, desc_advance(dV, kq * 4096), desc_advance(dP, kq * 512), idesc_pv, kq > 0 ? 1u : acc0, leader);
             if (leader) { tc_commit(&v_empty[k][vc]); tc_commit(&p_free[k][ps]); }
             ++npv;
             ++r_item;
@@ -677,21 +678,20 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           // P' = 64 exp2(x + lv - yref) = e * 64 exp2(m + lv - yref): the tile's V scale rides on the probability
           pp[q] = (q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
         }
-        uint8_t* dst = sP + ps * Cfg::kP8Bytes;
-        const uint32_t chunk = (uint32_t)kt >> 4, within = (uint32_t)kt & 15u;
-        if constexpr (GH == 1) {
-          const uint2 s0 = split_e4m3x2(pp[0], 0.f);
-          dst[0 * 128 + ((chunk ^ 0u) << 4) + within] = (uint8_t)s0.x;
-          dst[4 * 128 + ((chunk ^ 4u) << 4) + within] = (uint8_t)s0.y;
-        } else {
+        {   // the key's 16 bytes: leading parts of the (up to four) heads, their remainders, zeros
+          uint32_t lead = 0u, rem = 0u;
+          if constexpr (GH == 1) {
+            const uint2 s0 = split_e4m3x2(pp[0], 0.f);
+            lead = s0.x & 0xffu; rem = s0.y & 0xffu;
+          } else {
 #pragma unroll
-          for (int q = 0; q < GH; q += 2) {
-            const uint2 s01 = split_e4m3x2(pp[q], pp[q + 1]);
-            dst[(q + 0) * 128 + ((chunk ^ (uint32_t)(q + 0)) << 4) + within] = (uint8_t)s01.x;
-            dst[(q + 1) * 128 + ((chunk ^ (uint32_t)(q + 1)) << 4) + within] = (uint8_t)(s01.x >> 8);
-            dst[(q + 4) * 128 + ((chunk ^ (uint32_t)(q + 4)) << 4) + within] = (uint8_t)s01.y;
-            dst[(q + 5) * 128 + ((chunk ^ (uint32_t)(q + 5)) << 4) + within] = (uint8_t)(s01.y >> 8);
+            for (int q = 0; q < GH; q += 2) {
+              const uint2 s01 = split_e4m3x2(pp[q], pp[q + 1]);
+              lead |= (s01.x & 0xffffu) << (8 * q);
+              rem |= (s01.y & 0xffffu) << (8 * q);
+            }
           }
+          *reinterpret_cast<uint4*>(sP + ps * Cfg::kP8Bytes + kt * 16) = make_uint4(lead, rem, 0u, 0u);
         }
         fence_proxy_async_smem();
         __syncwarp();
