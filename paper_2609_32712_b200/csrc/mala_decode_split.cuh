@@ -307,11 +307,13 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     {
       const uint32_t leader = elect_one();
       constexpr uint32_t idesc_qk = make_idesc_bf16(128, 16, false, false);
-      constexpr uint32_t idesc_pv = make_idesc_bf16(128, 16, true, false);
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, 16, true, true);
       const uint64_t dQ0 = make_smem_desc(smem_u32(sQ), 16, 1024);
       const uint64_t dK0 = make_smem_desc(smem_u32(sK), 16, 1024);
       const uint64_t dV0 = make_smem_desc(smem_u32(sV), 16384, 1024);   // V tile read MN-major (M = channel)
-      const uint64_t dP0 = make_smem_desc(smem_u32(sP), 16, 1024);
+      // P^T is read MN-major without swizzle: per key the 16 rows as two 16-byte halves, each half of the tile a plane
+      // of 8-key core matrices 128 bytes apart (so that a softmax thread writes its key's values as one vector store)
+      const uint64_t dP0 = make_smem_desc(smem_u32(sP), 128, 2048) & ~((uint64_t)7 << 61);
       // cursor over (non-empty item, tile) in processing order; g = global tile number
       struct Cur { int item, ne, t, T, b, hkv, j0, g; bool valid; };
       auto first_item = [&](Cur& c, int from, int ne, int g) {
@@ -417,7 +419,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             const uint32_t acc0 = r_item > 0 ? 1u : 0u;
 #pragma unroll
             for (int k = 0; k < 8; ++k)   // k-step = 16 keys: 2 KB further on in the V tile, 32 B in a P^T panel
-              mma_ss(dO, desc_advance(dV, k * 2048), desc_advance(dP, (k >> 2) * 2048 + (k & 3) * 32), idesc_pv,
+              mma_ss(dO, desc_advance(dV, k * 2048), desc_advance(dP, k * 256), idesc_pv,
                      k > 0 ? 1u : acc0, leader);
             if (leader) { tc_commit(&v_empty[vc]); tc_commit(&p_free[ps]); }
             if (++vc == VS) { vc = 0; vcpar ^= 1; }
@@ -668,12 +670,19 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           if (!ok) break;
         }
         {
-          uint8_t* dst = sP + ps * DecCfg::kPBytes + (kt >> 6) * 2048;
-          const uint32_t col = (uint32_t)(kt & 63);
+          // the key's GH values of this group: rows rb .. rb + GH - 1 of the 16, i.e. GH * 2 bytes of half rb / 8
+          uint8_t* dst = sP + ps * DecCfg::kPBytes + (rb >> 3) * 2048 + (kt >> 3) * 128 + (kt & 7) * 16 + (rb & 7) * 2;
 #pragma unroll
-          for (int q = 0; q < GH; ++q) {
-            x[q] = (rb + q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
-            *reinterpret_cast<__nv_bfloat16*>(dst + sw128_offset((uint32_t)(rb + q), col)) = __float2bfloat16_rn(x[q]);
+          for (int q = 0; q < GH; ++q) x[q] = (rb + q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
+          if constexpr (GH == 1) {
+            *reinterpret_cast<__nv_bfloat16*>(dst) = __float2bfloat16_rn(x[0]);
+          } else {
+            uint32_t pk[GH / 2];
+#pragma unroll
+            for (int q = 0; q < GH; q += 2) pk[q / 2] = pack_bf16x2(x[q], x[q + 1]);
+            if constexpr (GH == 2) *reinterpret_cast<uint32_t*>(dst) = pk[0];
+            else if constexpr (GH == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(pk[0], pk[1]);
+            else *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
         fence_proxy_async_smem();
