@@ -77,6 +77,24 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, i
   return __all_sync(0xffffffffu, ok);
 }
 
+// The same for a warp that shares its scheduler with warps doing arithmetic: between two tests it sleeps for a few
+// dozen nanoseconds, so that its polling does not take their issue slots.
+__device__ __forceinline__ bool mbar_wait_warp_idle(uint64_t* bar, uint32_t parity, int* status) {
+  bool ok = true;
+  if (!mbar_try_wait(bar, parity)) {
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+      __nanosleep(32);
+      if (((++it) & 0xff) == 0) {
+        if (*(volatile int*)status != 0) { ok = false; break; }
+        if (clock64() - t0 > kWaitLimitCycles) { atomicCAS(status, 0, kDevTimeout); ok = false; break; }
+      }
+    }
+  }
+  return __all_sync(0xffffffffu, ok);
+}
+
 // One lane of a converged warp (1 in that lane, 0 in the others)
 __device__ __forceinline__ uint32_t elect_one() {
   uint32_t leader;
