@@ -888,6 +888,19 @@ def main():
                                   "rel_l2_o_vs_bf16_cache": float((o8.float() - o16.float()).norm() / o16.float().norm())}
                 f8[layout] = lay
                 del ka, va
+            # ... and in 256-key pages scattered over a shuffled pool (mala_decode_fp8_paged; scales per tile of a page)
+            kp8, vp8, bt8, _ = W.paginate(k8, v8, 256, seed=7)
+            sp = lambda sc: W.paginate_scales(sc, bt8, 256)
+            ksp, vsp = sp(ks8), sp(vs8)
+            pg8 = {}
+            for label, t_ in (("mala", tau), ("dense", 0.0)):
+                us = 1e3 * time_cuda(lambda: mala.decode_fp8_paged(qd, kp8, vp8, ksp, vsp, bt8, None, wd["scale"], t_,
+                                                                    dcfg.num_splits, ws=wsd, out=od, want_lse=False), 25, 100)
+                need = f8["key_major"][label]["needed_gb"] * 1e9
+                pg8[label] = {"us": us, "achieved_gbs": need / (us * 1e-6) / 1e9,
+                              "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+            f8["paged_256"] = pg8
+            del kp8, vp8, bt8, ksp, vsp
             row["e4m3_cache"] = f8
             del k8, v8, ks8, vs8
             if preset == "D":                       # work and fidelity against the dense decode, tau up to 1

@@ -201,6 +201,21 @@ int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float*
                     mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                     float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* mala_decode_fp8 over a paged 8-bit cache with one length per sequence: the layout of mala_decode_paged (one new token
+ * per sequence) with the storage of mala_decode_fp8.  kpages8, vpages8: 8-bit [num_pages, page_size, Hkv, d] views
+ * (strides in elements = bytes, multiples of 16), page_size a multiple of 128 (MALA_ERR_UNSUPPORTED otherwise: a scale
+ * belongs to a 128-key tile of a page); kscale, vscale: device fp32 [num_pages, Hkv, page_size/128], the scale of
+ * tile y of page x at [x][h][y].  block_table, seqlens, the split layout (Nk = max_pages_per_seq*page_size), the
+ * clamping of seqlens, entries outside the pool (read as zeros) and telemetry as in mala_decode_paged; slots of a
+ * mapped page beyond the sequence's length must hold codes other than e4m3's two NaN codes, 0x7f and 0xff (a
+ * zero-initialised or recycled page does): their keys are masked out of the scores, but their values are multiplied by
+ * zero probabilities.  d, Hq/Hkv and the workspace as in mala_decode_fp8. */
+int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const float* kscale, const float* vscale,
+                          const int32_t* block_table, const int32_t* seqlens, mala_tout o, float* lse_opt,
+                          const mala_stats* st, int B, int Hq, int Hkv, int num_pages, int page_size,
+                          int max_pages_per_seq, int d, float scale, float tau, int num_splits, void* ws, size_t ws_bytes,
+                          void* cuda_stream);
+
 /* Split-KV decode of Sq new tokens per sequence at once (a verification step of speculative decoding, or a short
  * chunk).  q, o [B,Sq,Hq,d]; lse_opt fp32 [B,Sq,Hq] or NULL; kcache, vcache [B,Nk,Hkv,d] with the keys and values of
  * the Sq new tokens already in the last Sq positions.  Token s (0 = oldest) sits at position Nk - Sq + s, attends to

@@ -509,6 +509,44 @@ int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float*
                            ws, status, (cudaStream_t)cuda_stream);
 }
 
+int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const float* kscale, const float* vscale,
+                          const int32_t* block_table, const int32_t* seqlens, mala_tout o, float* lse_opt,
+                          const mala_stats* st, int B, int Hq, int Hkv, int num_pages, int page_size,
+                          int max_pages_per_seq, int d, float scale, float tau, int num_splits, void* ws, size_t ws_bytes,
+                          void* cuda_stream) {
+  if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
+  if (page_size % 128 != 0 || (long long)max_pages_per_seq * page_size > 0x7fffffffLL ||
+      (long long)num_pages * Hkv * (page_size / 128) > 0x7fffffffLL)
+    return MALA_ERR_UNSUPPORTED;
+  const int Nk = max_pages_per_seq * page_size;   // the longest cache a sequence can hold
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  if (num_splits <= 0 || !ws || !kscale || !vscale) return MALA_ERR_INVALID_ARG;
+  if (Hq / Hkv > 4 || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  if ((((uintptr_t)block_table) & 3) != 0 || (((uintptr_t)seqlens) & 3) != 0) return MALA_ERR_MISALIGNED;
+  MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
+  auto check8 = [&](const mala_tin& t) -> int {   // 8-bit views: strides in elements = bytes, multiples of 16
+    if (!t.p) return MALA_ERR_INVALID_ARG;
+    if (!aligned16(t.p)) return MALA_ERR_MISALIGNED;
+    if ((num_pages > 1 && t.sb % 16) || (page_size > 1 && t.sn % 16) || (Hkv > 1 && t.sh % 16)) return MALA_ERR_MISALIGNED;
+    if ((num_pages > 1 && t.sb <= 0) || (page_size > 1 && t.sn <= 0) || (Hkv > 1 && t.sh <= 0)) return MALA_ERR_INVALID_ARG;
+    return MALA_OK;
+  };
+  MALA_TRY(check8(kpages8));
+  MALA_TRY(check8(vpages8));
+  MALA_TRY(check_view(o.p, o.sb, 8, o.sh, B, 1, Hq));
+  if ((((uintptr_t)ws) & 255) != 0 || (((uintptr_t)kscale) & 3) != 0 || (((uintptr_t)vscale) & 3) != 0) return MALA_ERR_MISALIGNED;
+  if (ws_bytes < decode_workspace_bytes(B, Hq, 128, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  DecPaging pg;
+  pg.block_table = block_table; pg.seqlens = seqlens; pg.bt_stride = max_pages_per_seq; pg.page_size = page_size;
+  pg.num_pages = num_pages;
+  return decode_fp8_launch(q, kpages8, vpages8, kscale, vscale, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau,
+                           num_splits, ws, status, (cudaStream_t)cuda_stream, &pg);
+}
+
 int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
                       int B, int Hq, int Hkv, int Nk, int Sq, int d, float scale, float tau, int num_splits, void* ws,
                       size_t ws_bytes, void* cuda_stream) {

@@ -83,6 +83,12 @@ struct DecF8Params {
   int B, Hq, Hkv, Nk, tps, num_splits, words, n_items, nt;
   float scale_log2, log2_tau;
   FastDiv by_splits, by_hkv;
+  // paged cache (block_table != null): K / V are [num_pages, page_size, Hkv, d], the scales [num_pages, Hkv, tpp];
+  // Nk = max_pages * page_size lays out the splits, a sequence holds seqlens[b] keys (null: Nk)
+  const int32_t* block_table;    // [B, max_pages]
+  const int32_t* seqlens;        // [B] or null
+  int num_pages, max_pages, tpp; // tpp = tiles (128 keys) per page
+  FastDiv by_tpp;
 };
 
 // NG_: streams (two: a third, with the registers moved from the issuing warps to the softmax groups and rings of two
@@ -137,7 +143,11 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
 // order, each stream taking the next one when it has finished its own; the tiles of the streams' current items are
 // interleaved round-robin.  pos counts the tiles of the sequence (ring slots are pos % depth).  The state is a few
 // integers and depends on tile counts only, so every role keeps its own copy in step.
-template <bool kDense, int GP, int NG_ = 2>
+// kPaged: the cache lies in pages (block table, one length per sequence).  The tiles' coordinates and scale indices
+// then come from the producer's page lookups through a small ring, and a tile's scales reach the softmax group with
+// its scores; over a contiguous cache every role computes them itself and the softmax group requests the next
+// tile's scales a tile ahead (3 % faster than the ring there).
+template <bool kDense, int GP, bool kPaged = false, int NG_ = 2>
 __global__ void __launch_bounds__(DecF8Cfg<NG_, kDense>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
@@ -159,6 +169,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[NG][4];
   __shared__ int ret_ring[NG][8];          // decision of the stream's tile g at g & 7 (vote warp -> PV warp)
+  __shared__ int t_row[NG][8], t_outer[NG][8], t_sidx[NG][8];   // TMA coordinates and scale index of tile g (producer ->)
+  __shared__ float sc_k[NG][4], sc_v[NG][4];                    // the scales of the tile in S^T slot g & 3 (S warp -> softmax)
   __shared__ float q_inv[NG][2][4];        // 2^-k of the query rows of a stream's item
   __shared__ __align__(16) float xch[NG][2][4][8];         // [stream][buffer][warp][row maxima 0..3, row sums 4..7]
   __shared__ __align__(16) float st_m[NG][2][4], st_l[NG][2][4], st_y[NG][2][4];   // a finished item's (m, l, yref)
@@ -213,12 +225,31 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   // Tiles, sequence, KV head, split and newest tile of a work item.  The KV head is the fastest index of an item's
   // number: the CTAs that run side by side then read the same keys of a key-major cache, each its own head's 128
   // bytes of every key's row, and the row is fetched from memory once, not once per head.
+  auto keys_of = [&](int b) -> int {   // keys the sequence holds
+    return (kPaged && p.seqlens) ? min(p.Nk, max(0, __ldg(p.seqlens + b))) : p.Nk;
+  };
   auto tiles_of = [&](int item) -> int {
     const int bs = (int)p.by_hkv.div((uint32_t)item);
-    const int split = bs - (int)p.by_splits.div((uint32_t)bs) * p.num_splits;
+    const int b = (int)p.by_splits.div((uint32_t)bs);
+    const int split = bs - b * p.num_splits;
     const int lo = split * p.tps * 128;
-    const int hi = min(p.Nk, lo + p.tps * 128);
+    const int hi = min(keys_of(b), lo + p.tps * 128);
     return hi > lo ? (hi - lo + 127) >> 7 : 0;
+  };
+  // where key block jt of sequence b lies: TMA row and outer coordinate, index of its scales (-1: no such page)
+  auto tile_coord = [&](int b, int hkv, int jt, int& row, int& outer, int& sidx) {
+    if (kPaged) {
+      const int x = (int)p.by_tpp.div((uint32_t)jt);
+      const int pg = __ldg(p.block_table + (size_t)b * p.max_pages + x);
+      const int in_page = jt - x * p.tpp;
+      row = in_page * 128;
+      outer = pg;
+      sidx = (pg >= 0 && pg < p.num_pages) ? (pg * p.Hkv + hkv) * p.tpp + in_page : -1;
+    } else {
+      row = jt * 128;
+      outer = b;
+      sidx = (b * p.Hkv + hkv) * p.nt + jt;
+    }
   };
   auto geometry = [&](int item, int& b, int& hkv, int& split, int& j0, int T) {
     const int bs = (int)p.by_hkv.div((uint32_t)item);
@@ -227,7 +258,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     split = bs - b * p.num_splits;
     j0 = split * p.tps + T - 1;
   };
-  auto scale_index = [&](int b, int hkv, int jt) -> int { return (b * p.Hkv + hkv) * p.nt + jt; };
+  auto scale_index_c = [&](int b, int hkv, int jt) -> int { return (b * p.Hkv + hkv) * p.nt + jt; };   // contiguous cache
   // the CTA's work items are blockIdx.x, + gridDim.x, ..; stream k takes the k-th, (k + NG)-th, .. of them
   const int item_step = NG * (int)gridDim.x;
 
@@ -263,15 +294,20 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           for (int t = 0; t < T && ok; ++t, ++g) {
             const int s = g % NK;
             const uint32_t ph = (uint32_t)((g / NK) & 1);
+            int row, outer, sidx;
+            tile_coord(b, hkv, j0 - t, row, outer, sidx);   // (a page lookup is in flight while the slot is waited for)
             ok = mbar_wait(&kr_empty[k][s], ph ^ 1u, status);
             if (!ok) break;
+            // The S warp and the vote warp take the tile's coordinates from here; they are at most seven tiles behind
+            // (K ring, S^T ring, votes outstanding) and see the stores through the K tile's barrier.
+            if (kPaged) { t_row[k][g & 7] = row; t_outer[k][g & 7] = outer; t_sidx[k][g & 7] = sidx; }
             mbar_arrive_expect_tx(&kr_full[k][s], RB);
-            tma_load_4d(sKr + s * RB, &tmK, &kr_full[k][s], 0, (j0 - t) * 128, hkv, b);
+            tma_load_4d(sKr + s * RB, &tmK, &kr_full[k][s], 0, row, hkv, outer);
             if (kDense) {   // every tile is retained: V follows K
               ok = mbar_wait(&v_empty[k][s], ph ^ 1u, status);
               if (!ok) break;
               mbar_arrive_expect_tx(&v_full[k][s], RB);
-              tma_load_4d(sVr + s * RB, &tmV, &v_full[k][s], 0, (j0 - t) * 128, hkv, b);
+              tma_load_4d(sVr + s * RB, &tmV, &v_full[k][s], 0, row, hkv, outer);
             }
           }
           ++ne;
@@ -327,6 +363,13 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
           if (ok) ok = mbar_wait_warp(&kr_full[k][kc], (uint32_t)((g / NK) & 1), status);
           if (!ok) break;
+          if (kPaged && leader) {   // the tile's scales travel with its scores (a page without scales holds zeros: any scale does)
+            const int sidx = *(volatile int*)&t_sidx[k][g & 7];
+            sc_k[k][sb] = sidx >= 0 ? __ldg(p.kscale + sidx) : 1.f;
+            sc_v[k][sb] = sidx >= 0 ? __ldg(p.vscale + sidx) : 1.f;
+            __threadfence_block();
+          }
+          __syncwarp();
           tc_fence_after();
           const uint32_t dS = tS + (uint32_t)sb * 16u;
           const uint64_t dK = desc_advance(dK0, kc * RB);
@@ -364,7 +407,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               if (!ok) break;
               if (leader) {
                 mbar_arrive_expect_tx(&v_full[k][vs], RB);
-                tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, (j0 - t) * 128, hkv, b);
+                if (kPaged) tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, *(volatile int*)&t_row[k][g & 7], hkv,
+                                        *(volatile int*)&t_outer[k][g & 7]);
+                else tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, (j0 - t) * 128, hkv, b);
               }
               ++nv;
             }
@@ -504,7 +549,6 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     constexpr int kLanesPerRow = 32 / GH;
     const int pub_row = lane / kLanesPerRow;
     const bool publisher = (lane % kLanesPerRow) == 0;
-    const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(p.Nk, 1)));
     int ne = 0, g = 0;                           // items and tiles of this stream so far
     int rg = 0;                                  // retained tiles so far: P8^T slot rg % PP
     uint32_t xc = 0;                             // exchanges so far (buffer and barrier phase xc & 1)
@@ -557,34 +601,41 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const int ip = ne & 1;
       const uint32_t colO = colO0 + (uint32_t)ip * 16u;
       uint32_t* bm_row = p.bitmask ? p.bitmask + ((size_t)(b * p.Hkv + hkv) * p.num_splits + split) * p.words : nullptr;
-      // the first tile of the stream's next non-empty item (for the look-ahead at this item's last tile)
       int nidx = -1;
-      for (int it2 = item + item_step; it2 < p.n_items; it2 += item_step) {
-        const int T2 = tiles_of(it2);
-        if (T2 > 0) {
-          int b2, h2, s2, j2;
-          geometry(it2, b2, h2, s2, j2, T2);
-          nidx = scale_index(b2, h2, j2);
-          break;
+      if constexpr (!kPaged) {
+        // the first tile of the stream's next non-empty item (for the look-ahead at this item's last tile)
+        for (int it2 = item + item_step; it2 < p.n_items; it2 += item_step) {
+          const int T2 = tiles_of(it2);
+          if (T2 > 0) {
+            int b2, h2, s2, j2;
+            geometry(it2, b2, h2, s2, j2, T2);
+            nidx = scale_index_c(b2, h2, j2);
+            break;
+          }
+        }
+        if (first) {
+          ks_nx = ld_scale(p.kscale, scale_index_c(b, hkv, j0));
+          vs_nx = ld_scale(p.vscale, scale_index_c(b, hkv, j0));
+          first = false;
         }
       }
-      if (first) {
-        ks_nx = ld_scale(p.kscale, scale_index(b, hkv, j0));
-        vs_nx = ld_scale(p.vscale, scale_index(b, hkv, j0));
-        first = false;
-      }
+      const int nk = keys_of(b);                 // keys of the sequence: the L of Eq. 3 and the tail mask
+      const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(nk, 1)));
       int r = 0;                                 // tiles of the item retained so far
       float m_ref[GH], l[GH], yref[GH], lgl[GH], c2q[GH];
 #pragma unroll
       for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; lgl[q] = -INFINITY; c2q[q] = c2; }
       for (int t = 0; t < T; ++t, ++g) {
-        const float ks = ks_nx, lv = __log2f(vs_nx);
-        if (t + 1 < T) {
-          ks_nx = ld_scale(p.kscale, scale_index(b, hkv, j0 - t - 1));
-          vs_nx = ld_scale(p.vscale, scale_index(b, hkv, j0 - t - 1));
-        } else if (nidx >= 0) {
-          ks_nx = ld_scale(p.kscale, nidx);
-          vs_nx = ld_scale(p.vscale, nidx);
+        float ks = ks_nx, lv = 0.f;
+        if constexpr (!kPaged) {
+          lv = __log2f(vs_nx);
+          if (t + 1 < T) {
+            ks_nx = ld_scale(p.kscale, scale_index_c(b, hkv, j0 - t - 1));
+            vs_nx = ld_scale(p.vscale, scale_index_c(b, hkv, j0 - t - 1));
+          } else if (nidx >= 0) {
+            ks_nx = ld_scale(p.kscale, nidx);
+            vs_nx = ld_scale(p.vscale, nidx);
+          }
         }
         const int sb = g & 3;
         ok = mbar_wait(&s_full[k][sb], (uint32_t)((g >> 2) & 1), status);
@@ -593,6 +644,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tc_fence_after();
         uint32_t sr[LDN];
         tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colS + (uint32_t)sb * 16u), sr);
+        if constexpr (kPaged) { ks = *(volatile float*)&sc_k[k][sb]; lv = __log2f(*(volatile float*)&sc_v[k][sb]); }
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
@@ -607,7 +659,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           float mx[GH];
 #pragma unroll
           for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
-            x[q] = (kpos < p.Nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
+            x[q] = (kpos < nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
             mx[q] = x[q];
           }
           RowReduce<GH, 16, true>::run(mx, lane);

@@ -83,6 +83,9 @@ def lib():
         L.mala_decode_fp8.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp,
                                       sz, vp]
         L.mala_decode_fp8.restype = i
+        L.mala_decode_fp8_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, vp, vp, _TOut, vp, ctypes.POINTER(_Stats),
+                                            i, i, i, i, i, i, i, f, f, i, vp, sz, vp]
+        L.mala_decode_fp8_paged.restype = i
         L.mala_decode_static.argtypes = [_TIn, _TIn, _TIn, _TOut, vp, i, i, i, i, i, f, f, i, vp]
         L.mala_decode_static.restype = i
         L.mala_test_expire_wait.argtypes = [ctypes.c_longlong, vp]
@@ -404,6 +407,36 @@ def decode_fp8(q, kcache8, vcache8, kscale, vscale, scale: float, tau: float, nu
                                ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_decode_fp8")
+    return o, lse, st
+
+
+def decode_fp8_paged(q, kpages8, vpages8, kscale, vscale, block_table, seqlens, scale: float, tau: float, num_splits: int,
+                     stats: bool = False, ws=None, out=None, want_lse: bool = True):
+    """mala_decode_fp8_paged: q [B,1,Hq,d] bf16; kpages8, vpages8 e4m3 codes [num_pages, page_size, Hkv, d];
+    kscale, vscale fp32 [num_pages, Hkv, page_size/128]; block_table int32 [B, max_pages_per_seq]; seqlens int32 [B] or
+    None.  Returns (o [B,1,Hq,d] bf16, lse [B,Hq] fp32 or None, Stats or None)."""
+    B, one, Hq, d = q.shape
+    assert one == 1
+    num_pages, page_size, Hkv = kpages8.shape[0], kpages8.shape[1], kpages8.shape[2]
+    assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.shape[0] == B
+    assert seqlens is None or (seqlens.dtype == torch.int32 and seqlens.is_contiguous() and seqlens.shape == (B,))
+    for t in (kscale, vscale):
+        assert t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (num_pages, Hkv, page_size // 128)
+    max_pages = block_table.shape[1]
+    Nk = max_pages * page_size
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    tps = -(-(-(-Nk // num_splits)) // 128)
+    st = Stats((B, Hkv, num_splits), -(-tps // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_DECODE, B, Hq, Hkv, Nk, 128, num_splits), q.device) if ws is None else ws
+    rc = lib().mala_decode_fp8_paged(_view(q, _TIn), _view8(kpages8), _view8(vpages8), kscale.data_ptr(),
+                                     vscale.data_ptr(), block_table.data_ptr(),
+                                     seqlens.data_ptr() if seqlens is not None else None, _view(o, _TOut),
+                                     lse.data_ptr() if lse is not None else None, ctypes.byref(st.c) if st else None,
+                                     B, Hq, Hkv, num_pages, page_size, max_pages, d, scale, tau, num_splits,
+                                     ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_decode_fp8_paged")
     return o, lse, st
 
 

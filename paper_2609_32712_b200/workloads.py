@@ -299,6 +299,27 @@ def custom_decode(B, Hq, Hkv, Nk, d, num_splits, group_types=None, seed=0, prese
     return make_decode(cfg, preset=preset, device=device)
 
 
+def paginate_scales(scales: torch.Tensor, block_table: torch.Tensor, page_size: int, tile: int = 128):
+    """The per-tile scales [B, Hkv, nt] of a contiguous 8-bit cache in the layout of its paged copy made by
+    ``paginate`` with the same ``page_size``: [num_pages, Hkv, page_size/tile], page block_table[b][x] holding the
+    scales of tiles x*tpp .. of sequence b; pages no sequence uses get scale 1."""
+    B, Hkv, nt = scales.shape
+    tpp = page_size // tile
+    mp = block_table.shape[1]
+    pool = B * mp + 3 if int(block_table.max()) >= B * mp else int(block_table.max()) + 1
+    pool = max(pool, int(block_table[block_table < B * mp + 3].max()) + 1)
+    out = torch.ones((pool, Hkv, tpp), dtype=torch.float32, device=scales.device)
+    pad = torch.ones((B, Hkv, mp * tpp), dtype=torch.float32, device=scales.device)
+    pad[:, :, :nt] = scales
+    bt = block_table.to(scales.device).long()
+    for b in range(B):
+        for x in range(mp):
+            pg = int(bt[b, x])
+            if 0 <= pg < pool:
+                out[pg] = pad[b, :, x * tpp:(x + 1) * tpp]
+    return out
+
+
 def quantize_cache_e4m3(x: torch.Tensor, tile: int = 128):
     """8-bit storage of a KV cache [B, Nk, Hkv, d]: e4m3 values with one fp32 scale per (sequence, KV head, tile of
     128 keys), scale = largest magnitude of the tile / 448 (the largest e4m3 value).  Returns (codes uint8

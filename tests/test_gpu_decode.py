@@ -394,3 +394,94 @@ def test_decode_fp8_refuses_what_it_does_not_support(mala):
     with pytest.raises(mala.MalaError) as e:     # eight query heads per KV head
         mala.decode_fp8(w["q"].cuda(), k8.cuda(), k8.cuda(), ks.cuda(), ks.cuda(), w["scale"], 0.0, 1)
     assert e.value.code == -2
+
+
+def _run_fp8_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0):
+    """mala_decode_fp8_paged against the paged oracle on the dequantised pages: the contiguous bf16 workload is cut
+    into pages of a shuffled pool (junk in unused slots, table entries outside the pool), the pool is quantised page by
+    page (one scale per 128-key tile of a page), and the oracle is handed scale * e4m3(code)."""
+    kp, vp, bt, lens = W.paginate(w["kcache"], w["vcache"], page_size, seqlens=seqlens, seed=seed)
+    k8, ks, kd = W.quantize_cache_e4m3(kp)      # (a pool [num_pages, page_size, Hkv, d] has the shape of a cache)
+    v8, vs, vd = W.quantize_cache_e4m3(vp)
+    q = w["q"].cuda()
+    B, _, Hq, d = q.shape
+    Hkv = kp.shape[2]
+    G = Hq // Hkv
+    o, lse, st = mala.decode_fp8_paged(q, k8.cuda(), v8.cuda(), ks.cuda(), vs.cuda(), bt.cuda(),
+                                       lens.cuda() if seqlens is not None else None, w["scale"], tau, num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    ln = lens.numpy() if seqlens is not None else None
+    ref = oracle.decode_paged(w["q"][:, 0], kd, vd, bt.numpy(), ln, w["scale"], tau, num_splits, 128)
+    ref_abs = oracle.decode_paged(w["q"][:, 0], kd, vd.abs(), bt.numpy(), ln, w["scale"], tau, num_splits, 128)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy()[:, 0], lse.cpu().numpy()
+    skipped = retained = 0
+    for b in range(B):
+        n = int(lens[b])
+        for g in range(Hkv):
+            for s in range(num_splits):
+                parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                                  tau, max(n, 1), 128)
+                assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
+            hs = slice(g * G, (g + 1) * G)
+            parity.check_output(o_c[b, hs], ref["o"][b, hs], a_ref=ref_abs["o"][b, hs])
+            if n > 0:
+                assert np.abs(lse_c[b, hs] - ref["lse"][b, hs]).max() <= parity.LSE_ABS
+            else:
+                assert np.isneginf(lse_c[b, hs]).all() and (o_c[b, hs] == 0).all()
+            skipped += int((ref["mask"][b, g] == 1).sum())
+            retained += int((ref["mask"][b, g] == 2).sum())
+    tot = st.totals.cpu().numpy()
+    assert tot[1] == retained + skipped
+    return dict(skipped=skipped, retained=retained)
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv,page,lens", [
+    (1024, 4, 8, 2, 128, None),                        # one tile per page, every sequence full
+    (2048, 4, 4, 1, 256, [2048, 1000, 129]),           # two tiles per page, ragged lengths, empty trailing splits
+    (1536, 3, 4, 2, 512, [1, 1536, 0, 700]),           # a split per page; one key; no key at all
+    (8192, 64, 8, 2, 128, [8192, 5000, 128, 3333]),    # more work items than SMs, one tile each
+    (6144, 6, 4, 4, 384, [6144, 6000, 385, 3000, 17]), # three tiles per page, one head per KV head
+])
+def test_decode_fp8_paged_literal(mala, oracle, Nk, S, Hq, Hkv, page, lens, tau):
+    B = 2 if lens is None else len(lens)
+    w = W.custom_decode(B, Hq, Hkv, Nk, 128, S, seed=Nk + S + page)
+    _run_fp8_paged(mala, oracle, w, tau, S, page, lens, seed=page)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+def test_decode_fp8_paged_gated_keys_skip_value_tiles(mala, oracle, tau):
+    w = W.custom_decode(3, 8, 2, 8192, 128, 8, group_types=["diffuse", "peaked"], seed=5, preset="D")
+    res = _run_fp8_paged(mala, oracle, w, tau, 8, 256, [8192, 4096 + 77, 2500], seed=9)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+
+
+def test_decode_fp8_paged_identity_table_equals_contiguous_call(mala):
+    # pages laid out in order are the contiguous cache: both entry points must give the same bits
+    w = W.custom_decode(2, 8, 2, 4096, 128, 8, group_types=["diffuse", "peaked"], seed=21, preset="D", device="cuda")
+    k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
+    v8, vs, _ = W.quantize_cache_e4m3(w["vcache"])
+    page = 512
+    npg = 4096 // page
+    kp = k8.view(2 * npg, page, 2, 128)
+    vp = v8.view(2 * npg, page, 2, 128)
+    # scales [B, Hkv, nt] -> [num_pages, Hkv, tiles per page]
+    to_pages = lambda sc: sc.view(2, 2, npg, page // 128).permute(0, 2, 1, 3).reshape(2 * npg, 2, page // 128).contiguous()
+    bt = torch.arange(2 * npg, dtype=torch.int32, device="cuda").view(2, npg)
+    for tau in (0.0, 1e-4):
+        o0, l0, _ = mala.decode_fp8(w["q"], k8, v8, ks, vs, w["scale"], tau, 8)
+        o1, l1, _ = mala.decode_fp8_paged(w["q"], kp, vp, to_pages(ks), to_pages(vs), bt, None, w["scale"], tau, 8)
+        assert torch.equal(o0, o1) and torch.equal(l0, l1)
+
+
+def test_decode_fp8_paged_rejects_pages_that_are_not_whole_tiles(mala):
+    w = W.custom_decode(1, 4, 1, 512, 128, 1, seed=1, device="cuda")
+    k8 = torch.zeros((8, 64, 1, 128), dtype=torch.uint8, device="cuda")       # pages of 64 keys
+    sc = torch.ones((8, 1, 0), dtype=torch.float32, device="cuda")            # (no whole tile, hence no scale)
+    bt = torch.arange(8, dtype=torch.int32, device="cuda").view(1, 8)
+    with pytest.raises(mala.MalaError) as e:
+        mala.decode_fp8_paged(w["q"], k8, k8, sc, sc, bt, None, w["scale"], 0.0, 1)
+    assert e.value.code == -2
