@@ -143,10 +143,11 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
 // order, each stream taking the next one when it has finished its own; the tiles of the streams' current items are
 // interleaved round-robin.  pos counts the tiles of the sequence (ring slots are pos % depth).  The state is a few
 // integers and depends on tile counts only, so every role keeps its own copy in step.
-// kPaged: the cache lies in pages (block table, one length per sequence).  The tiles' coordinates and scale indices
-// then come from the producer's page lookups through a small ring, and a tile's scales reach the softmax group with
-// its scores; over a contiguous cache every role computes them itself and the softmax group requests the next
-// tile's scales a tile ahead (3 % faster than the ring there).
+// kPaged: the cache lies in pages (block table, one length per sequence).  In either layout the producer works out
+// where a tile lies (a page lookup if paged) and publishes its TMA coordinates and the index of its scales in a small
+// ring; the vote warp takes the V copy's coordinates from there, and the S warp loads the tile's two scales and hands
+// them to the softmax group with the scores, so that the softmax chain carries no address arithmetic and no loads
+// (with the softmax group requesting the next tile's scales itself, a tile ahead, the contiguous step was 6 % slower).
 template <bool kDense, int GP, bool kPaged = false, int NG_ = 2>
 __global__ void __launch_bounds__(DecF8Cfg<NG_, kDense>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -258,7 +259,6 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     split = bs - b * p.num_splits;
     j0 = split * p.tps + T - 1;
   };
-  auto scale_index_c = [&](int b, int hkv, int jt) -> int { return (b * p.Hkv + hkv) * p.nt + jt; };   // contiguous cache
   // the CTA's work items are blockIdx.x, + gridDim.x, ..; stream k takes the k-th, (k + NG)-th, .. of them
   const int item_step = NG * (int)gridDim.x;
 
@@ -300,7 +300,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             if (!ok) break;
             // The S warp and the vote warp take the tile's coordinates from here; they are at most seven tiles behind
             // (K ring, S^T ring, votes outstanding) and see the stores through the K tile's barrier.
-            if (kPaged) { t_row[k][g & 7] = row; t_outer[k][g & 7] = outer; t_sidx[k][g & 7] = sidx; }
+            t_row[k][g & 7] = row; t_outer[k][g & 7] = outer; t_sidx[k][g & 7] = sidx;
             mbar_arrive_expect_tx(&kr_full[k][s], RB);
             tma_load_4d(sKr + s * RB, &tmK, &kr_full[k][s], 0, row, hkv, outer);
             if (kDense) {   // every tile is retained: V follows K
@@ -363,7 +363,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
           if (ok) ok = mbar_wait_warp(&kr_full[k][kc], (uint32_t)((g / NK) & 1), status);
           if (!ok) break;
-          if (kPaged && leader) {   // the tile's scales travel with its scores (a page without scales holds zeros: any scale does)
+          if (leader) {   // the tile's scales travel with its scores (a page without scales holds zeros: any scale does)
             const int sidx = *(volatile int*)&t_sidx[k][g & 7];
             sc_k[k][sb] = sidx >= 0 ? __ldg(p.kscale + sidx) : 1.f;
             sc_v[k][sb] = sidx >= 0 ? __ldg(p.vscale + sidx) : 1.f;
@@ -407,9 +407,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               if (!ok) break;
               if (leader) {
                 mbar_arrive_expect_tx(&v_full[k][vs], RB);
-                if (kPaged) tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, *(volatile int*)&t_row[k][g & 7], hkv,
-                                        *(volatile int*)&t_outer[k][g & 7]);
-                else tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, (j0 - t) * 128, hkv, b);
+                tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, *(volatile int*)&t_row[k][g & 7], hkv,
+                            *(volatile int*)&t_outer[k][g & 7]);
               }
               ++nv;
             }
@@ -584,15 +583,6 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       return true;
     };
-    // scales of the tile after this one (requested while this one is processed; loaded straight into the registers
-    // they are used from -- a copy would wait for the load at once)
-    auto ld_scale = [&](const float* base, int idx) -> float {
-      float v;
-      asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(base + idx));
-      return v;
-    };
-    float ks_nx = 1.f, vs_nx = 1.f;
-    bool first = true;
     for (int item = item0; item < p.n_items && ok; item += item_step) {
       const int T = tiles_of(item);
       if (T == 0) continue;
@@ -601,24 +591,6 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const int ip = ne & 1;
       const uint32_t colO = colO0 + (uint32_t)ip * 16u;
       uint32_t* bm_row = p.bitmask ? p.bitmask + ((size_t)(b * p.Hkv + hkv) * p.num_splits + split) * p.words : nullptr;
-      int nidx = -1;
-      if constexpr (!kPaged) {
-        // the first tile of the stream's next non-empty item (for the look-ahead at this item's last tile)
-        for (int it2 = item + item_step; it2 < p.n_items; it2 += item_step) {
-          const int T2 = tiles_of(it2);
-          if (T2 > 0) {
-            int b2, h2, s2, j2;
-            geometry(it2, b2, h2, s2, j2, T2);
-            nidx = scale_index_c(b2, h2, j2);
-            break;
-          }
-        }
-        if (first) {
-          ks_nx = ld_scale(p.kscale, scale_index_c(b, hkv, j0));
-          vs_nx = ld_scale(p.vscale, scale_index_c(b, hkv, j0));
-          first = false;
-        }
-      }
       const int nk = keys_of(b);                 // keys of the sequence: the L of Eq. 3 and the tail mask
       const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(nk, 1)));
       int r = 0;                                 // tiles of the item retained so far
@@ -626,17 +598,6 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
       for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; lgl[q] = -INFINITY; c2q[q] = c2; }
       for (int t = 0; t < T; ++t, ++g) {
-        float ks = ks_nx, lv = 0.f;
-        if constexpr (!kPaged) {
-          lv = __log2f(vs_nx);
-          if (t + 1 < T) {
-            ks_nx = ld_scale(p.kscale, scale_index_c(b, hkv, j0 - t - 1));
-            vs_nx = ld_scale(p.vscale, scale_index_c(b, hkv, j0 - t - 1));
-          } else if (nidx >= 0) {
-            ks_nx = ld_scale(p.kscale, nidx);
-            vs_nx = ld_scale(p.vscale, nidx);
-          }
-        }
         const int sb = g & 3;
         ok = mbar_wait(&s_full[k][sb], (uint32_t)((g >> 2) & 1), status);
         ok = __all_sync(0xffffffffu, ok);
@@ -644,7 +605,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         tc_fence_after();
         uint32_t sr[LDN];
         tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colS + (uint32_t)sb * 16u), sr);
-        if constexpr (kPaged) { ks = *(volatile float*)&sc_k[k][sb]; lv = __log2f(*(volatile float*)&sc_v[k][sb]); }
+        const float ks = *(volatile float*)&sc_k[k][sb], lv = __log2f(*(volatile float*)&sc_v[k][sb]);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
