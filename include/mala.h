@@ -194,7 +194,7 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
  *     k[b, n, h, :] = kscale[b, h, n / 128] * e4m3(kcache8[b, n, h, :]),   v likewise with vscale.
  * The result is that of mala_decode on those dequantised values (the step streams half the bytes).
  * kcache8, vcache8: 8-bit [B,Nk,Hkv,d] views, strides in ELEMENTS (= bytes), multiples of 16; kscale, vscale: device
- * fp32 [B,Hkv,ceil(Nk/128)].  d a multiple of 16, at most 128; Hq/Hkv <= 4 (MALA_ERR_UNSUPPORTED otherwise).  q, o,
+ * fp32 [B,Hkv,ceil(Nk/128)].  d a multiple of 16, at most 128; Hq/Hkv <= 8 (MALA_ERR_UNSUPPORTED otherwise).  q, o,
  * lse_opt, telemetry, splits and merge as in mala_decode.
  * Workspace: mala_workspace_bytes(MALA_OP_DECODE, B, Hq, Hkv, Nk, 128, num_splits). */
 int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float* kscale, const float* vscale,

@@ -486,7 +486,7 @@ int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float*
                     float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
   if (num_splits <= 0 || !ws || !kscale || !vscale) return MALA_ERR_INVALID_ARG;
-  if (Hq / Hkv > 4 || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  if (Hq / Hkv > 8 || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
   MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
   // 8-bit views: strides in elements = bytes, multiples of 16
   auto check8 = [&](const mala_tin& t) -> int {
@@ -521,7 +521,7 @@ int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const 
   const int Nk = max_pages_per_seq * page_size;   // the longest cache a sequence can hold
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
   if (num_splits <= 0 || !ws || !kscale || !vscale) return MALA_ERR_INVALID_ARG;
-  if (Hq / Hkv > 4 || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  if (Hq / Hkv > 8 || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
   if ((((uintptr_t)block_table) & 3) != 0 || (((uintptr_t)seqlens) & 3) != 0) return MALA_ERR_MISALIGNED;
   MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
   auto check8 = [&](const mala_tin& t) -> int {   // 8-bit views: strides in elements = bytes, multiples of 16

@@ -52,6 +52,7 @@ inline bool decode_set_attributes() {
 #define MALA_F8_ATTR(DENSE, GP) \
   ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess;
   MALA_F8_ATTR(false, 1) MALA_F8_ATTR(true, 1) MALA_F8_ATTR(false, 2) MALA_F8_ATTR(true, 2) MALA_F8_ATTR(false, 4) MALA_F8_ATTR(true, 4)
+  MALA_F8_ATTR(false, 8) MALA_F8_ATTR(true, 8)
 #undef MALA_F8_ATTR
 #undef MALA_DEC_ATTR_GP
 #undef MALA_DEC_ATTR
@@ -164,7 +165,7 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
                              float tau, int num_splits, void* ws, int* status, cudaStream_t stream,
                              const DecPaging* pg = nullptr) {
   const int G = Hq / Hkv;
-  if (G > 4 || d % 16 != 0 || d > 128 || d < 16) return MALA_ERR_UNSUPPORTED;
+  if (G > 8 || d % 16 != 0 || d > 128 || d < 16) return MALA_ERR_UNSUPPORTED;
   if (pg && (pg->page_size < 128 || pg->page_size % 128 != 0)) return MALA_ERR_UNSUPPORTED;
   const int per = (Nk + num_splits - 1) / num_splits;
   const int tps = (per + 127) / 128;
@@ -211,7 +212,8 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
   const bool dense = (tau == 0.f);
   if (G <= 1) { if (dense) MALA_F8_LAUNCH(true, 1); else MALA_F8_LAUNCH(false, 1); }
   else if (G <= 2) { if (dense) MALA_F8_LAUNCH(true, 2); else MALA_F8_LAUNCH(false, 2); }
-  else { if (dense) MALA_F8_LAUNCH(true, 4); else MALA_F8_LAUNCH(false, 4); }
+  else if (G <= 4) { if (dense) MALA_F8_LAUNCH(true, 4); else MALA_F8_LAUNCH(false, 4); }
+  else { if (dense) MALA_F8_LAUNCH(true, 8); else MALA_F8_LAUNCH(false, 8); }
 #undef MALA_F8_LAUNCH
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
   decode_merge_kernel<128><<<B * Hq, 128, 0, stream>>>(p.o_part, p.lse_part, (__nv_bfloat16*)o.p, o.sb, 0, o.sh, lse_opt, 1,

@@ -100,11 +100,11 @@ struct DecF8Cfg {
   static constexpr int kGroups = NG_;
   static constexpr int kKStages = kDense_ ? 3 : 2;       // raw K ring of a stream
   static constexpr int kVStages = kDense_ ? 3 : 4;       // raw V ring
-  static constexpr int kQBytes = 1024;                   // landing buffer of an item's queries as copied: 4 rows x 128 bf16
+  static constexpr int kQBytes = 2048;                   // landing buffer of an item's queries as copied: up to 8 rows x 128 bf16
   static constexpr int kQ8Bytes = 2048;                  // 16 rows x 128 e4m3, one per item parity
   static constexpr int kP8Bytes = 2048;                  // 16 rows x 128 e4m3
   static constexpr int kPPerGroup = 4;                   // P8^T slots of a stream: how far its softmax group may run ahead of its PVs
-  static constexpr int kStreamBytes = (kKStages + kVStages) * kRawBytes + 2 * kQBytes + 2 * kQ8Bytes + kPPerGroup * kP8Bytes;
+  static constexpr int kStreamBytes = (kKStages + kVStages) * kRawBytes + kQBytes + 2 * kQ8Bytes + kPPerGroup * kP8Bytes;
   static constexpr int kSmemBytes = kGroups * kStreamBytes + 1024;
   static constexpr int kThreads = 32 * (4 * kGroups) + 128 * kGroups + 128;   // issuing warps, softmax groups, epilogue group
   static constexpr uint32_t kColsPerStream = 96;         // S^T ring 4 x 16, O^T 2 x 16 (item parity)
@@ -156,7 +156,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   constexpr int RB = Cfg::kRawBytes, NK = Cfg::kKStages, NV = Cfg::kVStages, NG = Cfg::kGroups, PP = Cfg::kPPerGroup;
   static_assert(!kDense || NK == NV, "the dense producer walks both rings with one index");
   constexpr int GH = GP;                   // rows of a softmax group
-  constexpr int LDN = 8;                   // S^T / O^T columns a thread reads (leading parts 0..3, remainders 4..7)
+  constexpr int HALF = GP > 4 ? 8 : 4;     // rows (MMA columns) of the leading parts; the remainders follow them
+  constexpr int LDN = 2 * HALF;            // S^T / O^T columns a thread reads
   constexpr float kPScale = 64.f;          // P' of the key that sets the reference
   constexpr float kPGap = 2.8f;            // log2(448 / 64), rounded down: how far y may pass yref
   constexpr float kMGap = 60.f;            // ... and x the normalizer's reference (fp32)
@@ -164,7 +165,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   // per stream
-  __shared__ uint64_t qr_full[NG][2], qr_free[NG][2], q8_free[NG][2], kr_full[NG][NK], kr_empty[NG][NK], v_full[NG][NV],
+  __shared__ uint64_t qr_full[NG], qr_free[NG], q8_free[NG][2], kr_full[NG][NK], kr_empty[NG][NK], v_full[NG][NV],
       v_empty[NG][NV], s_full[NG][4], s_free[NG][4], vote_bar[NG][4], vote_read[NG][4], p_full[NG][PP], p_free[NG][PP],
       item_done[NG][2], st_full[NG][2], o_free[NG][2], grp_bar[NG], ret_full[NG][8], ret_free[NG][8], fin_bar[NG];
   __shared__ uint32_t tmem_base_s;
@@ -172,9 +173,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __shared__ int ret_ring[NG][8];          // decision of the stream's tile g at g & 7 (vote warp -> PV warp)
   __shared__ int t_row[NG][8], t_outer[NG][8], t_sidx[NG][8];   // TMA coordinates and scale index of tile g (producer ->)
   __shared__ float sc_k[NG][4], sc_v[NG][4];                    // the scales of the tile in S^T slot g & 3 (S warp -> softmax)
-  __shared__ float q_inv[NG][2][4];        // 2^-k of the query rows of a stream's item
-  __shared__ __align__(16) float xch[NG][2][4][8];         // [stream][buffer][warp][row maxima 0..3, row sums 4..7]
-  __shared__ __align__(16) float st_m[NG][2][4], st_l[NG][2][4], st_y[NG][2][4];   // a finished item's (m, l, yref)
+  __shared__ float q_inv[NG][2][8];        // 2^-k of the query rows of a stream's item
+  __shared__ __align__(16) float xch[NG][2][4][16];        // [stream][buffer][warp][row maxima 0..7, row sums 8..15]
+  __shared__ __align__(16) float st_m[NG][2][8], st_l[NG][2][8], st_y[NG][2][8];   // a finished item's (m, l, yref)
   __shared__ int st_r[NG][2];                              // ... and its retained tiles
   __shared__ int early_exit;
 
@@ -199,9 +200,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
     for (int k = 0; k < NG; ++k) {
-      mbar_init(&grp_bar[k], 4); mbar_init(&fin_bar[k], 1);
+      mbar_init(&grp_bar[k], 4); mbar_init(&fin_bar[k], 1); mbar_init(&qr_full[k], 1); mbar_init(&qr_free[k], 1);
       for (int i = 0; i < 2; ++i) {
-        mbar_init(&qr_full[k][i], 1); mbar_init(&qr_free[k][i], 1); mbar_init(&q8_free[k][i], 1);
+        mbar_init(&q8_free[k][i], 1);
         mbar_init(&item_done[k][i], 1); mbar_init(&st_full[k][i], 1); mbar_init(&o_free[k][i], 4);
       }
       for (int s = 0; s < PP; ++s) { mbar_init(&p_full[k][s], 4); mbar_init(&p_free[k][s], 1); }
@@ -285,12 +286,12 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           if (T == 0) continue;
           int b, hkv, split, j0;
           geometry(item, b, hkv, split, j0, T);
-          const int qs = ne & 1;
-          if (ne >= 2) ok = mbar_wait(&qr_free[k][qs], (uint32_t)(((ne >> 1) - 1) & 1), status);
+          // (one landing buffer: the S warp converts an item's queries at once, long before the next item starts)
+          if (ne >= 1) ok = mbar_wait(&qr_free[k], (uint32_t)((ne - 1) & 1), status);
           if (!ok) break;
-          mbar_arrive_expect_tx(&qr_full[k][qs], (uint32_t)R * 128u * 2u);   // two panels of R rows x 128 bytes
+          mbar_arrive_expect_tx(&qr_full[k], (uint32_t)R * 128u * 2u);   // two panels of R rows x 128 bytes
           for (int pn = 0; pn < 2; ++pn)
-            tma_load_4d(sQ + qs * Cfg::kQBytes + pn * 512, &tmQ, &qr_full[k][qs], pn * 64, hkv * G, 0, b);
+            tma_load_4d(sQ + pn * HALF * 128, &tmQ, &qr_full[k], pn * 64, hkv * G, 0, b);
           for (int t = 0; t < T && ok; ++t, ++g) {
             const int s = g % NK;
             const uint32_t ph = (uint32_t)((g / NK) & 1);
@@ -324,16 +325,16 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (T == 0) continue;
         const int ip = ne & 1;
         uint8_t* q8 = sQ8 + ip * Cfg::kQ8Bytes;
-        // the item's queries have landed: row qh (128 bf16 in two 64-column panels, rows qh and 4 + qh of the
-        // landing atom; lane = four consecutive columns) becomes rows qh and 4 + qh of the e4m3 operand, once the
+        // the item's queries have landed: row qh (128 bf16 in two 64-column panels, rows qh and HALF + qh of the
+        // landing buffer; lane = four consecutive columns) becomes rows qh and HALF + qh of the e4m3 operand, once the
         // MMAs of the item that had the operand's slot before have read it
-        ok = mbar_wait_warp(&qr_full[k][ip], (uint32_t)((ne >> 1) & 1), status);
+        ok = mbar_wait_warp(&qr_full[k], (uint32_t)(ne & 1), status);
         if (ok && ne >= 2) ok = mbar_wait_warp(&q8_free[k][ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
         if (!ok) break;
         for (int qh = 0; qh < R; ++qh) {
           const int e0 = lane * 4;
-          const int prow = qh + 4 * (e0 >> 6);
-          const uint8_t* src = sQ + ip * Cfg::kQBytes + prow * 128 + (((((e0 & 63) >> 3)) ^ prow) << 4) + (e0 & 7) * 2;
+          const int prow = qh + HALF * (e0 >> 6);     // row of the landing buffer: head qh of panel e0 / 64
+          const uint8_t* src = sQ + prow * 128 + (((((e0 & 63) >> 3)) ^ (prow & 7)) << 4) + (e0 & 7) * 2;
           const uint2 w2 = *reinterpret_cast<const uint2*>(src);
           float a[4] = {__uint_as_float(w2.x << 16), __uint_as_float(w2.x & 0xffff0000u), __uint_as_float(w2.y << 16),
                         __uint_as_float(w2.y & 0xffff0000u)};
@@ -345,14 +346,14 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           const int kk = ef == 0 ? 0 : min(max(134 - ef, -100), 100);
           const float up = __uint_as_float((uint32_t)(kk + 127) << 23), down = __uint_as_float((uint32_t)(127 - kk) << 23);
           const uint2 s01 = split_e4m3x2(a[0] * up, a[1] * up), s23 = split_e4m3x2(a[2] * up, a[3] * up);
-          const int r2 = 4 + qh;
+          const int r2 = HALF + qh;
           *reinterpret_cast<uint32_t*>(q8 + qh * 128 + (((e0 >> 4) ^ (qh & 7)) << 4) + (e0 & 15)) = s01.x | (s23.x << 16);
           *reinterpret_cast<uint32_t*>(q8 + r2 * 128 + (((e0 >> 4) ^ (r2 & 7)) << 4) + (e0 & 15)) = s01.y | (s23.y << 16);
           if (lane == 0) q_inv[k][ip][qh] = down;
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (leader) mbar_arrive(&qr_free[k][ip]);
+        if (leader) mbar_arrive(&qr_free[k]);
         const uint64_t dQ = desc_advance(dQ0, ip * Cfg::kQ8Bytes);
         for (int t = 0; t < T && ok; ++t, ++g) {
           const int sb = g & 3, kc = g % NK;
@@ -522,7 +523,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
       for (int q = 0; q < GH; ++q)
         if (q < R) {   // O^T is in units of 2^yref / 64, l in units of 2^m
-          const float num = fmaf(__uint_as_float(o[4 + q]), 0.0625f, __uint_as_float(o[q])) * fast_exp2(ys[q] - ms[q]);
+          const float num = fmaf(__uint_as_float(o[HALF + q]), 0.0625f, __uint_as_float(o[q])) * fast_exp2(ys[q] - ms[q]);
           p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = num / (ls[q] * kPScale);
           if (kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = (ms[q] + __log2f(ls[q])) * 0.6931471805599453f;
         }
@@ -559,7 +560,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     bool pending_sum = false;
     auto exchange = [&](float mx_w, float (&tmax)[GH], float (&l)[GH], float (&lgl)[GH]) -> bool {
       const int xb = xc & 1;
-      if (publisher) { xch[k][xb][w][pub_row] = mx_w; xch[k][xb][w][4 + pub_row] = psum_w; }
+      if (publisher) { xch[k][xb][w][pub_row] = mx_w; xch[k][xb][w][8 + pub_row] = psum_w; }
       __syncwarp();
       if (lane == 0) mbar_arrive(&grp_bar[k]);
       bool kk = mbar_wait(&grp_bar[k], xc & 1, status);
@@ -572,8 +573,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
       for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
       if (pending_sum) {
-        lds_row<GH>(xch[k][xb][0] + 4, a0); lds_row<GH>(xch[k][xb][1] + 4, a1);
-        lds_row<GH>(xch[k][xb][2] + 4, a2); lds_row<GH>(xch[k][xb][3] + 4, a3);
+        lds_row<GH>(xch[k][xb][0] + 8, a0); lds_row<GH>(xch[k][xb][1] + 8, a1);
+        lds_row<GH>(xch[k][xb][2] + 8, a2); lds_row<GH>(xch[k][xb][3] + 8, a3);
 #pragma unroll
         for (int q = 0; q < GH; ++q) {
           l[q] += (a0[q] + a1[q]) + (a2[q] + a3[q]);
@@ -620,7 +621,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           float mx[GH];
 #pragma unroll
           for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
-            x[q] = (kpos < nk && q < R) ? fmaf(__uint_as_float(sr[4 + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
+            x[q] = (kpos < nk && q < R) ? fmaf(__uint_as_float(sr[HALF + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
             mx[q] = x[q];
           }
           RowReduce<GH, 16, true>::run(mx, lane);
@@ -672,7 +673,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 #pragma unroll
             for (int q = 0; q < GH; ++q) {
               o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
-              o[4 + q] = __float_as_uint(__uint_as_float(o[4 + q]) * alpha[q]);
+              o[HALF + q] = __float_as_uint(__uint_as_float(o[HALF + q]) * alpha[q]);
             }
             tmem_st_cols<LDN>(tmem_addr(tb, lane_base, colO), o);
             tmem_wait_st();
@@ -691,20 +692,21 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           // P' = 64 exp2(x + lv - yref) = e * 64 exp2(m + lv - yref): the tile's V scale rides on the probability
           pp[q] = (q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
         }
-        {   // the key's 16 bytes: leading parts of the (up to four) heads, their remainders, zeros
-          uint32_t lead = 0u, rem = 0u;
+        {   // the key's 16 bytes: leading parts of the heads, their remainders (zeros behind them with up to four heads)
+          uint32_t lead[2] = {0u, 0u}, rem[2] = {0u, 0u};
           if constexpr (GH == 1) {
             const uint2 s0 = split_e4m3x2(pp[0], 0.f);
-            lead = s0.x & 0xffu; rem = s0.y & 0xffu;
+            lead[0] = s0.x & 0xffu; rem[0] = s0.y & 0xffu;
           } else {
 #pragma unroll
             for (int q = 0; q < GH; q += 2) {
               const uint2 s01 = split_e4m3x2(pp[q], pp[q + 1]);
-              lead |= (s01.x & 0xffffu) << (8 * q);
-              rem |= (s01.y & 0xffffu) << (8 * q);
+              lead[q >> 2] |= (s01.x & 0xffffu) << (8 * (q & 3));
+              rem[q >> 2] |= (s01.y & 0xffffu) << (8 * (q & 3));
             }
           }
-          *reinterpret_cast<uint4*>(sP + ps * Cfg::kP8Bytes + kt * 16) = make_uint4(lead, rem, 0u, 0u);
+          *reinterpret_cast<uint4*>(sP + ps * Cfg::kP8Bytes + kt * 16) =
+              HALF == 4 ? make_uint4(lead[0], rem[0], 0u, 0u) : make_uint4(lead[0], lead[1], rem[0], rem[1]);
         }
         fence_proxy_async_smem();
         __syncwarp();

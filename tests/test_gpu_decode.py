@@ -332,16 +332,17 @@ def _run_fp8(mala, oracle, w, tau, num_splits, rounding_bound=False):
 
 @pytest.mark.parametrize("tau", [0.0, 1e-4])
 @pytest.mark.parametrize("Nk,S,Hq,Hkv,d", [(128, 1, 4, 1, 128), (1024, 4, 8, 2, 128), (1000, 3, 4, 4, 128), (4096, 8, 2, 1, 128),
-                                            (700, 8, 2, 1, 64), (2100, 5, 6, 2, 96), (8192, 64, 8, 2, 128)])
+                                            (700, 8, 2, 1, 64), (2100, 5, 6, 2, 96), (8192, 64, 8, 2, 128),
+                                            (1024, 4, 8, 1, 128), (3000, 5, 16, 2, 128), (2100, 3, 6, 1, 64), (900, 2, 14, 2, 80)])
 def test_decode_fp8_cache_literal(mala, oracle, Nk, S, Hq, Hkv, d, tau):
     w = W.custom_decode(2, Hq, Hkv, Nk, d, S, seed=Nk + S)
     _run_fp8(mala, oracle, w, tau, S)
 
 
 @pytest.mark.parametrize("tau", [1e-4, 1.0])
-@pytest.mark.parametrize("Nk,S", [(8192, 8), (5000, 4)])
-def test_decode_fp8_cache_skips_value_tiles(mala, oracle, Nk, S, tau):
-    w = W.custom_decode(2, 8, 2, Nk, 128, S, group_types=["diffuse", "peaked"], seed=3, preset="D")
+@pytest.mark.parametrize("Nk,S,Hq", [(8192, 8, 8), (5000, 4, 8), (8192, 8, 16)])
+def test_decode_fp8_cache_skips_value_tiles(mala, oracle, Nk, S, Hq, tau):
+    w = W.custom_decode(2, Hq, 2, Nk, 128, S, group_types=["diffuse", "peaked"], seed=3, preset="D")
     res = _run_fp8(mala, oracle, w, tau, S)
     assert res["skipped"] > 0, "workload must exercise skipping"
     assert res["totals"][1] == res["retained"] + res["skipped"]
@@ -389,9 +390,9 @@ def test_decode_fp8_head_major_cache_view(mala, tau):
 
 
 def test_decode_fp8_refuses_what_it_does_not_support(mala):
-    w = W.custom_decode(1, 8, 1, 256, 128, 1, seed=1)
+    w = W.custom_decode(1, 16, 1, 256, 128, 1, seed=1)
     k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
-    with pytest.raises(mala.MalaError) as e:     # eight query heads per KV head
+    with pytest.raises(mala.MalaError) as e:     # sixteen query heads per KV head
         mala.decode_fp8(w["q"].cuda(), k8.cuda(), k8.cuda(), ks.cuda(), ks.cuda(), w["scale"], 0.0, 1)
     assert e.value.code == -2
 
@@ -445,6 +446,7 @@ def _run_fp8_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0)
     (1536, 3, 4, 2, 512, [1, 1536, 0, 700]),           # a split per page; one key; no key at all
     (8192, 64, 8, 2, 128, [8192, 5000, 128, 3333]),    # more work items than SMs, one tile each
     (6144, 6, 4, 4, 384, [6144, 6000, 385, 3000, 17]), # three tiles per page, one head per KV head
+    (4096, 8, 16, 2, 256, [4096, 2049, 300]),          # eight heads per KV head
 ])
 def test_decode_fp8_paged_literal(mala, oracle, Nk, S, Hq, Hkv, page, lens, tau):
     B = 2 if lens is None else len(lens)
