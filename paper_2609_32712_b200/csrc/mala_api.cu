@@ -81,6 +81,10 @@ static int device_setup(int dev, int** status_out) {
     ok = ok && set_smem(mala_fwd_kernel<128, false, true>, FwdCfg<128, false>::kSmemBytes);
     ok = ok && set_smem(mala_fwd_kernel<64, false, true>, FwdCfg<64, false>::kSmemBytes);
     ok = ok && set_smem(mala_fwd_kernel<64, true, true>, FwdCfg<64, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<256, true>, FwdCfg<256, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<256, false>, FwdCfg<256, false>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<256, true, true>, FwdCfg<256, true>::kSmemBytes);
+    ok = ok && set_smem(mala_fwd_kernel<256, false, true>, FwdCfg<256, false>::kSmemBytes);
     ok = ok && bwd_set_attributes();
     ok = ok && decode_set_attributes();
     if (!ok) return MALA_ERR_CUDA;
@@ -102,11 +106,11 @@ static int check_view(const void* p, int64_t sb, int64_t sn, int64_t sh, int B, 
   return MALA_OK;
 }
 
-static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float tau) {
+static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float tau, int dmax = 128) {
   if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0) return MALA_ERR_INVALID_ARG;
   if (!(tau >= 0.f) || !isfinite(tau)) return MALA_ERR_INVALID_ARG;
   if (!(scale > 0.f) || !isfinite(scale)) return MALA_ERR_INVALID_ARG;
-  if (!head_size_ok(d)) return MALA_ERR_UNSUPPORTED;
+  if (!head_size_ok(d, dmax)) return MALA_ERR_UNSUPPORTED;
   if (Hq % Hkv != 0) return MALA_ERR_UNSUPPORTED;
   if (B > 65535 || Hq > 65535) return MALA_ERR_UNSUPPORTED;
   return MALA_OK;
@@ -120,11 +124,11 @@ static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float
 
 static const float kLog2e = 1.4426950408889634f;
 
-// Forward (prefill) launch: two query blocks per CTA.
+// Forward (prefill) launch: two query blocks per CTA (one with D = 256).
 template <int D, bool kDense>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                       cudaStream_t stream) {
-  dim3 grid((p.Tr + 1) / 2, p.Hq, p.B * (p.num_splits > 1 ? p.num_splits : 1));
+  dim3 grid(FwdCfg<D, kDense>::kOne ? p.Tr : (p.Tr + 1) / 2, p.Hq, p.B * (p.num_splits > 1 ? p.num_splits : 1));
   if (p.ppt > 1)
     mala_fwd_kernel<D, kDense, true><<<grid, FwdCfg<D, kDense>::kThreads, FwdCfg<D, kDense>::kSmemBytes, stream>>>(tq, tk, tv, p);
   else
@@ -179,14 +183,14 @@ int mala_decode_suggest_splits(int B, int Hkv, int Nk, int sm_count) {
 
 int mala_tile_shape(int op, int d, int* Bq, int* Bk) {
   if (!Bq || !Bk) return MALA_ERR_INVALID_ARG;
-  if (!head_size_ok(d)) return MALA_ERR_UNSUPPORTED;
+  if (!head_size_ok(d, op == MALA_OP_FWD ? 256 : 128)) return MALA_ERR_UNSUPPORTED;
   if (op == MALA_OP_FWD || op == MALA_OP_BWD) { *Bq = 128; *Bk = 128; return MALA_OK; }
   if (op == MALA_OP_DECODE) { *Bq = 0; *Bk = 128; return MALA_OK; }
   return MALA_ERR_UNSUPPORTED;
 }
 
 size_t mala_workspace_bytes(int op, int B, int Hq, int Hkv, int N, int d, int num_splits) {
-  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || !head_size_ok(d)) return 0;
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || !head_size_ok(d, op == MALA_OP_FWD ? 256 : 128)) return 0;
   const int D = padded_head_size(d);
   if (op == MALA_OP_FWD) return num_splits > 1 ? fwd_split_workspace_bytes(B, Hq, N, D, num_splits) : 256;
   if (op == MALA_OP_BWD) return bwd_workspace_bytes(B, Hq, N, D);
@@ -246,11 +250,11 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
     if (cu || num_splits > 65535 || (long long)B * num_splits > 65535) return MALA_ERR_UNSUPPORTED;
     if (!ws) return MALA_ERR_INVALID_ARG;
     if ((((uintptr_t)ws) & 255) != 0) return MALA_ERR_MISALIGNED;
-    if (B > 0 && Hq > 0 && N > 0 && head_size_ok(d) &&
+    if (B > 0 && Hq > 0 && N > 0 && head_size_ok(d, 256) &&
         ws_bytes < fwd_split_workspace_bytes(B, Hq, N, padded_head_size(d), num_splits))
       return MALA_ERR_WORKSPACE_TOO_SMALL;
   }
-  MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau));
+  MALA_TRY(check_common(B, Hq, Hkv, N, d, scale, tau, 256));
   MALA_TRY(check_lengths(N, Nk, causal));
   if (!lse) return MALA_ERR_INVALID_ARG;
   const int Bt = cu ? 1 : B, Nt = cu ? total : N, Nkt = cu ? (cu_k ? total_k : total) : Nk;   // extents of the tensors
@@ -312,11 +316,15 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
     return MALA_ERR_CUDA;
   const bool dense = (tau == 0.f);
   int rc;
-  if (D == 128) rc = dense ? launch_fwd<128, true>(tq, tk, tv, p, stream) : launch_fwd<128, false>(tq, tk, tv, p, stream);
+  if (D == 256) rc = dense ? launch_fwd<256, true>(tq, tk, tv, p, stream) : launch_fwd<256, false>(tq, tk, tv, p, stream);
+  else if (D == 128) rc = dense ? launch_fwd<128, true>(tq, tk, tv, p, stream) : launch_fwd<128, false>(tq, tk, tv, p, stream);
   else rc = dense ? launch_fwd<64, true>(tq, tk, tv, p, stream) : launch_fwd<64, false>(tq, tk, tv, p, stream);
   if (rc != MALA_OK || num_splits == 1) return rc;
   const unsigned rows = (unsigned)((long long)B * Hq * N);
-  if (D == 128)
+  if (D == 256)
+    fwd_merge_splits_kernel<256><<<rows, 256, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
+                                                           num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal, d);
+  else if (D == 128)
     fwd_merge_splits_kernel<128><<<rows, 128, 0, stream>>>(p.o_part, p.lse_part, p.o, p.o_sb, p.o_sn, p.o_sh, lse, Hq, N,
                                                            num_splits, p.tps, p.Tk, p.koff, p.qshift, p.causal, d);
   else

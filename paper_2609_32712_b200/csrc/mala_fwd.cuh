@@ -1,4 +1,4 @@
-// MALA forward (Algorithm 1) for sm_100a, prefill version: two query blocks per CTA.
+// MALA forward (Algorithm 1) for sm_100a, prefill version: two query blocks per CTA (one with a head size above 128).
 //
 // One CTA owns the two consecutive 128-row query blocks A = 2c and B = 2c+1 of one (batch, query
 // head).  They share the K tiles; each block has its own UMMA-issuing warp, softmax warpgroup,
@@ -68,9 +68,14 @@ template <int D, bool kDense>
 struct FwdCfg {
   static constexpr int kPanels = D / 64;
   static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kKStages = 3;
+  // Head sizes above 128: a tile is 64 KB, so a CTA owns ONE query block (block A; the warps of block B find no
+  // block) with one Q tile, one K stage and one V stage, and its accumulators S (128 columns) and O (256) fill the
+  // tensor memory that two blocks of 128 columns fill otherwise.
+  static constexpr bool kOne = D > 128;
+  static constexpr int kKStages = kOne ? 1 : 3;
+  static constexpr int kBlocks = kOne ? 1 : 2;     // Q tiles and V stages
   // Q_A, Q_B, K ring, V_A, V_B
-  static constexpr int kSmemBytes = (2 + kKStages + 2) * kTileBytes + 1024;
+  static constexpr int kSmemBytes = (kBlocks + kKStages + kBlocks) * kTileBytes + 1024;
   static constexpr int kThreads = 384;
   static constexpr uint32_t kTmemCols = 512;
 };
@@ -82,11 +87,12 @@ __global__ void __launch_bounds__(384, 1)
 mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const FwdParams p) {
   using Cfg = FwdCfg<D, kDense>;
-  constexpr int KS = Cfg::kKStages, PAN = Cfg::kPanels;
+  constexpr int KS = Cfg::kKStages, PAN = Cfg::kPanels, VS = Cfg::kBlocks;
+  constexpr bool kOne = Cfg::kOne;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                               // [2] blocks A, B
-  uint8_t* sK = sQ + 2 * Cfg::kTileBytes;
+  uint8_t* sK = sQ + Cfg::kBlocks * Cfg::kTileBytes;
   uint8_t* sV = sK + KS * Cfg::kTileBytes;          // [2] blocks A, B
 
   __shared__ uint64_t q_full, k_full[KS], k_empty[KS], v_full[2], v_empty[2], s_full[2], vote_bar[2], p_full[2][2],
@@ -134,11 +140,11 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int Tr = p.cu ? (Nq + qshift + 127) / 128 : p.Tr;
   const int Tk = p.cu ? (Nkeys + 127) / 128 : p.Tk;
   const int bz = p.cu ? 0 : b;                        // outermost TMA coordinate
-  const int npairs = (Tr + 1) / 2;
+  const int npairs = kOne ? Tr : (Tr + 1) / 2;
   if ((int)blockIdx.x >= npairs) return;             // (a sequence shorter than the longest one)
   const int c = npairs - 1 - (int)blockIdx.x;        // longest pairs first
-  int iA = 2 * c, iB = 2 * c + 1;
-  bool hasB = iB < Tr;
+  int iA = kOne ? c : 2 * c, iB = kOne ? c : 2 * c + 1;
+  bool hasB = !kOne && iB < Tr;
   int dA = p.causal ? iA + koff : Tk - 1;            // newest key block with a legal key, per block
   const int dB = p.causal ? iB + koff : Tk - 1;
   int jlo = 0, jhi = Tk - 1;                         // key blocks of this CTA
@@ -213,18 +219,18 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       issued = u + 1;
       if (++s == KS) { s = 0; par ^= 1; }
       if (kDense) {
-        ok = mbar_wait_warp(&v_empty[u & 1], ((u >> 1) & 1) ^ 1, status);
+        ok = mbar_wait_warp(&v_empty[u % VS], ((u / VS) & 1) ^ 1, status);
         if (!ok) break;
-        if (lane == 0) mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
+        if (lane == 0) mbar_arrive_expect_tx(&v_full[u % VS], Cfg::kTileBytes);
         __syncwarp();
-        load_tile_small_warp(sV + (u & 1) * Cfg::kTileBytes, &tmV, &v_full[u & 1], j0 - u);
+        load_tile_small_warp(sV + (u % VS) * Cfg::kTileBytes, &tmV, &v_full[u % VS], j0 - u);
         v_issued = u + 1;
       }
     }
     if (!ok && lane == 0) {
       mbar_wait(&q_full, 0, status);
       for (int u = (issued > KS ? issued - KS : 0); u < issued; ++u) mbar_wait(&k_full[u % KS], (u / KS) & 1, status);
-      for (int u = (v_issued > 2 ? v_issued - 2 : 0); u < v_issued; ++u) mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
+      for (int u = (v_issued > VS ? v_issued - VS : 0); u < v_issued; ++u) mbar_wait(&v_full[u % VS], (u / VS) & 1, status);
     }
   } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer: Q_A, Q_B, K ring
@@ -251,18 +257,18 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         issued = u + 1;
         if (++s == KS) { s = 0; par ^= 1; }
         if (kDense) {   // dense: every tile is retained, so V(u) is prefetched into the shared 2-stage ring
-          ok = mbar_wait(&v_empty[u & 1], ((u >> 1) & 1) ^ 1, status);
+          ok = mbar_wait(&v_empty[u % VS], ((u / VS) & 1) ^ 1, status);
           if (!ok) break;
-          mbar_arrive_expect_tx(&v_full[u & 1], Cfg::kTileBytes);
+          mbar_arrive_expect_tx(&v_full[u % VS], Cfg::kTileBytes);
           for (int pn = 0; pn < PAN; ++pn)
-            tma_load_4d(sV + (u & 1) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u & 1], pn * 64, krow, hkv, kouter);
+            tma_load_4d(sV + (u % VS) * Cfg::kTileBytes + pn * 16384, &tmV, &v_full[u % VS], pn * 64, krow, hkv, kouter);
           v_issued = u + 1;
         }
       }
       if (!ok) {
         mbar_wait(&q_full, 0, status);
         for (int u = (issued > KS ? issued - KS : 0); u < issued; ++u) mbar_wait(&k_full[u % KS], (u / KS) & 1, status);
-        for (int u = (v_issued > 2 ? v_issued - 2 : 0); u < v_issued; ++u) mbar_wait(&v_full[u & 1], (u >> 1) & 1, status);
+        for (int u = (v_issued > VS ? v_issued - VS : 0); u < v_issued; ++u) mbar_wait(&v_full[u % VS], (u / VS) & 1, status);
       }
     }
   } else if (warp == 1 || warp == 2) {
@@ -303,9 +309,9 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         if (leader) mbar_arrive(&k_empty[s]);
         if (kDense) {                  // release the shared V stage too, paced by its arrival
-          ok = mbar_wait_warp(&v_full[u & 1], (u >> 1) & 1, status);
+          ok = mbar_wait_warp(&v_full[u % VS], (u / VS) & 1, status);
           if (!ok) break;
-          if (leader) mbar_arrive(&v_empty[u & 1]);
+          if (leader) mbar_arrive(&v_empty[u % VS]);
         }
         if (++s == KS) { s = 0; kpar ^= 1; }
       }
@@ -333,8 +339,8 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (retain) {
           // MALA: V is loaded on demand into this block's own stage (free once its previous PV retired);
           // dense: V(u) sits in the shared ring stage u & 1
-          const int vs = kDense ? (u & 1) : x;
-          const uint32_t vpar = kDense ? ((u >> 1) & 1) : (r & 1);
+          const int vs = kDense ? (u % VS) : x;
+          const uint32_t vpar = kDense ? ((u / VS) & 1) : (r & 1);
           if (!kDense) {
             ok = mbar_wait_warp(&v_empty[x], (r & 1) ^ 1, status);
             if (!ok) break;

@@ -28,11 +28,11 @@ inline PFN_tensorMapEncodeTiled tensor_map_encoder() {
 // Tensor map over a bf16 [B, N, H, d] view: coordinates (c, n, h, b), box = 64 columns x box_rows rows,
 // 128-byte swizzle, out-of-range rows read as zero.  Returns false if the driver rejects it
 // (base not 16-byte aligned, a stride not a multiple of 16 bytes, ...).
-// Head sizes: any multiple of 8 up to 128.  The kernels are built for D = 64 and D = 128 columns; a smaller head runs
-// on the next of the two with the missing columns read as zeros (TMA fills what lies beyond the tensor map's inner
-// extent d) and never stored.
-inline bool head_size_ok(int d) { return d >= 8 && d <= 128 && d % 8 == 0; }
-inline int padded_head_size(int d) { return d <= 64 ? 64 : 128; }
+// Head sizes: any multiple of 8 up to dmax (128; the forward and the decode step also take 256).  The kernels are built
+// for D = 64, 128 and 256 columns; a smaller head runs on the next of them with the missing columns read as zeros (TMA
+// fills what lies beyond the tensor map's inner extent d) and never stored.
+inline bool head_size_ok(int d, int dmax = 128) { return d >= 8 && d <= dmax && d % 8 == 0; }
+inline int padded_head_size(int d) { return d <= 64 ? 64 : (d <= 128 ? 128 : 256); }
 
 inline bool make_tensor_map_bnhd(CUtensorMap* out, const void* base, int B, int N, int H, int d, int64_t sb,
                                  int64_t sn, int64_t sh, int box_rows) {

@@ -1,6 +1,7 @@
-"""Head sizes other than 64 and 128 (any multiple of 8 up to 128): every entry point against the oracle.  The kernels
-run them on the next of their two column counts with the missing columns read as zeros, so what these cases guard is
-that nothing beyond column d is stored and that the zero columns change no result."""
+"""Head sizes other than 64 and 128 (any multiple of 8 up to 128; up to 256 in the forward): every entry point against
+the oracle.  The kernels run them on the next of their column counts with the missing columns read as zeros, so what
+these cases guard is that nothing beyond column d is stored and that the zero columns change no result; above 128 the
+forward runs one query block per CTA, which the cases at 256, 192 and 136 columns cover on every forward entry point."""
 import numpy as np
 import pytest
 import torch
@@ -9,6 +10,7 @@ from paper_2609_32712_b200 import workloads as W
 from tests import parity
 from tests.test_gpu_chunk import _chunk, _run, _run_bwd_any_offset, _run_fwd_any_offset, _run_split
 from tests.test_gpu_decode import _run_and_check, _run_multi, _run_paged
+from tests.test_gpu_fwd import _run_and_check as _run_fwd
 
 pytestmark = pytest.mark.gpu
 
@@ -89,8 +91,60 @@ def test_decode_gated_paged_several_tokens(mala, oracle, d, tau):
 
 
 def test_head_sizes_that_are_refused(mala):
-    for d in (4, 100, 136, 256):
+    for d in (4, 100, 260, 264, 512):
         q = torch.zeros(1, 256, 2, d, dtype=torch.bfloat16, device="cuda")
         with pytest.raises(mala.MalaError) as e:
             mala.fwd(q, q, q, 0.1, 0.0)
         assert e.value.code in (-2, -3)
+    for d in (136, 256):          # the backward stops at 128 columns
+        q = torch.zeros(1, 256, 2, d, dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros(1, 2, 256, dtype=torch.float32, device="cuda")
+        with pytest.raises(mala.MalaError) as e:
+            mala.bwd(q, q, q, q, q, lse, 0.1, 0.0)
+        assert e.value.code == -2
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("d,N,Hq,Hkv", [(256, 640, 4, 2), (256, 128, 1, 1), (192, 500, 2, 1), (136, 700, 2, 2), (160, 257, 2, 1),
+                                        (256, 1100, 2, 1)])
+def test_forward_above_128_columns_literal(mala, oracle, d, N, Hq, Hkv, tau):
+    w = W.custom_prefill(2, Hq, Hkv, N, d, seed=d + N)
+    _run_fwd(mala, oracle, w, tau)
+    _run_fwd(mala, oracle, w, tau, causal=False)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("d", [256, 192])
+def test_forward_above_128_columns_skipping_regime(mala, oracle, d, tau):
+    w = W.custom_prefill(1, 4, 2, 2048, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=d, preset="R")
+    res = _run_fwd(mala, oracle, w, tau, rounding_bound=True)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+
+
+@pytest.mark.parametrize("d", [256, 144])
+def test_forward_above_128_columns_chunks_and_key_ranges(mala, oracle, d):
+    w = W.custom_prefill(1, 4, 2, 1500, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=d + 1, preset="R")
+    _run_fwd_any_offset(mala, oracle, _chunk(w, 333), 1e-4)
+    _run_fwd_any_offset(mala, oracle, _chunk(w, 333), 1e-4, S=3)
+    _run_fwd_any_offset(mala, oracle, _chunk(w, 348), 0.0)
+    _run_split(mala, oracle, _chunk(w, 220), 1e-4, 4)
+    _run_split(mala, oracle, _chunk(w, 220), 0.0, 5)
+
+
+def test_forward_above_128_columns_stores_nothing_beyond_the_head_size(mala):
+    d, dw, N = 192, 256, 400
+    w = W.custom_prefill(1, 2, 1, N, d, seed=5)
+    q, k, v = (w[x].cuda() for x in ("q", "k", "v"))
+    ob = torch.full(q.shape[:-1] + (dw,), 7.0, dtype=torch.bfloat16, device="cuda")
+    o = ob[..., :d]
+    for tau in (0.0, 1e-4):
+        mala.fwd(q, k, v, w["scale"], tau, out=o)
+        torch.cuda.synchronize()
+        assert mala.device_status() == 0
+        assert (ob[..., d:] == 7.0).all() and not (ob[..., :d] == 7.0).all()
+        assert torch.equal(mala.fwd(q, k, v, w["scale"], tau)[0], o)
+    # the result on the inputs padded with zero columns to the kernel's width is the same
+    pad = lambda t: torch.cat([t, torch.zeros(t.shape[:-1] + (dw - d,), dtype=t.dtype, device=t.device)], dim=-1)
+    op, lsep, _ = mala.fwd(pad(q), pad(k), pad(v), w["scale"], 1e-4)
+    o1, lse1, _ = mala.fwd(q, k, v, w["scale"], 1e-4)
+    assert torch.equal(op[..., :d], o1) and torch.equal(lsep, lse1) and (op[..., d:] == 0).all()
