@@ -183,14 +183,14 @@ int mala_decode_suggest_splits(int B, int Hkv, int Nk, int sm_count) {
 
 int mala_tile_shape(int op, int d, int* Bq, int* Bk) {
   if (!Bq || !Bk) return MALA_ERR_INVALID_ARG;
-  if (!head_size_ok(d, op == MALA_OP_FWD ? 256 : 128)) return MALA_ERR_UNSUPPORTED;
+  if (!head_size_ok(d, op == MALA_OP_BWD ? 128 : 256)) return MALA_ERR_UNSUPPORTED;
   if (op == MALA_OP_FWD || op == MALA_OP_BWD) { *Bq = 128; *Bk = 128; return MALA_OK; }
   if (op == MALA_OP_DECODE) { *Bq = 0; *Bk = 128; return MALA_OK; }
   return MALA_ERR_UNSUPPORTED;
 }
 
 size_t mala_workspace_bytes(int op, int B, int Hq, int Hkv, int N, int d, int num_splits) {
-  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || !head_size_ok(d, op == MALA_OP_FWD ? 256 : 128)) return 0;
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || N <= 0 || !head_size_ok(d, op == MALA_OP_BWD ? 128 : 256)) return 0;
   const int D = padded_head_size(d);
   if (op == MALA_OP_FWD) return num_splits > 1 ? fwd_split_workspace_bytes(B, Hq, N, D, num_splits) : 256;
   if (op == MALA_OP_BWD) return bwd_workspace_bytes(B, Hq, N, D);
@@ -472,7 +472,7 @@ int mala_bwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_
 int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
                 int B, int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws,
                 size_t ws_bytes, void* cuda_stream) {
-  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau, 256));
   if (num_splits <= 0 || !ws) return MALA_ERR_INVALID_ARG;
   if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
   MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));
@@ -558,7 +558,7 @@ int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const 
 int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
                       int B, int Hq, int Hkv, int Nk, int Sq, int d, float scale, float tau, int num_splits, void* ws,
                       size_t ws_bytes, void* cuda_stream) {
-  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau, 256));
   if (num_splits <= 0 || Sq <= 0 || !ws) return MALA_ERR_INVALID_ARG;
   if ((Hq / Hkv) * Sq > 16 || Sq > Nk || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
   MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, Sq, Hq));
@@ -584,7 +584,7 @@ int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_
       (long long)max_pages_per_seq * page_size > 0x7fffffffLL)
     return MALA_ERR_UNSUPPORTED;
   const int Nk = max_pages_per_seq * page_size;   // the longest cache a sequence can hold
-  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau, 256));
   if (num_splits <= 0 || !ws) return MALA_ERR_INVALID_ARG;
   if ((Hq / Hkv) * Sq > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
   if ((((uintptr_t)block_table) & 3) != 0 || (((uintptr_t)seqlens) & 3) != 0) return MALA_ERR_MISALIGNED;
@@ -607,7 +607,7 @@ int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_
 
 int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, int B, int Hq,
                        int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* cuda_stream) {
-  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau, 256));
   if (num_splits <= 0) return MALA_ERR_INVALID_ARG;
   if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
   MALA_TRY(check_view(q.p, q.sb, 8, q.sh, B, 1, Hq));

@@ -46,7 +46,8 @@ inline bool decode_set_attributes() {
   bool ok = true;
 #define MALA_DEC_ATTR(DENSE, GP, MULTI) \
   ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess; \
-  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg::kSmemBytes) == cudaSuccess; \
+  ok = ok && cudaFuncSetAttribute(mala_decode_split_kernel<DENSE, GP, MULTI, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfgT<256>::kSmemBytes) == cudaSuccess;
 #define MALA_DEC_ATTR_GP(GP) MALA_DEC_ATTR(false, GP, false) MALA_DEC_ATTR(true, GP, false) MALA_DEC_ATTR(false, GP, true) MALA_DEC_ATTR(true, GP, true)
   MALA_DEC_ATTR_GP(1) MALA_DEC_ATTR_GP(2) MALA_DEC_ATTR_GP(4) MALA_DEC_ATTR_GP(8) MALA_DEC_ATTR_GP(16)
 #define MALA_F8_ATTR(DENSE, GP) \
@@ -73,7 +74,7 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
                                       const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                                       float tau, int num_splits, float* o_part, float* lse_part, int* status,
                                       cudaStream_t stream, const DecPaging* pg = nullptr, int Sq = 1) {
-  if (!head_size_ok(d)) return MALA_ERR_UNSUPPORTED;
+  if (!head_size_ok(d, 256)) return MALA_ERR_UNSUPPORTED;
   const int D = padded_head_size(d);
   const int G = Hq / Hkv;
   if (Sq < 1 || G * Sq > 16 || Sq > Nk) return MALA_ERR_UNSUPPORTED;
@@ -125,7 +126,8 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
   const int R = G * Sq;   // rows of a work item
 #define MALA_DEC_LAUNCH3(DENSE, GP, MULTI)                                                                           \
   {                                                                                                                  \
-    if (D == 128) mala_decode_split_kernel<DENSE, GP, MULTI, 128><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    if (D == 256) mala_decode_split_kernel<DENSE, GP, MULTI, 256><<<grid, DecCfg::kThreads, DecCfgT<256>::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    else if (D == 128) mala_decode_split_kernel<DENSE, GP, MULTI, 128><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p); \
     else mala_decode_split_kernel<DENSE, GP, MULTI, 64><<<grid, DecCfg::kThreads, DecCfg::kSmemBytes, stream>>>(tq, tk, tv, p);           \
   }
 #define MALA_DEC_LAUNCH2(DENSE, GP)          \
@@ -147,7 +149,10 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
 #undef MALA_DEC_LAUNCH2
 #undef MALA_DEC_LAUNCH3
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
-  if (D == 128)
+  if (D == 256)
+    decode_merge_kernel<256><<<B * Sq * Hq, 256, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
+                                                              Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits, d);
+  else if (D == 128)
     decode_merge_kernel<128><<<B * Sq * Hq, 128, 0, stream>>>(o_part, lse_part, (__nv_bfloat16*)o.p, o.sb,
                                                               Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits, d);
   else

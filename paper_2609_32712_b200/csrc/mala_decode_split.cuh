@@ -1,4 +1,4 @@
-// Split-KV decode, split kernel ("Fused decoding execution") for sm_100a, head size 128 or 64.
+// Split-KV decode, split kernel ("Fused decoding execution") for sm_100a, head size 64, 128 or 256.
 //
 // A work item is one split of one (batch, KV head): the G = Hq/Hkv <= 16 query heads that share the KV head
 // are processed together, L = Nk for every head, the tiles of the split are visited newest first with the
@@ -51,16 +51,21 @@ struct DecParams {
   float scale_log2, log2_tau;
 };
 
-struct DecCfg {
-  static constexpr int kTileBytes = 128 * 128 * 2;
-  static constexpr int kQBytes = 4096;                   // 16 rows x 128 columns, two 2 KB panels
+// D: columns of the kernel (64, 128 or 256).  With 256 a K / V tile is 64 KB (four panels), the rings hold two K
+// tiles and one V tile in the 192 KB that otherwise hold three and three, and O^T has a second pair of accumulators
+// for the channels 128 .. 255.
+template <int D>
+struct DecCfgT {
+  static constexpr int kTileBytes = D > 128 ? 128 * 256 * 2 : 128 * 128 * 2;
+  static constexpr int kQBytes = D > 128 ? 8192 : 4096;  // 16 rows x 128 (256) columns, 2 KB panels
   static constexpr int kPBytes = 4096;                   // P^T: 16 rows (heads) x 128 keys, two 2 KB panels
-  static constexpr int kKStages = 3, kVStages = 3, kPStages = 4, kSStages = 4;
+  static constexpr int kKStages = D > 128 ? 2 : 3, kVStages = D > 128 ? 1 : 3, kPStages = 4, kSStages = 4;
   static constexpr int kSmemBytes = 2 * kQBytes + (kKStages + kVStages) * kTileBytes + kPStages * kPBytes + 1024;
   static constexpr int kThreads = 384;                   // producer, UMMA warp, two idle warps, up to two softmax groups
-  static constexpr uint32_t kTmemCols = 128;             // S^T ring 4 x 16, O^T 2 x 16 (item parity)
-  static constexpr uint32_t kColO = 64;
+  static constexpr uint32_t kTmemCols = 128;             // S^T ring 4 x 16, O^T 2 x 16 (item parity), O^T of channels 128.. 2 x 16
+  static constexpr uint32_t kColO = 64, kColOHi = 96;
 };
+using DecCfg = DecCfgT<128>;
 
 // Warp-wide reduction of N independent values per lane (N a power of two <= 16) in N-ish shuffles instead of 5 N:
 // while more than one value is left, a lane hands the half of its values that its partner (lane ^ OFF) keeps to that
@@ -108,13 +113,15 @@ __device__ __forceinline__ void lds_row(const float* src, float (&dst)[N]) {
 // GP: the number of packed rows rounded up to a power of two (compile-time, so that the per-row loops of the
 // softmax group unroll without branches).  kMulti: several new tokens per sequence, i.e. rows that see
 // different numbers of keys (one token: every row sees all keys, and the per-row limits fold into scalars).
-// D: head size, 128 or 64.  The shared-memory stages keep their 128-wide size for D = 64 and only their first
+// D: head size, 64, 128 or 256.  The shared-memory stages keep their 128-wide size for D = 64 and only their first
 // 64-column panel is filled; O^T is then still accumulated as a 128-row MMA whose rows 64.. (fed from the unfilled
-// half of the V stage) are never read.
+// half of the V stage) are never read.  With D = 256 O^T is two 128-row MMAs per key step, on the tile's panels 0-1
+// and 2-3, into two accumulators; a softmax thread then owns the output channels kt and 128 + kt.
 template <bool kDense, int GP, bool kMulti, int D>
 __global__ void __launch_bounds__(384, 1)
 mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                          const __grid_constant__ CUtensorMap tmV, const DecParams p) {
+  using DecCfg = DecCfgT<D>;
   constexpr int KS = DecCfg::kKStages, VS = DecCfg::kVStages, TB = DecCfg::kTileBytes;
   constexpr int PAN = D / 64;                    // 64-column panels of a K / V / Q tile
   constexpr uint32_t kTileTx = 128u * D * 2u;    // bytes one K or V tile copy delivers
@@ -209,8 +216,9 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   // table lookups are one coalesced load and the copies are issued side by side (one lane alone cannot issue 16 to 32 copies per tile in a
   // tile's HBM time).  The barrier's expect_tx has been posted by then.
   auto load_tile_small_warp = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int b, int jt, int hkv) {
-    const int c = lane / PAN, pn = lane % PAN;
-    if (c < p.ppt) tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, small_page(b, jt, c));
+    const int pn = lane % PAN;
+    for (int c = lane / PAN; c < p.ppt; c += 32 / PAN)
+      tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, small_page(b, jt, c));
   };
 
   if (warp == 0 && p.ppt > 1) {
@@ -439,6 +447,12 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 #pragma unroll
           for (int k = 0; k < 8; ++k)   // k-step = 16 keys: 2 KB further on in the V tile, two core matrices of P^T
             mma_ss(dO, desc_advance(dV, k * 2048), desc_advance(dP, k * 256), idesc_pv, k > 0 ? 1u : acc0, leader);
+          if constexpr (D > 128) {      // channels 128 .. 255: the tile's panels 2 and 3, the second accumulator
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              mma_ss(dO + (DecCfg::kColOHi - DecCfg::kColO), desc_advance(dV, 32768 + k * 2048), desc_advance(dP, k * 256),
+                     idesc_pv, k > 0 ? 1u : acc0, leader);
+          }
           if (leader) { tc_commit(&v_empty[vc]); tc_commit(&p_free[ps]); }
           if (++vc == VS) { vc = 0; vcpar ^= 1; }
           ++npv;
@@ -572,6 +586,12 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             for (int k = 0; k < 8; ++k)   // k-step = 16 keys: 2 KB further on in the V tile, 32 B in a P^T panel
               mma_ss(dO, desc_advance(dV, k * 2048), desc_advance(dP, k * 256), idesc_pv,
                      k > 0 ? 1u : acc0, leader);
+            if constexpr (D > 128) {      // channels 128 .. 255: the tile's panels 2 and 3, the second accumulator
+#pragma unroll
+              for (int k = 0; k < 8; ++k)
+                mma_ss(dO + (DecCfg::kColOHi - DecCfg::kColO), desc_advance(dV, 32768 + k * 2048), desc_advance(dP, k * 256),
+                       idesc_pv, k > 0 ? 1u : acc0, leader);
+            }
             if (leader) { tc_commit(&v_empty[vc]); tc_commit(&p_free[ps]); }
             if (++vc == VS) { vc = 0; vcpar ^= 1; }
             ++npv;
@@ -653,17 +673,22 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       k = __all_sync(0xffffffffu, k);
       if (!k) return false;
       tc_fence_after();
-      uint32_t o[LDN];
+      uint32_t o[LDN], o2[D > 128 ? LDN : 1];
       tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, DecCfg::kColO + (uint32_t)pend_ip * 16u + (uint32_t)rb), o);
+      if constexpr (D > 128) tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, DecCfg::kColOHi + (uint32_t)pend_ip * 16u + (uint32_t)rb), o2);
       tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&o_free[pend_ip]);   // the accumulator may take the item after next
 #pragma unroll
       for (int q = 0; q < GH; ++q)
-        if (rb + q < R && kt < D)   // (a row that saw no key of the split: (0, -inf))
+        if (rb + q < R && kt < D) {   // (a row that saw no key of the split: (0, -inf))
           p.o_part[(pend_prow0 + rowoff[q]) * D + kt] =
               (!kMulti || pend_l[q] > 0.f) ? __uint_as_float(o[q]) / pend_l[q] : 0.f;
+          if constexpr (D > 128)
+            p.o_part[(pend_prow0 + rowoff[q]) * D + 128 + kt] =
+                (!kMulti || pend_l[q] > 0.f) ? __uint_as_float(o2[q]) / pend_l[q] : 0.f;
+        }
       pend = false;
       return true;
     };
@@ -685,6 +710,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         for (int q = 0; q < GH; ++q)
           if (rb + q < R) {
             if (kt < D) p.o_part[(prow0 + rowoff[q]) * D + kt] = 0.f;
+            if constexpr (D > 128) p.o_part[(prow0 + rowoff[q]) * D + 128 + kt] = 0.f;
             if (kt == q) p.lse_part[prow0 + rowoff[q]] = -INFINITY;
           }
         if (head && p.retained) p.retained[stat_row] = 0u;
@@ -809,6 +835,14 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 #pragma unroll
             for (int q = 0; q < GH; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
             tmem_st_cols<LDN>(tmem_addr(tb, lane_base, colO + (uint32_t)rb), o);
+            if constexpr (D > 128) {
+              constexpr uint32_t hi = DecCfg::kColOHi - DecCfg::kColO;
+              tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colO + hi + (uint32_t)rb), o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int q = 0; q < GH; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
+              tmem_st_cols<LDN>(tmem_addr(tb, lane_base, colO + hi + (uint32_t)rb), o);
+            }
             tmem_wait_st();
             tc_fence_before();
           }

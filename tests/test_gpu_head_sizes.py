@@ -1,7 +1,8 @@
-"""Head sizes other than 64 and 128 (any multiple of 8 up to 128; up to 256 in the forward): every entry point against
-the oracle.  The kernels run them on the next of their column counts with the missing columns read as zeros, so what
+"""Head sizes other than 64 and 128 (any multiple of 8 up to 128; up to 256 in the forward and the decode step): every
+entry point against the oracle.  The kernels run them on the next of their column counts with the missing columns read as zeros, so what
 these cases guard is that nothing beyond column d is stored and that the zero columns change no result; above 128 the
-forward runs one query block per CTA, which the cases at 256, 192 and 136 columns cover on every forward entry point."""
+forward runs one query block per CTA and the decode step 64 KB tiles with two output accumulators, which the cases
+at 136 to 256 columns cover on every forward and decode entry point."""
 import numpy as np
 import pytest
 import torch
@@ -148,3 +149,35 @@ def test_forward_above_128_columns_stores_nothing_beyond_the_head_size(mala):
     op, lsep, _ = mala.fwd(pad(q), pad(k), pad(v), w["scale"], 1e-4)
     o1, lse1, _ = mala.fwd(q, k, v, w["scale"], 1e-4)
     assert torch.equal(op[..., :d], o1) and torch.equal(lsep, lse1) and (op[..., d:] == 0).all()
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("d,Nk,S,Hq,Hkv", [(256, 1024, 4, 8, 2), (256, 1000, 3, 8, 1), (192, 4096, 8, 16, 1), (136, 300, 2, 6, 2),
+                                           (256, 2048, 4, 3, 1), (256, 128, 1, 1, 1)])
+def test_decode_above_128_columns_literal(mala, oracle, d, Nk, S, Hq, Hkv, tau):
+    w = W.custom_decode(2, Hq, Hkv, Nk, d, S, seed=Nk + d)
+    _run_and_check(mala, oracle, w, tau, S)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("d", [256, 160])
+def test_decode_above_128_columns_gated_paged_several_tokens(mala, oracle, d, tau):
+    w = W.custom_decode(2, 8, 2, 8192, d, 8, group_types=["diffuse", "peaked"], seed=3 + d, preset="D")
+    res = _run_and_check(mala, oracle, w, tau, 8)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+    _run_paged(mala, oracle, w, tau, 8, 256, [8192, 4096 + 77], seed=9)
+    _run_paged(mala, oracle, w, tau, 8, 16, [8192, 1000], seed=10)
+    _run_paged(mala, oracle, w, tau, 8, 8, [700, 8192], seed=11)
+    assert _run_multi(mala, oracle, w, 3, tau, 8) > 0
+
+
+def test_decode_above_128_columns_stores_nothing_beyond_the_head_size(mala):
+    d, dw = 192, 256
+    w = W.custom_decode(2, 8, 2, 3000, d, 4, seed=8, device="cuda")
+    ob = torch.full(w["q"].shape[:-1] + (dw,), 7.0, dtype=torch.bfloat16, device="cuda")
+    o = ob[..., :d]
+    mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 1e-4, 4, out=o)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert (ob[..., d:] == 7.0).all() and not (ob[..., :d] == 7.0).all()
+    assert torch.equal(mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 1e-4, 4)[0], o)
