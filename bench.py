@@ -354,6 +354,25 @@ def head_size_leg(cfg, preset, d, tau, it, peaks, dev):
     return row
 
 
+def head_size_256_fwd_leg(cfg, preset, tau, it, peaks, dev):
+    """The configuration's shapes with half the heads of twice the size (d = 256: the same FLOPs and bytes), forward only
+    (one query block per CTA; the backward stops at 128 columns)."""
+    import torch
+    from paper_2609_32712_b200 import mala, workloads as W
+    Hq, Hkv, d = cfg.Hq // 2, cfg.Hkv // 2, 256
+    w = W.custom_prefill(cfg.B, Hq, Hkv, cfg.N, d, head_types=cfg.head_types[:cfg.Hq // 2], seed=cfg.seed, preset=preset, device=dev)
+    q, k, v = w["q"], w["k"], w["v"]
+    o = torch.empty_like(q)
+    taus = {"mala": tau, "dense": 0.0}
+    f_t = time_alternating({lab: (lambda t_=t_: mala.fwd(q, k, v, w["scale"], t_, out=o)) for lab, t_ in taus.items()}, 3, it)
+    _, _, fs = mala.fwd(q, k, v, w["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    fr, fl = fs.totals.cpu().tolist()
+    return {"d": d, "Hq": Hq, "Hkv": Hkv, "mala": {"fwd_ms": f_t["mala"]}, "dense": {"fwd_ms": f_t["dense"]},
+            "fwd_retained_frac": fr / fl,
+            "dense_fwd_tensor_frac": fwd_executed_flops(fl, fl, d) / (f_t["dense"] * 1e-3) / 1e12 / peaks["tflops_sustained"]}
+
+
 def serving_prefill_leg(cfg, preset, tau, it, peaks, dev):
     """A serving-style prefill batch with the heads of a prefill configuration: eight sequences, a 2048-token chunk each
     behind prefixes of 0 ... 30720 tokens, packed (mala_fwd_varlen_prefix) and against a paged cache (mala_fwd_paged,
@@ -838,6 +857,8 @@ def main():
                     row["serving_prefill_8x2048"] = serving_prefill_leg(cc, preset, tau, it, peaks, dev)
                 if name == "cfg3":                  # the same shapes with 96-column heads (run on the 128-column kernels)
                     row["head_size_96"] = head_size_leg(cc, preset, 96, tau, it, peaks, dev)
+                if name == "cfg3":                  # half the heads, 256 columns each: the forward's one-block-per-CTA kernel
+                    row["head_size_256_fwd"] = head_size_256_fwd_leg(cc, preset, tau, it, peaks, dev)
                 if name == "cfg3" and preset == "R":
                     row["fidelity_vs_dense"] = fidelity(cs, (1e-4, 1e-2, 1.0), it)
                 detail[f"{name}_{preset}"] = row
@@ -903,6 +924,22 @@ def main():
             del kp8, vp8, bt8, ksp, vsp
             row["e4m3_cache"] = f8
             del k8, v8, ks8, vs8
+            # half the KV heads with 256 columns each (the same bytes per key): 64 KB tiles, two output accumulators
+            w2 = W.custom_decode(dcfg.B, dcfg.Hq // 2, dcfg.Hkv // 2, dcfg.Nk, 256, dcfg.num_splits,
+                                 group_types=dcfg.group_types[:dcfg.Hkv // 2], seed=dcfg.seed, preset=preset, device=dev)
+            o2 = torch.empty_like(w2["q"])
+            h256 = {"d": 256, "Hq": dcfg.Hq // 2, "Hkv": dcfg.Hkv // 2}
+            for label, t_ in (("mala", tau), ("dense", 0.0)):
+                us = 1e3 * time_cuda(lambda: mala.decode(w2["q"], w2["kcache"], w2["vcache"], w2["scale"], t_, dcfg.num_splits,
+                                                          ws=wsd, out=o2, want_lse=False), 25, 100)
+                _, _, st = mala.decode(w2["q"], w2["kcache"], w2["vcache"], w2["scale"], t_, dcfg.num_splits, ws=wsd, stats=True)
+                torch.cuda.synchronize()
+                ret, leg = st.totals.cpu().tolist()
+                need = (leg + ret) * TILE * 256 * 2
+                h256[label] = {"us": us, "retained_frac": ret / leg, "needed_gb": need / 1e9,
+                               "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+            row["head_size_256"] = h256
+            del w2, o2
             if preset == "D":                       # work and fidelity against the dense decode, tau up to 1
                 o0, lse0, _ = mala.decode(qd, kc, vc, wd["scale"], 0.0, dcfg.num_splits, ws=wsd)
                 o0, fid = o0.float(), {}

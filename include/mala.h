@@ -14,8 +14,11 @@
  *     never frees or retains one.  Tensors are bf16 views [B, N, H, d] given as a base pointer and
  *     element strides (sb, sn, sh); the last dimension is contiguous.  Base pointers must be
  *     16-byte aligned and all strides multiples of 8 elements (16 bytes).
- *   - d is a multiple of 8 between 8 and 128.  The kernels exist for 64 and 128 columns; another head size runs
- *     on the next of the two at that size's cost (the missing columns are read as zeros and never stored).
+ *   - d is a multiple of 8 between 8 and 256 for the forward calls (mala_fwd*) and the decode calls on a bf16 cache
+ *     (mala_decode, _multi, _paged, _static), between 8 and 128 for the backward calls and a multiple of 16 up to
+ *     128 for the calls on an e4m3 cache (the paper's symbols put no limit on d_h, Section 2.1; its models use 128).
+ *     The kernels exist for 64, 128 and 256 columns; another head size runs on the next of them at that size's cost
+ *     (the missing columns are read as zeros and never stored).
  *     Hq must be a multiple of Hkv; query head h uses key/value head h / (Hq / Hkv).  N may be any positive length (the last tile may be ragged).
  *   - scale (> 0, finite) multiplies the fp32 scores; lse is in nats, of the scaled scores, over
  *     the retained set.  tau >= 0, finite.
@@ -39,7 +42,7 @@ extern "C" {
 
 #define MALA_OK 0
 #define MALA_ERR_INVALID_ARG (-1)        /* NULL pointer, non-positive size, bad tau / scale */
-#define MALA_ERR_UNSUPPORTED (-2)        /* d not a multiple of 8 in 8..128, Hq % Hkv != 0, too many splits ... */
+#define MALA_ERR_UNSUPPORTED (-2)        /* d not a multiple of 8 in the call's range, Hq % Hkv != 0, too many splits ... */
 #define MALA_ERR_MISALIGNED (-3)         /* pointer / stride alignment rules above violated */
 #define MALA_ERR_WORKSPACE_TOO_SMALL (-4)
 #define MALA_ERR_WRONG_ARCH (-5)         /* current device is not compute capability 10.x */

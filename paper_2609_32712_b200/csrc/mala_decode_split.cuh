@@ -217,8 +217,13 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   // tile's HBM time).  The barrier's expect_tx has been posted by then.
   auto load_tile_small_warp = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int b, int jt, int hkv) {
     const int pn = lane % PAN;
-    for (int c = lane / PAN; c < p.ppt; c += 32 / PAN)
-      tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, small_page(b, jt, c));
+    if constexpr (PAN <= 2) {   // up to 16 copies of up to two panels: one per lane
+      const int c = lane / PAN;
+      if (c < p.ppt) tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, small_page(b, jt, c));
+    } else {
+      for (int c = lane / PAN; c < p.ppt; c += 32 / PAN)
+        tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, small_page(b, jt, c));
+    }
   };
 
   if (warp == 0 && p.ppt > 1) {

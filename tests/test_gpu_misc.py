@@ -105,9 +105,13 @@ def test_binding_reports_errors(mala):
     with pytest.raises(mala.MalaError) as e:
         mala.fwd(q, q, q, 0.1, -1.0)
     assert e.value.code == -1
-    q256 = torch.zeros(1, 256, 2, 256, dtype=torch.bfloat16, device="cuda")
+    q264 = torch.zeros(1, 256, 2, 264, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(mala.MalaError) as e:
-        mala.fwd(q256, q256, q256, 0.1, 0.0)
+        mala.fwd(q264, q264, q264, 0.1, 0.0)
+    assert e.value.code == -2
+    q256 = torch.zeros(1, 256, 2, 256, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(mala.MalaError) as e:        # the backward stops at 128 columns
+        mala.bwd(q256, q256, q256, q256, q256, lse, 0.1, 0.0)
     assert e.value.code == -2
     q17 = torch.zeros(1, 1, 34, 128, dtype=torch.bfloat16, device="cuda")
     kv1 = torch.zeros(1, 256, 2, 128, dtype=torch.bfloat16, device="cuda")

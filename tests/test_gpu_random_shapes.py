@@ -43,10 +43,17 @@ def test_random_cases_any_head_size(mala, oracle, seed):
     _sweep(mala, oracle, seed, list(range(8, 129, 8)), 40)
 
 
-def _sweep(mala, oracle, seed, head_sizes, n):
+@pytest.mark.parametrize("seed", [0, 7])
+def test_random_cases_head_sizes_above_128(mala, oracle, seed):
+    """The forward and the decode step (the backward stops at 128 columns)."""
+    _sweep(mala, oracle, seed, list(range(136, 257, 8)), 30, backward=False)
+
+
+def _sweep(mala, oracle, seed, head_sizes, n, backward=True):
     rng = random.Random(seed)
     for it in range(n):
-        kind = rng.choice(["fwdbwd", "chunk", "split", "varlen", "decode", "paged", "multi"])
+        kind = rng.choice(["fwdbwd", "chunk", "split", "varlen", "decode", "paged", "multi"] if backward else
+                          ["fwdbwd", "split", "decode", "paged", "multi"])
         tau = rng.choice([0.0, 1e-5, 1e-4, 1e-2, 1.0])
         d = rng.choice(head_sizes)
         preset = rng.choice(["literal", "R"])
@@ -54,8 +61,11 @@ def _sweep(mala, oracle, seed, head_sizes, n):
             Hq, Hkv = _heads(rng)
             N, causal = rng.randint(1, 1400), rng.random() < 0.8
             w = W.custom_prefill(rng.choice([1, 2]), Hq, Hkv, N, d, seed=rng.randint(0, 9999), preset=preset)
-            TF._run_and_check(mala, oracle, w, tau, causal=causal)
-            TB._run_isolated(mala, oracle, w, tau, causal=causal)
+            # (the sweep above 128 columns draws "planted" heads with |o| > 4, where half a bf16 ulp alone passes the
+            # absolute limit: its forward cases are held to the rounding bound instead, see parity.check_output)
+            TF._run_and_check(mala, oracle, w, tau, causal=causal, rounding_bound=not backward)
+            if backward:
+                TB._run_isolated(mala, oracle, w, tau, causal=causal)
         elif kind in ("chunk", "split"):
             Hq, Hkv = _heads(rng)
             Nq, off, causal = rng.randint(1, 700), 128 * rng.randint(0, 8), rng.random() < 0.8
@@ -74,7 +84,7 @@ def _sweep(mala, oracle, seed, head_sizes, n):
                 if causal and Nk > Nq + 1:   # the forward also from a position inside a tile, unsplit and split
                     c2 = TC._chunk(w, Nq + rng.randint(1, min(127, Nk - Nq)))
                     TC._run_fwd_any_offset(mala, oracle, c2, tau, rng.choice([1, S]))
-                    if len(head_sizes) > 2:   # (the newer sweep: the backward from that position as well)
+                    if len(head_sizes) > 2 and backward:   # (the newer sweep: the backward from that position as well)
                         TC._run_bwd_any_offset(mala, oracle, c2, tau)
         elif kind == "varlen":
             Hq, Hkv = _heads(rng)
