@@ -211,8 +211,8 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
   const int grid = p.n_items < sms ? p.n_items : sms;
 #define MALA_F8_LAUNCH(DENSE, GP)                                                                                      \
   do {                                                                                                                  \
-    if (pg) mala_decode_fp8_kernel<DENSE, GP, true><<<grid, DecF8Cfg<2, DENSE>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
-    else mala_decode_fp8_kernel<DENSE, GP, false><<<grid, DecF8Cfg<2, DENSE>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p);  \
+    if (pg) mala_decode_fp8_kernel<DENSE, GP, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    else mala_decode_fp8_kernel<DENSE, GP, false><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p);  \
   } while (0)
   const bool dense = (tau == 0.f);
   if (G <= 1) { if (dense) MALA_F8_LAUNCH(true, 1); else MALA_F8_LAUNCH(false, 1); }

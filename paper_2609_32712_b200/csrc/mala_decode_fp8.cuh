@@ -94,7 +94,10 @@ struct DecF8Params {
 // NG_: streams (two: a third, with the registers moved from the issuing warps to the softmax groups and rings of two
 // stages, gained the MALA kernel 4% and the dense kernel nothing).  kDense_: the dense kernel requests V with K and splits a stream's six stages evenly; the MALA kernel
 // requests V only after a tile's vote, a memory latency before its PV, and gives the V ring the larger share.
-template <int NG_, bool kDense_>
+// kSplit_: five to eight query heads per KV head.  A stream's softmax group is then eight warps, two threads per key:
+// warps 0-3 carry the heads 0-3 through the chain and warps 4-7 the heads 4-7 (both read the same TMEM lanes, their
+// own columns), so that a thread's chain is as long as with four heads; the two halves only meet in the tile's vote.
+template <int NG_, bool kDense_, bool kSplit_ = false>
 struct DecF8Cfg {
   static constexpr int kRawBytes = 128 * 128;            // one e4m3 tile
   static constexpr int kGroups = NG_;
@@ -106,7 +109,8 @@ struct DecF8Cfg {
   static constexpr int kPPerGroup = 4;                   // P8^T slots of a stream: how far its softmax group may run ahead of its PVs
   static constexpr int kStreamBytes = (kKStages + kVStages) * kRawBytes + kQBytes + 2 * kQ8Bytes + kPPerGroup * kP8Bytes;
   static constexpr int kSmemBytes = kGroups * kStreamBytes + 1024;
-  static constexpr int kThreads = 32 * (4 * kGroups) + 128 * kGroups + 128;   // issuing warps, softmax groups, epilogue group
+  static constexpr int kHalves = kSplit_ ? 2 : 1;        // warpgroups of a stream's softmax group
+  static constexpr int kThreads = 32 * (4 * kGroups) + 128 * kGroups * kHalves + 128;   // issuing warps, softmax groups, epilogue group
   static constexpr uint32_t kColsPerStream = 96;         // S^T ring 4 x 16, O^T 2 x 16 (item parity)
   static constexpr uint32_t kTmemCols = kGroups * kColsPerStream <= 128 ? 128 : 256;
 };
@@ -149,11 +153,14 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
 // them to the softmax group with the scores, so that the softmax chain carries no address arithmetic and no loads
 // (with the softmax group requesting the next tile's scales itself, a tile ahead, the contiguous step was 6 % slower).
 template <bool kDense, int GP, bool kPaged = false, int NG_ = 2>
-__global__ void __launch_bounds__(DecF8Cfg<NG_, kDense>::kThreads, 1)
+__global__ void __launch_bounds__(DecF8Cfg<NG_, kDense, (GP > 4)>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
-  using Cfg = DecF8Cfg<NG_, kDense>;
+  using Cfg = DecF8Cfg<NG_, kDense, (GP > 4)>;
   constexpr int RB = Cfg::kRawBytes, NK = Cfg::kKStages, NV = Cfg::kVStages, NG = Cfg::kGroups, PP = Cfg::kPPerGroup;
+  constexpr bool kSplit = GP > 4;          // two threads per key, four heads each
+  constexpr int HS = Cfg::kHalves;
+  constexpr int GS = kSplit ? 4 : GP;      // heads a softmax thread carries
   static_assert(!kDense || NK == NV, "the dense producer walks both rings with one index");
   constexpr int GH = GP;                   // rows of a softmax group
   constexpr int HALF = GP > 4 ? 8 : 4;     // rows (MMA columns) of the leading parts; the remainders follow them
@@ -167,14 +174,14 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   // per stream
   __shared__ uint64_t qr_full[NG], qr_free[NG], q8_free[NG][2], kr_full[NG][NK], kr_empty[NG][NK], v_full[NG][NV],
       v_empty[NG][NV], s_full[NG][4], s_free[NG][4], vote_bar[NG][4], vote_read[NG][4], p_full[NG][PP], p_free[NG][PP],
-      item_done[NG][2], st_full[NG][2], o_free[NG][2], grp_bar[NG], ret_full[NG][8], ret_free[NG][8], fin_bar[NG];
+      item_done[NG][2], st_full[NG][2], o_free[NG][2], grp_bar[NG][2], ret_full[NG][8], ret_free[NG][8], fin_bar[NG];
   __shared__ uint32_t tmem_base_s;
-  __shared__ int flag[NG][4];
+  __shared__ int flag[NG][2][8];           // [stream][half of the softmax group][tile g & 7]: that half's vote
   __shared__ int ret_ring[NG][8];          // decision of the stream's tile g at g & 7 (vote warp -> PV warp)
   __shared__ int t_row[NG][8], t_outer[NG][8], t_sidx[NG][8];   // TMA coordinates and scale index of tile g (producer ->)
   __shared__ float sc_k[NG][4], sc_v[NG][4];                    // the scales of the tile in S^T slot g & 3 (S warp -> softmax)
   __shared__ float q_inv[NG][2][8];        // 2^-k of the query rows of a stream's item
-  __shared__ __align__(16) float xch[NG][2][4][16];        // [stream][buffer][warp][row maxima 0..7, row sums 8..15]
+  __shared__ __align__(16) float xch[NG][2][2][4][16];     // [stream][half][buffer][warp][row maxima 0..7, row sums 8..15]
   __shared__ __align__(16) float st_m[NG][2][8], st_l[NG][2][8], st_y[NG][2][8];   // a finished item's (m, l, yref)
   __shared__ int st_r[NG][2];                              // ... and its retained tiles
   __shared__ int early_exit;
@@ -200,19 +207,22 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   if (tid == 0) {
     early_exit = (*(volatile int*)status != 0);
     for (int k = 0; k < NG; ++k) {
-      mbar_init(&grp_bar[k], 4); mbar_init(&fin_bar[k], 1); mbar_init(&qr_full[k], 1); mbar_init(&qr_free[k], 1);
+      mbar_init(&grp_bar[k][0], 4); mbar_init(&grp_bar[k][1], 4);
+      mbar_init(&fin_bar[k], 1); mbar_init(&qr_full[k], 1); mbar_init(&qr_free[k], 1);
       for (int i = 0; i < 2; ++i) {
         mbar_init(&q8_free[k][i], 1);
-        mbar_init(&item_done[k][i], 1); mbar_init(&st_full[k][i], 1); mbar_init(&o_free[k][i], 4);
+        mbar_init(&item_done[k][i], 1); mbar_init(&st_full[k][i], HS); mbar_init(&o_free[k][i], 4);
       }
-      for (int s = 0; s < PP; ++s) { mbar_init(&p_full[k][s], 4); mbar_init(&p_free[k][s], 1); }
+      for (int s = 0; s < PP; ++s) { mbar_init(&p_full[k][s], 4 * HS); mbar_init(&p_free[k][s], 1); }
       for (int s = 0; s < NK; ++s) { mbar_init(&kr_full[k][s], 1); mbar_init(&kr_empty[k][s], 1); }
       for (int s = 0; s < NV; ++s) { mbar_init(&v_full[k][s], 1); mbar_init(&v_empty[k][s], 1); }
       for (int s = 0; s < 4; ++s) {
-        mbar_init(&s_full[k][s], 1); mbar_init(&s_free[k][s], 4); mbar_init(&vote_bar[k][s], 1); mbar_init(&vote_read[k][s], 1);
-        flag[k][s] = 0;
+        mbar_init(&s_full[k][s], 1); mbar_init(&s_free[k][s], 4 * HS); mbar_init(&vote_bar[k][s], HS); mbar_init(&vote_read[k][s], 1);
       }
-      for (int s = 0; s < 8; ++s) { mbar_init(&ret_full[k][s], 1); mbar_init(&ret_free[k][s], 1); }
+      for (int s = 0; s < 8; ++s) {
+        mbar_init(&ret_full[k][s], 1); mbar_init(&ret_free[k][s], 1);
+        flag[k][0][s] = flag[k][1][s] = 0;
+      }
     }
     mbar_fence_init();
   }
@@ -399,7 +409,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ok = mbar_wait_warp(&vote_bar[k][g & 3], (uint32_t)((g >> 2) & 1), status);
             if (ok && g >= 8) ok = mbar_wait_warp(&ret_free[k][g & 7], (uint32_t)(((g >> 3) - 1) & 1), status);
             if (!ok) break;
-            const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[k][g & 3], 0) != 0;
+            const bool retain = __shfl_sync(0xffffffffu, *(volatile int*)&flag[k][0][g & 7] |
+                                                                  (kSplit ? *(volatile int*)&flag[k][1][g & 7] : 0), 0) != 0;
             __syncwarp();
             if (leader) mbar_arrive(&vote_read[k][g & 3]);
             if (retain) {
@@ -470,7 +481,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       mbar_wait_warp(&fin_bar[k], 0, status);
     }
     if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 400000) {} }
-  } else if (warp >= 8 * NG) {
+  } else if (warp >= 4 * NG + 4 * NG * HS) {
     // ------------------------------------------------------------------ epilogue group: thread = output channel
     // An item is written out when its last PV has completed and its stream has left its state: the partial output,
     // normalised by the split's own normalizer, and the log-sum-exp are stored and the item's accumulator and state
@@ -537,7 +548,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     }
   } else {
     // ------------------------------------------------------------------ softmax group of stream k: thread = key of the tile
-    const int k = (warp - 4 * NG) >> 2;
+    const int k = (warp - 4 * NG) / (4 * HS);
+    const int half = kSplit ? (((warp - 4 * NG) >> 2) & 1) : 0;   // which four of the (up to) eight heads
+    const int hb = half * 4;
     const int item0 = (int)blockIdx.x + k * (int)gridDim.x;
     uint8_t* sP = sP_of(k);
     const uint32_t colS = (uint32_t)k * Cfg::kColsPerStream, colO0 = colS + 64u;
@@ -545,8 +558,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const uint32_t lane_base = (uint32_t)w * 32u;
     const int kt = (int)lane_base + lane;
     const float c2 = p.scale_log2;
-    const bool head = (kt == 0);
-    constexpr int kLanesPerRow = 32 / GH;
+    const bool head = (kt == 0);               // (of this half: casts its vote, leaves its state)
+    constexpr int kLanesPerRow = 32 / GS;
     const int pub_row = lane / kLanesPerRow;
     const bool publisher = (lane % kLanesPerRow) == 0;
     int ne = 0, g = 0;                           // items and tiles of this stream so far
@@ -558,25 +571,25 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // adds the sums to l.
     float psum_w = 0.f;                          // this warp's sum of row pub_row, last retained tile
     bool pending_sum = false;
-    auto exchange = [&](float mx_w, float (&tmax)[GH], float (&l)[GH], float (&lgl)[GH]) -> bool {
+    auto exchange = [&](float mx_w, float (&tmax)[GS], float (&l)[GS], float (&lgl)[GS]) -> bool {
       const int xb = xc & 1;
-      if (publisher) { xch[k][xb][w][pub_row] = mx_w; xch[k][xb][w][8 + pub_row] = psum_w; }
+      if (publisher) { xch[k][half][xb][w][pub_row] = mx_w; xch[k][half][xb][w][8 + pub_row] = psum_w; }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&grp_bar[k]);
-      bool kk = mbar_wait(&grp_bar[k], xc & 1, status);
+      if (lane == 0) mbar_arrive(&grp_bar[k][half]);
+      bool kk = mbar_wait(&grp_bar[k][half], xc & 1, status);
       kk = __all_sync(0xffffffffu, kk);
       ++xc;
       if (!kk) return false;
-      float a0[GH], a1[GH], a2[GH], a3[GH];
-      lds_row<GH>(xch[k][xb][0], a0); lds_row<GH>(xch[k][xb][1], a1);
-      lds_row<GH>(xch[k][xb][2], a2); lds_row<GH>(xch[k][xb][3], a3);
+      float a0[GS], a1[GS], a2[GS], a3[GS];
+      lds_row<GS>(xch[k][half][xb][0], a0); lds_row<GS>(xch[k][half][xb][1], a1);
+      lds_row<GS>(xch[k][half][xb][2], a2); lds_row<GS>(xch[k][half][xb][3], a3);
 #pragma unroll
-      for (int q = 0; q < GH; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
+      for (int q = 0; q < GS; ++q) tmax[q] = fmaxf(fmaxf(a0[q], a1[q]), fmaxf(a2[q], a3[q]));
       if (pending_sum) {
-        lds_row<GH>(xch[k][xb][0] + 8, a0); lds_row<GH>(xch[k][xb][1] + 8, a1);
-        lds_row<GH>(xch[k][xb][2] + 8, a2); lds_row<GH>(xch[k][xb][3] + 8, a3);
+        lds_row<GS>(xch[k][half][xb][0] + 8, a0); lds_row<GS>(xch[k][half][xb][1] + 8, a1);
+        lds_row<GS>(xch[k][half][xb][2] + 8, a2); lds_row<GS>(xch[k][half][xb][3] + 8, a3);
 #pragma unroll
-        for (int q = 0; q < GH; ++q) {
+        for (int q = 0; q < GS; ++q) {
           l[q] += (a0[q] + a1[q]) + (a2[q] + a3[q]);
           lgl[q] = __log2f(l[q]);
         }
@@ -595,17 +608,27 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const int nk = keys_of(b);                 // keys of the sequence: the L of Eq. 3 and the tail mask
       const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(nk, 1)));
       int r = 0;                                 // tiles of the item retained so far
-      float m_ref[GH], l[GH], yref[GH], lgl[GH], c2q[GH];
+      float m_ref[GS], l[GS], yref[GS], lgl[GS], c2q[GS];
 #pragma unroll
-      for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; lgl[q] = -INFINITY; c2q[q] = c2; }
+      for (int q = 0; q < GS; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; lgl[q] = -INFINITY; c2q[q] = c2; }
       for (int t = 0; t < T; ++t, ++g) {
         const int sb = g & 3;
         ok = mbar_wait(&s_full[k][sb], (uint32_t)((g >> 2) & 1), status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        uint32_t sr[LDN];
-        tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colS + (uint32_t)sb * 16u), sr);
+        // the leading parts and the remainders of this thread's heads
+        uint32_t sr[kSplit ? 4 : LDN], sr2[kSplit ? 4 : 1];
+        if constexpr (kSplit) {
+          tmem_ld_cols<4>(tmem_addr(tb, lane_base, colS + (uint32_t)sb * 16u + (uint32_t)hb), sr);
+          tmem_ld_cols<4>(tmem_addr(tb, lane_base, colS + (uint32_t)sb * 16u + 8u + (uint32_t)hb), sr2);
+        } else {
+          tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colS + (uint32_t)sb * 16u), sr);
+        }
+        auto rem_of = [&](int q) -> float {
+          if constexpr (kSplit) return __uint_as_float(sr2[q]);
+          else return __uint_as_float(sr[HALF + q]);
+        };
         const float ks = *(volatile float*)&sc_k[k][sb], lv = __log2f(*(volatile float*)&sc_v[k][sb]);
         tmem_wait_ld();
         tc_fence_before();
@@ -613,18 +636,18 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (lane == 0) mbar_arrive(&s_free[k][sb]);
         if (t == 0) {
 #pragma unroll
-          for (int q = 0; q < GH; ++q) c2q[q] = c2 * *(volatile float*)&q_inv[k][ip][q];
+          for (int q = 0; q < GS; ++q) c2q[q] = c2 * *(volatile float*)&q_inv[k][ip][hb + q];
         }
         const int kpos = (j0 - t) * 128 + kt;
-        float x[GH], tmax[GH];
+        float x[GS], tmax[GS];
         {
-          float mx[GH];
+          float mx[GS];
 #pragma unroll
-          for (int q = 0; q < GH; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
-            x[q] = (kpos < nk && q < R) ? fmaf(__uint_as_float(sr[HALF + q]), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
+          for (int q = 0; q < GS; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
+            x[q] = (kpos < nk && hb + q < R) ? fmaf(rem_of(q), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
             mx[q] = x[q];
           }
-          RowReduce<GH, 16, true>::run(mx, lane);
+          RowReduce<GS, 16, true>::run(mx, lane);
           ok = exchange(mx[0], tmax, l, lgl);
           if (!ok) break;
         }
@@ -633,27 +656,34 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (!kDense && r > 0) {
           retain = false;
 #pragma unroll
-          for (int q = 0; q < GH; ++q) retain = retain || (q < R && !(((tmax[q] - (m_ref[q] + lgl[q])) - theta) < 0.f));
+          for (int q = 0; q < GS; ++q) retain = retain || (hb + q < R && !(((tmax[q] - (m_ref[q] + lgl[q])) - theta) < 0.f));
         }
         if (!kDense && head) {
-          *(volatile int*)&flag[k][g & 3] = retain ? 1 : 0;
+          *(volatile int*)&flag[k][half][g & 7] = retain ? 1 : 0;
           mbar_arrive(&vote_bar[k][g & 3]);
         }
+        if (!kDense && kSplit && !retain) {   // this half's heads would skip the tile: the other half's decide
+          ok = mbar_wait(&vote_bar[k][g & 3], (uint32_t)((g >> 2) & 1), status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          retain = (*(volatile int*)&flag[k][0][g & 7] | *(volatile int*)&flag[k][1][g & 7]) != 0;
+          retain = __all_sync(0xffffffffu, retain);
+        }
         if (!retain) continue;
-        if (head && bm_row) atomicOr(bm_row + ((T - 1 - t) >> 5), 1u << ((T - 1 - t) & 31));
+        if (head && half == 0 && bm_row) atomicOr(bm_row + ((T - 1 - t) >> 5), 1u << ((T - 1 - t) & 31));
         const int ps = rg % PP;
         if (r == 0) {
 #pragma unroll
-          for (int q = 0; q < GH; ++q) { m_ref[q] = tmax[q]; yref[q] = tmax[q] + lv; }   // (nothing accumulated yet)
+          for (int q = 0; q < GS; ++q) { m_ref[q] = tmax[q]; yref[q] = tmax[q] + lv; }   // (nothing accumulated yet)
         } else {
           // a maximum too far above a reference: the reference is raised, l follows here and O^T (whose earlier PVs
           // have to be complete) in TMEM
-          float alpha[GH];
+          float alpha[GS];
           bool touch = false;
 #pragma unroll
-          for (int q = 0; q < GH; ++q) {
+          for (int q = 0; q < GS; ++q) {
             alpha[q] = 1.f;
-            if (q < R && (tmax[q] + lv > yref[q] + kPGap || tmax[q] > m_ref[q] + kMGap)) {
+            if (hb + q < R && (tmax[q] + lv > yref[q] + kPGap || tmax[q] > m_ref[q] + kMGap)) {
               const float mn = fmaxf(m_ref[q], tmax[q]), yn = fmaxf(yref[q], tmax[q] + lv);
               l[q] *= fast_exp2(m_ref[q] - mn);
               alpha[q] = fast_exp2(yref[q] - yn);
@@ -667,15 +697,29 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            uint32_t o[LDN];
-            tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colO), o);
-            tmem_wait_ld();
+            if constexpr (kSplit) {
+              uint32_t o[4], o2[4];
+              tmem_ld_cols<4>(tmem_addr(tb, lane_base, colO + (uint32_t)hb), o);
+              tmem_ld_cols<4>(tmem_addr(tb, lane_base, colO + 8u + (uint32_t)hb), o2);
+              tmem_wait_ld();
 #pragma unroll
-            for (int q = 0; q < GH; ++q) {
-              o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
-              o[HALF + q] = __float_as_uint(__uint_as_float(o[HALF + q]) * alpha[q]);
+              for (int q = 0; q < 4; ++q) {
+                o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
+                o2[q] = __float_as_uint(__uint_as_float(o2[q]) * alpha[q]);
+              }
+              tmem_st_cols<4>(tmem_addr(tb, lane_base, colO + (uint32_t)hb), o);
+              tmem_st_cols<4>(tmem_addr(tb, lane_base, colO + 8u + (uint32_t)hb), o2);
+            } else {
+              uint32_t o[LDN];
+              tmem_ld_cols<LDN>(tmem_addr(tb, lane_base, colO), o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int q = 0; q < GS; ++q) {
+                o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha[q]);
+                o[HALF + q] = __float_as_uint(__uint_as_float(o[HALF + q]) * alpha[q]);
+              }
+              tmem_st_cols<LDN>(tmem_addr(tb, lane_base, colO), o);
             }
-            tmem_st_cols<LDN>(tmem_addr(tb, lane_base, colO), o);
             tmem_wait_st();
             tc_fence_before();
           }
@@ -685,33 +729,39 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
         }
-        float e[GH], pp[GH];
+        float e[GS], pp[GS];
 #pragma unroll
-        for (int q = 0; q < GH; ++q) {
-          e[q] = (q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
+        for (int q = 0; q < GS; ++q) {
+          e[q] = (hb + q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
           // P' = 64 exp2(x + lv - yref) = e * 64 exp2(m + lv - yref): the tile's V scale rides on the probability
-          pp[q] = (q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
+          pp[q] = (hb + q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
         }
-        {   // the key's 16 bytes: leading parts of the heads, their remainders (zeros behind them with up to four heads)
-          uint32_t lead[2] = {0u, 0u}, rem[2] = {0u, 0u};
-          if constexpr (GH == 1) {
+        {   // the key's 16 bytes: leading parts of the heads, their remainders (zeros behind them with up to four heads;
+            // with more, each half of the group writes its four bytes of either)
+          uint32_t lead = 0u, rem = 0u;
+          if constexpr (GS == 1) {
             const uint2 s0 = split_e4m3x2(pp[0], 0.f);
-            lead[0] = s0.x & 0xffu; rem[0] = s0.y & 0xffu;
+            lead = s0.x & 0xffu; rem = s0.y & 0xffu;
           } else {
 #pragma unroll
-            for (int q = 0; q < GH; q += 2) {
+            for (int q = 0; q < GS; q += 2) {
               const uint2 s01 = split_e4m3x2(pp[q], pp[q + 1]);
-              lead[q >> 2] |= (s01.x & 0xffffu) << (8 * (q & 3));
-              rem[q >> 2] |= (s01.y & 0xffffu) << (8 * (q & 3));
+              lead |= (s01.x & 0xffffu) << (8 * q);
+              rem |= (s01.y & 0xffffu) << (8 * q);
             }
           }
-          *reinterpret_cast<uint4*>(sP + ps * Cfg::kP8Bytes + kt * 16) =
-              HALF == 4 ? make_uint4(lead[0], rem[0], 0u, 0u) : make_uint4(lead[0], lead[1], rem[0], rem[1]);
+          uint8_t* prow = sP + ps * Cfg::kP8Bytes + kt * 16;
+          if constexpr (kSplit) {
+            *reinterpret_cast<uint32_t*>(prow + hb) = lead;
+            *reinterpret_cast<uint32_t*>(prow + 8 + hb) = rem;
+          } else {
+            *reinterpret_cast<uint4*>(prow) = make_uint4(lead, rem, 0u, 0u);
+          }
         }
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[k][ps]);
-        RowReduce<GH, 16, false>::run(e, lane);   // (the sums cross the group with the next tile's maxima)
+        RowReduce<GS, 16, false>::run(e, lane);   // (the sums cross the group with the next tile's maxima)
         psum_w = e[0];
         pending_sum = true;
         ++r;
@@ -719,7 +769,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       if (!ok) break;
       if (pending_sum) {   // the last retained tile's sums
-        float unused[GH];
+        float unused[GS];
         ok = exchange(-INFINITY, unused, l, lgl);
         if (!ok) break;
       }
@@ -731,8 +781,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (ne >= 2) ok = mbar_wait(&o_free[k][ip], (uint32_t)(((ne >> 1) - 1) & 1), status);
         if (ok) {
 #pragma unroll
-          for (int q = 0; q < GH; ++q) { st_m[k][ip][q] = m_ref[q]; st_l[k][ip][q] = l[q]; st_y[k][ip][q] = yref[q]; }
-          *(volatile int*)&st_r[k][ip] = r;
+          for (int q = 0; q < GS; ++q) { st_m[k][ip][hb + q] = m_ref[q]; st_l[k][ip][hb + q] = l[q]; st_y[k][ip][hb + q] = yref[q]; }
+          if (half == 0) *(volatile int*)&st_r[k][ip] = r;
           mbar_arrive(&st_full[k][ip]);
         }
       }
