@@ -40,8 +40,10 @@ def test_host_only_queries(mala):
     assert mala.tile_shape(mala.OP_FWD, 128) == (128, 128)
     assert mala.tile_shape(mala.OP_BWD, 64) == (128, 128)
     assert mala.tile_shape(mala.OP_DECODE, 128) == (0, 128)
-    with pytest.raises(mala.MalaError):
-        mala.tile_shape(mala.OP_FWD, 256)
+    assert mala.tile_shape(mala.OP_FWD, 256) == (128, 128) and mala.tile_shape(mala.OP_DECODE, 200) == (0, 128)
+    for op, d in ((mala.OP_FWD, 264), (mala.OP_BWD, 256), (mala.OP_BWD, 136), (mala.OP_DECODE, 512)):
+        with pytest.raises(mala.MalaError):   # the forward and the decode step take up to 256 columns, the backward 128
+            mala.tile_shape(op, d)
     # backward scratch: fp32 dQ accumulator + three fp32 per-row vectors, rows padded to whole tiles
     assert mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 64) == 2 * 1024 * 64 * 4 + 3 * 2 * 1024 * 4 + 256 + 256
     # (head sizes between the two kernel widths take the wider one's scratch)
@@ -49,6 +51,9 @@ def test_host_only_queries(mala):
     assert mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 40, 8) == mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 64, 8)
     assert mala.workspace_bytes(mala.OP_DECODE, 8, 32, 8, 131072, 128, 128) == 8 * 32 * 128 * 128 * 4 + 8 * 32 * 128 * 4
     assert mala.workspace_bytes(mala.OP_DECODE, 8, 32, 8, 131072, 128, 0) == 0
+    assert mala.workspace_bytes(mala.OP_DECODE, 8, 16, 4, 131072, 256, 128) == 8 * 16 * 128 * 256 * 4 + 8 * 16 * 128 * 4
+    assert mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 136, 8) == mala.workspace_bytes(mala.OP_DECODE, 2, 8, 2, 4096, 256, 8)
+    assert mala.workspace_bytes(mala.OP_BWD, 1, 2, 2, 1000, 256) == 0     # (no backward above 128 columns)
     assert mala.lib().mala_strerror(-4).decode() == "workspace too small"
     # split count for decode: the smallest one that fills the SMs evenly (queue = items per SM x tiles per item)
     # with at least six items per SM and two tiles per split
@@ -79,7 +84,7 @@ def test_argument_validation_codes(mala):
     assert f(B=0) == -1 and f(N=-3) == -1
     assert f(tau=-1.0) == -1 and f(tau=float("nan")) == -1 and f(scale=0.0) == -1 and f(scale=float("inf")) == -1
     assert f(lse=None) == -1
-    assert f(d=256) == -2 and f(d=100) == -2 and f(d=0) == -2 and f(Hq=3, Hkv=2) == -2
+    assert f(d=264) == -2 and f(d=512) == -2 and f(d=100) == -2 and f(d=0) == -2 and f(Hq=3, Hkv=2) == -2
     assert f(q=tin(off=2)) == -3 and f(q=tin(sn=130)) == -3
     # decode: too many packed heads, bad split count
     g = lambda **kw: L.mala_decode(tin(), tin(), tin(), tout(), None, None, 1, kw.get("Hq", 4), kw.get("Hkv", 1), 256,
@@ -89,6 +94,9 @@ def test_argument_validation_codes(mala):
     h = lambda ws, n: L.mala_bwd(tin(), tin(), tin(), tin(), tin(), base, tout(), tout(), tout(), None, 1, 2, 2, 4, 128,
                                  1, 0.1, 1e-4, ws, n, None)
     assert h(base, 16) == -4 and h(base + 16, 1 << 20) == -3
+    h256 = L.mala_bwd(tin(), tin(), tin(), tin(), tin(), base, tout(), tout(), tout(), None, 1, 2, 2, 4, 256, 1, 0.1,
+                      1e-4, base, 1 << 20, None)
+    assert h256 == -2                                                    # the backward stops at 128 columns
     if not torch.cuda.is_available():
         # valid arguments on a machine without a GPU: a loud CUDA error, never a silent fallback
         assert f() in (-5, -6)
