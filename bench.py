@@ -922,6 +922,20 @@ def main():
                               "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
             f8["paged_256"] = pg8
             del kp8, vp8, bt8, ksp, vsp
+            # ... and in 16-key pages (eight copies per tile; one scale per page, quantised page by page)
+            kp, vp, bt16, _ = W.paginate(kc, vc, 16, seed=7)
+            kp8, ksp, _ = W.quantize_cache_e4m3(kp, tile=16)
+            vp8, vsp, _ = W.quantize_cache_e4m3(vp, tile=16)
+            del kp, vp
+            pg8 = {}
+            for label, t_ in (("mala", tau), ("dense", 0.0)):
+                us = 1e3 * time_cuda(lambda: mala.decode_fp8_paged(qd, kp8, vp8, ksp, vsp, bt16, None, wd["scale"], t_,
+                                                                    dcfg.num_splits, ws=wsd, out=od, want_lse=False), 25, 100)
+                need = f8["key_major"][label]["needed_gb"] * 1e9
+                pg8[label] = {"us": us, "achieved_gbs": need / (us * 1e-6) / 1e9,
+                              "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+            f8["paged_16"] = pg8
+            del kp8, vp8, bt16, ksp, vsp
             row["e4m3_cache"] = f8
             del k8, v8, ks8, vs8
             # half the KV heads with 256 columns each (the same bytes per key): 64 KB tiles, two output accumulators

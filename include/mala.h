@@ -206,9 +206,11 @@ int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float*
 
 /* mala_decode_fp8 over a paged 8-bit cache with one length per sequence: the layout of mala_decode_paged (one new token
  * per sequence) with the storage of mala_decode_fp8.  kpages8, vpages8: 8-bit [num_pages, page_size, Hkv, d] views
- * (strides in elements = bytes, multiples of 16), page_size a multiple of 128 (MALA_ERR_UNSUPPORTED otherwise: a scale
- * belongs to a 128-key tile of a page); kscale, vscale: device fp32 [num_pages, Hkv, page_size/128], the scale of
- * tile y of page x at [x][h][y].  block_table, seqlens, the split layout (Nk = max_pages_per_seq*page_size), the
+ * (strides in elements = bytes, multiples of 16), page_size a multiple of 128, or 16, 32 or 64 (MALA_ERR_UNSUPPORTED
+ * otherwise); kscale, vscale: device fp32 [num_pages, Hkv, max(1, page_size/128)], the scale of tile y of page x at
+ * [x][h][y] -- one scale per 128-key tile of a page, or one per page where a page is smaller than a tile (a tile is then
+ * put together from 128 / page_size pages, each key scaled by its own page's scale; the skip rule's tile stays 128
+ * keys).  block_table, seqlens, the split layout (Nk = max_pages_per_seq*page_size), the
  * clamping of seqlens, entries outside the pool (read as zeros) and telemetry as in mala_decode_paged; slots of a
  * mapped page beyond the sequence's length must hold codes other than e4m3's two NaN codes, 0x7f and 0xff (a
  * zero-initialised or recycled page does): their keys are masked out of the scores, but their values are multiplied by

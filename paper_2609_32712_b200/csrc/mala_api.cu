@@ -523,8 +523,10 @@ int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const 
                           int max_pages_per_seq, int d, float scale, float tau, int num_splits, void* ws, size_t ws_bytes,
                           void* cuda_stream) {
   if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
-  if (page_size % 128 != 0 || (long long)max_pages_per_seq * page_size > 0x7fffffffLL ||
-      (long long)num_pages * Hkv * (page_size / 128) > 0x7fffffffLL)
+  // pages of whole tiles, or of 16, 32 or 64 keys (a tile is then put together from several pages)
+  if (!(page_size % 128 == 0 || page_size == 16 || page_size == 32 || page_size == 64) ||
+      (long long)max_pages_per_seq * page_size > 0x7fffffffLL ||
+      (long long)num_pages * Hkv * (page_size < 128 ? 1 : page_size / 128) > 0x7fffffffLL)
     return MALA_ERR_UNSUPPORTED;
   const int Nk = max_pages_per_seq * page_size;   // the longest cache a sequence can hold
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));

@@ -51,7 +51,7 @@ inline bool decode_set_attributes() {
 #define MALA_DEC_ATTR_GP(GP) MALA_DEC_ATTR(false, GP, false) MALA_DEC_ATTR(true, GP, false) MALA_DEC_ATTR(false, GP, true) MALA_DEC_ATTR(true, GP, true)
   MALA_DEC_ATTR_GP(1) MALA_DEC_ATTR_GP(2) MALA_DEC_ATTR_GP(4) MALA_DEC_ATTR_GP(8) MALA_DEC_ATTR_GP(16)
 #define MALA_F8_ATTR(DENSE, GP) \
-  ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess;
   MALA_F8_ATTR(false, 1) MALA_F8_ATTR(true, 1) MALA_F8_ATTR(false, 2) MALA_F8_ATTR(true, 2) MALA_F8_ATTR(false, 4) MALA_F8_ATTR(true, 4)
   MALA_F8_ATTR(false, 8) MALA_F8_ATTR(true, 8)
 #undef MALA_F8_ATTR
@@ -163,31 +163,36 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
 
 // Decode over an e4m3 cache with one fp32 scale per (sequence, KV head, 128-key tile): kc / vc are 8-bit [B,Nk,Hkv,d]
 // views (strides in elements), kscale / vscale fp32 [B,Hkv,ceil(Nk/128)].  Up to four query heads per KV head.
-// pg != null: kc / vc are [num_pages, page_size, Hkv, d] (page_size a multiple of 128), the scales
-// [num_pages, Hkv, page_size/128], and Nk = bt_stride * page_size lays out the splits.
+// pg != null: kc / vc are [num_pages, page_size, Hkv, d] (page_size a multiple of 128, or 16, 32 or 64), the scales
+// [num_pages, Hkv, max(1, page_size/128)], and Nk = bt_stride * page_size lays out the splits.
 inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* kscale, const float* vscale, mala_tout o,
                              float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                              float tau, int num_splits, void* ws, int* status, cudaStream_t stream,
                              const DecPaging* pg = nullptr) {
   const int G = Hq / Hkv;
   if (G > 8 || d % 16 != 0 || d > 128 || d < 16) return MALA_ERR_UNSUPPORTED;
-  if (pg && (pg->page_size < 128 || pg->page_size % 128 != 0)) return MALA_ERR_UNSUPPORTED;
+  const bool small = pg && pg->page_size < 128;
+  if (pg && !(pg->page_size % 128 == 0 || pg->page_size == 16 || pg->page_size == 32 || pg->page_size == 64))
+    return MALA_ERR_UNSUPPORTED;
+  const int box_rows = small ? pg->page_size : 128;
   const int per = (Nk + num_splits - 1) / num_splits;
   const int tps = (per + 127) / 128;
   if ((long long)B * Hkv * num_splits > 0x7fffffffLL || (long long)B * Hkv * ((Nk + 127) / 128) > 0x7fffffffLL)
     return MALA_ERR_UNSUPPORTED;
   CUtensorMap tq, tk, tv;
   if (!make_tensor_map_q_rows(&tq, q.p, B, 1, Hq, d, q.sb, 0, q.sh, G) ||
-      !make_tensor_map_u8_bnhd(&tk, kc.p, pg ? pg->num_pages : B, pg ? pg->page_size : Nk, Hkv, d, kc.sb, kc.sn, kc.sh) ||
-      !make_tensor_map_u8_bnhd(&tv, vc.p, pg ? pg->num_pages : B, pg ? pg->page_size : Nk, Hkv, d, vc.sb, vc.sn, vc.sh))
+      !make_tensor_map_u8_bnhd(&tk, kc.p, pg ? pg->num_pages : B, pg ? pg->page_size : Nk, Hkv, d, kc.sb, kc.sn, kc.sh, box_rows) ||
+      !make_tensor_map_u8_bnhd(&tv, vc.p, pg ? pg->num_pages : B, pg ? pg->page_size : Nk, Hkv, d, vc.sb, vc.sn, vc.sh, box_rows))
     return MALA_ERR_TENSOR_MAP;
   DecF8Params p;
   p.block_table = pg ? pg->block_table : nullptr;
   p.seqlens = pg ? pg->seqlens : nullptr;
   p.num_pages = pg ? pg->num_pages : 0;
   p.max_pages = pg ? pg->bt_stride : 0;
-  p.tpp = pg ? pg->page_size / 128 : 1;
+  p.tpp = (pg && !small) ? pg->page_size / 128 : 1;
   p.by_tpp.set((uint32_t)p.tpp);
+  p.ppt = 128 / box_rows;
+  p.prows = box_rows;
   p.o_part = (float*)ws;
   p.lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Hq * num_splits * 128 * sizeof(float)));
   p.retained = st ? st->retained_per_block : nullptr;
@@ -211,7 +216,8 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
   const int grid = p.n_items < sms ? p.n_items : sms;
 #define MALA_F8_LAUNCH(DENSE, GP)                                                                                      \
   do {                                                                                                                  \
-    if (pg) mala_decode_fp8_kernel<DENSE, GP, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    if (small) mala_decode_fp8_kernel<DENSE, GP, true, 2, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    else if (pg) mala_decode_fp8_kernel<DENSE, GP, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
     else mala_decode_fp8_kernel<DENSE, GP, false><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p);  \
   } while (0)
   const bool dense = (tau == 0.f);

@@ -89,6 +89,10 @@ struct DecF8Params {
   const int32_t* seqlens;        // [B] or null
   int num_pages, max_pages, tpp; // tpp = tiles (128 keys) per page
   FastDiv by_tpp;
+  // pages smaller than a tile (16, 32 or 64 keys; kSmall kernels): a tile is put together from ppt = 128 / page_size
+  // copies of prows = page_size rows, copy c of key block x from page block_table[b][x * ppt + c]; the scales are
+  // [num_pages, Hkv], one per (page, KV head)
+  int ppt, prows;
 };
 
 // NG_: streams (two: a third, with the registers moved from the issuing warps to the softmax groups and rings of two
@@ -152,7 +156,10 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
 // ring; the vote warp takes the V copy's coordinates from there, and the S warp loads the tile's two scales and hands
 // them to the softmax group with the scores, so that the softmax chain carries no address arithmetic and no loads
 // (with the softmax group requesting the next tile's scales itself, a tile ahead, the contiguous step was 6 % slower).
-template <bool kDense, int GP, bool kPaged = false, int NG_ = 2>
+// kSmall (with kPaged): pages smaller than a tile.  The producer and the vote warp issue a tile's copies from as many
+// lanes as it has pages, a key's scales are those of its page (a softmax thread is a key, so it reads its own), and
+// the reference of the 8-bit probabilities is kept against the largest V scale of the tile.
+template <bool kDense, int GP, bool kPaged = false, int NG_ = 2, bool kSmall = false>
 __global__ void __launch_bounds__(DecF8Cfg<NG_, kDense, (GP > 4)>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
@@ -178,8 +185,11 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __shared__ uint32_t tmem_base_s;
   __shared__ int flag[NG][2][8];           // [stream][half of the softmax group][tile g & 7]: that half's vote
   __shared__ int ret_ring[NG][8];          // decision of the stream's tile g at g & 7 (vote warp -> PV warp)
+  static_assert(!kSmall || kPaged, "small pages are pages");
   __shared__ int t_row[NG][8], t_outer[NG][8], t_sidx[NG][8];   // TMA coordinates and scale index of tile g (producer ->)
-  __shared__ float sc_k[NG][4], sc_v[NG][4];                    // the scales of the tile in S^T slot g & 3 (S warp -> softmax)
+  __shared__ int t_page[NG][8][8];                              // small pages: the up to eight pages of tile g
+  // the scales of the tile in S^T slot g & 3 (S warp -> softmax); small pages: one per page, and the largest V scale
+  __shared__ float sc_k[NG][4][8], sc_v[NG][4][8], sc_vmax[NG][4];
   __shared__ float q_inv[NG][2][8];        // 2^-k of the query rows of a stream's item
   __shared__ __align__(16) float xch[NG][2][2][4][16];     // [stream][half][buffer][warp][row maxima 0..7, row sums 8..15]
   __shared__ __align__(16) float st_m[NG][2][8], st_l[NG][2][8], st_y[NG][2][8];   // a finished item's (m, l, yref)
@@ -286,7 +296,46 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const uint32_t tO = tmem_addr(tb, 0, (uint32_t)k * Cfg::kColsPerStream + 64u);    // its two accumulators
     const uint32_t leader = elect_one();
     bool ok = true;
-    if (job == 0) {
+    if (job == 0 && kSmall) {
+      // ---- TMA producer, pages smaller than a tile: the loop below run by all 32 lanes (waits and counters
+      //      warp-uniform); lane c looks up the page of copy c and issues that copy
+      if (lane == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); }
+      int ne = 0, g = 0;
+      for (int item = item0; item < p.n_items && ok; item += item_step) {
+        const int T = tiles_of(item);
+        if (T == 0) continue;
+        int b, hkv, split, j0;
+        geometry(item, b, hkv, split, j0, T);
+        if (ne >= 1) ok = mbar_wait_warp(&qr_free[k], (uint32_t)((ne - 1) & 1), status);
+        if (!ok) break;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(&qr_full[k], (uint32_t)R * 128u * 2u);
+          for (int pn = 0; pn < 2; ++pn)
+            tma_load_4d(sQ + pn * HALF * 128, &tmQ, &qr_full[k], pn * 64, hkv * G, 0, b);
+        }
+        for (int t = 0; t < T && ok; ++t, ++g) {
+          const int s = g % NK;
+          const uint32_t ph = (uint32_t)((g / NK) & 1);
+          const int x = (j0 - t) * p.ppt + lane;   // (a table entry past the row's end reads as "no page": zeros)
+          const int pg = (lane < p.ppt && x < p.max_pages) ? __ldg(p.block_table + (size_t)b * p.max_pages + x) : -1;
+          ok = mbar_wait_warp(&kr_empty[k][s], ph ^ 1u, status);
+          if (!ok) break;
+          if (lane < 8) t_page[k][g & 7][lane] = pg;
+          __syncwarp();
+          if (lane == 0) mbar_arrive_expect_tx(&kr_full[k][s], RB);
+          __syncwarp();
+          if (lane < p.ppt) tma_load_4d(sKr + s * RB + lane * p.prows * 128, &tmK, &kr_full[k][s], 0, 0, hkv, pg);
+          if (kDense) {
+            ok = mbar_wait_warp(&v_empty[k][s], ph ^ 1u, status);
+            if (!ok) break;
+            if (lane == 0) mbar_arrive_expect_tx(&v_full[k][s], RB);
+            __syncwarp();
+            if (lane < p.ppt) tma_load_4d(sVr + s * RB + lane * p.prows * 128, &tmV, &v_full[k][s], 0, 0, hkv, pg);
+          }
+        }
+        ++ne;
+      }
+    } else if (job == 0) {
       // ---- TMA producer
       if (lane == 0) {
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -334,6 +383,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int T = tiles_of(item);
         if (T == 0) continue;
         const int ip = ne & 1;
+        int b_, hkv_ = 0, split_, j0_;
+        if constexpr (kSmall) geometry(item, b_, hkv_, split_, j0_, T);
         uint8_t* q8 = sQ8 + ip * Cfg::kQ8Bytes;
         // the item's queries have landed: row qh (128 bf16 in two 64-column panels, rows qh and HALF + qh of the
         // landing buffer; lane = four consecutive columns) becomes rows qh and HALF + qh of the e4m3 operand, once the
@@ -374,10 +425,23 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           }
           if (ok) ok = mbar_wait_warp(&kr_full[k][kc], (uint32_t)((g / NK) & 1), status);
           if (!ok) break;
-          if (leader) {   // the tile's scales travel with its scores (a page without scales holds zeros: any scale does)
+          if constexpr (kSmall) {   // one pair of scales per page of the tile, and the largest V scale
+            const int pg = lane < 8 ? *(volatile int*)&t_page[k][g & 7][lane] : -1;
+            const bool there = lane < p.ppt && pg >= 0 && pg < p.num_pages;
+            const float vsc = there ? __ldg(p.vscale + (size_t)pg * p.Hkv + hkv_) : 1.f;
+            if (lane < 8) {
+              sc_k[k][sb][lane] = there ? __ldg(p.kscale + (size_t)pg * p.Hkv + hkv_) : 1.f;
+              sc_v[k][sb][lane] = vsc;
+            }
+            float vmx = lane < p.ppt ? vsc : 0.f;
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) vmx = fmaxf(vmx, __shfl_xor_sync(0xffffffffu, vmx, o));
+            if (lane == 0) sc_vmax[k][sb] = vmx;
+            __threadfence_block();
+          } else if (leader) {   // the tile's scales travel with its scores (a page without scales holds zeros: any scale does)
             const int sidx = *(volatile int*)&t_sidx[k][g & 7];
-            sc_k[k][sb] = sidx >= 0 ? __ldg(p.kscale + sidx) : 1.f;
-            sc_v[k][sb] = sidx >= 0 ? __ldg(p.vscale + sidx) : 1.f;
+            sc_k[k][sb][0] = sidx >= 0 ? __ldg(p.kscale + sidx) : 1.f;
+            sc_v[k][sb][0] = sidx >= 0 ? __ldg(p.vscale + sidx) : 1.f;
             __threadfence_block();
           }
           __syncwarp();
@@ -417,7 +481,13 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               const int vs = nv % NV;
               if (nv >= NV) ok = mbar_wait_warp(&v_empty[k][vs], (uint32_t)(((nv / NV) - 1) & 1), status);
               if (!ok) break;
-              if (leader) {
+              if constexpr (kSmall) {
+                if (lane == 0) mbar_arrive_expect_tx(&v_full[k][vs], RB);
+                __syncwarp();
+                if (lane < p.ppt)
+                  tma_load_4d(sVr + vs * RB + lane * p.prows * 128, &tmV, &v_full[k][vs], 0, 0, hkv,
+                              *(volatile int*)&t_page[k][g & 7][lane]);
+              } else if (leader) {
                 mbar_arrive_expect_tx(&v_full[k][vs], RB);
                 tma_load_4d(sVr + vs * RB, &tmV, &v_full[k][vs], 0, *(volatile int*)&t_row[k][g & 7], hkv,
                             *(volatile int*)&t_outer[k][g & 7]);
@@ -557,6 +627,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     const int w = warp & 3;
     const uint32_t lane_base = (uint32_t)w * 32u;
     const int kt = (int)lane_base + lane;
+    const int pi = kSmall ? kt / p.prows : 0;  // small pages: the page of the tile this key lies in
     const float c2 = p.scale_log2;
     const bool head = (kt == 0);               // (of this half: casts its vote, leaves its state)
     constexpr int kLanesPerRow = 32 / GS;
@@ -629,7 +700,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           if constexpr (kSplit) return __uint_as_float(sr2[q]);
           else return __uint_as_float(sr[HALF + q]);
         };
-        const float ks = *(volatile float*)&sc_k[k][sb], lv = __log2f(*(volatile float*)&sc_v[k][sb]);
+        // (small pages: the key's own page's scales; the reference of P' follows the tile's largest V scale)
+        const float ks = *(volatile float*)&sc_k[k][sb][pi], lvk = __log2f(*(volatile float*)&sc_v[k][sb][pi]);
+        const float lv = kSmall ? __log2f(*(volatile float*)&sc_vmax[k][sb]) : lvk;
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
@@ -734,7 +807,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int q = 0; q < GS; ++q) {
           e[q] = (hb + q < R) ? fast_exp2(x[q] - m_ref[q]) : 0.f;
           // P' = 64 exp2(x + lv - yref) = e * 64 exp2(m + lv - yref): the tile's V scale rides on the probability
-          pp[q] = (hb + q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lv) - yref[q])) : 0.f;
+          pp[q] = (hb + q < R) ? e[q] * (kPScale * fast_exp2((m_ref[q] + lvk) - yref[q])) : 0.f;
         }
         {   // the key's 16 bytes: leading parts of the heads, their remainders (zeros behind them with up to four heads;
             // with more, each half of the group writes its four bytes of either)

@@ -51,15 +51,16 @@ inline bool make_tensor_map_bnhd(CUtensorMap* out, const void* base, int B, int 
 }
 
 // Tensor map over an 8-bit [B, N, H, d] view (strides in elements = bytes): coordinates (c, n, h, b), box = 128 columns
-// x 128 rows (one 16 KB tile), 128-byte swizzle; columns beyond d and rows beyond N read as zero.
+// x box_rows rows (128: one 16 KB tile; fewer: one page smaller than a tile), 128-byte swizzle; columns beyond d and rows
+// beyond N read as zero.
 inline bool make_tensor_map_u8_bnhd(CUtensorMap* out, const void* base, int B, int N, int H, int d, int64_t sb,
-                                    int64_t sn, int64_t sh) {
+                                    int64_t sn, int64_t sh, int box_rows = 128) {
   PFN_tensorMapEncodeTiled enc = tensor_map_encoder();
   if (!enc) return false;
   cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
   auto legal = [&](int64_t s, int n) -> cuuint64_t { return (n == 1 || s <= 0) ? (cuuint64_t)((d + 15) / 16 * 16) : (cuuint64_t)s; };
   cuuint64_t strides[3] = {legal(sn, N), legal(sh, H), legal(sb, B)};
-  cuuint32_t box[4] = {128u, 128u, 1u, 1u};
+  cuuint32_t box[4] = {128u, (cuuint32_t)box_rows, 1u, 1u};
   cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
   CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

@@ -413,7 +413,7 @@ def decode_fp8(q, kcache8, vcache8, kscale, vscale, scale: float, tau: float, nu
 def decode_fp8_paged(q, kpages8, vpages8, kscale, vscale, block_table, seqlens, scale: float, tau: float, num_splits: int,
                      stats: bool = False, ws=None, out=None, want_lse: bool = True):
     """mala_decode_fp8_paged: q [B,1,Hq,d] bf16; kpages8, vpages8 e4m3 codes [num_pages, page_size, Hkv, d];
-    kscale, vscale fp32 [num_pages, Hkv, page_size/128]; block_table int32 [B, max_pages_per_seq]; seqlens int32 [B] or
+    kscale, vscale fp32 [num_pages, Hkv, max(1, page_size/128)]; block_table int32 [B, max_pages_per_seq]; seqlens int32 [B] or
     None.  Returns (o [B,1,Hq,d] bf16, lse [B,Hq] fp32 or None, Stats or None)."""
     B, one, Hq, d = q.shape
     assert one == 1
@@ -421,7 +421,7 @@ def decode_fp8_paged(q, kpages8, vpages8, kscale, vscale, block_table, seqlens, 
     assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.shape[0] == B
     assert seqlens is None or (seqlens.dtype == torch.int32 and seqlens.is_contiguous() and seqlens.shape == (B,))
     for t in (kscale, vscale):
-        assert t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (num_pages, Hkv, page_size // 128)
+        assert t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (num_pages, Hkv, max(1, page_size // 128))
     max_pages = block_table.shape[1]
     Nk = max_pages * page_size
     o = torch.empty_like(q) if out is None else out

@@ -402,8 +402,9 @@ def _run_fp8_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0)
     into pages of a shuffled pool (junk in unused slots, table entries outside the pool), the pool is quantised page by
     page (one scale per 128-key tile of a page), and the oracle is handed scale * e4m3(code)."""
     kp, vp, bt, lens = W.paginate(w["kcache"], w["vcache"], page_size, seqlens=seqlens, seed=seed)
-    k8, ks, kd = W.quantize_cache_e4m3(kp)      # (a pool [num_pages, page_size, Hkv, d] has the shape of a cache)
-    v8, vs, vd = W.quantize_cache_e4m3(vp)
+    # (a pool [num_pages, page_size, Hkv, d] has the shape of a cache; pages smaller than a tile: one scale per page)
+    k8, ks, kd = W.quantize_cache_e4m3(kp, tile=min(128, page_size))
+    v8, vs, vd = W.quantize_cache_e4m3(vp, tile=min(128, page_size))
     q = w["q"].cuda()
     B, _, Hq, d = q.shape
     Hkv = kp.shape[2]
@@ -447,6 +448,10 @@ def _run_fp8_paged(mala, oracle, w, tau, num_splits, page_size, seqlens, seed=0)
     (8192, 64, 8, 2, 128, [8192, 5000, 128, 3333]),    # more work items than SMs, one tile each
     (6144, 6, 4, 4, 384, [6144, 6000, 385, 3000, 17]), # three tiles per page, one head per KV head
     (4096, 8, 16, 2, 256, [4096, 2049, 300]),          # eight heads per KV head
+    (2048, 4, 8, 2, 16, [2048, 1000, 129, 5]),         # pages of 16 keys: eight per tile, a scale per page
+    (1536, 3, 4, 1, 32, [1, 1536, 0, 700]),            # pages of 32 keys
+    (4096, 16, 16, 2, 64, [4096, 2049, 300]),          # pages of 64 keys, eight heads per KV head
+    (1040, 2, 6, 2, 16, [1040, 1025, 17]),             # a table whose last tile is partly past the row's end
 ])
 def test_decode_fp8_paged_literal(mala, oracle, Nk, S, Hq, Hkv, page, lens, tau):
     B = 2 if lens is None else len(lens)
@@ -479,11 +484,32 @@ def test_decode_fp8_paged_identity_table_equals_contiguous_call(mala):
         assert torch.equal(o0, o1) and torch.equal(l0, l1)
 
 
-def test_decode_fp8_paged_rejects_pages_that_are_not_whole_tiles(mala):
+def test_decode_fp8_paged_rejects_page_sizes_it_does_not_support(mala):
     w = W.custom_decode(1, 4, 1, 512, 128, 1, seed=1, device="cuda")
-    k8 = torch.zeros((8, 64, 1, 128), dtype=torch.uint8, device="cuda")       # pages of 64 keys
-    sc = torch.ones((8, 1, 0), dtype=torch.float32, device="cuda")            # (no whole tile, hence no scale)
-    bt = torch.arange(8, dtype=torch.int32, device="cuda").view(1, 8)
-    with pytest.raises(mala.MalaError) as e:
-        mala.decode_fp8_paged(w["q"], k8, k8, sc, sc, bt, None, w["scale"], 0.0, 1)
-    assert e.value.code == -2
+    for page in (8, 48, 192):          # (pages of whole tiles, or of 16, 32 or 64 keys)
+        k8 = torch.zeros((8, page, 1, 128), dtype=torch.uint8, device="cuda")
+        sc = torch.ones((8, 1, max(1, page // 128)), dtype=torch.float32, device="cuda")
+        bt = torch.arange(8, dtype=torch.int32, device="cuda").view(1, 8)
+        with pytest.raises(mala.MalaError) as e:
+            mala.decode_fp8_paged(w["q"], k8, k8, sc, sc, bt, None, w["scale"], 0.0, 1)
+        assert e.value.code == -2
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+@pytest.mark.parametrize("page", [16, 64])
+def test_decode_fp8_small_pages_gated_keys_skip_value_tiles(mala, oracle, page, tau):
+    w = W.custom_decode(3, 8, 2, 8192, 128, 8, group_types=["diffuse", "peaked"], seed=5, preset="D")
+    res = _run_fp8_paged(mala, oracle, w, tau, 8, page, [8192, 4096 + 77, 2500], seed=9)
+    assert res["skipped"] > 0, "workload must exercise skipping"
+
+
+def test_decode_fp8_small_pages_with_scales_far_apart(mala, oracle):
+    # the pages of a tile get V (and K) magnitudes a factor 2^10 apart: a key's probability is scaled by its own page's
+    # V scale while the 8-bit reference follows the tile's largest one
+    w = W.custom_decode(2, 4, 2, 2048, 128, 4, seed=77)
+    for name in ("kcache", "vcache"):
+        c = w[name].float()
+        f = torch.tensor([1.0, 2.0 ** -10, 2.0 ** -2, 2.0 ** -6])[(torch.arange(2048) // 16) % 4]
+        w[name] = (c * f[None, :, None, None] * (0.25 if name == "kcache" else 1.0)).to(torch.bfloat16)
+    for tau in (0.0, 1e-4):
+        _run_fp8_paged(mala, oracle, w, tau, 4, 16, [2048, 1500], seed=3)

@@ -170,3 +170,21 @@ def test_random_cases_decode_over_an_e4m3_cache(mala, oracle, seed):
         w = W.custom_decode(B, hkv * g, hkv, Nk, d, S, seed=rng.randint(0, 10**6), preset=preset)
         res = TD._run_fp8(mala, oracle, w, tau, S, rounding_bound=True)
         assert res["totals"][1] == res["retained"] + res["skipped"], (B, hkv, g, d, Nk, S, tau, preset)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_random_cases_decode_over_a_paged_e4m3_cache(mala, oracle, seed):
+    """Randomly drawn decode calls over an 8-bit cache in pages: pages of whole tiles and of 16, 32 and 64 keys (a
+    scale per page), group sizes 1 to 8, ragged lengths down to none, every tolerance, both presets."""
+    rng = random.Random(2000 + seed)
+    for it in range(10):
+        hkv, g = rng.choice([1, 2, 3]), rng.choice([1, 2, 4, 5, 8])
+        d = rng.choice([16, 64, 96, 128])
+        page = rng.choice([16, 32, 64, 128, 256])
+        B = rng.choice([1, 2, 4])
+        Nk = page * rng.randint(1, max(1, 6000 // page))
+        S = rng.choice([1, 2, 3, 8, 16])
+        tau = rng.choice([0.0, 1e-5, 1e-4, 1e-2, 1.0])
+        lens = [rng.choice([0, 1, Nk, rng.randint(0, Nk)]) for _ in range(B)]
+        w = W.custom_decode(B, hkv * g, hkv, Nk, d, S, seed=rng.randint(0, 10**6), preset=rng.choice(["literal", "D"]))
+        TD._run_fp8_paged(mala, oracle, w, tau, S, page, lens, seed=it)
