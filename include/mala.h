@@ -23,6 +23,11 @@
  *   - scale (> 0, finite) multiplies the fp32 scores; lse is in nats, of the scaled scores, over
  *     the retained set.  tau >= 0, finite.
  *   - Tile partition: mala_tile_shape() reports it; forward and backward use the same partition.
+ *   - Two environment variables, read once per process, change what a call does around its launches (both off by
+ *     default): MALA_NVTX=1 makes every launching call an NVTX range of its own name; MALA_DEBUG=1 makes error
+ *     reporting synchronous -- the call waits for its stream and returns MALA_ERR_CUDA or MALA_ERR_DEVICE_TIMEOUT
+ *     itself (with a line on stderr) instead of leaving the error to a later call.  A debug call therefore
+ *     synchronises, which a call otherwise never does.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t, may be NULL for the default
  *     stream), allocate nothing and never synchronise.  `ws` is caller-provided scratch of at
  *     least mala_workspace_bytes() bytes, 256-byte aligned; its contents are undefined afterwards.

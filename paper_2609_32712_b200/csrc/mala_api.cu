@@ -2,7 +2,11 @@
 // launches behind the C ABI declared in include/mala.h.  No torch types, no allocation, no sync.
 #include <cuda_runtime.h>
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <mutex>
+
+#include <nvtx3/nvToolsExt.h>
 
 #include "../../include/mala.h"
 #include "mala_bwd.cuh"
@@ -115,6 +119,45 @@ static int check_common(int B, int Hq, int Hkv, int N, int d, float scale, float
   if (B > 65535 || Hq > 65535) return MALA_ERR_UNSUPPORTED;
   return MALA_OK;
 }
+
+// Two environment variables, read once, change what a call does around its launches (both off by default):
+//   MALA_NVTX=1   every call that launches kernels is an NVTX range of its own name on the calling thread
+//   MALA_DEBUG=1  synchronous error reporting: the call waits for its stream, and a CUDA error or a recorded device
+//                 time-out comes back as the call's own return value (MALA_ERR_CUDA / MALA_ERR_DEVICE_TIMEOUT) with a line
+//                 on stderr, instead of surfacing at a later call.  (The call then synchronises, which it otherwise
+//                 never does; the status word stays set until mala_device_status clears it.)
+static int env_flag(const char* name) {
+  const char* v = getenv(name);
+  return (v && v[0] && v[0] != '0') ? 1 : 0;
+}
+static int nvtx_on() { static const int v = env_flag("MALA_NVTX"); return v; }
+static int debug_on() { static const int v = env_flag("MALA_DEBUG"); return v; }
+
+struct ApiScope {
+  const char* name;
+  cudaStream_t stream;
+  bool pushed;
+  ApiScope(const char* n, void* s) : name(n), stream((cudaStream_t)s), pushed(false) {
+    if (nvtx_on()) { nvtxRangePushA(name); pushed = true; }
+  }
+  ~ApiScope() { if (pushed) nvtxRangePop(); }
+  int finish(int rc) const {
+    if (rc != MALA_OK || !debug_on()) return rc;
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) {
+      fprintf(stderr, "[mala debug] %s: CUDA error %d (%s)\n", name, (int)e, cudaGetErrorString(e));
+      return MALA_ERR_CUDA;
+    }
+    int code = 0;
+    if (mala_device_status(&code, 0) != MALA_OK) return MALA_ERR_CUDA;
+    if (code != 0) {
+      fprintf(stderr, "[mala debug] %s: device status %d (a bounded wait expired)\n", name, code);
+      return MALA_ERR_DEVICE_TIMEOUT;
+    }
+    return MALA_OK;
+  }
+};
 
 #define MALA_TRY(expr)              \
   do {                              \
@@ -336,15 +379,17 @@ static int fwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse,
 int mala_fwd(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
              int Hkv, int N, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
              void* cuda_stream) {
+  ApiScope scope("mala_fwd", cuda_stream);
   (void)ws; (void)ws_bytes;
-  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, N, N, d, causal, scale, tau, cuda_stream);
+  return scope.finish(fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, N, N, d, causal, scale, tau, cuda_stream));
 }
 
 int mala_fwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B, int Hq,
                    int Hkv, int Nq, int Nk, int d, int causal, float scale, float tau, void* ws, size_t ws_bytes,
                    void* cuda_stream) {
+  ApiScope scope("mala_fwd_chunk", cuda_stream);
   (void)ws; (void)ws_bytes;
-  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, cuda_stream);
+  return scope.finish(fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, cuda_stream));
 }
 
 static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
@@ -380,22 +425,25 @@ static int bwd_impl(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dou
 int mala_fwd_chunk_split(mala_tin q, mala_tin k, mala_tin v, mala_tout o, float* lse, const mala_stats* st, int B,
                          int Hq, int Hkv, int Nq, int Nk, int d, int causal, float scale, float tau, int num_splits,
                          void* ws, size_t ws_bytes, void* cuda_stream) {
-  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, cuda_stream, nullptr, 0, num_splits,
-                  ws, ws_bytes);
+  ApiScope scope("mala_fwd_chunk_split", cuda_stream);
+  return scope.finish(fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, cuda_stream, nullptr, 0, num_splits,
+                  ws, ws_bytes));
 }
 
 int mala_bwd(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
              mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int N, int d, int causal,
              float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
-  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, N, N, d, causal, scale, tau, ws, ws_bytes,
-                  cuda_stream);
+  ApiScope scope("mala_bwd", cuda_stream);
+  return scope.finish(bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, N, N, d, causal, scale, tau, ws, ws_bytes,
+                  cuda_stream));
 }
 
 int mala_bwd_chunk(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse, mala_tout dq,
                    mala_tout dk, mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int Nq, int Nk, int d,
                    int causal, float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
-  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, ws, ws_bytes,
-                  cuda_stream);
+  ApiScope scope("mala_bwd_chunk", cuda_stream);
+  return scope.finish(bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, Nq, Nk, d, causal, scale, tau, ws, ws_bytes,
+                  cuda_stream));
 }
 
 static int check_packed(const int32_t* cu_seqlens, int B, int total, int max_seqlen) {
@@ -408,28 +456,31 @@ static int check_packed(const int32_t* cu_seqlens, int B, int total, int max_seq
 int mala_fwd_varlen(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu_seqlens, mala_tout o, float* lse,
                     const mala_stats* st, int B, int Hq, int Hkv, int total, int max_seqlen, int d, int causal,
                     float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_fwd_varlen", cuda_stream);
   (void)ws; (void)ws_bytes;
   MALA_TRY(check_packed(cu_seqlens, B, total, max_seqlen));
-  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau, cuda_stream,
-                  cu_seqlens, total);
+  return scope.finish(fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau, cuda_stream,
+                  cu_seqlens, total));
 }
 
 int mala_fwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,
                            mala_tout o, float* lse, const mala_stats* st, int B, int Hq, int Hkv, int total_q,
                            int total_k, int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau,
                            void* ws, size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_fwd_varlen_prefix", cuda_stream);
   (void)ws; (void)ws_bytes;
   MALA_TRY(check_packed(cu_seqlens_q, B, total_q, max_seqlen_q));
   MALA_TRY(check_packed(cu_seqlens_k, B, total_k, max_seqlen_k));
   if (causal && max_seqlen_k < max_seqlen_q) return MALA_ERR_UNSUPPORTED;
-  return fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen_q, max_seqlen_k, d, causal, scale, tau, cuda_stream,
-                  cu_seqlens_q, total_q, 1, nullptr, 0, cu_seqlens_k, total_k);
+  return scope.finish(fwd_impl(q, k, v, o, lse, st, B, Hq, Hkv, max_seqlen_q, max_seqlen_k, d, causal, scale, tau, cuda_stream,
+                  cu_seqlens_q, total_q, 1, nullptr, 0, cu_seqlens_k, total_k));
 }
 
 int mala_fwd_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* cu_seqlens_q, const int32_t* block_table,
                    const int32_t* seqlens_k, mala_tout o, float* lse, const mala_stats* st, int B, int Hq, int Hkv,
                    int total_q, int max_seqlen_q, int num_pages, int page_size, int max_pages_per_seq, int d, int causal,
                    float scale, float tau, void* ws, size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_fwd_paged", cuda_stream);
   (void)ws; (void)ws_bytes;
   MALA_TRY(check_packed(cu_seqlens_q, B, total_q, max_seqlen_q));
   if (!block_table || !seqlens_k || num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0) return MALA_ERR_INVALID_ARG;
@@ -443,17 +494,18 @@ int mala_fwd_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* 
   FwdPaging pg;
   pg.block_table = block_table; pg.seqlens_k = seqlens_k; pg.num_pages = num_pages; pg.page_size = page_size;
   pg.max_pages_per_seq = max_pages_per_seq;
-  return fwd_impl(q, kpages, vpages, o, lse, st, B, Hq, Hkv, max_seqlen_q, max_k, d, causal, scale, tau, cuda_stream,
-                  cu_seqlens_q, total_q, 1, nullptr, 0, nullptr, 0, &pg);
+  return scope.finish(fwd_impl(q, kpages, vpages, o, lse, st, B, Hq, Hkv, max_seqlen_q, max_k, d, causal, scale, tau, cuda_stream,
+                  cu_seqlens_q, total_q, 1, nullptr, 0, nullptr, 0, &pg));
 }
 
 int mala_bwd_varlen(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,
                     const int32_t* cu_seqlens, mala_tout dq, mala_tout dk, mala_tout dv, const mala_stats* st, int B,
                     int Hq, int Hkv, int total, int max_seqlen, int d, int causal, float scale, float tau, void* ws,
                     size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_bwd_varlen", cuda_stream);
   MALA_TRY(check_packed(cu_seqlens, B, total, max_seqlen));
-  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau,
-                  ws, ws_bytes, cuda_stream, cu_seqlens, total);
+  return scope.finish(bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, max_seqlen, max_seqlen, d, causal, scale, tau,
+                  ws, ws_bytes, cuda_stream, cu_seqlens, total));
 }
 
 int mala_bwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_tin dout, const float* lse,
@@ -461,17 +513,19 @@ int mala_bwd_varlen_prefix(mala_tin q, mala_tin k, mala_tin v, mala_tin o, mala_
                            mala_tout dv, const mala_stats* st, int B, int Hq, int Hkv, int total_q, int total_k,
                            int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, float tau, void* ws,
                            size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_bwd_varlen_prefix", cuda_stream);
   MALA_TRY(check_packed(cu_seqlens_q, B, total_q, max_seqlen_q));
   MALA_TRY(check_packed(cu_seqlens_k, B, total_k, max_seqlen_k));
   if ((long long)total_q + 384LL * B > 0x7fffffffLL) return MALA_ERR_UNSUPPORTED;
   if (causal && max_seqlen_k < max_seqlen_q) return MALA_ERR_UNSUPPORTED;
-  return bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, max_seqlen_q, max_seqlen_k, d, causal, scale, tau,
-                  ws, ws_bytes, cuda_stream, cu_seqlens_q, total_q, cu_seqlens_k, total_k);
+  return scope.finish(bwd_impl(q, k, v, o, dout, lse, dq, dk, dv, st, B, Hq, Hkv, max_seqlen_q, max_seqlen_k, d, causal, scale, tau,
+                  ws, ws_bytes, cuda_stream, cu_seqlens_q, total_q, cu_seqlens_k, total_k));
 }
 
 int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
                 int B, int Hq, int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* ws,
                 size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_decode", cuda_stream);
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau, 256));
   if (num_splits <= 0 || !ws) return MALA_ERR_INVALID_ARG;
   if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
@@ -485,13 +539,14 @@ int mala_decode(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
   MALA_TRY(device_setup(dev, &status));
-  return decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
-                       (cudaStream_t)cuda_stream);
+  return scope.finish(decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
+                       (cudaStream_t)cuda_stream));
 }
 
 int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float* kscale, const float* vscale,
                     mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                     float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_decode_fp8", cuda_stream);
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
   if (num_splits <= 0 || !ws || !kscale || !vscale) return MALA_ERR_INVALID_ARG;
   if (Hq / Hkv > 8 || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
@@ -513,8 +568,8 @@ int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float*
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
   MALA_TRY(device_setup(dev, &status));
-  return decode_fp8_launch(q, kcache8, vcache8, kscale, vscale, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits,
-                           ws, status, (cudaStream_t)cuda_stream);
+  return scope.finish(decode_fp8_launch(q, kcache8, vcache8, kscale, vscale, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits,
+                           ws, status, (cudaStream_t)cuda_stream));
 }
 
 int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const float* kscale, const float* vscale,
@@ -522,6 +577,7 @@ int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const 
                           const mala_stats* st, int B, int Hq, int Hkv, int num_pages, int page_size,
                           int max_pages_per_seq, int d, float scale, float tau, int num_splits, void* ws, size_t ws_bytes,
                           void* cuda_stream) {
+  ApiScope scope("mala_decode_fp8_paged", cuda_stream);
   if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
   // pages of whole tiles, or of 16, 32 or 64 keys (a tile is then put together from several pages)
   if (!(page_size % 128 == 0 || page_size == 16 || page_size == 32 || page_size == 64) ||
@@ -553,13 +609,14 @@ int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const 
   DecPaging pg;
   pg.block_table = block_table; pg.seqlens = seqlens; pg.bt_stride = max_pages_per_seq; pg.page_size = page_size;
   pg.num_pages = num_pages;
-  return decode_fp8_launch(q, kpages8, vpages8, kscale, vscale, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau,
-                           num_splits, ws, status, (cudaStream_t)cuda_stream, &pg);
+  return scope.finish(decode_fp8_launch(q, kpages8, vpages8, kscale, vscale, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau,
+                           num_splits, ws, status, (cudaStream_t)cuda_stream, &pg));
 }
 
 int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, const mala_stats* st,
                       int B, int Hq, int Hkv, int Nk, int Sq, int d, float scale, float tau, int num_splits, void* ws,
                       size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_decode_multi", cuda_stream);
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau, 256));
   if (num_splits <= 0 || Sq <= 0 || !ws) return MALA_ERR_INVALID_ARG;
   if ((Hq / Hkv) * Sq > 16 || Sq > Nk || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
@@ -573,14 +630,15 @@ int mala_decode_multi(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o,
   MALA_TRY(current_device_checked(&dev));
   int* status = nullptr;
   MALA_TRY(device_setup(dev, &status));
-  return decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
-                       (cudaStream_t)cuda_stream, nullptr, Sq);
+  return scope.finish(decode_launch(q, kcache, vcache, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
+                       (cudaStream_t)cuda_stream, nullptr, Sq));
 }
 
 int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_t* block_table,
                       const int32_t* seqlens, mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq,
                       int Hkv, int num_pages, int page_size, int max_pages_per_seq, int Sq, int d, float scale,
                       float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_decode_paged", cuda_stream);
   if (num_pages <= 0 || page_size <= 0 || max_pages_per_seq <= 0 || Sq <= 0 || !block_table) return MALA_ERR_INVALID_ARG;
   if (page_size < 8 || (page_size % 128 != 0 && 128 % page_size != 0) ||
       (long long)max_pages_per_seq * page_size > 0x7fffffffLL)
@@ -603,12 +661,13 @@ int mala_decode_paged(mala_tin q, mala_tin kpages, mala_tin vpages, const int32_
   DecPaging pg;
   pg.block_table = block_table; pg.seqlens = seqlens; pg.bt_stride = max_pages_per_seq; pg.page_size = page_size;
   pg.num_pages = num_pages;
-  return decode_launch(q, kpages, vpages, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
-                       (cudaStream_t)cuda_stream, &pg, Sq);
+  return scope.finish(decode_launch(q, kpages, vpages, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau, num_splits, ws, status,
+                       (cudaStream_t)cuda_stream, &pg, Sq));
 }
 
 int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o, float* lse_opt, int B, int Hq,
                        int Hkv, int Nk, int d, float scale, float tau, int num_splits, void* cuda_stream) {
+  ApiScope scope("mala_decode_static", cuda_stream);
   MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau, 256));
   if (num_splits <= 0) return MALA_ERR_INVALID_ARG;
   if (Hq / Hkv > 16 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
@@ -628,8 +687,8 @@ int mala_decode_static(mala_tin q, mala_tin kcache, mala_tin vcache, mala_tout o
   float* lse_part = (float*)(scratch + decode_align256((size_t)B * Hq * num_splits * padded_head_size(d) * sizeof(float)));
   // every (batch, head, split) entry of both arrays is written by the split kernel (empty splits
   // included) before the merge reads it, so nothing left over from an earlier call is ever read
-  return decode_launch_with_scratch(q, kcache, vcache, o, lse_opt, nullptr, B, Hq, Hkv, Nk, d, scale, tau, num_splits,
-                                    o_part, lse_part, status, (cudaStream_t)cuda_stream);
+  return scope.finish(decode_launch_with_scratch(q, kcache, vcache, o, lse_opt, nullptr, B, Hq, Hkv, Nk, d, scale, tau, num_splits,
+                                    o_part, lse_part, status, (cudaStream_t)cuda_stream));
 }
 
 }  // extern "C"

@@ -242,3 +242,34 @@ def test_an_expired_device_wait_is_reported_and_later_launches_do_nothing_until_
     assert np.abs(lse.cpu().numpy() - ref["lse"]).max() <= parity.LSE_ABS
     with pytest.raises(mala.MalaError):
         mala.test_expire_wait(0)
+
+
+def test_debug_mode_reports_errors_from_the_call_itself():
+    """MALA_DEBUG=1 (with MALA_NVTX=1 alongside): a call waits for its stream and returns a recorded device time-out
+    itself.  Run in a child process, since the variables are read once per process.  The time-out is the bounded wait
+    that nothing satisfies (mala_test_expire_wait), not a fault."""
+    import os, subprocess, sys, textwrap
+    code = textwrap.dedent("""
+        import torch
+        from paper_2609_32712_b200 import mala, workloads as W
+        w = W.custom_decode(1, 4, 1, 1024, 128, 2, seed=1, device="cuda")
+        o, lse, _ = mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 1e-4, 2)      # fine: returns 0
+        p = W.custom_prefill(1, 2, 1, 256, 64, seed=2, device="cuda")
+        mala.fwd(p["q"], p["k"], p["v"], p["scale"], 1e-4)
+        assert mala.lib().mala_test_expire_wait(20000, None) == 0                              # sets the status word
+        try:
+            mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 1e-4, 2)
+            print("NO ERROR")
+        except mala.MalaError as e:
+            print("CODE", e.code)
+        assert mala.device_status(clear=True) == -8
+        o2, lse2, _ = mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 1e-4, 2)    # recovered
+        assert torch.equal(o, o2) and torch.equal(lse, lse2)
+        print("DONE")
+    """)
+    env = dict(os.environ, MALA_DEBUG="1", MALA_NVTX="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    assert "CODE -8" in r.stdout and "DONE" in r.stdout, r.stdout + r.stderr[-1000:]
+    assert "[mala debug] mala_decode: device status" in r.stderr
