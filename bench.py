@@ -936,6 +936,22 @@ def main():
                               "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
             f8["paged_16"] = pg8
             del kp8, vp8, bt16, ksp, vsp
+            # ... and with eight query heads per KV head (64 query heads on the same cache: two threads per key)
+            q64 = qd.view(dcfg.B, 1, dcfg.Hkv, dcfg.Hq // dcfg.Hkv, dcfg.d)      # every group's heads, twice
+            q64 = torch.cat([q64, q64], dim=3).reshape(dcfg.B, 1, 2 * dcfg.Hq, dcfg.d).contiguous()
+            o64 = torch.empty_like(q64)
+            ws64 = torch.empty(mala.workspace_bytes(mala.OP_DECODE, dcfg.B, 2 * dcfg.Hq, dcfg.Hkv, dcfg.Nk, dcfg.d,
+                                                    dcfg.num_splits), dtype=torch.uint8, device=dev)
+            g8 = {}
+            for label, t_ in (("mala", tau), ("dense", 0.0)):
+                us = 1e3 * time_cuda(lambda: mala.decode_fp8(q64, k8, v8, ks8, vs8, wd["scale"], t_, dcfg.num_splits,
+                                                              ws=ws64, out=o64, want_lse=False), 25, 100)
+                us16 = 1e3 * time_cuda(lambda: mala.decode(q64, kc, vc, wd["scale"], t_, dcfg.num_splits, ws=ws64,
+                                                            out=o64, want_lse=False), 25, 100)
+                need = f8["key_major"][label]["needed_gb"] * 1e9
+                g8[label] = {"us": us, "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "bf16_cache_us": us16}
+            f8["eight_heads_per_kv_head"] = g8
+            del q64, o64, ws64
             row["e4m3_cache"] = f8
             del k8, v8, ks8, vs8
             # half the KV heads with 256 columns each (the same bytes per key): 64 KB tiles, two output accumulators
