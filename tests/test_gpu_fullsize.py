@@ -214,3 +214,100 @@ def test_cfg3_32k_chunk_of_the_last_8192_queries(mala, oracle, preset, tau):
     for (b, h, i) in dq_units:
         rows = slice(i * 128, (i + 1) * 128)
         parity.check_grad(dq[b, rows, h].float().cpu().numpy(), g["dq"][b, rows, h], f"dq block {i}")
+
+
+def _check_decode_units(oracle, q, kd, vd, scale, tau, S, units, G, o, lse, gm):
+    """Sampled (sequence, KV head) units of a decode call, each against the oracle on its own slice of the cache
+    (kd, vd: the values the call works on, fp32 or bf16, on the GPU; only the slices travel to the host)."""
+    for (b, g) in units:
+        hs = slice(g * G, (g + 1) * G)
+        n = kd.shape[1]
+        qs, ks, vs = q[b:b + 1, :, hs].cpu(), kd[b:b + 1, :, g:g + 1].cpu(), vd[b:b + 1, :, g:g + 1].cpu()
+        ref = oracle.decode(qs, ks, vs, scale, tau, S, 128)
+        ref_abs = oracle.decode(qs, ks, vs.abs(), scale, tau, S, 128)
+        tps = ref["mask"].shape[-1]
+        for s in range(S):
+            parity.check_mask(gm[b, g, s], ref["mask"][0, 0, s], ref["crit"][0, 0, s], list(range(tps - 1, -1, -1)), tau, n)
+        parity.check_output(o[b, 0, hs].float().cpu().numpy(), ref["o"][0], a_ref=ref_abs["o"][0])
+        assert np.abs(lse[b, hs].cpu().numpy() - ref["lse"][0]).max() <= parity.LSE_ABS
+
+
+@pytest.mark.parametrize("heads", [32, 64])
+@pytest.mark.parametrize("preset,tau", [("literal", 0.0), ("D", 1e-4)])
+def test_cfg5_decode_128k_over_an_e4m3_cache(mala, oracle, preset, tau, heads):
+    """The bench's e4m3 rows: cfg5 with the cache stored as e4m3 codes and a scale per tile, with cfg5's four and with
+    eight query heads per KV head (every group's heads twice)."""
+    cfg = W.decode_config("cfg5")
+    w = W.make_decode(cfg, preset=preset, device="cuda")
+    G0 = cfg.Hq // cfg.Hkv
+    q = w["q"]
+    if heads == 64:
+        q = q.view(cfg.B, 1, cfg.Hkv, G0, cfg.d)
+        q = torch.cat([q, q], dim=3).reshape(cfg.B, 1, 2 * cfg.Hq, cfg.d).contiguous()
+    k8, ks, kd = W.quantize_cache_e4m3(w["kcache"])
+    del w["kcache"]
+    v8, vs, vd = W.quantize_cache_e4m3(w["vcache"])
+    del w["vcache"]
+    o, lse, st = mala.decode_fp8(q, k8, v8, ks, vs, w["scale"], tau, cfg.num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert torch.isfinite(o.float()).all()
+    tps = -(-(-(-cfg.Nk // cfg.num_splits)) // 128)
+    gm = st.mask(tps).cpu().numpy()
+    _check_decode_units(oracle, q, kd, vd, w["scale"], tau, cfg.num_splits, [(0, 0), (5, 2), (7, 7)], heads // cfg.Hkv,
+                        o, lse, gm)
+    tot = st.totals.cpu().numpy()
+    assert tot[1] == cfg.B * cfg.Hkv * (cfg.Nk // 128) and (tot[0] == tot[1] if tau == 0.0 else tot[0] < tot[1])
+
+
+@pytest.mark.parametrize("preset,tau", [("literal", 0.0), ("D", 1e-4)])
+def test_cfg5_decode_128k_with_256_column_heads(mala, oracle, preset, tau):
+    """The bench's 256-column decode row: cfg5's bytes per key on half the heads of twice the size."""
+    cfg = W.decode_config("cfg5")
+    Hq, Hkv = cfg.Hq // 2, cfg.Hkv // 2
+    w = W.custom_decode(cfg.B, Hq, Hkv, cfg.Nk, 256, cfg.num_splits, group_types=cfg.group_types[:Hkv], seed=cfg.seed,
+                        preset=preset, device="cuda")
+    o, lse, st = mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], tau, cfg.num_splits, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert torch.isfinite(o.float()).all()
+    tps = -(-(-(-cfg.Nk // cfg.num_splits)) // 128)
+    gm = st.mask(tps).cpu().numpy()
+    _check_decode_units(oracle, w["q"], w["kcache"], w["vcache"], w["scale"], tau, cfg.num_splits, [(0, 0), (6, 3)],
+                        Hq // Hkv, o, lse, gm)
+    if tau == 0.0:
+        assert gm.all()
+
+
+@pytest.mark.parametrize("preset,tau", [("literal", 0.0), ("R", 1e-4)])
+def test_cfg3_32k_forward_with_256_column_heads(mala, oracle, preset, tau):
+    """The bench's 256-column forward row: cfg3's shape with half the heads of twice the size (one query block per CTA)."""
+    cfg = W.prefill_config("cfg3")
+    Hq, Hkv = cfg.Hq // 2, cfg.Hkv // 2
+    w = W.custom_prefill(cfg.B, Hq, Hkv, cfg.N, 256, head_types=cfg.head_types[:Hq], seed=cfg.seed, preset=preset,
+                         device="cuda")
+    q, k, v = w["q"], w["k"], w["v"]
+    T = cfg.N // 128
+    o, lse, st = mala.fwd(q, k, v, w["scale"], tau, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    assert torch.isfinite(o.float()).all()
+    fm = st.mask(T)
+    tri = torch.tril(torch.ones(T, T, dtype=torch.bool, device=fm.device))
+    assert not (fm & ~tri).any() and fm.diagonal(dim1=2, dim2=3).all()
+    if tau == 0.0:
+        assert (fm == tri).all()
+    else:
+        _, lse_d, _ = mala.fwd(q, k, v, w["scale"], 0.0)
+        eps = 1.0 - torch.exp(lse - lse_d)
+        assert eps.max() <= tau / (1 + tau) + 1e-3 and eps.min() >= -1e-3      # Proposition 1 (fp32 normalizers)
+        assert fm.sum() < tri.sum() * Hq
+    units = [(0, 1, T - 1), (0, 2, 100), (0, 5, 3), (0, 15, 200)]
+    ref = oracle.fwd(q, k, v, w["scale"], tau, 128, 128, units=units)
+    ref_abs = oracle.fwd(q, k, v.abs(), w["scale"], tau, 128, 128, units=units)
+    fmc = fm.cpu().numpy()
+    for (b, h, i) in units:
+        rows = slice(i * 128, (i + 1) * 128)
+        parity.check_mask(fmc[b, h, i], ref["mask"][b, h, i], ref["crit"][b, h, i], list(range(i, -1, -1)), tau, i * 128 + 1)
+        parity.check_output(o[b, rows, h].float().cpu().numpy(), ref["o"][b, rows, h], a_ref=ref_abs["o"][b, rows, h])
+        assert np.abs(lse[b, h, rows].cpu().numpy() - ref["lse"][b, h, rows]).max() <= parity.LSE_ABS
