@@ -2,7 +2,8 @@
 // storage type differs).  The decode step is bound by the bytes of K and V it streams, so an 8-bit cache halves its
 // time.  Keys and values are stored as e4m3 with one fp32 scale per (sequence, KV head, 128-key tile):
 //     k = kscale[b, h_kv, tile] * e4m3(k8),   v = vscale[b, h_kv, tile] * e4m3(v8)
-// and the kernel computes the operator of mala_decode on those dequantised values.
+// (paged caches: per tile of a page, or per page where a page is smaller than a tile) and the kernel computes the
+// operator of mala_decode on those dequantised values.
 //
 // The problem is laid out as in mala_decode_split_kernel (transposed: keys in the TMEM lanes, the packed query heads
 // as the N = 16 columns, persistent CTAs over (sequence, KV head, split) work items, V of a retained tile requested
@@ -13,9 +14,10 @@
 //   S^T = K8 Q8^T   each query row q becomes q1 = e4m3(q 2^k) and q2 = e4m3(16 (q 2^k - q1)), 2^k the power of two
 //                   that brings the row's largest magnitude into [128, 256).  A bf16 significand has 8 bits and q1
 //                   takes the leading 4, so q 2^k = q1 + q2 / 16 exactly, up to entries 2^-17 below the row's largest
-//                   (e4m3's subnormal floor).  The two rows are columns h and 4 + h of the MMA (hence at most four
-//                   heads per KV head), products of e4m3 values are exact in the fp32 accumulator, and a softmax
-//                   thread forms (S[h] + S[4 + h] / 16) * scale * kscale / 2^k.
+//                   (e4m3's subnormal floor).  The two rows are columns h and HALF + h of the MMA, HALF = 4 with up to
+//                   four heads per KV head and 8 with five to eight (hence at most eight heads), products of e4m3
+//                   values are exact in the fp32 accumulator, and a softmax thread forms
+//                   (S[h] + S[HALF + h] / 16) * scale * kscale / 2^k.
 //   O^T += V8^T P8^T  V8 is read MN-major.  A probability enters as P' = 64 exp2(y - yref) with y = x + log2(vscale)
 //                   the score of the key weighted by its V tile's scale and yref a running reference of the item
 //                   (so the tile's scale rides on P', inside e4m3's narrow range whatever its magnitude), split as
@@ -41,7 +43,8 @@
 //   warp NG + k       converts an item's queries, issues S^T of every tile
 //   warp 2NG + k      MALA kernel: takes the votes in order, requests the raw V copy of a retained tile
 //   warp 3NG + k      issues O^T += V8^T P8^T of every retained tile
-//   warps 4NG + 4k .. softmax group (thread = key of the tile), up to four packed query heads
+//   warps 4NG + 4k .. softmax group (thread = key of the tile), up to four packed query heads; with five to eight heads
+//                     the group is eight warps, warps 4NG + 8k .., two threads per key with four heads each
 // and for all streams
 //   last four warps   epilogue group (thread = output channel)
 #pragma once
