@@ -952,6 +952,22 @@ def main():
                 g8[label] = {"us": us, "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], "bf16_cache_us": us16}
             f8["eight_heads_per_kv_head"] = g8
             del q64, o64, ws64
+            # ... and two new tokens per sequence in one step (mala_decode_fp8_multi: eight rows per KV head, the same bytes)
+            q2 = qd.repeat(1, 2, 1, 1).contiguous()
+            o2t = torch.empty_like(q2)
+            ws2 = torch.empty(mala.workspace_bytes(mala.OP_DECODE, dcfg.B * 2, dcfg.Hq, dcfg.Hkv, dcfg.Nk, dcfg.d,
+                                                   dcfg.num_splits), dtype=torch.uint8, device=dev)
+            m2 = {}
+            for label, t_ in (("mala", tau), ("dense", 0.0)):
+                us = 1e3 * time_cuda(lambda: mala.decode_fp8_multi(q2, k8, v8, ks8, vs8, wd["scale"], t_, dcfg.num_splits,
+                                                                    ws=ws2, out=o2t, want_lse=False), 25, 100)
+                _, _, st = mala.decode_fp8_multi(q2, k8, v8, ks8, vs8, wd["scale"], t_, dcfg.num_splits, ws=ws2, stats=True)
+                ret, leg = st.totals.cpu().tolist()
+                need = (leg + ret) * TILE * dcfg.d
+                m2[label] = {"us": us, "retained_frac": ret / leg, "hbm_frac": need / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                             "two_single_steps_us": 2 * f8["key_major"][label]["us"]}
+            f8["multi_token_2"] = m2
+            del q2, o2t, ws2
             row["e4m3_cache"] = f8
             del k8, v8, ks8, vs8
             # half the KV heads with 256 columns each (the same bytes per key): 64 KB tiles, two output accumulators

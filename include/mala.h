@@ -209,6 +209,15 @@ int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float*
                     mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                     float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* mala_decode_fp8 with Sq new tokens per sequence: the rule and the layout of mala_decode_multi (q, o [B,Sq,Hq,d],
+ * lse_opt [B,Sq,Hq], the new tokens' keys and values in the last Sq positions of the caches, token s at position
+ * Nk - Sq + s with L = Nk - Sq + s + 1) on the storage of mala_decode_fp8.  Requires Sq * Hq/Hkv <= 8 and Sq <= Nk
+ * (MALA_ERR_UNSUPPORTED otherwise); Sq = 1 is mala_decode_fp8.
+ * Workspace: mala_workspace_bytes(MALA_OP_DECODE, B * Sq, Hq, Hkv, Nk, 128, num_splits). */
+int mala_decode_fp8_multi(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float* kscale, const float* vscale,
+                          mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int Sq, int d,
+                          float scale, float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* mala_decode_fp8 over a paged 8-bit cache with one length per sequence: the layout of mala_decode_paged (one new token
  * per sequence) with the storage of mala_decode_fp8.  kpages8, vpages8: 8-bit [num_pages, page_size, Hkv, d] views
  * (strides in elements = bytes, multiples of 16), page_size a multiple of 128, or 16, 32 or 64 (MALA_ERR_UNSUPPORTED

@@ -572,6 +572,34 @@ int mala_decode_fp8(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float*
                            ws, status, (cudaStream_t)cuda_stream));
 }
 
+int mala_decode_fp8_multi(mala_tin q, mala_tin kcache8, mala_tin vcache8, const float* kscale, const float* vscale,
+                          mala_tout o, float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int Sq, int d,
+                          float scale, float tau, int num_splits, void* ws, size_t ws_bytes, void* cuda_stream) {
+  ApiScope scope("mala_decode_fp8_multi", cuda_stream);
+  MALA_TRY(check_common(B, Hq, Hkv, Nk, d, scale, tau));
+  if (num_splits <= 0 || Sq <= 0 || !ws || !kscale || !vscale) return MALA_ERR_INVALID_ARG;
+  if ((Hq / Hkv) * Sq > 8 || Sq > Nk || d % 16 != 0 || num_splits > 65535) return MALA_ERR_UNSUPPORTED;
+  MALA_TRY(check_view(q.p, q.sb, q.sn, q.sh, B, Sq, Hq));
+  auto check8 = [&](const mala_tin& t) -> int {   // 8-bit views: strides in elements = bytes, multiples of 16
+    if (!t.p) return MALA_ERR_INVALID_ARG;
+    if (!aligned16(t.p)) return MALA_ERR_MISALIGNED;
+    if ((B > 1 && t.sb % 16) || (Nk > 1 && t.sn % 16) || (Hkv > 1 && t.sh % 16)) return MALA_ERR_MISALIGNED;
+    if ((B > 1 && t.sb <= 0) || (Nk > 1 && t.sn <= 0) || (Hkv > 1 && t.sh <= 0)) return MALA_ERR_INVALID_ARG;
+    return MALA_OK;
+  };
+  MALA_TRY(check8(kcache8));
+  MALA_TRY(check8(vcache8));
+  MALA_TRY(check_view(o.p, o.sb, o.sn, o.sh, B, Sq, Hq));
+  if ((((uintptr_t)ws) & 255) != 0 || (((uintptr_t)kscale) & 3) != 0 || (((uintptr_t)vscale) & 3) != 0) return MALA_ERR_MISALIGNED;
+  if (ws_bytes < decode_workspace_bytes(B * Sq, Hq, 128, num_splits)) return MALA_ERR_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  MALA_TRY(current_device_checked(&dev));
+  int* status = nullptr;
+  MALA_TRY(device_setup(dev, &status));
+  return scope.finish(decode_fp8_launch(q, kcache8, vcache8, kscale, vscale, o, lse_opt, st, B, Hq, Hkv, Nk, d, scale, tau,
+                                        num_splits, ws, status, (cudaStream_t)cuda_stream, nullptr, Sq));
+}
+
 int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const float* kscale, const float* vscale,
                           const int32_t* block_table, const int32_t* seqlens, mala_tout o, float* lse_opt,
                           const mala_stats* st, int B, int Hq, int Hkv, int num_pages, int page_size,

@@ -51,7 +51,7 @@ inline bool decode_set_attributes() {
 #define MALA_DEC_ATTR_GP(GP) MALA_DEC_ATTR(false, GP, false) MALA_DEC_ATTR(true, GP, false) MALA_DEC_ATTR(false, GP, true) MALA_DEC_ATTR(true, GP, true)
   MALA_DEC_ATTR_GP(1) MALA_DEC_ATTR_GP(2) MALA_DEC_ATTR_GP(4) MALA_DEC_ATTR_GP(8) MALA_DEC_ATTR_GP(16)
 #define MALA_F8_ATTR(DENSE, GP) \
-  ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess;
+  ok = ok && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, true, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess && cudaFuncSetAttribute(mala_decode_fp8_kernel<DENSE, GP, false, 2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecF8Cfg<2, DENSE>::kSmemBytes) == cudaSuccess;
   MALA_F8_ATTR(false, 1) MALA_F8_ATTR(true, 1) MALA_F8_ATTR(false, 2) MALA_F8_ATTR(true, 2) MALA_F8_ATTR(false, 4) MALA_F8_ATTR(true, 4)
   MALA_F8_ATTR(false, 8) MALA_F8_ATTR(true, 8)
 #undef MALA_F8_ATTR
@@ -168,9 +168,11 @@ inline int decode_launch_with_scratch(mala_tin q, mala_tin kc, mala_tin vc, mala
 inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* kscale, const float* vscale, mala_tout o,
                              float* lse_opt, const mala_stats* st, int B, int Hq, int Hkv, int Nk, int d, float scale,
                              float tau, int num_splits, void* ws, int* status, cudaStream_t stream,
-                             const DecPaging* pg = nullptr) {
+                             const DecPaging* pg = nullptr, int Sq = 1) {
   const int G = Hq / Hkv;
-  if (G > 8 || d % 16 != 0 || d > 128 || d < 16) return MALA_ERR_UNSUPPORTED;
+  const int R = G * Sq;   // rows of a work item
+  if (Sq < 1 || R > 8 || Sq > Nk || d % 16 != 0 || d > 128 || d < 16) return MALA_ERR_UNSUPPORTED;
+  if (Sq > 1 && pg) return MALA_ERR_UNSUPPORTED;   // (several tokens per step: contiguous caches only)
   const bool small = pg && pg->page_size < 128;
   if (pg && !(pg->page_size % 128 == 0 || pg->page_size == 16 || pg->page_size == 32 || pg->page_size == 64))
     return MALA_ERR_UNSUPPORTED;
@@ -180,7 +182,7 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
   if ((long long)B * Hkv * num_splits > 0x7fffffffLL || (long long)B * Hkv * ((Nk + 127) / 128) > 0x7fffffffLL)
     return MALA_ERR_UNSUPPORTED;
   CUtensorMap tq, tk, tv;
-  if (!make_tensor_map_q_rows(&tq, q.p, B, 1, Hq, d, q.sb, 0, q.sh, G) ||
+  if (!make_tensor_map_q_rows(&tq, q.p, B, Sq, Hq, d, q.sb, Sq > 1 ? q.sn : 0, q.sh, G) ||
       !make_tensor_map_u8_bnhd(&tk, kc.p, pg ? pg->num_pages : B, pg ? pg->page_size : Nk, Hkv, d, kc.sb, kc.sn, kc.sh, box_rows) ||
       !make_tensor_map_u8_bnhd(&tv, vc.p, pg ? pg->num_pages : B, pg ? pg->page_size : Nk, Hkv, d, vc.sb, vc.sn, vc.sh, box_rows))
     return MALA_ERR_TENSOR_MAP;
@@ -193,8 +195,9 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
   p.by_tpp.set((uint32_t)p.tpp);
   p.ppt = 128 / box_rows;
   p.prows = box_rows;
+  p.Sq = Sq;
   p.o_part = (float*)ws;
-  p.lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Hq * num_splits * 128 * sizeof(float)));
+  p.lse_part = (float*)((uint8_t*)ws + decode_align256((size_t)B * Sq * Hq * num_splits * 128 * sizeof(float)));
   p.retained = st ? st->retained_per_block : nullptr;
   p.bitmask = st ? st->tile_bitmask : nullptr;
   p.totals = st ? (unsigned long long*)st->totals : nullptr;
@@ -216,19 +219,20 @@ inline int decode_fp8_launch(mala_tin q, mala_tin kc, mala_tin vc, const float* 
   const int grid = p.n_items < sms ? p.n_items : sms;
 #define MALA_F8_LAUNCH(DENSE, GP)                                                                                      \
   do {                                                                                                                  \
-    if (small) mala_decode_fp8_kernel<DENSE, GP, true, 2, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    if (Sq > 1) mala_decode_fp8_kernel<DENSE, GP, false, 2, false, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
+    else if (small) mala_decode_fp8_kernel<DENSE, GP, true, 2, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
     else if (pg) mala_decode_fp8_kernel<DENSE, GP, true><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p); \
     else mala_decode_fp8_kernel<DENSE, GP, false><<<grid, DecF8Cfg<2, DENSE, (GP > 4)>::kThreads, DecF8Cfg<2, DENSE>::kSmemBytes, stream>>>(tq, tk, tv, p);  \
   } while (0)
   const bool dense = (tau == 0.f);
-  if (G <= 1) { if (dense) MALA_F8_LAUNCH(true, 1); else MALA_F8_LAUNCH(false, 1); }
-  else if (G <= 2) { if (dense) MALA_F8_LAUNCH(true, 2); else MALA_F8_LAUNCH(false, 2); }
-  else if (G <= 4) { if (dense) MALA_F8_LAUNCH(true, 4); else MALA_F8_LAUNCH(false, 4); }
+  if (R <= 1) { if (dense) MALA_F8_LAUNCH(true, 1); else MALA_F8_LAUNCH(false, 1); }
+  else if (R <= 2) { if (dense) MALA_F8_LAUNCH(true, 2); else MALA_F8_LAUNCH(false, 2); }
+  else if (R <= 4) { if (dense) MALA_F8_LAUNCH(true, 4); else MALA_F8_LAUNCH(false, 4); }
   else { if (dense) MALA_F8_LAUNCH(true, 8); else MALA_F8_LAUNCH(false, 8); }
 #undef MALA_F8_LAUNCH
   if (cudaGetLastError() != cudaSuccess) return MALA_ERR_CUDA;
-  decode_merge_kernel<128><<<B * Hq, 128, 0, stream>>>(p.o_part, p.lse_part, (__nv_bfloat16*)o.p, o.sb, 0, o.sh, lse_opt, 1,
-                                                      Hq, num_splits, d);
+  decode_merge_kernel<128><<<B * Sq * Hq, 128, 0, stream>>>(p.o_part, p.lse_part, (__nv_bfloat16*)o.p, o.sb,
+                                                           Sq > 1 ? o.sn : 0, o.sh, lse_opt, Sq, Hq, num_splits, d);
   return cudaGetLastError() == cudaSuccess ? MALA_OK : MALA_ERR_CUDA;
 }
 

@@ -96,6 +96,9 @@ struct DecF8Params {
   // copies of prows = page_size rows, copy c of key block x from page block_table[b][x * ppt + c]; the scales are
   // [num_pages, Hkv], one per (page, KV head)
   int ppt, prows;
+  // several new tokens per sequence (kMulti kernels): q, o are [B, Sq, Hq, d], the partials [B, Sq, Hq, splits, ..];
+  // row t * G + g of a work item is token t (0 = oldest, at position nk - Sq + t), head g of the group
+  int Sq;
 };
 
 // NG_: streams (two: a third, with the registers moved from the issuing warps to the softmax groups and rings of two
@@ -162,7 +165,9 @@ __device__ __forceinline__ uint2 split_e4m3x2(float a, float b) {
 // kSmall (with kPaged): pages smaller than a tile.  The producer and the vote warp issue a tile's copies from as many
 // lanes as it has pages, a key's scales are those of its page (a softmax thread is a key, so it reads its own), and
 // the reference of the 8-bit probabilities is kept against the largest V scale of the tile.
-template <bool kDense, int GP, bool kPaged = false, int NG_ = 2, bool kSmall = false>
+// kMulti: Sq > 1 new tokens per sequence, rows = Sq * G <= 8.  A row then sees the keys up to its own position,
+// has its own L (Section 2.1) and threshold, and a row that sees no key of a tile does not constrain the tile.
+template <bool kDense, int GP, bool kPaged = false, int NG_ = 2, bool kSmall = false, bool kMulti = false>
 __global__ void __launch_bounds__(DecF8Cfg<NG_, kDense, (GP > 4)>::kThreads, 1)
 mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const DecF8Params p) {
@@ -201,7 +206,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.Hq / p.Hkv;
-  const int R = G;
+  const int R = kMulti ? G * p.Sq : G;     // rows of a work item
   int* status = p.status;
 
   // the stream's part of shared memory
@@ -572,14 +577,19 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const int T = tiles_of(item);
       int b, hkv, split, j0;
       geometry(item, b, hkv, split, j0, T);
-      const size_t prow0 = ((size_t)b * p.Hq + hkv * G) * p.num_splits + split;
+      // row q of the item: token q / G, head q % G of the group; its partials lie rowoff(q) rows after the item's first
+      const size_t prow0 = ((size_t)b * (kMulti ? p.Sq : 1) * p.Hq + hkv * G) * p.num_splits + split;
+      auto rowoff = [&](int q) -> size_t {
+        if constexpr (kMulti) { const int tok = q / G; return ((size_t)tok * p.Hq + (size_t)(q - tok * G)) * p.num_splits; }
+        else return (size_t)q * p.num_splits;
+      };
       const size_t stat_row = (size_t)(b * p.Hkv + hkv) * p.num_splits + split;
       if (T == 0) {   // a split without keys: (0, -inf)
 #pragma unroll
         for (int q = 0; q < GH; ++q)
           if (q < R) {
-            p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = 0.f;
-            if (kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = -INFINITY;
+            p.o_part[(prow0 + rowoff(q)) * 128 + kt] = 0.f;
+            if (kt == q) p.lse_part[prow0 + rowoff(q)] = -INFINITY;
           }
         if (head && p.retained) p.retained[stat_row] = 0u;
         continue;
@@ -608,8 +618,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       for (int q = 0; q < GH; ++q)
         if (q < R) {   // O^T is in units of 2^yref / 64, l in units of 2^m
           const float num = fmaf(__uint_as_float(o[HALF + q]), 0.0625f, __uint_as_float(o[q])) * fast_exp2(ys[q] - ms[q]);
-          p.o_part[(prow0 + (size_t)q * p.num_splits) * 128 + kt] = num / (ls[q] * kPScale);
-          if (kt == q) p.lse_part[prow0 + (size_t)q * p.num_splits] = (ms[q] + __log2f(ls[q])) * 0.6931471805599453f;
+          const bool seen = !kMulti || ls[q] > 0.f;   // (a row that saw no key of the split: (0, -inf))
+          p.o_part[(prow0 + rowoff(q)) * 128 + kt] = seen ? num / (ls[q] * kPScale) : 0.f;
+          if (kt == q) p.lse_part[prow0 + rowoff(q)] = seen ? (ms[q] + __log2f(ls[q])) * 0.6931471805599453f : -INFINITY;
         }
       if (head) {
         if (p.retained) p.retained[stat_row] = (uint32_t)r_all;
@@ -681,6 +692,19 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       uint32_t* bm_row = p.bitmask ? p.bitmask + ((size_t)(b * p.Hkv + hkv) * p.num_splits + split) * p.words : nullptr;
       const int nk = keys_of(b);                 // keys of the sequence: the L of Eq. 3 and the tail mask
       const float theta = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(nk, 1)));
+      // several tokens: row q sees the keys before position lim[q] = nk - (Sq - 1 - its token), which is its L
+      int lim[kMulti ? GS : 1];
+      float theta_q[kMulti ? GS : 1];
+      if constexpr (kMulti) {
+#pragma unroll
+        for (int q = 0; q < GS; ++q) {
+          const int tok = (hb + q < R) ? (hb + q) / G : 0;
+          lim[q] = nk - (p.Sq - 1 - tok);
+          theta_q[q] = kDense ? -INFINITY : (p.log2_tau - log2f((float)max(lim[q], 1)));
+        }
+      }
+      auto lim_of = [&](int q) -> int { if constexpr (kMulti) return lim[q]; else return nk; };
+      auto theta_of = [&](int q) -> float { if constexpr (kMulti) return theta_q[q]; else return theta; };
       int r = 0;                                 // tiles of the item retained so far
       float m_ref[GS], l[GS], yref[GS], lgl[GS], c2q[GS];
 #pragma unroll
@@ -720,7 +744,7 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           float mx[GS];
 #pragma unroll
           for (int q = 0; q < GS; ++q) {   // the two e4m3 rows of the head, the row's 2^-k and the K tile's scale
-            x[q] = (kpos < nk && hb + q < R) ? fmaf(rem_of(q), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
+            x[q] = (kpos < lim_of(q) && hb + q < R) ? fmaf(rem_of(q), 0.0625f, __uint_as_float(sr[q])) * (c2q[q] * ks) : -INFINITY;
             mx[q] = x[q];
           }
           RowReduce<GS, 16, true>::run(mx, lane);
@@ -732,7 +756,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (!kDense && r > 0) {
           retain = false;
 #pragma unroll
-          for (int q = 0; q < GS; ++q) retain = retain || (hb + q < R && !(((tmax[q] - (m_ref[q] + lgl[q])) - theta) < 0.f));
+          for (int q = 0; q < GS; ++q)   // (several tokens: a row without a visible key in the tile does not constrain it)
+            retain = retain || (hb + q < R && (!kMulti || tmax[q] > -INFINITY) &&
+                                !(((tmax[q] - (m_ref[q] + lgl[q])) - theta_of(q)) < 0.f));
         }
         if (!kDense && head) {
           *(volatile int*)&flag[k][half][g & 7] = retain ? 1 : 0;
@@ -750,7 +776,10 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int ps = rg % PP;
         if (r == 0) {
 #pragma unroll
-          for (int q = 0; q < GS; ++q) { m_ref[q] = tmax[q]; yref[q] = tmax[q] + lv; }   // (nothing accumulated yet)
+          for (int q = 0; q < GS; ++q) {   // (nothing accumulated yet; finite also for a row that sees no key yet)
+            m_ref[q] = kMulti ? fmaxf(tmax[q], -1e30f) : tmax[q];
+            yref[q] = m_ref[q] + lv;
+          }
         } else {
           // a maximum too far above a reference: the reference is raised, l follows here and O^T (whose earlier PVs
           // have to be complete) in TMEM

@@ -83,6 +83,9 @@ def lib():
         L.mala_decode_fp8.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, f, f, i, vp,
                                       sz, vp]
         L.mala_decode_fp8.restype = i
+        L.mala_decode_fp8_multi.argtypes = [_TIn, _TIn, _TIn, vp, vp, _TOut, vp, ctypes.POINTER(_Stats), i, i, i, i, i, i, f,
+                                            f, i, vp, sz, vp]
+        L.mala_decode_fp8_multi.restype = i
         L.mala_decode_fp8_paged.argtypes = [_TIn, _TIn, _TIn, vp, vp, vp, vp, _TOut, vp, ctypes.POINTER(_Stats),
                                             i, i, i, i, i, i, i, f, f, i, vp, sz, vp]
         L.mala_decode_fp8_paged.restype = i
@@ -407,6 +410,29 @@ def decode_fp8(q, kcache8, vcache8, kscale, vscale, scale: float, tau: float, nu
                                ws.data_ptr(), ws.numel(), _stream())
     if rc != 0:
         raise MalaError(rc, "mala_decode_fp8")
+    return o, lse, st
+
+
+def decode_fp8_multi(q, kcache8, vcache8, kscale, vscale, scale: float, tau: float, num_splits: int, stats: bool = False,
+                     ws=None, out=None, want_lse: bool = True):
+    """mala_decode_fp8_multi: q [B,Sq,Hq,d] bf16, the Sq new tokens of each sequence (their keys / values are the last
+    Sq positions of the caches); caches and scales as for decode_fp8.  Returns (o [B,Sq,Hq,d] bf16, lse [B,Sq,Hq]
+    fp32 or None, Stats or None)."""
+    B, Sq, Hq, d = q.shape
+    Nk, Hkv = kcache8.shape[1], kcache8.shape[2]
+    assert kscale.dtype == torch.float32 and kscale.is_contiguous() and tuple(kscale.shape) == (B, Hkv, -(-Nk // 128))
+    assert vscale.dtype == torch.float32 and vscale.is_contiguous() and tuple(vscale.shape) == (B, Hkv, -(-Nk // 128))
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Sq, Hq), dtype=torch.float32, device=q.device) if want_lse else None
+    tps = -(-(-(-Nk // num_splits)) // 128)
+    st = Stats((B, Hkv, num_splits), -(-tps // 32), q.device) if stats else None
+    ws = _ws(workspace_bytes(OP_DECODE, B * Sq, Hq, Hkv, Nk, 128, num_splits), q.device) if ws is None else ws
+    rc = lib().mala_decode_fp8_multi(_view(q, _TIn), _view8(kcache8), _view8(vcache8), kscale.data_ptr(), vscale.data_ptr(),
+                                     _view(o, _TOut), lse.data_ptr() if lse is not None else None,
+                                     ctypes.byref(st.c) if st else None, B, Hq, Hkv, Nk, Sq, d, scale, tau, num_splits,
+                                     ws.data_ptr(), ws.numel(), _stream())
+    if rc != 0:
+        raise MalaError(rc, "mala_decode_fp8_multi")
     return o, lse, st
 
 

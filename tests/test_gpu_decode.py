@@ -513,3 +513,64 @@ def test_decode_fp8_small_pages_with_scales_far_apart(mala, oracle):
         w[name] = (c * f[None, :, None, None] * (0.25 if name == "kcache" else 1.0)).to(torch.bfloat16)
     for tau in (0.0, 1e-4):
         _run_fp8_paged(mala, oracle, w, tau, 4, 16, [2048, 1500], seed=3)
+
+
+def _run_fp8_multi(mala, oracle, w, Sq, tau, num_splits, seed=0):
+    """mala_decode_fp8_multi against the oracle's several-token decode on the dequantised cache (queries drawn as in
+    _run_multi)."""
+    k8, ks, kd = W.quantize_cache_e4m3(w["kcache"])
+    v8, vs, vd = W.quantize_cache_e4m3(w["vcache"])
+    B, Nk, Hkv, d = k8.shape
+    Hq = w["q"].shape[2]
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(1000 + seed)
+    q = w["q"].float().repeat(1, Sq, 1, 1)
+    q[..., : d - 1] += 0.5 * torch.randn((B, Sq, Hq, d - 1), generator=gen)   # (the last feature keeps the key gate)
+    q = q.to(torch.bfloat16)
+    o, lse, st = mala.decode_fp8_multi(q.cuda(), k8.cuda(), v8.cuda(), ks.cuda(), vs.cuda(), w["scale"], tau, num_splits,
+                                       stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    ref = oracle.decode_multi(q, kd, vd, w["scale"], tau, num_splits, 128)
+    ref_abs = oracle.decode_multi(q, kd, vd.abs(), w["scale"], tau, num_splits, 128)
+    tps = ref["mask"].shape[-1]
+    gm = st.mask(tps).cpu().numpy()
+    for b in range(B):
+        for g in range(Hkv):
+            for s in range(num_splits):
+                parity.check_mask(gm[b, g, s], ref["mask"][b, g, s], ref["crit"][b, g, s], list(range(tps - 1, -1, -1)),
+                                  tau, Nk - Sq + 1, 128)
+                assert int(st.retained[b, g, s]) == int(gm[b, g, s].sum())
+    parity.check_output(o.float().cpu().numpy(), ref["o"], a_ref=ref_abs["o"])
+    assert np.abs(lse.cpu().numpy() - ref["lse"]).max() <= parity.LSE_ABS
+    return int((ref["mask"] == 1).sum())
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("Nk,S,Hq,Hkv,Sq", [(1024, 4, 8, 2, 2), (1000, 3, 4, 4, 8), (2050, 4, 4, 2, 4), (1027, 2, 6, 2, 2),
+                                             (640, 5, 2, 1, 3), (4096, 8, 2, 2, 5), (1026, 2, 1, 1, 7)])
+def test_decode_fp8_multi_literal(mala, oracle, Nk, S, Hq, Hkv, Sq, tau):
+    """Several new tokens per step over an e4m3 cache, up to eight rows per KV head; (2050, 4), (1027, 2), (1026, 7): the
+    newest key block holds fewer keys than there are new tokens, so its first rows see none of it."""
+    w = W.custom_decode(2, Hq, Hkv, Nk, 128, S, seed=Nk + S + Sq)
+    _run_fp8_multi(mala, oracle, w, Sq, tau, S, seed=Sq)
+
+
+@pytest.mark.parametrize("tau", [1e-4, 1.0])
+def test_decode_fp8_multi_gated_keys_skip_value_tiles(mala, oracle, tau):
+    w = W.custom_decode(2, 8, 2, 8192, 128, 8, group_types=["diffuse", "peaked"], seed=3, preset="D")
+    assert _run_fp8_multi(mala, oracle, w, 2, tau, 8) > 0, "workload must exercise skipping"
+
+
+def test_decode_fp8_multi_of_one_token_equals_decode_fp8(mala):
+    w = W.custom_decode(2, 8, 2, 4096, 128, 8, group_types=["diffuse", "peaked"], seed=21, preset="D", device="cuda")
+    k8, ks, _ = W.quantize_cache_e4m3(w["kcache"])
+    v8, vs, _ = W.quantize_cache_e4m3(w["vcache"])
+    for tau in (0.0, 1e-4):
+        o0, l0, _ = mala.decode_fp8(w["q"], k8, v8, ks, vs, w["scale"], tau, 8)
+        o1, l1, _ = mala.decode_fp8_multi(w["q"], k8, v8, ks, vs, w["scale"], tau, 8)
+        assert torch.equal(o0, o1) and torch.equal(l0, l1.view_as(l0))
+    q3 = w["q"].repeat(1, 3, 1, 1)                      # (twelve rows per KV head: more than the kernel packs)
+    with pytest.raises(mala.MalaError) as e:
+        mala.decode_fp8_multi(q3, k8, v8, ks, vs, w["scale"], 0.0, 8)
+    assert e.value.code == -2

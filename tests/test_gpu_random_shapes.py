@@ -170,6 +170,8 @@ def test_random_cases_decode_over_an_e4m3_cache(mala, oracle, seed):
         w = W.custom_decode(B, hkv * g, hkv, Nk, d, S, seed=rng.randint(0, 10**6), preset=preset)
         res = TD._run_fp8(mala, oracle, w, tau, S, rounding_bound=True)
         assert res["totals"][1] == res["retained"] + res["skipped"], (B, hkv, g, d, Nk, S, tau, preset)
+        if g <= 4 and Nk >= 8:   # (several new tokens on the same cache, up to eight rows per KV head)
+            TD._run_fp8_multi(mala, oracle, w, rng.randint(2, 8 // g), tau, S, seed=Nk)
 
 
 @pytest.mark.parametrize("seed", [0, 1, 2])
