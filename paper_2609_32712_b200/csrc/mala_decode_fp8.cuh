@@ -391,8 +391,8 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const int T = tiles_of(item);
         if (T == 0) continue;
         const int ip = ne & 1;
-        int b_, hkv_ = 0, split_, j0_;
-        if constexpr (kSmall) geometry(item, b_, hkv_, split_, j0_, T);
+        int b_ = 0, hkv_ = 0, split_, j0_ = 0, nk_ = 0;
+        if constexpr (kSmall) { geometry(item, b_, hkv_, split_, j0_, T); nk_ = keys_of(b_); }
         uint8_t* q8 = sQ8 + ip * Cfg::kQ8Bytes;
         // the item's queries have landed: row qh (128 bf16 in two 64-column panels, rows qh and HALF + qh of the
         // landing buffer; lane = four consecutive columns) becomes rows qh and HALF + qh of the e4m3 operand, once the
@@ -441,10 +441,14 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
               sc_k[k][sb][lane] = there ? __ldg(p.kscale + (size_t)pg * p.Hkv + hkv_) : 1.f;
               sc_v[k][sb][lane] = vsc;
             }
-            float vmx = lane < p.ppt ? vsc : 0.f;
+            // the reference of the 8-bit probabilities follows the largest V scale among the pages that hold a key of
+            // the sequence: a page that is not there (scale 1) or lies wholly past the sequence's end (any scale) would
+            // push every real key's probability toward e4m3's subnormals
+            const bool counts = there && ((j0_ - t) * 128 + lane * p.prows) < nk_;
+            float vmx = counts ? vsc : 0.f;
 #pragma unroll
             for (int o = 4; o > 0; o >>= 1) vmx = fmaxf(vmx, __shfl_xor_sync(0xffffffffu, vmx, o));
-            if (lane == 0) sc_vmax[k][sb] = vmx;
+            if (lane == 0) sc_vmax[k][sb] = vmx > 0.f ? vmx : 1.f;
             __threadfence_block();
           } else if (leader) {   // the tile's scales travel with its scores (a page without scales holds zeros: any scale does)
             const int sidx = *(volatile int*)&t_sidx[k][g & 7];

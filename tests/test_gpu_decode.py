@@ -574,3 +574,14 @@ def test_decode_fp8_multi_of_one_token_equals_decode_fp8(mala):
     with pytest.raises(mala.MalaError) as e:
         mala.decode_fp8_multi(q3, k8, v8, ks, vs, w["scale"], 0.0, 8)
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("page", [16, 32])
+def test_decode_fp8_small_pages_absent_pages_do_not_set_the_reference(mala, oracle, page):
+    """Sequences that end inside a tile, with table entries outside the pool behind them, and values 2^-6 small: the
+    pages that are not there (scale 1) or lie past the sequence's end must not set the reference of the 8-bit
+    probabilities, or every real key's probability would fall into e4m3's subnormals."""
+    w = W.custom_decode(3, 8, 2, 4096, 64, 2, seed=462)
+    w["vcache"] = (w["vcache"].float() * 2.0 ** -6).to(torch.bfloat16)
+    for tau in (0.0, 1.0):
+        _run_fp8_paged(mala, oracle, w, tau, 2, page, [4096, 1497, 48 + page // 2], seed=3)
