@@ -228,7 +228,9 @@ int mala_decode_fp8_multi(mala_tin q, mala_tin kcache8, mala_tin vcache8, const 
  * clamping of seqlens, entries outside the pool (read as zeros) and telemetry as in mala_decode_paged; slots of a
  * mapped page beyond the sequence's length must hold codes other than e4m3's two NaN codes, 0x7f and 0xff (a
  * zero-initialised or recycled page does): their keys are masked out of the scores, but their values are multiplied by
- * zero probabilities.  d, Hq/Hkv and the workspace as in mala_decode_fp8. */
+ * zero probabilities.  (Where such slots share a scale with real keys -- the rest of the sequence's last page -- a
+ * scale orders of magnitude above the real values' costs those values, and the step's 8-bit probabilities, precision:
+ * quantise a page from the slots in use.)  d, Hq/Hkv and the workspace as in mala_decode_fp8. */
 int mala_decode_fp8_paged(mala_tin q, mala_tin kpages8, mala_tin vpages8, const float* kscale, const float* vscale,
                           const int32_t* block_table, const int32_t* seqlens, mala_tout o, float* lse_opt,
                           const mala_stats* st, int B, int Hq, int Hkv, int num_pages, int page_size,
