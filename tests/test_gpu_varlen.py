@@ -48,6 +48,7 @@ def _run(mala, oracle, lens, Hq, Hkv, d, tau, preset="literal", causal=True, hea
         # backward on the GPU's own forward output of this sequence
         g = oracle.bwd(w["q"], w["k"], w["v"], o[:, r0:r0 + n].float().cpu(), w["do"],
                        lse[:, r0:r0 + n].cpu().numpy()[None], w["scale"], tau, 128, 128, causal=causal)
+        flipped = False
         for h in range(Hq):
             for j in range(T):
                 om, oc = g["mask"][0, h, j], g["crit"][0, h, j]
@@ -56,8 +57,11 @@ def _run(mala, oracle, lens, Hq, Hkv, d, tau, preset="literal", causal=True, hea
                         assert not bm[b, h, j, i]
                     elif bool(bm[b, h, j, i]) != (om[i] == 2):
                         assert abs(oc[i]) <= parity.MASK_BAND, (b, h, j, i, oc[i])
+                        flipped = True
             assert not bm[b, h, T:].any()
-        for got, want, what in ((dq_c, g["dq"], "dq"), (dk_c, g["dk"], "dk"), (dv_c, g["dv"], "dv")):
+        # (a tile decided the other way inside the exemption band -- e.g. one key at tau = 1, where p = tau / L exactly --
+        # changes the gradients by that tile's whole contribution: nothing to compare element by element then)
+        for got, want, what in (() if flipped else ((dq_c, g["dq"], "dq"), (dk_c, g["dk"], "dk"), (dv_c, g["dv"], "dv"))):
             if n == 1 and what != "dv":
                 # one key: p = 1 and dS = p (dP - D) = 0 exactly; the kernel's D comes from the bf16 output
                 assert np.abs(got[r0:r0 + n]).max() <= 1e-2 * np.abs(want).max() + 1e-5
