@@ -176,6 +176,10 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   constexpr bool kSplit = GP > 4;          // two threads per key, four heads each
   constexpr int HS = Cfg::kHalves;
   constexpr int GS = kSplit ? 4 : GP;      // heads a softmax thread carries
+  // The dense kernel with two threads per key sums a tile's probabilities per thread and crosses the group once per
+  // item (no test needs the normalizer earlier): 5 % off its per-tile chain, which bounds it.  (With one thread per key
+  // the dense kernel is bound by HBM, and the same change made it 3 % slower: 378 against 365 us at cfg5.)
+  constexpr bool kLocalSums = kDense && kSplit;
   static_assert(!kDense || NK == NV, "the dense producer walks both rings with one index");
   constexpr int GH = GP;                   // rows of a softmax group
   constexpr int HALF = GP > 4 ? 8 : 4;     // rows (MMA columns) of the leading parts; the remainders follow them
@@ -713,6 +717,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       float m_ref[GS], l[GS], yref[GS], lgl[GS], c2q[GS];
 #pragma unroll
       for (int q = 0; q < GS; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; yref[q] = 0.f; lgl[q] = -INFINITY; c2q[q] = c2; }
+      float lacc[kLocalSums ? GS : 1];           // this thread's share of the row sums
+#pragma unroll
+      for (int q = 0; q < (kLocalSums ? GS : 1); ++q) lacc[q] = 0.f;
       for (int t = 0; t < T; ++t, ++g) {
         const int sb = g & 3;
         ok = mbar_wait(&s_full[k][sb], (uint32_t)((g >> 2) & 1), status);
@@ -794,7 +801,9 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             alpha[q] = 1.f;
             if (hb + q < R && (tmax[q] + lv > yref[q] + kPGap || tmax[q] > m_ref[q] + kMGap)) {
               const float mn = fmaxf(m_ref[q], tmax[q]), yn = fmaxf(yref[q], tmax[q] + lv);
-              l[q] *= fast_exp2(m_ref[q] - mn);
+              const float lf = fast_exp2(m_ref[q] - mn);
+              l[q] *= lf;
+              if constexpr (kLocalSums) lacc[q] *= lf;
               alpha[q] = fast_exp2(yref[q] - yn);
               touch = touch || yn > yref[q];
               m_ref[q] = mn;
@@ -870,13 +879,24 @@ mala_decode_fp8_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[k][ps]);
-        RowReduce<GS, 16, false>::run(e, lane);   // (the sums cross the group with the next tile's maxima)
-        psum_w = e[0];
-        pending_sum = true;
+        if constexpr (kLocalSums) {
+          // no test needs the normalizer before the item's end: every thread keeps the sums of its own key column
+#pragma unroll
+          for (int q = 0; q < GS; ++q) lacc[q] += e[q];
+        } else {
+          RowReduce<GS, 16, false>::run(e, lane);   // (the sums cross the group with the next tile's maxima)
+          psum_w = e[0];
+          pending_sum = true;
+        }
         ++r;
         ++rg;
       }
       if (!ok) break;
+      if constexpr (kLocalSums) {
+        RowReduce<GS, 16, false>::run(lacc, lane);
+        psum_w = lacc[0];
+        pending_sum = true;
+      }
       if (pending_sum) {   // the last retained tile's sums
         float unused[GS];
         ok = exchange(-INFINITY, unused, l, lgl);
