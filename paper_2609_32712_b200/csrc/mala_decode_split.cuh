@@ -129,6 +129,10 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   constexpr bool kInOrder = !kDense && NG == 1 && !kMulti;   // separate in-order issuing warps (see there)
   constexpr int GH = GP / NG;              // rows per group
   constexpr int LDN = NG == 1 ? 16 : GH;   // TMEM columns a softmax thread reads at a time
+  // The dense kernel at sixteen rows (bound by its softmax groups' instruction streams, not by HBM) sums a tile's
+  // probabilities per thread and crosses the group once per item: no test needs the normalizer earlier.  (The variants
+  // with fewer rows are bound by HBM and keep the per-tile sums, whose exchange rides with the maxima's.)
+  constexpr bool kLocalSums = kDense && GP >= 16;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                      // [2] item parity
@@ -727,6 +731,9 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       float psum = 0.f;   // this warp's sum of P of the last retained tile, for the row this lane publishes
 #pragma unroll
       for (int q = 0; q < GH; ++q) { m_ref[q] = -INFINITY; l[q] = 0.f; lgl[q] = -INFINITY; }
+      float lacc[kLocalSums ? GH : 1];   // this thread's share of the row sums
+#pragma unroll
+      for (int q = 0; q < (kLocalSums ? GH : 1); ++q) lacc[q] = 0.f;
       int r = 0;
       bool pending_sum = false;
       uint32_t bm_bits = 0;
@@ -822,6 +829,7 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             if (rb + q < R && tmax[q] > m_ref[q] + kRescaleGap) {   // lazy rescaling: the reference only moves when it has to
               alpha[q] = fast_exp2(m_ref[q] - tmax[q]);
               l[q] *= alpha[q];
+              if constexpr (kLocalSums) lacc[q] *= alpha[q];
               lgl[q] = __log2f(l[q]);
               m_ref[q] = tmax[q];
               resc = true;
@@ -878,14 +886,24 @@ mala_decode_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[ps]);
-        // this warp's per-row sums of the tile (fp32, before the bf16 cast); they travel with the next exchange
-        RowReduce<GH, 16, false>::run(x, lane);
-        psum = x[0];
-        pending_sum = true;
+        if constexpr (kLocalSums) {
+#pragma unroll
+          for (int q = 0; q < GH; ++q) lacc[q] += x[q];
+        } else {
+          // this warp's per-row sums of the tile (fp32, before the bf16 cast); they travel with the next exchange
+          RowReduce<GH, 16, false>::run(x, lane);
+          psum = x[0];
+          pending_sum = true;
+        }
         ++r;
         ++rg;
       }
       if (!ok) break;
+      if constexpr (kLocalSums) {
+        RowReduce<GH, 16, false>::run(lacc, lane);
+        psum = lacc[0];
+        pending_sum = true;
+      }
       if (pending_sum) {   // the sums of the last retained tile
         float dummy[GH];
         ok = exchange(-INFINITY, dummy);
