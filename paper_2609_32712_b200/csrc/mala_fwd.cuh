@@ -192,8 +192,10 @@ mala_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // x / PAN of panel x % PAN of a tile, so the table lookups are one coalesced load and the copies are issued side
     // by side instead of one after the other
     auto load_tile_small_warp = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int jt) {
-      const int c = lane / PAN, pn = lane % PAN, pg = jt * p.ppt + c;
-      if (c < p.ppt) {
+      const int pn = lane % PAN;
+      // (up to 16 copies of PAN panels: one per lane with up to two panels, two rounds with four)
+      for (int c = lane / PAN; c < p.ppt; c += 32 / PAN) {
+        const int pg = jt * p.ppt + c;
         const int outer = pg < p.bt_stride ? __ldg(p.block_table + (size_t)b * p.bt_stride + pg) : -1;
         tma_load_4d(dst + pn * 16384 + c * p.prows * 128, tm, bar, pn * 64, 0, hkv, outer);
       }

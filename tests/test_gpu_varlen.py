@@ -233,7 +233,7 @@ def test_varlen_prefix_backward_sequences_without_queries_get_zero_gradients(mal
 
 @pytest.mark.parametrize("tau", [0.0, 1e-4])
 @pytest.mark.parametrize("page,d", [(128, 128), (256, 128), (16, 128), (64, 128), (8, 64), (32, 96), (128, 40),
-                                    (256, 256), (16, 256), (128, 200)])
+                                    (256, 256), (16, 256), (128, 200), (8, 256), (8, 136)])
 def test_prefill_chunks_against_a_paged_cache(mala, oracle, tau, page, d):
     """Packed prefill chunks whose keys and values (prefix and chunk) lie in pages scattered over a shuffled pool."""
     Hq, Hkv = 4, 2
