@@ -181,3 +181,55 @@ def test_decode_above_128_columns_stores_nothing_beyond_the_head_size(mala):
     assert mala.device_status() == 0
     assert (ob[..., d:] == 7.0).all() and not (ob[..., :d] == 7.0).all()
     assert torch.equal(mala.decode(w["q"], w["kcache"], w["vcache"], w["scale"], 1e-4, 4)[0], o)
+
+
+@pytest.mark.parametrize("tau", [0.0, 1e-4])
+@pytest.mark.parametrize("d,causal", [(256, True), (168, True), (256, False)])
+def test_forward_above_128_columns_packed_sequences_behind_prefixes(mala, oracle, d, causal, tau):
+    """mala_fwd_varlen and mala_fwd_varlen_prefix (forward only) with one query block per CTA: sequences of different
+    lengths, chunks that start inside a tile, a chunk of one query."""
+    Hq, Hkv = 4, 2
+    nk = [900, 128, 517, 300, 64]
+    nq = [260, 128, 100, 1, 64]
+    ws = [W.custom_prefill(1, Hq, Hkv, n, d, head_types=["diffuse", "peaked", "peaked", "sink"], seed=60 + x, preset="R")
+          for x, n in enumerate(nk)]
+    q = torch.cat([w["q"][:, n - m:] for w, n, m in zip(ws, nk, nq)], dim=1).contiguous()
+    k = torch.cat([w["k"] for w in ws], dim=1).contiguous()
+    v = torch.cat([w["v"] for w in ws], dim=1).contiguous()
+    cq = torch.tensor(np.concatenate([[0], np.cumsum(nq)]), dtype=torch.int32)
+    ck = torch.tensor(np.concatenate([[0], np.cumsum(nk)]), dtype=torch.int32)
+    o, lse, st = mala.fwd_varlen_prefix(q.cuda(), k.cuda(), v.cuda(), cq.cuda(), ck.cuda(), max(nq), max(nk),
+                                        ws[0]["scale"], tau, causal=causal, stats=True)
+    o2, lse2, st2 = mala.fwd_varlen(torch.cat([w["q"] for w in ws], dim=1).contiguous().cuda(), k.cuda(), v.cuda(), ck.cuda(),
+                                    max(nk), ws[0]["scale"], tau, causal=causal, stats=True)
+    torch.cuda.synchronize()
+    assert mala.device_status() == 0
+    fm = st.mask(-(-max(nk) // 128)).cpu().numpy()
+    fm2 = st2.mask(-(-max(nk) // 128)).cpu().numpy()
+    o_c, lse_c = o.float().cpu().numpy()[0], lse.cpu().numpy()
+    o2_c, lse2_c = o2.float().cpu().numpy()[0], lse2.cpu().numpy()
+    for b, (w, n, m) in enumerate(zip(ws, nk, nq)):
+        off = n - m
+        shift = off % 128 if causal else 0
+        ref = oracle.fwd(w["q"][:, n - m:], w["k"], w["v"], w["scale"], tau, 128, 128, causal=causal, q_shift=shift)
+        ref_abs = oracle.fwd(w["q"][:, n - m:], w["k"], w["v"].abs(), w["scale"], tau, 128, 128, causal=causal, q_shift=shift)
+        Tq, Tk = ref["mask"].shape[2], ref["mask"].shape[3]
+        r0 = int(cq[b])
+        for h in range(Hq):
+            for i in range(Tq):
+                order = list(range(i + off // 128, -1, -1)) if causal else list(range(Tk - 1, -1, -1))
+                parity.check_mask(fm[b, h, i, :Tk], ref["mask"][0, h, i], ref["crit"][0, h, i], order, tau,
+                                  (max(i * 128 - shift, 0) + 1 + off) if causal else n)
+        parity.check_output(o_c[r0:r0 + m], ref["o"][0], a_ref=ref_abs["o"][0])
+        assert np.abs(lse_c[:, r0:r0 + m] - ref["lse"][0]).max() <= parity.LSE_ABS
+        # the whole sequence as its own packed sequence
+        full = oracle.fwd(w["q"], w["k"], w["v"], w["scale"], tau, 128, 128, causal=causal)
+        full_abs = oracle.fwd(w["q"], w["k"], w["v"].abs(), w["scale"], tau, 128, 128, causal=causal)
+        k0, T = int(ck[b]), -(-n // 128)
+        for h in range(Hq):
+            for i in range(T):
+                order = list(range(i, -1, -1)) if causal else list(range(T - 1, -1, -1))
+                parity.check_mask(fm2[b, h, i, :T], full["mask"][0, h, i], full["crit"][0, h, i], order, tau,
+                                  i * 128 + 1 if causal else n)
+        parity.check_output(o2_c[k0:k0 + n], full["o"][0], a_ref=full_abs["o"][0])
+        assert np.abs(lse2_c[:, k0:k0 + n] - full["lse"][0]).max() <= parity.LSE_ABS
